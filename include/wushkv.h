@@ -1,0 +1,191 @@
+/*
+ * wushkv.h - C ABI of the WUSH-KV serving hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, for ONE attention module on ONE GPU,
+ *   (1) calibration-time construction of the per-KV-head key transforms T_K
+ *       (WUSH closed form, Section 3 Eq. 1, specialised to keys by Eq. 4 / Algorithm 1),
+ *   (2) quantize-on-append: k' = T_K k for each new post-RoPE key, values taken as they
+ *       are (already in the weight-folded basis, Section 4.2), the per-token
+ *       percentile-clipped affine quantizer of Section 5.3 Eq. 6 at 2 or 4 bits, and packing of
+ *       codes + (scale, zero) into a paged cache (Algorithm 2 lines 3-4, 9-12),
+ *   (3) decode attention over that packed cache for one new query per sequence
+ *       (Algorithm 2 lines 3 and 5; Eq. 2; Eq. 3), reading the first S_sink and the most
+ *       recent positions from a bf16 copy (Section 4.4).
+ *
+ * General rules
+ *   - Every function returns an int status (WUSHKV_OK = 0).  No exceptions, no global state
+ *     except a cached device-attribute query.
+ *   - "host" / "device" beside a pointer says where the memory must live.  All memory is
+ *     owned by the caller before, during and after every call; the library allocates nothing
+ *     and keeps no pointer between calls.
+ *   - wushkv_append / wushkv_decode_attn / wushkv_unpack_debug only ENQUEUE work on the CUDA
+ *     stream passed in (a cudaStream_t cast to void*, NULL = default stream) and do not
+ *     synchronise.  Arguments are validated on the host before anything is launched; a bad
+ *     argument returns WUSHKV_EINVAL and launches nothing.
+ *   - Problems that only the device can see (a position beyond the page table, a page id
+ *     outside the pool, a copy that never arrived) never trap: the offending access is
+ *     skipped and a bit is OR-ed into *dev_status, which the caller reads when it likes.
+ *   - Head dimension d must be 128 and page_tokens must be 64.  bits is 2 or 4.  The query
+ *     group size n_q / n_kv must be an integer between 1 and 8.
+ *
+ * Conventions
+ *   - Vectors are rows [token][channel].  T is the paper's T stored row-major [out][in]:
+ *     k'[i] = sum_j T[i][j] k[j]  (k' = T k), and q'[i] = sum_j T_invT[i][j] q[j]
+ *     (q' = T^{-T} q) with T_invT = (T^{-1})^T.
+ *   - Positions are 0-based.  With S positions cached, the positions read from the packed
+ *     codes are [s_sink, s_sink + n) with n = floor((S - lag - s_keep - s_sink) / s_flush) * s_flush
+ *     when that is >= s_flush and 0 otherwise (closed form of Algorithm 2 lines 7-8);
+ *     every other position is read from its bf16 copy (sink buffer or ring buffer).
+ *   - bf16 / fp16 values cross the ABI as their 16-bit patterns (uint16_t).
+ */
+#ifndef WUSHKV_H
+#define WUSHKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes (return values) -------------------------------------------------------- */
+#define WUSHKV_OK        0
+#define WUSHKV_EINVAL    1  /* null pointer, unsupported shape, misaligned buffer, bad size   */
+#define WUSHKV_ENOTPD    2  /* damped Gram or Hessian not positive definite (Definition 1)    */
+#define WUSHKV_ECUDA     3  /* a CUDA runtime call or kernel launch failed                    */
+#define WUSHKV_ECAPACITY 4  /* workspace / ring buffer / page table too small for the request */
+
+/* ---- bits OR-ed into *dev_status by kernels ---------------------------------------------- */
+#define WUSHKV_DEV_PAGE_TABLE_FULL 1  /* a position needs page index >= max_pages: token skipped */
+#define WUSHKV_DEV_BAD_PAGE_ID     2  /* page table entry outside [0, n_pages): access skipped   */
+#define WUSHKV_DEV_BAD_SLOT        4  /* slot[b] outside [0, n_slots): sequence skipped          */
+#define WUSHKV_DEV_COPY_TIMEOUT    8  /* a staged page copy did not arrive within the wait limit */
+
+/*
+ * One layer's cache description.  Plain data; the caller fills it for every call.
+ *
+ * Packed pages (device): n_pages records of wushkv_page_bytes() bytes each, 256-byte aligned.
+ *   A page holds page_tokens consecutive positions of one sequence for all n_kv heads; the
+ *   per-(page, head) record keeps, contiguously, the K codes, the V codes and the four fp16
+ *   numbers (K step, K x_min, V step, V x_min) of each token (Eq. 6: Delta and the offset
+ *   x_min = -Delta z).  The bit layout inside a record is private to the library (it is
+ *   permuted to match the decode kernel's register fragments); read it back through
+ *   wushkv_unpack_debug.
+ * page_table (device): int32 [n_slots][max_pages]; entry [s][i] is the page that holds
+ *   positions [i*page_tokens, (i+1)*page_tokens) of slot s.
+ * sink_kv (device): bf16 [n_slots][n_kv][2][s_sink][d]; [..][0][p] is k' (= bf16(T_K k)) and
+ *   [..][1][p] is v of position p < s_sink.  May be NULL when s_sink == 0.
+ * ring_kv (device): bf16 [n_slots][n_kv][2][ring_cap][d]; position p lives in row p % ring_cap.
+ *   ring_cap >= s_keep + s_flush - 1 + boundary_lag.
+ * T_K, T_K_invT (device): fp32 [n_kv][d][d] as produced by wushkv_build_transforms.
+ * dev_status (device): one int32 that kernels OR error bits into; the caller zeroes it.
+ */
+typedef struct wushkv_cache {
+    int32_t n_q, n_kv, d, bits;
+    int32_t page_tokens, s_sink, s_keep, s_flush;
+    int32_t boundary_lag;  /* 0: read boundary from the current length (serving behaviour,
+                              Section 5.3); k: boundary of k positions ago (Algorithm 2 taken
+                              literally has k = positions appended in this step) */
+    int32_t n_slots, max_pages, ring_cap;
+    float kappa_k, kappa_v; /* clipping quantiles of Eq. 6 for keys and values, in [0, 1] */
+    float sm_scale;         /* 1 / tau of Eq. 2 */
+    int32_t reserved;
+    int64_t n_pages;
+    void* pages;
+    const int32_t* page_table;
+    void* sink_kv;
+    void* ring_kv;
+    const float* T_K;
+    const float* T_K_invT;
+    int32_t* dev_status;
+} wushkv_cache;
+
+/* Bytes of one page (all n_kv heads): n_kv * page_tokens * (2 * d * bits / 8 + 8).
+ * Returns 0 for an unsupported (bits, page_tokens, d). */
+size_t wushkv_page_bytes(int32_t n_kv, int32_t d, int32_t bits, int32_t page_tokens);
+
+/* Human-readable name of a status code (static storage). */
+const char* wushkv_status_string(int status);
+
+/*
+ * Gram / Hessian accumulation for the key transform: Eq. 4 and Algorithm 1 lines 4-5.
+ *   K (host): bf16 [n_tok][n_kv][d]  post-Norm post-RoPE keys of one calibration sequence.
+ *   Q (host): bf16 [n_tok][n_q][d]   post-Norm post-RoPE queries; head j belongs to KV head j / (n_q/n_kv).
+ *   M, H (host, in/out): float64 [n_kv][d][d];  M[h] += sum_t k k^T,  H[h] += 2 sum_g sum_t q q^T.
+ * Call once per calibration sequence (Algorithm 1 sums over sequences); the caller zeroes M, H first.
+ */
+int wushkv_accumulate_gram(int32_t n_kv, int32_t n_q, int32_t d, int64_t n_tok,
+                           const uint16_t* K, const uint16_t* Q, double* M, double* H);
+
+/*
+ * WUSH transforms from accumulated statistics: Section 3 Eq. 1 / Definition 1 applied per head
+ * (Algorithm 1 line 7).  Host pointers, host float64 arithmetic (Cholesky, cyclic Jacobi
+ * eigensolver, Sylvester Hadamard); runs once at calibration time.
+ *   M, H (host): float64 [n_heads][d][d] symmetric; gamma >= 0 the damping ratio.
+ *   T (host, out): fp32 [n_heads][d][d], T = c Had Lam^(-1/4) U^T L^T with eigenvalues
+ *       ascending and each eigenvector signed so that its largest-magnitude entry is positive;
+ *       every entry is rounded to the nearest bf16-representable value.
+ *   T_invT (host, out): fp32 [n_heads][d][d], transpose of the inverse of the ROUNDED T, so that
+ *       the insertion identity of Eq. 3 holds for the stored pair.
+ * d must be a power of two (<= 1024).  Returns WUSHKV_ENOTPD if a damped matrix is not
+ * positive definite (outputs of that head are then unspecified).
+ */
+int wushkv_build_transforms(int32_t n_heads, int32_t d, const double* M, const double* H, double gamma,
+                            float* T, float* T_invT);
+
+/*
+ * Quantize-on-append: Algorithm 2 lines 3-4 (key side) and 9-12, with Eq. 6 as the quantizer.
+ * For sequence b (0 <= b < batch) the new tokens are rows cu_new[b] .. cu_new[b+1]-1 of K_new /
+ * V_new and take positions seq_len[b], seq_len[b]+1, ...  Every new token is transformed
+ * (keys only), quantized from the fp32 transform output, packed into its page, and its bf16
+ * copy is written to the sink buffer (position < s_sink) and to the ring buffer (if it is among
+ * the last ring_cap positions after this call).  Finally seq_len[b] += number of new tokens.
+ *   slot (device): int32 [batch], cache slot of each sequence; slots must be distinct.
+ *   seq_len (device, in/out): int32 [batch].
+ *   cu_new (device): int32 [batch+1] prefix sums, cu_new[0] = 0, cu_new[batch] = total_new.
+ *   total_new, max_new (host): total and per-sequence maximum of new tokens.
+ *   K_new (device): bf16 [total_new][n_kv][d] post-Norm post-RoPE keys, 16-byte aligned.
+ *   V_new (device): bf16 [total_new][n_kv][d] values in the folded basis, 16-byte aligned.
+ * Chunks (max_new >= 128) take the tensor-core transform path; short appends a CUDA-core one.
+ * Both produce the same codes up to fp32 summation order.
+ */
+int wushkv_append(const wushkv_cache* cache, int32_t batch, const int32_t* slot, int32_t* seq_len,
+                  const int32_t* cu_new, int32_t total_new, int32_t max_new,
+                  const uint16_t* K_new, const uint16_t* V_new, void* stream);
+
+/* Bytes of scratch wushkv_decode_attn needs for (batch, max_seq_len); 0 on invalid arguments. */
+size_t wushkv_decode_workspace_bytes(const wushkv_cache* cache, int32_t batch, int32_t max_seq_len);
+
+/*
+ * Decode attention: Algorithm 2 line 3 (query side: q' = T_K^{-T} q) and line 5 (Eq. 2 for one
+ * query column that sees all seq_len[b] cached positions, softmax temperature 1/sm_scale),
+ * evaluated directly on the packed cache: quantized positions are dequantized in registers
+ * (x_hat = x_min + Delta * code), window positions are read from the bf16 buffers.  The
+ * context is split across thread blocks (partial softmax state per split) and merged by a
+ * final combine pass.  Call after wushkv_append of the step's token.
+ *   slot (device): int32 [batch];  seq_len (device): int32 [batch], each >= 1.
+ *   max_seq_len (host): upper bound of seq_len[b] (sizes the launch; no device read-back).
+ *   Q (device): bf16 [batch][n_q][d] post-Norm post-RoPE, NOT compensated; 16-byte aligned.
+ *   O (device, out): fp32 [batch][n_q][d] = V P in the folded value basis (the output
+ *       projection, Algorithm 2 line 6, is outside the library).
+ *   workspace (device): >= wushkv_decode_workspace_bytes(...) bytes, 256-byte aligned; contents
+ *       are scratch (no initialisation needed, nothing survives the call).
+ */
+int wushkv_decode_attn(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
+                       int32_t max_seq_len, const uint16_t* Q, float* O,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Read back the logical content of the packed cache (test / debugging aid): for positions
+ * pos0 .. pos0+n-1 of (slot, kv_head), which = 0 for keys, 1 for values:
+ *   codes (device, out): uint8 [n][d], one code per byte in channel order;
+ *   scale (device, out): fp32 [n] the stored step Delta;  zero (device, out): fp32 [n] the stored x_min.
+ * Positions are read wherever they are in the page table regardless of the windows.
+ */
+int wushkv_unpack_debug(const wushkv_cache* cache, int32_t slot, int32_t kv_head, int32_t which,
+                        int32_t pos0, int32_t n, uint8_t* codes, float* scale, float* zero, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WUSHKV_H */

@@ -1,0 +1,181 @@
+"""ctypes binding of libwushkv.so: the same entry points as ``include/wushkv.h``, argument
+marshalling only.  Every step of the hot path runs inside the library's CUDA kernels; PyTorch is
+used here for device memory and streams and nothing else.  There is no CPU fallback: importing
+this module without the built library raises."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libwushkv.so")
+
+OK, EINVAL, ENOTPD, ECUDA, ECAPACITY = 0, 1, 2, 3, 4
+DEV_PAGE_TABLE_FULL, DEV_BAD_PAGE_ID, DEV_BAD_SLOT, DEV_COPY_TIMEOUT = 1, 2, 4, 8
+
+EXPORTS = (
+    "wushkv_page_bytes", "wushkv_status_string", "wushkv_accumulate_gram", "wushkv_build_transforms",
+    "wushkv_append", "wushkv_decode_workspace_bytes", "wushkv_decode_attn", "wushkv_unpack_debug",
+)
+
+
+class WushkvError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({status_string(status)})")
+
+
+class wushkv_cache(C.Structure):
+    """Mirror of ``struct wushkv_cache``."""
+    _fields_ = [
+        ("n_q", C.c_int32), ("n_kv", C.c_int32), ("d", C.c_int32), ("bits", C.c_int32),
+        ("page_tokens", C.c_int32), ("s_sink", C.c_int32), ("s_keep", C.c_int32), ("s_flush", C.c_int32),
+        ("boundary_lag", C.c_int32),
+        ("n_slots", C.c_int32), ("max_pages", C.c_int32), ("ring_cap", C.c_int32),
+        ("kappa_k", C.c_float), ("kappa_v", C.c_float), ("sm_scale", C.c_float),
+        ("reserved", C.c_int32),
+        ("n_pages", C.c_int64),
+        ("pages", C.c_void_p), ("page_table", C.c_void_p), ("sink_kv", C.c_void_p), ("ring_kv", C.c_void_p),
+        ("T_K", C.c_void_p), ("T_K_invT", C.c_void_p), ("dev_status", C.c_void_p),
+    ]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2609_38121_b200.build` "
+            "(nvcc, sm_100a).  There is no fallback path.")
+    lib = C.CDLL(LIB_PATH)
+    lib.wushkv_page_bytes.restype = C.c_size_t
+    lib.wushkv_page_bytes.argtypes = [C.c_int32] * 4
+    lib.wushkv_status_string.restype = C.c_char_p
+    lib.wushkv_status_string.argtypes = [C.c_int]
+    lib.wushkv_accumulate_gram.restype = C.c_int
+    lib.wushkv_accumulate_gram.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_void_p, C.c_void_p,
+                                           C.c_void_p, C.c_void_p]
+    lib.wushkv_build_transforms.restype = C.c_int
+    lib.wushkv_build_transforms.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_double,
+                                            C.c_void_p, C.c_void_p]
+    lib.wushkv_append.restype = C.c_int
+    lib.wushkv_append.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                  C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.wushkv_decode_workspace_bytes.restype = C.c_size_t
+    lib.wushkv_decode_workspace_bytes.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_int32]
+    lib.wushkv_decode_attn.restype = C.c_int
+    lib.wushkv_decode_attn.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_void_p, C.c_void_p, C.c_int32,
+                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.wushkv_unpack_debug.restype = C.c_int
+    lib.wushkv_unpack_debug.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                        C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    return lib
+
+
+lib = _load()
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise WushkvError(status, where)
+
+
+def _ptr(t):
+    """Device or host pointer of a torch tensor / numpy array (None -> NULL)."""
+    if t is None:
+        return None
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return t.data_ptr()
+
+
+def _stream_ptr(stream):
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def status_string(status: int) -> str:
+    return lib.wushkv_status_string(int(status)).decode()
+
+
+def page_bytes(n_kv: int, d: int, bits: int, page_tokens: int) -> int:
+    return int(lib.wushkv_page_bytes(n_kv, d, bits, page_tokens))
+
+
+def accumulate_gram(K_bits: np.ndarray, Q_bits: np.ndarray, M: np.ndarray, H: np.ndarray):
+    """wushkv_accumulate_gram: K_bits uint16 [n_tok][n_kv][d], Q_bits uint16 [n_tok][n_q][d] (bf16
+    patterns), M and H float64 [n_kv][d][d] updated in place."""
+    K_bits = np.ascontiguousarray(K_bits, dtype=np.uint16)
+    Q_bits = np.ascontiguousarray(Q_bits, dtype=np.uint16)
+    assert M.dtype == np.float64 and H.dtype == np.float64 and M.flags.c_contiguous and H.flags.c_contiguous
+    n_tok, n_kv, d = K_bits.shape
+    _check(lib.wushkv_accumulate_gram(n_kv, Q_bits.shape[1], d, n_tok, K_bits.ctypes.data, Q_bits.ctypes.data,
+                                      M.ctypes.data, H.ctypes.data), "wushkv_accumulate_gram")
+
+
+def build_transforms(M: np.ndarray, H: np.ndarray, gamma: float):
+    """wushkv_build_transforms: returns (T, T_invT) as float32 [n_heads][d][d]."""
+    M = np.ascontiguousarray(M, dtype=np.float64)
+    H = np.ascontiguousarray(H, dtype=np.float64)
+    n, d, _ = M.shape
+    T = np.empty((n, d, d), dtype=np.float32)
+    TinvT = np.empty((n, d, d), dtype=np.float32)
+    _check(lib.wushkv_build_transforms(n, d, M.ctypes.data, H.ctypes.data, float(gamma), T.ctypes.data,
+                                       TinvT.ctypes.data), "wushkv_build_transforms")
+    return T, TinvT
+
+
+def append(cache: wushkv_cache, batch, slot, seq_len, cu_new, total_new, max_new, K_new, V_new, stream=None):
+    _check(lib.wushkv_append(C.byref(cache), batch, _ptr(slot), _ptr(seq_len), _ptr(cu_new), total_new, max_new,
+                             _ptr(K_new), _ptr(V_new), _stream_ptr(stream)), "wushkv_append")
+
+
+def decode_workspace_bytes(cache: wushkv_cache, batch: int, max_seq_len: int) -> int:
+    return int(lib.wushkv_decode_workspace_bytes(C.byref(cache), batch, max_seq_len))
+
+
+def decode_attn(cache: wushkv_cache, batch, slot, seq_len, max_seq_len, Q, O, workspace, workspace_bytes, stream=None):
+    _check(lib.wushkv_decode_attn(C.byref(cache), batch, _ptr(slot), _ptr(seq_len), max_seq_len, _ptr(Q), _ptr(O),
+                                  _ptr(workspace), workspace_bytes, _stream_ptr(stream)), "wushkv_decode_attn")
+
+
+def unpack_debug(cache: wushkv_cache, slot, kv_head, which, pos0, n, codes, scale, zero, stream=None):
+    _check(lib.wushkv_unpack_debug(C.byref(cache), slot, kv_head, which, pos0, n, _ptr(codes), _ptr(scale),
+                                   _ptr(zero), _stream_ptr(stream)), "wushkv_unpack_debug")
+
+
+class PagedCache:
+    """Owns the device buffers of one layer's cache (torch tensors) and the filled ``wushkv_cache``
+    descriptor.  Pure bookkeeping: page-table assignment and allocation, no arithmetic."""
+
+    def __init__(self, n_q, n_kv, bits, n_slots, max_seq_len, s_sink, s_keep, s_flush, kappa_k, kappa_v,
+                 T_K, T_K_invT, sm_scale=None, boundary_lag=0, ring_cap=None, device="cuda", page_order=None):
+        import torch
+        d, page_tokens = 128, 64
+        self.torch = torch
+        self.device = torch.device(device)
+        self.n_q, self.n_kv, self.bits, self.n_slots = n_q, n_kv, bits, n_slots
+        self.max_pages = (max_seq_len + page_tokens - 1) // page_tokens
+        n_pages = n_slots * self.max_pages
+        self.page_bytes = page_bytes(n_kv, d, bits, page_tokens)
+        self.pages = torch.zeros(n_pages * self.page_bytes, dtype=torch.uint8, device=self.device)
+        order = np.arange(n_pages) if page_order is None else np.asarray(page_order)
+        self.page_table = torch.from_numpy(order.reshape(n_slots, self.max_pages).astype(np.int32)).to(self.device)
+        self.ring_cap = ring_cap if ring_cap is not None else s_keep + s_flush - 1 + boundary_lag
+        self.sink_kv = torch.zeros((n_slots, n_kv, 2, max(s_sink, 1), d), dtype=torch.bfloat16, device=self.device)
+        self.ring_kv = torch.zeros((n_slots, n_kv, 2, self.ring_cap, d), dtype=torch.bfloat16, device=self.device)
+        self.T_K = torch.as_tensor(np.ascontiguousarray(T_K, dtype=np.float32)).to(self.device)
+        self.T_K_invT = torch.as_tensor(np.ascontiguousarray(T_K_invT, dtype=np.float32)).to(self.device)
+        self.dev_status = torch.zeros(1, dtype=torch.int32, device=self.device)
+        self.desc = wushkv_cache(
+            n_q=n_q, n_kv=n_kv, d=d, bits=bits, page_tokens=page_tokens, s_sink=s_sink, s_keep=s_keep, s_flush=s_flush,
+            boundary_lag=boundary_lag, n_slots=n_slots, max_pages=self.max_pages, ring_cap=self.ring_cap,
+            kappa_k=kappa_k, kappa_v=kappa_v, sm_scale=(sm_scale if sm_scale is not None else 1.0 / np.sqrt(d)),
+            reserved=0, n_pages=n_pages, pages=self.pages.data_ptr(), page_table=self.page_table.data_ptr(),
+            sink_kv=self.sink_kv.data_ptr(), ring_kv=self.ring_kv.data_ptr(), T_K=self.T_K.data_ptr(),
+            T_K_invT=self.T_K_invT.data_ptr(), dev_status=self.dev_status.data_ptr())
+
+    def status(self) -> int:
+        return int(self.dev_status.item())

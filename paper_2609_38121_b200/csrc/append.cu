@@ -1,0 +1,335 @@
+// Quantize-on-append (Algorithm 2 lines 3-4 and 9-12; quantizer: Section 5.3 Eq. 6).
+//
+// Warp-per-vector path: one warp owns one (new token, KV head) pair.  It computes k' = T_K k on
+// CUDA cores against a transposed copy of T_K in shared memory (keys only), then for k' and for v:
+// finds the clip range (min, max and the two order statistics around rank kappa*(d-1) of |x| by
+// repeated warp-wide maximum extraction), derives the fp16 step / offset, rounds the codes with
+// the STORED step and offset, and scatters the codes into the fragment-ordered page record.
+// The bf16 copies for the sink buffer and the recent ring are written by the same warp.
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+
+#include "host_common.h"
+#include "layout.cuh"
+
+namespace wushkv {
+
+constexpr unsigned FULL = 0xffffffffu;
+constexpr int TT_STRIDE = 132;   // floats per row of the transposed transform in shared memory
+
+struct ClipRule {     // rank rule of quantile_kappa(|x|) with linear interpolation
+    int rounds;       // extraction rounds: the last yields a[lo], the one before a[lo+1]
+    float frac;       // pos - lo
+};
+
+struct AppendParams {
+    CacheView c;
+    int batch, total_new, tokens_per_cta;
+    const int* slot;
+    const int* seq_len;
+    const int* cu_new;
+    const unsigned short* K_new;
+    const unsigned short* V_new;
+    ClipRule rule_k, rule_v;
+};
+
+__device__ __forceinline__ void cswap_desc(unsigned& a, unsigned& b) {
+    const unsigned hi = max(a, b), lo = min(a, b);
+    a = hi; b = lo;
+}
+
+__device__ __forceinline__ unsigned order_key(float x) {       // monotone float -> uint map
+    const unsigned u = __float_as_uint(x);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float order_key_inv(unsigned k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+// Eq. 6 for the 128-vector held as x[4] per lane (channels 4*lane .. 4*lane+3).  Returns the four
+// codes of this lane and the stored (fp16) step and offset.
+template <int BITS>
+__device__ __forceinline__ void quantize_vec(const float (&x)[4], ClipRule rule, int lane, int (&code)[4],
+                                             __half& step_h, __half& xmin_h) {
+    constexpr int LEVELS = (1 << BITS) - 1;
+    // ---- the two order statistics of |x| around rank kappa*(d-1)
+    unsigned u0 = __float_as_uint(x[0]) & 0x7fffffffu, u1 = __float_as_uint(x[1]) & 0x7fffffffu;
+    unsigned u2 = __float_as_uint(x[2]) & 0x7fffffffu, u3 = __float_as_uint(x[3]) & 0x7fffffffu;
+    cswap_desc(u0, u1); cswap_desc(u2, u3); cswap_desc(u0, u2); cswap_desc(u1, u3); cswap_desc(u1, u2);
+    unsigned a_lo = 0, a_hi = 0;
+    for (int r = 0; r < rule.rounds; ++r) {
+        const unsigned m = __reduce_max_sync(FULL, u0);
+        const unsigned owners = __ballot_sync(FULL, u0 == m);
+        if (lane == __ffs(owners) - 1) { u0 = u1; u1 = u2; u2 = u3; u3 = 0; }
+        a_hi = a_lo;
+        a_lo = m;
+    }
+    if (rule.rounds == 1) a_hi = a_lo;
+    const float alo = __uint_as_float(a_lo), ahi = __uint_as_float(a_hi);
+    const float q = alo + rule.frac * (ahi - alo);
+    // ---- extremes of x
+    const float lmin = fminf(fminf(x[0], x[1]), fminf(x[2], x[3]));
+    const float lmax = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+    const float vmin = order_key_inv(__reduce_min_sync(FULL, order_key(lmin)));
+    const float vmax = order_key_inv(__reduce_max_sync(FULL, order_key(lmax)));
+    const float x_min = fmaxf(vmin, -q);
+    const float x_max = fminf(vmax, q);
+    const float step = __fdiv_rn(x_max - x_min, static_cast<float>(LEVELS));
+    step_h = __float2half_rn(fminf(fmaxf(step, -65504.f), 65504.f));
+    xmin_h = __float2half_rn(fminf(fmaxf(x_min, -65504.f), 65504.f));
+    const float step_s = __half2float(step_h), xmin_s = __half2float(xmin_h);
+    const float inv = step_s > 0.f ? __frcp_rn(step_s) : 0.f;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const float t = rintf((x[e] - xmin_s) * inv);
+        code[e] = static_cast<int>(fminf(fmaxf(t, 0.f), static_cast<float>(LEVELS)));
+    }
+}
+
+// Scatter one token's K codes (lane holds channels 4*lane..+3) into the record; r = token row in page.
+template <int BITS>
+__device__ __forceinline__ void store_k_codes(unsigned char* rec, int r, const int (&code)[4], int lane) {
+    const int bi = r >> 4, rr = r & 15, g = rr & 7, rs = rr >> 3;
+    const int s = lane >> 2;                            // k-step of all four channels of this lane
+    const int sh = (BITS == 2) ? 2 * s : 4 * (s & 3);
+    unsigned wa = (static_cast<unsigned>(code[0]) << sh) | (static_cast<unsigned>(code[1]) << (16 + sh));
+    unsigned wb = (static_cast<unsigned>(code[2]) << sh) | (static_cast<unsigned>(code[3]) << (16 + sh));
+    wa |= __shfl_xor_sync(FULL, wa, 4);  wb |= __shfl_xor_sync(FULL, wb, 4);
+    wa |= __shfl_xor_sync(FULL, wa, 8);  wb |= __shfl_xor_sync(FULL, wb, 8);
+    if (BITS == 2) { wa |= __shfl_xor_sync(FULL, wa, 16); wb |= __shfl_xor_sync(FULL, wb, 16); }
+    const int w = (lane & 3) >> 1, ta = 2 * (lane & 1);
+    if (BITS == 2) {
+        if (lane < 4) {
+            unsigned char* p = rec + bi * 512 + 16 * (4 * g + ta) + 8 * rs + 4 * w;
+            *reinterpret_cast<unsigned*>(p) = wa;
+            *reinterpret_cast<unsigned*>(p + 16) = wb;
+        }
+    } else {
+        if ((lane & 12) == 0) {                         // lanes 0..3 (k-steps 0..3) and 16..19 (k-steps 4..7)
+            const int j = 2 * (lane >> 4) + w;
+            unsigned char* p = rec + bi * 1024 + 512 * rs + 16 * (4 * g + ta) + 4 * j;
+            *reinterpret_cast<unsigned*>(p) = wa;
+            *reinterpret_cast<unsigned*>(p + 16) = wb;
+        }
+    }
+}
+
+template <int BITS>
+__device__ __forceinline__ void store_v_codes(unsigned char* rec, int r, const int (&code)[4], int lane) {
+    const int bi = r >> 4, rr = r & 15, ps = rr >> 3, t = (rr & 7) >> 1, hi = rr & 1;
+    const int i = lane >> 2;                            // channel block of this lane's channels
+    const int sh = (BITS == 2) ? 2 * i : 4 * (i & 3);
+    unsigned wa = (static_cast<unsigned>(code[0]) << sh) | (static_cast<unsigned>(code[1]) << (16 + sh));
+    unsigned wb = (static_cast<unsigned>(code[2]) << sh) | (static_cast<unsigned>(code[3]) << (16 + sh));
+    wa |= __shfl_xor_sync(FULL, wa, 4);  wb |= __shfl_xor_sync(FULL, wb, 4);
+    wa |= __shfl_xor_sync(FULL, wa, 8);  wb |= __shfl_xor_sync(FULL, wb, 8);
+    if (BITS == 2) { wa |= __shfl_xor_sync(FULL, wa, 16); wb |= __shfl_xor_sync(FULL, wb, 16); }
+    const int rsel = (lane & 3) >> 1, g0 = 4 * (lane & 1);
+    unsigned char* base;
+    bool writer;
+    if (BITS == 2) {
+        writer = lane < 4;
+        base = rec + v_codes_offset(2) + bi * 512 + 4 * (2 * ps + rsel) + 2 * hi;
+    } else {
+        writer = (lane & 12) == 0;
+        base = rec + v_codes_offset(4) + bi * 1024 + 512 * ps + 4 * (2 * rsel + (lane >> 4)) + 2 * hi;
+    }
+    if (writer) {
+        *reinterpret_cast<unsigned short*>(base + 16 * (4 * (g0 + 0) + t)) = static_cast<unsigned short>(wa & 0xffffu);
+        *reinterpret_cast<unsigned short*>(base + 16 * (4 * (g0 + 1) + t)) = static_cast<unsigned short>(wa >> 16);
+        *reinterpret_cast<unsigned short*>(base + 16 * (4 * (g0 + 2) + t)) = static_cast<unsigned short>(wb & 0xffffu);
+        *reinterpret_cast<unsigned short*>(base + 16 * (4 * (g0 + 3) + t)) = static_cast<unsigned short>(wb >> 16);
+    }
+}
+
+// Where a new token goes; false (with a status bit) if it cannot be stored.
+struct TokenSlot {
+    int b, slot, pos, s_final;
+    unsigned char* rec;      // this head's record of the token's page
+    int r;                   // row inside the page
+};
+
+__device__ __forceinline__ bool locate_token(const AppendParams& P, int token, int head, TokenSlot& ts) {
+    int lo = 0, hi = P.batch;                 // largest b with cu_new[b] <= token
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(P.cu_new + mid) <= token) lo = mid; else hi = mid;
+    }
+    ts.b = lo;
+    ts.slot = __ldg(P.slot + lo);
+    const int s0 = __ldg(P.seq_len + lo);
+    const int first = __ldg(P.cu_new + lo), last = __ldg(P.cu_new + lo + 1);
+    ts.pos = s0 + (token - first);
+    ts.s_final = s0 + (last - first);
+    if (ts.slot < 0 || ts.slot >= P.c.n_slots || s0 < 0) { atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_SLOT); return false; }
+    const int pidx = ts.pos / PAGE_TOKENS;
+    if (pidx >= P.c.max_pages) { atomicOr(P.c.dev_status, WUSHKV_DEV_PAGE_TABLE_FULL); return false; }
+    const int page = __ldg(P.c.page_table + static_cast<long long>(ts.slot) * P.c.max_pages + pidx);
+    if (page < 0 || page >= P.c.n_pages) { atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_PAGE_ID); return false; }
+    ts.rec = P.c.pages + (static_cast<long long>(page) * P.c.n_kv + head) * record_bytes(P.c.bits);
+    ts.r = ts.pos % PAGE_TOKENS;
+    return true;
+}
+
+// bf16 copies for the sink buffer and the recent ring (Section 4.4): which = 0 keys, 1 values.
+__device__ __forceinline__ void store_window_copy(const AppendParams& P, const TokenSlot& ts, int head, int which,
+                                                  uint2 four_bf16, int lane) {
+    const CacheView& c = P.c;
+    if (ts.pos < c.s_sink) {
+        unsigned short* dst = c.sink_kv + (((static_cast<long long>(ts.slot) * c.n_kv + head) * 2 + which) * c.s_sink + ts.pos) * D;
+        reinterpret_cast<uint2*>(dst)[lane] = four_bf16;
+    }
+    if (ts.pos >= ts.s_final - c.ring_cap) {
+        unsigned short* dst = c.ring_kv + (((static_cast<long long>(ts.slot) * c.n_kv + head) * 2 + which) * c.ring_cap + ts.pos % c.ring_cap) * D;
+        reinterpret_cast<uint2*>(dst)[lane] = four_bf16;
+    }
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(256) append_rows_kernel(AppendParams P) {
+    extern __shared__ __align__(16) float Tt[];          // Tt[j * TT_STRIDE + i] = T[i][j]
+    const int head = blockIdx.y;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const float* T = P.c.T_K + static_cast<long long>(head) * D * D;
+    for (int idx = threadIdx.x; idx < D * D; idx += blockDim.x) {
+        const int i = idx >> 7, j = idx & 127;
+        Tt[j * TT_STRIDE + i] = __ldg(T + idx);
+    }
+    __syncthreads();
+    const int tok0 = blockIdx.x * P.tokens_per_cta;
+    const int tok1 = min(tok0 + P.tokens_per_cta, P.total_new);
+    for (int token = tok0 + warp; token < tok1; token += nwarps) {
+        TokenSlot ts;
+        if (!locate_token(P, token, head, ts)) continue;
+        const long long row = (static_cast<long long>(token) * P.c.n_kv + head) * D;
+        // ---------------- keys: k' = T k (Algorithm 2 line 3), fp32 accumulation of exact bf16 products
+        const uint2 kraw = __ldg(reinterpret_cast<const uint2*>(P.K_new + row) + lane);
+        float kin[4] = {bf16_bits_to_float(kraw.x & 0xffff), bf16_bits_to_float(kraw.x >> 16),
+                        bf16_bits_to_float(kraw.y & 0xffff), bf16_bits_to_float(kraw.y >> 16)};
+        float x[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+        for (int jj = 0; jj < 32; ++jj) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float kj = __shfl_sync(FULL, kin[e], jj);
+                const float4 tt = *reinterpret_cast<const float4*>(Tt + (4 * jj + e) * TT_STRIDE + 4 * lane);
+                x[0] = fmaf(tt.x, kj, x[0]); x[1] = fmaf(tt.y, kj, x[1]);
+                x[2] = fmaf(tt.z, kj, x[2]); x[3] = fmaf(tt.w, kj, x[3]);
+            }
+        }
+        int code[4];
+        __half step_h, xmin_h;
+        quantize_vec<BITS>(x, P.rule_k, lane, code, step_h, xmin_h);
+        store_k_codes<BITS>(ts.rec, ts.r, code, lane);
+        __half* meta = reinterpret_cast<__half*>(ts.rec + meta_location(BITS, ts.r));
+        if (lane == 0) { meta[0] = step_h; meta[1] = xmin_h; }
+        uint2 kb;
+        kb.x = float_to_bf16_bits(x[0]) | (static_cast<unsigned>(float_to_bf16_bits(x[1])) << 16);
+        kb.y = float_to_bf16_bits(x[2]) | (static_cast<unsigned>(float_to_bf16_bits(x[3])) << 16);
+        store_window_copy(P, ts, head, 0, kb, lane);
+        // ---------------- values: already in the folded basis, no transform
+        const uint2 vraw = __ldg(reinterpret_cast<const uint2*>(P.V_new + row) + lane);
+        float v[4] = {bf16_bits_to_float(vraw.x & 0xffff), bf16_bits_to_float(vraw.x >> 16),
+                      bf16_bits_to_float(vraw.y & 0xffff), bf16_bits_to_float(vraw.y >> 16)};
+        quantize_vec<BITS>(v, P.rule_v, lane, code, step_h, xmin_h);
+        store_v_codes<BITS>(ts.rec, ts.r, code, lane);
+        if (lane == 0) { meta[2] = step_h; meta[3] = xmin_h; }
+        store_window_copy(P, ts, head, 1, vraw, lane);
+    }
+}
+
+__global__ void advance_len_kernel(int batch, int* seq_len, const int* cu_new) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < batch) seq_len[b] += cu_new[b + 1] - cu_new[b];
+}
+
+__global__ void unpack_debug_kernel(CacheView c, int slot, int head, int which, int pos0, int n,
+                                    unsigned char* codes, float* scale, float* zero) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= n * D) return;
+    const int tok = idx >> 7, ch = idx & 127;
+    const int pos = pos0 + tok;
+    const int pidx = pos / PAGE_TOKENS, r = pos % PAGE_TOKENS;
+    if (pidx >= c.max_pages) { atomicOr(c.dev_status, WUSHKV_DEV_PAGE_TABLE_FULL); return; }
+    const int page = c.page_table[static_cast<long long>(slot) * c.max_pages + pidx];
+    if (page < 0 || page >= c.n_pages) { atomicOr(c.dev_status, WUSHKV_DEV_BAD_PAGE_ID); return; }
+    const unsigned char* rec = c.pages + (static_cast<long long>(page) * c.n_kv + head) * record_bytes(c.bits);
+    int off, bit;
+    if (which == 0) k_code_location(c.bits, r, ch, off, bit); else v_code_location(c.bits, r, ch, off, bit);
+    const unsigned hw = *reinterpret_cast<const unsigned short*>(rec + off);
+    codes[idx] = static_cast<unsigned char>((hw >> bit) & ((1u << c.bits) - 1u));
+    if (ch == 0) {
+        const __half* meta = reinterpret_cast<const __half*>(rec + meta_location(c.bits, r));
+        scale[tok] = __half2float(meta[2 * which]);
+        zero[tok] = __half2float(meta[2 * which + 1]);
+    }
+}
+
+static ClipRule make_rule(float kappa) {
+    const double pos = static_cast<double>(kappa) * (D - 1);
+    int lo = static_cast<int>(std::floor(pos));
+    lo = std::min(std::max(lo, 0), D - 1);
+    ClipRule r;
+    if (lo >= D - 1) { r.rounds = 1; r.frac = 0.f; }
+    else { r.rounds = D - lo; r.frac = static_cast<float>(pos - lo); }
+    return r;
+}
+
+}  // namespace wushkv
+
+using namespace wushkv;
+
+extern "C" int wushkv_append(const wushkv_cache* cache, int32_t batch, const int32_t* slot, int32_t* seq_len,
+                             const int32_t* cu_new, int32_t total_new, int32_t max_new,
+                             const uint16_t* K_new, const uint16_t* V_new, void* stream) {
+    AppendParams P;
+    const int rc = make_view(cache, P.c);
+    if (rc != WUSHKV_OK) return rc;
+    if (batch <= 0 || !slot || !seq_len || !cu_new || total_new < 0 || max_new < 0 || max_new > total_new) return WUSHKV_EINVAL;
+    if (total_new == 0) return WUSHKV_OK;
+    if (!K_new || !V_new || !aligned(K_new, 16) || !aligned(V_new, 16)) return WUSHKV_EINVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    P.batch = batch; P.total_new = total_new;
+    P.slot = slot; P.seq_len = seq_len; P.cu_new = cu_new;
+    P.K_new = K_new; P.V_new = V_new;
+    P.rule_k = make_rule(cache->kappa_k);
+    P.rule_v = make_rule(cache->kappa_v);
+    // enough CTAs to fill the machine, but at least 8 tokens each to amortise the transform load
+    const int want_ctas = std::max(1, 2 * sm_count() / P.c.n_kv);
+    int tpc = (total_new + want_ctas - 1) / want_ctas;
+    tpc = std::max(8, ((tpc + 7) / 8) * 8);
+    P.tokens_per_cta = tpc;
+    const dim3 grid((total_new + tpc - 1) / tpc, P.c.n_kv);
+    const size_t smem = static_cast<size_t>(D) * TT_STRIDE * sizeof(float);
+    cudaError_t e;
+    if (P.c.bits == 2) {
+        e = cudaFuncSetAttribute(append_rows_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return WUSHKV_ECUDA;
+        append_rows_kernel<2><<<grid, 256, smem, st>>>(P);
+    } else {
+        e = cudaFuncSetAttribute(append_rows_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return WUSHKV_ECUDA;
+        append_rows_kernel<4><<<grid, 256, smem, st>>>(P);
+    }
+    if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
+    advance_len_kernel<<<(batch + 127) / 128, 128, 0, st>>>(batch, seq_len, cu_new);
+    if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
+    return WUSHKV_OK;
+}
+
+extern "C" int wushkv_unpack_debug(const wushkv_cache* cache, int32_t slot, int32_t kv_head, int32_t which,
+                                   int32_t pos0, int32_t n, uint8_t* codes, float* scale, float* zero, void* stream) {
+    CacheView v;
+    const int rc = make_view(cache, v);
+    if (rc != WUSHKV_OK) return rc;
+    if (slot < 0 || slot >= v.n_slots || kv_head < 0 || kv_head >= v.n_kv || (which != 0 && which != 1) || pos0 < 0 || n < 0 ||
+        !codes || !scale || !zero)
+        return WUSHKV_EINVAL;
+    if (n == 0) return WUSHKV_OK;
+    const long long total = static_cast<long long>(n) * D;
+    unpack_debug_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        v, slot, kv_head, which, pos0, n, codes, scale, zero);
+    return cudaGetLastError() == cudaSuccess ? WUSHKV_OK : WUSHKV_ECUDA;
+}

@@ -1,0 +1,56 @@
+// Host-side argument validation shared by the entry points.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "../../include/wushkv.h"
+#include "layout.cuh"
+
+namespace wushkv {
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+// Checks the cache description and fills the device-side view.  Returns WUSHKV_OK or WUSHKV_EINVAL / ECAPACITY.
+inline int make_view(const wushkv_cache* c, CacheView& v) {
+    if (!c) return WUSHKV_EINVAL;
+    if (c->d != D || c->page_tokens != PAGE_TOKENS) return WUSHKV_EINVAL;
+    if (c->bits != 2 && c->bits != 4) return WUSHKV_EINVAL;
+    if (c->n_kv <= 0 || c->n_q <= 0 || c->n_q % c->n_kv != 0) return WUSHKV_EINVAL;
+    const int G = c->n_q / c->n_kv;
+    if (G < 1 || G > 8) return WUSHKV_EINVAL;
+    if (c->s_sink < 0 || c->s_keep < 1 || c->s_flush < 1 || c->boundary_lag < 0) return WUSHKV_EINVAL;
+    if (c->n_slots <= 0 || c->max_pages <= 0 || c->n_pages <= 0) return WUSHKV_EINVAL;
+    if (!(c->kappa_k >= 0.f && c->kappa_k <= 1.f) || !(c->kappa_v >= 0.f && c->kappa_v <= 1.f)) return WUSHKV_EINVAL;
+    if (!(c->sm_scale > 0.f)) return WUSHKV_EINVAL;
+    if (!c->pages || !c->page_table || !c->ring_kv || !c->T_K || !c->T_K_invT || !c->dev_status) return WUSHKV_EINVAL;
+    if (c->s_sink > 0 && !c->sink_kv) return WUSHKV_EINVAL;
+    if (!aligned(c->pages, 256) || !aligned(c->ring_kv, 16) || !aligned(c->sink_kv, 16) || !aligned(c->T_K, 16) ||
+        !aligned(c->T_K_invT, 16) || !aligned(c->page_table, 4) || !aligned(c->dev_status, 4))
+        return WUSHKV_EINVAL;
+    if (c->ring_cap < c->s_keep + c->s_flush - 1 + c->boundary_lag) return WUSHKV_ECAPACITY;
+    v.n_q = c->n_q; v.n_kv = c->n_kv; v.bits = c->bits;
+    v.s_sink = c->s_sink; v.s_keep = c->s_keep; v.s_flush = c->s_flush; v.lag = c->boundary_lag;
+    v.n_slots = c->n_slots; v.max_pages = c->max_pages; v.ring_cap = c->ring_cap; v.G = G;
+    v.n_pages = c->n_pages;
+    v.pages = static_cast<unsigned char*>(c->pages);
+    v.page_table = c->page_table;
+    v.sink_kv = static_cast<unsigned short*>(c->sink_kv);
+    v.ring_kv = static_cast<unsigned short*>(c->ring_kv);
+    v.T_K = c->T_K; v.T_K_invT = c->T_K_invT;
+    v.dev_status = c->dev_status;
+    v.sm_scale = c->sm_scale;
+    return WUSHKV_OK;
+}
+
+inline int sm_count() {
+    static int cached = 0;
+    if (cached == 0) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+        cached = n;
+    }
+    return cached;
+}
+
+}  // namespace wushkv

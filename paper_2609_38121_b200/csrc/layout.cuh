@@ -1,0 +1,109 @@
+// Physical layout of one packed (page, KV head) record and small shared device helpers.
+//
+// A record holds PAGE_TOKENS = 64 tokens as 4 blocks of 16 tokens:
+//     [K codes: 4 blocks][V codes: 4 blocks][meta: 4 blocks x 128 B]
+// with a code block of 16*16*bits/... = 512 B (2-bit) or 1024 B (4-bit).  Inside a code block
+// byte 16*L .. 16*L+15 (of each 512-byte half) belongs to lane L = 4*g + t of the decode warp,
+// so that one 16-byte shared-memory load per lane yields exactly the words that lane turns into
+// mma.m16n8k16 A-fragments with a mask (and one shift) per register:
+//
+//  K block (A = codes[16 tokens x 16 channels] per k-step s, channels 16s..16s+15):
+//    token row rr -> g = rr & 7, rs = rr >> 3;  channel ch -> s = ch >> 4, r16 = ch & 15,
+//    w = r16 >> 3, t = (r16 & 7) >> 1, hi = r16 & 1.
+//    2-bit: word (rs, w) of lane (g,t) at byte 16L + 8rs + 4w; code at bits 16hi + 2s.
+//    4-bit: 512-byte half rs; word j = 2(s>>2) + w at byte 512rs + 16L + 4j; code at bits 16hi + 4(s&3).
+//  V block (A = codes^T[16 channels x 16 tokens] per channel block i, channels 16i..16i+15):
+//    token rr -> ps = rr >> 3, t = (rr & 7) >> 1, hi = rr & 1;  channel ch -> i = ch >> 4,
+//    r16 = ch & 15, rsel = r16 >> 3, g = r16 & 7.
+//    2-bit: half-word hi of word (ps, rsel) at byte 16L + 4(2ps + rsel) + 2hi; code at bits 2i.
+//    4-bit: 512-byte half ps; word (rsel, j = i>>2) at byte 512ps + 16L + 4(2rsel + j) + 2hi; code at bits 4(i&3).
+//  meta block bi: token rr -> 8 bytes {K step, K x_min, V step, V x_min} (fp16) at 128bi + 16(rr&7) + 8(rr>>3).
+//
+// Masked out of a 16-bit lane and read as an fp16 bit pattern, a code field that lies inside bits
+// 0..10 is the exact value code * 2^(shift-24) (fp16 subnormals and the first binade are linear in
+// the bit pattern), so no int->float conversion is ever executed; the power-of-two factors are
+// folded into the query fragments and the output epilogue.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace wushkv {
+
+constexpr int D = 128;
+constexpr int PAGE_TOKENS = 64;
+constexpr int BLOCK_TOKENS = 16;
+constexpr int BLOCKS_PER_PAGE = PAGE_TOKENS / BLOCK_TOKENS;
+
+__host__ __device__ constexpr int code_block_bytes(int bits) { return BLOCK_TOKENS * D * bits / 8; }
+__host__ __device__ constexpr int k_codes_offset(int) { return 0; }
+__host__ __device__ constexpr int v_codes_offset(int bits) { return BLOCKS_PER_PAGE * code_block_bytes(bits); }
+__host__ __device__ constexpr int meta_offset(int bits) { return 2 * BLOCKS_PER_PAGE * code_block_bytes(bits); }
+__host__ __device__ constexpr int record_bytes(int bits) { return meta_offset(bits) + PAGE_TOKENS * 8; }
+
+// Byte offset (within the record) of the 16-bit half-word holding K code (token r, channel ch) and
+// the bit position of the code inside that half-word.
+__host__ __device__ inline void k_code_location(int bits, int r, int ch, int& byte_off, int& bit) {
+    const int bi = r >> 4, rr = r & 15, g = rr & 7, rs = rr >> 3;
+    const int s = ch >> 4, r16 = ch & 15, w = r16 >> 3, t = (r16 & 7) >> 1, hi = r16 & 1;
+    const int L = 4 * g + t;
+    if (bits == 2) {
+        byte_off = bi * 512 + 16 * L + 8 * rs + 4 * w + 2 * hi;
+        bit = 2 * s;
+    } else {
+        byte_off = bi * 1024 + 512 * rs + 16 * L + 4 * (2 * (s >> 2) + w) + 2 * hi;
+        bit = 4 * (s & 3);
+    }
+}
+
+__host__ __device__ inline void v_code_location(int bits, int r, int ch, int& byte_off, int& bit) {
+    const int bi = r >> 4, rr = r & 15, ps = rr >> 3, t = (rr & 7) >> 1, hi = rr & 1;
+    const int i = ch >> 4, r16 = ch & 15, rsel = r16 >> 3, g = r16 & 7;
+    const int L = 4 * g + t;
+    if (bits == 2) {
+        byte_off = v_codes_offset(2) + bi * 512 + 16 * L + 4 * (2 * ps + rsel) + 2 * hi;
+        bit = 2 * i;
+    } else {
+        byte_off = v_codes_offset(4) + bi * 1024 + 512 * ps + 16 * L + 4 * (2 * rsel + (i >> 2)) + 2 * hi;
+        bit = 4 * (i & 3);
+    }
+}
+
+__host__ __device__ inline int meta_location(int bits, int r) {
+    const int bi = r >> 4, rr = r & 15;
+    return meta_offset(bits) + 128 * bi + 16 * (rr & 7) + 8 * (rr >> 3);
+}
+
+// Number of positions read from the packed codes when S positions are cached (closed form of the
+// boundary recurrence of Algorithm 2 lines 7-8); they are [s_sink, s_sink + n).
+__host__ __device__ inline int n_quantized(int S, int s_sink, int s_keep, int s_flush) {
+    const int room = S - s_keep - s_sink;
+    if (room < s_flush) return 0;
+    return (room / s_flush) * s_flush;
+}
+
+// Device-side mirror of the parts of the cache description that kernels need.
+struct CacheView {
+    int n_q, n_kv, bits, s_sink, s_keep, s_flush, lag;
+    int n_slots, max_pages, ring_cap, G;
+    long long n_pages;
+    unsigned char* pages;
+    const int* page_table;
+    unsigned short* sink_kv;
+    unsigned short* ring_kv;
+    const float* T_K;
+    const float* T_K_invT;
+    int* dev_status;
+    float sm_scale;
+};
+
+__device__ __forceinline__ float bf16_bits_to_float(unsigned short b) {
+    return __uint_as_float(static_cast<unsigned>(b) << 16);
+}
+__device__ __forceinline__ unsigned short float_to_bf16_bits(float x) {   // round to nearest even
+    unsigned u = __float_as_uint(x);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return static_cast<unsigned short>((u >> 16) | 0x40);
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return static_cast<unsigned short>(u >> 16);
+}
+
+}  // namespace wushkv

@@ -1,0 +1,162 @@
+"""GPU parity tests proper: the CUDA library, called through its C ABI, against the float64 oracle on
+the same seeded inputs.  Sizes are what the oracle finishes in seconds while still spanning several
+pages, several splits and ragged tails."""
+import numpy as np
+import pytest
+
+from paper_2609_38121_b200 import workloads as W
+from tests.harness import CODE_MISMATCH_MAX, Layer
+
+pytestmark = pytest.mark.gpu
+
+
+def _wl(n_q, n_kv, seed, batch=1, theta=1e4, rmsnorm=False):
+    return W.LayerWorkload(dict(seed=seed, batch=batch, n_q=n_q, n_kv=n_kv, ctx=0, theta=theta, bits=2, s_sink=4,
+                                s_keep=64, rmsnorm=rmsnorm, ragged=None, prefill_chunk=0))
+
+
+def _check_window_copies(L):
+    """bf16 sink / ring contents: keys are bf16(T k) (rare one-ulp flips from fp32 vs fp64 summation
+    order are allowed), values are the input itself, bit for bit."""
+    for b in range(L.batch):
+        S = L.lengths[b]
+        if S == 0:
+            continue
+        kc, km, vc, vm, kb_o, vb_o = L.oracle[b].arrays()
+        kb, vb = L.gpu_window_arrays(b)
+        have = np.isfinite(kb[:, 0, 0])
+        assert have[:min(S, L.s_sink)].all() and have[max(0, S - L.cache.ring_cap):].all()
+        assert np.array_equal(vb[have], vb_o[have])
+        d = np.abs(kb[have] - kb_o[have])
+        ulp = np.maximum(np.abs(kb_o[have]), 1e-30) * 2.0 ** -7
+        assert np.all(d <= ulp), "bf16 key copy differs by more than one ulp"
+        assert np.mean(d > 0) < 2e-3
+
+
+@pytest.mark.parametrize("bits", [2, 4])
+def test_config0_tiny_layer(bits):
+    """Benchmark config 0: batch 1, 8 query / 2 KV heads, 2048 context, sink 4, recent 64."""
+    wl = W.LayerWorkload("cfg0")
+    L = Layer(wl, [2048], bits, 4, 64, 1)
+    L.fill()
+    assert L.seq_len.cpu().tolist() == [2048]
+    assert L.check_append_parity() <= CODE_MISMATCH_MAX
+    _check_window_copies(L)
+    assert L.check_decode_parity() <= 2e-3
+    assert L.cache.status() == 0
+
+
+@pytest.mark.parametrize("n_q,n_kv,bits", [(8, 1, 2), (8, 1, 4), (7, 1, 2), (14, 2, 4), (2, 2, 2), (6, 2, 2), (5, 1, 4), (3, 1, 2)])
+def test_group_sizes(n_q, n_kv, bits):
+    """Every query-group size 1..8 takes one of the two fragment modes; G = 7 with RMSNorm is the
+    Qwen-shaped layer of config 4, G = 8 the 70B-shaped layer of config 3."""
+    wl = _wl(n_q, n_kv, seed=10 + n_q, theta=1e6, rmsnorm=(n_q // n_kv == 7))
+    L = Layer(wl, [700], bits, 4, 128, 1)
+    L.fill()
+    assert L.check_append_parity() <= CODE_MISMATCH_MAX
+    assert L.check_decode_parity() <= 2e-3
+    assert L.cache.status() == 0
+
+
+@pytest.mark.parametrize("bits", [2, 4])
+def test_ragged_batch_shuffled_pages_and_flush_sizes(bits):
+    """Ragged lengths (config 2's structure, scaled down), page table in random order, S_flush > 1
+    so that the recent window breathes, and appends that straddle page boundaries."""
+    wl = _wl(8, 2, seed=21, batch=5, theta=5e5)
+    lengths = [1, 63, 64, 65, 1000]
+    for s_flush, lag in ((8, 0), (16, 1)):
+        L = Layer(wl, lengths, bits, 4, 64, s_flush, lag=lag, page_shuffle_seed=3, max_seq_len=1024)
+        steps = [[0, 10, 60, 3, 500], [1, 50, 3, 61, 436], [0, 2, 0, 0, 63], [0, 1, 1, 1, 1]]
+        for st in steps:
+            L.append_step(st)
+        assert L.seq_len.cpu().tolist() == lengths
+        assert L.check_append_parity() <= CODE_MISMATCH_MAX
+        _check_window_copies(L)
+        assert L.check_decode_parity() <= 2e-3
+        assert L.cache.status() == 0
+
+
+def test_window_edges_and_empty_sequences():
+    """Degenerate cases of Section 4.4: nothing cached, everything inside the sink, nothing quantized
+    yet (S <= S_sink + S_keep + S_flush - 1), exactly one flush group quantized."""
+    wl = _wl(4, 1, seed=30, batch=6)
+    s_sink, s_keep, s_flush = 4, 64, 8
+    lengths = [0, 3, 4, s_sink + s_keep + s_flush - 1, s_sink + s_keep + s_flush, 200]
+    L = Layer(wl, lengths, 2, s_sink, s_keep, s_flush, max_seq_len=256)
+    L.fill()
+    assert L.check_append_parity() <= CODE_MISMATCH_MAX
+    _check_window_copies(L)
+    assert L.check_decode_parity() <= 2e-3
+    assert L.cache.status() == 0
+
+
+def test_no_sink_and_kappa_one():
+    wl = _wl(4, 1, seed=31)
+    L = Layer(wl, [333], 4, 0, 1, 1, kappa_k=1.0, kappa_v=0.5)
+    L.fill()
+    assert L.check_append_parity() <= CODE_MISMATCH_MAX
+    assert L.check_decode_parity() <= 2e-3
+
+
+def test_decode_is_deterministic_and_split_invariant(monkeypatch):
+    """The split count changes only the summation order: outputs for different splits agree to fp32
+    rounding, and two identical calls agree bit for bit."""
+    wl = _wl(8, 2, seed=32)
+    L = Layer(wl, [3000], 2, 4, 64, 1)
+    L.fill()
+    outs = []
+    for cp in ("8", "8", "13", "64"):
+        monkeypatch.setenv("WUSHKV_CHUNK_PAGES", cp)
+        outs.append(L.decode()[0])
+    assert np.array_equal(outs[0], outs[1])
+    scale = np.max(np.abs(outs[0]))
+    assert np.max(np.abs(outs[2] - outs[0])) <= 1e-5 * scale
+    assert np.max(np.abs(outs[3] - outs[0])) <= 1e-5 * scale
+
+
+def test_device_side_errors_are_flagged_not_fatal():
+    """A position beyond the page table and a page id outside the pool set status bits; the calls
+    still return and the rest of the batch is processed."""
+    import torch
+    from paper_2609_38121_b200 import binding as B
+    wl = _wl(4, 1, seed=33, batch=2)
+    L = Layer(wl, [200, 200], 2, 4, 64, 1, max_seq_len=256)
+    L.fill()
+    assert L.cache.status() == 0
+    good, _ = L.decode()
+    # sequence 0 claims to be at the end of its page table: the append is skipped and flagged
+    L.seq_len[0] = 256
+    cu = torch.tensor([0, 1, 1], dtype=torch.int32, device="cuda")
+    tok = torch.zeros((1, 1, 128), dtype=torch.int16, device="cuda")
+    B.append(L.cache.desc, 2, L.slot, L.seq_len, cu, 1, 1, tok, tok)
+    torch.cuda.synchronize()
+    assert L.cache.status() & B.DEV_PAGE_TABLE_FULL
+    # a corrupt page table entry inside the quantized range is skipped by decode and flagged
+    L.seq_len[0] = 200
+    L.cache.dev_status.zero_()
+    L.cache.page_table[0, 1] = 10 ** 6
+    out, _ = L.decode()
+    assert L.cache.status() & B.DEV_BAD_PAGE_ID
+    assert np.all(np.isfinite(out))
+    assert np.array_equal(out[1], good[1])            # the healthy sequence is untouched
+
+
+def test_host_side_capacity_and_alignment_errors():
+    import torch
+    from paper_2609_38121_b200 import binding as B
+    wl = _wl(4, 1, seed=34)
+    L = Layer(wl, [100], 2, 4, 64, 1)
+    L.fill()
+    Q = torch.zeros((1, 4, 128), dtype=torch.int16, device="cuda")
+    Oo = torch.zeros((1, 4, 128), dtype=torch.float32, device="cuda")
+    ws = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.WushkvError) as e:
+        B.decode_attn(L.cache.desc, 1, L.slot, L.seq_len, 100, Q, Oo, ws, 16)
+    assert e.value.status == B.ECAPACITY
+    with pytest.raises(B.WushkvError) as e:
+        B.decode_attn(L.cache.desc, 1, L.slot, L.seq_len, 100, Q, Oo, ws[8:], (1 << 20) - 8)
+    assert e.value.status == B.EINVAL
+    L.cache.desc.ring_cap = 10
+    with pytest.raises(B.WushkvError) as e:
+        B.decode_attn(L.cache.desc, 1, L.slot, L.seq_len, 100, Q, Oo, ws, 1 << 20)
+    assert e.value.status == B.ECAPACITY
