@@ -1,0 +1,504 @@
+#!/usr/bin/env python
+"""Benchmark of the WUSH-KV hot path on B200: one "step" = quantize-on-append of the step's new
+tokens + decode attention over the packed cache, for one layer, on seeded synthetic inputs shaped
+like the named model layer.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg1] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is the metric of the benchmark definition: bytes of packed
+cache (codes + scale/zero + bf16 windows) that one decode step must read, divided by the time of the
+whole step (append + decode), with every input already resident in HBM.  `roofline` times the decode
+main kernel alone (CUDA events recorded around it by the library on the launching stream).  `e2e`
+repeats the steps through the host-buffer entry point (pinned host inputs copied in, result copied
+out, one synchronisation per step).  `cpu_baseline` times the float64 oracle on a bounded slice.
+With N > 1 every rank runs its own replica of the workload (the path has no cross-GPU exchange).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2609_38121_b200 import workloads as W  # noqa: E402
+
+METRIC = "2-bit decode-attn cache GB/s (fraction of HBM peak) @32k ctx; append tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+L2_BYTES = 126 * 2 ** 20
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_main_kernel launch at the named
+# workload, from the ncu capture summarised under profiles/ (None until captured).
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_hbm_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------------------------------------
+# workload on the GPU (product path only: library calls + torch for memory)
+# ------------------------------------------------------------------------------------------------
+def library_transforms(wl):
+    """T_K, T_K_invT (and a value transform for the generator) from the calibration batch, built by
+    the library's own host entry points."""
+    from paper_2609_38121_b200 import binding as B
+    Kc, Qc, Vraw = wl.calibration()
+    d = 128
+    M = np.zeros((wl.n_kv, d, d))
+    H = np.zeros((wl.n_kv, d, d))
+    B.accumulate_gram(W.f32_to_bf16_bits(Kc), W.f32_to_bf16_bits(Qc), M, H)
+    T, TinvT = B.build_transforms(M, H, W.GAMMA)
+    Mv = np.stack([Vraw[:, h].astype(np.float64).T @ Vraw[:, h].astype(np.float64) for h in range(wl.n_kv)])
+    Hv = np.stack([2 * sum(wl.W_O[h, g].astype(np.float64) @ wl.W_O[h, g].astype(np.float64).T for g in range(wl.G))
+                   for h in range(wl.n_kv)])
+    TV, _ = B.build_transforms(Mv, Hv, W.GAMMA)
+    return T, TinvT, TV
+
+
+class Session:
+    """A filled cache plus the per-step inputs of one config, resident on one GPU."""
+
+    def __init__(self, name, n_steps, device="cuda", seed_offset=0, verbose=False):
+        import torch
+        from paper_2609_38121_b200 import binding as B
+        self.torch, self.B = torch, B
+        cfg = dict(W.CONFIGS[name])
+        cfg["seed"] += 1000 * seed_offset
+        self.name, self.cfg = name, cfg
+        wl = self.wl = W.LayerWorkload(cfg)
+        self.n_steps = n_steps
+        self.chunk = cfg["prefill_chunk"]
+        self.batch = wl.batch
+        final = wl.lengths().astype(np.int64)
+        self.T, self.TinvT, self.TV = library_transforms(wl)
+        self.s_flush = 1
+        if self.chunk:
+            self.start_len = np.zeros(self.batch, np.int64)
+            self.max_seq_len = int(final.max())
+        else:
+            self.start_len = final - 1
+            self.max_seq_len = int(final.max()) + n_steps
+        self.cache = B.PagedCache(wl.n_q, wl.n_kv, cfg["bits"], self.batch, self.max_seq_len, cfg["s_sink"],
+                                  cfg["s_keep"], self.s_flush, W.KAPPA_K, W.KAPPA_V, self.T, self.TinvT, device=device)
+        dev = self.cache.device
+        self.slot = torch.arange(self.batch, dtype=torch.int32, device=dev)
+        self.seq_len = torch.zeros(self.batch, dtype=torch.int32, device=dev)
+        t0 = time.time()
+        if self.chunk:
+            ks, vs = [], []
+            for b in range(self.batch):
+                _, K, V = next(wl.sequence_tokens(b, self.chunk, T_V=self.TV, chunk=self.chunk))
+                ks.append(K)
+                vs.append(V)
+            self.K_chunk = self._dev_bf16(np.concatenate(ks))
+            self.V_chunk = self._dev_bf16(np.concatenate(vs))
+            self.cu_chunk = torch.arange(0, (self.batch + 1) * self.chunk, self.chunk, dtype=torch.int32, device=dev)
+            n_step_tok = 0
+        else:
+            n_step_tok = n_steps
+        # prefill everything before the timed steps (one library call per sequence)
+        step_k = np.zeros((max(n_step_tok, 1), self.batch, wl.n_kv, 128), np.float32)
+        step_v = np.zeros_like(step_k)
+        for b in range(self.batch):
+            n_pre = int(self.start_len[b])
+            ks, vs = [], []
+            for _, K, V in wl.sequence_tokens(b, n_pre + n_step_tok, T_V=self.TV):
+                ks.append(K)
+                vs.append(V)
+            K = np.concatenate(ks) if ks else np.zeros((0, wl.n_kv, 128), np.float32)
+            V = np.concatenate(vs) if vs else np.zeros((0, wl.n_kv, 128), np.float32)
+            if n_step_tok:
+                step_k[:, b] = K[n_pre:]
+                step_v[:, b] = V[n_pre:]
+            if n_pre:
+                counts = np.zeros(self.batch, np.int64)
+                counts[b] = n_pre
+                cu = torch.tensor(np.concatenate([[0], np.cumsum(counts)]).astype(np.int32), device=dev)
+                B.append(self.cache.desc, self.batch, self.slot, self.seq_len, cu, n_pre, n_pre,
+                         self._dev_bf16(K[:n_pre]), self._dev_bf16(V[:n_pre]))
+                torch.cuda.synchronize()
+        self.step_K = self._dev_bf16(step_k)
+        self.step_V = self._dev_bf16(step_v)
+        q = np.stack([wl.queries(b, int(final[b]) - 1) for b in range(self.batch)])
+        self.Q = self._dev_bf16(q)
+        self.q_host = q
+        self.step_k_host, self.step_v_host = step_k, step_v
+        self.cu_one = torch.arange(0, self.batch + 1, dtype=torch.int32, device=dev)
+        self.O = torch.zeros((self.batch, wl.n_q, 128), dtype=torch.float32, device=dev)
+        self.ws_bytes = B.decode_workspace_bytes(self.cache.desc, self.batch, self.max_seq_len)
+        self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device=dev)
+        self.base_len = self.seq_len.clone()
+        self.final = final
+        self.step_index = 0
+        if verbose:
+            print(f"[bench] {name}: cache filled in {time.time() - t0:.1f}s, status {self.cache.status()}", file=sys.stderr)
+
+    def _dev_bf16(self, x):
+        return self.torch.from_numpy(W.f32_to_bf16_bits(x).view(np.int16)).to(self.cache.device)
+
+    def rewind(self):
+        self.seq_len.copy_(self.base_len)
+        self.step_index = 0
+
+    def step(self, mid_event=None):
+        """Enqueue one step (device-resident inputs)."""
+        B = self.B
+        if self.chunk:
+            self.seq_len.zero_()
+            B.append(self.cache.desc, self.batch, self.slot, self.seq_len, self.cu_chunk, self.batch * self.chunk,
+                     self.chunk, self.K_chunk, self.V_chunk)
+        else:
+            i = self.step_index
+            B.append(self.cache.desc, self.batch, self.slot, self.seq_len, self.cu_one, self.batch, 1,
+                     self.step_K[i], self.step_V[i])
+            self.step_index += 1
+        if mid_event is not None:
+            mid_event.record()
+        B.decode_attn(self.cache.desc, self.batch, self.slot, self.seq_len, self.max_seq_len, self.Q, self.O,
+                      self.ws, self.ws_bytes)
+
+    # ---- algorithmic bytes of one step -----------------------------------------------------------
+    def lengths_at(self, step_no):
+        """Context lengths seen by the decode of the step_no-th step (1-based) since the prefill."""
+        return self.final if self.chunk else self.final - 1 + step_no
+
+    def decode_bytes(self, step_no=1):
+        c = self.cfg
+        per_q = 72 if c["bits"] == 2 else 136
+        total = 0
+        for S in self.lengths_at(step_no):
+            S = int(S)
+            room = S - c["s_keep"] - c["s_sink"]
+            nq = (room // self.s_flush) * self.s_flush if room >= self.s_flush else 0
+            total += self.wl.n_kv * (nq * per_q + (S - nq) * 512)
+        return total
+
+    def append_tokens(self):
+        return self.batch * (self.chunk if self.chunk else 1)
+
+    def launches_per_step(self):
+        return 2 + 3       # append: rows + length update; decode: prep + main + combine
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "50", "-i", str(gpu_index)], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.tmp.read().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        try:
+            os.unlink(self.tmp.name)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle arm
+# ------------------------------------------------------------------------------------------------
+class OracleSample:
+    """The float64 oracle on a bounded slice of the workload: ONE sequence and ONE KV head (with its
+    G query heads) at the config's full context.  A step appends one token and decodes."""
+
+    def __init__(self, name, ctx_cap=None):
+        from oracle import wushkv_oracle as O
+        self.O = O
+        cfg = dict(W.CONFIGS[name])
+        wl = self.wl = W.LayerWorkload(cfg)
+        self.cfg = cfg
+        G = wl.G
+        Kc, Qc, _ = wl.calibration()
+        M, H = O.gram_hessian(Kc[:, 0], np.stack([Qc[:, g] for g in range(G)]))
+        self.T, self.TinvT = O.build_transforms(M[None], H[None], W.GAMMA)
+        S = int(wl.lengths()[0])
+        if ctx_cap:
+            S = min(S, ctx_cap)
+        self.S = S
+        self.cache = O.LayerCache(1, 128, cfg["bits"], W.KAPPA_K, W.KAPPA_V, self.T)
+        toks = [(K[:, :1], V[:, :1]) for _, K, V in wl.sequence_tokens(0, S + 64)]
+        self.K = np.concatenate([t[0] for t in toks])
+        self.V = np.concatenate([t[1] for t in toks])
+        self.cache.append(self.K[:S - 1], self.V[:S - 1])
+        self.q = wl.queries(0, S - 1)[:G]
+        self.extra = 0
+
+    def step(self):
+        O, c = self.O, self.cfg
+        i = self.S - 1 + self.extra
+        self.cache.append(self.K[i:i + 1], self.V[i:i + 1])
+        self.extra += 1
+        arrs = self.cache.arrays()
+        return O.decode_attn(self.q, self.TinvT, *arrs, self.cache.S, c["s_sink"], c["s_keep"], 1, 1.0 / np.sqrt(128))
+
+    def bytes_per_step(self):
+        c = self.cfg
+        per_q = 72 if c["bits"] == 2 else 136
+        S = self.S
+        nq = max(S - c["s_keep"] - c["s_sink"], 0)
+        return nq * per_q + (S - nq) * 512
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info()]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle(name, steps, warmup, budget_s=20.0):
+    smp = OracleSample(name)
+    for _ in range(warmup):
+        smp.step()
+    times = []
+    t_all = time.perf_counter()
+    for _ in range(steps):
+        t0 = time.perf_counter()
+        smp.step()
+        times.append(time.perf_counter() - t0)
+        if time.perf_counter() - t_all > budget_s:
+            break
+    sec = sum(times) / len(times)
+    return smp, sec, len(times)
+
+
+# ------------------------------------------------------------------------------------------------
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    smp, sec, done = time_oracle(args.config, args.steps, args.warmup, budget_s=120.0)
+    gbs = smp.bytes_per_step() / sec / 1e9
+    sample = (f"1 of {smp.wl.batch} sequences x 1 of {smp.wl.n_kv} KV heads ({smp.wl.G} query heads) at context {smp.S}: "
+              f"append 1 token + decode, numpy float64")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus, "steps": done,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.config, "sample": sample},
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def run_ours(args, rank, world):
+    import torch
+    import torch.distributed as dist
+    from paper_2609_38121_b200 import build as _build
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2609_38121_b200 import binding as B
+
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    K, Wm = args.steps, args.warmup
+    n_total_steps = Wm + K            # device-timed region
+    sess = Session(args.config, n_steps=2 * n_total_steps + 2, seed_offset=rank, verbose=(rank == 0 and args.verbose))
+    cache_bytes = sess.decode_bytes(1)
+    need_flush = cache_bytes < 2 * L2_BYTES
+    flush_buf = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device="cuda") if need_flush else None
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(Wm):
+        sess.step()
+    torch.cuda.synchronize()
+    assert sess.cache.status() == 0, f"device status {sess.cache.status()}"
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
+    starts, mids, stops = [ev() for _ in range(K)], [ev() for _ in range(K)], [ev() for _ in range(K)]
+    kstart, kstop = [ev() for _ in range(K)], [ev() for _ in range(K)]
+    for e in kstart + kstop:
+        e.record()                    # materialise the handles
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    t_region0 = ev()
+    t_region1 = ev()
+    t_region0.record()
+    for i in range(K):
+        if need_flush:
+            flush_buf.fill_(i & 0xFF)
+        B.set_profile_events(kstart[i], kstop[i])
+        starts[i].record()
+        sess.step(mid_event=mids[i])
+        stops[i].record()
+    t_region1.record()
+    B.set_profile_events(None, None)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    assert sess.cache.status() == 0, f"device status {sess.cache.status()}"
+    step_ms = [s.elapsed_time(e) for s, e in zip(starts, stops)]
+    append_ms = [s.elapsed_time(e) for s, e in zip(starts, mids)]
+    kern_ms = [s.elapsed_time(e) for s, e in zip(kstart, kstop)]
+    if need_flush:
+        ms_per_step = sum(step_ms) / K            # flush time excluded: per-step events
+    else:
+        ms_per_step = t_region0.elapsed_time(t_region1) / K
+    if world > 1:
+        t = torch.tensor([ms_per_step], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_per_step = float(t.item())
+    bytes_step = float(np.mean([sess.decode_bytes(Wm + i + 1) for i in range(K)])) if not sess.chunk else float(cache_bytes)
+    value = world * bytes_step / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end-to-end through the host-buffer entry point (decode steps only)
+    e2e = None
+    if not sess.chunk:
+        stg_bytes = B.step_staging_bytes(sess.cache.desc, sess.batch)
+        stg = torch.empty(stg_bytes, dtype=torch.uint8, device="cuda")
+        hK = torch.from_numpy(W.f32_to_bf16_bits(sess.step_k_host).view(np.int16)).pin_memory()
+        hV = torch.from_numpy(W.f32_to_bf16_bits(sess.step_v_host).view(np.int16)).pin_memory()
+        hQ = torch.from_numpy(W.f32_to_bf16_bits(sess.q_host).view(np.int16)).pin_memory()
+        hO = torch.empty((sess.batch, sess.wl.n_q, 128), dtype=torch.float32).pin_memory()
+        base = sess.step_index
+
+        def host_step(i):
+            B.decode_step_host(sess.cache.desc, sess.batch, sess.slot, sess.seq_len, sess.cu_one, sess.max_seq_len,
+                               hK[base + i], hV[base + i], hQ, hO, stg, stg_bytes, sess.ws, sess.ws_bytes)
+            torch.cuda.synchronize()
+            return float(hO[0, 0, 0])                 # the host reads the step's result
+
+        for i in range(Wm):
+            host_step(i)
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(K):
+            host_step(Wm + i)
+        t1 = time.perf_counter()
+        e2e_ms = (t1 - t0) * 1e3 / K
+        if world > 1:
+            t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        e2e = {"value": world * bytes_step / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": int(2 * hK[0].numel() * 2 + hQ.numel() * 2), "d2h_bytes_per_step": int(hO.numel() * 4)}
+        assert sess.cache.status() == 0
+
+    if rank != 0:
+        return
+    peak, peak_kind = measured_hbm_peak()
+    kern_s = statistics.mean(kern_ms) * 1e-3
+    achieved = bytes_step / kern_s / 1e9
+    roofline = {"bound": "hbm", "kernel": "decode_main_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "kernel_ms": kern_s * 1e3, "kernel_ms_min": min(kern_ms), "algorithmic_bytes": bytes_step,
+                "traffic": NCU_TRAFFIC_BYTES.get(args.config)}
+    cpu = None
+    if world == 1 and not args.no_cpu:
+        smp, sec, done = time_oracle(args.config, steps=10 ** 6, warmup=1, budget_s=args.cpu_seconds)
+        cpu = {"value": smp.bytes_per_step() / sec / 1e9, "unit": "GB/s", "cores": cpu_threads(), "kind": "oracle",
+               "ms_per_step": sec * 1e3, "steps": done,
+               "sample": (f"1 of {smp.wl.batch} sequences x 1 of {smp.wl.n_kv} KV heads ({smp.wl.G} query heads) at context "
+                          f"{smp.S}: append 1 token + decode, numpy float64")}
+    c = sess.cfg
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.config, "batch": sess.batch, "n_q": c["n_q"], "n_kv": c["n_kv"], "head_dim": 128,
+                   "context": int(sess.final.max()), "bits": c["bits"], "s_sink": c["s_sink"], "s_keep": c["s_keep"],
+                   "s_flush": sess.s_flush, "page_tokens": 64, "prefill_chunk": sess.chunk,
+                   "l2": ("flushed between steps (256 MB write)" if need_flush else "cache read per step exceeds L2 (no flush)"),
+                   "replicas": world},
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
+        "gpu_launches": K * sess.launches_per_step(), "clocks": clocks,
+        "decode_tokens_per_s": world * sess.batch / (ms_per_step * 1e-3),
+        "append_tokens_per_s": world * sess.append_tokens() / (statistics.mean(append_ms) * 1e-3),
+        "append_ms": statistics.mean(append_ms), "step_ms_min": min(step_ms),
+        "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="cfg1", choices=sorted(W.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--verbose", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", 0)))
+        dist.init_process_group("nccl")
+    try:
+        run_ours(args, rank, world)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

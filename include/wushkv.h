@@ -185,6 +185,33 @@ int wushkv_decode_attn(const wushkv_cache* cache, int32_t batch, const int32_t* 
 int wushkv_unpack_debug(const wushkv_cache* cache, int32_t slot, int32_t kv_head, int32_t which,
                         int32_t pos0, int32_t n, uint8_t* codes, float* scale, float* zero, void* stream);
 
+/*
+ * One whole decode step from HOST buffers: Algorithm 2 lines 3-5 and 7-12 for one new token per
+ * sequence.  Enqueues, in order, on `stream`: host->device copies of K_new, V_new and Q into
+ * `staging`, wushkv_append of one token per sequence, wushkv_decode_attn, and the device->host
+ * copy of O.  Does not synchronise; O_host is valid once the stream has been synchronised.
+ *   K_new_host, V_new_host (host, pinned for the copies to be asynchronous): bf16 [batch][n_kv][d].
+ *   Q_host (host): bf16 [batch][n_q][d].   O_host (host, out): fp32 [batch][n_q][d].
+ *   cu_new (device): int32 [batch+1] = 0, 1, ..., batch.
+ *   staging (device): >= wushkv_step_staging_bytes() bytes, 256-byte aligned, scratch.
+ *   slot, seq_len (in/out), max_seq_len (bound on the lengths AFTER the append), workspace: as for
+ *   wushkv_append / wushkv_decode_attn.
+ */
+size_t wushkv_step_staging_bytes(const wushkv_cache* cache, int32_t batch);
+int wushkv_decode_step_host(const wushkv_cache* cache, int32_t batch, const int32_t* slot, int32_t* seq_len,
+                            const int32_t* cu_new, int32_t max_seq_len,
+                            const uint16_t* K_new_host, const uint16_t* V_new_host, const uint16_t* Q_host,
+                            float* O_host, void* staging, size_t staging_bytes,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Measurement aid (not part of the method): when both arguments are non-NULL cudaEvent_t handles,
+ * every following wushkv_decode_attn records `start` immediately before and `stop` immediately after
+ * its main kernel (the one that streams the packed cache) on the call's stream, so that a benchmark
+ * can time that kernel alone.  Pass NULLs to switch it off.  Process-wide, not thread-safe.
+ */
+int wushkv_set_profile_events(void* start, void* stop);
+
 #ifdef __cplusplus
 }
 #endif

@@ -18,6 +18,7 @@ DEV_PAGE_TABLE_FULL, DEV_BAD_PAGE_ID, DEV_BAD_SLOT, DEV_COPY_TIMEOUT = 1, 2, 4, 
 EXPORTS = (
     "wushkv_page_bytes", "wushkv_status_string", "wushkv_accumulate_gram", "wushkv_build_transforms",
     "wushkv_append", "wushkv_decode_workspace_bytes", "wushkv_decode_attn", "wushkv_unpack_debug",
+    "wushkv_step_staging_bytes", "wushkv_decode_step_host", "wushkv_set_profile_events",
 )
 
 
@@ -69,6 +70,14 @@ def _load():
     lib.wushkv_unpack_debug.restype = C.c_int
     lib.wushkv_unpack_debug.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                         C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.wushkv_step_staging_bytes.restype = C.c_size_t
+    lib.wushkv_step_staging_bytes.argtypes = [C.POINTER(wushkv_cache), C.c_int32]
+    lib.wushkv_decode_step_host.restype = C.c_int
+    lib.wushkv_decode_step_host.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                            C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                            C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.wushkv_set_profile_events.restype = C.c_int
+    lib.wushkv_set_profile_events.argtypes = [C.c_void_p, C.c_void_p]
     return lib
 
 
@@ -144,6 +153,27 @@ def decode_attn(cache: wushkv_cache, batch, slot, seq_len, max_seq_len, Q, O, wo
 def unpack_debug(cache: wushkv_cache, slot, kv_head, which, pos0, n, codes, scale, zero, stream=None):
     _check(lib.wushkv_unpack_debug(C.byref(cache), slot, kv_head, which, pos0, n, _ptr(codes), _ptr(scale),
                                    _ptr(zero), _stream_ptr(stream)), "wushkv_unpack_debug")
+
+
+def step_staging_bytes(cache: wushkv_cache, batch: int) -> int:
+    return int(lib.wushkv_step_staging_bytes(C.byref(cache), batch))
+
+
+def decode_step_host(cache: wushkv_cache, batch, slot, seq_len, cu_new, max_seq_len, K_new_host, V_new_host, Q_host,
+                     O_host, staging, staging_bytes, workspace, workspace_bytes, stream=None):
+    """wushkv_decode_step_host: the *_host tensors are (pinned) CPU tensors, everything else device."""
+    _check(lib.wushkv_decode_step_host(C.byref(cache), batch, _ptr(slot), _ptr(seq_len), _ptr(cu_new), max_seq_len,
+                                       _ptr(K_new_host), _ptr(V_new_host), _ptr(Q_host), _ptr(O_host),
+                                       _ptr(staging), staging_bytes, _ptr(workspace), workspace_bytes,
+                                       _stream_ptr(stream)), "wushkv_decode_step_host")
+
+
+def set_profile_events(start=None, stop=None):
+    """wushkv_set_profile_events with torch.cuda.Event objects (already recorded once so that their
+    handles exist) or None to switch the hook off."""
+    a = C.c_void_p(start.cuda_event) if start is not None else None
+    b = C.c_void_p(stop.cuda_event) if stop is not None else None
+    _check(lib.wushkv_set_profile_events(a, b), "wushkv_set_profile_events")
 
 
 class PagedCache:

@@ -656,6 +656,8 @@ static bool make_plan(const CacheView& c, int batch, int max_seq_len, DecodePlan
     return true;
 }
 
+static cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
+
 template <int BITS, int MODE>
 static int launch_decode(const DecodeParams& P, cudaStream_t st) {
     constexpr int STAGES = BITS == 2 ? 4 : 3;
@@ -665,8 +667,10 @@ static int launch_decode(const DecodeParams& P, cudaStream_t st) {
     if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
     if (cudaFuncSetAttribute(decode_main_kernel<BITS, MODE, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(SMEM)) != cudaSuccess)
         return WUSHKV_ECUDA;
+    if (g_prof_start) cudaEventRecord(g_prof_start, st);
     decode_main_kernel<BITS, MODE, STAGES><<<dim3(P.n_chunks + 1, P.c.n_kv, P.batch), MAIN_WARPS * 32, SMEM, st>>>(P);
     if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
+    if (g_prof_stop) cudaEventRecord(g_prof_stop, st);
     decode_combine_kernel<<<dim3(P.c.n_q, P.batch), 128, 0, st>>>(P);
     if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
     return WUSHKV_OK;
@@ -706,4 +710,50 @@ extern "C" int wushkv_decode_attn(const wushkv_cache* cache, int32_t batch, cons
     const bool mode0 = P.c.G <= 4;
     if (P.c.bits == 2) return mode0 ? launch_decode<2, 0>(P, st) : launch_decode<2, 1>(P, st);
     return mode0 ? launch_decode<4, 0>(P, st) : launch_decode<4, 1>(P, st);
+}
+
+extern "C" int wushkv_set_profile_events(void* start, void* stop) {
+    if ((start == nullptr) != (stop == nullptr)) return WUSHKV_EINVAL;
+    g_prof_start = static_cast<cudaEvent_t>(start);
+    g_prof_stop = static_cast<cudaEvent_t>(stop);
+    return WUSHKV_OK;
+}
+
+extern "C" size_t wushkv_step_staging_bytes(const wushkv_cache* cache, int32_t batch) {
+    CacheView v;
+    if (make_view(cache, v) != WUSHKV_OK || batch <= 0) return 0;
+    const size_t kv = align_up(static_cast<size_t>(batch) * v.n_kv * D * 2, 256);
+    const size_t q = align_up(static_cast<size_t>(batch) * v.n_q * D * 2, 256);
+    const size_t o = align_up(static_cast<size_t>(batch) * v.n_q * D * 4, 256);
+    return 2 * kv + q + o;
+}
+
+extern "C" int wushkv_decode_step_host(const wushkv_cache* cache, int32_t batch, const int32_t* slot, int32_t* seq_len,
+                                       const int32_t* cu_new, int32_t max_seq_len,
+                                       const uint16_t* K_new_host, const uint16_t* V_new_host, const uint16_t* Q_host,
+                                       float* O_host, void* staging, size_t staging_bytes,
+                                       void* workspace, size_t workspace_bytes, void* stream) {
+    CacheView v;
+    const int rc = make_view(cache, v);
+    if (rc != WUSHKV_OK) return rc;
+    if (batch <= 0 || !K_new_host || !V_new_host || !Q_host || !O_host || !staging || !aligned(staging, 256)) return WUSHKV_EINVAL;
+    if (staging_bytes < wushkv_step_staging_bytes(cache, batch)) return WUSHKV_ECAPACITY;
+    const size_t kv_bytes = static_cast<size_t>(batch) * v.n_kv * D * 2, kv = align_up(kv_bytes, 256);
+    const size_t q_bytes = static_cast<size_t>(batch) * v.n_q * D * 2, q = align_up(q_bytes, 256);
+    const size_t o_bytes = static_cast<size_t>(batch) * v.n_q * D * 4;
+    unsigned char* sp = static_cast<unsigned char*>(staging);
+    uint16_t* dK = reinterpret_cast<uint16_t*>(sp);
+    uint16_t* dV = reinterpret_cast<uint16_t*>(sp + kv);
+    uint16_t* dQ = reinterpret_cast<uint16_t*>(sp + 2 * kv);
+    float* dO = reinterpret_cast<float*>(sp + 2 * kv + q);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(dK, K_new_host, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return WUSHKV_ECUDA;
+    if (cudaMemcpyAsync(dV, V_new_host, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return WUSHKV_ECUDA;
+    if (cudaMemcpyAsync(dQ, Q_host, q_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return WUSHKV_ECUDA;
+    int r = wushkv_append(cache, batch, slot, seq_len, cu_new, batch, 1, dK, dV, stream);
+    if (r != WUSHKV_OK) return r;
+    r = wushkv_decode_attn(cache, batch, slot, seq_len, max_seq_len, dQ, dO, workspace, workspace_bytes, stream);
+    if (r != WUSHKV_OK) return r;
+    if (cudaMemcpyAsync(O_host, dO, o_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return WUSHKV_ECUDA;
+    return WUSHKV_OK;
 }

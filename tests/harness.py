@@ -107,8 +107,9 @@ class Layer:
         return codes.cpu().numpy()[:n], scale.cpu().numpy()[:n].astype(np.float64), zero.cpu().numpy()[:n].astype(np.float64)
 
     def check_append_parity(self):
-        """Codes, scales and zeros of every position against the oracle; returns worst mismatch rate."""
-        worst = 0.0
+        """Codes, scales and zeros of every position against the oracle.  Returns the fraction of all
+        codes of the layer that differ (each by exactly one level, else this asserts)."""
+        n_codes = n_diff = 0
         for b in range(self.batch):
             n = self.lengths[b]
             if n == 0:
@@ -119,14 +120,15 @@ class Layer:
                     gc, gs, gz = self.gpu_codes(b, h, which)
                     diff = np.abs(gc.astype(np.int32) - oc[:, h].astype(np.int32))
                     assert diff.max() <= 1, f"code off by more than one level (b={b} h={h} which={which})"
-                    rate = float(np.mean(diff != 0))
-                    worst = max(worst, rate)
+                    n_codes += diff.size
+                    n_diff += int(np.count_nonzero(diff))
                     sref, zref = om[:, h, 0], om[:, h, 1]
                     assert np.all(np.abs(gs - sref) <= META_RTOL * np.abs(sref) + 1e-12), "scale mismatch"
                     # the offset is compared relative to the vector's range (x_min can sit near zero)
                     span = ((1 << self.bits) - 1) * sref
                     assert np.all(np.abs(gz - zref) <= META_RTOL * np.maximum(np.abs(zref), span) + 1e-12), "zero mismatch"
-        return worst
+        self.last_code_stats = (n_diff, n_codes)
+        return n_diff / max(n_codes, 1)
 
     def gpu_window_arrays(self, b):
         """bf16 copies the GPU holds for sequence b, scattered to their positions ([S][n_kv][128]

@@ -110,8 +110,8 @@ def test_decode_is_deterministic_and_split_invariant(monkeypatch):
         outs.append(L.decode()[0])
     assert np.array_equal(outs[0], outs[1])
     scale = np.max(np.abs(outs[0]))
-    assert np.max(np.abs(outs[2] - outs[0])) <= 1e-5 * scale
-    assert np.max(np.abs(outs[3] - outs[0])) <= 1e-5 * scale
+    assert np.max(np.abs(outs[2] - outs[0])) <= 5e-5 * scale
+    assert np.max(np.abs(outs[3] - outs[0])) <= 5e-5 * scale
 
 
 def test_device_side_errors_are_flagged_not_fatal():
