@@ -205,6 +205,29 @@ int wushkv_decode_step_host(const wushkv_cache* cache, int32_t batch, const int3
                             void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * wushkv_decode_attn without a caller-provided workspace (the paper has no counterpart: this is
+ * an interface convenience).  It is meant for callers that cannot allocate device memory - for
+ * example because their framework took all of it for its own pool at start-up, because they are a
+ * plug-in that only ever receives input and output buffers, or because an allocation's implicit
+ * synchronisation has no place in their latency-critical loop.  The scratch is a fixed array of
+ * WUSHKV_STATIC_SCRATCH_BYTES inside the library's device image; each GPU that loads the library
+ * holds that much memory until the process exits.
+ *   - Arguments and results are exactly those of wushkv_decode_attn, minus workspace.
+ *   - A request whose wushkv_decode_workspace_bytes() exceeds WUSHKV_STATIC_SCRATCH_BYTES is
+ *     refused with WUSHKV_ECAPACITY and nothing is launched; use wushkv_decode_attn then.
+ *   - The call allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress,
+ *     with that device current); make that first call before starting any stream capture.
+ *   - All calls on a GPU share the one array, and it keeps whatever the last call left in it.
+ *     Nothing in it needs to be zero at entry (each call writes every value it later reads), but
+ *     two calls that overlap on the GPU - different streams, or different threads - race on it.
+ *     Serialise them (same stream, or an event between them).
+ */
+#define WUSHKV_STATIC_SCRATCH_BYTES (8u << 20)
+int wushkv_decode_attn_static(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
+                              int32_t max_seq_len, const uint16_t* Q, float* O, void* stream);
+
+/*
  * Measurement aid (not part of the method): when both arguments are non-NULL cudaEvent_t handles,
  * every following wushkv_decode_attn records `start` immediately before and `stop` immediately after
  * its main kernel (the one that streams the packed cache) on the call's stream, so that a benchmark

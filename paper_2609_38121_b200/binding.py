@@ -19,7 +19,9 @@ EXPORTS = (
     "wushkv_page_bytes", "wushkv_status_string", "wushkv_accumulate_gram", "wushkv_build_transforms",
     "wushkv_append", "wushkv_decode_workspace_bytes", "wushkv_decode_attn", "wushkv_unpack_debug",
     "wushkv_step_staging_bytes", "wushkv_decode_step_host", "wushkv_set_profile_events",
+    "wushkv_decode_attn_static",
 )
+STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class WushkvError(RuntimeError):
@@ -76,6 +78,9 @@ def _load():
     lib.wushkv_decode_step_host.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
                                             C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                             C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.wushkv_decode_attn_static.restype = C.c_int
+    lib.wushkv_decode_attn_static.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_void_p, C.c_void_p, C.c_int32,
+                                              C.c_void_p, C.c_void_p, C.c_void_p]
     lib.wushkv_set_profile_events.restype = C.c_int
     lib.wushkv_set_profile_events.argtypes = [C.c_void_p, C.c_void_p]
     return lib
@@ -153,6 +158,14 @@ def decode_attn(cache: wushkv_cache, batch, slot, seq_len, max_seq_len, Q, O, wo
 def unpack_debug(cache: wushkv_cache, slot, kv_head, which, pos0, n, codes, scale, zero, stream=None):
     _check(lib.wushkv_unpack_debug(C.byref(cache), slot, kv_head, which, pos0, n, _ptr(codes), _ptr(scale),
                                    _ptr(zero), _stream_ptr(stream)), "wushkv_unpack_debug")
+
+
+def decode_attn_static(cache: wushkv_cache, batch, slot, seq_len, max_seq_len, Q, O, stream=None):
+    """wushkv_decode_attn_static: decode attention for callers that cannot allocate device memory
+    (the workspace is a fixed array inside the library; requests needing more than
+    STATIC_SCRATCH_BYTES raise with status ECAPACITY; overlapping calls on one GPU race)."""
+    _check(lib.wushkv_decode_attn_static(C.byref(cache), batch, _ptr(slot), _ptr(seq_len), max_seq_len, _ptr(Q),
+                                         _ptr(O), _stream_ptr(stream)), "wushkv_decode_attn_static")
 
 
 def step_staging_bytes(cache: wushkv_cache, batch: int) -> int:

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libwushkv.so")
-SOURCES = ["api.cu", "transforms_host.cpp", "append.cu", "decode.cu"]
+SOURCES = ["api.cu", "transforms_host.cpp", "append.cu", "decode.cu", "decode_static.cu"]
 
 
 def _nvcc() -> str:
@@ -32,7 +32,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     srcs = [os.path.join(CSRC, s) for s in SOURCES if os.path.exists(os.path.join(CSRC, s))]
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "--use_fast_math" if False else "-DWUSHKV_BUILD", "-Xcompiler", "-fPIC,-O3", "-shared",
+           "-DWUSHKV_BUILD", "-Xcompiler", "-fPIC,-O3", "-shared",
            "-cudart", "shared", "-o", LIB] + srcs
     if verbose:
         cmd.insert(1, "-Xptxas")
