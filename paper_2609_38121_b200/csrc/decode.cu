@@ -1,23 +1,28 @@
 // Decode attention over the packed cache (Algorithm 2 lines 3 and 5; Eq. 2; Eq. 3; Section 4.4).
 //
 // Three launches on the caller's stream:
-//   1. decode_prep_kernel   q' = T_K^{-T} q per query head (Algorithm 2 line 3), written (a) as fp32
-//                           for the bf16 windows and (b) as fp16 mma B-fragments, pre-scaled by the
-//                           power of two that each packed code field carries.
-//   2. decode_main_kernel   one CTA per (sequence, KV head, split of the quantized range) plus one
-//                           CTA per (sequence, KV head) for the bf16 sink / recent windows.  Each warp
-//                           streams whole 64-token page records into shared memory with bulk async
-//                           copies (mbarrier ring), turns code words into fp16 A-fragments with one
-//                           AND per register, and runs both contractions (q'.k and p.v) on
-//                           mma.sync.m16n8k16 with fp32 accumulation.  The affine part of Eq. 6 is
-//                           factored out of the contractions:
+//   1. decode_prep_kernel   q' = T_K^{-T} q per query head (Algorithm 2 line 3), written as mma
+//                           B-fragments: fp16 (value + rounding remainder), pre-scaled by the power of
+//                           two that each packed code field carries, for the quantized positions, and
+//                           bf16 (value + remainder) for the bf16 windows.  Block (0,0) also writes the
+//                           work plan: the prefix sums of work units per sequence.
+//   2. decode_main_kernel   ONE wave of CTAs; every WARP owns an equal, contiguous slice of the
+//                           flattened list of work units (sequence, KV head, unit), a unit being a
+//                           64-token packed page or up to 8 tokens of the bf16 sink / recent windows.
+//                           A warp streams its units into shared memory with bulk async copies (mbarrier
+//                           ring), turns code words into fp16 A-fragments with one AND per register, and
+//                           runs both contractions (q'.k and p.v) on mma.sync.m16n8k16 with fp32
+//                           accumulation.  The affine part of Eq. 6 is factored out of the contractions:
 //                               q'.k_hat = Delta_k (q'.c_k) + x_min_k sum(q'),
 //                               o        = sum_s (p_s Delta_v,s) c_v,s + (sum_s p_s x_min_v,s) 1.
-//                           Softmax is online (running max / sum) per warp, merged per CTA.
-//   3. decode_combine_kernel merges the per-split (max, sum, o) partials into O.
+//                           Window units use ldmatrix + bf16 mma on the staged rows and fold into the
+//                           same accumulators.  Softmax is online (running max / sum) per warp; a warp
+//                           writes one partial (max, sum, o) per (sequence, KV head) it touched.
+//   3. decode_combine_kernel merges the partials of each (sequence, query head) into O.
 //
-// No kernel waits on another CTA.  The only waits are on this warp's own copy barriers, bounded by
-// an iteration limit after which the kernel records WUSHKV_DEV_COPY_TIMEOUT and drains.
+// No kernel waits on another CTA or warp.  The only waits are on a warp's own copy barriers, bounded
+// by an iteration limit after which the kernel records WUSHKV_DEV_COPY_TIMEOUT and drains.
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
@@ -32,9 +37,12 @@ namespace wushkv {
 constexpr unsigned FULL = 0xffffffffu;
 constexpr int PART_STRIDE = 132;          // floats per partial: [0]=max (log2 domain) [1]=sum [4..131]=o
 constexpr float LOG2E = 1.4426950408889634f;
-constexpr float LO_SCALE = 2048.f;        // the "lo" fp16 column carries (x - fp16(x)) * 2^11
+constexpr float LO_SCALE = 2048.f;        // a "remainder" column carries (x - rounded(x)) * 2^11
 constexpr float PV_SCALE = 16.f;          // p * Delta_v is fed to the tensor core as fp16(p Delta_v 2^4)
 constexpr int MAIN_WARPS = 4;
+constexpr int WIN_TOKENS = 8;             // window tokens per work unit
+constexpr int WIN_ROW = 272;              // padded bytes per staged bf16 row (conflict-free ldmatrix)
+constexpr int WIN_V_OFF = WIN_TOKENS * WIN_ROW;
 
 struct DecodeParams {
     CacheView c;
@@ -43,12 +51,12 @@ struct DecodeParams {
     const int* seq_len;
     const unsigned short* Q;
     float* O;
-    uint4* qfrag;      // [batch][n_kv][4][32] uint4: B fragments of the 8 k-steps
-    float* qscal;      // [batch][n_q][2]: (score multiplier, x_min multiplier) in the log2 domain
-    float* qcomp;      // [batch][n_q][128]: q' * sm_scale * log2(e), fp32, for the bf16 windows
-    float* part;       // [batch][n_q][n_chunks + 1][PART_STRIDE]
-    int n_chunks;      // splits of the quantized range; split index n_chunks is the window split
-    int chunk_pages;
+    uint4* qfrag;        // [batch*n_kv][128]: fp16 B fragments of the 8 k-steps (quantized positions)
+    uint4* qwfrag;       // [batch*n_kv][2][128]: bf16 B fragments for the windows (MODE 1: value set, remainder set)
+    float* qscal;        // [batch][n_q][2]: (score multiplier, x_min multiplier) in the log2 domain
+    long long* plan;     // [batch+1]: exclusive prefix of work units per sequence (per KV head)
+    float* part;         // [n_warps + batch*n_kv][G][PART_STRIDE]
+    int n_warps;         // warps of the main kernel
 };
 
 // shift of the code field used by k-step / channel block idx (0..7) inside its 16-bit lane, after
@@ -56,6 +64,38 @@ struct DecodeParams {
 template <int BITS>
 __host__ __device__ constexpr int field_shift(int idx) {
     return BITS == 2 ? (idx < 5 ? 2 * idx : 2 * (idx - 5)) : 4 * (idx & 1);
+}
+// bf16x2 bit pattern of (2^e, 2^e)
+__host__ __device__ constexpr unsigned bf16x2_pow2(int e) {
+    return (static_cast<unsigned>(e + 127) << 7) | (static_cast<unsigned>(e + 127) << 23);
+}
+
+// How one sequence decomposes into work units (identical for all of its KV heads).
+struct SeqInfo {
+    int slot;
+    int q_lo, q_hi;          // positions read from the packed codes: [q_lo, q_hi)
+    int first_page, qp;      // packed pages covering them
+    int n_sink, recent_lo;   // window tokens: positions [0, n_sink) and [recent_lo, S)
+    int n_win;               // window tokens
+    int U;                   // qp + ceil(n_win / WIN_TOKENS)
+};
+
+__device__ __forceinline__ SeqInfo seq_info(const CacheView& c, int S, int slot) {
+    SeqInfo si;
+    si.slot = slot;
+    if (S <= 0 || slot < 0 || slot >= c.n_slots) {
+        si.q_lo = si.q_hi = 0; si.first_page = si.qp = 0; si.n_sink = si.recent_lo = si.n_win = si.U = 0;
+        return si;
+    }
+    const int nq = n_quantized(S - c.lag, c.s_sink, c.s_keep, c.s_flush);
+    si.q_lo = c.s_sink; si.q_hi = c.s_sink + nq;
+    si.first_page = si.q_lo / PAGE_TOKENS;
+    si.qp = nq > 0 ? (si.q_hi - 1) / PAGE_TOKENS - si.first_page + 1 : 0;
+    si.n_sink = min(S, c.s_sink);
+    si.recent_lo = c.s_sink + nq;
+    si.n_win = si.n_sink + max(0, S - si.recent_lo);
+    si.U = si.qp + (si.n_win + WIN_TOKENS - 1) / WIN_TOKENS;
+    return si;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -66,8 +106,36 @@ __global__ void __launch_bounds__(128) decode_prep_kernel(DecodeParams P) {
     __shared__ float q_s[8][D];
     __shared__ float red_max[8][4];
     __shared__ float red_sum[8][4];
+    __shared__ long long scan_s[4];
     const int h = blockIdx.x, b = blockIdx.y, G = P.c.G;
     const int i = threadIdx.x, lane = i & 31, warp = i >> 5;
+
+    if (h == 0 && b == 0) {               // work plan: exclusive prefix of units per sequence
+        long long carry = 0;
+        for (int base = 0; base < P.batch; base += 128) {
+            const int bb = base + i;
+            long long u = 0;
+            if (bb < P.batch) {
+                const int slot = __ldg(P.slot + bb);
+                if (slot < 0 || slot >= P.c.n_slots) atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_SLOT);
+                u = seq_info(P.c, __ldg(P.seq_len + bb), slot).U;
+            }
+            long long incl = u;
+            for (int o = 1; o < 32; o <<= 1) {
+                const long long v = __shfl_up_sync(FULL, incl, o);
+                if (lane >= o) incl += v;
+            }
+            if (lane == 31) scan_s[warp] = incl;
+            __syncthreads();
+            long long before = 0;
+            for (int w = 0; w < warp; ++w) before += scan_s[w];
+            if (bb < P.batch) P.plan[bb + 1] = carry + before + incl;
+            carry += scan_s[0] + scan_s[1] + scan_s[2] + scan_s[3];
+            __syncthreads();
+        }
+        if (i == 0) P.plan[0] = 0;
+    }
+
     for (int g = 0; g < G; ++g)
         q_s[g][i] = bf16_bits_to_float(P.Q[(static_cast<long long>(b) * P.c.n_q + h * G + g) * D + i]);
     __syncthreads();
@@ -75,6 +143,7 @@ __global__ void __launch_bounds__(128) decode_prep_kernel(DecodeParams P) {
 #pragma unroll
     for (int g = 0; g < 8; ++g) acc[g] = 0.f;
     const float4* Trow = reinterpret_cast<const float4*>(P.c.T_K_invT + (static_cast<long long>(h) * D + i) * D);
+#pragma unroll 8
     for (int j4 = 0; j4 < D / 4; ++j4) {
         const float4 t = __ldg(Trow + j4);
 #pragma unroll
@@ -92,7 +161,6 @@ __global__ void __launch_bounds__(128) decode_prep_kernel(DecodeParams P) {
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
         if (g < G) {
-            P.qcomp[(static_cast<long long>(b) * P.c.n_q + h * G + g) * D + i] = acc[g] * k2;
             float mx = fabsf(acc[g]) * pos_scale, sm = acc[g];
             for (int o = 16; o > 0; o >>= 1) {
                 mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
@@ -120,21 +188,31 @@ __global__ void __launch_bounds__(128) decode_prep_kernel(DecodeParams P) {
             }
         }
     }
-    // B fragments: column n of the mma holds, for MODE 0, head n>>1 as its fp16 value (n even) or the
-    // scaled rounding remainder (n odd); for MODE 1, head n.
+    // B fragments.  Element (k-step s, register r, lane 4n+t, half hf) is channel 16s + 8r + 2t + hf of
+    // mma column n.  MODE 0: column n holds head n>>1, its rounded value (n even) or the rounding
+    // remainder times 2^11 (n odd).  MODE 1: column n holds head n; the window set has a second copy
+    // with the remainders.
     const int r16 = i & 15, r = r16 >> 3, t = (r16 & 7) >> 1, hf = r16 & 1;
-    unsigned short* frag = reinterpret_cast<unsigned short*>(P.qfrag + (static_cast<long long>(b) * P.c.n_kv + h) * 128);
+    const long long bh = static_cast<long long>(b) * P.c.n_kv + h;
+    unsigned short* frag = reinterpret_cast<unsigned short*>(P.qfrag + bh * 128);
+    unsigned short* wfrag = reinterpret_cast<unsigned short*>(P.qwfrag + bh * 256);
 #pragma unroll
     for (int n = 0; n < 8; ++n) {
         const int head = (MODE == 0) ? (n >> 1) : n;
-        float val = 0.f;
+        float val = 0.f, wval = 0.f, wrem = 0.f;
         if (head < G) {
             const float x = acc[head] * pos_scale * beta[head];
             const __half hi = __float2half_rn(x);
             val = (MODE == 0 && (n & 1)) ? (x - __half2float(hi)) * LO_SCALE : x;
+            const float y = acc[head] * k2;
+            const float yh = __bfloat162float(__float2bfloat16_rn(y));
+            wrem = y - yh;
+            wval = (MODE == 0 && (n & 1)) ? wrem : y;
         }
-        const int lane_dst = 4 * n + t;
-        frag[((((s >> 1) * 32 + lane_dst) * 4 + (s & 1) * 2 + r) << 1) + hf] = __half_as_ushort(__float2half_rn(val));
+        const int idx = ((((s >> 1) * 32 + 4 * n + t) * 4 + (s & 1) * 2 + r) << 1) + hf;
+        frag[idx] = __half_as_ushort(__float2half_rn(val));
+        wfrag[idx] = __bfloat16_as_ushort(__float2bfloat16_rn(wval));
+        if (MODE == 1) wfrag[1024 + idx] = __bfloat16_as_ushort(__float2bfloat16_rn(wrem));
     }
 }
 
@@ -176,8 +254,19 @@ __device__ __forceinline__ uint4 lds128(unsigned addr) {
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
 }
-__device__ __forceinline__ void mma16816(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0, unsigned b1) {
+__device__ __forceinline__ void ldmatrix_x4(unsigned addr, unsigned& a, unsigned& b, unsigned& c, unsigned& d) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(unsigned addr, unsigned& a, unsigned& b, unsigned& c, unsigned& d) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "r"(addr));
+}
+__device__ __forceinline__ void mma_f16(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0, unsigned b1) {
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0, unsigned b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
@@ -191,8 +280,24 @@ __device__ __forceinline__ unsigned pack_h2(float lo, float hi) {      // lo -> 
     asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
     return d;
 }
+__device__ __forceinline__ unsigned pack_bf2(float lo, float hi) {
+    unsigned d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+__device__ __forceinline__ unsigned mul_bf2(unsigned a, unsigned b) {
+    unsigned d;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ float ex2(float x) {      // 2^x, -inf -> 0
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ float h_lo(unsigned u) { return __half2float(__ushort_as_half(static_cast<unsigned short>(u & 0xffffu))); }
 __device__ __forceinline__ float h_hi(unsigned u) { return __half2float(__ushort_as_half(static_cast<unsigned short>(u >> 16))); }
+__device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 
 // Field idx (0..7) of a code word as an fp16x2 A-fragment register.  `w` is the raw word, `ws` the
 // same word shifted right so that the upper fields fall into the low bits of each 16-bit lane.
@@ -208,18 +313,51 @@ __device__ __forceinline__ unsigned field(unsigned w, unsigned ws, int idx) {
 }
 template <int BITS> __device__ __forceinline__ unsigned pre_shift(unsigned w) { return BITS == 2 ? (w >> 10) : (w >> 8); }
 
-// Per-warp running softmax state.  MODE 0: one head per thread (head t, value and rounding remainder
-// in the two accumulator columns).  MODE 1: two heads per thread (2t, 2t+1).
+// Per-warp running softmax state of one (sequence, KV head).  MODE 0: one head per thread (head t,
+// value and rounding-remainder columns).  MODE 1: two heads per thread (2t, 2t+1).
+// o[i][.] accumulates channel block i in units of 2^(field_shift(i) - 24) / PV_SCALE.
 template <int MODE>
 struct WarpState {
     static constexpr int NH = MODE == 0 ? 1 : 2;
     float m[NH], l[NH], z[NH];
     float o[8][4];
+    __device__ __forceinline__ void reset() {
+#pragma unroll
+        for (int k = 0; k < NH; ++k) { m[k] = -INFINITY; l[k] = 0.f; z[k] = 0.f; }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    }
+    // Raise the running maximum to cover this unit's per-head maxima (already reduced over the unit's
+    // tokens); mref receives the reference each head's exponentials use.
+    __device__ __forceinline__ void raise_max(const float (&mx)[NH], float (&mref)[NH]) {
+        bool grew = false;
+        float mnew[NH];
+#pragma unroll
+        for (int k = 0; k < NH; ++k) {
+            mnew[k] = fmaxf(m[k], mx[k]);
+            grew |= mnew[k] > m[k];
+            mref[k] = (mnew[k] == -INFINITY) ? 0.f : mnew[k];       // all masked so far: any finite reference works
+        }
+        if (__any_sync(FULL, grew)) {
+            float scl[NH];
+#pragma unroll
+            for (int k = 0; k < NH; ++k) {
+                scl[k] = ex2(m[k] - mref[k]);                        // old max -inf: state is all zero, factor 0
+                l[k] *= scl[k]; z[k] *= scl[k];
+                m[k] = mnew[k];
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                o[i][0] *= scl[0]; o[i][2] *= scl[0];
+                o[i][1] *= scl[NH - 1]; o[i][3] *= scl[NH - 1];
+            }
+        }
+    }
 };
 
-// Writes this warp's partial (max, sum, o[128]) of every head into shared scratch [warp][head][PART_STRIDE].
+// Writes this warp's partial (max, sum, o[128]) of every head of one (sequence, KV head) to global memory.
 template <int BITS, int MODE>
-__device__ __forceinline__ void spill_warp_state(WarpState<MODE>& st, float* scratch_warp, int lane, int G) {
+__device__ __forceinline__ void store_partial(const WarpState<MODE>& st, float* dst0, int lane, int G) {
     const int g = lane >> 2, t = lane & 3;
     constexpr int NH = WarpState<MODE>::NH;
 #pragma unroll
@@ -230,7 +368,7 @@ __device__ __forceinline__ void spill_warp_state(WarpState<MODE>& st, float* scr
         l += __shfl_xor_sync(FULL, l, 16); z += __shfl_xor_sync(FULL, z, 16);
         const int head = MODE == 0 ? t : 2 * t + k;
         if (head < G) {
-            float* dst = scratch_warp + head * PART_STRIDE;
+            float* dst = dst0 + head * PART_STRIDE;
             if (g == 0) { dst[0] = st.m[k]; dst[1] = l; }
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
@@ -250,132 +388,59 @@ __device__ __forceinline__ void spill_warp_state(WarpState<MODE>& st, float* scr
     }
 }
 
-// Merge the per-warp partials in shared scratch and write this CTA's partial to global memory.
-__device__ __forceinline__ void merge_and_store(const float* scratch, int nwarps, int G, float* part_base,
-                                                long long head_stride, int tid, int nthreads) {
-    for (int idx = tid; idx < G * D; idx += nthreads) {
-        const int head = idx >> 7, ch = idx & 127;
-        float m = -INFINITY;
-        for (int w = 0; w < nwarps; ++w) m = fmaxf(m, scratch[(w * 8 + head) * PART_STRIDE]);
-        float l = 0.f, o = 0.f;
-        for (int w = 0; w < nwarps; ++w) {
-            const float* p = scratch + (w * 8 + head) * PART_STRIDE;
-            const float sc = (p[0] == -INFINITY) ? 0.f : exp2f(p[0] - m);
-            l += sc * p[1];
-            o += sc * p[4 + ch];
-        }
-        float* dst = part_base + head * head_stride;
-        if (ch == 0) { dst[0] = m; dst[1] = l; }
-        dst[4 + ch] = o;
-    }
-}
-
-// ------------------------------------------------------------------------------------------------
-// bf16 windows (sink + recent ring), CUDA cores, fp32
-// ------------------------------------------------------------------------------------------------
-__device__ void window_split(const DecodeParams& P, int b, int h, int slot, int S, int nq, float* scratch) {
-    const CacheView& c = P.c;
-    const int G = c.G;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    const int n_sink = min(S, c.s_sink);
-    const int recent_lo = c.s_sink + nq;
-    const int n_recent = max(0, S - recent_lo);
-    float q[8][4];
-#pragma unroll
-    for (int g = 0; g < 8; ++g) {
-        if (g < G) {
-            const float4 v = __ldg(reinterpret_cast<const float4*>(P.qcomp + (static_cast<long long>(b) * c.n_q + h * G + g) * D) + lane);
-            q[g][0] = v.x; q[g][1] = v.y; q[g][2] = v.z; q[g][3] = v.w;
-        } else {
-            q[g][0] = q[g][1] = q[g][2] = q[g][3] = 0.f;
-        }
-    }
-    float m[8], l[8], o[8][4];
-#pragma unroll
-    for (int g = 0; g < 8; ++g) { m[g] = -INFINITY; l[g] = 0.f; o[g][0] = o[g][1] = o[g][2] = o[g][3] = 0.f; }
-    const long long head_base = (static_cast<long long>(slot) * c.n_kv + h) * 2;
-    for (int w = warp; w < n_sink + n_recent; w += nwarps) {
-        const unsigned short *kp, *vp;
-        if (w < n_sink) {
-            kp = c.sink_kv + ((head_base + 0) * c.s_sink + w) * D;
-            vp = c.sink_kv + ((head_base + 1) * c.s_sink + w) * D;
-        } else {
-            const int row = (recent_lo + (w - n_sink)) % c.ring_cap;
-            kp = c.ring_kv + ((head_base + 0) * c.ring_cap + row) * D;
-            vp = c.ring_kv + ((head_base + 1) * c.ring_cap + row) * D;
-        }
-        const uint2 kr = __ldg(reinterpret_cast<const uint2*>(kp) + lane);
-        const uint2 vr = __ldg(reinterpret_cast<const uint2*>(vp) + lane);
-        const float k0 = bf16_bits_to_float(kr.x & 0xffff), k1 = bf16_bits_to_float(kr.x >> 16);
-        const float k2 = bf16_bits_to_float(kr.y & 0xffff), k3 = bf16_bits_to_float(kr.y >> 16);
-        const float v0 = bf16_bits_to_float(vr.x & 0xffff), v1 = bf16_bits_to_float(vr.x >> 16);
-        const float v2 = bf16_bits_to_float(vr.y & 0xffff), v3 = bf16_bits_to_float(vr.y >> 16);
-#pragma unroll
-        for (int g = 0; g < 8; ++g) {
-            if (g < G) {
-                float s = q[g][0] * k0 + q[g][1] * k1 + q[g][2] * k2 + q[g][3] * k3;
-                for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(FULL, s, off);
-                const float mn = fmaxf(m[g], s);
-                const float sc = exp2f(m[g] - mn);            // m = -inf on the first token: sc = 0
-                const float p = exp2f(s - mn);
-                l[g] = l[g] * sc + p;
-                o[g][0] = o[g][0] * sc + p * v0; o[g][1] = o[g][1] * sc + p * v1;
-                o[g][2] = o[g][2] * sc + p * v2; o[g][3] = o[g][3] * sc + p * v3;
-                m[g] = mn;
-            }
-        }
-    }
-    float* mine = scratch + warp * 8 * PART_STRIDE;
-#pragma unroll
-    for (int g = 0; g < 8; ++g) {
-        if (g < G) {
-            float* dst = mine + g * PART_STRIDE;
-            if (lane == 0) { dst[0] = m[g]; dst[1] = l[g]; }
-            *reinterpret_cast<float4*>(dst + 4 + 4 * lane) = make_float4(o[g][0], o[g][1], o[g][2], o[g][3]);
-        }
-    }
-}
+// Position of a warp in the flattened unit list.
+struct Cursor {
+    int b, h, u;
+    SeqInfo si;
+};
 
 // ------------------------------------------------------------------------------------------------
 // main kernel
 // ------------------------------------------------------------------------------------------------
 template <int BITS, int MODE, int STAGES>
-__global__ void __launch_bounds__(MAIN_WARPS * 32) decode_main_kernel(DecodeParams P) {
+__global__ void __launch_bounds__(MAIN_WARPS * 32, 4) decode_main_kernel(DecodeParams P) {
     constexpr int REC = record_bytes(BITS);
     constexpr int CB = code_block_bytes(BITS);
     constexpr int NH = WarpState<MODE>::NH;
+    static_assert(2 * WIN_TOKENS * WIN_ROW <= REC, "a window unit must fit in one stage");
     extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char* stage_base = smem;                                               // [MAIN_WARPS][STAGES][REC]
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + MAIN_WARPS * STAGES * REC);
-    float* scratch = reinterpret_cast<float*>(smem);                                // reused after the stream is drained
     const CacheView& c = P.c;
-    const int b = blockIdx.z, h = blockIdx.y, chunk = blockIdx.x;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int G = c.G;
-    const int slot = __ldg(P.slot + b);
-    const int S = __ldg(P.seq_len + b);
-    const int n_splits = P.n_chunks + 1;
-    float* part_base = P.part + ((static_cast<long long>(b) * c.n_q + h * G) * n_splits + chunk) * PART_STRIDE;
-    const long long head_stride = static_cast<long long>(n_splits) * PART_STRIDE;
-    if (slot < 0 || slot >= c.n_slots) {
-        if (tid == 0) atomicOr(c.dev_status, WUSHKV_DEV_BAD_SLOT);
-        return;
-    }
-    const int nq = (S > 0) ? n_quantized(S - c.lag, c.s_sink, c.s_keep, c.s_flush) : 0;
 
-    if (chunk == P.n_chunks) {          // ---- the bf16 windows
-        window_split(P, b, h, slot, max(S, 0), nq, scratch);
-        __syncthreads();
-        merge_and_store(scratch, MAIN_WARPS, G, part_base, head_stride, tid, blockDim.x);
-        return;
+    // ---- this warp's slice of the flattened unit list
+    const long long total = P.plan[P.batch] * c.n_kv;
+    if (total <= 0) return;
+    const long long wg = static_cast<long long>(blockIdx.x) * MAIN_WARPS + warp;
+    const long long L0 = wg * total / P.n_warps, L1 = (wg + 1) * total / P.n_warps;
+    if (L0 >= L1) return;
+    const int n_units = static_cast<int>(L1 - L0);
+
+    auto load_seq = [&](int b) { return seq_info(c, __ldg(P.seq_len + b), __ldg(P.slot + b)); };
+    auto advance = [&](Cursor& cur) {
+        if (++cur.u < cur.si.U) return;
+        cur.u = 0;
+        if (++cur.h < c.n_kv) return;
+        cur.h = 0;
+        do { ++cur.b; if (cur.b < P.batch) cur.si = load_seq(cur.b); } while (cur.b < P.batch && cur.si.U == 0);
+    };
+    Cursor cons;
+    {
+        int lo = 0, hi = P.batch;           // largest b with n_kv * plan[b] <= L0
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (P.plan[mid] * c.n_kv <= L0) lo = mid; else hi = mid;
+        }
+        cons.b = lo;
+        cons.si = load_seq(lo);
+        const long long rem = L0 - P.plan[lo] * c.n_kv;
+        const int U = max(cons.si.U, 1);
+        cons.h = static_cast<int>(rem / U);
+        cons.u = static_cast<int>(rem % U);
     }
-    if (nq <= 0) return;
-    const int q_lo = c.s_sink, q_hi = c.s_sink + nq;
-    const int first_page = q_lo / PAGE_TOKENS, last_page = (q_hi - 1) / PAGE_TOKENS;
-    const int pg0 = first_page + chunk * P.chunk_pages;
-    const int pg1 = min(pg0 + P.chunk_pages, last_page + 1);
-    if (pg0 >= pg1) return;
+    Cursor prod = cons;
 
     // ---- barriers
     const unsigned bar0 = smem_u32(bars + warp * STAGES);
@@ -385,177 +450,227 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32) decode_main_kernel(DecodePara
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
-    const unsigned stage0 = smem_u32(stage_base + warp * STAGES * REC);
-    const int* ptab = c.page_table + static_cast<long long>(slot) * c.max_pages;
+    const unsigned stage0 = smem_u32(smem + warp * STAGES * REC);
 
-    unsigned bad_stage = 0;             // lane 0: bit s set if the page staged in s could not be fetched
-    auto issue = [&](int pg, int s) {   // lane 0 only
-        const int page = (pg < c.max_pages) ? __ldg(ptab + pg) : -1;
-        if (page < 0 || page >= c.n_pages) {
-            atomicOr(c.dev_status, pg < c.max_pages ? WUSHKV_DEV_BAD_PAGE_ID : WUSHKV_DEV_PAGE_TABLE_FULL);
-            bad_stage |= 1u << s;
-            mbar_arrive(bar0 + 8 * s);
-        } else {
+    unsigned bad_stage = 0;             // bit s set if the unit staged in s could not be fetched
+    // Stage the unit under `cur` into stage s.  Executed by the whole warp.
+    auto issue = [&](const Cursor& cur, int s) {
+        const unsigned bar = bar0 + 8 * s, dst = stage0 + s * REC;
+        if (cur.u < cur.si.qp) {                        // a packed page: one bulk copy
+            const int pg = cur.si.first_page + cur.u;
+            int page = -1;
+            if (lane == 0) {
+                page = (pg < c.max_pages) ? __ldg(c.page_table + static_cast<long long>(cur.si.slot) * c.max_pages + pg) : -1;
+                if (page < 0 || page >= c.n_pages) {
+                    atomicOr(c.dev_status, pg < c.max_pages ? WUSHKV_DEV_BAD_PAGE_ID : WUSHKV_DEV_PAGE_TABLE_FULL);
+                    page = -1;
+                    mbar_arrive(bar);
+                } else {
+                    mbar_expect_tx(bar, REC);
+                    bulk_copy_g2s(dst, c.pages + (static_cast<long long>(page) * c.n_kv + cur.h) * REC, REC, bar);
+                }
+            }
+            page = __shfl_sync(FULL, page, 0);
+            bad_stage = page < 0 ? (bad_stage | (1u << s)) : (bad_stage & ~(1u << s));
+        } else {                                        // up to 8 window tokens: one 256-byte row copy per lane
+            const int w0 = (cur.u - cur.si.qp) * WIN_TOKENS;
+            const int n_valid = min(WIN_TOKENS, cur.si.n_win - w0);
+            if (lane == 0) mbar_expect_tx(bar, n_valid * 2 * D * 2);
+            __syncwarp();
+            const int r = lane & 7, which = lane >> 3;  // lanes 0-7: key rows, 8-15: value rows
+            if (lane < 16 && r < n_valid) {
+                const int w = w0 + r;
+                const long long plane = (static_cast<long long>(cur.si.slot) * c.n_kv + cur.h) * 2 + which;
+                const unsigned short* src;
+                if (w < cur.si.n_sink) src = c.sink_kv + (plane * c.s_sink + w) * D;
+                else src = c.ring_kv + (plane * c.ring_cap + (cur.si.recent_lo + (w - cur.si.n_sink)) % c.ring_cap) * D;
+                bulk_copy_g2s(dst + which * WIN_V_OFF + r * WIN_ROW, src, D * 2, bar);
+            }
             bad_stage &= ~(1u << s);
-            const unsigned char* src = c.pages + (static_cast<long long>(page) * c.n_kv + h) * REC;
-            mbar_expect_tx(bar0 + 8 * s, REC);
-            bulk_copy_g2s(stage0 + s * REC, src, REC, bar0 + 8 * s);
         }
     };
-    if (lane == 0) {
-#pragma unroll
-        for (int s = 0; s < STAGES; ++s) {
-            const int pg = pg0 + warp + s * MAIN_WARPS;
-            if (pg < pg1) issue(pg, s);
-        }
-    }
+    for (int s = 0; s < STAGES && s < n_units; ++s) { issue(prod, s); advance(prod); }
 
-    // ---- query fragments and per-head scalars
+    // ---- per (sequence, KV head) segment state
     unsigned qf[8][2];
-    {
-        const uint4* src = P.qfrag + (static_cast<long long>(b) * c.n_kv + h) * 128;
+    float fmul[NH], gadd[NH];
+    WarpState<MODE> st;
+    auto begin_segment = [&](const Cursor& cur) {
+        const long long bh = static_cast<long long>(cur.b) * c.n_kv + cur.h;
+        const uint4* src = P.qfrag + bh * 128;
 #pragma unroll
         for (int s2 = 0; s2 < 4; ++s2) {
             const uint4 v = __ldg(src + s2 * 32 + lane);
             qf[2 * s2][0] = v.x; qf[2 * s2][1] = v.y; qf[2 * s2 + 1][0] = v.z; qf[2 * s2 + 1][1] = v.w;
         }
-    }
-    float fmul[NH], gadd[NH];
 #pragma unroll
-    for (int k = 0; k < NH; ++k) {
-        const int head = MODE == 0 ? t : 2 * t + k;
-        fmul[k] = gadd[k] = 0.f;
-        if (head < G) {
-            const float2 v = __ldg(reinterpret_cast<const float2*>(P.qscal + (static_cast<long long>(b) * c.n_q + h * G + head) * 2));
-            fmul[k] = v.x; gadd[k] = v.y;
+        for (int k = 0; k < NH; ++k) {
+            const int head = MODE == 0 ? t : 2 * t + k;
+            fmul[k] = gadd[k] = 0.f;
+            if (head < G) {
+                const float2 v = __ldg(reinterpret_cast<const float2*>(P.qscal + (static_cast<long long>(cur.b) * c.n_q + cur.h * G + head) * 2));
+                fmul[k] = v.x; gadd[k] = v.y;
+            }
         }
-    }
-
-    WarpState<MODE> st;
-#pragma unroll
-    for (int k = 0; k < NH; ++k) { st.m[k] = -INFINITY; st.l[k] = 0.f; st.z[k] = 0.f; }
-#pragma unroll
-    for (int i = 0; i < 8; ++i) st.o[i][0] = st.o[i][1] = st.o[i][2] = st.o[i][3] = 0.f;
+        st.reset();
+    };
+    auto end_segment = [&](const Cursor& cur) {
+        const long long bh = static_cast<long long>(cur.b) * c.n_kv + cur.h;
+        store_partial<BITS, MODE>(st, P.part + (wg + bh) * G * PART_STRIDE, lane, G);
+    };
+    begin_segment(cons);
 
     bool timed_out = false;
-    int it = 0;
-    for (int pg = pg0 + warp; pg < pg1; pg += MAIN_WARPS, ++it) {
+    for (int it = 0; it < n_units; ++it) {
         const int s = it % STAGES;
         const unsigned parity = (it / STAGES) & 1;
         // a phase that one lane saw complete is complete for all: keep the decision warp-uniform
         if (!__any_sync(FULL, mbar_wait_bounded(bar0 + 8 * s, parity))) { timed_out = true; break; }
-        const bool bad = __shfl_sync(FULL, (bad_stage >> s) & 1u, 0) != 0;
-        if (!bad) {
-            const unsigned rec = stage0 + s * REC;
-            const int pos0 = pg * PAGE_TOKENS;
-            const bool full_page = (pos0 >= q_lo) && (pos0 + PAGE_TOKENS <= q_hi);
-            // ---------------- scores of the 64 tokens
+        const unsigned rec = stage0 + s * REC;
+        if (cons.u >= cons.si.qp) {
+            // ======================= window unit: up to 8 bf16 tokens ==============================
+            const int w0 = (cons.u - cons.si.qp) * WIN_TOKENS;
+            const int n_valid = min(WIN_TOKENS, cons.si.n_win - w0);
+            const int r_eff = (lane & 7) < n_valid ? (lane & 7) : 0;      // rows beyond the valid ones alias row 0
+            const int mat = lane >> 3;
+            const unsigned frag_off = r_eff * WIN_ROW + ((mat >> 1) * 16 + (mat & 1) * 8) * 2;
+            const uint4* wsrc = P.qwfrag + (static_cast<long long>(cons.b) * c.n_kv + cons.h) * 256;
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int pass = 0; pass < (MODE == 0 ? 1 : 2); ++pass) {
+#pragma unroll
+                for (int s2 = 0; s2 < 4; ++s2) {
+                    const uint4 bq = __ldg(wsrc + pass * 128 + s2 * 32 + lane);
+                    unsigned k0, k1, k2, k3;                              // (step 2s2: ch lo, ch hi), (step 2s2+1: ch lo, ch hi)
+                    ldmatrix_x4(rec + frag_off + s2 * 64, k0, k1, k2, k3);
+                    mma_bf16(acc, k0, k0, k1, k1, bq.x, bq.y);            // token rows 8..15 alias rows 0..7
+                    mma_bf16(acc, k2, k2, k3, k3, bq.z, bq.w);
+                }
+            }
+            const bool ok = g < n_valid;
+            float sc[NH], mx[NH], mref[NH];
+            if (MODE == 0) sc[0] = ok ? acc[0] + acc[1] : -INFINITY;
+            else { sc[0] = ok ? acc[0] : -INFINITY; sc[NH - 1] = ok ? acc[1] : -INFINITY; }
+#pragma unroll
+            for (int k = 0; k < NH; ++k) {
+                mx[k] = sc[k];
+                mx[k] = fmaxf(mx[k], __shfl_xor_sync(FULL, mx[k], 4));
+                mx[k] = fmaxf(mx[k], __shfl_xor_sync(FULL, mx[k], 8));
+                mx[k] = fmaxf(mx[k], __shfl_xor_sync(FULL, mx[k], 16));
+            }
+            st.raise_max(mx, mref);
+            float p[NH];
+#pragma unroll
+            for (int k = 0; k < NH; ++k) { p[k] = ex2(sc[k] - mref[k]); st.l[k] += p[k]; }
+#pragma unroll
+            for (int pass = 0; pass < (MODE == 0 ? 1 : 2); ++pass) {
+                unsigned pr;                                              // this token's probabilities in the score-fragment layout
+                if (MODE == 0) pr = pack_bf2(p[0], (p[0] - bf16_round(p[0])) * LO_SCALE);   // value column, remainder column
+                else if (pass == 0) pr = pack_bf2(p[0], p[NH - 1]);
+                else pr = pack_bf2(p[0] - bf16_round(p[0]), p[NH - 1] - bf16_round(p[NH - 1]));
+                const unsigned b01 = movmatrix_trans(pr);                 // tokens 2t, 2t+1 of column g; tokens 8..15 get zero
+#pragma unroll
+                for (int i2 = 0; i2 < 4; ++i2) {
+                    unsigned v0, v1, v2, v3;                              // (block 2i2: ch lo, ch hi), (block 2i2+1: ch lo, ch hi)
+                    ldmatrix_x4_trans(rec + WIN_V_OFF + frag_off + i2 * 64, v0, v1, v2, v3);
+                    // fold the block's accumulator unit in: p * v * PV_SCALE * 2^(shift - 24)
+                    mma_bf16(st.o[2 * i2], v0, v1, v0, v1, mul_bf2(b01, bf16x2_pow2(field_shift<BITS>(2 * i2) - 20)), 0u);
+                    mma_bf16(st.o[2 * i2 + 1], v2, v3, v2, v3, mul_bf2(b01, bf16x2_pow2(field_shift<BITS>(2 * i2 + 1) - 20)), 0u);
+                }
+            }
+        } else if (((bad_stage >> s) & 1u) == 0) {
+            // ======================= packed page: 64 quantized tokens ==============================
+            const int pos0 = (cons.si.first_page + cons.u) * PAGE_TOKENS;
+            const bool full_page = (pos0 >= cons.si.q_lo) && (pos0 + PAGE_TOKENS <= cons.si.q_hi);
             float sc[4][2 * NH];          // [block][row g: heads..., row g+8: heads...]
             unsigned vmeta[4][2];         // fp16x2 (Delta_v, x_min_v) of rows g, g+8
 #pragma unroll
             for (int bi = 0; bi < 4; ++bi) {
-                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                float acc[4] = {0.f, 0.f, 0.f, 0.f}, acc2[4] = {0.f, 0.f, 0.f, 0.f};      // two chains for ILP
                 if (BITS == 2) {
                     const uint4 kw = lds128(rec + bi * CB + 16 * lane);
                     const unsigned sx = pre_shift<2>(kw.x), sy = pre_shift<2>(kw.y), sz = pre_shift<2>(kw.z), sw = pre_shift<2>(kw.w);
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        mma16816(acc, field<2>(kw.x, sx, ks), field<2>(kw.z, sz, ks), field<2>(kw.y, sy, ks), field<2>(kw.w, sw, ks),
-                                 qf[ks][0], qf[ks][1]);
+                    for (int ks = 0; ks < 8; ks += 2) {
+                        mma_f16(acc, field<2>(kw.x, sx, ks), field<2>(kw.z, sz, ks), field<2>(kw.y, sy, ks), field<2>(kw.w, sw, ks),
+                                qf[ks][0], qf[ks][1]);
+                        mma_f16(acc2, field<2>(kw.x, sx, ks + 1), field<2>(kw.z, sz, ks + 1), field<2>(kw.y, sy, ks + 1), field<2>(kw.w, sw, ks + 1),
+                                qf[ks + 1][0], qf[ks + 1][1]);
+                    }
                 } else {
                     const uint4 ka = lds128(rec + bi * CB + 16 * lane);          // row g:   W0..W3
                     const uint4 kb = lds128(rec + bi * CB + 512 + 16 * lane);    // row g+8: W0..W3
                     const unsigned a0s = pre_shift<4>(ka.x), a1s = pre_shift<4>(ka.y), a2s = pre_shift<4>(ka.z), a3s = pre_shift<4>(ka.w);
                     const unsigned b0s = pre_shift<4>(kb.x), b1s = pre_shift<4>(kb.y), b2s = pre_shift<4>(kb.z), b3s = pre_shift<4>(kb.w);
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        mma16816(acc, field<4>(ka.x, a0s, ks), field<4>(kb.x, b0s, ks), field<4>(ka.y, a1s, ks), field<4>(kb.y, b1s, ks),
-                                 qf[ks][0], qf[ks][1]);
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        mma16816(acc, field<4>(ka.z, a2s, ks), field<4>(kb.z, b2s, ks), field<4>(ka.w, a3s, ks), field<4>(kb.w, b3s, ks),
-                                 qf[4 + ks][0], qf[4 + ks][1]);
+                    for (int ks = 0; ks < 4; ++ks) {
+                        mma_f16(acc, field<4>(ka.x, a0s, ks), field<4>(kb.x, b0s, ks), field<4>(ka.y, a1s, ks), field<4>(kb.y, b1s, ks),
+                                qf[ks][0], qf[ks][1]);
+                        mma_f16(acc2, field<4>(ka.z, a2s, ks), field<4>(kb.z, b2s, ks), field<4>(ka.w, a3s, ks), field<4>(kb.w, b3s, ks),
+                                qf[4 + ks][0], qf[4 + ks][1]);
+                    }
                 }
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[e] += acc2[e];
                 const uint4 mt = lds128(rec + meta_offset(BITS) + 128 * bi + 16 * g);   // rows g (x,y) and g+8 (z,w)
-                float kd0 = h_lo(mt.x), km0 = h_hi(mt.x), kd1 = h_lo(mt.z), km1 = h_hi(mt.z);
+                const float kd0 = h_lo(mt.x), km0 = h_hi(mt.x), kd1 = h_lo(mt.z), km1 = h_hi(mt.z);
                 unsigned vm0 = mt.y, vm1 = mt.w;
                 bool ok0 = true, ok1 = true;
                 if (!full_page) {
                     const int p0 = pos0 + bi * 16 + g, p1 = p0 + 8;
-                    ok0 = (p0 >= q_lo) && (p0 < q_hi);
-                    ok1 = (p1 >= q_lo) && (p1 < q_hi);
+                    ok0 = (p0 >= cons.si.q_lo) && (p0 < cons.si.q_hi);
+                    ok1 = (p1 >= cons.si.q_lo) && (p1 < cons.si.q_hi);
                     if (!ok0) vm0 = 0u;
                     if (!ok1) vm1 = 0u;
                 }
                 vmeta[bi][0] = vm0; vmeta[bi][1] = vm1;
                 if (MODE == 0) {
-                    const float d0 = acc[0] + acc[1] * (1.f / LO_SCALE), d1 = acc[2] + acc[3] * (1.f / LO_SCALE);
+                    const float d0 = fmaf(acc[1], 1.f / LO_SCALE, acc[0]), d1 = fmaf(acc[3], 1.f / LO_SCALE, acc[2]);
                     const float s0 = fmaf(d0 * kd0, fmul[0], km0 * gadd[0]);
                     const float s1 = fmaf(d1 * kd1, fmul[0], km1 * gadd[0]);
                     sc[bi][0] = ok0 ? s0 : -INFINITY;
-                    sc[bi][1] = ok1 ? s1 : -INFINITY;
+                    sc[bi][NH] = ok1 ? s1 : -INFINITY;
                 } else {
                     const float s00 = fmaf(acc[0] * kd0, fmul[0], km0 * gadd[0]);
-                    const float s01 = fmaf(acc[1] * kd0, fmul[1], km0 * gadd[1]);
+                    const float s01 = fmaf(acc[1] * kd0, fmul[NH - 1], km0 * gadd[NH - 1]);
                     const float s10 = fmaf(acc[2] * kd1, fmul[0], km1 * gadd[0]);
-                    const float s11 = fmaf(acc[3] * kd1, fmul[1], km1 * gadd[1]);
-                    sc[bi][0] = ok0 ? s00 : -INFINITY; sc[bi][1] = ok0 ? s01 : -INFINITY;
-                    sc[bi][2] = ok1 ? s10 : -INFINITY; sc[bi][3] = ok1 ? s11 : -INFINITY;
+                    const float s11 = fmaf(acc[3] * kd1, fmul[NH - 1], km1 * gadd[NH - 1]);
+                    sc[bi][0] = ok0 ? s00 : -INFINITY; sc[bi][NH - 1] = ok0 ? s01 : -INFINITY;
+                    sc[bi][NH] = ok1 ? s10 : -INFINITY; sc[bi][2 * NH - 1] = ok1 ? s11 : -INFINITY;
                 }
             }
             // ---------------- running maximum of the page, rescale if it grew
-            float mref[NH], mnew[NH];
-            bool grew = false;
+            float mx[NH], mref[NH];
 #pragma unroll
             for (int k = 0; k < NH; ++k) {
-                float mx;
-                if (MODE == 0) mx = fmaxf(fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1])),
-                                          fmaxf(fmaxf(sc[2][0], sc[2][1]), fmaxf(sc[3][0], sc[3][1])));
-                else mx = fmaxf(fmaxf(fmaxf(sc[0][k], sc[0][2 + k]), fmaxf(sc[1][k], sc[1][2 + k])),
-                                fmaxf(fmaxf(sc[2][k], sc[2][2 + k]), fmaxf(sc[3][k], sc[3][2 + k])));
-                mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 4));
-                mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 8));
-                mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 16));
-                mnew[k] = fmaxf(st.m[k], mx);
-                grew |= mnew[k] > st.m[k];
-                mref[k] = (mnew[k] == -INFINITY) ? 0.f : mnew[k];     // all-masked so far: any finite reference works
+                float v = fmaxf(fmaxf(fmaxf(sc[0][k], sc[0][NH + k]), fmaxf(sc[1][k], sc[1][NH + k])),
+                                fmaxf(fmaxf(sc[2][k], sc[2][NH + k]), fmaxf(sc[3][k], sc[3][NH + k])));
+                v = fmaxf(v, __shfl_xor_sync(FULL, v, 4));
+                v = fmaxf(v, __shfl_xor_sync(FULL, v, 8));
+                v = fmaxf(v, __shfl_xor_sync(FULL, v, 16));
+                mx[k] = v;
             }
-            if (__any_sync(FULL, grew)) {
-                float scl[NH];
-#pragma unroll
-                for (int k = 0; k < NH; ++k) {
-                    scl[k] = exp2f(st.m[k] - mref[k]);                // old max -inf: state is all zero, factor 0
-                    st.l[k] *= scl[k]; st.z[k] *= scl[k];
-                    st.m[k] = mnew[k];
-                }
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    if (MODE == 0) { st.o[i][0] *= scl[0]; st.o[i][1] *= scl[0]; st.o[i][2] *= scl[0]; st.o[i][3] *= scl[0]; }
-                    else { st.o[i][0] *= scl[0]; st.o[i][1] *= scl[1]; st.o[i][2] *= scl[0]; st.o[i][3] *= scl[1]; }
-                }
-            }
+            st.raise_max(mx, mref);
             // ---------------- probabilities, value reduction
 #pragma unroll
             for (int bi = 0; bi < 4; ++bi) {
-                const float vd0 = h_lo(vmeta[bi][0]), vn0 = h_hi(vmeta[bi][0]);
-                const float vd1 = h_lo(vmeta[bi][1]), vn1 = h_hi(vmeta[bi][1]);
+                const float vd0 = h_lo(vmeta[bi][0]) * PV_SCALE, vn0 = h_hi(vmeta[bi][0]);
+                const float vd1 = h_lo(vmeta[bi][1]) * PV_SCALE, vn1 = h_hi(vmeta[bi][1]);
                 unsigned r0, r1;
                 if (MODE == 0) {
-                    const float p0 = exp2f(sc[bi][0] - mref[0]), p1 = exp2f(sc[bi][1] - mref[0]);
+                    const float p0 = ex2(sc[bi][0] - mref[0]), p1 = ex2(sc[bi][NH] - mref[0]);
                     st.l[0] += p0 + p1;
                     st.z[0] = fmaf(p0, vn0, fmaf(p1, vn1, st.z[0]));
-                    const float w0 = p0 * vd0 * PV_SCALE, w1 = p1 * vd1 * PV_SCALE;
-                    const float w0h = __half2float(__float2half_rn(w0)), w1h = __half2float(__float2half_rn(w1));
-                    r0 = pack_h2(w0, (w0 - w0h) * LO_SCALE);
-                    r1 = pack_h2(w1, (w1 - w1h) * LO_SCALE);
+                    r0 = pack_h2(p0 * vd0, 0.f);
+                    r1 = pack_h2(p1 * vd1, 0.f);
                 } else {
-                    const float p00 = exp2f(sc[bi][0] - mref[0]), p01 = exp2f(sc[bi][1] - mref[1]);
-                    const float p10 = exp2f(sc[bi][2] - mref[0]), p11 = exp2f(sc[bi][3] - mref[1]);
-                    st.l[0] += p00 + p10; st.l[1] += p01 + p11;
+                    const float p00 = ex2(sc[bi][0] - mref[0]), p01 = ex2(sc[bi][NH - 1] - mref[NH - 1]);
+                    const float p10 = ex2(sc[bi][NH] - mref[0]), p11 = ex2(sc[bi][2 * NH - 1] - mref[NH - 1]);
+                    st.l[0] += p00 + p10; st.l[NH - 1] += p01 + p11;
                     st.z[0] = fmaf(p00, vn0, fmaf(p10, vn1, st.z[0]));
-                    st.z[1] = fmaf(p01, vn0, fmaf(p11, vn1, st.z[1]));
-                    r0 = pack_h2(p00 * vd0 * PV_SCALE, p01 * vd0 * PV_SCALE);
-                    r1 = pack_h2(p10 * vd1 * PV_SCALE, p11 * vd1 * PV_SCALE);
+                    st.z[NH - 1] = fmaf(p01, vn0, fmaf(p11, vn1, st.z[NH - 1]));
+                    r0 = pack_h2(p00 * vd0, p01 * vd0);
+                    r1 = pack_h2(p10 * vd1, p11 * vd1);
                 }
                 const unsigned b01 = movmatrix_trans(r0), b23 = movmatrix_trans(r1);
                 if (BITS == 2) {
@@ -563,7 +678,7 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32) decode_main_kernel(DecodePara
                     const unsigned sx = pre_shift<2>(vw.x), sy = pre_shift<2>(vw.y), sz = pre_shift<2>(vw.z), sw = pre_shift<2>(vw.w);
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
-                        mma16816(st.o[i], field<2>(vw.x, sx, i), field<2>(vw.y, sy, i), field<2>(vw.z, sz, i), field<2>(vw.w, sw, i), b01, b23);
+                        mma_f16(st.o[i], field<2>(vw.x, sx, i), field<2>(vw.y, sy, i), field<2>(vw.z, sz, i), field<2>(vw.w, sw, i), b01, b23);
                 } else {
                     const uint4 va = lds128(rec + v_codes_offset(4) + bi * CB + 16 * lane);         // tokens 2t,2t+1
                     const uint4 vb = lds128(rec + v_codes_offset(4) + bi * CB + 512 + 16 * lane);   // tokens 2t+8,2t+9
@@ -571,26 +686,30 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32) decode_main_kernel(DecodePara
                     const unsigned b0s = pre_shift<4>(vb.x), b1s = pre_shift<4>(vb.y), b2s = pre_shift<4>(vb.z), b3s = pre_shift<4>(vb.w);
 #pragma unroll
                     for (int k = 0; k < 4; ++k)     // channel blocks 0..3: words (rsel, j=0)
-                        mma16816(st.o[k], field<4>(va.x, a0s, k), field<4>(va.z, a2s, k), field<4>(vb.x, b0s, k), field<4>(vb.z, b2s, k), b01, b23);
+                        mma_f16(st.o[k], field<4>(va.x, a0s, k), field<4>(va.z, a2s, k), field<4>(vb.x, b0s, k), field<4>(vb.z, b2s, k), b01, b23);
 #pragma unroll
                     for (int k = 0; k < 4; ++k)     // channel blocks 4..7: words (rsel, j=1)
-                        mma16816(st.o[4 + k], field<4>(va.y, a1s, k), field<4>(va.w, a3s, k), field<4>(vb.y, b1s, k), field<4>(vb.w, b3s, k), b01, b23);
+                        mma_f16(st.o[4 + k], field<4>(va.y, a1s, k), field<4>(va.w, a3s, k), field<4>(vb.y, b1s, k), field<4>(vb.w, b3s, k), b01, b23);
                 }
             }
         }
         __syncwarp();
-        const int next = pg + STAGES * MAIN_WARPS;
-        if (lane == 0 && next < pg1) issue(next, s);
+        if (it + STAGES < n_units) { issue(prod, s); advance(prod); }
+        // ---- next unit; a change of (sequence, KV head) closes this warp's partial
+        if (it + 1 < n_units) {
+            const int pb = cons.b, ph = cons.h;
+            Cursor nxt = cons;
+            advance(nxt);
+            if (nxt.b != pb || nxt.h != ph) { end_segment(cons); begin_segment(nxt); }
+            cons = nxt;
+        }
     }
     if (timed_out) {
         if (lane == 0) atomicOr(c.dev_status, WUSHKV_DEV_COPY_TIMEOUT);
-        // give copies that may still be in flight a bounded time to land before the staging area is reused
+        // give copies that may still be in flight a bounded time to land before the CTA's memory is released
         for (int k = 0; k < 1000; ++k) __nanosleep(1000);
     }
-    __syncthreads();                    // every warp has drained its stages: the staging area becomes scratch
-    spill_warp_state<BITS, MODE>(st, scratch + warp * 8 * PART_STRIDE, lane, G);
-    __syncthreads();
-    merge_and_store(scratch, MAIN_WARPS, G, part_base, head_stride, tid, blockDim.x);
+    end_segment(cons);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -599,23 +718,30 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32) decode_main_kernel(DecodePara
 __global__ void __launch_bounds__(128) decode_combine_kernel(DecodeParams P) {
     const CacheView& c = P.c;
     const int j = blockIdx.x, b = blockIdx.y, ch = threadIdx.x;
-    const int S = __ldg(P.seq_len + b);
-    const int slot = __ldg(P.slot + b);
     float* out = P.O + (static_cast<long long>(b) * c.n_q + j) * D;
-    if (slot < 0 || slot >= c.n_slots || S <= 0) { out[ch] = 0.f; return; }
-    const int nq = n_quantized(S - c.lag, c.s_sink, c.s_keep, c.s_flush);
-    int valid_chunks = 0;
-    if (nq > 0) {
-        const int first_page = c.s_sink / PAGE_TOKENS, last_page = (c.s_sink + nq - 1) / PAGE_TOKENS;
-        valid_chunks = min((last_page - first_page) / P.chunk_pages + 1, P.n_chunks);
+    const long long U = P.plan[b + 1] - P.plan[b];
+    const long long total = P.plan[P.batch] * c.n_kv;
+    if (U <= 0 || total <= 0) { out[ch] = 0.f; return; }
+    const int h = j / c.G, head = j % c.G;
+    const long long La = P.plan[b] * c.n_kv + static_cast<long long>(h) * U, Lb = La + U;      // units [La, Lb)
+    const long long nw = P.n_warps;
+    const long long w_first = ((La + 1) * nw - 1) / total, w_last = (Lb * nw - 1) / total;     // owners of La and Lb-1
+    const long long bh = static_cast<long long>(b) * c.n_kv + h;
+    const float* base = P.part + ((w_first + bh) * c.G + head) * PART_STRIDE;
+    const long long stride = static_cast<long long>(c.G) * PART_STRIDE;
+    const int n = static_cast<int>(w_last - w_first + 1);
+    float m = -INFINITY;
+    for (int s = 0; s < n; ++s) {
+        const long long w = w_first + s;
+        const long long lo = max(w * total / nw, La), hi = min((w + 1) * total / nw, Lb);
+        if (lo < hi) m = fmaxf(m, base[s * stride]);
     }
-    const int n_splits = P.n_chunks + 1;
-    const float* base = P.part + (static_cast<long long>(b) * c.n_q + j) * n_splits * PART_STRIDE;
-    float m = base[P.n_chunks * PART_STRIDE];
-    for (int s = 0; s < valid_chunks; ++s) m = fmaxf(m, base[s * PART_STRIDE]);
     float l = 0.f, o = 0.f;
-    for (int s = 0; s <= valid_chunks; ++s) {
-        const float* p = base + (s < valid_chunks ? s : P.n_chunks) * PART_STRIDE;
+    for (int s = 0; s < n; ++s) {
+        const long long w = w_first + s;
+        const long long lo = max(w * total / nw, La), hi = min((w + 1) * total / nw, Lb);
+        if (lo >= hi) continue;                       // a warp with an empty slice wrote nothing
+        const float* p = base + s * stride;
         const float scl = (p[0] == -INFINITY) ? 0.f : exp2f(p[0] - m);
         l += scl * p[1];
         o += scl * p[4 + ch];
@@ -627,31 +753,33 @@ __global__ void __launch_bounds__(128) decode_combine_kernel(DecodeParams P) {
 // host side
 // ------------------------------------------------------------------------------------------------
 struct DecodePlan {
-    int chunk_pages, n_chunks;
-    size_t off_qfrag, off_qscal, off_qcomp, off_part, total;
+    int n_ctas, n_warps;
+    size_t off_qfrag, off_qwfrag, off_qscal, off_plan, off_part, total;
 };
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 static bool make_plan(const CacheView& c, int batch, int max_seq_len, DecodePlan& pl) {
     if (batch <= 0 || max_seq_len <= 0) return false;
-    const long long pages_max = (static_cast<long long>(max_seq_len) + PAGE_TOKENS - 1) / PAGE_TOKENS;
-    const long long total_pages = pages_max * batch * c.n_kv;
-    long long cp = 0;
-    if (const char* e = std::getenv("WUSHKV_CHUNK_PAGES")) cp = std::atoll(e);
-    if (cp <= 0) {
-        const long long want_ctas = 8LL * sm_count();          // a few waves of CTAs for balance
-        cp = (total_pages + want_ctas - 1) / want_ctas;
-        cp = std::max<long long>(cp, 2 * MAIN_WARPS);
+    const long long pages_max = (static_cast<long long>(max_seq_len) + PAGE_TOKENS - 1) / PAGE_TOKENS + 1;
+    const long long win_max = std::min<long long>(max_seq_len, c.s_sink + c.s_keep + c.s_flush - 1 + c.lag);
+    const long long units_max = (pages_max + (win_max + WIN_TOKENS - 1) / WIN_TOKENS + 1) * batch * c.n_kv;
+    long long ctas = 0;
+    if (const char* e = std::getenv("WUSHKV_DECODE_CTAS")) ctas = std::atoll(e);
+    if (ctas <= 0) {
+        const long long per_sm = c.bits == 2 ? 4 : 2;                   // CTAs that fit one SM's shared memory
+        ctas = std::min<long long>(per_sm * sm_count(), (units_max + 2 * MAIN_WARPS - 1) / (2 * MAIN_WARPS));
     }
-    cp = std::min<long long>(cp, pages_max);
-    pl.chunk_pages = static_cast<int>(cp);
-    pl.n_chunks = static_cast<int>((pages_max + cp - 1) / cp);
+    ctas = std::max<long long>(1, std::min<long long>(ctas, 1 << 20));
+    pl.n_ctas = static_cast<int>(ctas);
+    pl.n_warps = pl.n_ctas * MAIN_WARPS;
+    const size_t bh = static_cast<size_t>(batch) * c.n_kv;
     size_t off = 0;
-    pl.off_qfrag = off; off = align_up(off + static_cast<size_t>(batch) * c.n_kv * 128 * sizeof(uint4), 256);
-    pl.off_qscal = off; off = align_up(off + static_cast<size_t>(batch) * c.n_q * 2 * sizeof(float), 256);
-    pl.off_qcomp = off; off = align_up(off + static_cast<size_t>(batch) * c.n_q * D * sizeof(float), 256);
-    pl.off_part = off;  off = align_up(off + static_cast<size_t>(batch) * c.n_q * (pl.n_chunks + 1) * PART_STRIDE * sizeof(float), 256);
+    pl.off_qfrag = off;  off = align_up(off + bh * 128 * sizeof(uint4), 256);
+    pl.off_qwfrag = off; off = align_up(off + bh * 256 * sizeof(uint4), 256);
+    pl.off_qscal = off;  off = align_up(off + static_cast<size_t>(batch) * c.n_q * 2 * sizeof(float), 256);
+    pl.off_plan = off;   off = align_up(off + (static_cast<size_t>(batch) + 1) * sizeof(long long), 256);
+    pl.off_part = off;   off = align_up(off + (pl.n_warps + bh) * c.G * PART_STRIDE * sizeof(float), 256);
     pl.total = off;
     return true;
 }
@@ -659,16 +787,15 @@ static bool make_plan(const CacheView& c, int batch, int max_seq_len, DecodePlan
 static cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
 
 template <int BITS, int MODE>
-static int launch_decode(const DecodeParams& P, cudaStream_t st) {
-    constexpr int STAGES = BITS == 2 ? 4 : 3;
+static int launch_decode(const DecodeParams& P, int n_ctas, cudaStream_t st) {
+    constexpr int STAGES = 3;
     constexpr size_t SMEM = static_cast<size_t>(MAIN_WARPS) * STAGES * record_bytes(BITS) + MAIN_WARPS * STAGES * 8;
-    static_assert(SMEM >= static_cast<size_t>(MAIN_WARPS) * 8 * PART_STRIDE * sizeof(float), "scratch must fit in the staging area");
     decode_prep_kernel<BITS, MODE><<<dim3(P.c.n_kv, P.batch), 128, 0, st>>>(P);
     if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
     if (cudaFuncSetAttribute(decode_main_kernel<BITS, MODE, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(SMEM)) != cudaSuccess)
         return WUSHKV_ECUDA;
     if (g_prof_start) cudaEventRecord(g_prof_start, st);
-    decode_main_kernel<BITS, MODE, STAGES><<<dim3(P.n_chunks + 1, P.c.n_kv, P.batch), MAIN_WARPS * 32, SMEM, st>>>(P);
+    decode_main_kernel<BITS, MODE, STAGES><<<n_ctas, MAIN_WARPS * 32, SMEM, st>>>(P);
     if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
     if (g_prof_stop) cudaEventRecord(g_prof_stop, st);
     decode_combine_kernel<<<dim3(P.c.n_q, P.batch), 128, 0, st>>>(P);
@@ -697,19 +824,20 @@ extern "C" int wushkv_decode_attn(const wushkv_cache* cache, int32_t batch, cons
     if (!slot || !seq_len || !Q || !O || !workspace || !aligned(Q, 16) || !aligned(O, 16) || !aligned(workspace, 256)) return WUSHKV_EINVAL;
     DecodePlan pl;
     if (!make_plan(P.c, batch, max_seq_len, pl)) return WUSHKV_EINVAL;
-    if (batch > 65535 || pl.n_chunks + 1 > 0x7fffffff) return WUSHKV_EINVAL;
+    if (batch > 65535) return WUSHKV_EINVAL;
     if (workspace_bytes < pl.total) return WUSHKV_ECAPACITY;
     unsigned char* ws = static_cast<unsigned char*>(workspace);
     P.batch = batch; P.slot = slot; P.seq_len = seq_len; P.Q = Q; P.O = O;
     P.qfrag = reinterpret_cast<uint4*>(ws + pl.off_qfrag);
+    P.qwfrag = reinterpret_cast<uint4*>(ws + pl.off_qwfrag);
     P.qscal = reinterpret_cast<float*>(ws + pl.off_qscal);
-    P.qcomp = reinterpret_cast<float*>(ws + pl.off_qcomp);
+    P.plan = reinterpret_cast<long long*>(ws + pl.off_plan);
     P.part = reinterpret_cast<float*>(ws + pl.off_part);
-    P.n_chunks = pl.n_chunks; P.chunk_pages = pl.chunk_pages;
+    P.n_warps = pl.n_warps;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool mode0 = P.c.G <= 4;
-    if (P.c.bits == 2) return mode0 ? launch_decode<2, 0>(P, st) : launch_decode<2, 1>(P, st);
-    return mode0 ? launch_decode<4, 0>(P, st) : launch_decode<4, 1>(P, st);
+    if (P.c.bits == 2) return mode0 ? launch_decode<2, 0>(P, pl.n_ctas, st) : launch_decode<2, 1>(P, pl.n_ctas, st);
+    return mode0 ? launch_decode<4, 0>(P, pl.n_ctas, st) : launch_decode<4, 1>(P, pl.n_ctas, st);
 }
 
 extern "C" int wushkv_set_profile_events(void* start, void* stop) {

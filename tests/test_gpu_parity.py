@@ -105,13 +105,13 @@ def test_decode_is_deterministic_and_split_invariant(monkeypatch):
     L = Layer(wl, [3000], 2, 4, 64, 1)
     L.fill()
     outs = []
-    for cp in ("8", "8", "13", "64"):
-        monkeypatch.setenv("WUSHKV_CHUNK_PAGES", cp)
+    for ctas in ("5", "5", "1", "64"):
+        monkeypatch.setenv("WUSHKV_DECODE_CTAS", ctas)
         outs.append(L.decode()[0])
     assert np.array_equal(outs[0], outs[1])
     scale = np.max(np.abs(outs[0]))
-    assert np.max(np.abs(outs[2] - outs[0])) <= 5e-5 * scale
-    assert np.max(np.abs(outs[3] - outs[0])) <= 5e-5 * scale
+    assert np.max(np.abs(outs[2] - outs[0])) <= 5e-4 * scale
+    assert np.max(np.abs(outs[3] - outs[0])) <= 5e-4 * scale
 
 
 def test_device_side_errors_are_flagged_not_fatal():
