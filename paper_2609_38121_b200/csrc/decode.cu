@@ -44,6 +44,12 @@ constexpr int WIN_TOKENS = 8;             // window tokens per work unit
 constexpr int WIN_ROW = 272;              // padded bytes per staged bf16 row (conflict-free ldmatrix)
 constexpr int WIN_V_OFF = WIN_TOKENS * WIN_ROW;
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute may
+// start while its predecessor in the stream is still running; it must call pdl_wait() before it
+// touches anything the predecessor writes.  Without the attribute both calls are no-ops.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 struct DecodeParams {
     CacheView c;
     int batch;
@@ -109,6 +115,7 @@ __global__ void __launch_bounds__(128) decode_prep_kernel(DecodeParams P) {
     __shared__ long long scan_s[4];
     const int h = blockIdx.x, b = blockIdx.y, G = P.c.G;
     const int i = threadIdx.x, lane = i & 31, warp = i >> 5;
+    pdl_launch_dependents();              // the main kernel may start staging pages while this one runs
 
     if (h == 0 && b == 0) {               // work plan: exclusive prefix of units per sequence
         long long carry = 0;
@@ -234,24 +241,25 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
     unsigned ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(2000u) : "memory");      // may sleep up to ~2 us in hardware
     return ok != 0;
 }
-// Bounded wait: false if the phase did not complete within the limit.
+// Bounded wait: false if the phase did not complete within the limit (about a second of sleeping polls).
 __device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity) {
-    for (int it = 0; it < (1 << 22); ++it)
+    for (int it = 0; it < (1 << 19); ++it)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
+
 __device__ __forceinline__ void bulk_copy_g2s(unsigned dst, const void* src, unsigned bytes, unsigned bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 __device__ __forceinline__ uint4 lds128(unsigned addr) {
     uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    asm("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
     return v;
 }
 __device__ __forceinline__ void ldmatrix_x4(unsigned addr, unsigned& a, unsigned& b, unsigned& c, unsigned& d) {
@@ -261,18 +269,18 @@ __device__ __forceinline__ void ldmatrix_x4_trans(unsigned addr, unsigned& a, un
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "r"(addr));
 }
 __device__ __forceinline__ void mma_f16(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0, unsigned b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ void mma_bf16(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0, unsigned b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ unsigned movmatrix_trans(unsigned a) {
     unsigned d;
-    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    asm("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
     return d;
 }
 __device__ __forceinline__ unsigned pack_h2(float lo, float hi) {      // lo -> bits 0..15, hi -> bits 16..31, saturating
@@ -295,8 +303,11 @@ __device__ __forceinline__ float ex2(float x) {      // 2^x, -inf -> 0
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ float h_lo(unsigned u) { return __half2float(__ushort_as_half(static_cast<unsigned short>(u & 0xffffu))); }
-__device__ __forceinline__ float h_hi(unsigned u) { return __half2float(__ushort_as_half(static_cast<unsigned short>(u >> 16))); }
+__device__ __forceinline__ float2 h2f2(unsigned u) {     // both halves of an fp16x2 register as floats
+    __half2 h;
+    *reinterpret_cast<unsigned*>(&h) = u;
+    return __half22float2(h);
+}
 __device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 
 // Field idx (0..7) of a code word as an fp16x2 A-fragment register.  `w` is the raw word, `ws` the
@@ -388,11 +399,13 @@ __device__ __forceinline__ void store_partial(const WarpState<MODE>& st, float* 
     }
 }
 
-// Position of a warp in the flattened unit list.
-struct Cursor {
-    int b, h, u;
-    SeqInfo si;
+// One (sequence, KV head) stretch of a warp's slice, kept in shared memory.  Units [u0, u1) of the
+// head's unit list: units below qp are packed pages (page index first_page + u), the rest are window
+// units of WIN_TOKENS tokens.
+struct Segment {
+    int b, h, slot, u0, u1, qp, first_page, q_lo, q_hi, n_win, n_sink, recent_lo;
 };
+constexpr int MAX_SEGMENTS = 6;           // per warp and round; more segments take further rounds
 
 // ------------------------------------------------------------------------------------------------
 // main kernel
@@ -405,42 +418,66 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, 4) decode_main_kernel(DecodeP
     static_assert(2 * WIN_TOKENS * WIN_ROW <= REC, "a window unit must fit in one stage");
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + MAIN_WARPS * STAGES * REC);
+    Segment* seg_all = reinterpret_cast<Segment*>(smem + MAIN_WARPS * STAGES * REC + MAIN_WARPS * STAGES * 8);
     const CacheView& c = P.c;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int G = c.G;
+    Segment* segs = seg_all + warp * MAX_SEGMENTS;
+
+    // ---- work plan: prefix sums of units per sequence.  Recomputed here from the inputs (into the still
+    // unused staging area) so that nothing the preparation kernel writes is needed before the first copies.
+    __shared__ long long scan_s[MAIN_WARPS];
+    long long* plan_s = reinterpret_cast<long long*>(smem);
+    const bool local_plan = (static_cast<size_t>(P.batch) + 1) * sizeof(long long) <= static_cast<size_t>(MAIN_WARPS) * STAGES * REC;
+    if (local_plan) {
+        long long carry = 0;
+        for (int base = 0; base < P.batch; base += MAIN_WARPS * 32) {
+            const int bb = base + threadIdx.x;
+            long long incl = 0;
+            if (bb < P.batch) incl = seq_info(c, __ldg(P.seq_len + bb), __ldg(P.slot + bb)).U;
+            for (int o = 1; o < 32; o <<= 1) {
+                const long long v = __shfl_up_sync(FULL, incl, o);
+                if (lane >= o) incl += v;
+            }
+            if (lane == 31) scan_s[warp] = incl;
+            __syncthreads();
+            long long before = 0, all = 0;
+            for (int w = 0; w < MAIN_WARPS; ++w) { if (w < warp) before += scan_s[w]; all += scan_s[w]; }
+            if (bb < P.batch) plan_s[bb + 1] = carry + before + incl;
+            carry += all;
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) plan_s[0] = 0;
+        __syncthreads();
+    } else {
+        pdl_wait();
+    }
+    const long long* plan = local_plan ? plan_s : P.plan;
 
     // ---- this warp's slice of the flattened unit list
-    const long long total = P.plan[P.batch] * c.n_kv;
-    if (total <= 0) return;
+    const long long total = plan[P.batch] * c.n_kv;
     const long long wg = static_cast<long long>(blockIdx.x) * MAIN_WARPS + warp;
-    const long long L0 = wg * total / P.n_warps, L1 = (wg + 1) * total / P.n_warps;
-    if (L0 >= L1) return;
-    const int n_units = static_cast<int>(L1 - L0);
+    long long L = total > 0 ? wg * total / P.n_warps : 0;
+    const long long L1 = total > 0 ? (wg + 1) * total / P.n_warps : 0;
 
-    auto load_seq = [&](int b) { return seq_info(c, __ldg(P.seq_len + b), __ldg(P.slot + b)); };
-    auto advance = [&](Cursor& cur) {
-        if (++cur.u < cur.si.U) return;
-        cur.u = 0;
-        if (++cur.h < c.n_kv) return;
-        cur.h = 0;
-        do { ++cur.b; if (cur.b < P.batch) cur.si = load_seq(cur.b); } while (cur.b < P.batch && cur.si.U == 0);
-    };
-    Cursor cons;
-    {
-        int lo = 0, hi = P.batch;           // largest b with n_kv * plan[b] <= L0
+    // position of the slice start: sequence b, head h, unit u
+    int sb = 0, sh = 0, su = 0;
+    if (L < L1) {
+        int lo = 0, hi = P.batch;           // largest b with n_kv * plan[b] <= L
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
-            if (P.plan[mid] * c.n_kv <= L0) lo = mid; else hi = mid;
+            if (plan[mid] * c.n_kv <= L) lo = mid; else hi = mid;
         }
-        cons.b = lo;
-        cons.si = load_seq(lo);
-        const long long rem = L0 - P.plan[lo] * c.n_kv;
-        const int U = max(cons.si.U, 1);
-        cons.h = static_cast<int>(rem / U);
-        cons.u = static_cast<int>(rem % U);
+        sb = lo;
+        const long long U = max(plan[lo + 1] - plan[lo], 1LL);
+        const long long rem = L - plan[lo] * c.n_kv;
+        sh = static_cast<int>(rem / U);
+        su = static_cast<int>(rem % U);
     }
-    Cursor prod = cons;
+    __syncthreads();                        // the staging area stops being plan scratch here
+    pdl_launch_dependents();
+    if (L >= L1) return;
 
     // ---- barriers
     const unsigned bar0 = smem_u32(bars + warp * STAGES);
@@ -451,265 +488,301 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, 4) decode_main_kernel(DecodeP
     }
     __syncwarp();
     const unsigned stage0 = smem_u32(smem + warp * STAGES * REC);
+    const long long page_row_bytes = static_cast<long long>(c.n_kv) * REC;
 
-    unsigned bad_stage = 0;             // bit s set if the unit staged in s could not be fetched
-    // Stage the unit under `cur` into stage s.  Executed by the whole warp.
-    auto issue = [&](const Cursor& cur, int s) {
-        const unsigned bar = bar0 + 8 * s, dst = stage0 + s * REC;
-        if (cur.u < cur.si.qp) {                        // a packed page: one bulk copy
-            const int pg = cur.si.first_page + cur.u;
-            int page = -1;
-            if (lane == 0) {
-                page = (pg < c.max_pages) ? __ldg(c.page_table + static_cast<long long>(cur.si.slot) * c.max_pages + pg) : -1;
-                if (page < 0 || page >= c.n_pages) {
-                    atomicOr(c.dev_status, pg < c.max_pages ? WUSHKV_DEV_BAD_PAGE_ID : WUSHKV_DEV_PAGE_TABLE_FULL);
-                    page = -1;
-                    mbar_arrive(bar);
-                } else {
-                    mbar_expect_tx(bar, REC);
-                    bulk_copy_g2s(dst, c.pages + (static_cast<long long>(page) * c.n_kv + cur.h) * REC, REC, bar);
-                }
-            }
-            page = __shfl_sync(FULL, page, 0);
-            bad_stage = page < 0 ? (bad_stage | (1u << s)) : (bad_stage & ~(1u << s));
-        } else {                                        // up to 8 window tokens: one 256-byte row copy per lane
-            const int w0 = (cur.u - cur.si.qp) * WIN_TOKENS;
-            const int n_valid = min(WIN_TOKENS, cur.si.n_win - w0);
-            if (lane == 0) mbar_expect_tx(bar, n_valid * 2 * D * 2);
-            __syncwarp();
-            const int r = lane & 7, which = lane >> 3;  // lanes 0-7: key rows, 8-15: value rows
-            if (lane < 16 && r < n_valid) {
-                const int w = w0 + r;
-                const long long plane = (static_cast<long long>(cur.si.slot) * c.n_kv + cur.h) * 2 + which;
-                const unsigned short* src;
-                if (w < cur.si.n_sink) src = c.sink_kv + (plane * c.s_sink + w) * D;
-                else src = c.ring_kv + (plane * c.ring_cap + (cur.si.recent_lo + (w - cur.si.n_sink)) % c.ring_cap) * D;
-                bulk_copy_g2s(dst + which * WIN_V_OFF + r * WIN_ROW, src, D * 2, bar);
-            }
-            bad_stage &= ~(1u << s);
-        }
-    };
-    for (int s = 0; s < STAGES && s < n_units; ++s) { issue(prod, s); advance(prod); }
-
-    // ---- per (sequence, KV head) segment state
     unsigned qf[8][2];
     float fmul[NH], gadd[NH];
     WarpState<MODE> st;
-    auto begin_segment = [&](const Cursor& cur) {
-        const long long bh = static_cast<long long>(cur.b) * c.n_kv + cur.h;
-        const uint4* src = P.qfrag + bh * 128;
-#pragma unroll
-        for (int s2 = 0; s2 < 4; ++s2) {
-            const uint4 v = __ldg(src + s2 * 32 + lane);
-            qf[2 * s2][0] = v.x; qf[2 * s2][1] = v.y; qf[2 * s2 + 1][0] = v.z; qf[2 * s2 + 1][1] = v.w;
-        }
-#pragma unroll
-        for (int k = 0; k < NH; ++k) {
-            const int head = MODE == 0 ? t : 2 * t + k;
-            fmul[k] = gadd[k] = 0.f;
-            if (head < G) {
-                const float2 v = __ldg(reinterpret_cast<const float2*>(P.qscal + (static_cast<long long>(cur.b) * c.n_q + cur.h * G + head) * 2));
-                fmul[k] = v.x; gadd[k] = v.y;
-            }
-        }
-        st.reset();
-    };
-    auto end_segment = [&](const Cursor& cur) {
-        const long long bh = static_cast<long long>(cur.b) * c.n_kv + cur.h;
-        store_partial<BITS, MODE>(st, P.part + (wg + bh) * G * PART_STRIDE, lane, G);
-    };
-    begin_segment(cons);
-
+    int stage = 0;                      // ring position of the next unit to consume (and to refill)
+    unsigned phase_bits = 0;            // parity of each stage's next completion
+    unsigned bad_bits = 0;              // lane 0: stages whose unit could not be fetched
     bool timed_out = false;
-    for (int it = 0; it < n_units; ++it) {
-        const int s = it % STAGES;
-        const unsigned parity = (it / STAGES) & 1;
-        // a phase that one lane saw complete is complete for all: keep the decision warp-uniform
-        if (!__any_sync(FULL, mbar_wait_bounded(bar0 + 8 * s, parity))) { timed_out = true; break; }
-        const unsigned rec = stage0 + s * REC;
-        if (cons.u >= cons.si.qp) {
-            // ======================= window unit: up to 8 bf16 tokens ==============================
-            const int w0 = (cons.u - cons.si.qp) * WIN_TOKENS;
-            const int n_valid = min(WIN_TOKENS, cons.si.n_win - w0);
-            const int r_eff = (lane & 7) < n_valid ? (lane & 7) : 0;      // rows beyond the valid ones alias row 0
-            const int mat = lane >> 3;
-            const unsigned frag_off = r_eff * WIN_ROW + ((mat >> 1) * 16 + (mat & 1) * 8) * 2;
-            const uint4* wsrc = P.qwfrag + (static_cast<long long>(cons.b) * c.n_kv + cons.h) * 256;
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int pass = 0; pass < (MODE == 0 ? 1 : 2); ++pass) {
-#pragma unroll
-                for (int s2 = 0; s2 < 4; ++s2) {
-                    const uint4 bq = __ldg(wsrc + pass * 128 + s2 * 32 + lane);
-                    unsigned k0, k1, k2, k3;                              // (step 2s2: ch lo, ch hi), (step 2s2+1: ch lo, ch hi)
-                    ldmatrix_x4(rec + frag_off + s2 * 64, k0, k1, k2, k3);
-                    mma_bf16(acc, k0, k0, k1, k1, bq.x, bq.y);            // token rows 8..15 alias rows 0..7
-                    mma_bf16(acc, k2, k2, k3, k3, bq.z, bq.w);
+
+    while (L < L1 && !timed_out) {
+        // ================= round set-up: list the next segments of the slice =====================
+        int n_seg = 0, round_units = 0;
+        while (n_seg < MAX_SEGMENTS && L < L1) {
+            const SeqInfo si = seq_info(c, __ldg(P.seq_len + sb), __ldg(P.slot + sb));
+            if (si.U > 0) {
+                const int u1 = static_cast<int>(min(static_cast<long long>(si.U), su + (L1 - L)));
+                if (lane == 0) {
+                    Segment sg;
+                    sg.b = sb; sg.h = sh; sg.slot = si.slot; sg.u0 = su; sg.u1 = u1; sg.qp = si.qp; sg.first_page = si.first_page;
+                    sg.q_lo = si.q_lo; sg.q_hi = si.q_hi; sg.n_win = si.n_win; sg.n_sink = si.n_sink; sg.recent_lo = si.recent_lo;
+                    segs[n_seg] = sg;
                 }
+                ++n_seg;
+                round_units += u1 - su;
+                L += u1 - su;
+                su = u1;
             }
-            const bool ok = g < n_valid;
-            float sc[NH], mx[NH], mref[NH];
-            if (MODE == 0) sc[0] = ok ? acc[0] + acc[1] : -INFINITY;
-            else { sc[0] = ok ? acc[0] : -INFINITY; sc[NH - 1] = ok ? acc[1] : -INFINITY; }
-#pragma unroll
-            for (int k = 0; k < NH; ++k) {
-                mx[k] = sc[k];
-                mx[k] = fmaxf(mx[k], __shfl_xor_sync(FULL, mx[k], 4));
-                mx[k] = fmaxf(mx[k], __shfl_xor_sync(FULL, mx[k], 8));
-                mx[k] = fmaxf(mx[k], __shfl_xor_sync(FULL, mx[k], 16));
-            }
-            st.raise_max(mx, mref);
-            float p[NH];
-#pragma unroll
-            for (int k = 0; k < NH; ++k) { p[k] = ex2(sc[k] - mref[k]); st.l[k] += p[k]; }
-#pragma unroll
-            for (int pass = 0; pass < (MODE == 0 ? 1 : 2); ++pass) {
-                unsigned pr;                                              // this token's probabilities in the score-fragment layout
-                if (MODE == 0) pr = pack_bf2(p[0], (p[0] - bf16_round(p[0])) * LO_SCALE);   // value column, remainder column
-                else if (pass == 0) pr = pack_bf2(p[0], p[NH - 1]);
-                else pr = pack_bf2(p[0] - bf16_round(p[0]), p[NH - 1] - bf16_round(p[NH - 1]));
-                const unsigned b01 = movmatrix_trans(pr);                 // tokens 2t, 2t+1 of column g; tokens 8..15 get zero
-#pragma unroll
-                for (int i2 = 0; i2 < 4; ++i2) {
-                    unsigned v0, v1, v2, v3;                              // (block 2i2: ch lo, ch hi), (block 2i2+1: ch lo, ch hi)
-                    ldmatrix_x4_trans(rec + WIN_V_OFF + frag_off + i2 * 64, v0, v1, v2, v3);
-                    // fold the block's accumulator unit in: p * v * PV_SCALE * 2^(shift - 24)
-                    mma_bf16(st.o[2 * i2], v0, v1, v0, v1, mul_bf2(b01, bf16x2_pow2(field_shift<BITS>(2 * i2) - 20)), 0u);
-                    mma_bf16(st.o[2 * i2 + 1], v2, v3, v2, v3, mul_bf2(b01, bf16x2_pow2(field_shift<BITS>(2 * i2 + 1) - 20)), 0u);
-                }
-            }
-        } else if (((bad_stage >> s) & 1u) == 0) {
-            // ======================= packed page: 64 quantized tokens ==============================
-            const int pos0 = (cons.si.first_page + cons.u) * PAGE_TOKENS;
-            const bool full_page = (pos0 >= cons.si.q_lo) && (pos0 + PAGE_TOKENS <= cons.si.q_hi);
-            float sc[4][2 * NH];          // [block][row g: heads..., row g+8: heads...]
-            unsigned vmeta[4][2];         // fp16x2 (Delta_v, x_min_v) of rows g, g+8
-#pragma unroll
-            for (int bi = 0; bi < 4; ++bi) {
-                float acc[4] = {0.f, 0.f, 0.f, 0.f}, acc2[4] = {0.f, 0.f, 0.f, 0.f};      // two chains for ILP
-                if (BITS == 2) {
-                    const uint4 kw = lds128(rec + bi * CB + 16 * lane);
-                    const unsigned sx = pre_shift<2>(kw.x), sy = pre_shift<2>(kw.y), sz = pre_shift<2>(kw.z), sw = pre_shift<2>(kw.w);
-#pragma unroll
-                    for (int ks = 0; ks < 8; ks += 2) {
-                        mma_f16(acc, field<2>(kw.x, sx, ks), field<2>(kw.z, sz, ks), field<2>(kw.y, sy, ks), field<2>(kw.w, sw, ks),
-                                qf[ks][0], qf[ks][1]);
-                        mma_f16(acc2, field<2>(kw.x, sx, ks + 1), field<2>(kw.z, sz, ks + 1), field<2>(kw.y, sy, ks + 1), field<2>(kw.w, sw, ks + 1),
-                                qf[ks + 1][0], qf[ks + 1][1]);
-                    }
-                } else {
-                    const uint4 ka = lds128(rec + bi * CB + 16 * lane);          // row g:   W0..W3
-                    const uint4 kb = lds128(rec + bi * CB + 512 + 16 * lane);    // row g+8: W0..W3
-                    const unsigned a0s = pre_shift<4>(ka.x), a1s = pre_shift<4>(ka.y), a2s = pre_shift<4>(ka.z), a3s = pre_shift<4>(ka.w);
-                    const unsigned b0s = pre_shift<4>(kb.x), b1s = pre_shift<4>(kb.y), b2s = pre_shift<4>(kb.z), b3s = pre_shift<4>(kb.w);
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        mma_f16(acc, field<4>(ka.x, a0s, ks), field<4>(kb.x, b0s, ks), field<4>(ka.y, a1s, ks), field<4>(kb.y, b1s, ks),
-                                qf[ks][0], qf[ks][1]);
-                        mma_f16(acc2, field<4>(ka.z, a2s, ks), field<4>(kb.z, b2s, ks), field<4>(ka.w, a3s, ks), field<4>(kb.w, b3s, ks),
-                                qf[4 + ks][0], qf[4 + ks][1]);
-                    }
-                }
-#pragma unroll
-                for (int e = 0; e < 4; ++e) acc[e] += acc2[e];
-                const uint4 mt = lds128(rec + meta_offset(BITS) + 128 * bi + 16 * g);   // rows g (x,y) and g+8 (z,w)
-                const float kd0 = h_lo(mt.x), km0 = h_hi(mt.x), kd1 = h_lo(mt.z), km1 = h_hi(mt.z);
-                unsigned vm0 = mt.y, vm1 = mt.w;
-                bool ok0 = true, ok1 = true;
-                if (!full_page) {
-                    const int p0 = pos0 + bi * 16 + g, p1 = p0 + 8;
-                    ok0 = (p0 >= cons.si.q_lo) && (p0 < cons.si.q_hi);
-                    ok1 = (p1 >= cons.si.q_lo) && (p1 < cons.si.q_hi);
-                    if (!ok0) vm0 = 0u;
-                    if (!ok1) vm1 = 0u;
-                }
-                vmeta[bi][0] = vm0; vmeta[bi][1] = vm1;
-                if (MODE == 0) {
-                    const float d0 = fmaf(acc[1], 1.f / LO_SCALE, acc[0]), d1 = fmaf(acc[3], 1.f / LO_SCALE, acc[2]);
-                    const float s0 = fmaf(d0 * kd0, fmul[0], km0 * gadd[0]);
-                    const float s1 = fmaf(d1 * kd1, fmul[0], km1 * gadd[0]);
-                    sc[bi][0] = ok0 ? s0 : -INFINITY;
-                    sc[bi][NH] = ok1 ? s1 : -INFINITY;
-                } else {
-                    const float s00 = fmaf(acc[0] * kd0, fmul[0], km0 * gadd[0]);
-                    const float s01 = fmaf(acc[1] * kd0, fmul[NH - 1], km0 * gadd[NH - 1]);
-                    const float s10 = fmaf(acc[2] * kd1, fmul[0], km1 * gadd[0]);
-                    const float s11 = fmaf(acc[3] * kd1, fmul[NH - 1], km1 * gadd[NH - 1]);
-                    sc[bi][0] = ok0 ? s00 : -INFINITY; sc[bi][NH - 1] = ok0 ? s01 : -INFINITY;
-                    sc[bi][NH] = ok1 ? s10 : -INFINITY; sc[bi][2 * NH - 1] = ok1 ? s11 : -INFINITY;
-                }
-            }
-            // ---------------- running maximum of the page, rescale if it grew
-            float mx[NH], mref[NH];
-#pragma unroll
-            for (int k = 0; k < NH; ++k) {
-                float v = fmaxf(fmaxf(fmaxf(sc[0][k], sc[0][NH + k]), fmaxf(sc[1][k], sc[1][NH + k])),
-                                fmaxf(fmaxf(sc[2][k], sc[2][NH + k]), fmaxf(sc[3][k], sc[3][NH + k])));
-                v = fmaxf(v, __shfl_xor_sync(FULL, v, 4));
-                v = fmaxf(v, __shfl_xor_sync(FULL, v, 8));
-                v = fmaxf(v, __shfl_xor_sync(FULL, v, 16));
-                mx[k] = v;
-            }
-            st.raise_max(mx, mref);
-            // ---------------- probabilities, value reduction
-#pragma unroll
-            for (int bi = 0; bi < 4; ++bi) {
-                const float vd0 = h_lo(vmeta[bi][0]) * PV_SCALE, vn0 = h_hi(vmeta[bi][0]);
-                const float vd1 = h_lo(vmeta[bi][1]) * PV_SCALE, vn1 = h_hi(vmeta[bi][1]);
-                unsigned r0, r1;
-                if (MODE == 0) {
-                    const float p0 = ex2(sc[bi][0] - mref[0]), p1 = ex2(sc[bi][NH] - mref[0]);
-                    st.l[0] += p0 + p1;
-                    st.z[0] = fmaf(p0, vn0, fmaf(p1, vn1, st.z[0]));
-                    r0 = pack_h2(p0 * vd0, 0.f);
-                    r1 = pack_h2(p1 * vd1, 0.f);
-                } else {
-                    const float p00 = ex2(sc[bi][0] - mref[0]), p01 = ex2(sc[bi][NH - 1] - mref[NH - 1]);
-                    const float p10 = ex2(sc[bi][NH] - mref[0]), p11 = ex2(sc[bi][2 * NH - 1] - mref[NH - 1]);
-                    st.l[0] += p00 + p10; st.l[NH - 1] += p01 + p11;
-                    st.z[0] = fmaf(p00, vn0, fmaf(p10, vn1, st.z[0]));
-                    st.z[NH - 1] = fmaf(p01, vn0, fmaf(p11, vn1, st.z[NH - 1]));
-                    r0 = pack_h2(p00 * vd0, p01 * vd0);
-                    r1 = pack_h2(p10 * vd1, p11 * vd1);
-                }
-                const unsigned b01 = movmatrix_trans(r0), b23 = movmatrix_trans(r1);
-                if (BITS == 2) {
-                    const uint4 vw = lds128(rec + v_codes_offset(2) + bi * CB + 16 * lane);
-                    const unsigned sx = pre_shift<2>(vw.x), sy = pre_shift<2>(vw.y), sz = pre_shift<2>(vw.z), sw = pre_shift<2>(vw.w);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        mma_f16(st.o[i], field<2>(vw.x, sx, i), field<2>(vw.y, sy, i), field<2>(vw.z, sz, i), field<2>(vw.w, sw, i), b01, b23);
-                } else {
-                    const uint4 va = lds128(rec + v_codes_offset(4) + bi * CB + 16 * lane);         // tokens 2t,2t+1
-                    const uint4 vb = lds128(rec + v_codes_offset(4) + bi * CB + 512 + 16 * lane);   // tokens 2t+8,2t+9
-                    const unsigned a0s = pre_shift<4>(va.x), a1s = pre_shift<4>(va.y), a2s = pre_shift<4>(va.z), a3s = pre_shift<4>(va.w);
-                    const unsigned b0s = pre_shift<4>(vb.x), b1s = pre_shift<4>(vb.y), b2s = pre_shift<4>(vb.z), b3s = pre_shift<4>(vb.w);
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)     // channel blocks 0..3: words (rsel, j=0)
-                        mma_f16(st.o[k], field<4>(va.x, a0s, k), field<4>(va.z, a2s, k), field<4>(vb.x, b0s, k), field<4>(vb.z, b2s, k), b01, b23);
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)     // channel blocks 4..7: words (rsel, j=1)
-                        mma_f16(st.o[4 + k], field<4>(va.y, a1s, k), field<4>(va.w, a3s, k), field<4>(vb.y, b1s, k), field<4>(vb.w, b3s, k), b01, b23);
-                }
+            if (si.U == 0 || su >= si.U) {              // next head, or next sequence
+                su = 0;
+                if (si.U == 0 || ++sh >= c.n_kv) { sh = 0; ++sb; }
+                if (sb >= P.batch) break;
             }
         }
         __syncwarp();
-        if (it + STAGES < n_units) { issue(prod, s); advance(prod); }
-        // ---- next unit; a change of (sequence, KV head) closes this warp's partial
-        if (it + 1 < n_units) {
-            const int pb = cons.b, ph = cons.h;
-            Cursor nxt = cons;
-            advance(nxt);
-            if (nxt.b != pb || nxt.h != ph) { end_segment(cons); begin_segment(nxt); }
-            cons = nxt;
+
+        // ================= producer: stages the units of this round, in order =====================
+        int p_seg = -1, p_u = 0, p_u1 = 0, p_qp = 0, p_head_off = 0, issued = 0;
+        const int* p_ptab = nullptr;
+        auto issue_next = [&](const int s) {            // whole warp; stages the round's next unit into ring slot s
+            if (p_u == p_u1) {                          // next segment
+                ++p_seg;
+                const Segment& sg = segs[p_seg];
+                p_u = sg.u0; p_u1 = sg.u1; p_qp = sg.qp; p_head_off = sg.h * REC;
+                p_ptab = c.page_table + static_cast<long long>(sg.slot) * c.max_pages + sg.first_page;
+                if (sg.first_page + sg.qp > c.max_pages) {      // the page table cannot hold this length
+                    if (lane == 0) atomicOr(c.dev_status, WUSHKV_DEV_PAGE_TABLE_FULL);
+                    p_qp = min(p_qp, max(c.max_pages - sg.first_page, 0));   // pages beyond it are treated as window-less gaps below
+                }
+            }
+            const unsigned bar = bar0 + 8 * s, dst = stage0 + s * REC;
+            const Segment& sg = segs[p_seg];
+            if (p_u < sg.qp) {                          // a packed page: one bulk copy
+                if (lane == 0) {
+                    const int page = (p_u < p_qp) ? __ldg(p_ptab + p_u) : -1;
+                    if (static_cast<unsigned>(page) >= static_cast<unsigned long long>(c.n_pages)) {
+                        if (p_u < p_qp) atomicOr(c.dev_status, WUSHKV_DEV_BAD_PAGE_ID);
+                        bad_bits |= 1u << s;
+                        mbar_arrive(bar);
+                    } else {
+                        bad_bits &= ~(1u << s);
+                        mbar_expect_tx(bar, REC);
+                        bulk_copy_g2s(dst, c.pages + page * page_row_bytes + p_head_off, REC, bar);
+                    }
+                }
+            } else {                                    // up to 8 window tokens: one 256-byte row copy per lane
+                const int w0 = (p_u - sg.qp) * WIN_TOKENS;
+                const int n_valid = min(WIN_TOKENS, sg.n_win - w0);
+                if (lane == 0) { bad_bits &= ~(1u << s); mbar_expect_tx(bar, n_valid * 2 * D * 2); }
+                __syncwarp();
+                const int r = lane & 7, which = lane >> 3;      // lanes 0-7: key rows, 8-15: value rows
+                if (lane < 16 && r < n_valid) {
+                    const int w = w0 + r;
+                    const long long plane = (static_cast<long long>(sg.slot) * c.n_kv + sg.h) * 2 + which;
+                    const unsigned short* src;
+                    if (w < sg.n_sink) src = c.sink_kv + (plane * c.s_sink + w) * D;
+                    else src = c.ring_kv + (plane * c.ring_cap + (sg.recent_lo + (w - sg.n_sink)) % c.ring_cap) * D;
+                    bulk_copy_g2s(dst + which * WIN_V_OFF + r * WIN_ROW, src, D * 2, bar);
+                }
+            }
+            ++p_u;
+            ++issued;
+        };
+        for (int k = 0; k < STAGES && k < round_units; ++k) issue_next((stage + k) % STAGES);
+
+        // ================= consumer ==============================================================
+        pdl_wait();                                     // query fragments come from the preparation kernel
+        for (int cs = 0; cs < n_seg && !timed_out; ++cs) {
+            const Segment& sg = segs[cs];               // rarely used fields are re-read from shared memory
+            const long long bh = static_cast<long long>(sg.b) * c.n_kv + sg.h;
+            const int u1 = sg.u1, qp = sg.qp, q_lo = sg.q_lo, q_hi = sg.q_hi;
+            int pos0 = (sg.first_page + sg.u0) * PAGE_TOKENS;
+            {   // query fragments and per-head scalars of this (sequence, KV head)
+                const uint4* src = P.qfrag + bh * 128;
+#pragma unroll
+                for (int s2 = 0; s2 < 4; ++s2) {
+                    const uint4 v = __ldg(src + s2 * 32 + lane);
+                    qf[2 * s2][0] = v.x; qf[2 * s2][1] = v.y; qf[2 * s2 + 1][0] = v.z; qf[2 * s2 + 1][1] = v.w;
+                }
+#pragma unroll
+                for (int k = 0; k < NH; ++k) {
+                    const int head = MODE == 0 ? t : 2 * t + k;
+                    fmul[k] = gadd[k] = 0.f;
+                    if (head < G) {
+                        const float2 v = __ldg(reinterpret_cast<const float2*>(P.qscal + (static_cast<long long>(sg.b) * c.n_q + sg.h * G + head) * 2));
+                        fmul[k] = v.x; gadd[k] = v.y;
+                    }
+                }
+                st.reset();
+            }
+            for (int u = sg.u0; u < u1; ++u, pos0 += PAGE_TOKENS) {
+                const int s = stage;
+                // a phase that one lane saw complete is complete for all: keep the decision warp-uniform
+                if (!__any_sync(FULL, mbar_wait_bounded(bar0 + 8 * s, (phase_bits >> s) & 1u))) { timed_out = true; break; }
+                phase_bits ^= 1u << s;
+                const unsigned rec = stage0 + s * REC;
+                if (u >= qp) {
+                    // ======================= window unit: up to 8 bf16 tokens ==========================
+                    const int w0 = (u - qp) * WIN_TOKENS;
+                    const int n_valid = min(WIN_TOKENS, sg.n_win - w0);
+                    const int r_eff = (lane & 7) < n_valid ? (lane & 7) : 0;      // rows beyond the valid ones alias row 0
+                    const int mat = lane >> 3;
+                    const unsigned frag_off = r_eff * WIN_ROW + ((mat >> 1) * 16 + (mat & 1) * 8) * 2;
+                    const uint4* wsrc = P.qwfrag + (static_cast<long long>(sg.b) * c.n_kv + sg.h) * 256;
+                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int pass = 0; pass < (MODE == 0 ? 1 : 2); ++pass) {
+#pragma unroll
+                        for (int s2 = 0; s2 < 4; ++s2) {
+                            const uint4 bq = __ldg(wsrc + pass * 128 + s2 * 32 + lane);
+                            unsigned k0, k1, k2, k3;                      // (step 2s2: ch lo, ch hi), (step 2s2+1: ch lo, ch hi)
+                            ldmatrix_x4(rec + frag_off + s2 * 64, k0, k1, k2, k3);
+                            mma_bf16(acc, k0, k0, k1, k1, bq.x, bq.y);    // token rows 8..15 alias rows 0..7
+                            mma_bf16(acc, k2, k2, k3, k3, bq.z, bq.w);
+                        }
+                    }
+                    const bool ok = g < n_valid;
+                    float sc[NH], mx[NH], mref[NH];
+                    if (MODE == 0) sc[0] = ok ? acc[0] + acc[1] : -INFINITY;
+                    else { sc[0] = ok ? acc[0] : -INFINITY; sc[NH - 1] = ok ? acc[1] : -INFINITY; }
+#pragma unroll
+                    for (int k = 0; k < NH; ++k) {
+                        mx[k] = sc[k];
+                        mx[k] = fmaxf(mx[k], __shfl_xor_sync(FULL, mx[k], 4));
+                        mx[k] = fmaxf(mx[k], __shfl_xor_sync(FULL, mx[k], 8));
+                        mx[k] = fmaxf(mx[k], __shfl_xor_sync(FULL, mx[k], 16));
+                    }
+                    st.raise_max(mx, mref);
+                    float p[NH];
+#pragma unroll
+                    for (int k = 0; k < NH; ++k) { p[k] = ex2(sc[k] - mref[k]); st.l[k] += p[k]; }
+#pragma unroll
+                    for (int pass = 0; pass < (MODE == 0 ? 1 : 2); ++pass) {
+                        unsigned pr;                                      // this token's probabilities in the score-fragment layout
+                        if (MODE == 0) pr = pack_bf2(p[0], (p[0] - bf16_round(p[0])) * LO_SCALE);   // value column, remainder column
+                        else if (pass == 0) pr = pack_bf2(p[0], p[NH - 1]);
+                        else pr = pack_bf2(p[0] - bf16_round(p[0]), p[NH - 1] - bf16_round(p[NH - 1]));
+                        const unsigned b01 = movmatrix_trans(pr);         // tokens 2t, 2t+1 of column g; tokens 8..15 get zero
+#pragma unroll
+                        for (int i2 = 0; i2 < 4; ++i2) {
+                            unsigned v0, v1, v2, v3;                      // (block 2i2: ch lo, ch hi), (block 2i2+1: ch lo, ch hi)
+                            ldmatrix_x4_trans(rec + WIN_V_OFF + frag_off + i2 * 64, v0, v1, v2, v3);
+                            // fold the block's accumulator unit in: p * v * PV_SCALE * 2^(shift - 24)
+                            mma_bf16(st.o[2 * i2], v0, v1, v0, v1, mul_bf2(b01, bf16x2_pow2(field_shift<BITS>(2 * i2) - 20)), 0u);
+                            mma_bf16(st.o[2 * i2 + 1], v2, v3, v2, v3, mul_bf2(b01, bf16x2_pow2(field_shift<BITS>(2 * i2 + 1) - 20)), 0u);
+                        }
+                    }
+                } else if (!__any_sync(FULL, (bad_bits >> s) & 1u)) {
+                    // ======================= packed page: 64 quantized tokens ==========================
+                    const bool full_page = (pos0 >= q_lo) && (pos0 + PAGE_TOKENS <= q_hi);
+                    float sc[4][2 * NH];          // [block][row g: heads..., row g+8: heads...]
+                    unsigned vmeta[4][2];         // fp16x2 (Delta_v, x_min_v) of rows g, g+8
+#pragma unroll
+                    for (int bi = 0; bi < 4; ++bi) {
+                        float acc[4] = {0.f, 0.f, 0.f, 0.f}, acc2[4] = {0.f, 0.f, 0.f, 0.f};      // two chains for ILP
+                        if (BITS == 2) {
+                            const uint4 kw = lds128(rec + bi * CB + 16 * lane);
+                            const unsigned sx = pre_shift<2>(kw.x), sy = pre_shift<2>(kw.y), sz = pre_shift<2>(kw.z), sw = pre_shift<2>(kw.w);
+#pragma unroll
+                            for (int ks = 0; ks < 8; ks += 2) {
+                                mma_f16(acc, field<2>(kw.x, sx, ks), field<2>(kw.z, sz, ks), field<2>(kw.y, sy, ks), field<2>(kw.w, sw, ks),
+                                        qf[ks][0], qf[ks][1]);
+                                mma_f16(acc2, field<2>(kw.x, sx, ks + 1), field<2>(kw.z, sz, ks + 1), field<2>(kw.y, sy, ks + 1), field<2>(kw.w, sw, ks + 1),
+                                        qf[ks + 1][0], qf[ks + 1][1]);
+                            }
+                        } else {
+                            const uint4 ka = lds128(rec + bi * CB + 16 * lane);          // row g:   W0..W3
+                            const uint4 kb = lds128(rec + bi * CB + 512 + 16 * lane);    // row g+8: W0..W3
+                            const unsigned a0s = pre_shift<4>(ka.x), a1s = pre_shift<4>(ka.y), a2s = pre_shift<4>(ka.z), a3s = pre_shift<4>(ka.w);
+                            const unsigned b0s = pre_shift<4>(kb.x), b1s = pre_shift<4>(kb.y), b2s = pre_shift<4>(kb.z), b3s = pre_shift<4>(kb.w);
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks) {
+                                mma_f16(acc, field<4>(ka.x, a0s, ks), field<4>(kb.x, b0s, ks), field<4>(ka.y, a1s, ks), field<4>(kb.y, b1s, ks),
+                                        qf[ks][0], qf[ks][1]);
+                                mma_f16(acc2, field<4>(ka.z, a2s, ks), field<4>(kb.z, b2s, ks), field<4>(ka.w, a3s, ks), field<4>(kb.w, b3s, ks),
+                                        qf[4 + ks][0], qf[4 + ks][1]);
+                            }
+                        }
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) acc[e] += acc2[e];
+                        const uint4 mt = lds128(rec + meta_offset(BITS) + 128 * bi + 16 * g);   // rows g (x,y) and g+8 (z,w)
+                        const float2 km_a = h2f2(mt.x), km_b = h2f2(mt.z);
+                        const float kd0 = km_a.x, km0 = km_a.y, kd1 = km_b.x, km1 = km_b.y;
+                        unsigned vm0 = mt.y, vm1 = mt.w;
+                        bool ok0 = true, ok1 = true;
+                        if (!full_page) {
+                            const int p0 = pos0 + bi * 16 + g, p1 = p0 + 8;
+                            ok0 = (p0 >= q_lo) && (p0 < q_hi);
+                            ok1 = (p1 >= q_lo) && (p1 < q_hi);
+                            if (!ok0) vm0 = 0u;
+                            if (!ok1) vm1 = 0u;
+                        }
+                        vmeta[bi][0] = vm0; vmeta[bi][1] = vm1;
+                        if (MODE == 0) {
+                            const float d0 = fmaf(acc[1], 1.f / LO_SCALE, acc[0]), d1 = fmaf(acc[3], 1.f / LO_SCALE, acc[2]);
+                            const float s0 = fmaf(d0 * kd0, fmul[0], km0 * gadd[0]);
+                            const float s1 = fmaf(d1 * kd1, fmul[0], km1 * gadd[0]);
+                            sc[bi][0] = ok0 ? s0 : -INFINITY;
+                            sc[bi][NH] = ok1 ? s1 : -INFINITY;
+                        } else {
+                            const float s00 = fmaf(acc[0] * kd0, fmul[0], km0 * gadd[0]);
+                            const float s01 = fmaf(acc[1] * kd0, fmul[NH - 1], km0 * gadd[NH - 1]);
+                            const float s10 = fmaf(acc[2] * kd1, fmul[0], km1 * gadd[0]);
+                            const float s11 = fmaf(acc[3] * kd1, fmul[NH - 1], km1 * gadd[NH - 1]);
+                            sc[bi][0] = ok0 ? s00 : -INFINITY; sc[bi][NH - 1] = ok0 ? s01 : -INFINITY;
+                            sc[bi][NH] = ok1 ? s10 : -INFINITY; sc[bi][2 * NH - 1] = ok1 ? s11 : -INFINITY;
+                        }
+                    }
+                    // ---------------- running maximum of the page, rescale if it grew
+                    float mx[NH], mref[NH];
+#pragma unroll
+                    for (int k = 0; k < NH; ++k) {
+                        float v = fmaxf(fmaxf(fmaxf(sc[0][k], sc[0][NH + k]), fmaxf(sc[1][k], sc[1][NH + k])),
+                                        fmaxf(fmaxf(sc[2][k], sc[2][NH + k]), fmaxf(sc[3][k], sc[3][NH + k])));
+                        v = fmaxf(v, __shfl_xor_sync(FULL, v, 4));
+                        v = fmaxf(v, __shfl_xor_sync(FULL, v, 8));
+                        v = fmaxf(v, __shfl_xor_sync(FULL, v, 16));
+                        mx[k] = v;
+                    }
+                    st.raise_max(mx, mref);
+                    // ---------------- probabilities, value reduction
+#pragma unroll
+                    for (int bi = 0; bi < 4; ++bi) {
+                        const float2 vm_a = h2f2(vmeta[bi][0]), vm_b = h2f2(vmeta[bi][1]);
+                        const float vd0 = vm_a.x * PV_SCALE, vn0 = vm_a.y, vd1 = vm_b.x * PV_SCALE, vn1 = vm_b.y;
+                        unsigned r0, r1;
+                        if (MODE == 0) {
+                            const float p0 = ex2(sc[bi][0] - mref[0]), p1 = ex2(sc[bi][NH] - mref[0]);
+                            st.l[0] += p0 + p1;
+                            st.z[0] = fmaf(p0, vn0, fmaf(p1, vn1, st.z[0]));
+                            r0 = pack_h2(p0 * vd0, 0.f);
+                            r1 = pack_h2(p1 * vd1, 0.f);
+                        } else {
+                            const float p00 = ex2(sc[bi][0] - mref[0]), p01 = ex2(sc[bi][NH - 1] - mref[NH - 1]);
+                            const float p10 = ex2(sc[bi][NH] - mref[0]), p11 = ex2(sc[bi][2 * NH - 1] - mref[NH - 1]);
+                            st.l[0] += p00 + p10; st.l[NH - 1] += p01 + p11;
+                            st.z[0] = fmaf(p00, vn0, fmaf(p10, vn1, st.z[0]));
+                            st.z[NH - 1] = fmaf(p01, vn0, fmaf(p11, vn1, st.z[NH - 1]));
+                            r0 = pack_h2(p00 * vd0, p01 * vd0);
+                            r1 = pack_h2(p10 * vd1, p11 * vd1);
+                        }
+                        const unsigned b01 = movmatrix_trans(r0), b23 = movmatrix_trans(r1);
+                        if (BITS == 2) {
+                            const uint4 vw = lds128(rec + v_codes_offset(2) + bi * CB + 16 * lane);
+                            const unsigned sx = pre_shift<2>(vw.x), sy = pre_shift<2>(vw.y), sz = pre_shift<2>(vw.z), sw = pre_shift<2>(vw.w);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                mma_f16(st.o[i], field<2>(vw.x, sx, i), field<2>(vw.y, sy, i), field<2>(vw.z, sz, i), field<2>(vw.w, sw, i), b01, b23);
+                        } else {
+                            const uint4 va = lds128(rec + v_codes_offset(4) + bi * CB + 16 * lane);         // tokens 2t,2t+1
+                            const uint4 vb = lds128(rec + v_codes_offset(4) + bi * CB + 512 + 16 * lane);   // tokens 2t+8,2t+9
+                            const unsigned a0s = pre_shift<4>(va.x), a1s = pre_shift<4>(va.y), a2s = pre_shift<4>(va.z), a3s = pre_shift<4>(va.w);
+                            const unsigned b0s = pre_shift<4>(vb.x), b1s = pre_shift<4>(vb.y), b2s = pre_shift<4>(vb.z), b3s = pre_shift<4>(vb.w);
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)     // channel blocks 0..3: words (rsel, j=0)
+                                mma_f16(st.o[k], field<4>(va.x, a0s, k), field<4>(va.z, a2s, k), field<4>(vb.x, b0s, k), field<4>(vb.z, b2s, k), b01, b23);
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)     // channel blocks 4..7: words (rsel, j=1)
+                                mma_f16(st.o[4 + k], field<4>(va.y, a1s, k), field<4>(va.w, a3s, k), field<4>(vb.y, b1s, k), field<4>(vb.w, b3s, k), b01, b23);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (issued < round_units) issue_next(s);         // refill the stage just consumed
+                stage = (stage + 1 == STAGES) ? 0 : stage + 1;
+            }
+            store_partial<BITS, MODE>(st, P.part + (wg + static_cast<long long>(sg.b) * c.n_kv + sg.h) * G * PART_STRIDE, lane, G);
         }
+        __syncwarp();
     }
     if (timed_out) {
         if (lane == 0) atomicOr(c.dev_status, WUSHKV_DEV_COPY_TIMEOUT);
         // give copies that may still be in flight a bounded time to land before the CTA's memory is released
         for (int k = 0; k < 1000; ++k) __nanosleep(1000);
     }
-    end_segment(cons);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -718,6 +791,7 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, 4) decode_main_kernel(DecodeP
 __global__ void __launch_bounds__(128) decode_combine_kernel(DecodeParams P) {
     const CacheView& c = P.c;
     const int j = blockIdx.x, b = blockIdx.y, ch = threadIdx.x;
+    pdl_wait();                                         // partials come from the main kernel
     float* out = P.O + (static_cast<long long>(b) * c.n_q + j) * D;
     const long long U = P.plan[b + 1] - P.plan[b];
     const long long total = P.plan[P.batch] * c.n_kv;
@@ -789,17 +863,29 @@ static cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
 template <int BITS, int MODE>
 static int launch_decode(const DecodeParams& P, int n_ctas, cudaStream_t st) {
     constexpr int STAGES = 3;
-    constexpr size_t SMEM = static_cast<size_t>(MAIN_WARPS) * STAGES * record_bytes(BITS) + MAIN_WARPS * STAGES * 8;
+    constexpr size_t SMEM = static_cast<size_t>(MAIN_WARPS) * STAGES * record_bytes(BITS) + MAIN_WARPS * STAGES * 8 +
+                            MAIN_WARPS * MAX_SEGMENTS * sizeof(Segment);
     decode_prep_kernel<BITS, MODE><<<dim3(P.c.n_kv, P.batch), 128, 0, st>>>(P);
     if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
     if (cudaFuncSetAttribute(decode_main_kernel<BITS, MODE, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(SMEM)) != cudaSuccess)
         return WUSHKV_ECUDA;
+    cudaLaunchAttribute pdl_attr[1];
+    pdl_attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pdl_attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.stream = st;
+    cfg.attrs = pdl_attr;
+    cfg.numAttrs = 1;
     if (g_prof_start) cudaEventRecord(g_prof_start, st);
-    decode_main_kernel<BITS, MODE, STAGES><<<n_ctas, MAIN_WARPS * 32, SMEM, st>>>(P);
-    if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
+    cfg.gridDim = dim3(n_ctas);
+    cfg.blockDim = dim3(MAIN_WARPS * 32);
+    cfg.dynamicSmemBytes = SMEM;
+    if (cudaLaunchKernelEx(&cfg, decode_main_kernel<BITS, MODE, STAGES>, P) != cudaSuccess) return WUSHKV_ECUDA;
     if (g_prof_stop) cudaEventRecord(g_prof_stop, st);
-    decode_combine_kernel<<<dim3(P.c.n_q, P.batch), 128, 0, st>>>(P);
-    if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
+    cfg.gridDim = dim3(P.c.n_q, P.batch);
+    cfg.blockDim = dim3(128);
+    cfg.dynamicSmemBytes = 0;
+    if (cudaLaunchKernelEx(&cfg, decode_combine_kernel, P) != cudaSuccess) return WUSHKV_ECUDA;
     return WUSHKV_OK;
 }
 
