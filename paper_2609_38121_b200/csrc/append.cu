@@ -28,7 +28,7 @@ struct AppendParams {
     CacheView c;
     int batch, total_new, tokens_per_cta;
     const int* slot;
-    const int* seq_len;
+    int* seq_len;
     const int* cu_new;
     const unsigned short* K_new;
     const unsigned short* V_new;
@@ -240,6 +240,82 @@ __global__ void __launch_bounds__(256) append_rows_kernel(AppendParams P) {
     }
 }
 
+// Decode-time append: exactly one new token per sequence (or none).  One CTA per sequence handles
+// all KV heads: every thread computes outputs of k' = T_K k as a row dot product (the rows of T_K
+// come straight from L2), then one warp per vector quantizes and packs keys and values.  The CTA
+// is the only reader of its sequence's length, so it also advances it: no second launch.
+template <int BITS>
+__global__ void __launch_bounds__(1024) append_token_kernel(AppendParams P) {
+    extern __shared__ __align__(16) float tok_s[];       // [n_kv][128] input key, [n_kv][128] transformed key
+    const int b = blockIdx.x;
+    const int n_kv = P.c.n_kv;
+    float* kin_s = tok_s;
+    float* kp_s = tok_s + n_kv * D;
+    const int first = __ldg(P.cu_new + b), n_new = __ldg(P.cu_new + b + 1) - first;
+    if (n_new <= 0) return;
+    const int s0 = __ldg(P.seq_len + b);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const long long row0 = static_cast<long long>(first) * n_kv * D;
+    for (int idx = threadIdx.x; idx < n_kv * D; idx += blockDim.x) kin_s[idx] = bf16_bits_to_float(__ldg(P.K_new + row0 + idx));
+    __syncthreads();
+    // k'[h][i] = sum_j T[h][i][j] k[h][j]: a warp takes 32 consecutive rows of one head; every row is
+    // read as one coalesced 512-byte line (lane L holds columns 4L..4L+3), the 32 partial sums per lane
+    // are then reduced across lanes with a transposing butterfly.
+    for (int task = warp; task < n_kv * 4; task += nwarps) {
+        const int h = task >> 2, r0 = (task & 3) * 32;
+        const float4 kv = *reinterpret_cast<const float4*>(kin_s + h * D + 4 * lane);
+        const float4* Tbase = reinterpret_cast<const float4*>(P.c.T_K + (static_cast<long long>(h) * D + r0) * D) + lane;
+        float part[32];
+#pragma unroll
+        for (int r = 0; r < 32; ++r) {
+            const float4 t = __ldg(Tbase + r * (D / 4));
+            part[r] = fmaf(t.x, kv.x, fmaf(t.y, kv.y, fmaf(t.z, kv.z, t.w * kv.w)));
+        }
+        kp_s[h * D + r0 + lane] = warp_transpose_reduce(part, lane);
+    }
+    __syncthreads();
+    TokenSlot ts;
+    ts.b = b; ts.slot = __ldg(P.slot + b); ts.pos = s0; ts.s_final = s0 + 1;
+    bool ok = true;
+    if (ts.slot < 0 || ts.slot >= P.c.n_slots || s0 < 0) { if (threadIdx.x == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_SLOT); ok = false; }
+    int page = -1;
+    if (ok) {
+        const int pidx = ts.pos / PAGE_TOKENS;
+        if (pidx >= P.c.max_pages) { if (threadIdx.x == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_PAGE_TABLE_FULL); ok = false; }
+        else {
+            page = __ldg(P.c.page_table + static_cast<long long>(ts.slot) * P.c.max_pages + pidx);
+            if (page < 0 || page >= P.c.n_pages) { if (threadIdx.x == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_PAGE_ID); ok = false; }
+        }
+    }
+    if (ok) {
+        ts.r = ts.pos % PAGE_TOKENS;
+        for (int v = warp; v < 2 * n_kv; v += nwarps) {
+            const int which = v >= n_kv ? 1 : 0, head = which ? v - n_kv : v;
+            ts.rec = P.c.pages + (static_cast<long long>(page) * n_kv + head) * record_bytes(BITS);
+            float x[4];
+            uint2 copy;
+            if (which == 0) {
+                const float4 kp = *reinterpret_cast<const float4*>(kp_s + head * D + 4 * lane);
+                x[0] = kp.x; x[1] = kp.y; x[2] = kp.z; x[3] = kp.w;
+                copy.x = float_to_bf16_bits(x[0]) | (static_cast<unsigned>(float_to_bf16_bits(x[1])) << 16);
+                copy.y = float_to_bf16_bits(x[2]) | (static_cast<unsigned>(float_to_bf16_bits(x[3])) << 16);
+            } else {
+                copy = __ldg(reinterpret_cast<const uint2*>(P.V_new + row0 + head * D) + lane);
+                x[0] = bf16_bits_to_float(copy.x & 0xffff); x[1] = bf16_bits_to_float(copy.x >> 16);
+                x[2] = bf16_bits_to_float(copy.y & 0xffff); x[3] = bf16_bits_to_float(copy.y >> 16);
+            }
+            int code[4];
+            __half step_h, xmin_h;
+            quantize_vec<BITS>(x, which ? P.rule_v : P.rule_k, lane, code, step_h, xmin_h);
+            if (which == 0) store_k_codes<BITS>(ts.rec, ts.r, code, lane); else store_v_codes<BITS>(ts.rec, ts.r, code, lane);
+            __half* meta = reinterpret_cast<__half*>(ts.rec + meta_location(BITS, ts.r));
+            if (lane == 0) { meta[2 * which] = step_h; meta[2 * which + 1] = xmin_h; }
+            store_window_copy(P, ts, head, which, copy, lane);
+        }
+    }
+    if (threadIdx.x == 0) P.seq_len[b] = s0 + 1;          // every read of the old length happened before the barriers above
+}
+
 __global__ void advance_len_kernel(int batch, int* seq_len, const int* cu_new) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b < batch) seq_len[b] += cu_new[b + 1] - cu_new[b];
@@ -296,6 +372,14 @@ extern "C" int wushkv_append(const wushkv_cache* cache, int32_t batch, const int
     P.K_new = K_new; P.V_new = V_new;
     P.rule_k = make_rule(cache->kappa_k);
     P.rule_v = make_rule(cache->kappa_v);
+    if (max_new == 1) {                 // decode-time append: one CTA per sequence, single launch
+        const int threads = std::min(1024, P.c.n_kv * D);
+        const size_t smem1 = static_cast<size_t>(2) * P.c.n_kv * D * sizeof(float);
+        if (smem1 > 48 * 1024) return WUSHKV_EINVAL;
+        if (P.c.bits == 2) append_token_kernel<2><<<batch, threads, smem1, st>>>(P);
+        else append_token_kernel<4><<<batch, threads, smem1, st>>>(P);
+        return cudaGetLastError() == cudaSuccess ? WUSHKV_OK : WUSHKV_ECUDA;
+    }
     // enough CTAs to fill the machine, but at least 8 tokens each to amortise the transform load
     const int want_ctas = std::max(1, 2 * sm_count() / P.c.n_kv);
     int tpc = (total_new + want_ctas - 1) / want_ctas;

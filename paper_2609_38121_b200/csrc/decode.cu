@@ -146,22 +146,40 @@ __global__ void __launch_bounds__(128) decode_prep_kernel(DecodeParams P) {
     for (int g = 0; g < G; ++g)
         q_s[g][i] = bf16_bits_to_float(P.Q[(static_cast<long long>(b) * P.c.n_q + h * G + g) * D + i]);
     __syncthreads();
-    float acc[8];
+    // q'[g][i] = sum_j T_invT[h][i][j] q[g][j].  Each warp takes 32 rows; a row is one coalesced
+    // 512-byte read (lane L holds columns 4L..4L+3); rows are handled 32/GP at a time so that the
+    // GP x rows partial sums fit a 32-value transposing butterfly (GP = 4 or 8 head slots).
+    __shared__ float qp_s[8][D];
+    {
+        constexpr int GP = MODE == 0 ? 4 : 8;           // MODE 0 serves G <= 4, MODE 1 serves G <= 8
+        constexpr int rows_per = 32 / GP;
+        const float4* Tbase = reinterpret_cast<const float4*>(P.c.T_K_invT + (static_cast<long long>(h) * D + warp * 32) * D) + lane;
+        float4 qv[8];
 #pragma unroll
-    for (int g = 0; g < 8; ++g) acc[g] = 0.f;
-    const float4* Trow = reinterpret_cast<const float4*>(P.c.T_K_invT + (static_cast<long long>(h) * D + i) * D);
-#pragma unroll 8
-    for (int j4 = 0; j4 < D / 4; ++j4) {
-        const float4 t = __ldg(Trow + j4);
+        for (int g = 0; g < 8; ++g) qv[g] = g < G ? *reinterpret_cast<const float4*>(&q_s[g][4 * lane]) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int r0 = 0; r0 < 32; r0 += rows_per) {
+            float part[32];
 #pragma unroll
-        for (int g = 0; g < 8; ++g) {
-            if (g < G) {
-                const float4 qv = *reinterpret_cast<const float4*>(&q_s[g][4 * j4]);
-                acc[g] = fmaf(t.x, qv.x, acc[g]); acc[g] = fmaf(t.y, qv.y, acc[g]);
-                acc[g] = fmaf(t.z, qv.z, acc[g]); acc[g] = fmaf(t.w, qv.w, acc[g]);
+            for (int k = 0; k < 32; ++k) part[k] = 0.f;
+#pragma unroll
+            for (int rr = 0; rr < 32; ++rr) {            // slot k = rr * GP + g for rr < rows_per
+                if (rr < rows_per) {
+                    const float4 t = __ldg(Tbase + (r0 + rr) * (D / 4));
+#pragma unroll
+                    for (int g = 0; g < 8; ++g)
+                        if (g < GP && rr * GP + g < 32)
+                            part[(rr * GP + g) & 31] = fmaf(t.x, qv[g].x, fmaf(t.y, qv[g].y, fmaf(t.z, qv[g].z, t.w * qv[g].w)));
+                }
             }
+            const float tot = warp_transpose_reduce(part, lane);
+            const int rr = lane / GP, g = lane % GP;
+            if (g < G) qp_s[g][warp * 32 + r0 + rr] = tot;
         }
     }
+    __syncthreads();
+    float acc[8];
+#pragma unroll
+    for (int g = 0; g < 8; ++g) acc[g] = g < G ? qp_s[g][i] : 0.f;
     const int s = i >> 4;
     const float pos_scale = exp2f(-static_cast<float>(field_shift<BITS>(s)));
     const float k2 = P.c.sm_scale * LOG2E;
@@ -788,10 +806,12 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, 4) decode_main_kernel(DecodeP
 // ------------------------------------------------------------------------------------------------
 // 3. combine
 // ------------------------------------------------------------------------------------------------
+// One CTA per (sequence, query head), one thread per channel.  The partials sit in L2, so the cost is
+// load latency: the loads of 8 partials are issued together before they are merged.
 __global__ void __launch_bounds__(128) decode_combine_kernel(DecodeParams P) {
     const CacheView& c = P.c;
     const int j = blockIdx.x, b = blockIdx.y, ch = threadIdx.x;
-    pdl_wait();                                         // partials come from the main kernel
+    pdl_wait();                                         // partials and the plan come from the earlier kernels
     float* out = P.O + (static_cast<long long>(b) * c.n_q + j) * D;
     const long long U = P.plan[b + 1] - P.plan[b];
     const long long total = P.plan[P.batch] * c.n_kv;
@@ -799,26 +819,42 @@ __global__ void __launch_bounds__(128) decode_combine_kernel(DecodeParams P) {
     const int h = j / c.G, head = j % c.G;
     const long long La = P.plan[b] * c.n_kv + static_cast<long long>(h) * U, Lb = La + U;      // units [La, Lb)
     const long long nw = P.n_warps;
-    const long long w_first = ((La + 1) * nw - 1) / total, w_last = (Lb * nw - 1) / total;     // owners of La and Lb-1
+    // warp w owns units [floor(w total / nw), floor((w+1) total / nw)); owners of La and Lb-1:
+    const long long w_first = ((La + 1) * nw - 1) / total, w_last = (Lb * nw - 1) / total;
     const long long bh = static_cast<long long>(b) * c.n_kv + h;
     const float* base = P.part + ((w_first + bh) * c.G + head) * PART_STRIDE;
     const long long stride = static_cast<long long>(c.G) * PART_STRIDE;
     const int n = static_cast<int>(w_last - w_first + 1);
-    float m = -INFINITY;
-    for (int s = 0; s < n; ++s) {
-        const long long w = w_first + s;
-        const long long lo = max(w * total / nw, La), hi = min((w + 1) * total / nw, Lb);
-        if (lo < hi) m = fmaxf(m, base[s * stride]);
-    }
-    float l = 0.f, o = 0.f;
-    for (int s = 0; s < n; ++s) {
-        const long long w = w_first + s;
-        const long long lo = max(w * total / nw, La), hi = min((w + 1) * total / nw, Lb);
-        if (lo >= hi) continue;                       // a warp with an empty slice wrote nothing
-        const float* p = base + s * stride;
-        const float scl = (p[0] == -INFINITY) ? 0.f : exp2f(p[0] - m);
-        l += scl * p[1];
-        o += scl * p[4 + ch];
+    // slice bounds advance by q = total / nw with a carry of r = total % nw (no division in the loop)
+    const long long q = total / nw, r = total % nw;
+    long long lo_w = w_first * total / nw, rem = (w_first * total) % nw;
+    float m = -INFINITY, l = 0.f, o = 0.f;
+    for (int s0 = 0; s0 < n; s0 += 8) {
+        float pm[8], pl[8], po[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            pm[k] = -INFINITY; pl[k] = 0.f; po[k] = 0.f;
+            if (s0 + k < n) {
+                long long hi_w = lo_w + q;
+                rem += r;
+                if (rem >= nw) { rem -= nw; ++hi_w; }
+                const bool wrote = max(lo_w, La) < min(hi_w, Lb);     // a warp with an empty slice wrote nothing
+                lo_w = hi_w;
+                if (wrote) {
+                    const float* p = base + (s0 + k) * stride;
+                    pm[k] = __ldcg(p); pl[k] = __ldcg(p + 1); po[k] = __ldcg(p + 4 + ch);
+                }
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            if (pm[k] == -INFINITY) continue;
+            const float mn = fmaxf(m, pm[k]);
+            const float sa = exp2f(m - mn), sb = exp2f(pm[k] - mn);   // m = -inf on the first partial: sa = 0
+            l = l * sa + pl[k] * sb;
+            o = o * sa + po[k] * sb;
+            m = mn;
+        }
     }
     out[ch] = l > 0.f ? o / l : 0.f;
 }

@@ -106,4 +106,20 @@ __device__ __forceinline__ unsigned short float_to_bf16_bits(float x) {   // rou
     return static_cast<unsigned short>(u >> 16);
 }
 
+// Sum v[i] over the 32 lanes of a warp for i = 0..31 at once: on return lane L holds the total of
+// v[L] in v[0].  31 shuffles instead of 32 x 5 (a butterfly that halves the live values each step).
+__device__ __forceinline__ float warp_transpose_reduce(float (&v)[32], int lane) {
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        const bool upper = (lane & off) != 0;
+#pragma unroll
+        for (int i = 0; i < off; ++i) {
+            const float send = upper ? v[i] : v[i + off];
+            const float keep = upper ? v[i + off] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+        }
+    }
+    return v[0];
+}
+
 }  // namespace wushkv
