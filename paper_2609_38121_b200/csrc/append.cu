@@ -9,7 +9,9 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cmath>
+#include <cstdlib>
 
 #include "host_common.h"
 #include "layout.cuh"
@@ -316,6 +318,196 @@ __global__ void __launch_bounds__(1024) append_token_kernel(AppendParams P) {
     if (threadIdx.x == 0) P.seq_len[b] = s0 + 1;          // every read of the old length happened before the barriers above
 }
 
+// ------------------------------------------------------------------------------------------------
+// Chunk (prefill) append: the key transform K' = K T_K^T of 128 tokens x one KV head is ONE
+// tcgen05 tile: A = the 128 x 128 bf16 key tile, B = T_K (bf16, [out][in] is already the K-major B
+// operand), D = 128 x 128 fp32 in tensor memory (lane = token, column = output channel).  bf16 x bf16
+// products are exact in fp32, so the result differs from the CUDA-core paths only by summation order.
+// A CTA keeps its head's T_K resident in shared memory and walks over token tiles; while the tensor
+// core works on the keys, the warps quantize the tile's values; the fp32 keys then come back through
+// tcgen05.ld into shared memory and take the same warp-per-vector quantizer.
+//
+// Shared-memory operand layout (no swizzle, K-major "interleaved"): the tile is cut into core matrices
+// of 8 rows x 16 bytes (8 bf16) stored as 128 contiguous bytes; core matrix (row group rg, k chunk kc)
+// sits at rg * SBO + kc * LBO with LBO = 128 B and SBO = 2048 B.  One MMA consumes K = 16, i.e. two
+// k chunks, so the descriptor start address advances by 256 B per k-step.
+// ------------------------------------------------------------------------------------------------
+constexpr int TC_TILE = 128;                 // tokens per tile (MMA M)
+constexpr int TC_LBO = 128, TC_SBO = 2048;   // bytes
+constexpr int TC_X_PITCH = 132;              // floats per row of the fp32 key tile in shared memory
+constexpr int TC_THREADS = 512;
+constexpr int TC_SMEM_B = 32768;                                   // T_K as bf16 operand
+constexpr int TC_SMEM_X = TC_TILE * TC_X_PITCH * 4;                // fp32 keys; its first 32 KB double as the A operand
+constexpr int TC_SMEM_TOTAL = TC_SMEM_B + TC_SMEM_X + 64;
+
+__device__ __forceinline__ unsigned long long umma_smem_desc(unsigned smem_addr) {
+    unsigned long long d = 0;
+    d |= static_cast<unsigned long long>((smem_addr >> 4) & 0x3FFFu);            // start address
+    d |= static_cast<unsigned long long>((TC_LBO >> 4) & 0x3FFFu) << 16;         // leading (k chunk) byte offset
+    d |= static_cast<unsigned long long>((TC_SBO >> 4) & 0x3FFFu) << 32;         // stride (row group) byte offset
+    d |= 1ull << 46;                                                             // descriptor version of sm_100
+    return d;                                                                    // base offset 0, no swizzle
+}
+// kind::f16 instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 128
+constexpr unsigned UMMA_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+
+__device__ __forceinline__ unsigned smem_addr_u32(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
+
+template <int BITS>
+__global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParams P) {
+    extern __shared__ __align__(1024) unsigned char tc_smem[];
+    unsigned char* sB = tc_smem;
+    unsigned char* sA = tc_smem + TC_SMEM_B;                         // A operand, later overwritten by the fp32 tile
+    float* sX = reinterpret_cast<float*>(tc_smem + TC_SMEM_B);
+    unsigned long long* mbar = reinterpret_cast<unsigned long long*>(tc_smem + TC_SMEM_B + TC_SMEM_X);
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(tc_smem + TC_SMEM_B + TC_SMEM_X + 16);
+    const int head = blockIdx.y;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_tiles = (P.total_new + TC_TILE - 1) / TC_TILE;
+
+    // ---- one-time set-up: tensor memory, barrier, T_K as bf16 operand
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr_u32(tmem_slot)), "r"(128u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr_u32(mbar)) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    {
+        const float* T = P.c.T_K + static_cast<long long>(head) * D * D;
+        const int r8 = lane & 7, cq = lane >> 3;
+        for (int item = warp; item < 64; item += TC_THREADS / 32) {     // 16 row groups x 4 groups of 4 k chunks
+            const int rg = item >> 2, kc = (item & 3) * 4 + cq;
+            const float4* src = reinterpret_cast<const float4*>(T + (rg * 8 + r8) * D + kc * 8);
+            const float4 a = __ldg(src), b = __ldg(src + 1);
+            uint4 v;
+            v.x = float_to_bf16_bits(a.x) | (static_cast<unsigned>(float_to_bf16_bits(a.y)) << 16);
+            v.y = float_to_bf16_bits(a.z) | (static_cast<unsigned>(float_to_bf16_bits(a.w)) << 16);
+            v.z = float_to_bf16_bits(b.x) | (static_cast<unsigned>(float_to_bf16_bits(b.y)) << 16);
+            v.w = float_to_bf16_bits(b.z) | (static_cast<unsigned>(float_to_bf16_bits(b.w)) << 16);
+            *reinterpret_cast<uint4*>(sB + rg * TC_SBO + kc * TC_LBO + r8 * 16) = v;
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const unsigned tmem_base = *tmem_slot;
+    unsigned phase = 0;
+    bool failed = false;
+
+    for (int tile = blockIdx.x; tile < n_tiles && !failed; tile += gridDim.x) {
+        const int tok0 = tile * TC_TILE;
+        // ---- A operand: key rows of this tile (zero rows past the end of the batch)
+        {
+            const int r8 = lane & 7, cq = lane >> 3;
+            for (int item = warp; item < 64; item += TC_THREADS / 32) {
+                const int rg = item >> 2, kc = (item & 3) * 4 + cq;
+                const int tok = tok0 + rg * 8 + r8;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (tok < P.total_new) v = __ldg(reinterpret_cast<const uint4*>(P.K_new + (static_cast<long long>(tok) * P.c.n_kv + head) * D + kc * 8));
+                *reinterpret_cast<uint4*>(sA + rg * TC_SBO + kc * TC_LBO + r8 * 16) = v;
+            }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // generic-proxy writes -> visible to the tensor core
+        __syncthreads();
+        // ---- one thread issues the 8 k-steps and commits them to the barrier
+        if (tid == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const unsigned long long adesc = umma_smem_desc(smem_addr_u32(sA)), bdesc = umma_smem_desc(smem_addr_u32(sB));
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const unsigned accumulate = ks > 0 ? 1u : 0u;
+                asm volatile(
+                    "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                    "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+                    ::"r"(tmem_base), "l"(adesc + static_cast<unsigned long long>(ks * 2 * TC_LBO >> 4)),
+                      "l"(bdesc + static_cast<unsigned long long>(ks * 2 * TC_LBO >> 4)), "r"(UMMA_IDESC), "r"(accumulate),
+                      "r"(0u), "r"(0u), "r"(0u), "r"(0u) : "memory");
+            }
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr_u32(mbar)) : "memory");
+        }
+        // ---- while the tensor core runs: values of this tile (no transform)
+        for (int v = warp; v < TC_TILE; v += TC_THREADS / 32) {
+            const int token = tok0 + v;
+            if (token >= P.total_new) break;
+            TokenSlot ts;
+            if (!locate_token(P, token, head, ts)) continue;
+            const uint2 vraw = __ldg(reinterpret_cast<const uint2*>(P.V_new + (static_cast<long long>(token) * P.c.n_kv + head) * D) + lane);
+            float x[4] = {bf16_bits_to_float(vraw.x & 0xffff), bf16_bits_to_float(vraw.x >> 16),
+                          bf16_bits_to_float(vraw.y & 0xffff), bf16_bits_to_float(vraw.y >> 16)};
+            int code[4];
+            __half step_h, xmin_h;
+            quantize_vec<BITS>(x, P.rule_v, lane, code, step_h, xmin_h);
+            store_v_codes<BITS>(ts.rec, ts.r, code, lane);
+            __half* meta = reinterpret_cast<__half*>(ts.rec + meta_location(BITS, ts.r));
+            if (lane == 0) { meta[2] = step_h; meta[3] = xmin_h; }
+            store_window_copy(P, ts, head, 1, vraw, lane);
+        }
+        // ---- wait for the MMAs (bounded), then tensor memory -> shared memory
+        {
+            bool done = false;
+            for (int it = 0; it < (1 << 20) && !done; ++it) {
+                unsigned ok;
+                asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                             : "=r"(ok) : "r"(smem_addr_u32(mbar)), "r"(phase), "r"(2000u) : "memory");
+                done = ok != 0;
+            }
+            if (!__syncthreads_and(done ? 1 : 0)) {          // uniform decision for the whole CTA
+                if (tid == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_COPY_TIMEOUT);
+                failed = true;
+                break;
+            }
+            phase ^= 1u;
+        }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        {
+            const int q = warp & 3, cg = warp >> 2;          // lane quadrant of this warp, 32-column group
+            unsigned r[32];
+            const unsigned taddr = tmem_base + (static_cast<unsigned>(q * 32) << 16) + static_cast<unsigned>(cg * 32);
+            asm volatile(
+                "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                  "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                  "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                  "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                : "r"(taddr) : "memory");
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            float* dst = sX + (q * 32 + lane) * TC_X_PITCH + cg * 32;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<uint4*>(dst + 4 * j) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        // ---- keys of this tile: quantize the fp32 rows
+        for (int v = warp; v < TC_TILE; v += TC_THREADS / 32) {
+            const int token = tok0 + v;
+            if (token >= P.total_new) break;
+            TokenSlot ts;
+            if (!locate_token(P, token, head, ts)) continue;
+            const float4 kp = *reinterpret_cast<const float4*>(sX + v * TC_X_PITCH + 4 * lane);
+            float x[4] = {kp.x, kp.y, kp.z, kp.w};
+            int code[4];
+            __half step_h, xmin_h;
+            quantize_vec<BITS>(x, P.rule_k, lane, code, step_h, xmin_h);
+            store_k_codes<BITS>(ts.rec, ts.r, code, lane);
+            __half* meta = reinterpret_cast<__half*>(ts.rec + meta_location(BITS, ts.r));
+            if (lane == 0) { meta[0] = step_h; meta[1] = xmin_h; }
+            uint2 kb;
+            kb.x = float_to_bf16_bits(x[0]) | (static_cast<unsigned>(float_to_bf16_bits(x[1])) << 16);
+            kb.y = float_to_bf16_bits(x[2]) | (static_cast<unsigned>(float_to_bf16_bits(x[3])) << 16);
+            store_window_copy(P, ts, head, 0, kb, lane);
+        }
+        __syncthreads();                                      // the fp32 tile becomes the next A operand
+    }
+    // ---- release tensor memory (also after a timeout: nothing of this CTA is in flight any more or ever will complete)
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(128u) : "memory");
+}
+
 __global__ void advance_len_kernel(int batch, int* seq_len, const int* cu_new) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b < batch) seq_len[b] += cu_new[b + 1] - cu_new[b];
@@ -378,6 +570,26 @@ extern "C" int wushkv_append(const wushkv_cache* cache, int32_t batch, const int
         if (smem1 > 48 * 1024) return WUSHKV_EINVAL;
         if (P.c.bits == 2) append_token_kernel<2><<<batch, threads, smem1, st>>>(P);
         else append_token_kernel<4><<<batch, threads, smem1, st>>>(P);
+        return cudaGetLastError() == cudaSuccess ? WUSHKV_OK : WUSHKV_ECUDA;
+    }
+    const char* path_env = std::getenv("WUSHKV_APPEND_PATH");          // "cuda" forces the CUDA-core chunk path (testing)
+    const bool force_cuda = path_env && path_env[0] == 'c';
+    if (max_new >= TC_TILE && !force_cuda) {    // prefill chunk: tensor-core transform
+        const int n_tiles = (total_new + TC_TILE - 1) / TC_TILE;
+        const int per_head = std::max(1, std::min(n_tiles, 2 * sm_count() / P.c.n_kv));
+        const dim3 grid_tc(per_head, P.c.n_kv);
+        cudaError_t e2;
+        if (P.c.bits == 2) {
+            e2 = cudaFuncSetAttribute(append_chunk_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_TOTAL);
+            if (e2 != cudaSuccess) return WUSHKV_ECUDA;
+            append_chunk_kernel<2><<<grid_tc, TC_THREADS, TC_SMEM_TOTAL, st>>>(P);
+        } else {
+            e2 = cudaFuncSetAttribute(append_chunk_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_TOTAL);
+            if (e2 != cudaSuccess) return WUSHKV_ECUDA;
+            append_chunk_kernel<4><<<grid_tc, TC_THREADS, TC_SMEM_TOTAL, st>>>(P);
+        }
+        if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
+        advance_len_kernel<<<(batch + 127) / 128, 128, 0, st>>>(batch, seq_len, cu_new);
         return cudaGetLastError() == cudaSuccess ? WUSHKV_OK : WUSHKV_ECUDA;
     }
     // enough CTAs to fill the machine, but at least 8 tokens each to amortise the transform load

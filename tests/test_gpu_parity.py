@@ -29,7 +29,9 @@ def _check_window_copies(L):
         assert np.array_equal(vb[have], vb_o[have])
         d = np.abs(kb[have] - kb_o[have])
         ulp = np.maximum(np.abs(kb_o[have]), 1e-30) * 2.0 ** -7
-        assert np.all(d <= ulp), "bf16 key copy differs by more than one ulp"
+        # fp32 accumulation error scales with the vector, not with an entry that cancels to almost zero
+        slack = 4e-6 * np.max(np.abs(kb_o[have]), axis=-1, keepdims=True)
+        assert np.all(d <= ulp + slack), "bf16 key copy differs by more than one ulp"
         assert np.mean(d > 0) < 2e-3
 
 
@@ -74,6 +76,24 @@ def test_ragged_batch_shuffled_pages_and_flush_sizes(bits):
         _check_window_copies(L)
         assert L.check_decode_parity() <= 2e-3
         assert L.cache.status() == 0
+
+
+@pytest.mark.parametrize("path", ["tensor", "cuda"])
+def test_prefill_chunk_paths(path, monkeypatch):
+    """Config 4's structure scaled down: several sequences appended as one chunk each in ONE call
+    (tile boundaries fall inside sequences and a ragged last tile), Qwen-shaped heads (G = 7, RMSNorm),
+    through the tensor-core transform and through the CUDA-core chunk path; then one decode step."""
+    if path == "cuda":
+        monkeypatch.setenv("WUSHKV_APPEND_PATH", "cuda")
+    wl = _wl(28, 4, seed=41, batch=3, theta=1e6, rmsnorm=True)
+    L = Layer(wl, [700, 131, 390], 2, 4, 128, 1)
+    L.append_step([699, 130, 389])
+    L.append_step([1, 1, 1])
+    assert L.seq_len.cpu().tolist() == [700, 131, 390]
+    assert L.check_append_parity() <= CODE_MISMATCH_MAX
+    _check_window_copies(L)
+    assert L.check_decode_parity() <= 2e-3
+    assert L.cache.status() == 0
 
 
 def test_window_edges_and_empty_sequences():
