@@ -147,6 +147,15 @@ class Session:
         if verbose:
             print(f"[bench] {name}: cache filled in {time.time() - t0:.1f}s, status {self.cache.status()}", file=sys.stderr)
 
+    def host_tokens(self, b):
+        """The (K, V) token rows of sequence b exactly as the constructor generated them (same stream,
+        same chunking), positions 0 .. : used by tests to recompute sampled pieces with the oracle."""
+        if self.chunk:
+            _, K, V = next(self.wl.sequence_tokens(b, self.chunk, T_V=self.TV, chunk=self.chunk))
+            return K, V
+        toks = list(self.wl.sequence_tokens(b, int(self.start_len[b]) + self.n_steps, T_V=self.TV))
+        return np.concatenate([t[1] for t in toks]), np.concatenate([t[2] for t in toks])
+
     def _dev_bf16(self, x):
         return self.torch.from_numpy(W.f32_to_bf16_bits(x).view(np.int16)).to(self.cache.device)
 

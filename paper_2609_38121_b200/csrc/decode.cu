@@ -57,7 +57,7 @@ struct DecodeParams {
     const int* seq_len;
     const unsigned short* Q;
     float* O;
-    uint4* qfrag;        // [batch*n_kv][128]: fp16 B fragments of the 8 k-steps (quantized positions)
+    uint4* qfrag;        // [batch*n_kv][2][128]: fp16 B fragments of the 8 k-steps (MODE 1: value set, remainder set)
     uint4* qwfrag;       // [batch*n_kv][2][128]: bf16 B fragments for the windows (MODE 1: value set, remainder set)
     float* qscal;        // [batch][n_q][2]: (score multiplier, x_min multiplier) in the log2 domain
     long long* plan;     // [batch+1]: exclusive prefix of work units per sequence (per KV head)
@@ -219,16 +219,17 @@ __global__ void __launch_bounds__(128) decode_prep_kernel(DecodeParams P) {
     // with the remainders.
     const int r16 = i & 15, r = r16 >> 3, t = (r16 & 7) >> 1, hf = r16 & 1;
     const long long bh = static_cast<long long>(b) * P.c.n_kv + h;
-    unsigned short* frag = reinterpret_cast<unsigned short*>(P.qfrag + bh * 128);
+    unsigned short* frag = reinterpret_cast<unsigned short*>(P.qfrag + bh * 256);
     unsigned short* wfrag = reinterpret_cast<unsigned short*>(P.qwfrag + bh * 256);
 #pragma unroll
     for (int n = 0; n < 8; ++n) {
         const int head = (MODE == 0) ? (n >> 1) : n;
-        float val = 0.f, wval = 0.f, wrem = 0.f;
+        float val = 0.f, rem = 0.f, wval = 0.f, wrem = 0.f;
         if (head < G) {
             const float x = acc[head] * pos_scale * beta[head];
             const __half hi = __float2half_rn(x);
-            val = (MODE == 0 && (n & 1)) ? (x - __half2float(hi)) * LO_SCALE : x;
+            rem = (x - __half2float(hi)) * LO_SCALE;
+            val = (MODE == 0 && (n & 1)) ? rem : x;
             const float y = acc[head] * k2;
             const float yh = __bfloat162float(__float2bfloat16_rn(y));
             wrem = y - yh;
@@ -236,6 +237,7 @@ __global__ void __launch_bounds__(128) decode_prep_kernel(DecodeParams P) {
         }
         const int idx = ((((s >> 1) * 32 + 4 * n + t) * 4 + (s & 1) * 2 + r) << 1) + hf;
         frag[idx] = __half_as_ushort(__float2half_rn(val));
+        if (MODE == 1) frag[1024 + idx] = __half_as_ushort(__float2half_rn(rem));
         wfrag[idx] = __bfloat16_as_ushort(__float2bfloat16_rn(wval));
         if (MODE == 1) wfrag[1024 + idx] = __bfloat16_as_ushort(__float2bfloat16_rn(wrem));
     }
@@ -429,7 +431,7 @@ constexpr int MAX_SEGMENTS = 6;           // per warp and round; more segments t
 // main kernel
 // ------------------------------------------------------------------------------------------------
 template <int BITS, int MODE, int STAGES>
-__global__ void __launch_bounds__(MAIN_WARPS * 32, 4) decode_main_kernel(DecodeParams P) {
+__global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ? 4 : 3))) decode_main_kernel(DecodeParams P) {
     constexpr int REC = record_bytes(BITS);
     constexpr int CB = code_block_bytes(BITS);
     constexpr int NH = WarpState<MODE>::NH;
@@ -599,7 +601,7 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, 4) decode_main_kernel(DecodeP
             const int u1 = sg.u1, qp = sg.qp, q_lo = sg.q_lo, q_hi = sg.q_hi;
             int pos0 = (sg.first_page + sg.u0) * PAGE_TOKENS;
             {   // query fragments and per-head scalars of this (sequence, KV head)
-                const uint4* src = P.qfrag + bh * 128;
+                const uint4* src = P.qfrag + bh * 256;
 #pragma unroll
                 for (int s2 = 0; s2 < 4; ++s2) {
                     const uint4 v = __ldg(src + s2 * 32 + lane);
@@ -703,6 +705,37 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, 4) decode_main_kernel(DecodeP
                                 mma_f16(acc2, field<4>(ka.z, a2s, ks), field<4>(kb.z, b2s, ks), field<4>(ka.w, a3s, ks), field<4>(kb.w, b3s, ks),
                                         qf[4 + ks][0], qf[4 + ks][1]);
                             }
+                        }
+                        if (MODE == 1) {
+                            // two heads per column pair leave no room for a remainder column: a second pass over
+                            // the same A fragments with the remainder fragments (re-read per block: L1 hits)
+                            float accr[4] = {0.f, 0.f, 0.f, 0.f}, accr2[4] = {0.f, 0.f, 0.f, 0.f};
+                            const uint4* rsrc = P.qfrag + bh * 256 + 128 + lane;
+                            if (BITS == 2) {
+                                const uint4 kw = lds128(rec + bi * CB + 16 * lane);
+                                const unsigned sx = pre_shift<2>(kw.x), sy = pre_shift<2>(kw.y), sz = pre_shift<2>(kw.z), sw = pre_shift<2>(kw.w);
+#pragma unroll
+                                for (int s2 = 0; s2 < 4; ++s2) {
+                                    const uint4 rq = __ldg(rsrc + s2 * 32);
+                                    mma_f16(accr, field<2>(kw.x, sx, 2 * s2), field<2>(kw.z, sz, 2 * s2), field<2>(kw.y, sy, 2 * s2), field<2>(kw.w, sw, 2 * s2), rq.x, rq.y);
+                                    mma_f16(accr2, field<2>(kw.x, sx, 2 * s2 + 1), field<2>(kw.z, sz, 2 * s2 + 1), field<2>(kw.y, sy, 2 * s2 + 1), field<2>(kw.w, sw, 2 * s2 + 1), rq.z, rq.w);
+                                }
+                            } else {
+                                const uint4 ka = lds128(rec + bi * CB + 16 * lane);
+                                const uint4 kb = lds128(rec + bi * CB + 512 + 16 * lane);
+                                const unsigned a0s = pre_shift<4>(ka.x), a1s = pre_shift<4>(ka.y), a2s = pre_shift<4>(ka.z), a3s = pre_shift<4>(ka.w);
+                                const unsigned b0s = pre_shift<4>(kb.x), b1s = pre_shift<4>(kb.y), b2s = pre_shift<4>(kb.z), b3s = pre_shift<4>(kb.w);
+#pragma unroll
+                                for (int s2 = 0; s2 < 2; ++s2) {
+                                    const uint4 rq = __ldg(rsrc + s2 * 32), rq2 = __ldg(rsrc + (s2 + 2) * 32);
+                                    mma_f16(accr, field<4>(ka.x, a0s, 2 * s2), field<4>(kb.x, b0s, 2 * s2), field<4>(ka.y, a1s, 2 * s2), field<4>(kb.y, b1s, 2 * s2), rq.x, rq.y);
+                                    mma_f16(accr, field<4>(ka.x, a0s, 2 * s2 + 1), field<4>(kb.x, b0s, 2 * s2 + 1), field<4>(ka.y, a1s, 2 * s2 + 1), field<4>(kb.y, b1s, 2 * s2 + 1), rq.z, rq.w);
+                                    mma_f16(accr2, field<4>(ka.z, a2s, 2 * s2), field<4>(kb.z, b2s, 2 * s2), field<4>(ka.w, a3s, 2 * s2), field<4>(kb.w, b3s, 2 * s2), rq2.x, rq2.y);
+                                    mma_f16(accr2, field<4>(ka.z, a2s, 2 * s2 + 1), field<4>(kb.z, b2s, 2 * s2 + 1), field<4>(ka.w, a3s, 2 * s2 + 1), field<4>(kb.w, b3s, 2 * s2 + 1), rq2.z, rq2.w);
+                                }
+                            }
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) acc[e] = fmaf(accr[e] + accr2[e], 1.f / LO_SCALE, acc[e]);
                         }
 #pragma unroll
                         for (int e = 0; e < 4; ++e) acc[e] += acc2[e];
@@ -877,7 +910,7 @@ static bool make_plan(const CacheView& c, int batch, int max_seq_len, DecodePlan
     long long ctas = 0;
     if (const char* e = std::getenv("WUSHKV_DECODE_CTAS")) ctas = std::atoll(e);
     if (ctas <= 0) {
-        const long long per_sm = c.bits == 2 ? 4 : 2;                   // CTAs that fit one SM's shared memory
+        const long long per_sm = c.bits == 4 ? 2 : (c.G <= 4 ? 4 : 3);  // CTAs per SM (shared memory at 4 bits, registers for G > 4)
         ctas = std::min<long long>(per_sm * sm_count(), (units_max + 2 * MAIN_WARPS - 1) / (2 * MAIN_WARPS));
     }
     ctas = std::max<long long>(1, std::min<long long>(ctas, 1 << 20));
@@ -885,7 +918,7 @@ static bool make_plan(const CacheView& c, int batch, int max_seq_len, DecodePlan
     pl.n_warps = pl.n_ctas * MAIN_WARPS;
     const size_t bh = static_cast<size_t>(batch) * c.n_kv;
     size_t off = 0;
-    pl.off_qfrag = off;  off = align_up(off + bh * 128 * sizeof(uint4), 256);
+    pl.off_qfrag = off;  off = align_up(off + bh * 256 * sizeof(uint4), 256);
     pl.off_qwfrag = off; off = align_up(off + bh * 256 * sizeof(uint4), 256);
     pl.off_qscal = off;  off = align_up(off + static_cast<size_t>(batch) * c.n_q * 2 * sizeof(float), 256);
     pl.off_plan = off;   off = align_up(off + (static_cast<size_t>(batch) + 1) * sizeof(long long), 256);

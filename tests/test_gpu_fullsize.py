@@ -1,0 +1,100 @@
+"""Parity at the benchmark configs' FULL sizes, in the launch configuration bench.py times: the cache
+is built by the same `bench.Session` (library transforms, tensor-core chunk append for the prefill,
+single-token append + decode for the step), and the float64 oracle recomputes sampled pieces:
+the codes / scale / zero of sampled token ranges from the regenerated inputs, and the decode output
+of sampled (sequence, KV head) groups from the library's own cache content."""
+import numpy as np
+import pytest
+
+import bench
+from oracle import wushkv_oracle as O
+from paper_2609_38121_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def _unpack(sess, b, h, which, pos0, n):
+    import torch
+    B = sess.B
+    codes = torch.empty((n, 128), dtype=torch.uint8, device="cuda")
+    scale = torch.empty(n, dtype=torch.float32, device="cuda")
+    zero = torch.empty(n, dtype=torch.float32, device="cuda")
+    B.unpack_debug(sess.cache.desc, b, h, which, pos0, n, codes, scale, zero)
+    torch.cuda.synchronize()
+    return codes.cpu().numpy(), scale.cpu().numpy().astype(np.float64), zero.cpu().numpy().astype(np.float64)
+
+
+def _check_append_samples(sess, b, ranges):
+    """Oracle quantization of regenerated tokens of sequence b against the packed cache."""
+    cfg, wl = sess.cfg, sess.wl
+    S = int(sess.seq_len[b].item())
+    K, V = sess.host_tokens(b)
+    n_codes = n_diff = 0
+    T = sess.T.astype(np.float64)
+    for (p0, n) in ranges:
+        p0 = max(0, min(p0, S - n))
+        for h in range(wl.n_kv):
+            for which in (0, 1):
+                gc, gs, gz = _unpack(sess, b, h, which, p0, n)
+                for i in range(n):
+                    x = O.key_transform(T[h], K[p0 + i, h][None])[0] if which == 0 else V[p0 + i, h].astype(np.float64)
+                    c, dl, z = O.quantize(x, cfg["bits"], W.KAPPA_K if which == 0 else W.KAPPA_V)
+                    diff = np.abs(gc[i].astype(np.int32) - c.astype(np.int32))
+                    assert diff.max() <= 1
+                    n_codes += diff.size
+                    n_diff += int(np.count_nonzero(diff))
+                    assert abs(gs[i] - dl) <= 1e-3 * abs(dl) + 1e-12
+                    assert abs(gz[i] - z) <= 1e-3 * max(abs(z), ((1 << cfg["bits"]) - 1) * dl) + 1e-12
+    return n_diff / n_codes
+
+
+def _check_decode_group(sess, out, b, h):
+    """Oracle decode of KV head h of sequence b (its G query heads) on the library's cache content."""
+    cfg, wl = sess.cfg, sess.wl
+    G = wl.G
+    S = int(sess.seq_len[b].item())
+    kc, ks, kz = _unpack(sess, b, h, 0, 0, S)
+    vc, vs, vz = _unpack(sess, b, h, 1, 0, S)
+    km = np.stack([ks, kz], axis=1)[:, None, :]
+    vm = np.stack([vs, vz], axis=1)[:, None, :]
+    c = sess.cache
+    kb = np.full((S, 1, 128), np.nan)
+    vb = np.full((S, 1, 128), np.nan)
+    sink = c.sink_kv[b, h].float().cpu().numpy().astype(np.float64)      # [2][s_sink][d]
+    ring = c.ring_kv[b, h].float().cpu().numpy().astype(np.float64)      # [2][ring_cap][d]
+    for p in range(min(S, cfg["s_sink"])):
+        kb[p, 0], vb[p, 0] = sink[0, p], sink[1, p]
+    for p in range(max(cfg["s_sink"], S - c.ring_cap), S):
+        kb[p, 0], vb[p, 0] = ring[0, p % c.ring_cap], ring[1, p % c.ring_cap]
+    q = sess.q_host[b, h * G:(h + 1) * G].astype(np.float64)
+    ref = O.decode_attn(q, sess.TinvT[h:h + 1].astype(np.float64), kc[:, None], km, vc[:, None], vm, kb, vb, S,
+                        cfg["s_sink"], cfg["s_keep"], sess.s_flush, 1.0 / np.sqrt(128))
+    assert np.all(np.isfinite(ref))
+    got = out[b, h * G:(h + 1) * G]
+    return np.max(np.abs(got - ref)) / np.max(np.abs(ref))
+
+
+@pytest.mark.parametrize("name,groups", [
+    ("cfg1", [(0, 0), (7, 3), (15, 7)]),          # Llama-3-8B-shaped, batch 16 x 32768, 2-bit
+    ("cfg2", [(0, 0), (31, 5), (63, 7)]),         # 4-bit, batch 64, ragged 1024..8192
+    ("cfg3", [(0, 0), (0, 5)]),                   # 70B-shaped, batch 1 x 131072, G = 8
+    ("cfg4", [(0, 0), (5, 2), (7, 3)]),           # Qwen-shaped, 8 x 8192-token chunk, G = 7, then decode
+])
+def test_full_size_config(name, groups):
+    import torch
+    sess = bench.Session(name, n_steps=4)
+    sess.step()                                   # one bench step: append + decode
+    torch.cuda.synchronize()
+    assert sess.cache.status() == 0
+    S_all = sess.seq_len.cpu().numpy()
+    assert np.array_equal(S_all, sess.lengths_at(1))
+    out = sess.O.cpu().numpy().astype(np.float64)
+    assert np.all(np.isfinite(out))
+    # sampled token ranges: the start (sink, first page), a page boundary in the middle, the very end
+    b0 = groups[1][0]
+    S = int(S_all[b0])
+    rate = _check_append_samples(sess, b0, [(0, 6), (S // 2 - 3, 6), (S - 6, 6)])
+    assert rate <= 1e-4 or rate * 3 * 6 * 2 * sess.wl.n_kv * 128 <= 2      # at most a couple of tie flips in the sample
+    for (b, h) in groups:
+        err = _check_decode_group(sess, out, b, h)
+        assert err <= 2e-3, f"{name}: sequence {b} KV head {h}: {err:.3e}"
