@@ -293,6 +293,12 @@ __device__ __forceinline__ void mma_f16(float (&c)[4], unsigned a0, unsigned a1,
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// first MMA of a chain: D = A B (no accumulator registers to initialise)
+__device__ __forceinline__ void mma_f16_zero(float (&d)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0, unsigned b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
+}
 __device__ __forceinline__ void mma_bf16(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0, unsigned b1) {
     asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
@@ -682,12 +688,14 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ?
                     unsigned vmeta[4][2];         // fp16x2 (Delta_v, x_min_v) of rows g, g+8
 #pragma unroll
                     for (int bi = 0; bi < 4; ++bi) {
-                        float acc[4] = {0.f, 0.f, 0.f, 0.f}, acc2[4] = {0.f, 0.f, 0.f, 0.f};      // two chains for ILP
+                        float acc[4], acc2[4];                                                  // two chains for ILP
                         if (BITS == 2) {
                             const uint4 kw = lds128(rec + bi * CB + 16 * lane);
                             const unsigned sx = pre_shift<2>(kw.x), sy = pre_shift<2>(kw.y), sz = pre_shift<2>(kw.z), sw = pre_shift<2>(kw.w);
+                            mma_f16_zero(acc, field<2>(kw.x, sx, 0), field<2>(kw.z, sz, 0), field<2>(kw.y, sy, 0), field<2>(kw.w, sw, 0), qf[0][0], qf[0][1]);
+                            mma_f16_zero(acc2, field<2>(kw.x, sx, 1), field<2>(kw.z, sz, 1), field<2>(kw.y, sy, 1), field<2>(kw.w, sw, 1), qf[1][0], qf[1][1]);
 #pragma unroll
-                            for (int ks = 0; ks < 8; ks += 2) {
+                            for (int ks = 2; ks < 8; ks += 2) {
                                 mma_f16(acc, field<2>(kw.x, sx, ks), field<2>(kw.z, sz, ks), field<2>(kw.y, sy, ks), field<2>(kw.w, sw, ks),
                                         qf[ks][0], qf[ks][1]);
                                 mma_f16(acc2, field<2>(kw.x, sx, ks + 1), field<2>(kw.z, sz, ks + 1), field<2>(kw.y, sy, ks + 1), field<2>(kw.w, sw, ks + 1),
@@ -698,8 +706,10 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ?
                             const uint4 kb = lds128(rec + bi * CB + 512 + 16 * lane);    // row g+8: W0..W3
                             const unsigned a0s = pre_shift<4>(ka.x), a1s = pre_shift<4>(ka.y), a2s = pre_shift<4>(ka.z), a3s = pre_shift<4>(ka.w);
                             const unsigned b0s = pre_shift<4>(kb.x), b1s = pre_shift<4>(kb.y), b2s = pre_shift<4>(kb.z), b3s = pre_shift<4>(kb.w);
+                            mma_f16_zero(acc, field<4>(ka.x, a0s, 0), field<4>(kb.x, b0s, 0), field<4>(ka.y, a1s, 0), field<4>(kb.y, b1s, 0), qf[0][0], qf[0][1]);
+                            mma_f16_zero(acc2, field<4>(ka.z, a2s, 0), field<4>(kb.z, b2s, 0), field<4>(ka.w, a3s, 0), field<4>(kb.w, b3s, 0), qf[4][0], qf[4][1]);
 #pragma unroll
-                            for (int ks = 0; ks < 4; ++ks) {
+                            for (int ks = 1; ks < 4; ++ks) {
                                 mma_f16(acc, field<4>(ka.x, a0s, ks), field<4>(kb.x, b0s, ks), field<4>(ka.y, a1s, ks), field<4>(kb.y, b1s, ks),
                                         qf[ks][0], qf[ks][1]);
                                 mma_f16(acc2, field<4>(ka.z, a2s, ks), field<4>(kb.z, b2s, ks), field<4>(ka.w, a3s, ks), field<4>(kb.w, b3s, ks),
