@@ -249,6 +249,7 @@ __global__ void __launch_bounds__(256) append_rows_kernel(AppendParams P) {
 template <int BITS>
 __global__ void __launch_bounds__(1024) append_token_kernel(AppendParams P) {
     extern __shared__ __align__(16) float tok_s[];       // [n_kv][128] input key, [n_kv][128] transformed key
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a dependent launched programmatically may start; it waits for us itself
     const int b = blockIdx.x;
     const int n_kv = P.c.n_kv;
     float* kin_s = tok_s;

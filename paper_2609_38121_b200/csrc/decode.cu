@@ -115,6 +115,7 @@ __global__ void __launch_bounds__(128) decode_prep_kernel(DecodeParams P) {
     __shared__ long long scan_s[4];
     const int h = blockIdx.x, b = blockIdx.y, G = P.c.G;
     const int i = threadIdx.x, lane = i & 31, warp = i >> 5;
+    pdl_wait();                           // everything this kernel reads may come from the kernel before it
     pdl_launch_dependents();              // the main kernel may start staging pages while this one runs
 
     if (h == 0 && b == 0) {               // work plan: exclusive prefix of units per sequence
@@ -944,10 +945,6 @@ static int launch_decode(const DecodeParams& P, int n_ctas, cudaStream_t st) {
     constexpr int STAGES = 3;
     constexpr size_t SMEM = static_cast<size_t>(MAIN_WARPS) * STAGES * record_bytes(BITS) + MAIN_WARPS * STAGES * 8 +
                             MAIN_WARPS * MAX_SEGMENTS * sizeof(Segment);
-    decode_prep_kernel<BITS, MODE><<<dim3(P.c.n_kv, P.batch), 128, 0, st>>>(P);
-    if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
-    if (cudaFuncSetAttribute(decode_main_kernel<BITS, MODE, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(SMEM)) != cudaSuccess)
-        return WUSHKV_ECUDA;
     cudaLaunchAttribute pdl_attr[1];
     pdl_attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     pdl_attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -955,6 +952,12 @@ static int launch_decode(const DecodeParams& P, int n_ctas, cudaStream_t st) {
     cfg.stream = st;
     cfg.attrs = pdl_attr;
     cfg.numAttrs = 1;
+    cfg.gridDim = dim3(P.c.n_kv, P.batch);
+    cfg.blockDim = dim3(128);
+    cfg.dynamicSmemBytes = 0;
+    if (cudaLaunchKernelEx(&cfg, decode_prep_kernel<BITS, MODE>, P) != cudaSuccess) return WUSHKV_ECUDA;
+    if (cudaFuncSetAttribute(decode_main_kernel<BITS, MODE, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(SMEM)) != cudaSuccess)
+        return WUSHKV_ECUDA;
     if (g_prof_start) cudaEventRecord(g_prof_start, st);
     cfg.gridDim = dim3(n_ctas);
     cfg.blockDim = dim3(MAIN_WARPS * 32);
