@@ -204,6 +204,25 @@ class Session:
 
 
 # ------------------------------------------------------------------------------------------------
+# multi-GPU aggregation (replicas only: no data-path collective, just the slowest rank's time)
+# ------------------------------------------------------------------------------------------------
+def max_over_ranks(ms, device="cuda"):
+    """Slowest rank's time per step (all ranks get it).  A no-op outside torch.distributed."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(bytes_per_rank_step, ms_per_step, world):
+    """Whole-job GB/s: every rank moved `bytes_per_rank_step` per step, the job took the slowest rank's time."""
+    return world * bytes_per_rank_step / (ms_per_step * 1e-3) / 1e9
+
+
+# ------------------------------------------------------------------------------------------------
 # clocks
 # ------------------------------------------------------------------------------------------------
 class ClockSampler:
@@ -417,12 +436,9 @@ def run_ours(args, rank, world):
     step_ms = [s_.elapsed_time(e_) for s_, e_ in zip(starts, stops)]
     append_ms = [s_.elapsed_time(e_) for s_, e_ in zip(starts, mids)]
     kern_ms = [s_.elapsed_time(e_) for s_, e_ in zip(kstart, kstop)]
-    if world > 1:
-        t = torch.tensor([ms_per_step], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_per_step = float(t.item())
+    ms_per_step = max_over_ranks(ms_per_step)
     bytes_step = float(np.mean([sess.decode_bytes(Wm + i + 1) for i in range(K)])) if not sess.chunk else float(cache_bytes)
-    value = world * bytes_step / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_value(bytes_step, ms_per_step, world)
 
     # ---- end-to-end through the host-buffer entry point (decode steps only)
     e2e = None
@@ -450,11 +466,8 @@ def run_ours(args, rank, world):
             host_step(Wm + i)
         t1 = time.perf_counter()
         e2e_ms = (t1 - t0) * 1e3 / K
-        if world > 1:
-            t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
-        e2e = {"value": world * bytes_step / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms,
+        e2e_ms = max_over_ranks(e2e_ms)
+        e2e = {"value": whole_job_value(bytes_step, e2e_ms, world), "unit": "GB/s", "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": int(2 * hK[0].numel() * 2 + hQ.numel() * 2), "d2h_bytes_per_step": int(hO.numel() * 4)}
         assert sess.cache.status() == 0
 

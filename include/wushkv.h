@@ -13,8 +13,9 @@
  *       recent positions from a bf16 copy (Section 4.4).
  *
  * General rules
- *   - Every function returns an int status (WUSHKV_OK = 0).  No exceptions, no global state
- *     except a cached device-attribute query.
+ *   - Every function returns an int status (WUSHKV_OK = 0).  No exceptions.  Global state is
+ *     limited to a cached device-attribute query, the optional event pair of
+ *     wushkv_set_profile_events and the built-in scratch of wushkv_decode_attn_static.
  *   - "host" / "device" beside a pointer says where the memory must live.  All memory is
  *     owned by the caller before, during and after every call; the library allocates nothing
  *     and keeps no pointer between calls.
@@ -146,8 +147,10 @@ int wushkv_build_transforms(int32_t n_heads, int32_t d, const double* M, const d
  *   total_new, max_new (host): total and per-sequence maximum of new tokens.
  *   K_new (device): bf16 [total_new][n_kv][d] post-Norm post-RoPE keys, 16-byte aligned.
  *   V_new (device): bf16 [total_new][n_kv][d] values in the folded basis, 16-byte aligned.
- * Chunks (max_new >= 128) take the tensor-core transform path; short appends a CUDA-core one.
- * Both produce the same codes up to fp32 summation order.
+ * Chunks (max_new >= 128) take the tensor-core transform path (tcgen05, fp32 accumulation in
+ * tensor memory), max_new == 1 a single-launch decode-time path, anything else a CUDA-core path.
+ * All produce the same codes up to fp32 summation order.  Environment variable
+ * WUSHKV_APPEND_PATH=cuda forces the CUDA-core path for chunks (testing aid).
  */
 int wushkv_append(const wushkv_cache* cache, int32_t batch, const int32_t* slot, int32_t* seq_len,
                   const int32_t* cu_new, int32_t total_new, int32_t max_new,
@@ -170,6 +173,9 @@ size_t wushkv_decode_workspace_bytes(const wushkv_cache* cache, int32_t batch, i
  *       projection, Algorithm 2 line 6, is outside the library).
  *   workspace (device): >= wushkv_decode_workspace_bytes(...) bytes, 256-byte aligned; contents
  *       are scratch (no initialisation needed, nothing survives the call).
+ * The kernels of one call are chained by programmatic dependent launch; the first of them waits
+ * for the kernel before it in the stream before it reads anything, so any producer of Q, seq_len or
+ * the cache may precede the call directly.
  */
 int wushkv_decode_attn(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
                        int32_t max_seq_len, const uint16_t* Q, float* O,
