@@ -335,11 +335,12 @@ __global__ void __launch_bounds__(1024) append_token_kernel(AppendParams P) {
 // ------------------------------------------------------------------------------------------------
 constexpr int TC_TILE = 128;                 // tokens per tile (MMA M)
 constexpr int TC_LBO = 128, TC_SBO = 2048;   // bytes
-constexpr int TC_X_PITCH = 132;              // floats per row of the fp32 key tile in shared memory
+constexpr int TC_X_PITCH = 136;              // floats per row of the fp32 key tile (== 8 mod 32: conflict-free quad reads)
 constexpr int TC_THREADS = 512;
 constexpr int TC_SMEM_B = 32768;                                   // T_K as bf16 operand
 constexpr int TC_SMEM_X = TC_TILE * TC_X_PITCH * 4;                // fp32 keys; its first 32 KB double as the A operand
-constexpr int TC_SMEM_TOTAL = TC_SMEM_B + TC_SMEM_X + 64;
+constexpr int TC_SMEM_ROWS = TC_TILE * 32;                          // per-row token lookup (RowInfo)
+constexpr int TC_SMEM_TOTAL = TC_SMEM_B + TC_SMEM_X + TC_SMEM_ROWS + 64;
 
 __device__ __forceinline__ unsigned long long umma_smem_desc(unsigned smem_addr) {
     unsigned long long d = 0;
@@ -354,7 +355,108 @@ constexpr unsigned UMMA_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3
 
 __device__ __forceinline__ unsigned smem_addr_u32(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
 
-template <int BITS>
+// ---- quad-per-vector quantizer of the chunk path --------------------------------------------------
+// Four adjacent lanes own one 128-vector, 32 entries each.  The clipping quantile needs the two
+// order statistics around rank kappa*(d-1) of |x|, i.e. the `rounds`-th and (`rounds`-1)-th largest;
+// each lane keeps the KK largest of its entries with bitonic networks on registers and the quad merges
+// the four lists with two exchanges.  All network indices are compile-time constants.
+struct RowInfo {                 // where one token of the tile goes (filled once per tile and head)
+    long long rec_off;           // byte offset of the head's record in the page pool, < 0: skip the token
+    int r, pos, s_final, slot;
+    int pad[2];
+};
+
+__device__ __forceinline__ void ce_desc_u(unsigned& a, unsigned& b) {
+    const unsigned hi = max(a, b), lo = min(a, b);
+    a = hi; b = lo;
+}
+template <int N>
+__device__ __forceinline__ void bitonic_sort_desc(unsigned (&a)[N]) {
+#pragma unroll
+    for (int k = 2; k <= N; k <<= 1)
+#pragma unroll
+        for (int j = k >> 1; j > 0; j >>= 1)
+#pragma unroll
+            for (int i = 0; i < N; ++i) {
+                const int l = i ^ j;
+                if (l > i) { if ((i & k) == 0) ce_desc_u(a[i], a[l]); else ce_desc_u(a[l], a[i]); }
+            }
+}
+template <int N>
+__device__ __forceinline__ void bitonic_merge_desc(unsigned (&a)[N]) {      // bitonic sequence -> descending
+#pragma unroll
+    for (int j = N >> 1; j > 0; j >>= 1)
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+            const int l = i ^ j;
+            if (l > i) ce_desc_u(a[i], a[l]);
+        }
+}
+template <int N>
+__device__ __forceinline__ void keep_largest(unsigned (&top)[N], const unsigned (&other)[N]) {   // both descending
+#pragma unroll
+    for (int i = 0; i < N; ++i) top[i] = max(top[i], other[N - 1 - i]);
+    bitonic_merge_desc<N>(top);
+}
+
+// Clip range, stored step / offset and the 32 codes of this lane's entries x[32] (Eq. 6); all four
+// lanes of the quad return the same step_h / xmin_h.
+template <int BITS, int KK>
+__device__ __forceinline__ void quad_quantize(const float (&x)[32], ClipRule rule, int (&code)[32], __half& step_h, __half& xmin_h) {
+    constexpr int LEVELS = (1 << BITS) - 1;
+    unsigned top[KK];
+#pragma unroll
+    for (int g0 = 0; g0 < 32; g0 += KK) {
+        unsigned tmp[KK];
+#pragma unroll
+        for (int i = 0; i < KK; ++i) tmp[i] = __float_as_uint(x[g0 + i]) & 0x7fffffffu;
+        bitonic_sort_desc<KK>(tmp);
+        if (g0 == 0) {
+#pragma unroll
+            for (int i = 0; i < KK; ++i) top[i] = tmp[i];
+        } else {
+            keep_largest<KK>(top, tmp);
+        }
+    }
+#pragma unroll
+    for (int off = 1; off <= 2; off <<= 1) {
+        unsigned other[KK];
+#pragma unroll
+        for (int i = 0; i < KK; ++i) other[i] = __shfl_xor_sync(FULL, top[i], off);
+        keep_largest<KK>(top, other);
+    }
+    unsigned a_lo = 0, a_hi = 0;
+#pragma unroll
+    for (int i = 0; i < KK; ++i) {
+        if (i == rule.rounds - 1) a_lo = top[i];
+        if (i == rule.rounds - 2) a_hi = top[i];
+    }
+    if (rule.rounds == 1) a_hi = a_lo;
+    const float alo = __uint_as_float(a_lo), ahi = __uint_as_float(a_hi);
+    const float q = alo + rule.frac * (ahi - alo);
+    float lmin = x[0], lmax = x[0];
+#pragma unroll
+    for (int i = 1; i < 32; ++i) { lmin = fminf(lmin, x[i]); lmax = fmaxf(lmax, x[i]); }
+    lmin = fminf(lmin, __shfl_xor_sync(FULL, lmin, 1)); lmax = fmaxf(lmax, __shfl_xor_sync(FULL, lmax, 1));
+    lmin = fminf(lmin, __shfl_xor_sync(FULL, lmin, 2)); lmax = fmaxf(lmax, __shfl_xor_sync(FULL, lmax, 2));
+    const float x_min = fmaxf(lmin, -q);
+    const float x_max = fminf(lmax, q);
+    const float step = __fdiv_rn(x_max - x_min, static_cast<float>(LEVELS));
+    step_h = __float2half_rn(fminf(fmaxf(step, -65504.f), 65504.f));
+    xmin_h = __float2half_rn(fminf(fmaxf(x_min, -65504.f), 65504.f));
+    const float step_s = __half2float(step_h), xmin_s = __half2float(xmin_h);
+    const float inv = step_s > 0.f ? __frcp_rn(step_s) : 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        // clamp, then round to nearest even by adding 1.5 * 2^23: the code is in the low mantissa bits
+        const float t = fminf(fmaxf((x[i] - xmin_s) * inv, 0.f), static_cast<float>(LEVELS));
+        code[i] = static_cast<int>(__float_as_uint(t + 12582912.f) & 0xFu);
+    }
+}
+
+// KK_K / KK_V: list length of the quad quantizer for keys / values (8 or 16, >= the rule's rounds), or 0 for
+// the warp-per-vector quantizer (any kappa).
+template <int BITS, int KK_K, int KK_V>
 __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParams P) {
     extern __shared__ __align__(1024) unsigned char tc_smem[];
     unsigned char* sB = tc_smem;
@@ -362,6 +464,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
     float* sX = reinterpret_cast<float*>(tc_smem + TC_SMEM_B);
     unsigned long long* mbar = reinterpret_cast<unsigned long long*>(tc_smem + TC_SMEM_B + TC_SMEM_X);
     unsigned* tmem_slot = reinterpret_cast<unsigned*>(tc_smem + TC_SMEM_B + TC_SMEM_X + 16);
+    RowInfo* rows = reinterpret_cast<RowInfo*>(tc_smem + TC_SMEM_B + TC_SMEM_X + 64);
     const int head = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_tiles = (P.total_new + TC_TILE - 1) / TC_TILE;
@@ -410,6 +513,15 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
                 *reinterpret_cast<uint4*>(sA + rg * TC_SBO + kc * TC_LBO + r8 * 16) = v;
             }
         }
+        if (tid < TC_TILE) {                                  // where each token of the tile goes
+            RowInfo ri;
+            ri.rec_off = -1; ri.r = 0; ri.pos = 0; ri.s_final = 0; ri.slot = 0; ri.pad[0] = ri.pad[1] = 0;
+            TokenSlot ts;
+            if (tok0 + tid < P.total_new && locate_token(P, tok0 + tid, head, ts)) {
+                ri.rec_off = ts.rec - P.c.pages; ri.r = ts.r; ri.pos = ts.pos; ri.s_final = ts.s_final; ri.slot = ts.slot;
+            }
+            rows[tid] = ri;
+        }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // generic-proxy writes -> visible to the tensor core
         __syncthreads();
         // ---- one thread issues the 8 k-steps and commits them to the barrier
@@ -429,21 +541,80 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
             asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr_u32(mbar)) : "memory");
         }
         // ---- while the tensor core runs: values of this tile (no transform)
-        for (int v = warp; v < TC_TILE; v += TC_THREADS / 32) {
-            const int token = tok0 + v;
-            if (token >= P.total_new) break;
-            TokenSlot ts;
-            if (!locate_token(P, token, head, ts)) continue;
-            const uint2 vraw = __ldg(reinterpret_cast<const uint2*>(P.V_new + (static_cast<long long>(token) * P.c.n_kv + head) * D) + lane);
-            float x[4] = {bf16_bits_to_float(vraw.x & 0xffff), bf16_bits_to_float(vraw.x >> 16),
-                          bf16_bits_to_float(vraw.y & 0xffff), bf16_bits_to_float(vraw.y >> 16)};
-            int code[4];
+        if (KK_V > 0) {
+            constexpr int KQ = KK_V > 0 ? KK_V : 8;
+            const int row = 8 * warp + (lane >> 2), qd = lane & 3;
+            const RowInfo ri = rows[row];
+            const bool live = ri.rec_off >= 0;
+            const unsigned short* vsrc = P.V_new + (static_cast<long long>(tok0 + row) * P.c.n_kv + head) * D + 4 * qd;
+            float x[32];
+            uint2 raw[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                raw[k] = live ? __ldg(reinterpret_cast<const uint2*>(vsrc + 16 * k)) : make_uint2(0u, 0u);
+                x[4 * k + 0] = bf16_bits_to_float(raw[k].x & 0xffff); x[4 * k + 1] = bf16_bits_to_float(raw[k].x >> 16);
+                x[4 * k + 2] = bf16_bits_to_float(raw[k].y & 0xffff); x[4 * k + 3] = bf16_bits_to_float(raw[k].y >> 16);
+            }
+            int code[32];
             __half step_h, xmin_h;
-            quantize_vec<BITS>(x, P.rule_v, lane, code, step_h, xmin_h);
-            store_v_codes<BITS>(ts.rec, ts.r, code, lane);
-            __half* meta = reinterpret_cast<__half*>(ts.rec + meta_location(BITS, ts.r));
-            if (lane == 0) { meta[2] = step_h; meta[3] = xmin_h; }
-            store_window_copy(P, ts, head, 1, vraw, lane);
+            quad_quantize<BITS, KQ>(x, P.rule_v, code, step_h, xmin_h);
+            if (live) {
+                unsigned char* rec = P.c.pages + ri.rec_off;
+                const int bi = ri.r >> 4, rr = ri.r & 15, ps = rr >> 3, t = (rr & 7) >> 1, hi = rr & 1;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {                 // channel residue c16 = 4 qd + e: one half-word per 8 (or 4) channel blocks
+                    const int c16 = 4 * qd + e, g = c16 & 7, rsel = c16 >> 3;
+                    if (BITS == 2) {
+                        unsigned hw = 0;
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) hw |= static_cast<unsigned>(code[4 * k + e]) << (2 * k);
+                        *reinterpret_cast<unsigned short*>(rec + v_codes_offset(2) + bi * 512 + 16 * (4 * g + t) + 4 * (2 * ps + rsel) + 2 * hi) =
+                            static_cast<unsigned short>(hw);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            unsigned hw = 0;
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) hw |= static_cast<unsigned>(code[4 * (4 * j + k) + e]) << (4 * k);
+                            *reinterpret_cast<unsigned short*>(rec + v_codes_offset(4) + bi * 1024 + 512 * ps + 16 * (4 * g + t) + 4 * (2 * rsel + j) + 2 * hi) =
+                                static_cast<unsigned short>(hw);
+                        }
+                    }
+                }
+                if (qd == 0) {
+                    __half* meta = reinterpret_cast<__half*>(rec + meta_location(BITS, ri.r));
+                    meta[2] = step_h; meta[3] = xmin_h;
+                }
+                const CacheView& c = P.c;
+                const long long plane = (static_cast<long long>(ri.slot) * c.n_kv + head) * 2 + 1;
+                if (ri.pos < c.s_sink) {
+                    unsigned short* dst = c.sink_kv + (plane * c.s_sink + ri.pos) * D + 4 * qd;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) *reinterpret_cast<uint2*>(dst + 16 * k) = raw[k];
+                }
+                if (ri.pos >= ri.s_final - c.ring_cap) {
+                    unsigned short* dst = c.ring_kv + (plane * c.ring_cap + ri.pos % c.ring_cap) * D + 4 * qd;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) *reinterpret_cast<uint2*>(dst + 16 * k) = raw[k];
+                }
+            }
+        } else {
+            for (int v = warp; v < TC_TILE; v += TC_THREADS / 32) {
+                const int token = tok0 + v;
+                if (token >= P.total_new) break;
+                TokenSlot ts;
+                if (!locate_token(P, token, head, ts)) continue;
+                const uint2 vraw = __ldg(reinterpret_cast<const uint2*>(P.V_new + (static_cast<long long>(token) * P.c.n_kv + head) * D) + lane);
+                float x[4] = {bf16_bits_to_float(vraw.x & 0xffff), bf16_bits_to_float(vraw.x >> 16),
+                              bf16_bits_to_float(vraw.y & 0xffff), bf16_bits_to_float(vraw.y >> 16)};
+                int code[4];
+                __half step_h, xmin_h;
+                quantize_vec<BITS>(x, P.rule_v, lane, code, step_h, xmin_h);
+                store_v_codes<BITS>(ts.rec, ts.r, code, lane);
+                __half* meta = reinterpret_cast<__half*>(ts.rec + meta_location(BITS, ts.r));
+                if (lane == 0) { meta[2] = step_h; meta[3] = xmin_h; }
+                store_window_copy(P, ts, head, 1, vraw, lane);
+            }
         }
         // ---- wait for the MMAs (bounded), then tensor memory -> shared memory
         {
@@ -483,23 +654,79 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
         // ---- keys of this tile: quantize the fp32 rows
-        for (int v = warp; v < TC_TILE; v += TC_THREADS / 32) {
-            const int token = tok0 + v;
-            if (token >= P.total_new) break;
-            TokenSlot ts;
-            if (!locate_token(P, token, head, ts)) continue;
-            const float4 kp = *reinterpret_cast<const float4*>(sX + v * TC_X_PITCH + 4 * lane);
-            float x[4] = {kp.x, kp.y, kp.z, kp.w};
-            int code[4];
+        if (KK_K > 0) {
+            constexpr int KQ = KK_K > 0 ? KK_K : 8;
+            const int row = 8 * warp + (lane >> 2), qd = lane & 3;
+            const RowInfo ri = rows[row];
+            const bool live = ri.rec_off >= 0;
+            float x[32];                                      // entry 4k + j: channel 16k + 2qd + (j & 1) + 8 (j >> 1)
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const float2 a = *reinterpret_cast<const float2*>(sX + row * TC_X_PITCH + 16 * k + 2 * qd);
+                const float2 b = *reinterpret_cast<const float2*>(sX + row * TC_X_PITCH + 16 * k + 2 * qd + 8);
+                x[4 * k + 0] = a.x; x[4 * k + 1] = a.y; x[4 * k + 2] = b.x; x[4 * k + 3] = b.y;
+            }
+            int code[32];
             __half step_h, xmin_h;
-            quantize_vec<BITS>(x, P.rule_k, lane, code, step_h, xmin_h);
-            store_k_codes<BITS>(ts.rec, ts.r, code, lane);
-            __half* meta = reinterpret_cast<__half*>(ts.rec + meta_location(BITS, ts.r));
-            if (lane == 0) { meta[0] = step_h; meta[1] = xmin_h; }
-            uint2 kb;
-            kb.x = float_to_bf16_bits(x[0]) | (static_cast<unsigned>(float_to_bf16_bits(x[1])) << 16);
-            kb.y = float_to_bf16_bits(x[2]) | (static_cast<unsigned>(float_to_bf16_bits(x[3])) << 16);
-            store_window_copy(P, ts, head, 0, kb, lane);
+            quad_quantize<BITS, KQ>(x, P.rule_k, code, step_h, xmin_h);
+            if (live) {
+                unsigned char* rec = P.c.pages + ri.rec_off;
+                const int bi = ri.r >> 4, rr = ri.r & 15, g = rr & 7, rs = rr >> 3;
+                if (BITS == 2) {
+                    uint2 w = make_uint2(0u, 0u);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        w.x |= (static_cast<unsigned>(code[4 * k + 0]) << (2 * k)) | (static_cast<unsigned>(code[4 * k + 1]) << (16 + 2 * k));
+                        w.y |= (static_cast<unsigned>(code[4 * k + 2]) << (2 * k)) | (static_cast<unsigned>(code[4 * k + 3]) << (16 + 2 * k));
+                    }
+                    *reinterpret_cast<uint2*>(rec + bi * 512 + 16 * (4 * g + qd) + 8 * rs) = w;
+                } else {
+                    unsigned w[4] = {0u, 0u, 0u, 0u};         // word 2 (k >> 2) + (j >> 1), field k & 3
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        w[2 * (k >> 2) + 0] |= (static_cast<unsigned>(code[4 * k + 0]) << (4 * (k & 3))) | (static_cast<unsigned>(code[4 * k + 1]) << (16 + 4 * (k & 3)));
+                        w[2 * (k >> 2) + 1] |= (static_cast<unsigned>(code[4 * k + 2]) << (4 * (k & 3))) | (static_cast<unsigned>(code[4 * k + 3]) << (16 + 4 * (k & 3)));
+                    }
+                    *reinterpret_cast<uint4*>(rec + bi * 1024 + 512 * rs + 16 * (4 * g + qd)) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+                if (qd == 0) {
+                    __half* meta = reinterpret_cast<__half*>(rec + meta_location(BITS, ri.r));
+                    meta[0] = step_h; meta[1] = xmin_h;
+                }
+                const CacheView& c = P.c;
+                const long long plane = (static_cast<long long>(ri.slot) * c.n_kv + head) * 2 + 0;
+                const bool to_sink = ri.pos < c.s_sink, to_ring = ri.pos >= ri.s_final - c.ring_cap;
+                if (to_sink || to_ring) {
+                    unsigned short* d_sink = c.sink_kv + (plane * c.s_sink + ri.pos) * D + 2 * qd;
+                    unsigned short* d_ring = c.ring_kv + (plane * c.ring_cap + ri.pos % c.ring_cap) * D + 2 * qd;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const unsigned lo = float_to_bf16_bits(x[4 * k + 0]) | (static_cast<unsigned>(float_to_bf16_bits(x[4 * k + 1])) << 16);
+                        const unsigned hi2 = float_to_bf16_bits(x[4 * k + 2]) | (static_cast<unsigned>(float_to_bf16_bits(x[4 * k + 3])) << 16);
+                        if (to_sink) { *reinterpret_cast<unsigned*>(d_sink + 16 * k) = lo; *reinterpret_cast<unsigned*>(d_sink + 16 * k + 8) = hi2; }
+                        if (to_ring) { *reinterpret_cast<unsigned*>(d_ring + 16 * k) = lo; *reinterpret_cast<unsigned*>(d_ring + 16 * k + 8) = hi2; }
+                    }
+                }
+            }
+        } else {
+            for (int v = warp; v < TC_TILE; v += TC_THREADS / 32) {
+                const int token = tok0 + v;
+                if (token >= P.total_new) break;
+                TokenSlot ts;
+                if (!locate_token(P, token, head, ts)) continue;
+                const float4 kp = *reinterpret_cast<const float4*>(sX + v * TC_X_PITCH + 4 * lane);
+                float x[4] = {kp.x, kp.y, kp.z, kp.w};
+                int code[4];
+                __half step_h, xmin_h;
+                quantize_vec<BITS>(x, P.rule_k, lane, code, step_h, xmin_h);
+                store_k_codes<BITS>(ts.rec, ts.r, code, lane);
+                __half* meta = reinterpret_cast<__half*>(ts.rec + meta_location(BITS, ts.r));
+                if (lane == 0) { meta[0] = step_h; meta[1] = xmin_h; }
+                uint2 kb;
+                kb.x = float_to_bf16_bits(x[0]) | (static_cast<unsigned>(float_to_bf16_bits(x[1])) << 16);
+                kb.y = float_to_bf16_bits(x[2]) | (static_cast<unsigned>(float_to_bf16_bits(x[3])) << 16);
+                store_window_copy(P, ts, head, 0, kb, lane);
+            }
         }
         __syncthreads();                                      // the fp32 tile becomes the next A operand
     }
@@ -579,16 +806,30 @@ extern "C" int wushkv_append(const wushkv_cache* cache, int32_t batch, const int
         const int n_tiles = (total_new + TC_TILE - 1) / TC_TILE;
         const int per_head = std::max(1, std::min(n_tiles, 2 * sm_count() / P.c.n_kv));
         const dim3 grid_tc(per_head, P.c.n_kv);
-        cudaError_t e2;
+        // list length of the quad quantizer: the rule's rounds must fit (kappa >= ~0.945 -> 8, >= ~0.882 -> 16)
+        const int need = std::max(P.rule_k.rounds, P.rule_v.rounds);
+        const int kk_k = need > 16 ? 0 : (P.rule_k.rounds <= 8 ? 8 : 16);
+        const int kk_v = need > 16 ? 0 : (P.rule_v.rounds <= 8 ? 8 : 16);
+        auto launch = [&](auto kernel) -> bool {
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_TOTAL) != cudaSuccess) return false;
+            kernel<<<grid_tc, TC_THREADS, TC_SMEM_TOTAL, st>>>(P);
+            return true;
+        };
+        bool ok;
         if (P.c.bits == 2) {
-            e2 = cudaFuncSetAttribute(append_chunk_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_TOTAL);
-            if (e2 != cudaSuccess) return WUSHKV_ECUDA;
-            append_chunk_kernel<2><<<grid_tc, TC_THREADS, TC_SMEM_TOTAL, st>>>(P);
+            if (kk_k == 0) ok = launch(append_chunk_kernel<2, 0, 0>);
+            else if (kk_k == 8 && kk_v == 8) ok = launch(append_chunk_kernel<2, 8, 8>);
+            else if (kk_k == 8) ok = launch(append_chunk_kernel<2, 8, 16>);
+            else if (kk_v == 8) ok = launch(append_chunk_kernel<2, 16, 8>);
+            else ok = launch(append_chunk_kernel<2, 16, 16>);
         } else {
-            e2 = cudaFuncSetAttribute(append_chunk_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_TOTAL);
-            if (e2 != cudaSuccess) return WUSHKV_ECUDA;
-            append_chunk_kernel<4><<<grid_tc, TC_THREADS, TC_SMEM_TOTAL, st>>>(P);
+            if (kk_k == 0) ok = launch(append_chunk_kernel<4, 0, 0>);
+            else if (kk_k == 8 && kk_v == 8) ok = launch(append_chunk_kernel<4, 8, 8>);
+            else if (kk_k == 8) ok = launch(append_chunk_kernel<4, 8, 16>);
+            else if (kk_v == 8) ok = launch(append_chunk_kernel<4, 16, 8>);
+            else ok = launch(append_chunk_kernel<4, 16, 16>);
         }
+        if (!ok) return WUSHKV_ECUDA;
         if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
         advance_len_kernel<<<(batch + 127) / 128, 128, 0, st>>>(batch, seq_len, cu_new);
         return cudaGetLastError() == cudaSuccess ? WUSHKV_OK : WUSHKV_ECUDA;
