@@ -166,6 +166,12 @@ class Session:
     def step(self, mid_event=None):
         """Enqueue one step (device-resident inputs)."""
         B = self.B
+        if not self.chunk and mid_event is None:        # the fused call a user makes for a decode step
+            i = self.step_index
+            B.decode_step(self.cache.desc, self.batch, self.slot, self.seq_len, self.cu_one, self.max_seq_len,
+                          self.step_K[i], self.step_V[i], self.Q, self.O, self.ws, self.ws_bytes)
+            self.step_index += 1
+            return
         if self.chunk:
             self.seq_len.zero_()
             B.append(self.cache.desc, self.batch, self.slot, self.seq_len, self.cu_chunk, self.batch * self.chunk,
@@ -225,51 +231,100 @@ def whole_job_value(bytes_per_rank_step, ms_per_step, world):
 # ------------------------------------------------------------------------------------------------
 # clocks
 # ------------------------------------------------------------------------------------------------
-class ClockSampler:
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-             "clocks_event_reasons.sw_power_cap")
+_CLOCK_POLL_SRC = r"""
+import sys, time
+import pynvml as N
+N.nvmlInit()
+key = sys.argv[1]
+try:
+    h = N.nvmlDeviceGetHandleByUUID(key) if key.startswith("GPU-") else N.nvmlDeviceGetHandleByIndex(int(key))
+except Exception:
+    h = N.nvmlDeviceGetHandleByIndex(0)
+mx = N.nvmlDeviceGetMaxClockInfo(h, N.NVML_CLOCK_SM)
+w = sys.stdout.write
+while True:
+    t = time.monotonic_ns()
+    sm = N.nvmlDeviceGetClockInfo(h, N.NVML_CLOCK_SM)
+    try:
+        r = N.nvmlDeviceGetCurrentClocksEventReasons(h)
+    except Exception:
+        r = N.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+    w("%d,%d,%d,%d\n" % (t, sm, mx, r))
+    sys.stdout.flush()
+    time.sleep(0.0003)
+"""
 
-    def __init__(self, gpu_index):
+
+def device_key(local):
+    """NVML name of CUDA device `local`: its UUID (CUDA_VISIBLE_DEVICES may renumber), else the index."""
+    try:
+        import torch
+        return "GPU-" + str(torch.cuda.get_device_properties(local).uuid)
+    except Exception:
+        return str(local)
+
+
+class ClockSampler:
+    """Reads (never sets) the SM clock and the clock-event reasons of one GPU through NVML from a
+    child process, a few thousand times a second, so that a timed region of a few milliseconds
+    still holds samples; `mark()` brackets the region on the system-wide monotonic clock."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown"}
+
+    def __init__(self, device_key):
         self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
-        self.proc = None
+        self.t0 = self.t1 = None
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "50", "-i", str(gpu_index)], stdout=self.tmp, stderr=subprocess.DEVNULL)
+            self.proc = subprocess.Popen([sys.executable, "-c", _CLOCK_POLL_SRC, str(device_key)],
+                                         stdout=self.tmp, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
+        deadline = time.time() + 10.0                       # wait for the first sample
+        while self.proc is not None and time.time() < deadline and os.path.getsize(self.tmp.name) == 0:
+            if self.proc.poll() is not None:
+                self.proc = None
+                break
+            time.sleep(0.01)
+
+    def mark(self):
+        if self.t0 is None:
+            self.t0 = time.monotonic_ns()
+        else:
+            self.t1 = time.monotonic_ns()
 
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.proc is None:
-            return out
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
         self.tmp.flush()
         self.tmp.seek(0)
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = []
         for line in self.tmp.read().splitlines():
-            f = [x.strip() for x in line.split(",")]
-            if len(f) < 9:
-                continue
-            try:
-                sm.append(float(f[1]))
-                mx.append(float(f[2]))
-            except ValueError:
-                continue
-            for nm, val in zip(names, f[5:9]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
+            f = line.split(",")
+            if len(f) == 4:
+                try:
+                    rows.append(tuple(int(x) for x in f))
+                except ValueError:
+                    pass
         try:
             os.unlink(self.tmp.name)
         except OSError:
             pass
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        t0, t1 = self.t0 or 0, self.t1 or (1 << 62)
+        inside = [r for r in rows if t0 <= r[0] <= t1]
+        if not inside and rows:                              # region shorter than the sampling period
+            mid = (t0 + t1) // 2
+            inside = sorted(rows, key=lambda r: abs(r[0] - mid))[:2]
+            out["nearest"] = True
+        if inside:
+            bits = 0
+            for r in inside:
+                bits |= r[3]
+            out.update(sm_mhz=statistics.median(r[1] for r in inside), sm_max_mhz=max(r[2] for r in inside),
+                       reasons=sorted(n for b, n in self.REASONS.items() if bits & b), samples=len(inside))
         return out
 
 
@@ -394,9 +449,11 @@ def run_ours(args, rank, world):
 
     ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
     starts, stops = [ev() for _ in range(K)], [ev() for _ in range(K)]
-    sampler = ClockSampler(local) if rank == 0 else None
+    sampler = ClockSampler(device_key(local)) if rank == 0 else None
     # ---- region A: K whole steps, device-timed; this gives `value`
     barrier()
+    if sampler:
+        sampler.mark()
     t_region0, t_region1 = ev(), ev()
     t_region0.record()
     for i in range(K):
@@ -431,6 +488,8 @@ def run_ours(args, rank, world):
         stops[i].record()
     B.set_profile_events(None, None)
     barrier()
+    if sampler:
+        sampler.mark()
     clocks = sampler.stop() if sampler else None
     assert sess.cache.status() == 0, f"device status {sess.cache.status()}"
     step_ms = [s_.elapsed_time(e_) for s_, e_ in zip(starts, stops)]

@@ -192,10 +192,26 @@ int wushkv_unpack_debug(const wushkv_cache* cache, int32_t slot, int32_t kv_head
                         int32_t pos0, int32_t n, uint8_t* codes, float* scale, float* zero, void* stream);
 
 /*
+ * One whole decode step from DEVICE buffers: Algorithm 2 lines 3-5 and 7-12 for one new token per
+ * sequence, i.e. wushkv_append of one token per sequence followed by wushkv_decode_attn over the
+ * extended cache, with the same results as those two calls.  Because the library knows here what
+ * runs ahead of the query preparation (its own append kernel, which begins only after all earlier
+ * work in the stream has finished), it transforms the queries while the new token is being
+ * quantized instead of after it.
+ *   K_new, V_new (device): bf16 [batch][n_kv][d].   Q (device): bf16 [batch][n_q][d], 16-byte aligned.
+ *   O (device, out): fp32 [batch][n_q][d].   cu_new (device): int32 [batch+1] = 0, 1, ..., batch.
+ *   slot, seq_len (in/out), max_seq_len (bound on the lengths AFTER the append), workspace: as for
+ *   wushkv_append / wushkv_decode_attn.  The decode half is validated before anything is appended.
+ */
+int wushkv_decode_step(const wushkv_cache* cache, int32_t batch, const int32_t* slot, int32_t* seq_len,
+                       const int32_t* cu_new, int32_t max_seq_len,
+                       const uint16_t* K_new, const uint16_t* V_new, const uint16_t* Q, float* O,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * One whole decode step from HOST buffers: Algorithm 2 lines 3-5 and 7-12 for one new token per
  * sequence.  Enqueues, in order, on `stream`: host->device copies of K_new, V_new and Q into
- * `staging`, wushkv_append of one token per sequence, wushkv_decode_attn, and the device->host
- * copy of O.  Does not synchronise; O_host is valid once the stream has been synchronised.
+ * `staging`, wushkv_decode_step on the staged copies, and the device->host copy of O.  Does not synchronise; O_host is valid once the stream has been synchronised.
  *   K_new_host, V_new_host (host, pinned for the copies to be asynchronous): bf16 [batch][n_kv][d].
  *   Q_host (host): bf16 [batch][n_q][d].   O_host (host, out): fp32 [batch][n_q][d].
  *   cu_new (device): int32 [batch+1] = 0, 1, ..., batch.

@@ -18,7 +18,7 @@ DEV_PAGE_TABLE_FULL, DEV_BAD_PAGE_ID, DEV_BAD_SLOT, DEV_COPY_TIMEOUT = 1, 2, 4, 
 EXPORTS = (
     "wushkv_page_bytes", "wushkv_status_string", "wushkv_accumulate_gram", "wushkv_build_transforms",
     "wushkv_append", "wushkv_decode_workspace_bytes", "wushkv_decode_attn", "wushkv_unpack_debug",
-    "wushkv_step_staging_bytes", "wushkv_decode_step_host", "wushkv_set_profile_events",
+    "wushkv_decode_step", "wushkv_step_staging_bytes", "wushkv_decode_step_host", "wushkv_set_profile_events",
     "wushkv_decode_attn_static",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
@@ -72,6 +72,9 @@ def _load():
     lib.wushkv_unpack_debug.restype = C.c_int
     lib.wushkv_unpack_debug.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                         C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.wushkv_decode_step.restype = C.c_int
+    lib.wushkv_decode_step.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
     lib.wushkv_step_staging_bytes.restype = C.c_size_t
     lib.wushkv_step_staging_bytes.argtypes = [C.POINTER(wushkv_cache), C.c_int32]
     lib.wushkv_decode_step_host.restype = C.c_int
@@ -166,6 +169,14 @@ def decode_attn_static(cache: wushkv_cache, batch, slot, seq_len, max_seq_len, Q
     STATIC_SCRATCH_BYTES raise with status ECAPACITY; overlapping calls on one GPU race)."""
     _check(lib.wushkv_decode_attn_static(C.byref(cache), batch, _ptr(slot), _ptr(seq_len), max_seq_len, _ptr(Q),
                                          _ptr(O), _stream_ptr(stream)), "wushkv_decode_attn_static")
+
+
+def decode_step(cache: wushkv_cache, batch, slot, seq_len, cu_new, max_seq_len, K_new, V_new, Q, O, workspace,
+                workspace_bytes, stream=None):
+    """wushkv_decode_step: append one token per sequence, then decode over the extended cache (device tensors)."""
+    _check(lib.wushkv_decode_step(C.byref(cache), batch, _ptr(slot), _ptr(seq_len), _ptr(cu_new), max_seq_len,
+                                  _ptr(K_new), _ptr(V_new), _ptr(Q), _ptr(O), _ptr(workspace), workspace_bytes,
+                                  _stream_ptr(stream)), "wushkv_decode_step")
 
 
 def step_staging_bytes(cache: wushkv_cache, batch: int) -> int:

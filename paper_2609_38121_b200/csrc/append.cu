@@ -249,7 +249,11 @@ __global__ void __launch_bounds__(256) append_rows_kernel(AppendParams P) {
 template <int BITS>
 __global__ void __launch_bounds__(1024) append_token_kernel(AppendParams P) {
     extern __shared__ __align__(16) float tok_s[];       // [n_kv][128] input key, [n_kv][128] transformed key
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a dependent launched programmatically may start; it waits for us itself
+    // Launched programmatically: the CTAs may be resident before the kernel ahead in the stream has
+    // finished, so wait for it (and its memory) first; then let the next kernel's CTAs come in early
+    // too (that kernel waits for this one itself).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int b = blockIdx.x;
     const int n_kv = P.c.n_kv;
     float* kin_s = tok_s;
@@ -796,9 +800,19 @@ extern "C" int wushkv_append(const wushkv_cache* cache, int32_t batch, const int
         const int threads = std::min(1024, P.c.n_kv * D);
         const size_t smem1 = static_cast<size_t>(2) * P.c.n_kv * D * sizeof(float);
         if (smem1 > 48 * 1024) return WUSHKV_EINVAL;
-        if (P.c.bits == 2) append_token_kernel<2><<<batch, threads, smem1, st>>>(P);
-        else append_token_kernel<4><<<batch, threads, smem1, st>>>(P);
-        return cudaGetLastError() == cudaSuccess ? WUSHKV_OK : WUSHKV_ECUDA;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(batch);
+        cfg.blockDim = dim3(threads);
+        cfg.dynamicSmemBytes = smem1;
+        cfg.stream = st;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const cudaError_t e1 = P.c.bits == 2 ? cudaLaunchKernelEx(&cfg, append_token_kernel<2>, P)
+                                             : cudaLaunchKernelEx(&cfg, append_token_kernel<4>, P);
+        return e1 == cudaSuccess ? WUSHKV_OK : WUSHKV_ECUDA;
     }
     const char* path_env = std::getenv("WUSHKV_APPEND_PATH");          // "cuda" forces the CUDA-core chunk path (testing)
     const bool force_cuda = path_env && path_env[0] == 'c';

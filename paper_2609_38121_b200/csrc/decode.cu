@@ -63,6 +63,7 @@ struct DecodeParams {
     long long* plan;     // [batch+1]: exclusive prefix of work units per sequence (per KV head)
     float* part;         // [n_warps + batch*n_kv][G][PART_STRIDE]
     int n_warps;         // warps of the main kernel
+    int q_early;         // 1: Q was final before the kernel ahead of the preparation kernel started
 };
 
 // shift of the code field used by k-step / channel block idx (0..7) inside its 16-bit lane, after
@@ -107,58 +108,42 @@ __device__ __forceinline__ SeqInfo seq_info(const CacheView& c, int S, int slot)
 // ------------------------------------------------------------------------------------------------
 // 1. query preparation
 // ------------------------------------------------------------------------------------------------
+constexpr int PREP_THREADS = 512;                   // 16 warps share the 128 rows of T_K^{-T}
+constexpr int PREP_ROWS = D / (PREP_THREADS / 32);   // rows per warp
 template <int BITS, int MODE>
-__global__ void __launch_bounds__(128) decode_prep_kernel(DecodeParams P) {
+__global__ void __launch_bounds__(PREP_THREADS) decode_prep_kernel(DecodeParams P) {
     __shared__ float q_s[8][D];
     __shared__ float red_max[8][4];
     __shared__ float red_sum[8][4];
     __shared__ long long scan_s[4];
     const int h = blockIdx.x, b = blockIdx.y, G = P.c.G;
     const int i = threadIdx.x, lane = i & 31, warp = i >> 5;
-    pdl_wait();                           // everything this kernel reads may come from the kernel before it
-    pdl_launch_dependents();              // the main kernel may start staging pages while this one runs
+    // Normally everything this kernel reads may come from the kernel ahead of it.  In the fused step
+    // (q_early) that kernel is the single-token append, which started only after all earlier work had
+    // finished: Q is final already and only the lengths (for the work plan) have to wait for it, so the
+    // transform of the queries runs beside the append.  The main kernel reads the lengths and stages
+    // pages as soon as it starts, so the plan CTA holds its launch signal back until the append is done.
+    const bool plan_cta = h == 0 && b == 0;
+    if (!P.q_early) pdl_wait();
+    if (!(P.q_early && plan_cta)) pdl_launch_dependents();   // the main kernel may start staging pages while this one runs
 
-    if (h == 0 && b == 0) {               // work plan: exclusive prefix of units per sequence
-        long long carry = 0;
-        for (int base = 0; base < P.batch; base += 128) {
-            const int bb = base + i;
-            long long u = 0;
-            if (bb < P.batch) {
-                const int slot = __ldg(P.slot + bb);
-                if (slot < 0 || slot >= P.c.n_slots) atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_SLOT);
-                u = seq_info(P.c, __ldg(P.seq_len + bb), slot).U;
-            }
-            long long incl = u;
-            for (int o = 1; o < 32; o <<= 1) {
-                const long long v = __shfl_up_sync(FULL, incl, o);
-                if (lane >= o) incl += v;
-            }
-            if (lane == 31) scan_s[warp] = incl;
-            __syncthreads();
-            long long before = 0;
-            for (int w = 0; w < warp; ++w) before += scan_s[w];
-            if (bb < P.batch) P.plan[bb + 1] = carry + before + incl;
-            carry += scan_s[0] + scan_s[1] + scan_s[2] + scan_s[3];
-            __syncthreads();
-        }
-        if (i == 0) P.plan[0] = 0;
-    }
-
-    for (int g = 0; g < G; ++g)
-        q_s[g][i] = bf16_bits_to_float(P.Q[(static_cast<long long>(b) * P.c.n_q + h * G + g) * D + i]);
+    for (int k = i; k < G * D; k += PREP_THREADS)
+        q_s[k >> 7][k & (D - 1)] = bf16_bits_to_float(P.Q[(static_cast<long long>(b) * P.c.n_q + h * G) * D + k]);
     __syncthreads();
-    // q'[g][i] = sum_j T_invT[h][i][j] q[g][j].  Each warp takes 32 rows; a row is one coalesced
-    // 512-byte read (lane L holds columns 4L..4L+3); rows are handled 32/GP at a time so that the
-    // GP x rows partial sums fit a 32-value transposing butterfly (GP = 4 or 8 head slots).
+    // q'[g][i] = sum_j T_invT[h][i][j] q[g][j].  Each of the 16 warps takes 8 rows, all of their loads in
+    // flight together; a row is one coalesced 512-byte read (lane L holds columns 4L..4L+3); rows are
+    // handled 32/GP at a time so that the GP x rows partial sums fit a 32-value transposing butterfly
+    // (GP = 4 or 8 head slots).
     __shared__ float qp_s[8][D];
     {
         constexpr int GP = MODE == 0 ? 4 : 8;           // MODE 0 serves G <= 4, MODE 1 serves G <= 8
         constexpr int rows_per = 32 / GP;
-        const float4* Tbase = reinterpret_cast<const float4*>(P.c.T_K_invT + (static_cast<long long>(h) * D + warp * 32) * D) + lane;
+        const float4* Tbase = reinterpret_cast<const float4*>(P.c.T_K_invT + (static_cast<long long>(h) * D + warp * PREP_ROWS) * D) + lane;
         float4 qv[8];
 #pragma unroll
         for (int g = 0; g < 8; ++g) qv[g] = g < G ? *reinterpret_cast<const float4*>(&q_s[g][4 * lane]) : make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int r0 = 0; r0 < 32; r0 += rows_per) {
+#pragma unroll
+        for (int r0 = 0; r0 < PREP_ROWS; r0 += rows_per) {
             float part[32];
 #pragma unroll
             for (int k = 0; k < 32; ++k) part[k] = 0.f;
@@ -174,10 +159,37 @@ __global__ void __launch_bounds__(128) decode_prep_kernel(DecodeParams P) {
             }
             const float tot = warp_transpose_reduce(part, lane);
             const int rr = lane / GP, g = lane % GP;
-            if (g < G) qp_s[g][warp * 32 + r0 + rr] = tot;
+            if (g < G) qp_s[g][warp * PREP_ROWS + r0 + rr] = tot;
         }
     }
     __syncthreads();
+    if (plan_cta) {                       // work plan: exclusive prefix of units per sequence
+        if (P.q_early) { pdl_wait(); pdl_launch_dependents(); }     // the lengths come from the append
+        long long carry = 0;
+        for (int base = 0; base < P.batch; base += 128) {
+            const int bb = base + i;
+            long long u = 0;
+            if (i < 128 && bb < P.batch) {
+                const int slot = __ldg(P.slot + bb);
+                if (slot < 0 || slot >= P.c.n_slots) atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_SLOT);
+                u = seq_info(P.c, __ldg(P.seq_len + bb), slot).U;
+            }
+            long long incl = u;
+            for (int o = 1; o < 32; o <<= 1) {
+                const long long v = __shfl_up_sync(FULL, incl, o);
+                if (lane >= o) incl += v;
+            }
+            if (lane == 31 && warp < 4) scan_s[warp] = incl;
+            __syncthreads();
+            long long before = 0;
+            for (int w = 0; w < warp && w < 4; ++w) before += scan_s[w];
+            if (i < 128 && bb < P.batch) P.plan[bb + 1] = carry + before + incl;
+            carry += scan_s[0] + scan_s[1] + scan_s[2] + scan_s[3];
+            __syncthreads();
+        }
+        if (i == 0) P.plan[0] = 0;
+    }
+    if (i >= 128) return;                 // the fragment stage has one thread per channel
     float acc[8];
 #pragma unroll
     for (int g = 0; g < 8; ++g) acc[g] = g < G ? qp_s[g][i] : 0.f;
@@ -195,7 +207,7 @@ __global__ void __launch_bounds__(128) decode_prep_kernel(DecodeParams P) {
             if (lane == 0) { red_max[g][warp] = mx; red_sum[g][warp] = sm; }
         }
     }
-    __syncthreads();
+    asm volatile("bar.sync 1, 128;" ::: "memory");       // the four remaining warps only
     float beta[8];
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
@@ -689,33 +701,29 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ?
                     unsigned vmeta[4][2];         // fp16x2 (Delta_v, x_min_v) of rows g, g+8
 #pragma unroll
                     for (int bi = 0; bi < 4; ++bi) {
-                        float acc[4], acc2[4];                                                  // two chains for ILP
+                        float acc[4];                 // one chain per block; the four blocks of a page are independent
                         if (BITS == 2) {
                             const uint4 kw = lds128(rec + bi * CB + 16 * lane);
                             const unsigned sx = pre_shift<2>(kw.x), sy = pre_shift<2>(kw.y), sz = pre_shift<2>(kw.z), sw = pre_shift<2>(kw.w);
                             mma_f16_zero(acc, field<2>(kw.x, sx, 0), field<2>(kw.z, sz, 0), field<2>(kw.y, sy, 0), field<2>(kw.w, sw, 0), qf[0][0], qf[0][1]);
-                            mma_f16_zero(acc2, field<2>(kw.x, sx, 1), field<2>(kw.z, sz, 1), field<2>(kw.y, sy, 1), field<2>(kw.w, sw, 1), qf[1][0], qf[1][1]);
 #pragma unroll
-                            for (int ks = 2; ks < 8; ks += 2) {
+                            for (int ks = 1; ks < 8; ++ks)
                                 mma_f16(acc, field<2>(kw.x, sx, ks), field<2>(kw.z, sz, ks), field<2>(kw.y, sy, ks), field<2>(kw.w, sw, ks),
                                         qf[ks][0], qf[ks][1]);
-                                mma_f16(acc2, field<2>(kw.x, sx, ks + 1), field<2>(kw.z, sz, ks + 1), field<2>(kw.y, sy, ks + 1), field<2>(kw.w, sw, ks + 1),
-                                        qf[ks + 1][0], qf[ks + 1][1]);
-                            }
                         } else {
                             const uint4 ka = lds128(rec + bi * CB + 16 * lane);          // row g:   W0..W3
                             const uint4 kb = lds128(rec + bi * CB + 512 + 16 * lane);    // row g+8: W0..W3
                             const unsigned a0s = pre_shift<4>(ka.x), a1s = pre_shift<4>(ka.y), a2s = pre_shift<4>(ka.z), a3s = pre_shift<4>(ka.w);
                             const unsigned b0s = pre_shift<4>(kb.x), b1s = pre_shift<4>(kb.y), b2s = pre_shift<4>(kb.z), b3s = pre_shift<4>(kb.w);
                             mma_f16_zero(acc, field<4>(ka.x, a0s, 0), field<4>(kb.x, b0s, 0), field<4>(ka.y, a1s, 0), field<4>(kb.y, b1s, 0), qf[0][0], qf[0][1]);
-                            mma_f16_zero(acc2, field<4>(ka.z, a2s, 0), field<4>(kb.z, b2s, 0), field<4>(ka.w, a3s, 0), field<4>(kb.w, b3s, 0), qf[4][0], qf[4][1]);
 #pragma unroll
-                            for (int ks = 1; ks < 4; ++ks) {
+                            for (int ks = 1; ks < 4; ++ks)
                                 mma_f16(acc, field<4>(ka.x, a0s, ks), field<4>(kb.x, b0s, ks), field<4>(ka.y, a1s, ks), field<4>(kb.y, b1s, ks),
                                         qf[ks][0], qf[ks][1]);
-                                mma_f16(acc2, field<4>(ka.z, a2s, ks), field<4>(kb.z, b2s, ks), field<4>(ka.w, a3s, ks), field<4>(kb.w, b3s, ks),
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks)
+                                mma_f16(acc, field<4>(ka.z, a2s, ks), field<4>(kb.z, b2s, ks), field<4>(ka.w, a3s, ks), field<4>(kb.w, b3s, ks),
                                         qf[4 + ks][0], qf[4 + ks][1]);
-                            }
                         }
                         if (MODE == 1) {
                             // two heads per column pair leave no room for a remainder column: a second pass over
@@ -748,8 +756,6 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ?
 #pragma unroll
                             for (int e = 0; e < 4; ++e) acc[e] = fmaf(accr[e] + accr2[e], 1.f / LO_SCALE, acc[e]);
                         }
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) acc[e] += acc2[e];
                         const uint4 mt = lds128(rec + meta_offset(BITS) + 128 * bi + 16 * g);   // rows g (x,y) and g+8 (z,w)
                         const float2 km_a = h2f2(mt.x), km_b = h2f2(mt.z);
                         const float kd0 = km_a.x, km0 = km_a.y, kd1 = km_b.x, km1 = km_b.y;
@@ -856,6 +862,7 @@ __global__ void __launch_bounds__(128) decode_combine_kernel(DecodeParams P) {
     const CacheView& c = P.c;
     const int j = blockIdx.x, b = blockIdx.y, ch = threadIdx.x;
     pdl_wait();                                         // partials and the plan come from the earlier kernels
+    pdl_launch_dependents();                            // a programmatically launched successor waits for us itself
     float* out = P.O + (static_cast<long long>(b) * c.n_q + j) * D;
     const long long U = P.plan[b + 1] - P.plan[b];
     const long long total = P.plan[P.batch] * c.n_kv;
@@ -953,11 +960,17 @@ static int launch_decode(const DecodeParams& P, int n_ctas, cudaStream_t st) {
     cfg.attrs = pdl_attr;
     cfg.numAttrs = 1;
     cfg.gridDim = dim3(P.c.n_kv, P.batch);
-    cfg.blockDim = dim3(128);
+    cfg.blockDim = dim3(PREP_THREADS);
     cfg.dynamicSmemBytes = 0;
     if (cudaLaunchKernelEx(&cfg, decode_prep_kernel<BITS, MODE>, P) != cudaSuccess) return WUSHKV_ECUDA;
-    if (cudaFuncSetAttribute(decode_main_kernel<BITS, MODE, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(SMEM)) != cudaSuccess)
-        return WUSHKV_ECUDA;
+    static bool smem_opted_in[64] = {};      // once per device and kernel instance
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return WUSHKV_ECUDA;
+    if (dev < 0 || dev >= 64 || !smem_opted_in[dev]) {
+        if (cudaFuncSetAttribute(decode_main_kernel<BITS, MODE, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(SMEM)) != cudaSuccess)
+            return WUSHKV_ECUDA;
+        if (dev >= 0 && dev < 64) smem_opted_in[dev] = true;
+    }
     if (g_prof_start) cudaEventRecord(g_prof_start, st);
     cfg.gridDim = dim3(n_ctas);
     cfg.blockDim = dim3(MAIN_WARPS * 32);
@@ -983,10 +996,11 @@ extern "C" size_t wushkv_decode_workspace_bytes(const wushkv_cache* cache, int32
     return pl.total;
 }
 
-extern "C" int wushkv_decode_attn(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
-                                  int32_t max_seq_len, const uint16_t* Q, float* O,
-                                  void* workspace, size_t workspace_bytes, void* stream) {
+static int decode_attn_impl(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
+                            int32_t max_seq_len, const uint16_t* Q, float* O,
+                            void* workspace, size_t workspace_bytes, void* stream, int q_early) {
     DecodeParams P;
+    P.q_early = q_early;
     const int rc = make_view(cache, P.c);
     if (rc != WUSHKV_OK) return rc;
     if (!slot || !seq_len || !Q || !O || !workspace || !aligned(Q, 16) || !aligned(O, 16) || !aligned(workspace, 256)) return WUSHKV_EINVAL;
@@ -1006,6 +1020,31 @@ extern "C" int wushkv_decode_attn(const wushkv_cache* cache, int32_t batch, cons
     const bool mode0 = P.c.G <= 4;
     if (P.c.bits == 2) return mode0 ? launch_decode<2, 0>(P, pl.n_ctas, st) : launch_decode<2, 1>(P, pl.n_ctas, st);
     return mode0 ? launch_decode<4, 0>(P, pl.n_ctas, st) : launch_decode<4, 1>(P, pl.n_ctas, st);
+}
+
+extern "C" int wushkv_decode_attn(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
+                                  int32_t max_seq_len, const uint16_t* Q, float* O,
+                                  void* workspace, size_t workspace_bytes, void* stream) {
+    return decode_attn_impl(cache, batch, slot, seq_len, max_seq_len, Q, O, workspace, workspace_bytes, stream, 0);
+}
+
+extern "C" int wushkv_decode_step(const wushkv_cache* cache, int32_t batch, const int32_t* slot, int32_t* seq_len,
+                                  const int32_t* cu_new, int32_t max_seq_len,
+                                  const uint16_t* K_new, const uint16_t* V_new, const uint16_t* Q, float* O,
+                                  void* workspace, size_t workspace_bytes, void* stream) {
+    if (batch <= 0 || !Q || !O || !workspace) return WUSHKV_EINVAL;
+    // validate the decode half before anything is appended
+    CacheView v;
+    int r = make_view(cache, v);
+    if (r != WUSHKV_OK) return r;
+    DecodePlan pl;
+    if (!make_plan(v, batch, max_seq_len, pl) || batch > 65535 || !aligned(Q, 16) || !aligned(O, 16) || !aligned(workspace, 256)) return WUSHKV_EINVAL;
+    if (workspace_bytes < pl.total) return WUSHKV_ECAPACITY;
+    r = wushkv_append(cache, batch, slot, seq_len, cu_new, batch, 1, K_new, V_new, stream);
+    if (r != WUSHKV_OK) return r;
+    // the single-token append kernel is now the kernel ahead of the query preparation, and it started
+    // only after all earlier work in the stream: the preparation may read Q without waiting for it
+    return decode_attn_impl(cache, batch, slot, seq_len, max_seq_len, Q, O, workspace, workspace_bytes, stream, 1);
 }
 
 extern "C" int wushkv_set_profile_events(void* start, void* stop) {
@@ -1046,9 +1085,7 @@ extern "C" int wushkv_decode_step_host(const wushkv_cache* cache, int32_t batch,
     if (cudaMemcpyAsync(dK, K_new_host, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return WUSHKV_ECUDA;
     if (cudaMemcpyAsync(dV, V_new_host, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return WUSHKV_ECUDA;
     if (cudaMemcpyAsync(dQ, Q_host, q_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return WUSHKV_ECUDA;
-    int r = wushkv_append(cache, batch, slot, seq_len, cu_new, batch, 1, dK, dV, stream);
-    if (r != WUSHKV_OK) return r;
-    r = wushkv_decode_attn(cache, batch, slot, seq_len, max_seq_len, dQ, dO, workspace, workspace_bytes, stream);
+    const int r = wushkv_decode_step(cache, batch, slot, seq_len, cu_new, max_seq_len, dK, dV, dQ, dO, workspace, workspace_bytes, stream);
     if (r != WUSHKV_OK) return r;
     if (cudaMemcpyAsync(O_host, dO, o_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return WUSHKV_ECUDA;
     return WUSHKV_OK;

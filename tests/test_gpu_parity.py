@@ -134,6 +134,50 @@ def test_decode_is_deterministic_and_split_invariant(monkeypatch):
     assert np.max(np.abs(outs[3] - outs[0])) <= 5e-4 * scale
 
 
+@pytest.mark.parametrize("bits,n_q,n_kv", [(2, 8, 2), (4, 14, 2)])
+def test_fused_step_equals_append_then_decode(bits, n_q, n_kv):
+    """wushkv_decode_step (queries transformed beside the append) gives, bit for bit, the cache and the
+    outputs of wushkv_append + wushkv_decode_attn; several steps are enqueued back to back."""
+    import torch
+    from paper_2609_38121_b200 import binding as B
+    wl = _wl(n_q, n_kv, seed=41)
+    lengths, steps = [700, 67, 3, 333], 3
+    first = [n - steps for n in lengths]
+    two, one = Layer(wl, lengths, bits, 4, 64, 1), Layer(wl, lengths, bits, 4, 64, 1)
+    two.append_step(first, oracle_too=False)
+    one.append_step(first, oracle_too=False)
+    dev = one.cache.device
+    qs = [np.stack([wl.queries(b, first[b] + i) for b in range(len(lengths))]) for i in range(steps)]
+    ref = []
+    for i in range(steps):
+        two.append_step([1] * len(lengths), oracle_too=False)
+        ref.append(two.decode(queries=qs[i])[0])
+    bits16 = lambda x: torch.from_numpy(W.f32_to_bf16_bits(x).view(np.int16)).to(dev)  # noqa: E731
+    Ks = [bits16(np.stack([one.tokens[b][0][first[b] + i] for b in range(len(lengths))])) for i in range(steps)]
+    Vs = [bits16(np.stack([one.tokens[b][1][first[b] + i] for b in range(len(lengths))])) for i in range(steps)]
+    Qs = [bits16(q) for q in qs]
+    outs = [torch.full((len(lengths), n_q, 128), float("nan"), dtype=torch.float32, device=dev) for _ in range(steps)]
+    cu = torch.arange(len(lengths) + 1, dtype=torch.int32, device=dev)
+    nbytes = B.decode_workspace_bytes(one.cache.desc, one.batch, one.max_seq_len)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    torch.cuda.synchronize()
+    for i in range(steps):                                   # no host synchronisation between the steps
+        B.decode_step(one.cache.desc, one.batch, one.slot, one.seq_len, cu, one.max_seq_len, Ks[i], Vs[i], Qs[i],
+                      outs[i], ws, nbytes)
+    torch.cuda.synchronize()
+    assert one.cache.status() == 0
+    assert one.seq_len.cpu().tolist() == lengths
+    for i in range(steps):
+        assert np.array_equal(outs[i].cpu().numpy().astype(np.float64), ref[i]), f"step {i}"
+    for b in range(len(lengths)):
+        for h in range(n_kv):
+            for which in (0, 1):
+                for x, y in zip(one.gpu_codes(b, h, which), two.gpu_codes(b, h, which)):
+                    assert np.array_equal(x, y)
+        for x, y in zip(one.gpu_window_arrays(b), two.gpu_window_arrays(b)):
+            assert np.array_equal(x, y, equal_nan=True)
+
+
 def test_device_side_errors_are_flagged_not_fatal():
     """A position beyond the page table and a page id outside the pool set status bits; the calls
     still return and the rest of the batch is processed."""
