@@ -38,7 +38,13 @@ constexpr unsigned FULL = 0xffffffffu;
 constexpr int PART_STRIDE = 132;          // floats per partial: [0]=max (log2 domain) [1]=sum [4..131]=o
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LO_SCALE = 2048.f;        // a "remainder" column carries (x - rounded(x)) * 2^11
-constexpr float PV_SCALE = 16.f;          // p * Delta_v is fed to the tensor core as fp16(p Delta_v 2^4)
+// Exponentials are taken against (running reference - LOG2_PV): every probability, and with it l, z and
+// o of a partial, carries the common factor 2^LOG2_PV, which cancels in the final ratio and keeps
+// fp16(p Delta_v) out of the subnormals.  The reference is only raised (and the state rescaled) when
+// a unit's maximum exceeds it by more than MAX_SLACK, so p <= 2^(LOG2_PV + MAX_SLACK) and
+// p Delta_v stays finite in fp16 for Delta_v < 2^(16 - LOG2_PV - MAX_SLACK) = 1024.
+constexpr float LOG2_PV = 3.f;
+constexpr float MAX_SLACK = 3.f;
 constexpr int MAIN_WARPS = 4;
 constexpr int WIN_TOKENS = 8;             // window tokens per work unit
 constexpr int WIN_ROW = 272;              // padded bytes per staged bf16 row (conflict-free ldmatrix)
@@ -365,36 +371,35 @@ template <int BITS> __device__ __forceinline__ unsigned pre_shift(unsigned w) { 
 
 // Per-warp running softmax state of one (sequence, KV head).  MODE 0: one head per thread (head t,
 // value and rounding-remainder columns).  MODE 1: two heads per thread (2t, 2t+1).
-// o[i][.] accumulates channel block i in units of 2^(field_shift(i) - 24) / PV_SCALE.
+// o[i][.] accumulates channel block i in units of 2^(field_shift(i) - 24); l, z and o carry the
+// common factor 2^LOG2_PV.  m is the reference of the partial, not necessarily its exact maximum.
 template <int MODE>
 struct WarpState {
     static constexpr int NH = MODE == 0 ? 1 : 2;
-    float m[NH], l[NH], z[NH];
+    float m[NH], mr[NH], l[NH], z[NH];
     float o[8][4];
     __device__ __forceinline__ void reset() {
 #pragma unroll
-        for (int k = 0; k < NH; ++k) { m[k] = -INFINITY; l[k] = 0.f; z[k] = 0.f; }
+        for (int k = 0; k < NH; ++k) { m[k] = -INFINITY; mr[k] = 0.f; l[k] = 0.f; z[k] = 0.f; }
 #pragma unroll
         for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
     }
-    // Raise the running maximum to cover this unit's per-head maxima (already reduced over the unit's
-    // tokens); mref receives the reference each head's exponentials use.
-    __device__ __forceinline__ void raise_max(const float (&mx)[NH], float (&mref)[NH]) {
+    // Make the running reference cover this unit's per-head maxima (already reduced over the unit's
+    // tokens) to within MAX_SLACK; mr is what the exponentials subtract.
+    __device__ __forceinline__ void raise_max(const float (&mx)[NH]) {
         bool grew = false;
-        float mnew[NH];
 #pragma unroll
-        for (int k = 0; k < NH; ++k) {
-            mnew[k] = fmaxf(m[k], mx[k]);
-            grew |= mnew[k] > m[k];
-            mref[k] = (mnew[k] == -INFINITY) ? 0.f : mnew[k];       // all masked so far: any finite reference works
-        }
+        for (int k = 0; k < NH; ++k) grew |= mx[k] > m[k] + MAX_SLACK;      // reference -inf: any finite score
         if (__any_sync(FULL, grew)) {
             float scl[NH];
 #pragma unroll
             for (int k = 0; k < NH; ++k) {
-                scl[k] = ex2(m[k] - mref[k]);                        // old max -inf: state is all zero, factor 0
+                const float mnew = fmaxf(m[k], mx[k]);
+                const float ref = (mnew == -INFINITY) ? 0.f : mnew;          // all masked so far: any finite reference works
+                scl[k] = ex2(m[k] - ref);                                    // old reference -inf: state is all zero, factor 0
                 l[k] *= scl[k]; z[k] *= scl[k];
-                m[k] = mnew[k];
+                m[k] = mnew;
+                mr[k] = ref - LOG2_PV;
             }
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
@@ -422,7 +427,7 @@ __device__ __forceinline__ void store_partial(const WarpState<MODE>& st, float* 
             if (g == 0) { dst[0] = st.m[k]; dst[1] = l; }
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                const float osc = exp2f(static_cast<float>(24 - field_shift<BITS>(i))) / PV_SCALE;
+                const float osc = exp2f(static_cast<float>(24 - field_shift<BITS>(i)));
                 float lo_ch, hi_ch;
                 if (MODE == 0) {
                     lo_ch = (st.o[i][0] + st.o[i][1] * (1.f / LO_SCALE)) * osc + z;
@@ -664,7 +669,7 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ?
                         }
                     }
                     const bool ok = g < n_valid;
-                    float sc[NH], mx[NH], mref[NH];
+                    float sc[NH], mx[NH];
                     if (MODE == 0) sc[0] = ok ? acc[0] + acc[1] : -INFINITY;
                     else { sc[0] = ok ? acc[0] : -INFINITY; sc[NH - 1] = ok ? acc[1] : -INFINITY; }
 #pragma unroll
@@ -674,10 +679,10 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ?
                         mx[k] = fmaxf(mx[k], __shfl_xor_sync(FULL, mx[k], 8));
                         mx[k] = fmaxf(mx[k], __shfl_xor_sync(FULL, mx[k], 16));
                     }
-                    st.raise_max(mx, mref);
+                    st.raise_max(mx);
                     float p[NH];
 #pragma unroll
-                    for (int k = 0; k < NH; ++k) { p[k] = ex2(sc[k] - mref[k]); st.l[k] += p[k]; }
+                    for (int k = 0; k < NH; ++k) { p[k] = ex2(sc[k] - st.mr[k]); st.l[k] += p[k]; }
 #pragma unroll
                     for (int pass = 0; pass < (MODE == 0 ? 1 : 2); ++pass) {
                         unsigned pr;                                      // this token's probabilities in the score-fragment layout
@@ -689,9 +694,9 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ?
                         for (int i2 = 0; i2 < 4; ++i2) {
                             unsigned v0, v1, v2, v3;                      // (block 2i2: ch lo, ch hi), (block 2i2+1: ch lo, ch hi)
                             ldmatrix_x4_trans(rec + WIN_V_OFF + frag_off + i2 * 64, v0, v1, v2, v3);
-                            // fold the block's accumulator unit in: p * v * PV_SCALE * 2^(shift - 24)
-                            mma_bf16(st.o[2 * i2], v0, v1, v0, v1, mul_bf2(b01, bf16x2_pow2(field_shift<BITS>(2 * i2) - 20)), 0u);
-                            mma_bf16(st.o[2 * i2 + 1], v2, v3, v2, v3, mul_bf2(b01, bf16x2_pow2(field_shift<BITS>(2 * i2 + 1) - 20)), 0u);
+                            // fold the block's accumulator unit in: p * v * 2^(shift - 24)
+                            mma_bf16(st.o[2 * i2], v0, v1, v0, v1, mul_bf2(b01, bf16x2_pow2(field_shift<BITS>(2 * i2) - 24)), 0u);
+                            mma_bf16(st.o[2 * i2 + 1], v2, v3, v2, v3, mul_bf2(b01, bf16x2_pow2(field_shift<BITS>(2 * i2 + 1) - 24)), 0u);
                         }
                     }
                 } else if (!__any_sync(FULL, (bad_bits >> s) & 1u)) {
@@ -759,33 +764,36 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ?
                         const uint4 mt = lds128(rec + meta_offset(BITS) + 128 * bi + 16 * g);   // rows g (x,y) and g+8 (z,w)
                         const float2 km_a = h2f2(mt.x), km_b = h2f2(mt.z);
                         const float kd0 = km_a.x, km0 = km_a.y, kd1 = km_b.x, km1 = km_b.y;
-                        unsigned vm0 = mt.y, vm1 = mt.w;
-                        bool ok0 = true, ok1 = true;
-                        if (!full_page) {
-                            const int p0 = pos0 + bi * 16 + g, p1 = p0 + 8;
-                            ok0 = (p0 >= q_lo) && (p0 < q_hi);
-                            ok1 = (p1 >= q_lo) && (p1 < q_hi);
-                            if (!ok0) vm0 = 0u;
-                            if (!ok1) vm1 = 0u;
-                        }
-                        vmeta[bi][0] = vm0; vmeta[bi][1] = vm1;
+                        vmeta[bi][0] = mt.y; vmeta[bi][1] = mt.w;
                         if (MODE == 0) {
                             const float d0 = fmaf(acc[1], 1.f / LO_SCALE, acc[0]), d1 = fmaf(acc[3], 1.f / LO_SCALE, acc[2]);
-                            const float s0 = fmaf(d0 * kd0, fmul[0], km0 * gadd[0]);
-                            const float s1 = fmaf(d1 * kd1, fmul[0], km1 * gadd[0]);
-                            sc[bi][0] = ok0 ? s0 : -INFINITY;
-                            sc[bi][NH] = ok1 ? s1 : -INFINITY;
+                            sc[bi][0] = fmaf(d0 * kd0, fmul[0], km0 * gadd[0]);
+                            sc[bi][NH] = fmaf(d1 * kd1, fmul[0], km1 * gadd[0]);
                         } else {
-                            const float s00 = fmaf(acc[0] * kd0, fmul[0], km0 * gadd[0]);
-                            const float s01 = fmaf(acc[1] * kd0, fmul[NH - 1], km0 * gadd[NH - 1]);
-                            const float s10 = fmaf(acc[2] * kd1, fmul[0], km1 * gadd[0]);
-                            const float s11 = fmaf(acc[3] * kd1, fmul[NH - 1], km1 * gadd[NH - 1]);
-                            sc[bi][0] = ok0 ? s00 : -INFINITY; sc[bi][NH - 1] = ok0 ? s01 : -INFINITY;
-                            sc[bi][NH] = ok1 ? s10 : -INFINITY; sc[bi][2 * NH - 1] = ok1 ? s11 : -INFINITY;
+                            sc[bi][0] = fmaf(acc[0] * kd0, fmul[0], km0 * gadd[0]);
+                            sc[bi][NH - 1] = fmaf(acc[1] * kd0, fmul[NH - 1], km0 * gadd[NH - 1]);
+                            sc[bi][NH] = fmaf(acc[2] * kd1, fmul[0], km1 * gadd[0]);
+                            sc[bi][2 * NH - 1] = fmaf(acc[3] * kd1, fmul[NH - 1], km1 * gadd[NH - 1]);
+                        }
+                    }
+                    if (!full_page) {             // first / last page of the quantized range: mask the tokens outside it
+#pragma unroll
+                        for (int bi = 0; bi < 4; ++bi) {
+                            const int p0 = pos0 + bi * 16 + g, p1 = p0 + 8;
+                            if (p0 < q_lo || p0 >= q_hi) {
+                                vmeta[bi][0] = 0u;
+#pragma unroll
+                                for (int k = 0; k < NH; ++k) sc[bi][k] = -INFINITY;
+                            }
+                            if (p1 < q_lo || p1 >= q_hi) {
+                                vmeta[bi][1] = 0u;
+#pragma unroll
+                                for (int k = 0; k < NH; ++k) sc[bi][NH + k] = -INFINITY;
+                            }
                         }
                     }
                     // ---------------- running maximum of the page, rescale if it grew
-                    float mx[NH], mref[NH];
+                    float mx[NH];
 #pragma unroll
                     for (int k = 0; k < NH; ++k) {
                         float v = fmaxf(fmaxf(fmaxf(sc[0][k], sc[0][NH + k]), fmaxf(sc[1][k], sc[1][NH + k])),
@@ -795,22 +803,22 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ?
                         v = fmaxf(v, __shfl_xor_sync(FULL, v, 16));
                         mx[k] = v;
                     }
-                    st.raise_max(mx, mref);
+                    st.raise_max(mx);
                     // ---------------- probabilities, value reduction
 #pragma unroll
                     for (int bi = 0; bi < 4; ++bi) {
                         const float2 vm_a = h2f2(vmeta[bi][0]), vm_b = h2f2(vmeta[bi][1]);
-                        const float vd0 = vm_a.x * PV_SCALE, vn0 = vm_a.y, vd1 = vm_b.x * PV_SCALE, vn1 = vm_b.y;
+                        const float vd0 = vm_a.x, vn0 = vm_a.y, vd1 = vm_b.x, vn1 = vm_b.y;
                         unsigned r0, r1;
                         if (MODE == 0) {
-                            const float p0 = ex2(sc[bi][0] - mref[0]), p1 = ex2(sc[bi][NH] - mref[0]);
+                            const float p0 = ex2(sc[bi][0] - st.mr[0]), p1 = ex2(sc[bi][NH] - st.mr[0]);
                             st.l[0] += p0 + p1;
                             st.z[0] = fmaf(p0, vn0, fmaf(p1, vn1, st.z[0]));
                             r0 = pack_h2(p0 * vd0, 0.f);
                             r1 = pack_h2(p1 * vd1, 0.f);
                         } else {
-                            const float p00 = ex2(sc[bi][0] - mref[0]), p01 = ex2(sc[bi][NH - 1] - mref[NH - 1]);
-                            const float p10 = ex2(sc[bi][NH] - mref[0]), p11 = ex2(sc[bi][2 * NH - 1] - mref[NH - 1]);
+                            const float p00 = ex2(sc[bi][0] - st.mr[0]), p01 = ex2(sc[bi][NH - 1] - st.mr[NH - 1]);
+                            const float p10 = ex2(sc[bi][NH] - st.mr[0]), p11 = ex2(sc[bi][2 * NH - 1] - st.mr[NH - 1]);
                             st.l[0] += p00 + p10; st.l[NH - 1] += p01 + p11;
                             st.z[0] = fmaf(p00, vn0, fmaf(p10, vn1, st.z[0]));
                             st.z[NH - 1] = fmaf(p01, vn0, fmaf(p11, vn1, st.z[NH - 1]));
