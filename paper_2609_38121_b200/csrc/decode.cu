@@ -65,7 +65,7 @@ struct DecodeParams {
     float* O;
     uint4* qfrag;        // [batch*n_kv][2][128]: fp16 B fragments of the 8 k-steps (MODE 1: value set, remainder set)
     uint4* qwfrag;       // [batch*n_kv][2][128]: bf16 B fragments for the windows (MODE 1: value set, remainder set)
-    float* qscal;        // [batch][n_q][2]: (score multiplier, x_min multiplier) in the log2 domain
+    float* qscal;        // [batch][n_q][2]: score multiplier (log2 domain, > 0), x_min multiplier divided by it
     long long* plan;     // [batch+1]: exclusive prefix of work units per sequence (per KV head)
     float* part;         // [n_warps + batch*n_kv][G][PART_STRIDE]
     int n_warps;         // warps of the main kernel
@@ -227,8 +227,8 @@ __global__ void __launch_bounds__(PREP_THREADS) decode_prep_kernel(DecodeParams 
             if (i == 0) {
                 const float sum = red_sum[g][0] + red_sum[g][1] + red_sum[g][2] + red_sum[g][3];
                 float* qs = P.qscal + (static_cast<long long>(b) * P.c.n_q + h * G + g) * 2;
-                qs[0] = k2 * 16777216.f / beta[g];
-                qs[1] = k2 * sum;
+                qs[0] = k2 * 16777216.f / beta[g];            // score = qs[0] * (Delta_k * (codes . q'') + x_min_k * qs[1])
+                qs[1] = sum * beta[g] * (1.f / 16777216.f);
             }
         }
     }
@@ -384,9 +384,10 @@ struct WarpState {
 #pragma unroll
         for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
     }
-    // Make the running reference cover this unit's per-head maxima (already reduced over the unit's
-    // tokens) to within MAX_SLACK; mr is what the exponentials subtract.
-    __device__ __forceinline__ void raise_max(const float (&mx)[NH]) {
+    // Make the running reference cover this unit's maxima to within MAX_SLACK.  mx holds each lane's
+    // maximum over its own tokens; the warp-wide reduction is only needed when some lane is past the
+    // slack, which after the first unit of a slice is rare.  mr is what the exponentials subtract.
+    __device__ __forceinline__ void raise_max(float (&mx)[NH]) {
         bool grew = false;
 #pragma unroll
         for (int k = 0; k < NH; ++k) grew |= mx[k] > m[k] + MAX_SLACK;      // reference -inf: any finite score
@@ -394,6 +395,9 @@ struct WarpState {
             float scl[NH];
 #pragma unroll
             for (int k = 0; k < NH; ++k) {
+                mx[k] = fmaxf(mx[k], __shfl_xor_sync(FULL, mx[k], 4));       // over the 8 token rows of the fragment
+                mx[k] = fmaxf(mx[k], __shfl_xor_sync(FULL, mx[k], 8));
+                mx[k] = fmaxf(mx[k], __shfl_xor_sync(FULL, mx[k], 16));
                 const float mnew = fmaxf(m[k], mx[k]);
                 const float ref = (mnew == -INFINITY) ? 0.f : mnew;          // all masked so far: any finite reference works
                 scl[k] = ex2(m[k] - ref);                                    // old reference -inf: state is all zero, factor 0
@@ -634,7 +638,7 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ?
 #pragma unroll
                 for (int k = 0; k < NH; ++k) {
                     const int head = MODE == 0 ? t : 2 * t + k;
-                    fmul[k] = gadd[k] = 0.f;
+                    fmul[k] = 1.f; gadd[k] = 0.f;             // unused head slots stay finite
                     if (head < G) {
                         const float2 v = __ldg(reinterpret_cast<const float2*>(P.qscal + (static_cast<long long>(sg.b) * c.n_q + sg.h * G + head) * 2));
                         fmul[k] = v.x; gadd[k] = v.y;
@@ -673,12 +677,7 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ?
                     if (MODE == 0) sc[0] = ok ? acc[0] + acc[1] : -INFINITY;
                     else { sc[0] = ok ? acc[0] : -INFINITY; sc[NH - 1] = ok ? acc[1] : -INFINITY; }
 #pragma unroll
-                    for (int k = 0; k < NH; ++k) {
-                        mx[k] = sc[k];
-                        mx[k] = fmaxf(mx[k], __shfl_xor_sync(FULL, mx[k], 4));
-                        mx[k] = fmaxf(mx[k], __shfl_xor_sync(FULL, mx[k], 8));
-                        mx[k] = fmaxf(mx[k], __shfl_xor_sync(FULL, mx[k], 16));
-                    }
+                    for (int k = 0; k < NH; ++k) mx[k] = sc[k];
                     st.raise_max(mx);
                     float p[NH];
 #pragma unroll
@@ -767,13 +766,13 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ?
                         vmeta[bi][0] = mt.y; vmeta[bi][1] = mt.w;
                         if (MODE == 0) {
                             const float d0 = fmaf(acc[1], 1.f / LO_SCALE, acc[0]), d1 = fmaf(acc[3], 1.f / LO_SCALE, acc[2]);
-                            sc[bi][0] = fmaf(d0 * kd0, fmul[0], km0 * gadd[0]);
-                            sc[bi][NH] = fmaf(d1 * kd1, fmul[0], km1 * gadd[0]);
+                            sc[bi][0] = fmaf(km0, gadd[0], d0 * kd0);
+                            sc[bi][NH] = fmaf(km1, gadd[0], d1 * kd1);
                         } else {
-                            sc[bi][0] = fmaf(acc[0] * kd0, fmul[0], km0 * gadd[0]);
-                            sc[bi][NH - 1] = fmaf(acc[1] * kd0, fmul[NH - 1], km0 * gadd[NH - 1]);
-                            sc[bi][NH] = fmaf(acc[2] * kd1, fmul[0], km1 * gadd[0]);
-                            sc[bi][2 * NH - 1] = fmaf(acc[3] * kd1, fmul[NH - 1], km1 * gadd[NH - 1]);
+                            sc[bi][0] = fmaf(km0, gadd[0], acc[0] * kd0);
+                            sc[bi][NH - 1] = fmaf(km0, gadd[NH - 1], acc[1] * kd0);
+                            sc[bi][NH] = fmaf(km1, gadd[0], acc[2] * kd1);
+                            sc[bi][2 * NH - 1] = fmaf(km1, gadd[NH - 1], acc[3] * kd1);
                         }
                     }
                     if (!full_page) {             // first / last page of the quantized range: mask the tokens outside it
@@ -796,12 +795,9 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ?
                     float mx[NH];
 #pragma unroll
                     for (int k = 0; k < NH; ++k) {
-                        float v = fmaxf(fmaxf(fmaxf(sc[0][k], sc[0][NH + k]), fmaxf(sc[1][k], sc[1][NH + k])),
-                                        fmaxf(fmaxf(sc[2][k], sc[2][NH + k]), fmaxf(sc[3][k], sc[3][NH + k])));
-                        v = fmaxf(v, __shfl_xor_sync(FULL, v, 4));
-                        v = fmaxf(v, __shfl_xor_sync(FULL, v, 8));
-                        v = fmaxf(v, __shfl_xor_sync(FULL, v, 16));
-                        mx[k] = v;
+                        const float v = fmaxf(fmaxf(fmaxf(sc[0][k], sc[0][NH + k]), fmaxf(sc[1][k], sc[1][NH + k])),
+                                              fmaxf(fmaxf(sc[2][k], sc[2][NH + k]), fmaxf(sc[3][k], sc[3][NH + k])));
+                        mx[k] = v * fmul[k];          // scores are kept divided by the head's multiplier (> 0)
                     }
                     st.raise_max(mx);
                     // ---------------- probabilities, value reduction
@@ -811,14 +807,14 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ?
                         const float vd0 = vm_a.x, vn0 = vm_a.y, vd1 = vm_b.x, vn1 = vm_b.y;
                         unsigned r0, r1;
                         if (MODE == 0) {
-                            const float p0 = ex2(sc[bi][0] - st.mr[0]), p1 = ex2(sc[bi][NH] - st.mr[0]);
+                            const float p0 = ex2(fmaf(sc[bi][0], fmul[0], -st.mr[0])), p1 = ex2(fmaf(sc[bi][NH], fmul[0], -st.mr[0]));
                             st.l[0] += p0 + p1;
                             st.z[0] = fmaf(p0, vn0, fmaf(p1, vn1, st.z[0]));
                             r0 = pack_h2(p0 * vd0, 0.f);
                             r1 = pack_h2(p1 * vd1, 0.f);
                         } else {
-                            const float p00 = ex2(sc[bi][0] - st.mr[0]), p01 = ex2(sc[bi][NH - 1] - st.mr[NH - 1]);
-                            const float p10 = ex2(sc[bi][NH] - st.mr[0]), p11 = ex2(sc[bi][2 * NH - 1] - st.mr[NH - 1]);
+                            const float p00 = ex2(fmaf(sc[bi][0], fmul[0], -st.mr[0])), p01 = ex2(fmaf(sc[bi][NH - 1], fmul[NH - 1], -st.mr[NH - 1]));
+                            const float p10 = ex2(fmaf(sc[bi][NH], fmul[0], -st.mr[0])), p11 = ex2(fmaf(sc[bi][2 * NH - 1], fmul[NH - 1], -st.mr[NH - 1]));
                             st.l[0] += p00 + p10; st.l[NH - 1] += p01 + p11;
                             st.z[0] = fmaf(p00, vn0, fmaf(p10, vn1, st.z[0]));
                             st.z[NH - 1] = fmaf(p01, vn0, fmaf(p11, vn1, st.z[NH - 1]));
