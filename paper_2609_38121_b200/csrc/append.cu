@@ -261,6 +261,10 @@ __global__ void __launch_bounds__(1024) append_token_kernel(AppendParams P) {
     const int first = __ldg(P.cu_new + b), n_new = __ldg(P.cu_new + b + 1) - first;
     if (n_new <= 0) return;
     const int s0 = __ldg(P.seq_len + b);
+    const int slot0 = __ldg(P.slot + b);                 // the page lookup does not depend on the transform: start it now
+    int page = -1;
+    if (slot0 >= 0 && slot0 < P.c.n_slots && s0 >= 0 && s0 / PAGE_TOKENS < P.c.max_pages)
+        page = __ldg(P.c.page_table + static_cast<long long>(slot0) * P.c.max_pages + s0 / PAGE_TOKENS);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const long long row0 = static_cast<long long>(first) * n_kv * D;
     for (int idx = threadIdx.x; idx < n_kv * D; idx += blockDim.x) kin_s[idx] = bf16_bits_to_float(__ldg(P.K_new + row0 + idx));
@@ -282,17 +286,13 @@ __global__ void __launch_bounds__(1024) append_token_kernel(AppendParams P) {
     }
     __syncthreads();
     TokenSlot ts;
-    ts.b = b; ts.slot = __ldg(P.slot + b); ts.pos = s0; ts.s_final = s0 + 1;
+    ts.b = b; ts.slot = slot0; ts.pos = s0; ts.s_final = s0 + 1;
     bool ok = true;
     if (ts.slot < 0 || ts.slot >= P.c.n_slots || s0 < 0) { if (threadIdx.x == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_SLOT); ok = false; }
-    int page = -1;
     if (ok) {
         const int pidx = ts.pos / PAGE_TOKENS;
         if (pidx >= P.c.max_pages) { if (threadIdx.x == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_PAGE_TABLE_FULL); ok = false; }
-        else {
-            page = __ldg(P.c.page_table + static_cast<long long>(ts.slot) * P.c.max_pages + pidx);
-            if (page < 0 || page >= P.c.n_pages) { if (threadIdx.x == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_PAGE_ID); ok = false; }
-        }
+        else if (page < 0 || page >= P.c.n_pages) { if (threadIdx.x == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_PAGE_ID); ok = false; }
     }
     if (ok) {
         ts.r = ts.pos % PAGE_TOKENS;

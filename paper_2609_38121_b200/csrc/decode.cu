@@ -860,54 +860,76 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ?
 // ------------------------------------------------------------------------------------------------
 // 3. combine
 // ------------------------------------------------------------------------------------------------
-// One CTA per (sequence, query head), one thread per channel.  The partials sit in L2, so the cost is
-// load latency: the loads of 8 partials are issued together before they are merged.
-__global__ void __launch_bounds__(128) decode_combine_kernel(DecodeParams P) {
+// One CTA per (sequence, query head): up to 8 thread groups of one thread per channel, each merging a
+// contiguous share of the head's partials.  The partials sit in L2, so the cost is load latency: a
+// group issues the loads of COMBINE_BATCH partials together before it merges them.
+constexpr int COMBINE_BATCH = 8;        // loads in flight per thread
+template <int MAX_GROUPS>
+__global__ void __launch_bounds__(128 * MAX_GROUPS) decode_combine_kernel(DecodeParams P) {
+    __shared__ float red_m[MAX_GROUPS], red_l[MAX_GROUPS], red_o[MAX_GROUPS][D];
     const CacheView& c = P.c;
-    const int j = blockIdx.x, b = blockIdx.y, ch = threadIdx.x;
+    const int j = blockIdx.x, b = blockIdx.y, ch = threadIdx.x, grp = threadIdx.y, n_grp = blockDim.y;
     pdl_wait();                                         // partials and the plan come from the earlier kernels
     pdl_launch_dependents();                            // a programmatically launched successor waits for us itself
     float* out = P.O + (static_cast<long long>(b) * c.n_q + j) * D;
     const long long U = P.plan[b + 1] - P.plan[b];
     const long long total = P.plan[P.batch] * c.n_kv;
-    if (U <= 0 || total <= 0) { out[ch] = 0.f; return; }
+    if (U <= 0 || total <= 0) { if (grp == 0) out[ch] = 0.f; return; }
     const int h = j / c.G, head = j % c.G;
     const long long La = P.plan[b] * c.n_kv + static_cast<long long>(h) * U, Lb = La + U;      // units [La, Lb)
     const long long nw = P.n_warps;
     // warp w owns units [floor(w total / nw), floor((w+1) total / nw)); owners of La and Lb-1:
     const long long w_first = ((La + 1) * nw - 1) / total, w_last = (Lb * nw - 1) / total;
     const long long bh = static_cast<long long>(b) * c.n_kv + h;
-    const float* base = P.part + ((w_first + bh) * c.G + head) * PART_STRIDE;
     const long long stride = static_cast<long long>(c.G) * PART_STRIDE;
     const int n = static_cast<int>(w_last - w_first + 1);
+    // thread group grp merges the contiguous share [k0, k1) of the n partials
+    const int share = (n + n_grp - 1) / n_grp;
+    const int k0 = min(grp * share, n), k1 = min(k0 + share, n);
+    const float* base = P.part + ((w_first + k0 + bh) * c.G + head) * PART_STRIDE;
     // slice bounds advance by q = total / nw with a carry of r = total % nw (no division in the loop)
     const long long q = total / nw, r = total % nw;
-    long long lo_w = w_first * total / nw, rem = (w_first * total) % nw;
+    long long lo_w = (w_first + k0) * total / nw, rem = ((w_first + k0) * total) % nw;
     float m = -INFINITY, l = 0.f, o = 0.f;
-    for (int s0 = 0; s0 < n; s0 += 8) {
-        float pm[8], pl[8], po[8];
+    for (int s0 = k0; s0 < k1; s0 += COMBINE_BATCH) {
+        float pm[COMBINE_BATCH], pl[COMBINE_BATCH], po[COMBINE_BATCH];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
+        for (int k = 0; k < COMBINE_BATCH; ++k) {
             pm[k] = -INFINITY; pl[k] = 0.f; po[k] = 0.f;
-            if (s0 + k < n) {
+            if (s0 + k < k1) {
                 long long hi_w = lo_w + q;
                 rem += r;
                 if (rem >= nw) { rem -= nw; ++hi_w; }
                 const bool wrote = max(lo_w, La) < min(hi_w, Lb);     // a warp with an empty slice wrote nothing
                 lo_w = hi_w;
                 if (wrote) {
-                    const float* p = base + (s0 + k) * stride;
+                    const float* p = base + (s0 - k0 + k) * stride;
                     pm[k] = __ldcg(p); pl[k] = __ldcg(p + 1); po[k] = __ldcg(p + 4 + ch);
                 }
             }
         }
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
+        for (int k = 0; k < COMBINE_BATCH; ++k) {
             if (pm[k] == -INFINITY) continue;
             const float mn = fmaxf(m, pm[k]);
             const float sa = exp2f(m - mn), sb = exp2f(pm[k] - mn);   // m = -inf on the first partial: sa = 0
             l = l * sa + pl[k] * sb;
             o = o * sa + po[k] * sb;
+            m = mn;
+        }
+    }
+    if (MAX_GROUPS > 1 && n_grp > 1) {                  // merge the groups' states, in group order
+        if (ch == 0) { red_m[grp] = m; red_l[grp] = l; }
+        red_o[grp][ch] = o;
+        __syncthreads();
+        if (grp != 0) return;
+        for (int k = 1; k < n_grp; ++k) {
+            const float pm = red_m[k];
+            if (pm == -INFINITY) continue;
+            const float mn = fmaxf(m, pm);
+            const float sa = exp2f(m - mn), sb = exp2f(pm - mn);
+            l = l * sa + red_l[k] * sb;
+            o = o * sa + red_o[k][ch] * sb;
             m = mn;
         }
     }
@@ -981,10 +1003,19 @@ static int launch_decode(const DecodeParams& P, int n_ctas, cudaStream_t st) {
     cfg.dynamicSmemBytes = SMEM;
     if (cudaLaunchKernelEx(&cfg, decode_main_kernel<BITS, MODE, STAGES>, P) != cudaSuccess) return WUSHKV_ECUDA;
     if (g_prof_stop) cudaEventRecord(g_prof_stop, st);
+    // Partials per (sequence, KV head) are about n_warps / (batch n_kv).  Short lists go to one thread
+    // group per CTA (a few rounds of COMBINE_BATCH loads); a long list (few sequences, long context)
+    // is shared by 8 groups.
+    const long long per_head = P.n_warps / (static_cast<long long>(P.batch) * P.c.n_kv) + 2;
     cfg.gridDim = dim3(P.c.n_q, P.batch);
-    cfg.blockDim = dim3(128);
     cfg.dynamicSmemBytes = 0;
-    if (cudaLaunchKernelEx(&cfg, decode_combine_kernel, P) != cudaSuccess) return WUSHKV_ECUDA;
+    if (per_head <= 4 * COMBINE_BATCH) {
+        cfg.blockDim = dim3(128, 1);
+        if (cudaLaunchKernelEx(&cfg, decode_combine_kernel<1>, P) != cudaSuccess) return WUSHKV_ECUDA;
+    } else {
+        cfg.blockDim = dim3(128, 8);
+        if (cudaLaunchKernelEx(&cfg, decode_combine_kernel<8>, P) != cudaSuccess) return WUSHKV_ECUDA;
+    }
     return WUSHKV_OK;
 }
 
