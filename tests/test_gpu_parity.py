@@ -178,6 +178,18 @@ def test_fused_step_equals_append_then_decode(bits, n_q, n_kv):
             assert np.array_equal(x, y, equal_nan=True)
 
 
+@pytest.mark.parametrize("bits", [2, 4])
+def test_tensor_memory_score_path(bits, monkeypatch):
+    """The alternative main kernel (scores by tcgen05 from e4m3 code bytes in tensor memory, selected by
+    WUSHKV_DECODE_PATH=tc for G <= 4) meets the same tolerance on a ragged, shuffled-page batch."""
+    monkeypatch.setenv("WUSHKV_DECODE_PATH", "tc")
+    wl = _wl(8, 2, seed=52, batch=5)
+    L = Layer(wl, [1500, 0, 65, 300, 2], bits, 4, 64, 1, page_shuffle_seed=5)
+    L.fill()
+    assert L.check_decode_parity() <= 2e-3
+    assert L.cache.status() == 0
+
+
 def test_device_side_errors_are_flagged_not_fatal():
     """A position beyond the page table and a page id outside the pool set status bits; the calls
     still return and the rest of the batch is processed."""
