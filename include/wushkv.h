@@ -216,6 +216,10 @@ int wushkv_decode_step(const wushkv_cache* cache, int32_t batch, const int32_t* 
  *   Q_host (host): bf16 [batch][n_q][d].   O_host (host, out): fp32 [batch][n_q][d].
  *   cu_new (device): int32 [batch+1] = 0, 1, ..., batch.
  *   staging (device): >= wushkv_step_staging_bytes() bytes, 256-byte aligned, scratch.
+ *   When all four host buffers are pinned and mapped into the device's address space (cudaHostAlloc or
+ *   cudaHostRegister under unified addressing) and 16-byte aligned, no copy is enqueued: the kernels read
+ *   K_new, V_new and Q and write O in place over the bus.  Otherwise (or with WUSHKV_HOST_IO=copy in the
+ *   environment) the copies go through `staging`.  Results are identical either way.
  *   slot, seq_len (in/out), max_seq_len (bound on the lengths AFTER the append), workspace: as for
  *   wushkv_append / wushkv_decode_attn.
  */

@@ -178,6 +178,49 @@ def test_fused_step_equals_append_then_decode(bits, n_q, n_kv):
             assert np.array_equal(x, y, equal_nan=True)
 
 
+@pytest.mark.parametrize("mode", ["mapped", "copy"])
+def test_host_step_equals_device_step(mode, monkeypatch):
+    """wushkv_decode_step_host (pinned host buffers read and written in place, or staged copies when
+    WUSHKV_HOST_IO=copy) gives the outputs and the cache of wushkv_decode_step, bit for bit."""
+    import torch
+    from paper_2609_38121_b200 import binding as B
+    if mode == "copy":
+        monkeypatch.setenv("WUSHKV_HOST_IO", "copy")
+    wl = _wl(8, 2, seed=43)
+    lengths, steps = [400, 70, 2], 2
+    first = [n - steps for n in lengths]
+    dev_l, host_l = Layer(wl, lengths, 2, 4, 64, 1), Layer(wl, lengths, 2, 4, 64, 1)
+    dev_l.append_step(first, oracle_too=False)
+    host_l.append_step(first, oracle_too=False)
+    dev = dev_l.cache.device
+    nb = len(lengths)
+    bits16 = lambda x: torch.from_numpy(W.f32_to_bf16_bits(x).view(np.int16))  # noqa: E731
+    cu = torch.arange(nb + 1, dtype=torch.int32, device=dev)
+    nbytes = B.decode_workspace_bytes(dev_l.cache.desc, nb, dev_l.max_seq_len)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    stg_bytes = B.step_staging_bytes(host_l.cache.desc, nb)
+    stg = torch.empty(stg_bytes, dtype=torch.uint8, device=dev)
+    for i in range(steps):
+        K = bits16(np.stack([dev_l.tokens[b][0][first[b] + i] for b in range(nb)]))
+        V = bits16(np.stack([dev_l.tokens[b][1][first[b] + i] for b in range(nb)]))
+        Q = bits16(np.stack([wl.queries(b, first[b] + i) for b in range(nb)]))
+        O_dev = torch.full((nb, 8, 128), float("nan"), dtype=torch.float32, device=dev)
+        B.decode_step(dev_l.cache.desc, nb, dev_l.slot, dev_l.seq_len, cu, dev_l.max_seq_len, K.to(dev), V.to(dev), Q.to(dev),
+                      O_dev, ws, nbytes)
+        hK, hV, hQ = K.pin_memory(), V.pin_memory(), Q.pin_memory()
+        hO = torch.full((nb, 8, 128), float("nan"), dtype=torch.float32).pin_memory()
+        B.decode_step_host(host_l.cache.desc, nb, host_l.slot, host_l.seq_len, cu, host_l.max_seq_len, hK, hV, hQ, hO,
+                           stg, stg_bytes, ws, nbytes)
+        torch.cuda.synchronize()
+        assert np.array_equal(hO.numpy(), O_dev.cpu().numpy()), f"step {i}"
+    assert host_l.seq_len.cpu().tolist() == lengths and host_l.cache.status() == 0
+    for b in range(nb):
+        for h in range(2):
+            for which in (0, 1):
+                for x, y in zip(host_l.gpu_codes(b, h, which), dev_l.gpu_codes(b, h, which)):
+                    assert np.array_equal(x, y)
+
+
 @pytest.mark.parametrize("bits", [2, 4])
 def test_tensor_memory_score_path(bits, monkeypatch):
     """The alternative main kernel (scores by tcgen05 from e4m3 code bytes in tensor memory, selected by
