@@ -176,6 +176,12 @@ size_t wushkv_decode_workspace_bytes(const wushkv_cache* cache, int32_t batch, i
  * The kernels of one call are chained by programmatic dependent launch; the first of them waits
  * for the kernel before it in the stream before it reads anything, so any producer of Q, seq_len or
  * the cache may precede the call directly.
+ * Range: probabilities times the stored value step are fed to the tensor core in fp16 with up to
+ * 2^6 of headroom, so a stored Delta_v of 1024 or more (a value range beyond ~3000 at 2 bits)
+ * saturates and loses accuracy; keys have no such limit.
+ * Environment (testing aids): WUSHKV_DECODE_CTAS=<n> fixes the number of thread blocks of the main
+ * kernel (the split count); WUSHKV_DECODE_PATH=tc selects, for n_q / n_kv <= 4, an alternative main
+ * kernel that computes the scores with tcgen05 (same results to rounding, slower).
  */
 int wushkv_decode_attn(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
                        int32_t max_seq_len, const uint16_t* Q, float* O,

@@ -18,10 +18,14 @@
 //                           Window units use ldmatrix + bf16 mma on the staged rows and fold into the
 //                           same accumulators.  Softmax is online (running max / sum) per warp; a warp
 //                           writes one partial (max, sum, o) per (sequence, KV head) it touched.
+//  2b. decode_main_tc_kernel  opt-in alternative to 2 for G <= 4 (WUSHKV_DECODE_PATH=tc): the scores come from
+//                           tcgen05.mma on e4m3 code bytes held in tensor memory; a CTA's four warps share
+//                           128-token tiles.  Measured slower than 2; kept with its parity test.
 //   3. decode_combine_kernel merges the partials of each (sequence, query head) into O.
 //
-// No kernel waits on another CTA or warp.  The only waits are on a warp's own copy barriers, bounded
-// by an iteration limit after which the kernel records WUSHKV_DEV_COPY_TIMEOUT and drains.
+// No kernel waits on another CTA.  The only waits are on a warp's (2b: a CTA's) own copy and MMA
+// barriers, bounded by an iteration limit after which the kernel records WUSHKV_DEV_COPY_TIMEOUT and
+// drains; in 2b the four warps of a CTA also meet at CTA barriers, whose outcome carries that flag.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
