@@ -178,6 +178,30 @@ def test_fused_step_equals_append_then_decode(bits, n_q, n_kv):
             assert np.array_equal(x, y, equal_nan=True)
 
 
+@pytest.mark.parametrize("log2_scale", [-6, 5])
+def test_value_scale_invariance(log2_scale):
+    """Scaling every value by a power of two scales the stored steps and offsets exactly and leaves the
+    codes unchanged, so the outputs must scale with it up to what the fp16 operand p * Delta_v of the
+    value contraction loses at the ends of its range (tiny probabilities fall into the subnormals at the
+    low end; at the high end the stored step must stay below 1024, which with this workload's outlier
+    channels is reached at a scale of 2^6)."""
+    wl = _wl(8, 2, seed=61)
+    outs = []
+    for f in (1.0, 2.0 ** log2_scale):
+        L = Layer(wl, [900, 130], 2, 4, 64, 1)
+        L.tokens = [(K, V * np.float32(f)) for (K, V) in L.tokens]
+        L.append_step([n - 1 for n in L.lengths], oracle_too=False)
+        L.append_step([1] * L.batch, oracle_too=False)
+        outs.append(L.decode()[0])
+        if f != 1.0:
+            codes_scaled = L.gpu_codes(0, 1, 1)[0]
+        else:
+            codes_plain = L.gpu_codes(0, 1, 1)[0]
+    assert np.array_equal(codes_scaled, codes_plain)
+    assert np.all(np.isfinite(outs[1]))
+    assert np.max(np.abs(outs[1] * 2.0 ** -log2_scale - outs[0])) <= 5e-4 * np.max(np.abs(outs[0]))
+
+
 @pytest.mark.parametrize("mode", ["mapped", "copy"])
 def test_host_step_equals_device_step(mode, monkeypatch):
     """wushkv_decode_step_host (pinned host buffers read and written in place, or staged copies when
