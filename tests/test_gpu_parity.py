@@ -178,6 +178,29 @@ def test_fused_step_equals_append_then_decode(bits, n_q, n_kv):
             assert np.array_equal(x, y, equal_nan=True)
 
 
+def test_batch_larger_than_the_in_kernel_plan():
+    """7000 short sequences: the work plan no longer fits the main kernel's staging area (it is read from
+    the preparation kernel's copy instead), a warp's slice spans many (sequence, head) segments and
+    takes several rounds, and most sequences are sink-only or nothing-quantized."""
+    wl = _wl(2, 1, seed=71, batch=7000)
+    rng = np.random.default_rng(71)
+    lengths = [int(x) for x in rng.integers(0, 6, size=7000)]
+    lengths[17] = 300
+    L = Layer(wl, lengths, 2, 1, 2, 1)
+    L.fill()
+    Og, Q = L.decode()
+    assert L.cache.status() == 0
+    worst = 0.0
+    for b in list(range(0, 7000, 97)) + [17, 6999]:
+        if lengths[b] == 0:
+            assert np.all(Og[b] == 0)
+            continue
+        ref = L.oracle_decode_on_gpu_cache(b, Q[b])
+        worst = max(worst, np.max(np.abs(Og[b] - ref)) / np.max(np.abs(ref)))
+    assert worst <= 2e-3
+    assert all(np.all(Og[b] == 0) for b in range(7000) if lengths[b] == 0)
+
+
 @pytest.mark.parametrize("log2_scale", [-6, 5])
 def test_value_scale_invariance(log2_scale):
     """Scaling every value by a power of two scales the stored steps and offsets exactly and leaves the
