@@ -78,6 +78,7 @@ struct DecodeParams {
     unsigned char* qb8;  // [batch*n_kv][2048]: e4m3 query operand of the tensor-memory kernel (null: not used)
     float* qscal8;       // [batch][n_q][2]: the same two scalars as qscal for the e4m3 operand
     int slice_shift;     // log2 of the warps that share one slice of the unit list (0: each warp its own, 2: a CTA)
+    int stream_pages;    // 1: the packed pages of a step cannot stay in L2 anyway: copy them with an evict-first hint
 };
 
 // shift of the code field used by k-step / channel block idx (0..7) inside its 16-bit lane, after
@@ -366,6 +367,17 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity)
 __device__ __forceinline__ void bulk_copy_g2s(unsigned dst, const void* src, unsigned bytes, unsigned bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// The same copy for data that is read once per step (packed pages): evict-first in L2, so that the
+// stream does not push out what the step's other kernels re-read (transforms, fragments, partials).
+__device__ __forceinline__ unsigned long long l2_evict_first_policy() {
+    unsigned long long pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void bulk_copy_g2s_stream(unsigned dst, const void* src, unsigned bytes, unsigned bar, unsigned long long pol) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(pol) : "memory");
 }
 __device__ __forceinline__ uint4 lds128(unsigned addr) {
     uint4 v;
@@ -657,6 +669,7 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ?
     __syncwarp();
     const unsigned stage0 = smem_u32(smem + warp * STAGES * REC);
     const long long page_row_bytes = static_cast<long long>(c.n_kv) * REC;
+    const unsigned long long stream_policy = l2_evict_first_policy();
 
     unsigned qf[8][2];
     float fmul[NH], gadd[NH];
@@ -718,7 +731,8 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ?
                     } else {
                         bad_bits &= ~(1u << s);
                         mbar_expect_tx(bar, REC);
-                        bulk_copy_g2s(dst, c.pages + page * page_row_bytes + p_head_off, REC, bar);
+                        if (P.stream_pages) bulk_copy_g2s_stream(dst, c.pages + page * page_row_bytes + p_head_off, REC, bar, stream_policy);
+                        else bulk_copy_g2s(dst, c.pages + page * page_row_bytes + p_head_off, REC, bar);
                     }
                 }
             } else {                                    // up to 8 window tokens: one 256-byte row copy per lane
@@ -1374,7 +1388,7 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 3 : 4)) decode_m
 // contiguous share of the head's partials.  The partials sit in L2, so the cost is load latency: a
 // group issues the loads of COMBINE_BATCH partials together before it merges them.
 constexpr int COMBINE_BATCH = 8;        // loads in flight per thread
-template <int MAX_GROUPS>
+template <int MAX_GROUPS, int GS>      // GS: log2 of the warps per slice (compile-time copy of slice_shift)
 __global__ void __launch_bounds__(128 * MAX_GROUPS) decode_combine_kernel(DecodeParams P) {
     __shared__ float red_m[MAX_GROUPS], red_l[MAX_GROUPS], red_o[MAX_GROUPS][D];
     const CacheView& c = P.c;
@@ -1390,7 +1404,7 @@ __global__ void __launch_bounds__(128 * MAX_GROUPS) decode_combine_kernel(Decode
     // The unit list is cut into ns equal slices, slice i = [floor(i total / ns), floor((i+1) total / ns)); a
     // slice belongs to one warp (slice_shift 0) or to the four warps of a CTA (slice_shift 2), and every
     // warp of a slice that meets [La, Lb) wrote a partial, at slot (slice + bh) * warps_per_slice + warp.
-    const int gs = P.slice_shift, group_mask = (1 << gs) - 1;
+    constexpr int gs = GS, group_mask = (1 << gs) - 1;
     const long long ns = static_cast<long long>(P.n_warps) >> gs;
     const long long s_first = ((La + 1) * ns - 1) / total, s_last = (Lb * ns - 1) / total;   // owners of La and Lb-1
     const long long bh = static_cast<long long>(b) * c.n_kv + h;
@@ -1546,12 +1560,13 @@ static int launch_decode(const DecodeParams& P, int n_ctas, cudaStream_t st) {
     const long long per_head = P.n_warps / (static_cast<long long>(P.batch) * P.c.n_kv) + 2;
     cfg.gridDim = dim3(P.c.n_q, P.batch);
     cfg.dynamicSmemBytes = 0;
+    const bool shared_slices = P.slice_shift != 0;
     if (per_head <= 4 * COMBINE_BATCH) {
         cfg.blockDim = dim3(128, 1);
-        if (cudaLaunchKernelEx(&cfg, decode_combine_kernel<1>, P) != cudaSuccess) return WUSHKV_ECUDA;
+        if (cudaLaunchKernelEx(&cfg, shared_slices ? decode_combine_kernel<1, 2> : decode_combine_kernel<1, 0>, P) != cudaSuccess) return WUSHKV_ECUDA;
     } else {
         cfg.blockDim = dim3(128, 8);
-        if (cudaLaunchKernelEx(&cfg, decode_combine_kernel<8>, P) != cudaSuccess) return WUSHKV_ECUDA;
+        if (cudaLaunchKernelEx(&cfg, shared_slices ? decode_combine_kernel<8, 2> : decode_combine_kernel<8, 0>, P) != cudaSuccess) return WUSHKV_ECUDA;
     }
     return WUSHKV_OK;
 }
@@ -1591,6 +1606,19 @@ static int decode_attn_impl(const wushkv_cache* cache, int32_t batch, const int3
     P.qb8 = pl.tensor_scores ? ws + pl.off_qb8 : nullptr;
     P.qscal8 = pl.tensor_scores ? reinterpret_cast<float*>(ws + pl.off_qscal8) : nullptr;
     P.slice_shift = pl.tensor_scores ? 2 : 0;
+    {   // upper bound of the packed bytes one step reads against the L2 size
+        static int l2_bytes[64] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return WUSHKV_ECUDA;
+        int l2 = (dev >= 0 && dev < 64) ? l2_bytes[dev] : 0;
+        if (l2 == 0) {
+            if (cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess) return WUSHKV_ECUDA;
+            if (dev >= 0 && dev < 64) l2_bytes[dev] = l2;
+        }
+        const double step_bytes = static_cast<double>(batch) * P.c.n_kv * ((max_seq_len + PAGE_TOKENS - 1) / PAGE_TOKENS) *
+                                  (P.c.bits == 2 ? record_bytes(2) : record_bytes(4));
+        P.stream_pages = step_bytes > static_cast<double>(l2) ? 1 : 0;
+    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool mode0 = P.c.G <= 4;
     if (P.c.bits == 2) return mode0 ? launch_decode<2, 0>(P, pl.n_ctas, st) : launch_decode<2, 1>(P, pl.n_ctas, st);
