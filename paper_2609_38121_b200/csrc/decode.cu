@@ -591,7 +591,7 @@ constexpr int MAX_SEGMENTS = 6;           // per warp and round; more segments t
 // main kernel
 // ------------------------------------------------------------------------------------------------
 template <int BITS, int MODE, int STAGES>
-__global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 2 : (MODE == 0 ? 4 : 3))) decode_main_kernel(DecodeParams P) {
+__global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 3 : (MODE == 0 ? 4 : 3))) decode_main_kernel(DecodeParams P) {
     constexpr int REC = record_bytes(BITS);
     constexpr int CB = code_block_bytes(BITS);
     constexpr int NH = WarpState<MODE>::NH;
@@ -1494,7 +1494,7 @@ static bool make_plan(const CacheView& c, int batch, int max_seq_len, DecodePlan
     if (const char* e = std::getenv("WUSHKV_DECODE_CTAS")) ctas = std::atoll(e);
     if (ctas <= 0) {
         // CTAs per SM: shared memory at 4 bits, registers for G > 4
-        const long long per_sm = pl.tensor_scores ? (c.bits == 4 ? 3 : 4) : (c.bits == 4 ? 2 : (c.G <= 4 ? 4 : 3));
+        const long long per_sm = pl.tensor_scores ? (c.bits == 4 ? 3 : 4) : (c.bits == 4 ? 3 : (c.G <= 4 ? 4 : 3));
         ctas = std::min<long long>(per_sm * sm_count(), (units_max + 2 * MAIN_WARPS - 1) / (2 * MAIN_WARPS));
     }
     ctas = std::max<long long>(1, std::min<long long>(ctas, 1 << 20));
@@ -1517,7 +1517,7 @@ static cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
 
 template <int BITS, int MODE>
 static int launch_decode(const DecodeParams& P, int n_ctas, cudaStream_t st) {
-    constexpr int STAGES = 3;
+    constexpr int STAGES = BITS == 4 ? 2 : 3;      // 4-bit records are twice as large: two stages keep three CTAs on an SM
     constexpr size_t SMEM = static_cast<size_t>(MAIN_WARPS) * STAGES * record_bytes(BITS) + MAIN_WARPS * STAGES * 8 +
                             MAIN_WARPS * MAX_SEGMENTS * sizeof(Segment);
     constexpr size_t SMEM_TC = static_cast<size_t>(TC_STAGES) * 2 * record_bytes(BITS) + 2 * QB_BYTES + (TC_STAGES + 1) * 8 + 32 +
