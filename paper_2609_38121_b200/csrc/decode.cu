@@ -1517,7 +1517,7 @@ static cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
 
 template <int BITS, int MODE>
 static int launch_decode(const DecodeParams& P, int n_ctas, cudaStream_t st) {
-    constexpr int STAGES = BITS == 4 ? 2 : 3;      // 4-bit records are twice as large: two stages keep three CTAs on an SM
+    constexpr int STAGES = 2;      // 4-bit records are twice as large: two stages keep three CTAs on an SM
     constexpr size_t SMEM = static_cast<size_t>(MAIN_WARPS) * STAGES * record_bytes(BITS) + MAIN_WARPS * STAGES * 8 +
                             MAIN_WARPS * MAX_SEGMENTS * sizeof(Segment);
     constexpr size_t SMEM_TC = static_cast<size_t>(TC_STAGES) * 2 * record_bytes(BITS) + 2 * QB_BYTES + (TC_STAGES + 1) * 8 + 32 +
