@@ -267,6 +267,9 @@ __global__ void __launch_bounds__(1024) append_token_kernel(AppendParams P) {
         page = __ldg(P.c.page_table + static_cast<long long>(slot0) * P.c.max_pages + s0 / PAGE_TOKENS);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const long long row0 = static_cast<long long>(first) * n_kv * D;
+    // a warp that will quantize a value vector requests it now; it is used after the transform
+    uint2 v_pre = make_uint2(0u, 0u);
+    if (warp >= n_kv && warp < 2 * n_kv) v_pre = __ldg(reinterpret_cast<const uint2*>(P.V_new + row0 + (warp - n_kv) * D) + lane);
     for (int idx = threadIdx.x; idx < n_kv * D; idx += blockDim.x) kin_s[idx] = bf16_bits_to_float(__ldg(P.K_new + row0 + idx));
     __syncthreads();
     // k'[h][i] = sum_j T[h][i][j] k[h][j]: a warp takes 32 consecutive rows of one head; every row is
@@ -307,7 +310,7 @@ __global__ void __launch_bounds__(1024) append_token_kernel(AppendParams P) {
                 copy.x = float_to_bf16_bits(x[0]) | (static_cast<unsigned>(float_to_bf16_bits(x[1])) << 16);
                 copy.y = float_to_bf16_bits(x[2]) | (static_cast<unsigned>(float_to_bf16_bits(x[3])) << 16);
             } else {
-                copy = __ldg(reinterpret_cast<const uint2*>(P.V_new + row0 + head * D) + lane);
+                copy = (v == warp) ? v_pre : __ldg(reinterpret_cast<const uint2*>(P.V_new + row0 + head * D) + lane);
                 x[0] = bf16_bits_to_float(copy.x & 0xffff); x[1] = bf16_bits_to_float(copy.x >> 16);
                 x[2] = bf16_bits_to_float(copy.y & 0xffff); x[3] = bf16_bits_to_float(copy.y >> 16);
             }
