@@ -38,7 +38,7 @@ FALLBACK_HBM_GBS = 6650.0
 L2_BYTES = 126 * 2 ** 20
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_main_kernel launch at the named
 # workload, from the ncu capture summarised under profiles/ (None until captured).
-NCU_TRAFFIC_BYTES = {"cfg1": 311490048 + 4783360}     # profiles/decode_main_kernel_cfg1.md
+NCU_TRAFFIC_BYTES = {"cfg1": 310668544 + 3688960, "cfg2": 362961408 + 3549440}     # profiles/decode_main_kernel_cfg1.md, _cfg2.md
 
 
 def measured_hbm_peak():
