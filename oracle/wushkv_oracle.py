@@ -233,7 +233,7 @@ def quantize_rows(X, bits: int, kappa: float):
 def pack_codes(codes, bits: int) -> np.ndarray:
     """Reference bit packing (storage definition only): channel i occupies
     bits [bits*(i % per), bits*(i % per + 1)) of byte i // per, per = 8/bits.
-    The CUDA library is free to permute its physical layout; parity is judged
+    The CUDA library is free to permute its physical layout; parity is checked
     on logical codes."""
     codes = np.asarray(codes, dtype=np.uint8)
     per = 8 // bits
