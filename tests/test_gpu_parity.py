@@ -78,6 +78,22 @@ def test_ragged_batch_shuffled_pages_and_flush_sizes(bits):
         assert L.cache.status() == 0
 
 
+@pytest.mark.parametrize("s_sink,s_keep,s_flush", [(64, 256, 8), (16, 128, 16), (4, 64, 64)])
+def test_serving_window_sizes(s_sink, s_keep, s_flush):
+    """The window sizes of the paper's downstream (Section 5.3: 64 / 256 / 8) and perplexity (Section 5.2:
+    16 / 128 / 16) runs, and a page-sized flush: long sink and recent windows, a boundary that moves in
+    steps of S_flush, lengths around the point where quantization starts."""
+    wl = _wl(8, 2, seed=23, batch=4)
+    edge = s_sink + s_keep + s_flush
+    lengths = [1100, edge - 1, edge, edge + s_flush + 3]
+    L = Layer(wl, lengths, 2, s_sink, s_keep, s_flush)
+    L.fill()
+    assert L.check_append_parity() <= CODE_MISMATCH_MAX
+    _check_window_copies(L)
+    assert L.check_decode_parity() <= 2e-3
+    assert L.cache.status() == 0
+
+
 @pytest.mark.parametrize("path", ["tensor", "cuda"])
 def test_prefill_chunk_paths(path, monkeypatch):
     """Config 4's structure scaled down: several sequences appended as one chunk each in ONE call
