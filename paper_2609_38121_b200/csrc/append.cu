@@ -346,6 +346,9 @@ constexpr int TC_X_PITCH = 136;              // floats per row of the fp32 key t
 constexpr int TC_THREADS = 512;
 constexpr int TC_SMEM_B = 32768;                                   // T_K as bf16 operand
 constexpr int TC_SMEM_X = TC_TILE * TC_X_PITCH * 4;                // fp32 keys; its first 32 KB double as the A operand
+constexpr int TC_SMEM_A = TC_TILE * D * 2;                         // the A operand
+constexpr int TC_V_PITCH = 288;                                    // bytes per staged value row (72 words: quad reads spread over all banks)
+static_assert(TC_SMEM_A + TC_TILE * TC_V_PITCH <= TC_SMEM_X, "the staged value rows must fit behind the A operand");
 constexpr int TC_SMEM_ROWS = TC_TILE * 32;                          // per-row token lookup (RowInfo)
 constexpr int TC_SMEM_TOTAL = TC_SMEM_B + TC_SMEM_X + TC_SMEM_ROWS + 64;
 
@@ -361,6 +364,10 @@ __device__ __forceinline__ unsigned long long umma_smem_desc(unsigned smem_addr)
 constexpr unsigned UMMA_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
 __device__ __forceinline__ unsigned smem_addr_u32(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
+// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros without reading
+__device__ __forceinline__ void cp_async16(unsigned dst, const void* src, unsigned src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
 
 // ---- quad-per-vector quantizer of the chunk path --------------------------------------------------
 // Four adjacent lanes own one 128-vector, 32 entries each.  The clipping quantile needs the two
@@ -469,6 +476,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
     unsigned char* sB = tc_smem;
     unsigned char* sA = tc_smem + TC_SMEM_B;                         // A operand, later overwritten by the fp32 tile
     float* sX = reinterpret_cast<float*>(tc_smem + TC_SMEM_B);
+    unsigned char* sV = tc_smem + TC_SMEM_B + TC_SMEM_A;             // value rows of the tile, until the fp32 tile arrives
     unsigned long long* mbar = reinterpret_cast<unsigned long long*>(tc_smem + TC_SMEM_B + TC_SMEM_X);
     unsigned* tmem_slot = reinterpret_cast<unsigned*>(tc_smem + TC_SMEM_B + TC_SMEM_X + 16);
     RowInfo* rows = reinterpret_cast<RowInfo*>(tc_smem + TC_SMEM_B + TC_SMEM_X + 64);
@@ -509,16 +517,27 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
 
     for (int tile = blockIdx.x; tile < n_tiles && !failed; tile += gridDim.x) {
         const int tok0 = tile * TC_TILE;
-        // ---- A operand: key rows of this tile (zero rows past the end of the batch)
+        // ---- A operand: key rows of this tile (zero rows past the end of the batch), and the value rows of the
+        // tile into the part of the fp32 tile that is free until the MMAs are done; both as 16-byte
+        // asynchronous copies, so that no register waits for them
         {
             const int r8 = lane & 7, cq = lane >> 3;
             for (int item = warp; item < 64; item += TC_THREADS / 32) {
                 const int rg = item >> 2, kc = (item & 3) * 4 + cq;
                 const int tok = tok0 + rg * 8 + r8;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (tok < P.total_new) v = __ldg(reinterpret_cast<const uint4*>(P.K_new + (static_cast<long long>(tok) * P.c.n_kv + head) * D + kc * 8));
-                *reinterpret_cast<uint4*>(sA + rg * TC_SBO + kc * TC_LBO + r8 * 16) = v;
+                const bool in_range = tok < P.total_new;
+                cp_async16(smem_addr_u32(sA + rg * TC_SBO + kc * TC_LBO + r8 * 16),
+                           P.K_new + (static_cast<long long>(in_range ? tok : 0) * P.c.n_kv + head) * D + kc * 8, in_range ? 16u : 0u);
             }
+            if (KK_V > 0) {
+                for (int item = tid; item < TC_TILE * 16; item += TC_THREADS) {
+                    const int row = item >> 4, ch = item & 15;
+                    const bool in_range = tok0 + row < P.total_new;
+                    cp_async16(smem_addr_u32(sV + row * TC_V_PITCH + ch * 16),
+                               P.V_new + (static_cast<long long>(in_range ? tok0 + row : 0) * P.c.n_kv + head) * D + ch * 8, in_range ? 16u : 0u);
+                }
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
         }
         if (tid < TC_TILE) {                                  // where each token of the tile goes
             RowInfo ri;
@@ -529,6 +548,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
             }
             rows[tid] = ri;
         }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // generic-proxy writes -> visible to the tensor core
         __syncthreads();
         // ---- one thread issues the 8 k-steps and commits them to the barrier
@@ -553,12 +573,12 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
             const int row = 8 * warp + (lane >> 2), qd = lane & 3;
             const RowInfo ri = rows[row];
             const bool live = ri.rec_off >= 0;
-            const unsigned short* vsrc = P.V_new + (static_cast<long long>(tok0 + row) * P.c.n_kv + head) * D + 4 * qd;
+            const unsigned char* vrow = sV + row * TC_V_PITCH + 8 * qd;
             float x[32];
             uint2 raw[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
-                raw[k] = live ? __ldg(reinterpret_cast<const uint2*>(vsrc + 16 * k)) : make_uint2(0u, 0u);
+                raw[k] = live ? *reinterpret_cast<const uint2*>(vrow + 32 * k) : make_uint2(0u, 0u);
                 x[4 * k + 0] = bf16_bits_to_float(raw[k].x & 0xffff); x[4 * k + 1] = bf16_bits_to_float(raw[k].x >> 16);
                 x[4 * k + 2] = bf16_bits_to_float(raw[k].y & 0xffff); x[4 * k + 3] = bf16_bits_to_float(raw[k].y >> 16);
             }
