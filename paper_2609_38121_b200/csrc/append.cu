@@ -384,17 +384,24 @@ __device__ __forceinline__ void ce_desc_u(unsigned& a, unsigned& b) {
     const unsigned hi = max(a, b), lo = min(a, b);
     a = hi; b = lo;
 }
-template <int N>
-__device__ __forceinline__ void bitonic_sort_desc(unsigned (&a)[N]) {
-#pragma unroll
-    for (int k = 2; k <= N; k <<= 1)
-#pragma unroll
-        for (int j = k >> 1; j > 0; j >>= 1)
-#pragma unroll
-            for (int i = 0; i < N; ++i) {
-                const int l = i ^ j;
-                if (l > i) { if ((i & k) == 0) ce_desc_u(a[i], a[l]); else ce_desc_u(a[l], a[i]); }
-            }
+// Sorting networks with the fewest known comparators (19 for 8 keys: Batcher's odd-even merge sort;
+// 60 for 16 keys: Green's network), descending; both checked exhaustively with the 0-1 principle.
+__device__ __forceinline__ void sort_desc(unsigned (&a)[8]) {
+    ce_desc_u(a[0], a[1]); ce_desc_u(a[2], a[3]); ce_desc_u(a[0], a[2]); ce_desc_u(a[1], a[3]); ce_desc_u(a[1], a[2]); ce_desc_u(a[4], a[5]); ce_desc_u(a[6], a[7]); ce_desc_u(a[4], a[6]);
+    ce_desc_u(a[5], a[7]); ce_desc_u(a[5], a[6]); ce_desc_u(a[0], a[4]); ce_desc_u(a[2], a[6]); ce_desc_u(a[2], a[4]); ce_desc_u(a[1], a[5]); ce_desc_u(a[3], a[7]); ce_desc_u(a[3], a[5]);
+    ce_desc_u(a[1], a[2]); ce_desc_u(a[3], a[4]); ce_desc_u(a[5], a[6]);
+}
+__device__ __forceinline__ void sort_desc(unsigned (&a)[16]) {
+    ce_desc_u(a[0], a[13]); ce_desc_u(a[1], a[12]); ce_desc_u(a[2], a[15]); ce_desc_u(a[3], a[14]); ce_desc_u(a[4], a[8]); ce_desc_u(a[5], a[6]); ce_desc_u(a[7], a[11]); ce_desc_u(a[9], a[10]);
+    ce_desc_u(a[0], a[5]); ce_desc_u(a[1], a[7]); ce_desc_u(a[2], a[9]); ce_desc_u(a[3], a[4]); ce_desc_u(a[6], a[13]); ce_desc_u(a[8], a[14]); ce_desc_u(a[10], a[15]); ce_desc_u(a[11], a[12]);
+    ce_desc_u(a[0], a[1]); ce_desc_u(a[2], a[3]); ce_desc_u(a[4], a[5]); ce_desc_u(a[6], a[8]); ce_desc_u(a[7], a[9]); ce_desc_u(a[10], a[11]); ce_desc_u(a[12], a[13]); ce_desc_u(a[14], a[15]);
+    ce_desc_u(a[0], a[2]); ce_desc_u(a[1], a[3]); ce_desc_u(a[4], a[10]); ce_desc_u(a[5], a[11]); ce_desc_u(a[6], a[7]); ce_desc_u(a[8], a[9]); ce_desc_u(a[12], a[14]); ce_desc_u(a[13], a[15]);
+    ce_desc_u(a[1], a[2]); ce_desc_u(a[3], a[12]); ce_desc_u(a[4], a[6]); ce_desc_u(a[5], a[7]); ce_desc_u(a[8], a[10]); ce_desc_u(a[9], a[11]); ce_desc_u(a[13], a[14]);
+    ce_desc_u(a[1], a[4]); ce_desc_u(a[2], a[6]); ce_desc_u(a[5], a[8]); ce_desc_u(a[7], a[10]); ce_desc_u(a[9], a[13]); ce_desc_u(a[11], a[14]);
+    ce_desc_u(a[2], a[4]); ce_desc_u(a[3], a[6]); ce_desc_u(a[9], a[12]); ce_desc_u(a[11], a[13]);
+    ce_desc_u(a[3], a[5]); ce_desc_u(a[6], a[8]); ce_desc_u(a[7], a[9]); ce_desc_u(a[10], a[12]);
+    ce_desc_u(a[3], a[4]); ce_desc_u(a[5], a[6]); ce_desc_u(a[7], a[8]); ce_desc_u(a[9], a[10]); ce_desc_u(a[11], a[12]);
+    ce_desc_u(a[6], a[7]); ce_desc_u(a[8], a[9]);
 }
 template <int N>
 __device__ __forceinline__ void bitonic_merge_desc(unsigned (&a)[N]) {      // bitonic sequence -> descending
@@ -424,7 +431,7 @@ __device__ __forceinline__ void quad_quantize(const float (&x)[32], ClipRule rul
         unsigned tmp[KK];
 #pragma unroll
         for (int i = 0; i < KK; ++i) tmp[i] = __float_as_uint(x[g0 + i]) & 0x7fffffffu;
-        bitonic_sort_desc<KK>(tmp);
+        sort_desc(tmp);
         if (g0 == 0) {
 #pragma unroll
             for (int i = 0; i < KK; ++i) top[i] = tmp[i];
