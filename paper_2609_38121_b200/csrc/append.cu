@@ -1,6 +1,11 @@
 // Quantize-on-append (Algorithm 2 lines 3-4 and 9-12; quantizer: Section 5.3 Eq. 6).
 //
-// Warp-per-vector path: one warp owns one (new token, KV head) pair.  It computes k' = T_K k on
+// Three kernels, chosen by wushkv_append from the shape of the call:
+//   append_chunk_kernel  prefill chunks (max_new >= 128): key transform on tcgen05, four lanes per vector
+//                        for the quantizer (described where it is defined, further down);
+//   append_token_kernel  one token per sequence (a decode step): one CTA per sequence, single launch;
+//   append_rows_kernel   everything else, and the chunk path when WUSHKV_APPEND_PATH=cuda.
+// The last two share the warp-per-vector path: one warp owns one (new token, KV head) pair.  It computes k' = T_K k on
 // CUDA cores against a transposed copy of T_K in shared memory (keys only), then for k' and for v:
 // finds the clip range (min, max and the two order statistics around rank kappa*(d-1) of |x| by
 // repeated warp-wide maximum extraction), derives the fp16 step / offset, rounds the codes with
@@ -331,9 +336,12 @@ __global__ void __launch_bounds__(1024) append_token_kernel(AppendParams P) {
 // tcgen05 tile: A = the 128 x 128 bf16 key tile, B = T_K (bf16, [out][in] is already the K-major B
 // operand), D = 128 x 128 fp32 in tensor memory (lane = token, column = output channel).  bf16 x bf16
 // products are exact in fp32, so the result differs from the CUDA-core paths only by summation order.
-// A CTA keeps its head's T_K resident in shared memory and walks over token tiles; while the tensor
-// core works on the keys, the warps quantize the tile's values; the fp32 keys then come back through
-// tcgen05.ld into shared memory and take the same warp-per-vector quantizer.
+// A CTA keeps its head's T_K resident in shared memory and walks over token tiles.  The key tile (straight
+// into the operand layout) and the tile's value rows arrive by 16-byte cp.async copies; while the tensor
+// core works on the keys, the warps quantize the values out of shared memory (they are parked in the part
+// of the fp32 tile that stays free until the MMAs are done); the fp32 keys then come back through
+// tcgen05.ld into shared memory and are quantized the same way: four lanes per vector, each keeping the
+// largest 8 or 16 of its 32 entries with sorting networks on registers (quad_quantize).
 //
 // Shared-memory operand layout (no swizzle, K-major "interleaved"): the tile is cut into core matrices
 // of 8 rows x 16 bytes (8 bf16) stored as 128 contiguous bytes; core matrix (row group rg, k chunk kc)
