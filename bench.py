@@ -206,7 +206,8 @@ class Session:
         return self.batch * (self.chunk if self.chunk else 1)
 
     def launches_per_step(self):
-        return 2 + 3       # append: rows + length update; decode: prep + main + combine
+        # chunk append: transform/quantize kernel + length update; token append: one kernel; decode: prep + main + combine
+        return (2 if self.chunk else 1) + 3
 
 
 # ------------------------------------------------------------------------------------------------
