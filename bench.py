@@ -9,8 +9,9 @@ Prints ONE JSON line (rank 0).  `value` is the metric of the benchmark definitio
 cache (codes + scale/zero + bf16 windows) that one decode step must read, divided by the time of the
 whole step (append + decode), with every input already resident in HBM.  `roofline` times the decode
 main kernel alone (CUDA events recorded around it by the library on the launching stream).  `e2e`
-repeats the steps through the host-buffer entry point (pinned host inputs copied in, result copied
-out, one synchronisation per step).  `cpu_baseline` times the float64 oracle on a bounded slice.
+repeats the steps through the host-buffer entry point (the step's new token and queries come from pinned
+host memory, the outputs go back to it, one synchronisation per step; the library reads and writes
+pinned buffers in place over the bus and falls back to staged copies otherwise).  `cpu_baseline` times the float64 oracle on a bounded slice.
 With N > 1 every rank runs its own replica of the workload (the path has no cross-GPU exchange).
 """
 from __future__ import annotations
@@ -38,7 +39,8 @@ FALLBACK_HBM_GBS = 6650.0
 L2_BYTES = 126 * 2 ** 20
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_main_kernel launch at the named
 # workload, from the ncu capture summarised under profiles/ (None until captured).
-NCU_TRAFFIC_BYTES = {"cfg1": 310668544 + 3688960, "cfg2": 362961408 + 3549440}     # profiles/decode_main_kernel_cfg1.md, _cfg2.md
+NCU_TRAFFIC_BYTES = {"cfg1": 310668544 + 3688960, "cfg2": 362961408 + 3549440,
+                     "cfg3": 76140032 + 3253760}      # profiles/decode_main_kernel_cfg1.md, _cfg2.md, _cfg3.md
 
 
 def measured_hbm_peak():
