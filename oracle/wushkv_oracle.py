@@ -19,7 +19,7 @@ Conventions
 * Positions are 0-based; the paper's ``S_start < s <= S_quant`` (1-based) is
   the 0-based half-open range ``[S_start, S_quant)``.
 
-Parity pins (tests/test_oracle_*.py) cover every function below; none is
+Parity pins (tests/test_oracle_*.py, tests/test_golden.py) cover every function below; none is
 "parity unpinned" against the mathematics.  What the paper itself does not fix
 (quantile interpolation rule, tie rounding, storage precision of scale and
 zero, the boundary used at attention time) cannot be pinned to the paper; each
