@@ -53,6 +53,9 @@ def test_host_validation_rejects_bad_arguments_without_cuda():
     desc = B.wushkv_cache()                                  # all zero
     assert B.lib.wushkv_append(C.byref(desc), 1, None, None, None, 1, 1, None, None, None) == B.EINVAL
     assert B.lib.wushkv_decode_attn(C.byref(desc), 1, None, None, 64, None, None, None, 0, None) == B.EINVAL
+    assert B.lib.wushkv_decode_step(C.byref(desc), 1, None, None, None, 64, None, None, None, None, None, 0, None) == B.EINVAL
+    assert B.lib.wushkv_decode_step_host(C.byref(desc), 1, None, None, None, 64, None, None, None, None, None, 0, None, 0,
+                                         None) != B.OK
     assert B.lib.wushkv_decode_workspace_bytes(C.byref(desc), 1, 64) == 0
     assert B.lib.wushkv_build_transforms(1, 12, None, None, 0.0, None, None) == B.EINVAL
     with pytest.raises(B.WushkvError):
