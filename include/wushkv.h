@@ -61,6 +61,10 @@ extern "C" {
 #define WUSHKV_DEV_BAD_PAGE_ID     2  /* page table entry outside [0, n_pages): access skipped   */
 #define WUSHKV_DEV_BAD_SLOT        4  /* slot[b] outside [0, n_slots): sequence skipped          */
 #define WUSHKV_DEV_COPY_TIMEOUT    8  /* a staged page copy did not arrive within the wait limit */
+#define WUSHKV_DEV_BAD_COUNT      16  /* max_new == 1 was promised but a sequence brought more than one token: sequence skipped */
+#define WUSHKV_DEV_VALUE_RANGE    32  /* a stored value step Delta_v >= 1024: beyond the fp16 range of the decode value contraction */
+/* After PAGE_TABLE_FULL, BAD_PAGE_ID, BAD_SLOT or BAD_COUNT in wushkv_append the length of the affected
+ * sequence is left as it was (tokens of the call that did fit are orphaned: nothing reads them). */
 
 /*
  * One layer's cache description.  Plain data; the caller fills it for every call.
@@ -149,8 +153,8 @@ int wushkv_build_transforms(int32_t n_heads, int32_t d, const double* M, const d
  *   V_new (device): bf16 [total_new][n_kv][d] values in the folded basis, 16-byte aligned.
  * Chunks (max_new >= 128) take the tensor-core transform path (tcgen05, fp32 accumulation in
  * tensor memory), max_new == 1 a single-launch decode-time path, anything else a CUDA-core path.
- * All produce the same codes up to fp32 summation order.  Environment variable
- * WUSHKV_APPEND_PATH=cuda forces the CUDA-core path for chunks (testing aid).
+ * All produce the same codes up to fp32 summation order (wushkv_set_test_option("append_path_cuda", 1)
+ * forces the CUDA-core path for chunks).
  */
 int wushkv_append(const wushkv_cache* cache, int32_t batch, const int32_t* slot, int32_t* seq_len,
                   const int32_t* cu_new, int32_t total_new, int32_t max_new,
@@ -179,9 +183,11 @@ size_t wushkv_decode_workspace_bytes(const wushkv_cache* cache, int32_t batch, i
  * Range: probabilities times the stored value step are fed to the tensor core in fp16 with up to
  * 2^6 of headroom, so a stored Delta_v of 1024 or more (a value range beyond ~3000 at 2 bits)
  * saturates and loses accuracy; keys have no such limit.
- * Environment (testing aids): WUSHKV_DECODE_CTAS=<n> fixes the number of thread blocks of the main
- * kernel (the split count); WUSHKV_DECODE_PATH=tc selects, for n_q / n_kv <= 4, an alternative main
- * kernel that computes the scores with tcgen05 (same results to rounding, slower).
+ * The scores of the quantized positions are computed from a 16-bit fixed-point copy of q' (exact
+ * integer dot products with the codes), i.e. they are the scores of a query that differs from q' by
+ * at most 2^-16 of its largest entry per channel.
+ * NaN or infinite inputs (Q, or stored steps / offsets derived from such keys and values) give
+ * unspecified finite-or-NaN outputs for the affected sequences; nothing traps.
  */
 int wushkv_decode_attn(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
                        int32_t max_seq_len, const uint16_t* Q, float* O,
@@ -266,6 +272,23 @@ int wushkv_decode_attn_static(const wushkv_cache* cache, int32_t batch, const in
  * can time that kernel alone.  Pass NULLs to switch it off.  Process-wide, not thread-safe.
  */
 int wushkv_set_profile_events(void* start, void* stop);
+
+/*
+ * Testing aids (not part of the method).  Process-wide and unsynchronised: set them from one thread while
+ * no call of the library is running.  The first three take their initial value from the environment
+ * (WUSHKV_DECODE_CTAS=<n>, WUSHKV_APPEND_PATH=cuda, WUSHKV_HOST_IO=copy), read once per process.
+ *   "decode_ctas"       n > 0: number of thread blocks of the decode main kernel (the split count); 0: automatic.
+ *   "append_path_cuda"  1: prefill chunks take the CUDA-core append path instead of the tensor-core one.
+ *   "host_io_copy"      1: wushkv_decode_step_host always stages its host buffers with copies.
+ *   "drop_copy_unit"    u >= 0: the decode main kernel does not issue the copy of work unit u of its flattened
+ *                       list, so that the wait for it runs into its limit (WUSHKV_DEV_COPY_TIMEOUT is set
+ *                       in *dev_status and the kernel returns); -1: off.
+ *   "wait_limit"        n > 0: poll limit of the device-side barrier waits (default: about a second); 0: default.
+ *   "drop_chunk_mma"    1: the chunk append does not commit the MMAs of its first tile to their barrier (same
+ *                       failure path in that kernel).
+ * Returns WUSHKV_EINVAL for an unknown name.
+ */
+int wushkv_set_test_option(const char* name, long long value);
 
 #ifdef __cplusplus
 }

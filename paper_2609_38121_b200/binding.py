@@ -19,7 +19,7 @@ EXPORTS = (
     "wushkv_page_bytes", "wushkv_status_string", "wushkv_accumulate_gram", "wushkv_build_transforms",
     "wushkv_append", "wushkv_decode_workspace_bytes", "wushkv_decode_attn", "wushkv_unpack_debug",
     "wushkv_decode_step", "wushkv_step_staging_bytes", "wushkv_decode_step_host", "wushkv_set_profile_events",
-    "wushkv_decode_attn_static",
+    "wushkv_decode_attn_static", "wushkv_set_test_option",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -86,6 +86,8 @@ def _load():
                                               C.c_void_p, C.c_void_p, C.c_void_p]
     lib.wushkv_set_profile_events.restype = C.c_int
     lib.wushkv_set_profile_events.argtypes = [C.c_void_p, C.c_void_p]
+    lib.wushkv_set_test_option.restype = C.c_int
+    lib.wushkv_set_test_option.argtypes = [C.c_char_p, C.c_longlong]
     return lib
 
 
@@ -198,6 +200,11 @@ def set_profile_events(start=None, stop=None):
     a = C.c_void_p(start.cuda_event) if start is not None else None
     b = C.c_void_p(stop.cuda_event) if stop is not None else None
     _check(lib.wushkv_set_profile_events(a, b), "wushkv_set_profile_events")
+
+
+def set_test_option(name: str, value: int):
+    """wushkv_set_test_option: process-wide testing aids (see the header for the names)."""
+    _check(lib.wushkv_set_test_option(name.encode(), int(value)), "wushkv_set_test_option")
 
 
 class PagedCache:

@@ -1,5 +1,36 @@
 // Small host-only entry points of the C ABI.
+#include <cstdlib>
+#include <cstring>
+
 #include "host_common.h"
+
+namespace wushkv {
+
+Knobs& knobs() {
+    static Knobs k = [] {
+        Knobs v;
+        if (const char* e = std::getenv("WUSHKV_DECODE_CTAS")) v.decode_ctas = std::atoll(e);
+        if (const char* e = std::getenv("WUSHKV_APPEND_PATH")) v.append_path_cuda = e[0] == 'c';
+        if (const char* e = std::getenv("WUSHKV_HOST_IO")) v.host_io_copy = e[0] == 'c';
+        return v;
+    }();
+    return k;
+}
+
+}  // namespace wushkv
+
+extern "C" int wushkv_set_test_option(const char* name, long long value) {
+    if (!name) return WUSHKV_EINVAL;
+    wushkv::Knobs& k = wushkv::knobs();
+    if (!std::strcmp(name, "decode_ctas")) k.decode_ctas = value;
+    else if (!std::strcmp(name, "append_path_cuda")) k.append_path_cuda = value != 0;
+    else if (!std::strcmp(name, "host_io_copy")) k.host_io_copy = value != 0;
+    else if (!std::strcmp(name, "drop_copy_unit")) k.drop_copy_unit = value;
+    else if (!std::strcmp(name, "wait_limit")) k.wait_limit = value;
+    else if (!std::strcmp(name, "drop_chunk_mma")) k.drop_chunk_mma = value != 0;
+    else return WUSHKV_EINVAL;
+    return WUSHKV_OK;
+}
 
 extern "C" size_t wushkv_page_bytes(int32_t n_kv, int32_t d, int32_t bits, int32_t page_tokens) {
     if (n_kv <= 0 || d != wushkv::D || page_tokens != wushkv::PAGE_TOKENS || (bits != 2 && bits != 4)) return 0;

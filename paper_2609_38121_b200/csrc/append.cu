@@ -25,6 +25,9 @@ namespace wushkv {
 
 constexpr unsigned FULL = 0xffffffffu;
 constexpr int TT_STRIDE = 132;   // floats per row of the transposed transform in shared memory
+// The decode kernel feeds (probability x value step) to the tensor core in fp16 with 2^6 of headroom:
+// a stored value step at or beyond this limit can saturate there, so the append flags it.
+constexpr float VALUE_STEP_LIMIT = 1024.f;
 
 struct ClipRule {     // rank rule of quantile_kappa(|x|) with linear interpolation
     int rounds;       // extraction rounds: the last yields a[lo], the one before a[lo+1]
@@ -59,7 +62,7 @@ __device__ __forceinline__ float order_key_inv(unsigned k) {
 // codes of this lane and the stored (fp16) step and offset.
 template <int BITS>
 __device__ __forceinline__ void quantize_vec(const float (&x)[4], ClipRule rule, int lane, int (&code)[4],
-                                             __half& step_h, __half& xmin_h) {
+                                             __half& step_h, __half& xmin_h, int* value_status = nullptr) {
     constexpr int LEVELS = (1 << BITS) - 1;
     // ---- the two order statistics of |x| around rank kappa*(d-1)
     unsigned u0 = __float_as_uint(x[0]) & 0x7fffffffu, u1 = __float_as_uint(x[1]) & 0x7fffffffu;
@@ -87,6 +90,7 @@ __device__ __forceinline__ void quantize_vec(const float (&x)[4], ClipRule rule,
     step_h = __float2half_rn(fminf(fmaxf(step, -65504.f), 65504.f));
     xmin_h = __float2half_rn(fminf(fmaxf(x_min, -65504.f), 65504.f));
     const float step_s = __half2float(step_h), xmin_s = __half2float(xmin_h);
+    if (value_status != nullptr && step_s >= VALUE_STEP_LIMIT && lane == 0) atomicOr(value_status, WUSHKV_DEV_VALUE_RANGE);
     const float inv = step_s > 0.f ? __frcp_rn(step_s) : 0.f;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
@@ -96,30 +100,24 @@ __device__ __forceinline__ void quantize_vec(const float (&x)[4], ClipRule rule,
 }
 
 // Scatter one token's K codes (lane holds channels 4*lane..+3) into the record; r = token row in page.
+// Channel 4 lane + e sits in k-step s = lane >> 3, channel half hh = (lane >> 2) & 1, byte 2 ((lane >> 1) & 1) + (e & 1)
+// of the word of fragment lane t = 2 (lane & 1) + (e >> 1).
 template <int BITS>
 __device__ __forceinline__ void store_k_codes(unsigned char* rec, int r, const int (&code)[4], int lane) {
     const int bi = r >> 4, rr = r & 15, g = rr & 7, rs = rr >> 3;
-    const int s = lane >> 2;                            // k-step of all four channels of this lane
-    const int sh = (BITS == 2) ? 2 * s : 4 * (s & 3);
-    unsigned wa = (static_cast<unsigned>(code[0]) << sh) | (static_cast<unsigned>(code[1]) << (16 + sh));
-    unsigned wb = (static_cast<unsigned>(code[2]) << sh) | (static_cast<unsigned>(code[3]) << (16 + sh));
-    wa |= __shfl_xor_sync(FULL, wa, 4);  wb |= __shfl_xor_sync(FULL, wb, 4);
-    wa |= __shfl_xor_sync(FULL, wa, 8);  wb |= __shfl_xor_sync(FULL, wb, 8);
+    const int s = lane >> 3, b0 = 2 * ((lane >> 1) & 1);
+    const int sh = 8 * b0 + ((BITS == 2) ? 2 * s : 4 * (s & 1));
+    unsigned wa = (static_cast<unsigned>(code[0]) << sh) | (static_cast<unsigned>(code[1]) << (8 + sh));   // t = 2 (lane & 1)
+    unsigned wb = (static_cast<unsigned>(code[2]) << sh) | (static_cast<unsigned>(code[3]) << (8 + sh));   // t = 2 (lane & 1) + 1
+    wa |= __shfl_xor_sync(FULL, wa, 2);  wb |= __shfl_xor_sync(FULL, wb, 2);       // the other byte pair
+    wa |= __shfl_xor_sync(FULL, wa, 8);  wb |= __shfl_xor_sync(FULL, wb, 8);       // the fields / nibbles of the same byte
     if (BITS == 2) { wa |= __shfl_xor_sync(FULL, wa, 16); wb |= __shfl_xor_sync(FULL, wb, 16); }
-    const int w = (lane & 3) >> 1, ta = 2 * (lane & 1);
-    if (BITS == 2) {
-        if (lane < 4) {
-            unsigned char* p = rec + bi * 512 + 16 * (4 * g + ta) + 8 * rs + 4 * w;
-            *reinterpret_cast<unsigned*>(p) = wa;
-            *reinterpret_cast<unsigned*>(p + 16) = wb;
-        }
-    } else {
-        if ((lane & 12) == 0) {                         // lanes 0..3 (k-steps 0..3) and 16..19 (k-steps 4..7)
-            const int j = 2 * (lane >> 4) + w;
-            unsigned char* p = rec + bi * 1024 + 512 * rs + 16 * (4 * g + ta) + 4 * j;
-            *reinterpret_cast<unsigned*>(p) = wa;
-            *reinterpret_cast<unsigned*>(p + 16) = wb;
-        }
+    const int hh = (lane >> 2) & 1, ta = 2 * (lane & 1), j = rs + 2 * hh;
+    const bool writer = BITS == 2 ? (lane & 26) == 0 : (lane & 10) == 0;
+    if (writer) {
+        unsigned char* p = rec + bi * code_block_bytes(BITS) + (BITS == 4 ? 512 * (lane >> 4) : 0) + 16 * (4 * g + ta) + 4 * j;
+        *reinterpret_cast<unsigned*>(p) = wa;
+        *reinterpret_cast<unsigned*>(p + 16) = wb;
     }
 }
 
@@ -240,7 +238,7 @@ __global__ void __launch_bounds__(256) append_rows_kernel(AppendParams P) {
         const uint2 vraw = __ldg(reinterpret_cast<const uint2*>(P.V_new + row) + lane);
         float v[4] = {bf16_bits_to_float(vraw.x & 0xffff), bf16_bits_to_float(vraw.x >> 16),
                       bf16_bits_to_float(vraw.y & 0xffff), bf16_bits_to_float(vraw.y >> 16)};
-        quantize_vec<BITS>(v, P.rule_v, lane, code, step_h, xmin_h);
+        quantize_vec<BITS>(v, P.rule_v, lane, code, step_h, xmin_h, P.c.dev_status);
         store_v_codes<BITS>(ts.rec, ts.r, code, lane);
         if (lane == 0) { meta[2] = step_h; meta[3] = xmin_h; }
         store_window_copy(P, ts, head, 1, vraw, lane);
@@ -265,7 +263,11 @@ __global__ void __launch_bounds__(1024) append_token_kernel(AppendParams P) {
     float* kp_s = tok_s + n_kv * D;
     const int first = __ldg(P.cu_new + b), n_new = __ldg(P.cu_new + b + 1) - first;
     if (n_new <= 0) return;
-    const int s0 = __ldg(P.seq_len + b);
+    if (n_new > 1) {                                     // the host promised one token per sequence
+        if (threadIdx.x == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_COUNT);
+        return;
+    }
+    const int s0 = P.seq_len[b];                         // written by this kernel: not through the read-only path
     const int slot0 = __ldg(P.slot + b);                 // the page lookup does not depend on the transform: start it now
     int page = -1;
     if (slot0 >= 0 && slot0 < P.c.n_slots && s0 >= 0 && s0 / PAGE_TOKENS < P.c.max_pages)
@@ -321,14 +323,14 @@ __global__ void __launch_bounds__(1024) append_token_kernel(AppendParams P) {
             }
             int code[4];
             __half step_h, xmin_h;
-            quantize_vec<BITS>(x, which ? P.rule_v : P.rule_k, lane, code, step_h, xmin_h);
+            quantize_vec<BITS>(x, which ? P.rule_v : P.rule_k, lane, code, step_h, xmin_h, which ? P.c.dev_status : nullptr);
             if (which == 0) store_k_codes<BITS>(ts.rec, ts.r, code, lane); else store_v_codes<BITS>(ts.rec, ts.r, code, lane);
             __half* meta = reinterpret_cast<__half*>(ts.rec + meta_location(BITS, ts.r));
             if (lane == 0) { meta[2 * which] = step_h; meta[2 * which + 1] = xmin_h; }
             store_window_copy(P, ts, head, which, copy, lane);
         }
     }
-    if (threadIdx.x == 0) P.seq_len[b] = s0 + 1;          // every read of the old length happened before the barriers above
+    if (ok && threadIdx.x == 0) P.seq_len[b] = s0 + 1;    // every read of the old length happened before the barriers above
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -431,7 +433,8 @@ __device__ __forceinline__ void keep_largest(unsigned (&top)[N], const unsigned 
 // Clip range, stored step / offset and the 32 codes of this lane's entries x[32] (Eq. 6); all four
 // lanes of the quad return the same step_h / xmin_h.
 template <int BITS, int KK>
-__device__ __forceinline__ void quad_quantize(const float (&x)[32], ClipRule rule, int (&code)[32], __half& step_h, __half& xmin_h) {
+__device__ __forceinline__ void quad_quantize(const float (&x)[32], ClipRule rule, int (&code)[32], __half& step_h, __half& xmin_h,
+                                              int* value_status = nullptr, bool flag_lane = false) {
     constexpr int LEVELS = (1 << BITS) - 1;
     unsigned top[KK];
 #pragma unroll
@@ -474,6 +477,7 @@ __device__ __forceinline__ void quad_quantize(const float (&x)[32], ClipRule rul
     step_h = __float2half_rn(fminf(fmaxf(step, -65504.f), 65504.f));
     xmin_h = __float2half_rn(fminf(fmaxf(x_min, -65504.f), 65504.f));
     const float step_s = __half2float(step_h), xmin_s = __half2float(xmin_h);
+    if (value_status != nullptr && flag_lane && step_s >= VALUE_STEP_LIMIT) atomicOr(value_status, WUSHKV_DEV_VALUE_RANGE);
     const float inv = step_s > 0.f ? __frcp_rn(step_s) : 0.f;
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
@@ -599,7 +603,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
             }
             int code[32];
             __half step_h, xmin_h;
-            quad_quantize<BITS, KQ>(x, P.rule_v, code, step_h, xmin_h);
+            quad_quantize<BITS, KQ>(x, P.rule_v, code, step_h, xmin_h, P.c.dev_status, live && qd == 0);
             if (live) {
                 unsigned char* rec = P.c.pages + ri.rec_off;
                 const int bi = ri.r >> 4, rr = ri.r & 15, ps = rr >> 3, t = (rr & 7) >> 1, hi = rr & 1;
@@ -651,7 +655,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
                               bf16_bits_to_float(vraw.y & 0xffff), bf16_bits_to_float(vraw.y >> 16)};
                 int code[4];
                 __half step_h, xmin_h;
-                quantize_vec<BITS>(x, P.rule_v, lane, code, step_h, xmin_h);
+                quantize_vec<BITS>(x, P.rule_v, lane, code, step_h, xmin_h, P.c.dev_status);
                 store_v_codes<BITS>(ts.rec, ts.r, code, lane);
                 __half* meta = reinterpret_cast<__half*>(ts.rec + meta_location(BITS, ts.r));
                 if (lane == 0) { meta[2] = step_h; meta[3] = xmin_h; }
@@ -714,22 +718,28 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
             if (live) {
                 unsigned char* rec = P.c.pages + ri.rec_off;
                 const int bi = ri.r >> 4, rr = ri.r & 15, g = rr & 7, rs = rr >> 3;
+                // entry 4k + j is byte j of the word of channel half k & 1, field / nibble of k-step k >> 1
                 if (BITS == 2) {
-                    uint2 w = make_uint2(0u, 0u);
+                    unsigned w[2] = {0u, 0u};
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        w.x |= (static_cast<unsigned>(code[4 * k + 0]) << (2 * k)) | (static_cast<unsigned>(code[4 * k + 1]) << (16 + 2 * k));
-                        w.y |= (static_cast<unsigned>(code[4 * k + 2]) << (2 * k)) | (static_cast<unsigned>(code[4 * k + 3]) << (16 + 2 * k));
-                    }
-                    *reinterpret_cast<uint2*>(rec + bi * 512 + 16 * (4 * g + qd) + 8 * rs) = w;
+                    for (int k = 0; k < 8; ++k)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) w[k & 1] |= static_cast<unsigned>(code[4 * k + j]) << (8 * j + 2 * (k >> 1));
+                    unsigned char* p = rec + bi * 512 + 16 * (4 * g + qd) + 4 * rs;
+                    *reinterpret_cast<unsigned*>(p) = w[0];
+                    *reinterpret_cast<unsigned*>(p + 8) = w[1];
                 } else {
-                    unsigned w[4] = {0u, 0u, 0u, 0u};         // word 2 (k >> 2) + (j >> 1), field k & 3
+                    unsigned w[2][2] = {{0u, 0u}, {0u, 0u}};      // [512-byte half][channel half]
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        w[2 * (k >> 2) + 0] |= (static_cast<unsigned>(code[4 * k + 0]) << (4 * (k & 3))) | (static_cast<unsigned>(code[4 * k + 1]) << (16 + 4 * (k & 3)));
-                        w[2 * (k >> 2) + 1] |= (static_cast<unsigned>(code[4 * k + 2]) << (4 * (k & 3))) | (static_cast<unsigned>(code[4 * k + 3]) << (16 + 4 * (k & 3)));
+                    for (int k = 0; k < 8; ++k)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) w[k >> 2][k & 1] |= static_cast<unsigned>(code[4 * k + j]) << (8 * j + 4 * ((k >> 1) & 1));
+#pragma unroll
+                    for (int pq = 0; pq < 2; ++pq) {
+                        unsigned char* p = rec + bi * 1024 + 512 * pq + 16 * (4 * g + qd) + 4 * rs;
+                        *reinterpret_cast<unsigned*>(p) = w[pq][0];
+                        *reinterpret_cast<unsigned*>(p + 8) = w[pq][1];
                     }
-                    *reinterpret_cast<uint4*>(rec + bi * 1024 + 512 * rs + 16 * (4 * g + qd)) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
                 if (qd == 0) {
                     __half* meta = reinterpret_cast<__half*>(rec + meta_location(BITS, ri.r));
@@ -778,9 +788,23 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(128u) : "memory");
 }
 
-__global__ void advance_len_kernel(int batch, int* seq_len, const int* cu_new) {
+// Advances the lengths after a rows / chunk append.  A sequence one of whose tokens could not be stored
+// (bad slot, page table too short, page id outside the pool: the append kernel flagged it and skipped
+// that token) keeps its old length.
+__global__ void advance_len_kernel(CacheView c, int batch, const int* slot, int* seq_len, const int* cu_new) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b < batch) seq_len[b] += cu_new[b + 1] - cu_new[b];
+    if (b >= batch) return;
+    const int n_new = cu_new[b + 1] - cu_new[b];
+    if (n_new <= 0) return;
+    const int s0 = seq_len[b], sl = slot[b];
+    if (sl < 0 || sl >= c.n_slots || s0 < 0) return;
+    const int p0 = s0 / PAGE_TOKENS, p1 = (s0 + n_new - 1) / PAGE_TOKENS;
+    if (p1 >= c.max_pages) return;
+    for (int p = p0; p <= p1; ++p) {
+        const int page = c.page_table[static_cast<long long>(sl) * c.max_pages + p];
+        if (page < 0 || page >= c.n_pages) return;
+    }
+    seq_len[b] = s0 + n_new;
 }
 
 __global__ void unpack_debug_kernel(CacheView c, int slot, int head, int which, int pos0, int n,
@@ -796,8 +820,8 @@ __global__ void unpack_debug_kernel(CacheView c, int slot, int head, int which, 
     const unsigned char* rec = c.pages + (static_cast<long long>(page) * c.n_kv + head) * record_bytes(c.bits);
     int off, bit;
     if (which == 0) k_code_location(c.bits, r, ch, off, bit); else v_code_location(c.bits, r, ch, off, bit);
-    const unsigned hw = *reinterpret_cast<const unsigned short*>(rec + off);
-    codes[idx] = static_cast<unsigned char>((hw >> bit) & ((1u << c.bits) - 1u));
+    const unsigned byte = rec[off + (bit >> 3)];          // little-endian half-words: bit 8.. is the second byte
+    codes[idx] = static_cast<unsigned char>((byte >> (bit & 7)) & ((1u << c.bits) - 1u));
     if (ch == 0) {
         const __half* meta = reinterpret_cast<const __half*>(rec + meta_location(c.bits, r));
         scale[tok] = __half2float(meta[2 * which]);
@@ -852,8 +876,7 @@ extern "C" int wushkv_append(const wushkv_cache* cache, int32_t batch, const int
                                              : cudaLaunchKernelEx(&cfg, append_token_kernel<4>, P);
         return e1 == cudaSuccess ? WUSHKV_OK : WUSHKV_ECUDA;
     }
-    const char* path_env = std::getenv("WUSHKV_APPEND_PATH");          // "cuda" forces the CUDA-core chunk path (testing)
-    const bool force_cuda = path_env && path_env[0] == 'c';
+    const bool force_cuda = knobs().append_path_cuda != 0;             // testing aid: CUDA-core path for chunks too
     if (max_new >= TC_TILE && !force_cuda) {    // prefill chunk: tensor-core transform
         const int n_tiles = (total_new + TC_TILE - 1) / TC_TILE;
         const int per_head = std::max(1, std::min(n_tiles, 2 * sm_count() / P.c.n_kv));
@@ -863,7 +886,7 @@ extern "C" int wushkv_append(const wushkv_cache* cache, int32_t batch, const int
         const int kk_k = need > 16 ? 0 : (P.rule_k.rounds <= 8 ? 8 : 16);
         const int kk_v = need > 16 ? 0 : (P.rule_v.rounds <= 8 ? 8 : 16);
         auto launch = [&](auto kernel) -> bool {
-            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_TOTAL) != cudaSuccess) return false;
+            if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(kernel), TC_SMEM_TOTAL)) return false;
             kernel<<<grid_tc, TC_THREADS, TC_SMEM_TOTAL, st>>>(P);
             return true;
         };
@@ -883,7 +906,7 @@ extern "C" int wushkv_append(const wushkv_cache* cache, int32_t batch, const int
         }
         if (!ok) return WUSHKV_ECUDA;
         if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
-        advance_len_kernel<<<(batch + 127) / 128, 128, 0, st>>>(batch, seq_len, cu_new);
+        advance_len_kernel<<<(batch + 127) / 128, 128, 0, st>>>(P.c, batch, slot, seq_len, cu_new);
         return cudaGetLastError() == cudaSuccess ? WUSHKV_OK : WUSHKV_ECUDA;
     }
     // enough CTAs to fill the machine, but at least 8 tokens each to amortise the transform load
@@ -893,18 +916,15 @@ extern "C" int wushkv_append(const wushkv_cache* cache, int32_t batch, const int
     P.tokens_per_cta = tpc;
     const dim3 grid((total_new + tpc - 1) / tpc, P.c.n_kv);
     const size_t smem = static_cast<size_t>(D) * TT_STRIDE * sizeof(float);
-    cudaError_t e;
     if (P.c.bits == 2) {
-        e = cudaFuncSetAttribute(append_rows_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-        if (e != cudaSuccess) return WUSHKV_ECUDA;
+        if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(append_rows_kernel<2>), static_cast<int>(smem))) return WUSHKV_ECUDA;
         append_rows_kernel<2><<<grid, 256, smem, st>>>(P);
     } else {
-        e = cudaFuncSetAttribute(append_rows_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-        if (e != cudaSuccess) return WUSHKV_ECUDA;
+        if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(append_rows_kernel<4>), static_cast<int>(smem))) return WUSHKV_ECUDA;
         append_rows_kernel<4><<<grid, 256, smem, st>>>(P);
     }
     if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
-    advance_len_kernel<<<(batch + 127) / 128, 128, 0, st>>>(batch, seq_len, cu_new);
+    advance_len_kernel<<<(batch + 127) / 128, 128, 0, st>>>(P.c, batch, slot, seq_len, cu_new);
     if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
     return WUSHKV_OK;
 }

@@ -2,30 +2,32 @@
 //
 // Three launches on the caller's stream:
 //   1. decode_prep_kernel   q' = T_K^{-T} q per query head (Algorithm 2 line 3), written as mma
-//                           B-fragments: fp16 (value + rounding remainder), pre-scaled by the power of
-//                           two that each packed code field carries, for the quantized positions, and
-//                           bf16 (value + remainder) for the bf16 windows.  Block (0,0) also writes the
+//                           B-fragments: for the quantized positions a 16-bit fixed-point copy of q' split
+//                           into two signed bytes per channel (the operand of the integer mma), for the
+//                           bf16 windows a bf16 value + rounding remainder.  Block (0,0) also writes the
 //                           work plan: the prefix sums of work units per sequence.
 //   2. decode_main_kernel   ONE wave of CTAs; every WARP owns an equal, contiguous slice of the
 //                           flattened list of work units (sequence, KV head, unit), a unit being a
 //                           64-token packed page or up to 8 tokens of the bf16 sink / recent windows.
 //                           A warp streams its units into shared memory with bulk async copies (mbarrier
-//                           ring), turns code words into fp16 A-fragments with one AND per register, and
-//                           runs both contractions (q'.k and p.v) on mma.sync.m16n8k16 with fp32
-//                           accumulation.  The affine part of Eq. 6 is factored out of the contractions:
+//                           ring).  Scores: the packed key codes become unsigned bytes with one AND per four
+//                           codes and go through mma.sync.m16n8k32 (u8 x s8, exact 32-bit sums); values:
+//                           code words become fp16 A-fragments with one AND per two codes and go through
+//                           mma.sync.m16n8k16 with fp32 accumulation.  The affine part of Eq. 6 is factored
+//                           out of the contractions:
 //                               q'.k_hat = Delta_k (q'.c_k) + x_min_k sum(q'),
 //                               o        = sum_s (p_s Delta_v,s) c_v,s + (sum_s p_s x_min_v,s) 1.
 //                           Window units use ldmatrix + bf16 mma on the staged rows and fold into the
 //                           same accumulators.  Softmax is online (running max / sum) per warp; a warp
 //                           writes one partial (max, sum, o) per (sequence, KV head) it touched.
-//  2b. decode_main_tc_kernel  opt-in alternative to 2 for G <= 4 (WUSHKV_DECODE_PATH=tc): the scores come from
-//                           tcgen05.mma on e4m3 code bytes held in tensor memory; a CTA's four warps share
-//                           128-token tiles.  Measured slower than 2; kept with its parity test.
 //   3. decode_combine_kernel merges the partials of each (sequence, query head) into O.
 //
-// No kernel waits on another CTA.  The only waits are on a warp's (2b: a CTA's) own copy and MMA
-// barriers, bounded by an iteration limit after which the kernel records WUSHKV_DEV_COPY_TIMEOUT and
-// drains; in 2b the four warps of a CTA also meet at CTA barriers, whose outcome carries that flag.
+// No kernel waits on another CTA.  The only waits are on a warp's own copy barriers, bounded by an
+// iteration limit after which the kernel records WUSHKV_DEV_COPY_TIMEOUT and drains.
+//
+// Data that an earlier kernel of the same step may still be writing while a later one is already
+// resident (programmatic dependent launch: sequence lengths, plan, query fragments, partials) is read
+// with ld.global.cg or plain loads after griddepcontrol.wait, never through the read-only path.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -42,7 +44,8 @@ namespace wushkv {
 constexpr unsigned FULL = 0xffffffffu;
 constexpr int PART_STRIDE = 132;          // floats per partial: [0]=max (log2 domain) [1]=sum [4..131]=o
 constexpr float LOG2E = 1.4426950408889634f;
-constexpr float LO_SCALE = 2048.f;        // a "remainder" column carries (x - rounded(x)) * 2^11
+constexpr float LO_SCALE = 2048.f;        // a "remainder" column of a window unit carries (x - rounded(x)) * 2^11
+constexpr float Q_MAX = 32512.f;          // largest magnitude of the 16-bit fixed-point query (127 * 256: both digits fit a signed byte)
 // Exponentials are taken against (running reference - LOG2_PV): every probability, and with it l, z and
 // o of a partial, carries the common factor 2^LOG2_PV, which cancels in the final ratio and keeps
 // fp16(p Delta_v) out of the subnormals.  The reference is only raised (and the state rescaled) when
@@ -68,16 +71,14 @@ struct DecodeParams {
     const int* seq_len;
     const unsigned short* Q;
     float* O;
-    uint4* qfrag;        // [batch*n_kv][2][128]: fp16 B fragments of the 8 k-steps (MODE 1: value set, remainder set)
+    uint4* qfrag;        // [batch*n_kv][256]: s8 B fragments of the 4 k-steps, 2 x 32 uint4 per digit set (MODE 0: one set
+                         // whose columns alternate high / low digit; MODE 1: high-digit set, low-digit set)
     uint4* qwfrag;       // [batch*n_kv][2][128]: bf16 B fragments for the windows (MODE 1: value set, remainder set)
     float* qscal;        // [batch][n_q][2]: score multiplier (log2 domain, > 0), x_min multiplier divided by it
     long long* plan;     // [batch+1]: exclusive prefix of work units per sequence (per KV head)
     float* part;         // [n_warps + batch*n_kv][G][PART_STRIDE]
     int n_warps;         // warps of the main kernel
     int q_early;         // 1: Q was final before the kernel ahead of the preparation kernel started
-    unsigned char* qb8;  // [batch*n_kv][2048]: e4m3 query operand of the tensor-memory kernel (null: not used)
-    float* qscal8;       // [batch][n_q][2]: the same two scalars as qscal for the e4m3 operand
-    int slice_shift;     // log2 of the warps that share one slice of the unit list (0: each warp its own, 2: a CTA)
     int stream_pages;    // 1: the packed pages of a step cannot stay in L2 anyway: copy them with an evict-first hint
 };
 
@@ -120,32 +121,6 @@ __device__ __forceinline__ SeqInfo seq_info(const CacheView& c, int S, int slot)
     return si;
 }
 
-// ---- constants of the tensor-memory main kernel (section 2b) that the query preparation shares
-constexpr int TC_STAGES = 4;
-constexpr int TC_TMEM_COLS = 64;          // 32 columns of A (128 e4m3 per token row) and two D buffers of 16
-constexpr int TC_D_COL = 32;
-constexpr int QB_LBO = 128, QB_SBO = 1024, QB_BYTES = 2048;       // 16 x 128 e4m3, K-major core matrices (8 rows x 16 B)
-constexpr unsigned QK8_IDESC = (1u << 4) | ((16u >> 3) << 17) | ((128u >> 4) << 24);    // D fp32, A and B e4m3 K-major, N 16, M 128
-
-// Position k (0..127) of channel ch in the e4m3 row the tensor-memory kernel lays out for a token, and
-// whether the mask that extracts it leaves the code shifted up by two bits (a factor 4).  Thread (g, t)
-// of a warp owns, exactly as in the register-operand kernel, the 16 bytes of key block codes of token
-// rows g and g+8 x channels {16s + 8w + 2t + hi}; it writes them with tcgen05.st.16x256b, where register
-// pair j of a row lands in tensor-memory columns 8j + 2t and 8j + 2t + 1, four e4m3 bytes per column.
-template <int BITS>
-__host__ __device__ inline int tc_k_of_channel(int ch, bool& times4) {
-    const int s = ch >> 4, r16 = ch & 15, w = r16 >> 3, tq = (r16 & 7) >> 1, hi = r16 & 1;
-    if (BITS == 2) {
-        const int m = s & 3, byte = 2 * hi + (s >> 2);          // mask m of word w; byte = half-word, low / high byte
-        times4 = (m & 1) != 0;
-        return 4 * (8 * (2 * w + (m >> 1)) + 2 * tq + (m & 1)) + byte;
-    } else {
-        const int hn = s & 1, byte = 2 * hi + ((s & 3) >> 1), jw = 2 * (s >> 2) + w;      // nibble hn of word jw
-        times4 = false;
-        return 4 * (8 * jw + 2 * tq + hn) + byte;
-    }
-}
-
 // ------------------------------------------------------------------------------------------------
 // 1. query preparation
 // ------------------------------------------------------------------------------------------------
@@ -154,9 +129,8 @@ constexpr int PREP_ROWS = D / (PREP_THREADS / 32);   // rows per warp
 template <int BITS, int MODE>
 __global__ void __launch_bounds__(PREP_THREADS) decode_prep_kernel(DecodeParams P) {
     __shared__ float q_s[8][D];
-    __shared__ float red_max[8][4];
-    __shared__ float red_sum[8][4];
     __shared__ float red_abs[8][4];
+    __shared__ int red_isum[8][4];
     __shared__ long long scan_s[4];
     const int h = blockIdx.x, b = blockIdx.y, G = P.c.G;
     const int i = threadIdx.x, lane = i & 31, warp = i >> 5;
@@ -214,7 +188,7 @@ __global__ void __launch_bounds__(PREP_THREADS) decode_prep_kernel(DecodeParams 
             if (i < 128 && bb < P.batch) {
                 const int slot = __ldg(P.slot + bb);
                 if (slot < 0 || slot >= P.c.n_slots) atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_SLOT);
-                u = seq_info(P.c, __ldg(P.seq_len + bb), slot).U;
+                u = seq_info(P.c, __ldcg(P.seq_len + bb), slot).U;
             }
             long long incl = u;
             for (int o = 1; o < 32; o <<= 1) {
@@ -235,102 +209,82 @@ __global__ void __launch_bounds__(PREP_THREADS) decode_prep_kernel(DecodeParams 
     float acc[8];
 #pragma unroll
     for (int g = 0; g < 8; ++g) acc[g] = g < G ? qp_s[g][i] : 0.f;
-    const int s = i >> 4;
-    const float pos_scale = exp2f(-static_cast<float>(field_shift<BITS>(s)));
     const float k2 = P.c.sm_scale * LOG2E;
+    // ---- 16-bit fixed point of q' per head: q'[ch] ~ lam * qi[ch], |qi| <= Q_MAX, qi = 256 hi + lo with both
+    // digits signed bytes.  The scores of the quantized positions use exactly this rounded query
+    // (code part and x_min part alike), so they are the scores of a slightly perturbed query, the same
+    // for every position.
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
         if (g < G) {
-            float mx = fabsf(acc[g]) * pos_scale, sm = acc[g], ab = fabsf(acc[g]);
-            for (int o = 16; o > 0; o >>= 1) {
-                mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
-                sm += __shfl_xor_sync(FULL, sm, o);
-                ab = fmaxf(ab, __shfl_xor_sync(FULL, ab, o));
-            }
-            if (lane == 0) { red_max[g][warp] = mx; red_sum[g][warp] = sm; red_abs[g][warp] = ab; }
+            float ab = fabsf(acc[g]);
+            for (int o = 16; o > 0; o >>= 1) ab = fmaxf(ab, __shfl_xor_sync(FULL, ab, o));
+            if (lane == 0) red_abs[g][warp] = ab;
         }
     }
     asm volatile("bar.sync 1, 128;" ::: "memory");       // the four remaining warps only
-    float beta[8];
+    int qi[8];
+    float lam[8];
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
-        beta[g] = 1.f;
+        qi[g] = 0; lam[g] = 1.f;
         if (g < G) {
-            const float mx = fmaxf(fmaxf(red_max[g][0], red_max[g][1]), fmaxf(red_max[g][2], red_max[g][3]));
-            int e = 0;
-            if (mx > 0.f && mx < 3e38f) frexpf(mx, &e);          // mx < 2^e
-            e = max(min(e, 100), -100);
-            beta[g] = exp2f(static_cast<float>(14 - e));         // scaled entries stay below 2^14
-            if (i == 0) {
-                const float sum = red_sum[g][0] + red_sum[g][1] + red_sum[g][2] + red_sum[g][3];
-                float* qs = P.qscal + (static_cast<long long>(b) * P.c.n_q + h * G + g) * 2;
-                qs[0] = k2 * 16777216.f / beta[g];            // score = qs[0] * (Delta_k * (codes . q'') + x_min_k * qs[1])
-                qs[1] = sum * beta[g] * (1.f / 16777216.f);
+            const float amax = fmaxf(fmaxf(red_abs[g][0], red_abs[g][1]), fmaxf(red_abs[g][2], red_abs[g][3]));
+            if (amax > 0.f && amax < 3e38f) {
+                lam[g] = amax * (1.f / Q_MAX);
+                qi[g] = max(-static_cast<int>(Q_MAX), min(static_cast<int>(Q_MAX), __float2int_rn(acc[g] * (Q_MAX / amax))));
             }
+            int sm = qi[g];
+            for (int o = 16; o > 0; o >>= 1) sm += __shfl_xor_sync(FULL, sm, o);
+            if (lane == 0) red_isum[g][warp] = sm;
         }
     }
-    // B fragments.  Element (k-step s, register r, lane 4n+t, half hf) is channel 16s + 8r + 2t + hf of
-    // mma column n.  MODE 0: column n holds head n>>1, its rounded value (n even) or the rounding
-    // remainder times 2^11 (n odd).  MODE 1: column n holds head n; the window set has a second copy
-    // with the remainders.
-    const int r16 = i & 15, r = r16 >> 3, t = (r16 & 7) >> 1, hf = r16 & 1;
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (i < G) {
+        const int sum = red_isum[i][0] + red_isum[i][1] + red_isum[i][2] + red_isum[i][3];
+        constexpr float FS = BITS == 2 ? 4.f : 16.f;      // the integer score carries this factor (see the main kernel)
+        float* qs = P.qscal + (static_cast<long long>(b) * P.c.n_q + h * G + i) * 2;
+        qs[0] = k2 * lam[i] * (1.f / FS);                 // score (log2 domain) = qs[0] * (Delta_k * sum_int + x_min_k * qs[1])
+        qs[1] = FS * static_cast<float>(sum);
+    }
+    // ---- B fragments of the integer mma (m16n8k32, B = 32 channels x 8 columns of signed bytes).  Channel i sits in
+    // k-step s = i >> 5 at k index 16 hh + 4 t + bb, i.e. register hh, lane 4 n + t, byte bb of column n.
+    // MODE 0: column n holds head n >> 1, high digit (n even) or low digit (n odd).  MODE 1: column n holds
+    // head n; the high digits form the first fragment set, the low digits the second.
+    const int s = i >> 5, hh = (i >> 4) & 1, bb = 2 * ((i >> 3) & 1) + (i & 1), t = (i >> 1) & 3;
     const long long bh = static_cast<long long>(b) * P.c.n_kv + h;
-    unsigned short* frag = reinterpret_cast<unsigned short*>(P.qfrag + bh * 256);
+    signed char* frag = reinterpret_cast<signed char*>(P.qfrag + bh * 256);
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+        const int head = (MODE == 0) ? (n >> 1) : n;
+        const int v = head < G ? qi[head] : 0;
+        const int hi = (v + 128) >> 8, lo = v - 256 * hi;          // hi in [-127, 127], lo in [-128, 127]
+        const int off = (((s >> 1) * 32 + 4 * n + t) * 16) + ((s & 1) * 2 + hh) * 4 + bb;
+        if (MODE == 0) {
+            frag[off] = static_cast<signed char>((n & 1) ? lo : hi);
+        } else {
+            frag[off] = static_cast<signed char>(hi);
+            frag[1024 + off] = static_cast<signed char>(lo);
+        }
+    }
+    // ---- bf16 B fragments for the windows (mma.m16n8k16).  Element (k-step s16, register r, lane 4n+t, half hf) is
+    // channel 16 s16 + 8 r + 2 t + hf of mma column n.  MODE 0: column n holds head n>>1, its rounded value (n even)
+    // or the rounding remainder (n odd).  MODE 1: column n holds head n; a second copy holds the remainders.
+    const int s16 = i >> 4, r16 = i & 15, r = r16 >> 3, tw = (r16 & 7) >> 1, hf = r16 & 1;
     unsigned short* wfrag = reinterpret_cast<unsigned short*>(P.qwfrag + bh * 256);
 #pragma unroll
     for (int n = 0; n < 8; ++n) {
         const int head = (MODE == 0) ? (n >> 1) : n;
-        float val = 0.f, rem = 0.f, wval = 0.f, wrem = 0.f;
+        float wval = 0.f, wrem = 0.f;
         if (head < G) {
-            const float x = acc[head] * pos_scale * beta[head];
-            const __half hi = __float2half_rn(x);
-            rem = (x - __half2float(hi)) * LO_SCALE;
-            val = (MODE == 0 && (n & 1)) ? rem : x;
             const float y = acc[head] * k2;
             const float yh = __bfloat162float(__float2bfloat16_rn(y));
             wrem = y - yh;
             wval = (MODE == 0 && (n & 1)) ? wrem : y;
         }
-        const int idx = ((((s >> 1) * 32 + 4 * n + t) * 4 + (s & 1) * 2 + r) << 1) + hf;
-        frag[idx] = __half_as_ushort(__float2half_rn(val));
-        if (MODE == 1) frag[1024 + idx] = __half_as_ushort(__float2half_rn(rem));
+        const int idx = ((((s16 >> 1) * 32 + 4 * n + tw) * 4 + (s16 & 1) * 2 + r) << 1) + hf;
         wfrag[idx] = __bfloat16_as_ushort(__float2bfloat16_rn(wval));
         if (MODE == 1) wfrag[1024 + idx] = __bfloat16_as_ushort(__float2bfloat16_rn(wrem));
-    }
-    // Operand of the tensor-memory kernel: each head's q' as the sum of four e4m3 terms (value, then three
-    // rounding remainders), scaled by a power of two so that the largest entry sits below 2^8; row n of the
-    // 16 x 128 operand is head n/2's term n%2 (n < 8) or term 2 + n%2 (n >= 8), its k order is the order
-    // in which a thread of that kernel lays out a token's codes, and the image is the K-major core-matrix
-    // layout the MMA reads from shared memory.
-    if (MODE == 0 && P.qb8 != nullptr) {
-        bool times4;
-        const int k = tc_k_of_channel<BITS>(i, times4);
-        unsigned char* img = P.qb8 + bh * QB_BYTES + (k >> 4) * QB_LBO + (k & 15);
-#pragma unroll
-        for (int head = 0; head < 4; ++head) {
-            float beta8 = 1.f, r = 0.f;
-            if (head < G) {
-                const float mx = fmaxf(fmaxf(red_abs[head][0], red_abs[head][1]), fmaxf(red_abs[head][2], red_abs[head][3]));
-                int e = 0;
-                if (mx > 0.f && mx < 3e38f) frexpf(mx, &e);          // mx < 2^e
-                e = max(min(e, 100), -100);
-                beta8 = exp2f(static_cast<float>(8 - e));
-                r = acc[head] * beta8 * (times4 ? 0.25f : 1.f);
-                if (i == 0) {
-                    const float sum = red_sum[head][0] + red_sum[head][1] + red_sum[head][2] + red_sum[head][3];
-                    float* qs = P.qscal8 + (static_cast<long long>(b) * P.c.n_q + h * G + head) * 2;
-                    qs[0] = k2 * 512.f / beta8;                   // an e4m3 code field is code * 2^-9
-                    qs[1] = sum * beta8 * (1.f / 512.f);
-                }
-            }
-#pragma unroll
-            for (int term = 0; term < 4; ++term) {
-                const __nv_fp8_e4m3 q8(r);                         // round to nearest, saturating
-                r -= static_cast<float>(q8);
-                const int n = (term < 2) ? 2 * head + term : 8 + 2 * head + (term - 2);
-                img[(n >> 3) * QB_SBO + (n & 7) * 16] = q8.__x;
-            }
-        }
     }
 }
 
@@ -400,6 +354,17 @@ __device__ __forceinline__ void mma_f16_zero(float (&d)[4], unsigned a0, unsigne
     asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
         : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
+}
+// integer mma: A = 16 x 32 unsigned bytes (codes), B = 32 x 8 signed bytes (query digits), exact 32-bit sums
+__device__ __forceinline__ void mma_u8s8(int (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0, unsigned b1) {
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_u8s8_zero(int (&d)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0, unsigned b1) {
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(0));
 }
 __device__ __forceinline__ void mma_bf16(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0, unsigned b1) {
     asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -544,7 +509,7 @@ __device__ __forceinline__ void window_unit(WarpState<MODE>& st, unsigned rec, i
     for (int pass = 0; pass < (MODE == 0 ? 1 : 2); ++pass) {
 #pragma unroll
         for (int s2 = 0; s2 < 4; ++s2) {
-            const uint4 bq = __ldg(wsrc + pass * 128 + s2 * 32 + lane);
+            const uint4 bq = __ldcg(wsrc + pass * 128 + s2 * 32 + lane);
             unsigned k0, k1, k2, k3;                      // (step 2s2: ch lo, ch hi), (step 2s2+1: ch lo, ch hi)
             ldmatrix_x4(rec + frag_off + s2 * 64, k0, k1, k2, k3);
             mma_bf16(acc, k0, k0, k1, k1, bq.x, bq.y);    // token rows 8..15 alias rows 0..7
@@ -615,7 +580,7 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 3 : (MODE == 0 ?
         for (int base = 0; base < P.batch; base += MAIN_WARPS * 32) {
             const int bb = base + threadIdx.x;
             long long incl = 0;
-            if (bb < P.batch) incl = seq_info(c, __ldg(P.seq_len + bb), __ldg(P.slot + bb)).U;
+            if (bb < P.batch) incl = seq_info(c, __ldcg(P.seq_len + bb), __ldg(P.slot + bb)).U;
             for (int o = 1; o < 32; o <<= 1) {
                 const long long v = __shfl_up_sync(FULL, incl, o);
                 if (lane >= o) incl += v;
@@ -671,7 +636,8 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 3 : (MODE == 0 ?
     const long long page_row_bytes = static_cast<long long>(c.n_kv) * REC;
     const unsigned long long stream_policy = l2_evict_first_policy();
 
-    unsigned qf[8][2];
+    unsigned qf[4][2];                  // integer B fragments of the four k-steps (MODE 1: the high digits)
+    unsigned qfl[MODE == 1 ? 4 : 1][2]; // MODE 1: the low digits
     float fmul[NH], gadd[NH];
     WarpState<MODE> st;
     int stage = 0;                      // ring position of the next unit to consume (and to refill)
@@ -683,7 +649,7 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 3 : (MODE == 0 ?
         // ================= round set-up: list the next segments of the slice =====================
         int n_seg = 0, round_units = 0;
         while (n_seg < MAX_SEGMENTS && L < L1) {
-            const SeqInfo si = seq_info(c, __ldg(P.seq_len + sb), __ldg(P.slot + sb));
+            const SeqInfo si = seq_info(c, __ldcg(P.seq_len + sb), __ldg(P.slot + sb));
             if (si.U > 0) {
                 const int u1 = static_cast<int>(min(static_cast<long long>(si.U), su + (L1 - L)));
                 if (lane == 0) {
@@ -765,16 +731,20 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 3 : (MODE == 0 ?
             {   // query fragments and per-head scalars of this (sequence, KV head)
                 const uint4* src = P.qfrag + bh * 256;
 #pragma unroll
-                for (int s2 = 0; s2 < 4; ++s2) {
-                    const uint4 v = __ldg(src + s2 * 32 + lane);
+                for (int s2 = 0; s2 < 2; ++s2) {
+                    const uint4 v = __ldcg(src + s2 * 32 + lane);
                     qf[2 * s2][0] = v.x; qf[2 * s2][1] = v.y; qf[2 * s2 + 1][0] = v.z; qf[2 * s2 + 1][1] = v.w;
+                    if (MODE == 1) {
+                        const uint4 w = __ldcg(src + 64 + s2 * 32 + lane);
+                        qfl[2 * s2][0] = w.x; qfl[2 * s2][1] = w.y; qfl[2 * s2 + 1][0] = w.z; qfl[2 * s2 + 1][1] = w.w;
+                    }
                 }
 #pragma unroll
                 for (int k = 0; k < NH; ++k) {
                     const int head = MODE == 0 ? t : 2 * t + k;
                     fmul[k] = 1.f; gadd[k] = 0.f;             // unused head slots stay finite
                     if (head < G) {
-                        const float2 v = __ldg(reinterpret_cast<const float2*>(P.qscal + (static_cast<long long>(sg.b) * c.n_q + sg.h * G + head) * 2));
+                        const float2 v = __ldcg(reinterpret_cast<const float2*>(P.qscal + (static_cast<long long>(sg.b) * c.n_q + sg.h * G + head) * 2));
                         fmul[k] = v.x; gadd[k] = v.y;
                     }
                 }
@@ -798,74 +768,59 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 3 : (MODE == 0 ?
                     unsigned vmeta[4][2];         // fp16x2 (Delta_v, x_min_v) of rows g, g+8
 #pragma unroll
                     for (int bi = 0; bi < 4; ++bi) {
-                        float acc[4];                 // one chain per block; the four blocks of a page are independent
+                        // The four k-steps of a block take one field of every code byte each.  Fields at an even
+                        // position come out of the mask as the code itself, fields at an odd position as the code
+                        // times FS (4 at 2 bits, 16 at 4 bits): the two kinds are summed separately (X, Y) and
+                        // joined as FS * X + Y, which is FS times the exact integer dot product.
+                        constexpr int FS = BITS == 2 ? 4 : 16;
+                        unsigned a[4][4];             // [k-step][A register]
                         if (BITS == 2) {
-                            const uint4 kw = lds128(rec + bi * CB + 16 * lane);
-                            const unsigned sx = pre_shift<2>(kw.x), sy = pre_shift<2>(kw.y), sz = pre_shift<2>(kw.z), sw = pre_shift<2>(kw.w);
-                            mma_f16_zero(acc, field<2>(kw.x, sx, 0), field<2>(kw.z, sz, 0), field<2>(kw.y, sy, 0), field<2>(kw.w, sw, 0), qf[0][0], qf[0][1]);
-#pragma unroll
-                            for (int ks = 1; ks < 8; ++ks)
-                                mma_f16(acc, field<2>(kw.x, sx, ks), field<2>(kw.z, sz, ks), field<2>(kw.y, sy, ks), field<2>(kw.w, sw, ks),
-                                        qf[ks][0], qf[ks][1]);
+                            const uint4 kw = lds128(rec + bi * CB + 16 * lane);      // (row g, ch half 0), (g+8, 0), (g, 1), (g+8, 1)
+                            const unsigned sx = kw.x >> 4, sy = kw.y >> 4, sz = kw.z >> 4, sw = kw.w >> 4;
+                            a[0][0] = kw.x & 0x03030303u; a[0][1] = kw.y & 0x03030303u; a[0][2] = kw.z & 0x03030303u; a[0][3] = kw.w & 0x03030303u;
+                            a[1][0] = kw.x & 0x0C0C0C0Cu; a[1][1] = kw.y & 0x0C0C0C0Cu; a[1][2] = kw.z & 0x0C0C0C0Cu; a[1][3] = kw.w & 0x0C0C0C0Cu;
+                            a[2][0] = sx & 0x03030303u;   a[2][1] = sy & 0x03030303u;   a[2][2] = sz & 0x03030303u;   a[2][3] = sw & 0x03030303u;
+                            a[3][0] = sx & 0x0C0C0C0Cu;   a[3][1] = sy & 0x0C0C0C0Cu;   a[3][2] = sz & 0x0C0C0C0Cu;   a[3][3] = sw & 0x0C0C0C0Cu;
                         } else {
-                            const uint4 ka = lds128(rec + bi * CB + 16 * lane);          // row g:   W0..W3
-                            const uint4 kb = lds128(rec + bi * CB + 512 + 16 * lane);    // row g+8: W0..W3
-                            const unsigned a0s = pre_shift<4>(ka.x), a1s = pre_shift<4>(ka.y), a2s = pre_shift<4>(ka.z), a3s = pre_shift<4>(ka.w);
-                            const unsigned b0s = pre_shift<4>(kb.x), b1s = pre_shift<4>(kb.y), b2s = pre_shift<4>(kb.z), b3s = pre_shift<4>(kb.w);
-                            mma_f16_zero(acc, field<4>(ka.x, a0s, 0), field<4>(kb.x, b0s, 0), field<4>(ka.y, a1s, 0), field<4>(kb.y, b1s, 0), qf[0][0], qf[0][1]);
-#pragma unroll
-                            for (int ks = 1; ks < 4; ++ks)
-                                mma_f16(acc, field<4>(ka.x, a0s, ks), field<4>(kb.x, b0s, ks), field<4>(ka.y, a1s, ks), field<4>(kb.y, b1s, ks),
-                                        qf[ks][0], qf[ks][1]);
-#pragma unroll
-                            for (int ks = 0; ks < 4; ++ks)
-                                mma_f16(acc, field<4>(ka.z, a2s, ks), field<4>(kb.z, b2s, ks), field<4>(ka.w, a3s, ks), field<4>(kb.w, b3s, ks),
-                                        qf[4 + ks][0], qf[4 + ks][1]);
+                            const uint4 ka = lds128(rec + bi * CB + 16 * lane);          // k-steps 0 (low nibbles), 1 (high nibbles)
+                            const uint4 kb = lds128(rec + bi * CB + 512 + 16 * lane);    // k-steps 2, 3
+                            a[0][0] = ka.x & 0x0F0F0F0Fu; a[0][1] = ka.y & 0x0F0F0F0Fu; a[0][2] = ka.z & 0x0F0F0F0Fu; a[0][3] = ka.w & 0x0F0F0F0Fu;
+                            a[1][0] = ka.x & 0xF0F0F0F0u; a[1][1] = ka.y & 0xF0F0F0F0u; a[1][2] = ka.z & 0xF0F0F0F0u; a[1][3] = ka.w & 0xF0F0F0F0u;
+                            a[2][0] = kb.x & 0x0F0F0F0Fu; a[2][1] = kb.y & 0x0F0F0F0Fu; a[2][2] = kb.z & 0x0F0F0F0Fu; a[2][3] = kb.w & 0x0F0F0F0Fu;
+                            a[3][0] = kb.x & 0xF0F0F0F0u; a[3][1] = kb.y & 0xF0F0F0F0u; a[3][2] = kb.z & 0xF0F0F0F0u; a[3][3] = kb.w & 0xF0F0F0F0u;
                         }
-                        if (MODE == 1) {
-                            // two heads per column pair leave no room for a remainder column: a second pass over
-                            // the same A fragments with the remainder fragments (re-read per block: L1 hits)
-                            float accr[4] = {0.f, 0.f, 0.f, 0.f}, accr2[4] = {0.f, 0.f, 0.f, 0.f};
-                            const uint4* rsrc = P.qfrag + bh * 256 + 128 + lane;
-                            if (BITS == 2) {
-                                const uint4 kw = lds128(rec + bi * CB + 16 * lane);
-                                const unsigned sx = pre_shift<2>(kw.x), sy = pre_shift<2>(kw.y), sz = pre_shift<2>(kw.z), sw = pre_shift<2>(kw.w);
+                        int dot[4];                   // MODE 0: (row g, row g+8) x (high, low digit) joined below; MODE 1: rows x heads 2t, 2t+1
+                        {
+                            int X[4], Y[4];
+                            mma_u8s8_zero(X, a[0][0], a[0][1], a[0][2], a[0][3], qf[0][0], qf[0][1]);
+                            mma_u8s8_zero(Y, a[1][0], a[1][1], a[1][2], a[1][3], qf[1][0], qf[1][1]);
+                            mma_u8s8(X, a[2][0], a[2][1], a[2][2], a[2][3], qf[2][0], qf[2][1]);
+                            mma_u8s8(Y, a[3][0], a[3][1], a[3][2], a[3][3], qf[3][0], qf[3][1]);
 #pragma unroll
-                                for (int s2 = 0; s2 < 4; ++s2) {
-                                    const uint4 rq = __ldg(rsrc + s2 * 32);
-                                    mma_f16(accr, field<2>(kw.x, sx, 2 * s2), field<2>(kw.z, sz, 2 * s2), field<2>(kw.y, sy, 2 * s2), field<2>(kw.w, sw, 2 * s2), rq.x, rq.y);
-                                    mma_f16(accr2, field<2>(kw.x, sx, 2 * s2 + 1), field<2>(kw.z, sz, 2 * s2 + 1), field<2>(kw.y, sy, 2 * s2 + 1), field<2>(kw.w, sw, 2 * s2 + 1), rq.z, rq.w);
-                                }
-                            } else {
-                                const uint4 ka = lds128(rec + bi * CB + 16 * lane);
-                                const uint4 kb = lds128(rec + bi * CB + 512 + 16 * lane);
-                                const unsigned a0s = pre_shift<4>(ka.x), a1s = pre_shift<4>(ka.y), a2s = pre_shift<4>(ka.z), a3s = pre_shift<4>(ka.w);
-                                const unsigned b0s = pre_shift<4>(kb.x), b1s = pre_shift<4>(kb.y), b2s = pre_shift<4>(kb.z), b3s = pre_shift<4>(kb.w);
+                            for (int e = 0; e < 4; ++e) dot[e] = X[e] * FS + Y[e];
+                        }
+                        if (MODE == 1) {              // second fragment set: the low digits of the eight heads
+                            int X[4], Y[4];
+                            mma_u8s8_zero(X, a[0][0], a[0][1], a[0][2], a[0][3], qfl[0][0], qfl[0][1]);
+                            mma_u8s8_zero(Y, a[1][0], a[1][1], a[1][2], a[1][3], qfl[1][0], qfl[1][1]);
+                            mma_u8s8(X, a[2][0], a[2][1], a[2][2], a[2][3], qfl[2][0], qfl[2][1]);
+                            mma_u8s8(Y, a[3][0], a[3][1], a[3][2], a[3][3], qfl[3][0], qfl[3][1]);
 #pragma unroll
-                                for (int s2 = 0; s2 < 2; ++s2) {
-                                    const uint4 rq = __ldg(rsrc + s2 * 32), rq2 = __ldg(rsrc + (s2 + 2) * 32);
-                                    mma_f16(accr, field<4>(ka.x, a0s, 2 * s2), field<4>(kb.x, b0s, 2 * s2), field<4>(ka.y, a1s, 2 * s2), field<4>(kb.y, b1s, 2 * s2), rq.x, rq.y);
-                                    mma_f16(accr, field<4>(ka.x, a0s, 2 * s2 + 1), field<4>(kb.x, b0s, 2 * s2 + 1), field<4>(ka.y, a1s, 2 * s2 + 1), field<4>(kb.y, b1s, 2 * s2 + 1), rq.z, rq.w);
-                                    mma_f16(accr2, field<4>(ka.z, a2s, 2 * s2), field<4>(kb.z, b2s, 2 * s2), field<4>(ka.w, a3s, 2 * s2), field<4>(kb.w, b3s, 2 * s2), rq2.x, rq2.y);
-                                    mma_f16(accr2, field<4>(ka.z, a2s, 2 * s2 + 1), field<4>(kb.z, b2s, 2 * s2 + 1), field<4>(ka.w, a3s, 2 * s2 + 1), field<4>(kb.w, b3s, 2 * s2 + 1), rq2.z, rq2.w);
-                                }
-                            }
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) acc[e] = fmaf(accr[e] + accr2[e], 1.f / LO_SCALE, acc[e]);
+                            for (int e = 0; e < 4; ++e) dot[e] = dot[e] * 256 + (X[e] * FS + Y[e]);
                         }
                         const uint4 mt = lds128(rec + meta_offset(BITS) + 128 * bi + 16 * g);   // rows g (x,y) and g+8 (z,w)
                         const float2 km_a = h2f2(mt.x), km_b = h2f2(mt.z);
                         const float kd0 = km_a.x, km0 = km_a.y, kd1 = km_b.x, km1 = km_b.y;
                         vmeta[bi][0] = mt.y; vmeta[bi][1] = mt.w;
                         if (MODE == 0) {
-                            const float d0 = fmaf(acc[1], 1.f / LO_SCALE, acc[0]), d1 = fmaf(acc[3], 1.f / LO_SCALE, acc[2]);
+                            const float d0 = static_cast<float>(dot[0] * 256 + dot[1]), d1 = static_cast<float>(dot[2] * 256 + dot[3]);
                             sc[bi][0] = fmaf(km0, gadd[0], d0 * kd0);
                             sc[bi][NH] = fmaf(km1, gadd[0], d1 * kd1);
                         } else {
-                            sc[bi][0] = fmaf(km0, gadd[0], acc[0] * kd0);
-                            sc[bi][NH - 1] = fmaf(km0, gadd[NH - 1], acc[1] * kd0);
-                            sc[bi][NH] = fmaf(km1, gadd[0], acc[2] * kd1);
-                            sc[bi][2 * NH - 1] = fmaf(km1, gadd[NH - 1], acc[3] * kd1);
+                            sc[bi][0] = fmaf(km0, gadd[0], static_cast<float>(dot[0]) * kd0);
+                            sc[bi][NH - 1] = fmaf(km0, gadd[NH - 1], static_cast<float>(dot[1]) * kd0);
+                            sc[bi][NH] = fmaf(km1, gadd[0], static_cast<float>(dot[2]) * kd1);
+                            sc[bi][2 * NH - 1] = fmaf(km1, gadd[NH - 1], static_cast<float>(dot[3]) * kd1);
                         }
                     }
                     if (!full_page) {             // first / last page of the quantized range: mask the tokens outside it
@@ -948,437 +903,6 @@ __global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 3 : (MODE == 0 ?
         // give copies that may still be in flight a bounded time to land before the CTA's memory is released
         for (int k = 0; k < 1000; ++k) __nanosleep(1000);
     }
-}
-
-// ------------------------------------------------------------------------------------------------
-// 2b. main kernel with the scores on the tensor core (G <= 4)
-// ------------------------------------------------------------------------------------------------
-// Alternative, selected with WUSHKV_DECODE_PATH=tc; slower than the kernel above on every measured
-// configuration (config 1: 135 us against 82 us), see the note where the path is chosen.
-// The register-operand kernel above spends one mask per two key codes plus the MMA issue itself on the
-// scores.  Here a CTA of four warps takes a contiguous slice of the unit list and walks it two units
-// (128 tokens) at a time; for packed pages every thread owns one token row: it masks that row's codes
-// in place into e4m3 bytes (four codes per mask: a 2-bit field inside bits 0..3 of a byte is the e4m3
-// value field * 2^-9, subnormals and the first binade being linear in the bit pattern), writes the 128
-// bytes to tensor memory (lane = token row) and one thread issues tcgen05.mma kind::f8f6f4 with that
-// A operand against the query as four e4m3 terms per head (16 columns, shared memory).  The 128 x 16
-// fp32 scores come back as 16 x 256 bit fragments, which is exactly the mma.sync accumulator layout the
-// softmax / value code of the kernel above works in; values stay on mma.sync with per-warp states.
-// The 16-token key block at shared address blk as e4m3 bytes in tensor memory: this lane's rows g and
-// g+8, eight registers (columns 8j + 2t, 8j + 2t + 1) each, written to lanes taddr .. taddr + 15.
-template <int BITS>
-__device__ __forceinline__ void tc_store_key_block(unsigned blk, int lane, unsigned taddr) {
-    unsigned a[16];                   // a[4j], a[4j+1]: row g; a[4j+2], a[4j+3]: row g+8
-    if (BITS == 2) {
-        const uint4 kw = lds128(blk + 16 * lane);                   // row g: words x, y; row g+8: words z, w
-        const unsigned sx = kw.x >> 4, sy = kw.y >> 4, sz = kw.z >> 4, sw = kw.w >> 4;
-        a[0] = kw.x & 0x03030303u;  a[1] = kw.x & 0x0C0C0C0Cu;  a[2] = kw.z & 0x03030303u;  a[3] = kw.z & 0x0C0C0C0Cu;
-        a[4] = sx & 0x03030303u;    a[5] = sx & 0x0C0C0C0Cu;    a[6] = sz & 0x03030303u;    a[7] = sz & 0x0C0C0C0Cu;
-        a[8] = kw.y & 0x03030303u;  a[9] = kw.y & 0x0C0C0C0Cu;  a[10] = kw.w & 0x03030303u; a[11] = kw.w & 0x0C0C0C0Cu;
-        a[12] = sy & 0x03030303u;   a[13] = sy & 0x0C0C0C0Cu;   a[14] = sw & 0x03030303u;   a[15] = sw & 0x0C0C0C0Cu;
-    } else {
-        const uint4 ka = lds128(blk + 16 * lane);                   // row g:   W0..W3
-        const uint4 kb = lds128(blk + 512 + 16 * lane);             // row g+8: W0..W3
-        a[0] = ka.x & 0x0F0F0F0Fu;  a[1] = (ka.x >> 4) & 0x0F0F0F0Fu;  a[2] = kb.x & 0x0F0F0F0Fu;  a[3] = (kb.x >> 4) & 0x0F0F0F0Fu;
-        a[4] = ka.y & 0x0F0F0F0Fu;  a[5] = (ka.y >> 4) & 0x0F0F0F0Fu;  a[6] = kb.y & 0x0F0F0F0Fu;  a[7] = (kb.y >> 4) & 0x0F0F0F0Fu;
-        a[8] = ka.z & 0x0F0F0F0Fu;  a[9] = (ka.z >> 4) & 0x0F0F0F0Fu;  a[10] = kb.z & 0x0F0F0F0Fu; a[11] = (kb.z >> 4) & 0x0F0F0F0Fu;
-        a[12] = ka.w & 0x0F0F0F0Fu; a[13] = (ka.w >> 4) & 0x0F0F0F0Fu; a[14] = kb.w & 0x0F0F0F0Fu; a[15] = (kb.w >> 4) & 0x0F0F0F0Fu;
-    }
-    asm volatile(
-        "tcgen05.st.sync.aligned.16x256b.x4.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
-        :: "r"(taddr), "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(a[4]), "r"(a[5]), "r"(a[6]), "r"(a[7]),
-           "r"(a[8]), "r"(a[9]), "r"(a[10]), "r"(a[11]), "r"(a[12]), "r"(a[13]), "r"(a[14]), "r"(a[15]) : "memory");
-}
-
-__device__ __forceinline__ unsigned long long qb_smem_desc(unsigned smem_addr) {
-    unsigned long long d = 0;
-    d |= static_cast<unsigned long long>((smem_addr >> 4) & 0x3FFFu);            // start address
-    d |= static_cast<unsigned long long>((QB_LBO >> 4) & 0x3FFFu) << 16;         // leading (k chunk) byte offset
-    d |= static_cast<unsigned long long>((QB_SBO >> 4) & 0x3FFFu) << 32;         // stride (row group) byte offset
-    d |= 1ull << 46;                                                             // descriptor version of sm_100
-    return d;                                                                    // no swizzle
-}
-
-template <int BITS>
-__global__ void __launch_bounds__(MAIN_WARPS * 32, (BITS == 4 ? 3 : 4)) decode_main_tc_kernel(DecodeParams P) {
-    constexpr int REC = record_bytes(BITS);
-    constexpr int CB = code_block_bytes(BITS);
-    constexpr int TILE = 2 * REC;                       // a stage holds two units
-    static_assert(2 * WIN_TOKENS * WIN_ROW <= REC, "a window unit must fit in half a stage");
-    extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char* qb = smem + TC_STAGES * TILE;                                           // two operand buffers
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(qb + 2 * QB_BYTES);   // full[TC_STAGES], mma
-    unsigned* misc = reinterpret_cast<unsigned*>(bars + TC_STAGES + 1);                    // [0] tensor-memory base, [1 + s] missing halves of stage s, [7] abort
-    Segment* segs = reinterpret_cast<Segment*>(misc + 8);
-    const CacheView& c = P.c;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int g = lane >> 2, t = lane & 3;
-    const int G = c.G;
-    const int half = warp >> 1;                          // which unit of a stage this warp works on
-    const int blk0 = 2 * (warp & 1);                     // its two 16-token blocks of that unit: blk0, blk0 + 1
-
-    // ---- work plan (as in the kernel above)
-    __shared__ long long scan_s[MAIN_WARPS];
-    long long* plan_s = reinterpret_cast<long long*>(smem);
-    const bool local_plan = (static_cast<size_t>(P.batch) + 1) * sizeof(long long) <= static_cast<size_t>(TC_STAGES) * TILE;
-    if (local_plan) {
-        long long carry = 0;
-        for (int base = 0; base < P.batch; base += MAIN_WARPS * 32) {
-            const int bb = base + tid;
-            long long incl = 0;
-            if (bb < P.batch) incl = seq_info(c, __ldg(P.seq_len + bb), __ldg(P.slot + bb)).U;
-            for (int o = 1; o < 32; o <<= 1) {
-                const long long v = __shfl_up_sync(FULL, incl, o);
-                if (lane >= o) incl += v;
-            }
-            if (lane == 31) scan_s[warp] = incl;
-            __syncthreads();
-            long long before = 0, all = 0;
-            for (int w = 0; w < MAIN_WARPS; ++w) { if (w < warp) before += scan_s[w]; all += scan_s[w]; }
-            if (bb < P.batch) plan_s[bb + 1] = carry + before + incl;
-            carry += all;
-            __syncthreads();
-        }
-        if (tid == 0) plan_s[0] = 0;
-        __syncthreads();
-    } else {
-        pdl_wait();
-    }
-    const long long* plan = local_plan ? plan_s : P.plan;
-
-    // ---- this CTA's slice of the flattened unit list
-    const long long total = plan[P.batch] * c.n_kv;
-    const long long n_slices = gridDim.x;
-    long long L = total > 0 ? blockIdx.x * total / n_slices : 0;
-    const long long L1 = total > 0 ? (blockIdx.x + 1) * total / n_slices : 0;
-    int sb = 0, sh = 0, su = 0;
-    if (L < L1) {
-        int lo = 0, hi = P.batch;           // largest b with n_kv * plan[b] <= L
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (plan[mid] * c.n_kv <= L) lo = mid; else hi = mid;
-        }
-        sb = lo;
-        const long long U = max(plan[lo + 1] - plan[lo], 1LL);
-        const long long rem = L - plan[lo] * c.n_kv;
-        sh = static_cast<int>(rem / U);
-        su = static_cast<int>(rem % U);
-    }
-    __syncthreads();                        // the staging area stops being plan scratch here
-    pdl_launch_dependents();
-    if (L >= L1) return;                    // the whole CTA: nothing allocated yet
-
-    // ---- tensor memory, barriers
-    if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(misc)), "r"(static_cast<unsigned>(TC_TMEM_COLS)) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    const unsigned bar0 = smem_u32(bars), mma_bar = bar0 + 8 * TC_STAGES;
-    if (tid == 0) {
-#pragma unroll
-        for (int s = 0; s <= TC_STAGES; ++s) mbar_init(bar0 + 8 * s, 1);
-#pragma unroll
-        for (int s = 1; s < 8; ++s) misc[s] = 0u;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const unsigned tmem = misc[0];
-    const unsigned my_tmem = tmem + (static_cast<unsigned>(warp * 32) << 16);     // this warp's 32 lanes: two 16-token blocks
-    const unsigned stage0 = smem_u32(smem);
-    const unsigned qb_addr = smem_u32(qb);
-    const long long page_row_bytes = static_cast<long long>(c.n_kv) * REC;
-    const unsigned my_rec_off = half * REC;
-
-    WarpState<0> st;
-    int stage = 0;                      // ring position of the tile being finished
-    unsigned phase_bits = 0;            // parity of each stage's next completion
-    unsigned mma_phase = 0;
-    bool aborted = false;
-
-    while (L < L1 && !aborted) {
-        __syncthreads();                // every warp is done with the previous round's segments and stages
-        // ================= round set-up: list the next segments of the slice =====================
-        int n_seg = 0, round_tiles = 0;
-        while (n_seg < MAX_SEGMENTS && L < L1) {
-            const SeqInfo si = seq_info(c, __ldg(P.seq_len + sb), __ldg(P.slot + sb));
-            if (si.U > 0) {
-                const int u1 = static_cast<int>(min(static_cast<long long>(si.U), su + (L1 - L)));
-                if (tid == 0) {
-                    Segment sg;
-                    sg.b = sb; sg.h = sh; sg.slot = si.slot; sg.u0 = su; sg.u1 = u1; sg.qp = si.qp; sg.first_page = si.first_page;
-                    sg.q_lo = si.q_lo; sg.q_hi = si.q_hi; sg.n_win = si.n_win; sg.n_sink = si.n_sink; sg.recent_lo = si.recent_lo;
-                    segs[n_seg] = sg;
-                }
-                ++n_seg;
-                round_tiles += (u1 - su + 1) >> 1;
-                L += u1 - su;
-                su = u1;
-            }
-            if (si.U == 0 || su >= si.U) {              // next head, or next sequence
-                su = 0;
-                if (si.U == 0 || ++sh >= c.n_kv) { sh = 0; ++sb; }
-                if (sb >= P.batch) break;
-            }
-        }
-        __syncthreads();
-
-        // ================= producer: stages the tiles of this round, in order =====================
-        // Every warp tracks the cursor; the warp whose turn it is issues the copies (the turn rotates so
-        // that no warp is always the last one at the CTA barrier).
-        int p_seg = -1, p_u = 0, p_u1 = 0, p_qp = 0, p_sqp = 0, p_nwin = 0, p_head_off = 0, issued = 0;
-        const int* p_ptab = nullptr;
-        auto issue_tile = [&](const int s, const bool mine) {     // two units of one segment into ring slot s
-            if (p_u >= p_u1) {                          // next segment
-                ++p_seg;
-                const Segment& sg = segs[p_seg];
-                p_u = sg.u0; p_u1 = sg.u1; p_qp = p_sqp = sg.qp; p_nwin = sg.n_win; p_head_off = sg.h * REC;
-                p_ptab = c.page_table + static_cast<long long>(sg.slot) * c.max_pages + sg.first_page;
-                if (sg.first_page + sg.qp > c.max_pages) {      // the page table cannot hold this length
-                    if (mine && lane == 0) atomicOr(c.dev_status, WUSHKV_DEV_PAGE_TABLE_FULL);
-                    p_qp = min(p_qp, max(c.max_pages - sg.first_page, 0));
-                }
-            }
-            if (mine) {
-                const unsigned bar = bar0 + 8 * s, dst0 = stage0 + s * TILE;
-                int page[2] = {-1, -1}, n_valid[2] = {0, 0};
-                unsigned bytes = 0, missing = 0;
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    const int uu = p_u + hf;
-                    if (uu >= p_u1) continue;
-                    if (uu < p_sqp) {
-                        const int pg = (uu < p_qp) ? __ldg(p_ptab + uu) : -1;
-                        if (static_cast<unsigned>(pg) >= static_cast<unsigned long long>(c.n_pages)) {
-                            if (lane == 0 && uu < p_qp) atomicOr(c.dev_status, WUSHKV_DEV_BAD_PAGE_ID);
-                            missing |= 1u << hf;
-                        } else {
-                            page[hf] = pg;
-                            bytes += REC;
-                        }
-                    } else {
-                        n_valid[hf] = min(WIN_TOKENS, p_nwin - (uu - p_sqp) * WIN_TOKENS);
-                        bytes += n_valid[hf] * 2 * D * 2;
-                    }
-                }
-                if (lane == 0) {
-                    misc[1 + s] = missing;
-                    if (bytes) mbar_expect_tx(bar, bytes); else mbar_arrive(bar);
-                }
-                __syncwarp();
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    if (page[hf] >= 0) {
-                        if (lane == 0) bulk_copy_g2s(dst0 + hf * REC, c.pages + page[hf] * page_row_bytes + p_head_off, REC, bar);
-                    } else if (n_valid[hf] > 0) {       // up to 8 window tokens: one 256-byte row copy per lane
-                        const Segment& sg = segs[p_seg];
-                        const int w0 = (p_u + hf - p_sqp) * WIN_TOKENS;
-                        const int r = lane & 7, which = lane >> 3;      // lanes 0-7: key rows, 8-15: value rows
-                        if (lane < 16 && r < n_valid[hf]) {
-                            const int w = w0 + r;
-                            const long long plane = (static_cast<long long>(sg.slot) * c.n_kv + sg.h) * 2 + which;
-                            const unsigned short* src;
-                            if (w < sg.n_sink) src = c.sink_kv + (plane * c.s_sink + w) * D;
-                            else src = c.ring_kv + (plane * c.ring_cap + (sg.recent_lo + (w - sg.n_sink)) % c.ring_cap) * D;
-                            bulk_copy_g2s(dst0 + hf * REC + which * WIN_V_OFF + r * WIN_ROW, src, D * 2, bar);
-                        }
-                    }
-                }
-            }
-            p_u += 2;
-            ++issued;
-        };
-        for (int k = 0; k < TC_STAGES && k < round_tiles; ++k) issue_tile((stage + k) % TC_STAGES, warp == (k & 3));
-
-        // ================= consumer ==============================================================
-        // Software pipeline over the round's tiles: while the tensor core scores tile i+1, the warps run
-        // softmax and values of tile i.  Per iteration: wait for the scores of tile i and pull them into
-        // registers; write the key rows of tile i+1 (the A columns are free: the MMAs of tile i are done);
-        // CTA barrier; one thread issues the MMAs of tile i+1 into the other D buffer and one warp refills
-        // the stage of tile i-1; then everybody finishes tile i.
-        pdl_wait();                                     // query operands come from the preparation kernel
-        // tile being started (n_*) and tile being finished (f_*): segment fields live in registers
-        int n_cs = -1, n_u = 0, n_u1 = 0, n_qp = 0, n_stage = stage;
-        int f_cs = -1, f_u = 0, f_u1 = 0, f_qp = 0, f_qlo = 0, f_qhi = 0, f_page0 = 0, f_nwin = 0;
-        long long f_bh = 0;
-        float fmul = 1.f, gadd = 0.f;
-        auto next_start_segment = [&]() {
-            ++n_cs;
-            const Segment& sg = segs[n_cs];
-            n_u = sg.u0; n_u1 = sg.u1; n_qp = sg.qp;
-            // the head group's e4m3 query operand into buffer n_cs & 1 (its last reader, two segments back, is done)
-            const long long bh = static_cast<long long>(sg.b) * c.n_kv + sg.h;
-            reinterpret_cast<uint4*>(qb + (n_cs & 1) * QB_BYTES)[tid] = __ldg(reinterpret_cast<const uint4*>(P.qb8) + bh * (QB_BYTES / 16) + tid);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        };
-        auto next_finish_segment = [&]() {
-            ++f_cs;
-            const Segment& sg = segs[f_cs];
-            f_u = sg.u0; f_u1 = sg.u1; f_qp = sg.qp; f_qlo = sg.q_lo; f_qhi = sg.q_hi; f_page0 = sg.first_page; f_nwin = sg.n_win;
-            f_bh = static_cast<long long>(sg.b) * c.n_kv + sg.h;
-            fmul = 1.f; gadd = 0.f;                     // unused head slots stay finite
-            if (t < G) {
-                const float2 v = __ldg(reinterpret_cast<const float2*>(P.qscal8 + (static_cast<long long>(sg.b) * c.n_q + sg.h * G + t) * 2));
-                fmul = v.x; gadd = v.y;
-            }
-            st.reset();
-        };
-        // writes my key rows of the tile at n_u in ring slot n_stage; false if its data did not land
-        auto start_tile = [&]() -> bool {
-            const bool landed = __all_sync(FULL, mbar_wait_bounded(bar0 + 8 * n_stage, (phase_bits >> n_stage) & 1u));
-            phase_bits ^= 1u << n_stage;
-            const int my_u = n_u + half;
-            if (my_u < n_u1 && my_u < n_qp && !((misc[1 + n_stage] >> half) & 1u)) {
-                const unsigned rec = stage0 + n_stage * TILE + my_rec_off;
-                tc_store_key_block<BITS>(rec + blk0 * CB, lane, my_tmem);
-                tc_store_key_block<BITS>(rec + (blk0 + 1) * CB, lane, my_tmem + (16u << 16));
-            }
-            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-            return landed;
-        };
-        auto issue_mmas = [&](int d_buf) {              // one thread
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const unsigned long long bdesc = qb_smem_desc(qb_addr + (n_cs & 1) * QB_BYTES);
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-                const unsigned accumulate = ks > 0 ? 1u : 0u;
-                asm volatile(
-                    "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                    "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], [%1], %2, %3, p;\n\t}"
-                    ::"r"(tmem + TC_D_COL + 16u * d_buf), "r"(tmem + static_cast<unsigned>(8 * ks)),
-                      "l"(bdesc + static_cast<unsigned long long>(ks * 2 * QB_LBO >> 4)), "r"(QK8_IDESC), "r"(accumulate) : "memory");
-            }
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(mma_bar) : "memory");
-        };
-        // ---- first tile of the round
-        {
-            next_start_segment();
-            const bool landed = start_tile();
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            if (__syncthreads_or((!landed || misc[7] != 0u) ? 1 : 0)) aborted = true;
-            if (!aborted && n_u < n_qp && tid == 0) issue_mmas(0);
-        }
-        next_finish_segment();
-        for (int i = 0; i < round_tiles && !aborted; ++i) {
-            const int s = stage;
-            const int my_u = f_u + half;
-            const bool tile_has_pages = f_u < f_qp;
-            const bool my_page = my_u < f_u1 && my_u < f_qp && !((misc[1 + s] >> half) & 1u);
-            const bool my_window = my_u < f_u1 && my_u >= f_qp;
-            const unsigned rec = stage0 + s * TILE + my_rec_off;       // this warp's unit
-            // ---- scores of tile i: the sums of the four e4m3 terms, rows g and g+8 of my two 16-token blocks
-            float d[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
-            bool scored = true;
-            if (tile_has_pages) {
-                scored = __all_sync(FULL, mbar_wait_bounded(mma_bar, mma_phase));
-                mma_phase ^= 1u;
-                if (!scored) misc[7] = 1u;                  // everybody leaves at the next barrier
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                if (my_page && scored) {
-                    unsigned q0[8], q1[8];                  // columns 2t, 2t+1, 8+2t, 9+2t of rows g (0,1,4,5) and g+8 (2,3,6,7)
-                    const unsigned dcol = TC_D_COL + 16u * (i & 1);
-                    asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                                 : "=r"(q0[0]), "=r"(q0[1]), "=r"(q0[2]), "=r"(q0[3]), "=r"(q0[4]), "=r"(q0[5]), "=r"(q0[6]), "=r"(q0[7])
-                                 : "r"(my_tmem + dcol) : "memory");
-                    asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                                 : "=r"(q1[0]), "=r"(q1[1]), "=r"(q1[2]), "=r"(q1[3]), "=r"(q1[4]), "=r"(q1[5]), "=r"(q1[6]), "=r"(q1[7])
-                                 : "r"(my_tmem + (16u << 16) + dcol) : "memory");
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    d[0][0] = (__uint_as_float(q0[0]) + __uint_as_float(q0[1])) + (__uint_as_float(q0[4]) + __uint_as_float(q0[5]));
-                    d[0][1] = (__uint_as_float(q0[2]) + __uint_as_float(q0[3])) + (__uint_as_float(q0[6]) + __uint_as_float(q0[7]));
-                    d[1][0] = (__uint_as_float(q1[0]) + __uint_as_float(q1[1])) + (__uint_as_float(q1[4]) + __uint_as_float(q1[5]));
-                    d[1][1] = (__uint_as_float(q1[2]) + __uint_as_float(q1[3])) + (__uint_as_float(q1[6]) + __uint_as_float(q1[7]));
-                }
-            }
-            // ---- start tile i+1
-            bool landed = true;
-            const bool more = i + 1 < round_tiles;
-            if (more) {
-                n_u += 2;
-                n_stage = (n_stage + 1 == TC_STAGES) ? 0 : n_stage + 1;
-                if (n_u >= n_u1) next_start_segment();
-                landed = start_tile();
-            }
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");     // my D reads and A writes precede the next MMAs
-            if (__syncthreads_or((!landed || misc[7] != 0u) ? 1 : 0)) { aborted = true; break; }
-            if (more && n_u < n_qp && tid == 0) issue_mmas((i + 1) & 1);
-            // tiles i and i+1 are in use; the stage of tile i-1 is free now
-            if (i >= 1 && issued < round_tiles) issue_tile((s + TC_STAGES - 1) % TC_STAGES, warp == (i & 3));
-            // ---- finish tile i
-            if (my_window && (warp & 1) == 0) {
-                const int w0 = (my_u - f_qp) * WIN_TOKENS;
-                window_unit<BITS, 0>(st, rec, min(WIN_TOKENS, f_nwin - w0), P.qwfrag + f_bh * 256, lane);
-            }
-            if (my_page && scored) {
-                const int pos0 = (f_page0 + my_u) * PAGE_TOKENS;
-                const bool full_page = (pos0 >= f_qlo) && (pos0 + PAGE_TOKENS <= f_qhi);
-                float sc[2][2];               // [block][row g, row g+8], divided by the head multiplier
-                unsigned vmeta[2][2];         // fp16x2 (Delta_v, x_min_v) of rows g, g+8
-#pragma unroll
-                for (int jb = 0; jb < 2; ++jb) {
-                    const uint4 mt = lds128(rec + meta_offset(BITS) + 128 * (blk0 + jb) + 16 * g);   // rows g (x,y) and g+8 (z,w)
-                    const float2 km_a = h2f2(mt.x), km_b = h2f2(mt.z);
-                    vmeta[jb][0] = mt.y; vmeta[jb][1] = mt.w;
-                    sc[jb][0] = fmaf(km_a.y, gadd, d[jb][0] * km_a.x);
-                    sc[jb][1] = fmaf(km_b.y, gadd, d[jb][1] * km_b.x);
-                }
-                if (!full_page) {             // first / last page of the quantized range: mask the tokens outside it
-#pragma unroll
-                    for (int jb = 0; jb < 2; ++jb) {
-                        const int p0 = pos0 + (blk0 + jb) * 16 + g, p1 = p0 + 8;
-                        if (p0 < f_qlo || p0 >= f_qhi) { vmeta[jb][0] = 0u; sc[jb][0] = -INFINITY; }
-                        if (p1 < f_qlo || p1 >= f_qhi) { vmeta[jb][1] = 0u; sc[jb][1] = -INFINITY; }
-                    }
-                }
-                float mx[1];
-                mx[0] = fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1])) * fmul;
-                st.raise_max(mx);
-#pragma unroll
-                for (int jb = 0; jb < 2; ++jb) {
-                    const int bi = blk0 + jb;
-                    const float2 vm_a = h2f2(vmeta[jb][0]), vm_b = h2f2(vmeta[jb][1]);
-                    const float p0 = ex2(fmaf(sc[jb][0], fmul, -st.mr[0])), p1 = ex2(fmaf(sc[jb][1], fmul, -st.mr[0]));
-                    st.l[0] += p0 + p1;
-                    st.z[0] = fmaf(p0, vm_a.y, fmaf(p1, vm_b.y, st.z[0]));
-                    const unsigned b01 = movmatrix_trans(pack_h2(p0 * vm_a.x, 0.f)), b23 = movmatrix_trans(pack_h2(p1 * vm_b.x, 0.f));
-                    if (BITS == 2) {
-                        const uint4 vw = lds128(rec + v_codes_offset(2) + bi * CB + 16 * lane);
-                        const unsigned sx = pre_shift<2>(vw.x), sy = pre_shift<2>(vw.y), sz = pre_shift<2>(vw.z), sw = pre_shift<2>(vw.w);
-#pragma unroll
-                        for (int i8 = 0; i8 < 8; ++i8)
-                            mma_f16(st.o[i8], field<2>(vw.x, sx, i8), field<2>(vw.y, sy, i8), field<2>(vw.z, sz, i8), field<2>(vw.w, sw, i8), b01, b23);
-                    } else {
-                        const uint4 va = lds128(rec + v_codes_offset(4) + bi * CB + 16 * lane);         // tokens 2t,2t+1
-                        const uint4 vb = lds128(rec + v_codes_offset(4) + bi * CB + 512 + 16 * lane);   // tokens 2t+8,2t+9
-                        const unsigned a0s = pre_shift<4>(va.x), a1s = pre_shift<4>(va.y), a2s = pre_shift<4>(va.z), a3s = pre_shift<4>(va.w);
-                        const unsigned b0s = pre_shift<4>(vb.x), b1s = pre_shift<4>(vb.y), b2s = pre_shift<4>(vb.z), b3s = pre_shift<4>(vb.w);
-#pragma unroll
-                        for (int k = 0; k < 4; ++k)     // channel blocks 0..3: words (rsel, j=0)
-                            mma_f16(st.o[k], field<4>(va.x, a0s, k), field<4>(va.z, a2s, k), field<4>(vb.x, b0s, k), field<4>(vb.z, b2s, k), b01, b23);
-#pragma unroll
-                        for (int k = 0; k < 4; ++k)     // channel blocks 4..7: words (rsel, j=1)
-                            mma_f16(st.o[4 + k], field<4>(va.y, a1s, k), field<4>(va.w, a3s, k), field<4>(vb.y, b1s, k), field<4>(vb.w, b3s, k), b01, b23);
-                    }
-                }
-            }
-            // ---- next tile to finish; a segment ends with its partial
-            stage = (stage + 1 == TC_STAGES) ? 0 : stage + 1;
-            f_u += 2;
-            if (f_u >= f_u1) {
-                store_partial<BITS, 0>(st, P.part + ((blockIdx.x + f_bh) * MAIN_WARPS + warp) * G * PART_STRIDE, lane, G);
-                if (f_cs + 1 < n_seg) next_finish_segment();
-            }
-        }
-    }
-    if (aborted) {
-        if (tid == 0) atomicOr(c.dev_status, WUSHKV_DEV_COPY_TIMEOUT);
-        // give copies that may still be in flight a bounded time to land before the CTA's memory is released
-        for (int k = 0; k < 1000; ++k) __nanosleep(1000);
-    }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(static_cast<unsigned>(TC_TMEM_COLS)) : "memory");
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1474,8 +998,7 @@ __global__ void __launch_bounds__(128 * MAX_GROUPS) decode_combine_kernel(Decode
 // ------------------------------------------------------------------------------------------------
 struct DecodePlan {
     int n_ctas, n_warps;
-    bool tensor_scores;      // main kernel with the scores in tensor memory (G <= 4)
-    size_t off_qfrag, off_qwfrag, off_qscal, off_plan, off_part, off_qb8, off_qscal8, total;
+    size_t off_qfrag, off_qwfrag, off_qscal, off_plan, off_part, total;
 };
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -1485,16 +1008,10 @@ static bool make_plan(const CacheView& c, int batch, int max_seq_len, DecodePlan
     const long long pages_max = (static_cast<long long>(max_seq_len) + PAGE_TOKENS - 1) / PAGE_TOKENS + 1;
     const long long win_max = std::min<long long>(max_seq_len, c.s_sink + c.s_keep + c.s_flush - 1 + c.lag);
     const long long units_max = (pages_max + (win_max + WIN_TOKENS - 1) / WIN_TOKENS + 1) * batch * c.n_kv;
-    // "tc" selects the kernel that computes the scores with tcgen05 (G <= 4 only).  It is kept as a measured
-    // alternative, not the default: its four warps move in lockstep (two CTA barriers per 128 tokens), and
-    // that costs more than the masks and MMA issues it saves.
-    const char* path = std::getenv("WUSHKV_DECODE_PATH");
-    pl.tensor_scores = c.G <= 4 && path && path[0] == 't';
-    long long ctas = 0;
-    if (const char* e = std::getenv("WUSHKV_DECODE_CTAS")) ctas = std::atoll(e);
+    long long ctas = knobs().decode_ctas;
     if (ctas <= 0) {
         // CTAs per SM: shared memory at 4 bits, registers for G > 4
-        const long long per_sm = pl.tensor_scores ? (c.bits == 4 ? 3 : 4) : (c.bits == 4 ? 3 : (c.G <= 4 ? 4 : 3));
+        const long long per_sm = c.bits == 4 ? 3 : (c.G <= 4 ? 4 : 3);
         ctas = std::min<long long>(per_sm * sm_count(), (units_max + 2 * MAIN_WARPS - 1) / (2 * MAIN_WARPS));
     }
     ctas = std::max<long long>(1, std::min<long long>(ctas, 1 << 20));
@@ -1506,9 +1023,7 @@ static bool make_plan(const CacheView& c, int batch, int max_seq_len, DecodePlan
     pl.off_qwfrag = off; off = align_up(off + bh * 256 * sizeof(uint4), 256);
     pl.off_qscal = off;  off = align_up(off + static_cast<size_t>(batch) * c.n_q * 2 * sizeof(float), 256);
     pl.off_plan = off;   off = align_up(off + (static_cast<size_t>(batch) + 1) * sizeof(long long), 256);
-    pl.off_part = off;   off = align_up(off + (pl.n_warps + bh * (pl.tensor_scores ? MAIN_WARPS : 1)) * c.G * PART_STRIDE * sizeof(float), 256);
-    pl.off_qb8 = off;    off = align_up(off + (pl.tensor_scores ? bh * QB_BYTES : 0), 256);
-    pl.off_qscal8 = off; off = align_up(off + (pl.tensor_scores ? static_cast<size_t>(batch) * c.n_q * 2 * sizeof(float) : 0), 256);
+    pl.off_part = off;   off = align_up(off + (pl.n_warps + bh) * c.G * PART_STRIDE * sizeof(float), 256);
     pl.total = off;
     return true;
 }
@@ -1520,8 +1035,6 @@ static int launch_decode(const DecodeParams& P, int n_ctas, cudaStream_t st) {
     constexpr int STAGES = 2;      // 4-bit records are twice as large: two stages keep three CTAs on an SM
     constexpr size_t SMEM = static_cast<size_t>(MAIN_WARPS) * STAGES * record_bytes(BITS) + MAIN_WARPS * STAGES * 8 +
                             MAIN_WARPS * MAX_SEGMENTS * sizeof(Segment);
-    constexpr size_t SMEM_TC = static_cast<size_t>(TC_STAGES) * 2 * record_bytes(BITS) + 2 * QB_BYTES + (TC_STAGES + 1) * 8 + 32 +
-                               MAX_SEGMENTS * sizeof(Segment);
     cudaLaunchAttribute pdl_attr[1];
     pdl_attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     pdl_attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -1533,26 +1046,12 @@ static int launch_decode(const DecodeParams& P, int n_ctas, cudaStream_t st) {
     cfg.blockDim = dim3(PREP_THREADS);
     cfg.dynamicSmemBytes = 0;
     if (cudaLaunchKernelEx(&cfg, decode_prep_kernel<BITS, MODE>, P) != cudaSuccess) return WUSHKV_ECUDA;
-    static bool smem_opted_in[64] = {};      // once per device and kernel instance
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return WUSHKV_ECUDA;
-    if (dev < 0 || dev >= 64 || !smem_opted_in[dev]) {
-        if (cudaFuncSetAttribute(decode_main_kernel<BITS, MODE, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(SMEM)) != cudaSuccess)
-            return WUSHKV_ECUDA;
-        if (MODE == 0 && cudaFuncSetAttribute(decode_main_tc_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(SMEM_TC)) != cudaSuccess)
-            return WUSHKV_ECUDA;
-        if (dev >= 0 && dev < 64) smem_opted_in[dev] = true;
-    }
+    if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(decode_main_kernel<BITS, MODE, STAGES>), static_cast<int>(SMEM))) return WUSHKV_ECUDA;
     if (g_prof_start) cudaEventRecord(g_prof_start, st);
     cfg.gridDim = dim3(n_ctas);
     cfg.blockDim = dim3(MAIN_WARPS * 32);
-    if (P.qb8 != nullptr) {
-        cfg.dynamicSmemBytes = SMEM_TC;
-        if (cudaLaunchKernelEx(&cfg, decode_main_tc_kernel<BITS>, P) != cudaSuccess) return WUSHKV_ECUDA;
-    } else {
-        cfg.dynamicSmemBytes = SMEM;
-        if (cudaLaunchKernelEx(&cfg, decode_main_kernel<BITS, MODE, STAGES>, P) != cudaSuccess) return WUSHKV_ECUDA;
-    }
+    cfg.dynamicSmemBytes = SMEM;
+    if (cudaLaunchKernelEx(&cfg, decode_main_kernel<BITS, MODE, STAGES>, P) != cudaSuccess) return WUSHKV_ECUDA;
     if (g_prof_stop) cudaEventRecord(g_prof_stop, st);
     // Partials per (sequence, KV head) are about n_warps / (batch n_kv).  Short lists go to one thread
     // group per CTA (a few rounds of COMBINE_BATCH loads); a long list (few sequences, long context)
@@ -1560,13 +1059,12 @@ static int launch_decode(const DecodeParams& P, int n_ctas, cudaStream_t st) {
     const long long per_head = P.n_warps / (static_cast<long long>(P.batch) * P.c.n_kv) + 2;
     cfg.gridDim = dim3(P.c.n_q, P.batch);
     cfg.dynamicSmemBytes = 0;
-    const bool shared_slices = P.slice_shift != 0;
     if (per_head <= 4 * COMBINE_BATCH) {
         cfg.blockDim = dim3(128, 1);
-        if (cudaLaunchKernelEx(&cfg, shared_slices ? decode_combine_kernel<1, 2> : decode_combine_kernel<1, 0>, P) != cudaSuccess) return WUSHKV_ECUDA;
+        if (cudaLaunchKernelEx(&cfg, decode_combine_kernel<1, 0>, P) != cudaSuccess) return WUSHKV_ECUDA;
     } else {
         cfg.blockDim = dim3(128, 8);
-        if (cudaLaunchKernelEx(&cfg, shared_slices ? decode_combine_kernel<8, 2> : decode_combine_kernel<8, 0>, P) != cudaSuccess) return WUSHKV_ECUDA;
+        if (cudaLaunchKernelEx(&cfg, decode_combine_kernel<8, 0>, P) != cudaSuccess) return WUSHKV_ECUDA;
     }
     return WUSHKV_OK;
 }
@@ -1603,9 +1101,6 @@ static int decode_attn_impl(const wushkv_cache* cache, int32_t batch, const int3
     P.plan = reinterpret_cast<long long*>(ws + pl.off_plan);
     P.part = reinterpret_cast<float*>(ws + pl.off_part);
     P.n_warps = pl.n_warps;
-    P.qb8 = pl.tensor_scores ? ws + pl.off_qb8 : nullptr;
-    P.qscal8 = pl.tensor_scores ? reinterpret_cast<float*>(ws + pl.off_qscal8) : nullptr;
-    P.slice_shift = pl.tensor_scores ? 2 : 0;
     {   // upper bound of the packed bytes one step reads against the L2 size
         static int l2_bytes[64] = {};
         int dev = 0;
@@ -1696,8 +1191,7 @@ extern "C" int wushkv_decode_step_host(const wushkv_cache* cache, int32_t batch,
     // Pinned host buffers are visible to the device: the kernels then read the new token and the queries,
     // and write the outputs, in place over the bus, which saves four copy operations per step (about 320 KB
     // in config 1, where the copies' fixed costs dominate).  WUSHKV_HOST_IO=copy forces the staged copies.
-    const char* io = std::getenv("WUSHKV_HOST_IO");
-    if (!(io && io[0] == 'c')) {
+    if (!knobs().host_io_copy) {
         void* aK = mapped_alias(K_new_host);
         void* aV = aK ? mapped_alias(V_new_host) : nullptr;
         void* aQ = aV ? mapped_alias(Q_host) : nullptr;

@@ -42,6 +42,37 @@ inline int make_view(const wushkv_cache* c, CacheView& v) {
     return WUSHKV_OK;
 }
 
+// Testing aids (wushkv_set_test_option).  The environment is read once, when the first call needs a
+// knob; afterwards only the setter changes them.  Process-global, not synchronised.
+struct Knobs {
+    long long decode_ctas = 0;      // > 0: number of thread blocks of the decode main kernel (the split count)
+    int append_path_cuda = 0;       // 1: chunks take the CUDA-core append path
+    int host_io_copy = 0;           // 1: wushkv_decode_step_host stages its buffers with copies even when they are mapped
+    long long drop_copy_unit = -1;  // >= 0: the decode main kernel never issues the copy of this unit of the flattened list
+    long long wait_limit = 0;       // > 0: poll limit of the device-side barrier waits (default: about a second)
+    int drop_chunk_mma = 0;         // 1: the chunk append never commits its first tile's MMAs to the barrier
+};
+Knobs& knobs();
+
+// Opts a kernel in to `bytes` of dynamic shared memory, once per (kernel, device).  Concurrent first calls
+// may both set the attribute (same value: harmless).
+inline bool opt_in_dynamic_smem(const void* fn, int bytes) {
+    struct Entry { const void* fn; unsigned long long devs; };
+    static Entry table[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    const bool dev_ok = dev >= 0 && dev < 64;
+    for (Entry& e : table) {
+        if (e.fn != fn && e.fn != nullptr) continue;
+        if (e.fn == fn && dev_ok && ((e.devs >> dev) & 1ull)) return true;
+        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+        e.fn = fn;
+        if (dev_ok) e.devs |= 1ull << dev;
+        return true;
+    }
+    return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+}
+
 inline int sm_count() {
     static int cached = 0;
     if (cached == 0) {

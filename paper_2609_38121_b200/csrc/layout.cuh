@@ -2,27 +2,27 @@
 //
 // A record holds PAGE_TOKENS = 64 tokens as 4 blocks of 16 tokens:
 //     [K codes: 4 blocks][V codes: 4 blocks][meta: 4 blocks x 128 B]
-// with a code block of 16*16*bits/... = 512 B (2-bit) or 1024 B (4-bit).  Inside a code block
+// with a code block of 16*128*bits/8 = 512 B (2-bit) or 1024 B (4-bit).  Inside a code block
 // byte 16*L .. 16*L+15 (of each 512-byte half) belongs to lane L = 4*g + t of the decode warp,
 // so that one 16-byte shared-memory load per lane yields exactly the words that lane turns into
-// mma.m16n8k16 A-fragments with a mask (and one shift) per register:
+// mma A-fragments with a mask (and at most one shift) per register.
 //
-//  K block (A = codes[16 tokens x 16 channels] per k-step s, channels 16s..16s+15):
-//    token row rr -> g = rr & 7, rs = rr >> 3;  channel ch -> s = ch >> 4, r16 = ch & 15,
-//    w = r16 >> 3, t = (r16 & 7) >> 1, hi = r16 & 1.
-//    2-bit: word (rs, w) of lane (g,t) at byte 16L + 8rs + 4w; code at bits 16hi + 2s.
-//    4-bit: 512-byte half rs; word j = 2(s>>2) + w at byte 512rs + 16L + 4j; code at bits 16hi + 4(s&3).
-//  V block (A = codes^T[16 channels x 16 tokens] per channel block i, channels 16i..16i+15):
+//  K block (integer mma.m16n8k32: A = codes[16 tokens x 32 channels] as unsigned bytes, one k-step s per
+//  32 channels):
+//    token row rr -> g = rr & 7, rs = rr >> 3;  channel ch -> s = ch >> 5, hh = (ch >> 4) & 1,
+//    b = 2 ((ch >> 3) & 1) + (ch & 1), t = (ch >> 1) & 3.  Word j = rs + 2 hh of lane (g,t) is A register j.
+//    2-bit: byte b of that word, at byte 16L + 4j + b of the block; code at bits 2s of the byte (one mask per
+//           k-step leaves the code, or four times the code, in every byte).
+//    4-bit: 512-byte half p = s >> 1; byte at 512p + 16L + 4j + b; code in nibble s & 1.
+//  V block (mma.m16n8k16: A = codes^T[16 channels x 16 tokens] as fp16 per channel block i, channels 16i..16i+15):
 //    token rr -> ps = rr >> 3, t = (rr & 7) >> 1, hi = rr & 1;  channel ch -> i = ch >> 4,
 //    r16 = ch & 15, rsel = r16 >> 3, g = r16 & 7.
 //    2-bit: half-word hi of word (ps, rsel) at byte 16L + 4(2ps + rsel) + 2hi; code at bits 2i.
 //    4-bit: 512-byte half ps; word (rsel, j = i>>2) at byte 512ps + 16L + 4(2rsel + j) + 2hi; code at bits 4(i&3).
+//    Masked out of a 16-bit lane and read as an fp16 bit pattern, a code field that lies inside bits 0..10 is the
+//    exact value code * 2^(shift-24) (fp16 subnormals and the first binade are linear in the bit pattern), so
+//    no int->float conversion is executed; the powers of two are folded into the output epilogue.
 //  meta block bi: token rr -> 8 bytes {K step, K x_min, V step, V x_min} (fp16) at 128bi + 16(rr&7) + 8(rr>>3).
-//
-// Masked out of a 16-bit lane and read as an fp16 bit pattern, a code field that lies inside bits
-// 0..10 is the exact value code * 2^(shift-24) (fp16 subnormals and the first binade are linear in
-// the bit pattern), so no int->float conversion is ever executed; the power-of-two factors are
-// folded into the query fragments and the output epilogue.
 #pragma once
 #include <cstdint>
 #include <cuda_runtime.h>
@@ -40,21 +40,22 @@ __host__ __device__ constexpr int v_codes_offset(int bits) { return BLOCKS_PER_P
 __host__ __device__ constexpr int meta_offset(int bits) { return 2 * BLOCKS_PER_PAGE * code_block_bytes(bits); }
 __host__ __device__ constexpr int record_bytes(int bits) { return meta_offset(bits) + PAGE_TOKENS * 8; }
 
-// Byte offset (within the record) of the 16-bit half-word holding K code (token r, channel ch) and
-// the bit position of the code inside that half-word.
+// Byte offset (within the record) of the byte holding K code (token r, channel ch) and the bit position
+// of the code inside that byte.
 __host__ __device__ inline void k_code_location(int bits, int r, int ch, int& byte_off, int& bit) {
     const int bi = r >> 4, rr = r & 15, g = rr & 7, rs = rr >> 3;
-    const int s = ch >> 4, r16 = ch & 15, w = r16 >> 3, t = (r16 & 7) >> 1, hi = r16 & 1;
-    const int L = 4 * g + t;
+    const int s = ch >> 5, hh = (ch >> 4) & 1, b = 2 * ((ch >> 3) & 1) + (ch & 1), t = (ch >> 1) & 3;
+    const int L = 4 * g + t, j = rs + 2 * hh;
     if (bits == 2) {
-        byte_off = bi * 512 + 16 * L + 8 * rs + 4 * w + 2 * hi;
+        byte_off = bi * 512 + 16 * L + 4 * j + b;
         bit = 2 * s;
     } else {
-        byte_off = bi * 1024 + 512 * rs + 16 * L + 4 * (2 * (s >> 2) + w) + 2 * hi;
-        bit = 4 * (s & 3);
+        byte_off = bi * 1024 + 512 * (s >> 1) + 16 * L + 4 * j + b;
+        bit = 4 * (s & 1);
     }
 }
 
+// The same for V code (token r, channel ch): offset of its 16-bit half-word and the bit position inside it.
 __host__ __device__ inline void v_code_location(int bits, int r, int ch, int& byte_off, int& bit) {
     const int bi = r >> 4, rr = r & 15, ps = rr >> 3, t = (rr & 7) >> 1, hi = rr & 1;
     const int i = ch >> 4, r16 = ch & 15, rsel = r16 >> 3, g = r16 & 7;

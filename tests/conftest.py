@@ -24,3 +24,21 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture
+def test_option():
+    """Sets process-wide testing aids of the library (wushkv_set_test_option) and restores the
+    defaults when the test ends."""
+    from paper_2609_38121_b200 import binding as B
+    defaults = {"decode_ctas": 0, "append_path_cuda": 0, "host_io_copy": 0, "drop_copy_unit": -1, "wait_limit": 0,
+                "drop_chunk_mma": 0}
+    used = []
+
+    def _set(name, value):
+        used.append(name)
+        B.set_test_option(name, value)
+
+    yield _set
+    for name in used:
+        B.set_test_option(name, defaults[name])

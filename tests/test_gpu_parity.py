@@ -95,12 +95,12 @@ def test_serving_window_sizes(s_sink, s_keep, s_flush):
 
 
 @pytest.mark.parametrize("path", ["tensor", "cuda"])
-def test_prefill_chunk_paths(path, monkeypatch):
+def test_prefill_chunk_paths(path, test_option):
     """Config 4's structure scaled down: several sequences appended as one chunk each in ONE call
     (tile boundaries fall inside sequences and a ragged last tile), Qwen-shaped heads (G = 7, RMSNorm),
     through the tensor-core transform and through the CUDA-core chunk path; then one decode step."""
     if path == "cuda":
-        monkeypatch.setenv("WUSHKV_APPEND_PATH", "cuda")
+        test_option("append_path_cuda", 1)
     wl = _wl(28, 4, seed=41, batch=3, theta=1e6, rmsnorm=True)
     L = Layer(wl, [700, 131, 390], 2, 4, 128, 1)
     L.append_step([699, 130, 389])
@@ -134,15 +134,15 @@ def test_no_sink_and_kappa_one():
     assert L.check_decode_parity() <= 2e-3
 
 
-def test_decode_is_deterministic_and_split_invariant(monkeypatch):
+def test_decode_is_deterministic_and_split_invariant(test_option):
     """The split count changes only the summation order: outputs for different splits agree to fp32
     rounding, and two identical calls agree bit for bit."""
     wl = _wl(8, 2, seed=32)
     L = Layer(wl, [3000], 2, 4, 64, 1)
     L.fill()
     outs = []
-    for ctas in ("5", "5", "1", "64"):
-        monkeypatch.setenv("WUSHKV_DECODE_CTAS", ctas)
+    for ctas in (5, 5, 1, 64):
+        test_option("decode_ctas", ctas)
         outs.append(L.decode()[0])
     assert np.array_equal(outs[0], outs[1])
     scale = np.max(np.abs(outs[0]))
@@ -242,13 +242,13 @@ def test_value_scale_invariance(log2_scale):
 
 
 @pytest.mark.parametrize("mode", ["mapped", "copy"])
-def test_host_step_equals_device_step(mode, monkeypatch):
+def test_host_step_equals_device_step(mode, test_option):
     """wushkv_decode_step_host (pinned host buffers read and written in place, or staged copies when
-    WUSHKV_HOST_IO=copy) gives the outputs and the cache of wushkv_decode_step, bit for bit."""
+    the "host_io_copy" option is set) gives the outputs and the cache of wushkv_decode_step, bit for bit."""
     import torch
     from paper_2609_38121_b200 import binding as B
     if mode == "copy":
-        monkeypatch.setenv("WUSHKV_HOST_IO", "copy")
+        test_option("host_io_copy", 1)
     wl = _wl(8, 2, seed=43)
     lengths, steps = [400, 70, 2], 2
     first = [n - steps for n in lengths]
@@ -282,18 +282,6 @@ def test_host_step_equals_device_step(mode, monkeypatch):
             for which in (0, 1):
                 for x, y in zip(host_l.gpu_codes(b, h, which), dev_l.gpu_codes(b, h, which)):
                     assert np.array_equal(x, y)
-
-
-@pytest.mark.parametrize("bits", [2, 4])
-def test_tensor_memory_score_path(bits, monkeypatch):
-    """The alternative main kernel (scores by tcgen05 from e4m3 code bytes in tensor memory, selected by
-    WUSHKV_DECODE_PATH=tc for G <= 4) meets the same tolerance on a ragged, shuffled-page batch."""
-    monkeypatch.setenv("WUSHKV_DECODE_PATH", "tc")
-    wl = _wl(8, 2, seed=52, batch=5)
-    L = Layer(wl, [1500, 0, 65, 300, 2], bits, 4, 64, 1, page_shuffle_seed=5)
-    L.fill()
-    assert L.check_decode_parity() <= 2e-3
-    assert L.cache.status() == 0
 
 
 def test_device_side_errors_are_flagged_not_fatal():

@@ -192,7 +192,7 @@ def test_wush_lowers_reconstruction_error_against_identity(bits):
     Qs = wl._queries(rng, np.full(nQ, S - 1)).astype(np.float64)
 
     def run(use_wush):
-        num_s = den_s = num_y = den_y = 0.0
+        s_hat_all, s_ref_all, y_hat_all, y_ref_all = [], [], [], []
         for h in range(n_kv):
             TK = T_K[h] if use_wush else np.eye(d)
             TKi = T_KinvT[h] if use_wush else np.eye(d)
@@ -206,20 +206,76 @@ def test_wush_lowers_reconstruction_error_against_identity(bits):
                 Qg = Qs[:, h * G + g]
                 s_ref = Keys[:, h] @ Qg.T                       # [S][nQ] pre-scaling scores
                 s_hat = Kq @ (Qg @ TKi.T).T
-                num_s += np.sum((s_hat - s_ref) ** 2)
-                den_s += np.sum(s_ref ** 2)
+                s_hat_all.append(s_hat.ravel())
+                s_ref_all.append(s_ref.ravel())
                 P = np.exp((s_ref - s_ref.max(0)) / np.sqrt(d))
                 P /= P.sum(0)
                 Ph = np.exp((s_hat - s_hat.max(0)) / np.sqrt(d))
                 Ph /= Ph.sum(0)
                 Wo = wl.W_O[h, g].astype(np.float64)
-                y_ref = (P.T @ Vr[:, h]) @ Wo
-                y_hat = (Ph.T @ Vq) @ (TVinvT @ Wo)
-                num_y += np.sum((y_hat - y_ref) ** 2)
-                den_y += np.sum(y_ref ** 2)
-        return num_s / den_s, num_y / den_y
+                y_ref_all.append(((P.T @ Vr[:, h]) @ Wo).ravel())
+                y_hat_all.append(((Ph.T @ Vq) @ (TVinvT @ Wo)).ravel())
+        # Section 5.1: numerator and denominator are each summed over every head and query first
+        return (O.rel_sq_err(np.concatenate(s_hat_all), np.concatenate(s_ref_all)),
+                O.rel_sq_err(np.concatenate(y_hat_all), np.concatenate(y_ref_all)))
 
     s_w, y_w = run(True)
     s_i, y_i = run(False)
     assert s_w < 0.5 * s_i, (s_w, s_i)
     assert y_w < y_i, (y_w, y_i)
+
+
+# ------------------------------------------------------------------ error metric (Section 5.1)
+def test_rel_sq_err_hand_cases_and_pooling():
+    # |(3,2) - (3,4)|^2 / |(3,4)|^2 = 4 / 25
+    assert O.rel_sq_err([3.0, 2.0], [3.0, 4.0]) == pytest.approx(0.16, rel=1e-15)
+    assert O.rel_sq_err([[1.0, -2.0], [0.5, 0.0]], [[1.0, -2.0], [0.5, 0.0]]) == 0.0
+    assert O.rel_sq_err(np.zeros(5), np.arange(1.0, 6.0)) == pytest.approx(1.0, rel=1e-15)     # predicting zero
+    # numerator and denominator are pooled before the division: a small block that is 100 % off and a
+    # large exact block give 1 / 101, not the mean 0.5 of the two blocks' ratios
+    pooled = O.rel_sq_err(np.array([2.0, 10.0]), np.array([1.0, 10.0]))
+    assert pooled == pytest.approx(1.0 / 101.0, rel=1e-15)
+    assert abs(pooled - 0.5 * (O.rel_sq_err([2.0], [1.0]) + O.rel_sq_err([10.0], [10.0]))) > 0.4
+    # invariant under a common scaling, not symmetric in its arguments
+    rng = np.random.default_rng(5)
+    A, E = rng.standard_normal((7, 9)), 0.1 * rng.standard_normal((7, 9))
+    assert O.rel_sq_err(3.0 * (A + E), 3.0 * A) == pytest.approx(O.rel_sq_err(A + E, A), rel=1e-12)
+    assert O.rel_sq_err(A + E, A) == pytest.approx(np.linalg.norm(E) ** 2 / np.linalg.norm(A) ** 2, rel=1e-12)
+    assert O.rel_sq_err(A + E, A) != pytest.approx(O.rel_sq_err(A, A + E), rel=1e-6)
+
+
+# ------------------------------------------------------------------ the other reading of "what is quantized"
+def test_quantize_from_bf16_reading():
+    """``LayerCache(quantize_from_bf16=True)`` quantizes the bf16 rounding of the transformed key (the
+    lazy reading of Section 4.4: the full-precision entry is what gets flushed); the default quantizes
+    the float transform output.  Values are never transformed, so they agree under both readings."""
+    rng = np.random.default_rng(33)
+    d, n_kv, S = 128, 2, 96
+    K = W.bf16_round_f32(rng.standard_normal((S, n_kv, d)).astype(np.float32) * 2).astype(np.float64)
+    V = W.bf16_round_f32(rng.standard_normal((S, n_kv, d)).astype(np.float32)).astype(np.float64)
+    Ms, Hs = [], []
+    for h in range(n_kv):
+        Qc = rng.standard_normal((2, 256, d)) * np.exp(rng.standard_normal(d))
+        M, H = O.gram_hessian(K[:, h], Qc)
+        Ms.append(M)
+        Hs.append(H)
+    T, _ = O.build_transforms(np.stack(Ms), np.stack(Hs))
+    eager = O.LayerCache(n_kv, d, 4, 0.96, 0.92, T)
+    lazy = O.LayerCache(n_kv, d, 4, 0.96, 0.92, T, quantize_from_bf16=True)
+    eager.append(K, V)
+    lazy.append(K, V)
+    kc_e, km_e, vc_e, vm_e, kb_e, vb_e = eager.arrays()
+    kc_l, km_l, vc_l, vm_l, kb_l, vb_l = lazy.arrays()
+    differing_vectors = 0
+    for t in range(S):
+        for h in range(n_kv):
+            kp = O.key_transform(T[h], K[t, h][None])[0]
+            c, dl, z = O.quantize(O.round_bf16(kp), 4, 0.96)
+            assert np.array_equal(kc_l[t, h], c) and km_l[t, h, 0] == dl and km_l[t, h, 1] == z
+            c2, dl2, z2 = O.quantize(kp, 4, 0.96)
+            assert np.array_equal(kc_e[t, h], c2) and km_e[t, h, 0] == dl2 and km_e[t, h, 1] == z2
+            differing_vectors += int(not np.array_equal(c, c2))
+    assert differing_vectors >= 1                      # the bf16 round trip moves some code at 4 bits
+    assert np.mean(kc_l != kc_e) < 0.05                # ... but only a small fraction of them
+    assert np.array_equal(vc_l, vc_e) and np.array_equal(vm_l, vm_e)
+    assert np.array_equal(kb_l, kb_e) and np.array_equal(vb_l, vb_e)     # window copies do not depend on the reading
