@@ -79,11 +79,8 @@ struct DecodeParams {
     uint4* qwfrag;       // [batch*n_kv][2][128]: bf16 B fragments for the windows (MODE 1: value set, remainder set)
     float* qscal;        // [batch][n_q][2]: score multiplier (log2 domain, > 0), x_min multiplier divided by it
     long long* plan;     // [batch+1]: exclusive prefix of work units per sequence (per KV head)
-    float* part;         // [n_ctas + batch*n_kv][G][PART_STRIDE]: the partial of main-kernel CTA c for (sequence, KV head) index bh is slot c + bh
-    int* part_state;     // [n_ctas + batch*n_kv]: lock / "holds a partial" word of each slot that is merged in the workspace (zeroed by the preparation kernel)
-    int n_ctas;          // CTAs of the main kernel
-    int wait_limit;      // poll limit of the device-side barrier waits (0: default)
-    long long drop_unit; // testing aid: flattened index of a unit whose copy is never issued (-1: none)
+    float* part;         // [n_warps + batch*n_kv][G][PART_STRIDE]
+    int n_warps;         // warps of the main kernel
     int q_early;         // 1: Q was final before the kernel ahead of the preparation kernel started
     int stream_pages;    // 1: the packed pages of a step cannot stay in L2 anyway: copy them with an evict-first hint
 };
@@ -146,11 +143,6 @@ __global__ void __launch_bounds__(PREP_THREADS) decode_prep_kernel(DecodeParams 
     // transform of the queries runs beside the append.  The main kernel reads the lengths and stages
     // pages as soon as it starts, so the plan CTA holds its launch signal back until the append is done.
     const bool plan_cta = h == 0 && b == 0;
-    {   // slot states of the main kernel's workspace merges (read there only after this kernel has completed)
-        const int n_slots = P.n_ctas + P.batch * P.c.n_kv;
-        const int gid = (b * gridDim.x + h) * PREP_THREADS + i, gsz = gridDim.x * gridDim.y * PREP_THREADS;
-        for (int k = gid; k < n_slots; k += gsz) P.part_state[k] = 0;
-    }
     if (!P.q_early) pdl_wait();
     if (!(P.q_early && plan_cta)) pdl_launch_dependents();   // the main kernel may start staging pages while this one runs
 
@@ -323,8 +315,8 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
     return ok != 0;
 }
 // Bounded wait: false if the phase did not complete within the limit (about a second of sleeping polls).
-__device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity, int limit) {
-    for (int it = 0; it < limit; ++it)
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity) {
+    for (int it = 0; it < (1 << 19); ++it)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -473,26 +465,11 @@ struct WarpState {
     }
 };
 
-// Folds this warp's partial (max, sum, o[128] of every head) of one (sequence, KV head) into the CTA's partial of
-// that pair.  dst0 / state may point to shared memory (the CTA's first segments) or to the workspace (any further
-// ones); state: bit 0 lock, bit 1 "holds a partial".  All warps that merge into one slot belong to one CTA.
-// Returns false if the lock could not be taken within the limit.
+// Writes this warp's partial (max, sum, o[128]) of every head of one (sequence, KV head) to global memory.
 template <int BITS, int MODE>
-__device__ __forceinline__ bool merge_partial(const WarpState<MODE>& st, float* dst0, int* state, int lane, int G, int spin_limit) {
+__device__ __forceinline__ void store_partial(const WarpState<MODE>& st, float* dst0, int lane, int G) {
     const int g = lane >> 2, t = lane & 3;
     constexpr int NH = WarpState<MODE>::NH;
-    int v = 0;
-    bool ok = true;
-    if (lane == 0) {
-        ok = false;
-        for (int it = 0; it < spin_limit && !ok; ++it) {
-            v = *reinterpret_cast<volatile int*>(state);
-            if (!(v & 1) && atomicCAS(state, v, v | 1) == v) ok = true; else __nanosleep(64);
-        }
-    }
-    if (!__shfl_sync(FULL, ok, 0)) return false;
-    const bool init = (__shfl_sync(FULL, v, 0) & 2) != 0;
-    __threadfence();
 #pragma unroll
     for (int k = 0; k < NH; ++k) {
         float l = st.l[k], z = st.z[k];
@@ -500,13 +477,9 @@ __device__ __forceinline__ bool merge_partial(const WarpState<MODE>& st, float* 
         l += __shfl_xor_sync(FULL, l, 8);  z += __shfl_xor_sync(FULL, z, 8);
         l += __shfl_xor_sync(FULL, l, 16); z += __shfl_xor_sync(FULL, z, 16);
         const int head = MODE == 0 ? t : 2 * t + k;
-        const bool live = head < G;
-        volatile float* dst = dst0 + (live ? head : 0) * PART_STRIDE;
-        const float m_old = init ? dst[0] : -INFINITY, l_old = init ? dst[1] : 0.f;
-        const float m_w = st.m[k];
-        const float mn = fmaxf(m_old, m_w);
-        const float sa = m_old == -INFINITY ? 0.f : ex2(m_old - mn), sb = m_w == -INFINITY ? 0.f : ex2(m_w - mn);
-        if (live) {
+        if (head < G) {
+            float* dst = dst0 + head * PART_STRIDE;
+            if (g == 0) { dst[0] = st.m[k]; dst[1] = l; }
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const float osc = exp2f(static_cast<float>(24 - field_shift<BITS>(i)));
@@ -518,18 +491,11 @@ __device__ __forceinline__ bool merge_partial(const WarpState<MODE>& st, float* 
                     lo_ch = st.o[i][k] * osc + z;
                     hi_ch = st.o[i][2 + k] * osc + z;
                 }
-                volatile float* po = dst + 4 + 16 * i + g;
-                po[0] = (init ? po[0] * sa : 0.f) + lo_ch * sb;
-                po[8] = (init ? po[8] * sa : 0.f) + hi_ch * sb;
+                dst[4 + 16 * i + g] = lo_ch;
+                dst[4 + 16 * i + g + 8] = hi_ch;
             }
         }
-        __syncwarp();                           // every lane has read the old reference and sum
-        if (live && g == 0) { dst[0] = mn; dst[1] = l_old * sa + l * sb; }
     }
-    __threadfence();
-    __syncwarp();
-    if (lane == 0) atomicExch(state, 2);
-    return true;
 }
 
 // One window unit: up to 8 bf16 tokens staged at shared-memory address rec (key rows, then value rows at
@@ -593,7 +559,7 @@ constexpr int MAX_SEGMENTS = 6;           // per warp and round; more segments t
 // main kernel
 // ------------------------------------------------------------------------------------------------
 #ifndef WUSHKV_ABL
-#define WUSHKV_ABL 0        // timing experiments only: 1 no value contraction, 2 no key contraction, 4 start-up skew between the CTAs of an SM, 8 no page copies
+#define WUSHKV_ABL 0        // timing experiments only: 1 no value contraction, 2 no key contraction, 8 no page copies, 16 per-warp time stamps
 #endif
 #if WUSHKV_ABL & 16
 __device__ unsigned long long g_timeline[8192 * 4];
@@ -603,26 +569,16 @@ __device__ __forceinline__ unsigned long long gtime() { unsigned long long t; as
 #define TL(slot) do { } while (0)
 #endif
 
-__host__ __device__ constexpr int merge_slots(int mode) { return mode == 0 ? 4 : 2; }        // segments of a CTA merged in shared memory
-__host__ __device__ constexpr int merge_heads(int mode) { return mode == 0 ? 4 : 8; }
-
 template <int BITS, int MODE, int STAGES>
 __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_kernel(DecodeParams P) {
     constexpr int MAIN_WARPS = main_warps(BITS, MODE);
     constexpr int REC = record_bytes(BITS);
     constexpr int CB = code_block_bytes(BITS);
     constexpr int NH = WarpState<MODE>::NH;
-    constexpr int MSLOTS = merge_slots(MODE), MSLOT_FLOATS = merge_heads(MODE) * PART_STRIDE;
     static_assert(2 * WIN_TOKENS * WIN_ROW <= REC, "a window unit must fit in one stage");
     extern __shared__ __align__(128) unsigned char smem[];
-    constexpr size_t OFF_BARS = static_cast<size_t>(MAIN_WARPS) * STAGES * REC;
-    constexpr size_t OFF_SEGS = OFF_BARS + MAIN_WARPS * STAGES * 8;
-    constexpr size_t OFF_MERGE = (OFF_SEGS + MAIN_WARPS * MAX_SEGMENTS * sizeof(Segment) + 15) / 16 * 16;
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + OFF_BARS);
-    Segment* seg_all = reinterpret_cast<Segment*>(smem + OFF_SEGS);
-    float* merge_s = reinterpret_cast<float*>(smem + OFF_MERGE);                    // [MSLOTS][heads][PART_STRIDE]
-    __shared__ int merge_state[MSLOTS];
-    __shared__ int bh_first_s;              // (sequence, KV head) index of the first unit of the CTA's slice
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + MAIN_WARPS * STAGES * REC);
+    Segment* seg_all = reinterpret_cast<Segment*>(smem + MAIN_WARPS * STAGES * REC + MAIN_WARPS * STAGES * 8);
     const CacheView& c = P.c;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
@@ -631,24 +587,16 @@ __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_ke
     TL(0);
 
     // ---- work plan: prefix sums of units per sequence.  Recomputed here from the inputs (into the still
-    // unused staging area, with the lengths and slots beside it) so that nothing the preparation kernel
-    // writes is needed before the first copies.
+    // unused staging area) so that nothing the preparation kernel writes is needed before the first copies.
     __shared__ long long scan_s[MAIN_WARPS];
     long long* plan_s = reinterpret_cast<long long*>(smem);
-    int* lens_s = reinterpret_cast<int*>(plan_s + P.batch + 1);
-    int* slots_s = lens_s + P.batch;
-    const bool local_plan = (static_cast<size_t>(P.batch) + 1) * 16 <= static_cast<size_t>(MAIN_WARPS) * STAGES * REC;
-    if (threadIdx.x < MSLOTS) merge_state[threadIdx.x] = 0;
+    const bool local_plan = (static_cast<size_t>(P.batch) + 1) * sizeof(long long) <= static_cast<size_t>(MAIN_WARPS) * STAGES * REC;
     if (local_plan) {
         long long carry = 0;
         for (int base = 0; base < P.batch; base += MAIN_WARPS * 32) {
             const int bb = base + threadIdx.x;
             long long incl = 0;
-            if (bb < P.batch) {
-                const int S = __ldcg(P.seq_len + bb), sl = __ldg(P.slot + bb);
-                lens_s[bb] = S; slots_s[bb] = sl;
-                incl = seq_info(c, S, sl).U;
-            }
+            if (bb < P.batch) incl = seq_info(c, __ldcg(P.seq_len + bb), __ldg(P.slot + bb)).U;
             for (int o = 1; o < 32; o <<= 1) {
                 const long long v = __shfl_up_sync(FULL, incl, o);
                 if (lane >= o) incl += v;
@@ -668,17 +616,15 @@ __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_ke
     }
     const long long* plan = local_plan ? plan_s : P.plan;
 
-    // ---- the CTA's slice of the flattened unit list (equal cuts over the CTAs, which is what the combine
-    // kernel reconstructs), and this warp's equal share of it
+    // ---- this warp's slice of the flattened unit list
     const long long total = plan[P.batch] * c.n_kv;
-    const long long Lc = total > 0 ? blockIdx.x * total / gridDim.x : 0;
-    const int n_cta_units = static_cast<int>((total > 0 ? (blockIdx.x + 1) * total / gridDim.x : 0) - Lc);
-    long long L = Lc + static_cast<long long>(warp) * n_cta_units / MAIN_WARPS;
-    const long long L1 = Lc + static_cast<long long>(warp + 1) * n_cta_units / MAIN_WARPS;
+    const long long wg = static_cast<long long>(blockIdx.x) * MAIN_WARPS + warp;
+    long long L = total > 0 ? wg * total / P.n_warps : 0;
+    const long long L1 = total > 0 ? (wg + 1) * total / P.n_warps : 0;
 
     // position of the slice start: sequence b, head h, unit u
     int sb = 0, sh = 0, su = 0;
-    if (L < L1 || warp == 0) {
+    if (L < L1) {
         int lo = 0, hi = P.batch;           // largest b with n_kv * plan[b] <= L
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
@@ -690,7 +636,9 @@ __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_ke
         sh = static_cast<int>(rem / U);
         su = static_cast<int>(rem % U);
     }
-    if (threadIdx.x == 0) bh_first_s = sb * c.n_kv + sh;
+    __syncthreads();                        // the staging area stops being plan scratch here
+    pdl_launch_dependents();
+    if (L >= L1) return;
 
     // ---- barriers
     const unsigned bar0 = smem_u32(bars + warp * STAGES);
@@ -699,17 +647,26 @@ __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_ke
         for (int s = 0; s < STAGES; ++s) mbar_init(bar0 + 8 * s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    __syncwarp();
     const unsigned stage0 = smem_u32(smem + warp * STAGES * REC);
     const long long page_row_bytes = static_cast<long long>(c.n_kv) * REC;
     const unsigned long long stream_policy = l2_evict_first_policy();
 
-    // Lists the next (up to MAX_SEGMENTS) segments of the slice into shared memory; returns their unit count.
-    int n_seg = 0;
-    auto list_round = [&](const bool from_smem) -> int {
-        int round_units = 0;
-        n_seg = 0;
+    if (WUSHKV_ABL & 8) { for (int k = lane; k < STAGES * REC / 4; k += 32) reinterpret_cast<unsigned*>(smem + warp * STAGES * REC)[k] = 0u; __syncwarp(); }
+    unsigned qf[4][2];                  // integer B fragments of the four k-steps (MODE 1: the high digits)
+    unsigned qfl[MODE == 1 ? 4 : 1][2]; // MODE 1: the low digits
+    float fmul[NH], gadd[NH];
+    WarpState<MODE> st;
+    int stage = 0;                      // ring position of the next unit to consume (and to refill)
+    unsigned phase_bits = 0;            // parity of each stage's next completion
+    unsigned bad_bits = 0;              // lane 0: stages whose unit could not be fetched
+    bool timed_out = false;
+
+    while (L < L1 && !timed_out) {
+        // ================= round set-up: list the next segments of the slice =====================
+        int n_seg = 0, round_units = 0;
         while (n_seg < MAX_SEGMENTS && L < L1) {
-            const SeqInfo si = from_smem ? seq_info(c, lens_s[sb], slots_s[sb]) : seq_info(c, __ldcg(P.seq_len + sb), __ldg(P.slot + sb));
+            const SeqInfo si = seq_info(c, __ldcg(P.seq_len + sb), __ldg(P.slot + sb));
             if (si.U > 0) {
                 const int u1 = static_cast<int>(min(static_cast<long long>(si.U), su + (L1 - L)));
                 if (lane == 0) {
@@ -730,34 +687,8 @@ __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_ke
             }
         }
         __syncwarp();
-        return round_units;
-    };
-    // the first round is listed while the lengths are still in shared memory
-    int round_units = list_round(local_plan);
-    __syncthreads();                        // the staging area stops being plan scratch here
-    pdl_launch_dependents();
-    const int bh_first = bh_first_s;
-    const int spin_limit = 1 << 22;
-    const int wait_limit = P.wait_limit > 0 ? P.wait_limit : (1 << 19);      // polls that may sleep ~2 us each: about a second
-
-    if (WUSHKV_ABL & 8) { for (int k = lane; k < STAGES * REC / 4; k += 32) reinterpret_cast<unsigned*>(smem + warp * STAGES * REC)[k] = 0u; __syncwarp(); }
-    unsigned qf[4][2];                  // integer B fragments of the four k-steps (MODE 1: the high digits)
-    unsigned qfl[MODE == 1 ? 4 : 1][2]; // MODE 1: the low digits
-    float fmul[NH], gadd[NH];
-    WarpState<MODE> st;
-    int stage = 0;                      // ring position of the next unit to consume (and to refill)
-    unsigned phase_bits = 0;            // parity of each stage's next completion
-    unsigned bad_bits = 0;              // lane 0: stages whose unit could not be fetched
-    bool timed_out = false;
-    bool first_round = true;
-
-    while ((first_round ? round_units > 0 : L < L1) && !timed_out) {
-        // ================= round set-up: list the next segments of the slice =====================
-        if (!first_round) round_units = list_round(false);
-        first_round = false;
 
         // ================= producer: stages the units of this round, in order =====================
-        const long long round_L0 = L - round_units;      // flattened index of the round's first unit
         int p_seg = -1, p_u = 0, p_u1 = 0, p_qp = 0, p_head_off = 0, issued = 0;
         const int* p_ptab = nullptr;
         auto issue_next = [&](const int s) {            // whole warp; stages the round's next unit into ring slot s
@@ -786,9 +717,7 @@ __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_ke
                     } else {
                         bad_bits &= ~(1u << s);
                         mbar_expect_tx(bar, REC);
-                        if (P.drop_unit >= 0 && P.drop_unit == round_L0 + issued) {
-                            // testing aid: this copy is never issued, the wait for it runs into its limit
-                        } else if (P.stream_pages) bulk_copy_g2s_stream(dst, c.pages + page * page_row_bytes + p_head_off, REC, bar, stream_policy);
+                        if (P.stream_pages) bulk_copy_g2s_stream(dst, c.pages + page * page_row_bytes + p_head_off, REC, bar, stream_policy);
                         else bulk_copy_g2s(dst, c.pages + page * page_row_bytes + p_head_off, REC, bar);
                     }
                 }
@@ -845,7 +774,7 @@ __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_ke
             for (int u = sg.u0; u < u1; ++u, pos0 += PAGE_TOKENS) {
                 const int s = stage;
                 // a phase that one lane saw complete is complete for all: keep the decision warp-uniform
-                if (!__any_sync(FULL, mbar_wait_bounded(bar0 + 8 * s, (phase_bits >> s) & 1u, wait_limit))) { timed_out = true; break; }
+                if (!__any_sync(FULL, mbar_wait_bounded(bar0 + 8 * s, (phase_bits >> s) & 1u))) { timed_out = true; break; }
                 phase_bits ^= 1u << s;
 #if WUSHKV_ABL & 16
                 if (lane == 0 && g_timeline[((blockIdx.x * 16 + warp) & 8191) * 4 + 2] == 0) g_timeline[((blockIdx.x * 16 + warp) & 8191) * 4 + 2] = gtime();
@@ -991,12 +920,7 @@ __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_ke
                 if (issued < round_units) issue_next(s);         // refill the stage just consumed
                 stage = (stage + 1 == STAGES) ? 0 : stage + 1;
             }
-            {   // fold this warp's state into the CTA's partial of the segment
-                const int bh_seg = sg.b * c.n_kv + sg.h, ls = bh_seg - bh_first;
-                float* dst0 = ls < MSLOTS ? merge_s + ls * MSLOT_FLOATS : P.part + (static_cast<long long>(blockIdx.x) + bh_seg) * G * PART_STRIDE;
-                int* state = ls < MSLOTS ? &merge_state[ls] : P.part_state + blockIdx.x + bh_seg;
-                if (!merge_partial<BITS, MODE>(st, dst0, state, lane, G, spin_limit)) timed_out = true;
-            }
+            store_partial<BITS, MODE>(st, P.part + (wg + static_cast<long long>(sg.b) * c.n_kv + sg.h) * G * PART_STRIDE, lane, G);
         }
         __syncwarp();
     }
@@ -1006,26 +930,16 @@ __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_ke
         // give copies that may still be in flight a bounded time to land before the CTA's memory is released
         for (int k = 0; k < 1000; ++k) __nanosleep(1000);
     }
-    // ---- the CTA's partials of its first segments leave shared memory (every warp gets here)
-    __syncthreads();
-#pragma unroll 1
-    for (int ls = 0; ls < MSLOTS; ++ls) {
-        if (!(merge_state[ls] & 2)) continue;
-        float* dst = P.part + (static_cast<long long>(blockIdx.x) + bh_first + ls) * G * PART_STRIDE;
-        for (int k = threadIdx.x; k < G * PART_STRIDE; k += MAIN_WARPS * 32) dst[k] = merge_s[ls * MSLOT_FLOATS + k];
-    }
 }
 
 // ------------------------------------------------------------------------------------------------
 // 3. combine
 // ------------------------------------------------------------------------------------------------
 // One CTA per (sequence, query head): up to 8 thread groups of one thread per channel, each merging a
-// contiguous share of the head's partials.  Every CTA of the main kernel whose slice meets the units of the
-// head's (sequence, KV head) wrote exactly one partial for it, at slot (CTA + index of the pair); the slices
-// are equal cuts of the flattened unit list, so the covering CTAs follow from the plan alone.  The partials
-// sit in L2, so the cost is load latency: a group issues the loads of COMBINE_BATCH partials together.
+// contiguous share of the head's partials.  The partials sit in L2, so the cost is load latency: a
+// group issues the loads of COMBINE_BATCH partials together before it merges them.
 constexpr int COMBINE_BATCH = 8;        // loads in flight per thread
-template <int MAX_GROUPS>
+template <int MAX_GROUPS, int GS>      // GS: log2 of the warps per slice (compile-time copy of slice_shift)
 __global__ void __launch_bounds__(128 * MAX_GROUPS) decode_combine_kernel(DecodeParams P) {
     __shared__ float red_m[MAX_GROUPS], red_l[MAX_GROUPS], red_o[MAX_GROUPS][D];
     const CacheView& c = P.c;
@@ -1038,16 +952,26 @@ __global__ void __launch_bounds__(128 * MAX_GROUPS) decode_combine_kernel(Decode
     if (U <= 0 || total <= 0) { if (grp == 0) out[ch] = 0.f; return; }
     const int h = j / c.G, head = j % c.G;
     const long long La = P.plan[b] * c.n_kv + static_cast<long long>(h) * U, Lb = La + U;      // units [La, Lb)
-    // slice i of the main kernel = [floor(i total / ns), floor((i+1) total / ns))
-    const long long ns = P.n_ctas;
+    // The unit list is cut into ns equal slices, slice i = [floor(i total / ns), floor((i+1) total / ns)); a
+    // slice belongs to one warp (slice_shift 0) or to the four warps of a CTA (slice_shift 2), and every
+    // warp of a slice that meets [La, Lb) wrote a partial, at slot (slice + bh) * warps_per_slice + warp.
+    constexpr int gs = GS, group_mask = (1 << gs) - 1;
+    const long long ns = static_cast<long long>(P.n_warps) >> gs;
     const long long s_first = ((La + 1) * ns - 1) / total, s_last = (Lb * ns - 1) / total;   // owners of La and Lb-1
     const long long bh = static_cast<long long>(b) * c.n_kv + h;
     const long long stride = static_cast<long long>(c.G) * PART_STRIDE;
-    const int n = static_cast<int>(s_last - s_first + 1);
+    const int n = static_cast<int>(s_last - s_first + 1) << gs;
     // thread group grp merges the contiguous share [k0, k1) of the n partials
     const int share = (n + n_grp - 1) / n_grp;
     const int k0 = min(grp * share, n), k1 = min(k0 + share, n);
-    const float* base = P.part + ((s_first + bh + k0) * c.G + head) * PART_STRIDE;
+    const float* base = P.part + ((((s_first + bh) << gs) + k0) * c.G + head) * PART_STRIDE;
+    // slice bounds advance by q = total / ns with a carry of r = total % ns (no division in the loop)
+    const long long q = total / ns, r = total % ns;
+    const long long sl0 = s_first + (k0 >> gs);
+    long long lo_w = sl0 * total / ns, rem = (sl0 * total) % ns;
+    long long hi_w = lo_w + q;
+    rem += r;
+    if (rem >= ns) { rem -= ns; ++hi_w; }
     float m = -INFINITY, l = 0.f, o = 0.f;
     for (int s0 = k0; s0 < k1; s0 += COMBINE_BATCH) {
         float pm[COMBINE_BATCH], pl[COMBINE_BATCH], po[COMBINE_BATCH];
@@ -1055,8 +979,17 @@ __global__ void __launch_bounds__(128 * MAX_GROUPS) decode_combine_kernel(Decode
         for (int k = 0; k < COMBINE_BATCH; ++k) {
             pm[k] = -INFINITY; pl[k] = 0.f; po[k] = 0.f;
             if (s0 + k < k1) {
-                const float* p = base + (s0 - k0 + k) * stride;
-                pm[k] = __ldcg(p); pl[k] = __ldcg(p + 1); po[k] = __ldcg(p + 4 + ch);
+                const bool wrote = max(lo_w, La) < min(hi_w, Lb);     // a slice that misses the range wrote nothing
+                if (((s0 + k + 1) & group_mask) == 0) {               // next partial belongs to the next slice
+                    lo_w = hi_w;
+                    hi_w = lo_w + q;
+                    rem += r;
+                    if (rem >= ns) { rem -= ns; ++hi_w; }
+                }
+                if (wrote) {
+                    const float* p = base + (s0 - k0 + k) * stride;
+                    pm[k] = __ldcg(p); pl[k] = __ldcg(p + 1); po[k] = __ldcg(p + 4 + ch);
+                }
             }
         }
 #pragma unroll
@@ -1091,8 +1024,8 @@ __global__ void __launch_bounds__(128 * MAX_GROUPS) decode_combine_kernel(Decode
 // host side
 // ------------------------------------------------------------------------------------------------
 struct DecodePlan {
-    int n_ctas;
-    size_t off_qfrag, off_qwfrag, off_qscal, off_plan, off_part, off_state, total;
+    int n_ctas, n_warps;
+    size_t off_qfrag, off_qwfrag, off_qscal, off_plan, off_part, total;
 };
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -1110,14 +1043,14 @@ static bool make_plan(const CacheView& c, int batch, int max_seq_len, DecodePlan
     }
     ctas = std::max<long long>(1, std::min<long long>(ctas, 1 << 20));
     pl.n_ctas = static_cast<int>(ctas);
+    pl.n_warps = pl.n_ctas * warps;
     const size_t bh = static_cast<size_t>(batch) * c.n_kv;
     size_t off = 0;
     pl.off_qfrag = off;  off = align_up(off + bh * 256 * sizeof(uint4), 256);
     pl.off_qwfrag = off; off = align_up(off + bh * 256 * sizeof(uint4), 256);
     pl.off_qscal = off;  off = align_up(off + static_cast<size_t>(batch) * c.n_q * 2 * sizeof(float), 256);
     pl.off_plan = off;   off = align_up(off + (static_cast<size_t>(batch) + 1) * sizeof(long long), 256);
-    pl.off_part = off;   off = align_up(off + (pl.n_ctas + bh) * c.G * PART_STRIDE * sizeof(float), 256);
-    pl.off_state = off;  off = align_up(off + (pl.n_ctas + bh) * sizeof(int), 256);
+    pl.off_part = off;   off = align_up(off + (pl.n_warps + bh) * c.G * PART_STRIDE * sizeof(float), 256);
     pl.total = off;
     return true;
 }
@@ -1128,10 +1061,8 @@ template <int BITS, int MODE>
 static int launch_decode(const DecodeParams& P, int n_ctas, cudaStream_t st) {
     constexpr int MAIN_WARPS = main_warps(BITS, MODE);
     constexpr int STAGES = 2;      // per-warp ring depth
-    constexpr size_t SMEM = (static_cast<size_t>(MAIN_WARPS) * STAGES * record_bytes(BITS) + MAIN_WARPS * STAGES * 8 +
-                             MAIN_WARPS * MAX_SEGMENTS * sizeof(Segment) + 15) / 16 * 16 +
-                            static_cast<size_t>(merge_slots(MODE)) * merge_heads(MODE) * PART_STRIDE * sizeof(float);
-    static_assert(SMEM <= 227 * 1024, "shared memory of the main kernel");
+    constexpr size_t SMEM = static_cast<size_t>(MAIN_WARPS) * STAGES * record_bytes(BITS) + MAIN_WARPS * STAGES * 8 +
+                            MAIN_WARPS * MAX_SEGMENTS * sizeof(Segment);
     cudaLaunchAttribute pdl_attr[1];
     pdl_attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     pdl_attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -1150,17 +1081,18 @@ static int launch_decode(const DecodeParams& P, int n_ctas, cudaStream_t st) {
     cfg.dynamicSmemBytes = SMEM;
     if (cudaLaunchKernelEx(&cfg, decode_main_kernel<BITS, MODE, STAGES>, P) != cudaSuccess) return WUSHKV_ECUDA;
     if (g_prof_stop) cudaEventRecord(g_prof_stop, st);
-    // One partial per (CTA, sequence, KV head): a head's list is as long as the number of CTAs its units span.
-    // Short lists go to one thread group per CTA; a long one (few sequences, long context) is shared by 8 groups.
-    const long long per_head = P.n_ctas / (static_cast<long long>(P.batch) * P.c.n_kv) + 2;
+    // Partials per (sequence, KV head) are about n_warps / (batch n_kv).  Short lists go to one thread
+    // group per CTA (a few rounds of COMBINE_BATCH loads); a long list (few sequences, long context)
+    // is shared by 8 groups.
+    const long long per_head = P.n_warps / (static_cast<long long>(P.batch) * P.c.n_kv) + 2;
     cfg.gridDim = dim3(P.c.n_q, P.batch);
     cfg.dynamicSmemBytes = 0;
-    if (per_head <= 2 * COMBINE_BATCH) {
+    if (per_head <= 4 * COMBINE_BATCH) {
         cfg.blockDim = dim3(128, 1);
-        if (cudaLaunchKernelEx(&cfg, decode_combine_kernel<1>, P) != cudaSuccess) return WUSHKV_ECUDA;
+        if (cudaLaunchKernelEx(&cfg, decode_combine_kernel<1, 0>, P) != cudaSuccess) return WUSHKV_ECUDA;
     } else {
         cfg.blockDim = dim3(128, 8);
-        if (cudaLaunchKernelEx(&cfg, decode_combine_kernel<8>, P) != cudaSuccess) return WUSHKV_ECUDA;
+        if (cudaLaunchKernelEx(&cfg, decode_combine_kernel<8, 0>, P) != cudaSuccess) return WUSHKV_ECUDA;
     }
     return WUSHKV_OK;
 }
@@ -1196,10 +1128,7 @@ static int decode_attn_impl(const wushkv_cache* cache, int32_t batch, const int3
     P.qscal = reinterpret_cast<float*>(ws + pl.off_qscal);
     P.plan = reinterpret_cast<long long*>(ws + pl.off_plan);
     P.part = reinterpret_cast<float*>(ws + pl.off_part);
-    P.part_state = reinterpret_cast<int*>(ws + pl.off_state);
-    P.n_ctas = pl.n_ctas;
-    P.wait_limit = static_cast<int>(std::min<long long>(std::max<long long>(knobs().wait_limit, 0), 1 << 30));
-    P.drop_unit = knobs().drop_copy_unit;
+    P.n_warps = pl.n_warps;
     {   // upper bound of the packed bytes one step reads against the L2 size
         static int l2_bytes[64] = {};
         int dev = 0;

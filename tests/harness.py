@@ -13,11 +13,6 @@ from paper_2609_38121_b200 import workloads as W
 CODE_MISMATCH_MAX = 1e-4
 META_RTOL = 1e-3
 DECODE_TOL = 2e-3
-# Two decode calls on the same inputs: the main kernel hands work units to whichever warp is free, so which
-# units share a partial softmax state (and with it the reference that fp16(p * Delta_v) is rounded
-# against, and the fp32 summation order) varies from run to run, exactly as it does with the split
-# count.  Outputs of repeated or equivalent calls therefore agree to this fraction of |O|max, not bit for bit.
-REORDER_TOL = 5e-4
 
 
 def oracle_transforms(wl):
