@@ -11,7 +11,11 @@ whole step (append + decode), with every input already resident in HBM.  `roofli
 main kernel alone (CUDA events recorded around it by the library on the launching stream).  `e2e`
 repeats the steps through the host-buffer entry point (the step's new token and queries come from pinned
 host memory, the outputs go back to it, one synchronisation per step; the library reads and writes
-pinned buffers in place over the bus and falls back to staged copies otherwise).  `cpu_baseline` times the float64 oracle on a bounded slice.
+pinned buffers in place over the bus and falls back to staged copies otherwise).  `sustained` repeats the
+device-resident steps back to back for at least a second with the SM clock sampled throughout (the short
+regions run at the burst clock of a cool GPU); `value_sustained` is `value` over that leg.  For the prefill
+config (cfg4) `roofline` describes the chunk append kernel, the dominant kernel there.  `cpu_baseline` times
+the float64 oracle on a bounded slice, append and decode separately, with one thread and with all cores.
 With N > 1 every rank runs its own replica of the workload (the path has no cross-GPU exchange).
 """
 from __future__ import annotations
@@ -37,10 +41,10 @@ METRIC = "2-bit decode-attn cache GB/s (fraction of HBM peak) @32k ctx; append t
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 L2_BYTES = 126 * 2 ** 20
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode_main_kernel launch at the named
-# workload, from the ncu capture summarised under profiles/ (None until captured).
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel at the named workload,
+# from one ncu capture each (None where not captured).
 NCU_TRAFFIC_BYTES = {"cfg1": 310668544 + 3688960, "cfg2": 362961408 + 3549440,
-                     "cfg3": 76140032 + 3253760}      # profiles/decode_main_kernel_cfg1.md, _cfg2.md, _cfg3.md
+                     "cfg3": 76140032 + 3253760, "cfg4": None}
 
 
 def measured_hbm_peak():
@@ -294,7 +298,7 @@ class ClockSampler:
         else:
             self.t1 = time.monotonic_ns()
 
-    def stop(self):
+    def stop(self, bins=False):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is not None:
             self.proc.terminate()
@@ -328,6 +332,11 @@ class ClockSampler:
                 bits |= r[3]
             out.update(sm_mhz=statistics.median(r[1] for r in inside), sm_max_mhz=max(r[2] for r in inside),
                        reasons=sorted(n for b, n in self.REASONS.items() if bits & b), samples=len(inside))
+            if bins:                                         # share of the samples at each SM clock
+                hist = {}
+                for r in inside:
+                    hist[r[1]] = hist.get(r[1], 0) + 1
+                out["sm_mhz_bins"] = {str(k): round(v / len(inside), 4) for k, v in sorted(hist.items())}
         return out
 
 
@@ -360,13 +369,19 @@ class OracleSample:
         self.q = wl.queries(0, S - 1)[:G]
         self.extra = 0
 
-    def step(self):
-        O, c = self.O, self.cfg
+    def append_one(self):
         i = self.S - 1 + self.extra
         self.cache.append(self.K[i:i + 1], self.V[i:i + 1])
         self.extra += 1
+
+    def decode(self):
+        O, c = self.O, self.cfg
         arrs = self.cache.arrays()
         return O.decode_attn(self.q, self.TinvT, *arrs, self.cache.S, c["s_sink"], c["s_keep"], 1, 1.0 / np.sqrt(128))
+
+    def step(self):
+        self.append_one()
+        return self.decode()
 
     def bytes_per_step(self):
         c = self.cfg
@@ -399,6 +414,44 @@ def time_oracle(name, steps, warmup, budget_s=20.0):
             break
     sec = sum(times) / len(times)
     return smp, sec, len(times)
+
+
+def time_oracle_split(name, budget_s=16.0):
+    """Append (one token) and decode of the oracle sample timed separately, with the numerical libraries
+    limited to one thread and with all cores.  Returns (sample, {"append_ms": {...}, "decode_ms": {...}})."""
+    smp = OracleSample(name)
+    smp.step()                                           # warm-up of both halves
+    try:
+        from threadpoolctl import threadpool_limits
+    except Exception:
+        threadpool_limits = None
+    out = {"append_ms": {}, "decode_ms": {}, "steps": {}}
+    legs = [("1", 1), ("all", None)] if threadpool_limits else [("all", None)]
+    for label, limit in legs:
+        ctx = threadpool_limits(limits=limit) if (threadpool_limits and limit) else None
+        if ctx:
+            ctx.__enter__()
+        try:
+            ta, td, n = 0.0, 0.0, 0
+            t_all = time.perf_counter()
+            while n < 3 or (time.perf_counter() - t_all) < budget_s / len(legs):
+                t0 = time.perf_counter()
+                smp.append_one()
+                t1 = time.perf_counter()
+                smp.decode()
+                t2 = time.perf_counter()
+                ta += t1 - t0
+                td += t2 - t1
+                n += 1
+                if n >= 10 ** 6:
+                    break
+            out["append_ms"][label] = ta / n * 1e3
+            out["decode_ms"][label] = td / n * 1e3
+            out["steps"][label] = n
+        finally:
+            if ctx:
+                ctx.__exit__(None, None, None)
+    return smp, out
 
 
 # ------------------------------------------------------------------------------------------------
@@ -502,6 +555,42 @@ def run_ours(args, rank, world):
     bytes_step = float(np.mean([sess.decode_bytes(Wm + i + 1) for i in range(K)])) if not sess.chunk else float(cache_bytes)
     value = whole_job_value(bytes_step, ms_per_step, world)
 
+    # ---- region C (decode configs): at least a second of back-to-back steps, clocks sampled throughout and binned.
+    # The few-millisecond regions above run at the burst clock of a cool GPU; this is what a serving loop holds.
+    sustained = None
+    if not sess.chunk and not args.no_sustained:
+        sampler_c = ClockSampler(device_key(local)) if rank == 0 else None
+        n_avail = sess.step_K.shape[0]
+        done, reps = 0, 0
+        barrier()
+        if sampler_c:
+            sampler_c.mark()
+        c0, c1 = ev(), ev()
+        c0.record()
+        t_wall = time.perf_counter()
+        while True:
+            sess.rewind()
+            for _ in range(n_avail):
+                sess.step()
+            done += n_avail
+            reps += 1
+            if reps % 8 == 0:
+                torch.cuda.synchronize()
+                if time.perf_counter() - t_wall >= args.sustained_seconds:
+                    break
+        c1.record()
+        barrier()
+        if sampler_c:
+            sampler_c.mark()
+        sus_ms = max_over_ranks(c0.elapsed_time(c1) / done)
+        clk_c = sampler_c.stop(bins=True) if sampler_c else None
+        sess.rewind()
+        sess.step_index = 0
+        bytes_sus = float(np.mean([sess.decode_bytes(i + 1) for i in range(n_avail)]))
+        sustained = {"steps": done, "seconds": c0.elapsed_time(c1) * 1e-3, "ms_per_step": sus_ms,
+                     "value": whole_job_value(bytes_sus, sus_ms, world), "clocks": clk_c}
+        assert sess.cache.status() == 0
+
     # ---- end-to-end through the host-buffer entry point (decode steps only)
     e2e = None
     if not sess.chunk:
@@ -536,19 +625,42 @@ def run_ours(args, rank, world):
     if rank != 0:
         return
     peak, peak_kind = measured_hbm_peak()
-    kern_s = statistics.mean(kern_ms) * 1e-3
-    achieved = bytes_step / kern_s / 1e9
-    roofline = {"bound": "hbm", "kernel": "decode_main_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "kernel_ms": kern_s * 1e3, "kernel_ms_min": min(kern_ms), "algorithmic_bytes": bytes_step,
-                "traffic": NCU_TRAFFIC_BYTES.get(args.config)}
+    sm_mhz = (clocks or {}).get("sm_mhz")
+    if sess.chunk:
+        # prefill config: the dominant kernel is the chunk append (tensor-core transform + quantize + pack); its
+        # algorithmic bytes are the bf16 keys and values read plus the packed records written
+        per_tok = 2 * 128 * 2 + (72 if sess.cfg["bits"] == 2 else 136)
+        app_bytes = float(sess.append_tokens() * sess.wl.n_kv * per_tok)
+        app_s = statistics.mean(append_ms) * 1e-3
+        achieved = app_bytes / app_s / 1e9
+        roofline = {"bound": "hbm", "kernel": "append_chunk_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                    "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                    "kernel_ms": app_s * 1e3, "kernel_ms_min": min(append_ms), "algorithmic_bytes": app_bytes,
+                    "traffic": NCU_TRAFFIC_BYTES.get(args.config),
+                    "kernel_cycles": (app_s * 1e6 * sm_mhz) if sm_mhz else None,
+                    "note": "timed from the step's start to the event after wushkv_append (chunk kernel + length update); "
+                            "the kernel's busiest unit is the integer/logic pipe of the percentile selection, not HBM",
+                    "decode_main_kernel_ms": statistics.mean(kern_ms)}
+    else:
+        kern_s = statistics.mean(kern_ms) * 1e-3
+        achieved = bytes_step / kern_s / 1e9
+        roofline = {"bound": "hbm", "kernel": "decode_main_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                    "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                    "kernel_ms": kern_s * 1e3, "kernel_ms_min": min(kern_ms), "algorithmic_bytes": bytes_step,
+                    "traffic": NCU_TRAFFIC_BYTES.get(args.config),
+                    "kernel_cycles": (kern_s * 1e6 * sm_mhz) if sm_mhz else None}
     cpu = None
     if world == 1 and not args.no_cpu:
-        smp, sec, done = time_oracle(args.config, steps=10 ** 6, warmup=1, budget_s=args.cpu_seconds)
-        cpu = {"value": smp.bytes_per_step() / sec / 1e9, "unit": "GB/s", "cores": cpu_threads(), "kind": "oracle",
-               "ms_per_step": sec * 1e3, "steps": done,
+        smp, split = time_oracle_split(args.config, budget_s=args.cpu_seconds)
+        dec_all = split["decode_ms"]["all"]
+        cpu = {"value": smp.bytes_per_step() / (dec_all * 1e-3) / 1e9, "unit": "GB/s", "cores": cpu_threads(), "kind": "oracle",
+               "decode_ms": split["decode_ms"], "append_ms": split["append_ms"], "steps": split["steps"],
+               "append_tokens_per_s": {k: 1e3 / v for k, v in split["append_ms"].items()},
+               "host_cores": os.cpu_count(),
                "sample": (f"1 of {smp.wl.batch} sequences x 1 of {smp.wl.n_kv} KV heads ({smp.wl.G} query heads) at context "
-                          f"{smp.S}: append 1 token + decode, numpy float64")}
+                          f"{smp.S}, numpy float64; value = decode bytes of the slice / decode time with all cores; "
+                          f"append = one token (transform + both quantizers) of that head; keys '1' / 'all' = threads allowed "
+                          f"to the numerical libraries")}
     c = sess.cfg
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": Wm,
@@ -560,6 +672,7 @@ def run_ours(args, rank, world):
                    "l2": ("flushed between steps (256 MB write)" if need_flush else "cache read per step exceeds L2 (no flush)"),
                    "replicas": world},
         "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
+        "value_sustained": sustained["value"] if sustained else None, "sustained": sustained,
         "gpu_launches": K * sess.launches_per_step(), "clocks": clocks,
         "decode_tokens_per_s": world * sess.batch / (ms_per_step * 1e-3),
         "append_tokens_per_s": world * sess.append_tokens() / (statistics.mean(append_ms) * 1e-3),
@@ -578,6 +691,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--no-sustained", action="store_true", help="skip the second-long back-to-back leg")
+    ap.add_argument("--sustained-seconds", type=float, default=1.0)
     ap.add_argument("--verbose", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)

@@ -13,7 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libwushkv.so")
 
 OK, EINVAL, ENOTPD, ECUDA, ECAPACITY = 0, 1, 2, 3, 4
-DEV_PAGE_TABLE_FULL, DEV_BAD_PAGE_ID, DEV_BAD_SLOT, DEV_COPY_TIMEOUT = 1, 2, 4, 8
+DEV_PAGE_TABLE_FULL, DEV_BAD_PAGE_ID, DEV_BAD_SLOT, DEV_COPY_TIMEOUT, DEV_BAD_COUNT, DEV_VALUE_RANGE = 1, 2, 4, 8, 16, 32
 
 EXPORTS = (
     "wushkv_page_bytes", "wushkv_status_string", "wushkv_accumulate_gram", "wushkv_build_transforms",

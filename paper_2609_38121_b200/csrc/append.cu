@@ -43,6 +43,8 @@ struct AppendParams {
     const unsigned short* K_new;
     const unsigned short* V_new;
     ClipRule rule_k, rule_v;
+    int wait_limit;          // poll limit of the chunk kernel's MMA barrier wait (0: default, about two seconds)
+    int drop_mma_commit;     // testing aid: the first tile's MMAs are never committed to their barrier
 };
 
 __device__ __forceinline__ void cswap_desc(unsigned& a, unsigned& b) {
@@ -584,7 +586,8 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
                       "l"(bdesc + static_cast<unsigned long long>(ks * 2 * TC_LBO >> 4)), "r"(UMMA_IDESC), "r"(accumulate),
                       "r"(0u), "r"(0u), "r"(0u), "r"(0u) : "memory");
             }
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr_u32(mbar)) : "memory");
+            if (!(P.drop_mma_commit && tile == 0))       // (testing aid: without the commit the wait below runs into its limit)
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr_u32(mbar)) : "memory");
         }
         // ---- while the tensor core runs: values of this tile (no transform)
         if (KK_V > 0) {
@@ -665,14 +668,26 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
         // ---- wait for the MMAs (bounded), then tensor memory -> shared memory
         {
             bool done = false;
-            for (int it = 0; it < (1 << 20) && !done; ++it) {
+            const int mma_wait_limit = P.wait_limit > 0 ? P.wait_limit : (1 << 20);
+            for (int it = 0; it < mma_wait_limit && !done; ++it) {
                 unsigned ok;
                 asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
                              : "=r"(ok) : "r"(smem_addr_u32(mbar)), "r"(phase), "r"(2000u) : "memory");
                 done = ok != 0;
             }
             if (!__syncthreads_and(done ? 1 : 0)) {          // uniform decision for the whole CTA
-                if (tid == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_COPY_TIMEOUT);
+                if (tid == 0) {
+                    atomicOr(P.c.dev_status, WUSHKV_DEV_COPY_TIMEOUT);
+                    // commit whatever was issued once more and give it a bounded time, so that no MMA is still
+                    // writing tensor memory when it is released below
+                    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr_u32(mbar)) : "memory");
+                }
+                for (int it = 0; it < 512; ++it) {
+                    unsigned ok;
+                    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                                 : "=r"(ok) : "r"(smem_addr_u32(mbar)), "r"(phase), "r"(2000u) : "memory");
+                    if (ok) break;
+                }
                 failed = true;
                 break;
             }
@@ -858,6 +873,8 @@ extern "C" int wushkv_append(const wushkv_cache* cache, int32_t batch, const int
     P.K_new = K_new; P.V_new = V_new;
     P.rule_k = make_rule(cache->kappa_k);
     P.rule_v = make_rule(cache->kappa_v);
+    P.wait_limit = static_cast<int>(std::min<long long>(std::max<long long>(knobs().wait_limit, 0), 1 << 30));
+    P.drop_mma_commit = knobs().drop_chunk_mma;
     if (max_new == 1) {                 // decode-time append: one CTA per sequence, single launch
         const int threads = std::min(1024, P.c.n_kv * D);
         const size_t smem1 = static_cast<size_t>(2) * P.c.n_kv * D * sizeof(float);

@@ -81,6 +81,8 @@ struct DecodeParams {
     long long* plan;     // [batch+1]: exclusive prefix of work units per sequence (per KV head)
     float* part;         // [n_warps + batch*n_kv][G][PART_STRIDE]
     int n_warps;         // warps of the main kernel
+    int wait_limit;      // poll limit of the device-side barrier waits (0: default, about a second)
+    long long drop_unit; // testing aid: flattened index of a unit whose copy is never issued (-1: none)
     int q_early;         // 1: Q was final before the kernel ahead of the preparation kernel started
     int stream_pages;    // 1: the packed pages of a step cannot stay in L2 anyway: copy them with an evict-first hint
 };
@@ -315,8 +317,8 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
     return ok != 0;
 }
 // Bounded wait: false if the phase did not complete within the limit (about a second of sleeping polls).
-__device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity) {
-    for (int it = 0; it < (1 << 19); ++it)
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity, int limit) {
+    for (int it = 0; it < limit; ++it)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -661,6 +663,7 @@ __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_ke
     unsigned phase_bits = 0;            // parity of each stage's next completion
     unsigned bad_bits = 0;              // lane 0: stages whose unit could not be fetched
     bool timed_out = false;
+    const int wait_limit = P.wait_limit > 0 ? P.wait_limit : (1 << 19);      // polls that may sleep ~2 us each: about a second
 
     while (L < L1 && !timed_out) {
         // ================= round set-up: list the next segments of the slice =====================
@@ -689,6 +692,7 @@ __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_ke
         __syncwarp();
 
         // ================= producer: stages the units of this round, in order =====================
+        const long long round_L0 = L - round_units;      // flattened index of the round's first unit
         int p_seg = -1, p_u = 0, p_u1 = 0, p_qp = 0, p_head_off = 0, issued = 0;
         const int* p_ptab = nullptr;
         auto issue_next = [&](const int s) {            // whole warp; stages the round's next unit into ring slot s
@@ -717,7 +721,9 @@ __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_ke
                     } else {
                         bad_bits &= ~(1u << s);
                         mbar_expect_tx(bar, REC);
-                        if (P.stream_pages) bulk_copy_g2s_stream(dst, c.pages + page * page_row_bytes + p_head_off, REC, bar, stream_policy);
+                        if (P.drop_unit >= 0 && P.drop_unit == round_L0 + issued) {
+                            // testing aid: the copy is announced but never issued, so the wait for it runs into its limit
+                        } else if (P.stream_pages) bulk_copy_g2s_stream(dst, c.pages + page * page_row_bytes + p_head_off, REC, bar, stream_policy);
                         else bulk_copy_g2s(dst, c.pages + page * page_row_bytes + p_head_off, REC, bar);
                     }
                 }
@@ -774,7 +780,7 @@ __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_ke
             for (int u = sg.u0; u < u1; ++u, pos0 += PAGE_TOKENS) {
                 const int s = stage;
                 // a phase that one lane saw complete is complete for all: keep the decision warp-uniform
-                if (!__any_sync(FULL, mbar_wait_bounded(bar0 + 8 * s, (phase_bits >> s) & 1u))) { timed_out = true; break; }
+                if (!__any_sync(FULL, mbar_wait_bounded(bar0 + 8 * s, (phase_bits >> s) & 1u, wait_limit))) { timed_out = true; break; }
                 phase_bits ^= 1u << s;
 #if WUSHKV_ABL & 16
                 if (lane == 0 && g_timeline[((blockIdx.x * 16 + warp) & 8191) * 4 + 2] == 0) g_timeline[((blockIdx.x * 16 + warp) & 8191) * 4 + 2] = gtime();
@@ -927,8 +933,11 @@ __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_ke
     TL(3);
     if (timed_out) {
         if (lane == 0) atomicOr(c.dev_status, WUSHKV_DEV_COPY_TIMEOUT);
-        // give copies that may still be in flight a bounded time to land before the CTA's memory is released
-        for (int k = 0; k < 1000; ++k) __nanosleep(1000);
+        // Copies of this warp's other stages may still be in flight: wait for each (bounded; a stage with nothing
+        // pending simply runs the limit out) before the CTA's shared memory can be released.
+        const int drain_limit = min(wait_limit, 1 << 9);
+#pragma unroll
+        for (int s = 0; s < STAGES; ++s) mbar_wait_bounded(bar0 + 8 * s, (phase_bits >> s) & 1u, drain_limit);
     }
 }
 
@@ -1060,7 +1069,10 @@ static cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
 template <int BITS, int MODE>
 static int launch_decode(const DecodeParams& P, int n_ctas, cudaStream_t st) {
     constexpr int MAIN_WARPS = main_warps(BITS, MODE);
-    constexpr int STAGES = 2;      // per-warp ring depth
+#ifndef WUSHKV_STAGES_2BIT
+#define WUSHKV_STAGES_2BIT 2
+#endif
+    constexpr int STAGES = (BITS == 2 && MODE == 0) ? WUSHKV_STAGES_2BIT : 2;      // per-warp ring depth
     constexpr size_t SMEM = static_cast<size_t>(MAIN_WARPS) * STAGES * record_bytes(BITS) + MAIN_WARPS * STAGES * 8 +
                             MAIN_WARPS * MAX_SEGMENTS * sizeof(Segment);
     cudaLaunchAttribute pdl_attr[1];
@@ -1129,6 +1141,8 @@ static int decode_attn_impl(const wushkv_cache* cache, int32_t batch, const int3
     P.plan = reinterpret_cast<long long*>(ws + pl.off_plan);
     P.part = reinterpret_cast<float*>(ws + pl.off_part);
     P.n_warps = pl.n_warps;
+    P.wait_limit = static_cast<int>(std::min<long long>(std::max<long long>(knobs().wait_limit, 0), 1 << 30));
+    P.drop_unit = knobs().drop_copy_unit;
     {   // upper bound of the packed bytes one step reads against the L2 size
         static int l2_bytes[64] = {};
         int dev = 0;
