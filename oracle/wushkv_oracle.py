@@ -19,8 +19,9 @@ Conventions
 * Positions are 0-based; the paper's ``S_start < s <= S_quant`` (1-based) is
   the 0-based half-open range ``[S_start, S_quant)``.
 
-Parity pins (tests/test_oracle_*.py, tests/test_golden.py) cover every function below; none is
-"parity unpinned" against the mathematics.  What the paper itself does not fix
+Parity pins (tests/test_oracle_*.py, tests/test_golden.py) cover every function below (the error metric
+and the quantize-from-bf16 reading in test_oracle_attention.py, the QuEST quantizer in test_oracle_quest.py,
+chunk attention in test_oracle_chunk_attn.py); none is "parity unpinned" against the mathematics.  What the paper itself does not fix
 (quantile interpolation rule, tie rounding, storage precision of scale and
 zero, the boundary used at attention time) cannot be pinned to the paper; each
 such reading is listed where it is taken.
@@ -230,6 +231,82 @@ def quantize_rows(X, bits: int, kappa: float):
     return codes, delta, xmin
 
 
+# --------------------------------------------------------------------------
+# QuEST quantizer  (Section 4.3, Eq. 5; Lemma 1)
+# --------------------------------------------------------------------------
+
+
+def _gauss_grid_mse(alpha: float, bits: int) -> float:
+    """E[(Q_alpha(z) - z)^2] for z ~ N(0, 1) and the 2^b levels evenly spaced from -alpha to +alpha with
+    nearest-level rounding (the fixed-scale grid of Section 4.3), in closed form from the Gaussian
+    density and distribution function."""
+    import math
+    n = 1 << bits
+    step = 2.0 * alpha / (n - 1)
+    levels = [-alpha + k * step for k in range(n)]
+    edges = [-math.inf] + [0.5 * (levels[k] + levels[k + 1]) for k in range(n - 1)] + [math.inf]
+    pdf = lambda t: 0.0 if math.isinf(t) else math.exp(-0.5 * t * t) / math.sqrt(2.0 * math.pi)   # noqa: E731
+    cdf = lambda t: 0.5 * (1.0 + math.erf(t / math.sqrt(2.0)))                                      # noqa: E731
+    tpdf = lambda t: 0.0 if math.isinf(t) else t * pdf(t)                                            # noqa: E731
+    mse = 0.0
+    for k in range(n):
+        a, b, c = edges[k], edges[k + 1], levels[k]
+        m0 = cdf(b) - cdf(a)                    # integral of the density
+        m1 = pdf(a) - pdf(b)                    # integral of z * density
+        m2 = m0 + tpdf(a) - tpdf(b)             # integral of z^2 * density
+        mse += m2 - 2.0 * c * m1 + c * c * m0
+    return mse
+
+
+def quest_alpha(bits: int) -> float:
+    """alpha_b of Eq. 5: the endpoint of the 2^b-level evenly spaced grid that minimises the mean squared
+    error on a standard Gaussian (Section 4.3; the paper prints no value).  Golden-section search on the
+    closed-form error, which is unimodal in alpha on (0, 8)."""
+    lo, hi = 1e-3, 8.0
+    r = (np.sqrt(5.0) - 1.0) / 2.0
+    x1, x2 = hi - r * (hi - lo), lo + r * (hi - lo)
+    f1, f2 = _gauss_grid_mse(x1, bits), _gauss_grid_mse(x2, bits)
+    for _ in range(200):
+        if f1 < f2:
+            hi, x2, f2 = x2, x1, f1
+            x1 = hi - r * (hi - lo)
+            f1 = _gauss_grid_mse(x1, bits)
+        else:
+            lo, x1, f1 = x1, x2, f2
+            x2 = lo + r * (hi - lo)
+            f2 = _gauss_grid_mse(x2, bits)
+    return float(0.5 * (lo + hi))
+
+
+_QUEST_ALPHA = {}
+
+
+def quest_quantize(x, bits: int):
+    """Eq. 5 for one token-head group ``x`` ([d]): step Delta = 2 alpha_b (2^b - 1)^-1 d^-1/2 ||x||, bin index
+    floor(x / Delta) clamped to [-2^(b-1), 2^(b-1) - 1], reconstruction at the bin centre Delta (index + 1/2);
+    the zero group maps to zero.  Returns (codes uint8 [d] = index + 2^(b-1), delta, x_min) in the same
+    storage format as ``quantize``: x_hat = x_min + delta * code with x_min = -delta (2^b - 1) / 2.
+
+    Readings (storage, as for Eq. 6): the step is stored in fp16 and the bin indices are computed with the
+    stored step; the stored offset is the fp16 rounding of -delta (2^b - 1) / 2."""
+    x = np.asarray(x, dtype=np.float64)
+    d = x.shape[0]
+    if bits not in _QUEST_ALPHA:
+        _QUEST_ALPHA[bits] = quest_alpha(bits)
+    half = 1 << (bits - 1)
+    levels = (1 << bits) - 1
+    rms = np.sqrt(np.sum(x * x) / d)
+    delta = 2.0 * _QUEST_ALPHA[bits] / levels * rms
+    delta_s = float(round_fp16(delta))
+    xmin_s = float(round_fp16(-delta_s * levels / 2.0))
+    if delta_s > 0.0:
+        idx = np.clip(np.floor(x / delta_s), -half, half - 1)
+    else:
+        idx = np.full_like(x, -half)
+        xmin_s = 0.0                                 # Q(0) = 0: every code reconstructs to zero
+    return (idx + half).astype(np.uint8), delta_s, xmin_s
+
+
 def pack_codes(codes, bits: int) -> np.ndarray:
     """Reference bit packing (storage definition only): channel i occupies
     bits [bits*(i % per), bits*(i % per + 1)) of byte i // per, per = 8/bits.
@@ -293,7 +370,9 @@ class LayerCache:
     quantizing could change it, and that variant is available through
     ``quantize_from_bf16``)."""
 
-    def __init__(self, n_kv, d, bits, kappa_k, kappa_v, T, quantize_from_bf16=False):
+    def __init__(self, n_kv, d, bits, kappa_k, kappa_v, T, quantize_from_bf16=False, quantizer="affine"):
+        assert quantizer in ("affine", "quest")      # Eq. 6 (percentile-clipped affine) or Eq. 5 (QuEST; kappa unused)
+        self.quantizer = quantizer
         self.n_kv, self.d, self.bits = n_kv, d, bits
         self.kappa_k, self.kappa_v = kappa_k, kappa_v
         self.T = np.asarray(T, dtype=np.float64)
@@ -319,8 +398,12 @@ class LayerCache:
                 kp = key_transform(self.T[h], K_new[t, h][None, :])[0]
                 kb[h] = round_bf16(kp)
                 src = kb[h] if self.from_bf16 else kp
-                kc[h], km[h, 0], km[h, 1] = quantize(src, self.bits, self.kappa_k)
-                vc[h], vm[h, 0], vm[h, 1] = quantize(V_new[t, h], self.bits, self.kappa_v)
+                if self.quantizer == "quest":
+                    kc[h], km[h, 0], km[h, 1] = quest_quantize(src, self.bits)
+                    vc[h], vm[h, 0], vm[h, 1] = quest_quantize(V_new[t, h], self.bits)
+                else:
+                    kc[h], km[h, 0], km[h, 1] = quantize(src, self.bits, self.kappa_k)
+                    vc[h], vm[h, 0], vm[h, 1] = quantize(V_new[t, h], self.bits, self.kappa_v)
             self.k_codes.append(kc)
             self.v_codes.append(vc)
             self.k_meta.append(km)
@@ -386,6 +469,41 @@ def decode_attn(q, T_invT, k_codes, k_meta, v_codes, v_meta, k_bf16, v_bf16, S,
             j = h * G + g
             qc = query_compensation(T_invT[h], q[j][None, :])[0]
             out[j] = attention_one_query(qc, K_eff, V_eff, sm_scale)
+    return out
+
+
+def chunk_attn(q_chunk, T_invT, k_codes, k_meta, v_codes, v_meta, k_bf16, v_bf16, S, n_new,
+               s_sink, s_keep, s_flush, sm_scale, lag=0):
+    """Algorithm 2 lines 3 and 5 for a chunk of ``n_new`` > = 1 new positions of one sequence, AFTER they
+    were appended (line 4): the cache holds S positions, the chunk is positions [S - n_new, S).
+    q_chunk: [n_new][n_q][d] post-RoPE queries of the chunk (not compensated).  Chunk position i attends to
+    positions 0 .. S - n_new + i (causal inside the chunk).  Returns O [n_new][n_q][d].
+
+    Which copy each position is read from (Section 4.4; Section 5.3): positions of the chunk itself are
+    read from their bf16 copies ("each new chunk is first appended in full precision and is used to compute
+    its attention output"; the serving integration "updates cache storage before attention, while still
+    using the current ... prefill chunk's K/V in BF16"); every older position follows the window rule at
+    the cache length S - lag, as in ``effective_kv``.  Readings: lag = 0 is the serving behaviour;
+    lag = n_new is Algorithm 2 taken literally (the boundary is only moved in lines 7-8, after
+    attention)."""
+    q_chunk = np.asarray(q_chunk, dtype=np.float64)
+    n_new_, n_q, d = q_chunk.shape
+    assert n_new_ == n_new and 1 <= n_new <= S
+    n_kv = T_invT.shape[0]
+    G = n_q // n_kv
+    S0 = S - n_new
+    out = np.empty((n_new, n_q, d))
+    for h in range(n_kv):
+        K_eff, V_eff = effective_kv(k_codes[:, h], k_meta[:, h], v_codes[:, h], v_meta[:, h],
+                                    k_bf16[:, h], v_bf16[:, h], S, s_sink, s_keep, s_flush, lag)
+        K_eff[S0:S] = np.asarray(k_bf16[S0:S, h], dtype=np.float64)      # the chunk is read in full precision
+        V_eff[S0:S] = np.asarray(v_bf16[S0:S, h], dtype=np.float64)
+        for g in range(G):
+            j = h * G + g
+            qc = query_compensation(T_invT[h], q_chunk[:, j])            # [n_new][d]
+            for i in range(n_new):
+                n_vis = S0 + i + 1
+                out[i, j] = attention_one_query(qc[i], K_eff[:n_vis], V_eff[:n_vis], sm_scale)
     return out
 
 
