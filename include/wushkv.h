@@ -56,6 +56,10 @@ extern "C" {
 #define WUSHKV_ECUDA     3  /* a CUDA runtime call or kernel launch failed                    */
 #define WUSHKV_ECAPACITY 4  /* workspace / ring buffer / page table too small for the request */
 
+/* ---- quantizers (wushkv_cache.quantizer) ---------------------------------------------------- */
+#define WUSHKV_QUANTIZER_AFFINE 0
+#define WUSHKV_QUANTIZER_QUEST  1
+
 /* ---- bits OR-ed into *dev_status by kernels ---------------------------------------------- */
 #define WUSHKV_DEV_PAGE_TABLE_FULL 1  /* a position needs page index >= max_pages: token skipped */
 #define WUSHKV_DEV_BAD_PAGE_ID     2  /* page table entry outside [0, n_pages): access skipped   */
@@ -94,7 +98,10 @@ typedef struct wushkv_cache {
     int32_t n_slots, max_pages, ring_cap;
     float kappa_k, kappa_v; /* clipping quantiles of Eq. 6 for keys and values, in [0, 1] */
     float sm_scale;         /* 1 / tau of Eq. 2 */
-    int32_t reserved;
+    int32_t quantizer;      /* WUSHKV_QUANTIZER_AFFINE (0): percentile-clipped affine, Section 5.3 Eq. 6;
+                               WUSHKV_QUANTIZER_QUEST (1): QuEST, Section 4.3 Eq. 5 (step from the group's RMS, bin-centre
+                               reconstruction, Q(0) = 0; kappa_k / kappa_v unused).  Both are stored as (step, offset, codes)
+                               with x_hat = offset + step * code, so decode reads either. */
     int64_t n_pages;
     void* pages;
     const int32_t* page_table;
@@ -192,6 +199,28 @@ size_t wushkv_decode_workspace_bytes(const wushkv_cache* cache, int32_t batch, i
 int wushkv_decode_attn(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
                        int32_t max_seq_len, const uint16_t* Q, float* O,
                        void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Chunk (prefill) attention: Algorithm 2 line 3 (q' = T_K^{-T} q, k' = T_K k) and line 5 for a chunk of new
+ * positions, evaluated AFTER wushkv_append has stored the chunk (line 4).  Chunk position i of sequence b attends
+ * to cached positions 0 .. seq_len[b] - n_new[b] + i (causal inside the chunk).  The chunk's own keys and values
+ * are read in full precision (k' rounded to bf16, as the cache's window copies hold it; Section 4.4: "each new
+ * chunk is first appended in full precision and is used to compute its attention output"; Section 5.3), older
+ * positions by the window rule at length seq_len[b] - boundary_lag: sink and recent window from the bf16 buffers,
+ * the quantized middle from the packed pages.  boundary_lag = n_new reproduces Algorithm 2 literally (boundary
+ * moved after attention); ring_cap must then cover s_keep + s_flush - 1 + boundary_lag positions.
+ *   slot, cu_new, total_new, max_new, K_new, V_new: exactly what the preceding wushkv_append received.
+ *   seq_len (device): int32 [batch], the lengths AFTER that append.
+ *   Q_new (device): bf16 [total_new][n_q][d] post-Norm post-RoPE queries of the chunk, NOT compensated.
+ *   O (device, out): fp32 [total_new][n_q][d] in the folded value basis.
+ *   workspace (device): >= wushkv_prefill_workspace_bytes() bytes, 256-byte aligned, scratch.
+ * Both contractions run on tensor cores (fp16 operands, fp32 accumulation); q' is rounded to fp16.
+ */
+size_t wushkv_prefill_workspace_bytes(const wushkv_cache* cache, int32_t batch, int32_t total_new);
+int wushkv_prefill_attn(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
+                        const int32_t* cu_new, int32_t total_new, int32_t max_new,
+                        const uint16_t* K_new, const uint16_t* V_new, const uint16_t* Q_new, float* O,
+                        void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Read back the logical content of the packed cache (test / debugging aid): for positions

@@ -13,13 +13,14 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libwushkv.so")
 
 OK, EINVAL, ENOTPD, ECUDA, ECAPACITY = 0, 1, 2, 3, 4
+QUANTIZER_AFFINE, QUANTIZER_QUEST = 0, 1
 DEV_PAGE_TABLE_FULL, DEV_BAD_PAGE_ID, DEV_BAD_SLOT, DEV_COPY_TIMEOUT, DEV_BAD_COUNT, DEV_VALUE_RANGE = 1, 2, 4, 8, 16, 32
 
 EXPORTS = (
     "wushkv_page_bytes", "wushkv_status_string", "wushkv_accumulate_gram", "wushkv_build_transforms",
     "wushkv_append", "wushkv_decode_workspace_bytes", "wushkv_decode_attn", "wushkv_unpack_debug",
     "wushkv_decode_step", "wushkv_step_staging_bytes", "wushkv_decode_step_host", "wushkv_set_profile_events",
-    "wushkv_decode_attn_static", "wushkv_set_test_option",
+    "wushkv_decode_attn_static", "wushkv_set_test_option", "wushkv_prefill_workspace_bytes", "wushkv_prefill_attn",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -38,7 +39,7 @@ class wushkv_cache(C.Structure):
         ("boundary_lag", C.c_int32),
         ("n_slots", C.c_int32), ("max_pages", C.c_int32), ("ring_cap", C.c_int32),
         ("kappa_k", C.c_float), ("kappa_v", C.c_float), ("sm_scale", C.c_float),
-        ("reserved", C.c_int32),
+        ("quantizer", C.c_int32),
         ("n_pages", C.c_int64),
         ("pages", C.c_void_p), ("page_table", C.c_void_p), ("sink_kv", C.c_void_p), ("ring_kv", C.c_void_p),
         ("T_K", C.c_void_p), ("T_K_invT", C.c_void_p), ("dev_status", C.c_void_p),
@@ -86,6 +87,11 @@ def _load():
                                               C.c_void_p, C.c_void_p, C.c_void_p]
     lib.wushkv_set_profile_events.restype = C.c_int
     lib.wushkv_set_profile_events.argtypes = [C.c_void_p, C.c_void_p]
+    lib.wushkv_prefill_workspace_bytes.restype = C.c_size_t
+    lib.wushkv_prefill_workspace_bytes.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_int32]
+    lib.wushkv_prefill_attn.restype = C.c_int
+    lib.wushkv_prefill_attn.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                        C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
     lib.wushkv_set_test_option.restype = C.c_int
     lib.wushkv_set_test_option.argtypes = [C.c_char_p, C.c_longlong]
     return lib
@@ -202,6 +208,18 @@ def set_profile_events(start=None, stop=None):
     _check(lib.wushkv_set_profile_events(a, b), "wushkv_set_profile_events")
 
 
+def prefill_workspace_bytes(cache: wushkv_cache, batch: int, total_new: int) -> int:
+    return int(lib.wushkv_prefill_workspace_bytes(C.byref(cache), batch, total_new))
+
+
+def prefill_attn(cache: wushkv_cache, batch, slot, seq_len, cu_new, total_new, max_new, K_new, V_new, Q_new, O, workspace,
+                 workspace_bytes, stream=None):
+    """wushkv_prefill_attn: attention outputs of an appended chunk over the mixed cache (device tensors)."""
+    _check(lib.wushkv_prefill_attn(C.byref(cache), batch, _ptr(slot), _ptr(seq_len), _ptr(cu_new), total_new, max_new,
+                                   _ptr(K_new), _ptr(V_new), _ptr(Q_new), _ptr(O), _ptr(workspace), workspace_bytes,
+                                   _stream_ptr(stream)), "wushkv_prefill_attn")
+
+
 def set_test_option(name: str, value: int):
     """wushkv_set_test_option: process-wide testing aids (see the header for the names)."""
     _check(lib.wushkv_set_test_option(name.encode(), int(value)), "wushkv_set_test_option")
@@ -212,7 +230,7 @@ class PagedCache:
     descriptor.  Pure bookkeeping: page-table assignment and allocation, no arithmetic."""
 
     def __init__(self, n_q, n_kv, bits, n_slots, max_seq_len, s_sink, s_keep, s_flush, kappa_k, kappa_v,
-                 T_K, T_K_invT, sm_scale=None, boundary_lag=0, ring_cap=None, device="cuda", page_order=None):
+                 T_K, T_K_invT, sm_scale=None, boundary_lag=0, ring_cap=None, device="cuda", page_order=None, quantizer=0):
         import torch
         d, page_tokens = 128, 64
         self.torch = torch
@@ -234,7 +252,7 @@ class PagedCache:
             n_q=n_q, n_kv=n_kv, d=d, bits=bits, page_tokens=page_tokens, s_sink=s_sink, s_keep=s_keep, s_flush=s_flush,
             boundary_lag=boundary_lag, n_slots=n_slots, max_pages=self.max_pages, ring_cap=self.ring_cap,
             kappa_k=kappa_k, kappa_v=kappa_v, sm_scale=(sm_scale if sm_scale is not None else 1.0 / np.sqrt(d)),
-            reserved=0, n_pages=n_pages, pages=self.pages.data_ptr(), page_table=self.page_table.data_ptr(),
+            quantizer=quantizer, n_pages=n_pages, pages=self.pages.data_ptr(), page_table=self.page_table.data_ptr(),
             sink_kv=self.sink_kv.data_ptr(), ring_kv=self.ring_kv.data_ptr(), T_K=self.T_K.data_ptr(),
             T_K_invT=self.T_K_invT.data_ptr(), dev_status=self.dev_status.data_ptr())
 

@@ -29,9 +29,10 @@ constexpr int TT_STRIDE = 132;   // floats per row of the transposed transform i
 // a stored value step at or beyond this limit can saturate there, so the append flags it.
 constexpr float VALUE_STEP_LIMIT = 1024.f;
 
-struct ClipRule {     // rank rule of quantile_kappa(|x|) with linear interpolation
-    int rounds;       // extraction rounds: the last yields a[lo], the one before a[lo+1]
-    float frac;       // pos - lo
+struct ClipRule {     // how the step and offset of a group are chosen
+    int rounds;       // Eq. 6: extraction rounds of quantile_kappa(|x|): the last yields a[lo], the one before a[lo+1]
+    float frac;       // Eq. 6: pos - lo of the linear interpolation
+    float quest;      // Eq. 5 (QuEST) when > 0: 2 alpha_b / ((2^b - 1) sqrt(d)), the step per unit norm; 0 selects Eq. 6
 };
 
 struct AppendParams {
@@ -66,6 +67,24 @@ template <int BITS>
 __device__ __forceinline__ void quantize_vec(const float (&x)[4], ClipRule rule, int lane, int (&code)[4],
                                              __half& step_h, __half& xmin_h, int* value_status = nullptr) {
     constexpr int LEVELS = (1 << BITS) - 1;
+    if (rule.quest > 0.f) {
+        // Eq. 5: step from the group's norm, bin index floor(x / step) in [-2^(b-1), 2^(b-1) - 1], offset -step (2^b - 1) / 2
+        float ss = x[0] * x[0] + x[1] * x[1] + x[2] * x[2] + x[3] * x[3];
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(FULL, ss, o);
+        step_h = __float2half_rn(fminf(rule.quest * sqrtf(ss), 65504.f));
+        const float step_s = __half2float(step_h);
+        xmin_h = __float2half_rn(-0.5f * static_cast<float>(LEVELS) * step_s);
+        if (value_status != nullptr && step_s >= VALUE_STEP_LIMIT && lane == 0) atomicOr(value_status, WUSHKV_DEV_VALUE_RANGE);
+        const float inv = step_s > 0.f ? __frcp_rn(step_s) : 0.f;
+        constexpr float HALF = static_cast<float>(1 << (BITS - 1));
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float t = floorf(x[e] * inv) + HALF;
+            code[e] = step_s > 0.f ? static_cast<int>(fminf(fmaxf(t, 0.f), static_cast<float>(LEVELS))) : 0;
+        }
+        if (!(step_s > 0.f)) xmin_h = __float2half_rn(0.f);
+        return;
+    }
     // ---- the two order statistics of |x| around rank kappa*(d-1)
     unsigned u0 = __float_as_uint(x[0]) & 0x7fffffffu, u1 = __float_as_uint(x[1]) & 0x7fffffffu;
     unsigned u2 = __float_as_uint(x[2]) & 0x7fffffffu, u3 = __float_as_uint(x[3]) & 0x7fffffffu;
@@ -438,6 +457,25 @@ template <int BITS, int KK>
 __device__ __forceinline__ void quad_quantize(const float (&x)[32], ClipRule rule, int (&code)[32], __half& step_h, __half& xmin_h,
                                               int* value_status = nullptr, bool flag_lane = false) {
     constexpr int LEVELS = (1 << BITS) - 1;
+    if (rule.quest > 0.f) {                     // Eq. 5 (see quantize_vec)
+        float ss = 0.f;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) ss = fmaf(x[i], x[i], ss);
+        ss += __shfl_xor_sync(FULL, ss, 1);
+        ss += __shfl_xor_sync(FULL, ss, 2);
+        step_h = __float2half_rn(fminf(rule.quest * sqrtf(ss), 65504.f));
+        const float step_s = __half2float(step_h);
+        xmin_h = __float2half_rn(step_s > 0.f ? -0.5f * static_cast<float>(LEVELS) * step_s : 0.f);
+        if (value_status != nullptr && flag_lane && step_s >= VALUE_STEP_LIMIT) atomicOr(value_status, WUSHKV_DEV_VALUE_RANGE);
+        const float inv = step_s > 0.f ? __frcp_rn(step_s) : 0.f;
+        constexpr float HALF = static_cast<float>(1 << (BITS - 1));
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const float t = fminf(fmaxf(floorf(x[i] * inv) + HALF, 0.f), static_cast<float>(LEVELS));
+            code[i] = step_s > 0.f ? static_cast<int>(t) : 0;
+        }
+        return;
+    }
     unsigned top[KK];
 #pragma unroll
     for (int g0 = 0; g0 < 32; g0 += KK) {
@@ -844,11 +882,46 @@ __global__ void unpack_debug_kernel(CacheView c, int slot, int head, int which, 
     }
 }
 
+// alpha_b of Eq. 5: the endpoint of the evenly spaced 2^b-level grid with the least mean squared error on a
+// standard Gaussian (the paper prints no value).  Ternary search on the closed-form error.
+static double quest_grid_mse(double alpha, int bits) {
+    const int n = 1 << bits;
+    const double step = 2.0 * alpha / (n - 1), s2pi = std::sqrt(2.0 * 3.14159265358979323846);
+    auto pdf = [&](double t) { return std::isinf(t) ? 0.0 : std::exp(-0.5 * t * t) / s2pi; };
+    auto cdf = [&](double t) { return 0.5 * std::erfc(-t / std::sqrt(2.0)); };
+    double mse = 0.0;
+    for (int k = 0; k < n; ++k) {
+        const double c = -alpha + k * step;
+        const double a = k == 0 ? -INFINITY : c - 0.5 * step, b = k == n - 1 ? INFINITY : c + 0.5 * step;
+        const double m0 = cdf(b) - cdf(a), m1 = pdf(a) - pdf(b);
+        const double m2 = m0 + (std::isinf(a) ? 0.0 : a * pdf(a)) - (std::isinf(b) ? 0.0 : b * pdf(b));
+        mse += m2 - 2.0 * c * m1 + c * c * m0;
+    }
+    return mse;
+}
+static double quest_alpha(int bits) {
+    double lo = 1e-3, hi = 8.0;
+    for (int it = 0; it < 200; ++it) {
+        const double a = lo + (hi - lo) / 3.0, b = hi - (hi - lo) / 3.0;
+        if (quest_grid_mse(a, bits) < quest_grid_mse(b, bits)) hi = b; else lo = a;
+    }
+    return 0.5 * (lo + hi);
+}
+static ClipRule make_quest_rule(int bits) {
+    static double alpha[5] = {0, 0, 0, 0, 0};          // per bit width, computed on first use
+    if (alpha[bits] == 0) alpha[bits] = quest_alpha(bits);
+    ClipRule r;
+    r.rounds = 1; r.frac = 0.f;
+    r.quest = static_cast<float>(2.0 * alpha[bits] / (((1 << bits) - 1) * std::sqrt(static_cast<double>(D))));
+    return r;
+}
+
 static ClipRule make_rule(float kappa) {
     const double pos = static_cast<double>(kappa) * (D - 1);
     int lo = static_cast<int>(std::floor(pos));
     lo = std::min(std::max(lo, 0), D - 1);
     ClipRule r;
+    r.quest = 0.f;
     if (lo >= D - 1) { r.rounds = 1; r.frac = 0.f; }
     else { r.rounds = D - lo; r.frac = static_cast<float>(pos - lo); }
     return r;
@@ -871,8 +944,12 @@ extern "C" int wushkv_append(const wushkv_cache* cache, int32_t batch, const int
     P.batch = batch; P.total_new = total_new;
     P.slot = slot; P.seq_len = seq_len; P.cu_new = cu_new;
     P.K_new = K_new; P.V_new = V_new;
-    P.rule_k = make_rule(cache->kappa_k);
-    P.rule_v = make_rule(cache->kappa_v);
+    if (cache->quantizer == WUSHKV_QUANTIZER_QUEST) {
+        P.rule_k = P.rule_v = make_quest_rule(cache->bits);
+    } else {
+        P.rule_k = make_rule(cache->kappa_k);
+        P.rule_v = make_rule(cache->kappa_v);
+    }
     P.wait_limit = static_cast<int>(std::min<long long>(std::max<long long>(knobs().wait_limit, 0), 1 << 30));
     P.drop_mma_commit = knobs().drop_chunk_mma;
     if (max_new == 1) {                 // decode-time append: one CTA per sequence, single launch

@@ -22,6 +22,7 @@ inline int make_view(const wushkv_cache* c, CacheView& v) {
     if (c->n_slots <= 0 || c->max_pages <= 0 || c->n_pages <= 0) return WUSHKV_EINVAL;
     if (!(c->kappa_k >= 0.f && c->kappa_k <= 1.f) || !(c->kappa_v >= 0.f && c->kappa_v <= 1.f)) return WUSHKV_EINVAL;
     if (!(c->sm_scale > 0.f)) return WUSHKV_EINVAL;
+    if (c->quantizer != WUSHKV_QUANTIZER_AFFINE && c->quantizer != WUSHKV_QUANTIZER_QUEST) return WUSHKV_EINVAL;
     if (!c->pages || !c->page_table || !c->ring_kv || !c->T_K || !c->T_K_invT || !c->dev_status) return WUSHKV_EINVAL;
     if (c->s_sink > 0 && !c->sink_kv) return WUSHKV_EINVAL;
     if (!aligned(c->pages, 256) || !aligned(c->ring_kv, 16) || !aligned(c->sink_kv, 16) || !aligned(c->T_K, 16) ||

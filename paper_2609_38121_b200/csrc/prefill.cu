@@ -1,0 +1,469 @@
+// Chunk (prefill) attention over the mixed cache: Algorithm 2 line 3 (query / key transforms) and line 5 for a
+// chunk of S' > 1 new positions, after the chunk has been appended (line 4); Sections 4.4 and 5.3.
+//
+// Chunk position i of a sequence attends to every cached position up to itself.  Positions of the chunk are read
+// in full precision (k' = bf16(T_K k), v as given: "each new chunk is first appended in full precision and is used
+// to compute its attention output"), older positions follow the window rule: the sink and the recent window from
+// their bf16 copies, the quantized middle from the packed pages (x_hat = x_min + Delta * code, Eq. 6 / Eq. 5).
+//
+// Two launches:
+//   1. prefill_prep_kernel   q' = T_K^{-T} q and k' = T_K k of the chunk (fp32 accumulation), written as fp16
+//                            operands of the attention kernel (k' through its bf16 rounding, the value the cache's
+//                            window copies hold), the chunk's values as fp16, and sum_c q'_c per query row.
+//   2. prefill_attn_kernel   one CTA per (sequence, query head, 64 query rows): four warps, 16 rows each, stream
+//                            64-key tiles of the three sources through shared memory and keep an online softmax
+//                            (flash-attention recurrence) per row.  Both contractions run on mma.sync.m16n8k16
+//                            (fp16 operands, fp32 accumulation).  The affine part of the quantizer is factored out
+//                            of the contractions, per key j of a tile:
+//                                score_ij = Delta_k,j (q'_i . c_k,j) + x_min_k,j sum(q'_i)
+//                                o_i     += (p_ij Delta_v,j) c_v,j + (p_ij x_min_v,j) 1
+//                            so packed pages are staged as their integer codes (exact in fp16) and full-precision
+//                            rows with Delta = 1, x_min = 0.
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+
+#include "host_common.h"
+#include "layout.cuh"
+
+namespace wushkv {
+
+namespace {
+
+constexpr unsigned FULLM = 0xffffffffu;
+constexpr float LOG2E_F = 1.4426950408889634f;
+constexpr int BM = 64;                    // query rows per CTA
+constexpr int BN = 64;                    // keys per tile (= one packed page)
+constexpr int TILE_PITCH = D + 8;         // halves per staged row: 272 bytes, conflict-free for ldmatrix
+constexpr int PF_THREADS = 128;
+
+struct PrefillParams {
+    CacheView c;
+    int batch, total_new;
+    const int* slot;
+    const int* seq_len;                   // lengths after the chunk was appended
+    const int* cu_new;
+    const unsigned short* K_new;          // bf16 [total_new][n_kv][D] post-RoPE
+    const unsigned short* V_new;          // bf16 [total_new][n_kv][D]
+    const unsigned short* Q_new;          // bf16 [total_new][n_q][D] post-RoPE
+    float* O;                             // [total_new][n_q][D]
+    __half* KP;                           // [total_new][n_kv][D]  fp16(bf16(T_K k))
+    __half* VP;                           // [total_new][n_kv][D]  fp16(v)
+    __half* QP;                           // [total_new][n_q][D]   fp16(T_K^{-T} q)
+    float* qsum;                          // [total_new][n_q]      sum over channels of the fp16 q'
+    int tiles_per_seq;                    // ceil(max_new / BM)
+};
+
+__device__ __forceinline__ unsigned smem_addr(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void ldsm_x4(unsigned addr, unsigned& a, unsigned& b, unsigned& c, unsigned& d) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(unsigned addr, unsigned& a, unsigned& b, unsigned& c, unsigned& d) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "r"(addr));
+}
+__device__ __forceinline__ void hmma(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0, unsigned b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float fast_ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ unsigned pack_half2(float lo, float hi) {
+    unsigned d;
+    asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+// ------------------------------------------------------------------------------------------------
+// 1. transforms of the chunk (Algorithm 2 line 3)
+// ------------------------------------------------------------------------------------------------
+// One CTA per (tile of 32 tokens, head slot); head slots 0 .. n_kv-1 are the key heads, the rest the query heads.
+// The 128 x 128 transform sits transposed in shared memory; thread (channel i, token group) accumulates 16 tokens.
+constexpr int PREP_TOK = 32;
+__global__ void __launch_bounds__(256) prefill_prep_kernel(PrefillParams P) {
+    extern __shared__ __align__(16) float sm[];
+    float* Tt = sm;                               // [D][D + 1]: Tt[j][i] = T[i][j]
+    float* X = sm + D * (D + 1);                  // [PREP_TOK][D]
+    const int hs = blockIdx.y, tok0 = blockIdx.x * PREP_TOK;
+    const bool is_key = hs < P.c.n_kv;
+    const int head = is_key ? hs : hs - P.c.n_kv;
+    const int kvh = is_key ? head : head / P.c.G;
+    const float* T = (is_key ? P.c.T_K : P.c.T_K_invT) + static_cast<long long>(kvh) * D * D;
+    for (int idx = threadIdx.x; idx < D * D; idx += 256) {
+        const int i = idx >> 7, j = idx & 127;
+        Tt[j * (D + 1) + i] = __ldg(T + idx);
+    }
+    const int n_heads = is_key ? P.c.n_kv : P.c.n_q;
+    const unsigned short* src = is_key ? P.K_new : P.Q_new;
+    for (int idx = threadIdx.x; idx < PREP_TOK * D; idx += 256) {
+        const int tk = idx >> 7, ch = idx & 127;
+        const int tok = tok0 + tk;
+        X[idx] = tok < P.total_new ? bf16_bits_to_float(__ldg(src + (static_cast<long long>(tok) * n_heads + head) * D + ch)) : 0.f;
+    }
+    __syncthreads();
+    const int i = threadIdx.x & 127, tg = threadIdx.x >> 7;          // output channel, token group (16 tokens each)
+    float acc[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) acc[k] = 0.f;
+    for (int j = 0; j < D; ++j) {
+        const float tji = Tt[j * (D + 1) + i];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) acc[k] = fmaf(tji, X[(tg * 16 + k) * D + j], acc[k]);
+    }
+    __syncthreads();                                                  // X is reused for the row sums
+    float* rowsum = X;                                                // [PREP_TOK][4 warps of this token group]
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+        const int tok = tok0 + tg * 16 + k;
+        float val = acc[k];
+        __half hv;
+        if (is_key) hv = __float2half_rn(bf16_bits_to_float(float_to_bf16_bits(val)));   // the cache holds bf16(k')
+        else hv = __float2half_rn(val);
+        if (tok < P.total_new) {
+            __half* dst = (is_key ? P.KP : P.QP) + (static_cast<long long>(tok) * n_heads + head) * D + i;
+            *dst = hv;
+        }
+        if (!is_key) {                                                // sum of the rounded q' over the 128 channels
+            float s = __half2float(hv);
+            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(FULLM, s, o);
+            if ((threadIdx.x & 31) == 0) rowsum[(tg * 16 + k) * 4 + ((threadIdx.x & 127) >> 5)] = s;
+        }
+    }
+    if (is_key) {                                                     // the chunk's values as fp16 (no transform)
+        for (int idx = threadIdx.x; idx < PREP_TOK * D; idx += 256) {
+            const int tk = idx >> 7, ch = idx & 127, tok = tok0 + tk;
+            if (tok < P.total_new) {
+                const long long off = (static_cast<long long>(tok) * P.c.n_kv + head) * D + ch;
+                P.VP[off] = __float2half_rn(bf16_bits_to_float(__ldg(P.V_new + off)));
+            }
+        }
+        return;
+    }
+    __syncthreads();
+    if (threadIdx.x < PREP_TOK) {
+        const int tok = tok0 + threadIdx.x;
+        if (tok < P.total_new)
+            P.qsum[static_cast<long long>(tok) * P.c.n_q + head] =
+                rowsum[threadIdx.x * 4] + rowsum[threadIdx.x * 4 + 1] + rowsum[threadIdx.x * 4 + 2] + rowsum[threadIdx.x * 4 + 3];
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// 2. attention
+// ------------------------------------------------------------------------------------------------
+struct TileSmem {
+    __half K[BN][TILE_PITCH];
+    __half V[BN][TILE_PITCH];
+    float4 meta[BN];          // per key: Delta_k, x_min_k, Delta_v, x_min_v (1, 0, 1, 0 for a full-precision row)
+    int pos[BN];              // cached position of the key, -1: not a key of this tile
+    unsigned char raw[8704];  // one packed record
+};
+
+template <int BITS>
+__global__ void __launch_bounds__(PF_THREADS) prefill_attn_kernel(PrefillParams P) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    TileSmem& ts = *reinterpret_cast<TileSmem*>(smem_raw);
+    const CacheView& c = P.c;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const int qt = blockIdx.x % P.tiles_per_seq, b = blockIdx.x / P.tiles_per_seq;
+    const int jq = blockIdx.y, h = jq / c.G;
+    const int first = __ldg(P.cu_new + b), n_new = __ldg(P.cu_new + b + 1) - first;
+    if (qt * BM >= n_new) return;
+    const int S = __ldg(P.seq_len + b), sl = __ldg(P.slot + b);
+    if (sl < 0 || sl >= c.n_slots || S < n_new) {
+        if (tid == 0) atomicOr(c.dev_status, WUSHKV_DEV_BAD_SLOT);
+        return;
+    }
+    const int S0 = S - n_new;                                   // first position of the chunk
+    // ---- where older positions are read from (window rule at length S - lag, Section 4.4)
+    const int nq = n_quantized(S - c.lag, c.s_sink, c.s_keep, c.s_flush);
+    const int q_lo = c.s_sink, q_hi = min(c.s_sink + nq, S0);   // quantized positions below the chunk
+    const int a_hi = min(c.s_sink, S0);                         // sink positions below the chunk: [0, a_hi)
+    const int c_lo = max(q_hi, a_hi);                           // recent-window positions below the chunk: [c_lo, S0)
+    const int n_old_fp = a_hi + max(S0 - c_lo, 0);              // full-precision old positions, as one index space
+    const float k2 = c.sm_scale * LOG2E_F;
+
+    // ---- this warp's 16 query rows as A fragments (kept in registers), and their channel sums
+    const int row0 = qt * BM + warp * 16;                       // chunk-relative row of fragment row 0
+    const int ra = min(row0 + g, n_new - 1), rb = min(row0 + g + 8, n_new - 1);
+    unsigned qa[8][4];
+    {
+        const __half* q0 = P.QP + (static_cast<long long>(first + ra) * c.n_q + jq) * D;
+        const __half* q1 = P.QP + (static_cast<long long>(first + rb) * c.n_q + jq) * D;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            qa[ks][0] = __ldcg(reinterpret_cast<const unsigned*>(q0 + 16 * ks + 2 * t));
+            qa[ks][1] = __ldcg(reinterpret_cast<const unsigned*>(q1 + 16 * ks + 2 * t));
+            qa[ks][2] = __ldcg(reinterpret_cast<const unsigned*>(q0 + 16 * ks + 8 + 2 * t));
+            qa[ks][3] = __ldcg(reinterpret_cast<const unsigned*>(q1 + 16 * ks + 8 + 2 * t));
+        }
+    }
+    const float qs_a = __ldcg(P.qsum + static_cast<long long>(first + ra) * c.n_q + jq);
+    const float qs_b = __ldcg(P.qsum + static_cast<long long>(first + rb) * c.n_q + jq);
+    const int pos_a = S0 + row0 + g, pos_b = pos_a + 8;         // cached positions of the two rows (causal limit)
+
+    float o[16][4];
+#pragma unroll
+    for (int nb = 0; nb < 16; ++nb) o[nb][0] = o[nb][1] = o[nb][2] = o[nb][3] = 0.f;
+    float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f, z_a = 0.f, z_b = 0.f;
+
+    // One staged tile: scores, online softmax, value reduction.
+    auto consume = [&]() {
+        float s[8][4];
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb) s[nb][0] = s[nb][1] = s[nb][2] = s[nb][3] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+#pragma unroll
+            for (int nb2 = 0; nb2 < 4; ++nb2) {                 // two key blocks of 8 per ldmatrix.x4
+                unsigned b0, b1, b2, b3;
+                ldsm_x4(smem_addr(&ts.K[16 * nb2 + 8 * (lane >> 4) + (lane & 7)][16 * ks + 8 * ((lane >> 3) & 1)]), b0, b1, b2, b3);
+                hmma(s[2 * nb2], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
+                hmma(s[2 * nb2 + 1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b2, b3);
+            }
+        }
+        // affine part, masks, row maxima (log2 domain)
+        float mx_a = -INFINITY, mx_b = -INFINITY;
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int col = 8 * nb + 2 * t + e;
+                const float4 mt = ts.meta[col];
+                const int kp = ts.pos[col];
+                const float va = (kp >= 0 && kp <= pos_a) ? k2 * fmaf(mt.y, qs_a, mt.x * s[nb][e]) : -INFINITY;
+                const float vb = (kp >= 0 && kp <= pos_b) ? k2 * fmaf(mt.y, qs_b, mt.x * s[nb][2 + e]) : -INFINITY;
+                s[nb][e] = va; s[nb][2 + e] = vb;
+                mx_a = fmaxf(mx_a, va); mx_b = fmaxf(mx_b, vb);
+            }
+        }
+        mx_a = fmaxf(mx_a, __shfl_xor_sync(FULLM, mx_a, 1)); mx_a = fmaxf(mx_a, __shfl_xor_sync(FULLM, mx_a, 2));
+        mx_b = fmaxf(mx_b, __shfl_xor_sync(FULLM, mx_b, 1)); mx_b = fmaxf(mx_b, __shfl_xor_sync(FULLM, mx_b, 2));
+        const float mn_a = fmaxf(m_a, mx_a), mn_b = fmaxf(m_b, mx_b);
+        const float ref_a = mn_a == -INFINITY ? 0.f : mn_a, ref_b = mn_b == -INFINITY ? 0.f : mn_b;
+        const float al_a = fast_ex2(m_a - ref_a), al_b = fast_ex2(m_b - ref_b);     // old reference -inf: state is zero, factor 0
+        m_a = mn_a; m_b = mn_b;
+        l_a *= al_a; z_a *= al_a; l_b *= al_b; z_b *= al_b;
+#pragma unroll
+        for (int nb = 0; nb < 16; ++nb) { o[nb][0] *= al_a; o[nb][1] *= al_a; o[nb][2] *= al_b; o[nb][3] *= al_b; }
+        unsigned pa[4][4];                                      // A fragments of (p Delta_v) for the four 16-key steps
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb) {
+            float w[4];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const float4 mt = ts.meta[8 * nb + 2 * t + e];
+                const float p0 = fast_ex2(s[nb][e] - ref_a), p1 = fast_ex2(s[nb][2 + e] - ref_b);
+                l_a += p0; l_b += p1;
+                z_a = fmaf(p0, mt.w, z_a); z_b = fmaf(p1, mt.w, z_b);
+                w[e] = p0 * mt.z; w[2 + e] = p1 * mt.z;
+            }
+            pa[nb >> 1][(nb & 1) * 2 + 0] = pack_half2(w[0], w[1]);
+            pa[nb >> 1][(nb & 1) * 2 + 1] = pack_half2(w[2], w[3]);
+        }
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb) {
+#pragma unroll
+            for (int nb2 = 0; nb2 < 8; ++nb2) {                 // two channel blocks of 8 per ldmatrix.x4.trans
+                unsigned b0, b1, b2, b3;
+                ldsm_x4_t(smem_addr(&ts.V[16 * kb + 8 * ((lane >> 3) & 1) + (lane & 7)][16 * nb2 + 8 * (lane >> 4)]), b0, b1, b2, b3);
+                hmma(o[2 * nb2], pa[kb][0], pa[kb][1], pa[kb][2], pa[kb][3], b0, b1);
+                hmma(o[2 * nb2 + 1], pa[kb][0], pa[kb][1], pa[kb][2], pa[kb][3], b2, b3);
+            }
+        }
+    };
+
+    // ---- (1) full-precision old positions: sink [0, a_hi) and recent window [c_lo, S0), bf16 rows
+    for (int base = 0; base < n_old_fp; base += BN) {
+        __syncthreads();
+        for (int item = tid; item < BN * 16; item += PF_THREADS) {          // 16-byte pieces: 8 channels of one row
+            const int r = item >> 4, piece = item & 15, idx = base + r;
+            uint4 kh = make_uint4(0, 0, 0, 0), vh = kh;
+            if (idx < n_old_fp) {
+                const long long plane = (static_cast<long long>(sl) * c.n_kv + h) * 2;
+                const unsigned short *ksrc, *vsrc;
+                if (idx < a_hi) {
+                    ksrc = c.sink_kv + (plane * c.s_sink + idx) * D;
+                    vsrc = c.sink_kv + ((plane + 1) * c.s_sink + idx) * D;
+                } else {
+                    const int p = c_lo + (idx - a_hi);
+                    ksrc = c.ring_kv + (plane * c.ring_cap + p % c.ring_cap) * D;
+                    vsrc = c.ring_kv + ((plane + 1) * c.ring_cap + p % c.ring_cap) * D;
+                }
+                const uint4 kb16 = *reinterpret_cast<const uint4*>(ksrc + 8 * piece), vb16 = *reinterpret_cast<const uint4*>(vsrc + 8 * piece);
+                const unsigned kw[4] = {kb16.x, kb16.y, kb16.z, kb16.w}, vw[4] = {vb16.x, vb16.y, vb16.z, vb16.w};
+                unsigned ko[4], vo[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    ko[e] = pack_half2(bf16_bits_to_float(kw[e] & 0xffff), bf16_bits_to_float(kw[e] >> 16));
+                    vo[e] = pack_half2(bf16_bits_to_float(vw[e] & 0xffff), bf16_bits_to_float(vw[e] >> 16));
+                }
+                kh = make_uint4(ko[0], ko[1], ko[2], ko[3]); vh = make_uint4(vo[0], vo[1], vo[2], vo[3]);
+            }
+            *reinterpret_cast<uint4*>(&ts.K[r][8 * piece]) = kh;
+            *reinterpret_cast<uint4*>(&ts.V[r][8 * piece]) = vh;
+            if (piece == 0) {
+                ts.meta[r] = make_float4(1.f, 0.f, 1.f, 0.f);
+                ts.pos[r] = idx < n_old_fp ? (idx < a_hi ? idx : c_lo + (idx - a_hi)) : -1;
+            }
+        }
+        __syncthreads();
+        consume();
+    }
+
+    // ---- (2) quantized positions below the chunk: one packed page per tile, staged as integer codes
+    if (q_hi > q_lo) {
+        constexpr int REC = record_bytes(BITS);
+        const int page_first = q_lo / PAGE_TOKENS, page_last = (q_hi - 1) / PAGE_TOKENS;
+        for (int pg = page_first; pg <= page_last; ++pg) {
+            __syncthreads();
+            int page = -1;
+            if (pg < c.max_pages) page = __ldg(c.page_table + static_cast<long long>(sl) * c.max_pages + pg);
+            const bool page_ok = page >= 0 && page < c.n_pages;
+            if (!page_ok && tid == 0) atomicOr(c.dev_status, pg < c.max_pages ? WUSHKV_DEV_BAD_PAGE_ID : WUSHKV_DEV_PAGE_TABLE_FULL);
+            if (page_ok) {
+                const uint4* src = reinterpret_cast<const uint4*>(c.pages + (static_cast<long long>(page) * c.n_kv + h) * REC);
+                for (int k = tid; k < REC / 16; k += PF_THREADS) reinterpret_cast<uint4*>(ts.raw)[k] = __ldg(src + k);
+            }
+            __syncthreads();
+            // thread -> token r = tid & 63, channels (tid >> 6) * 64 .. + 63, two at a time
+            {
+                const int r = tid & 63, ch0 = (tid >> 6) * 64;
+                const int pos = pg * PAGE_TOKENS + r;
+                const bool live = page_ok && pos >= q_lo && pos < q_hi;
+                constexpr unsigned MASK = (1u << BITS) - 1u;
+                for (int ch = ch0; ch < ch0 + 64; ch += 2) {
+                    float k0 = 0.f, k1 = 0.f, v0 = 0.f, v1 = 0.f;
+                    if (live) {
+                        int off, bit;
+                        k_code_location(BITS, r, ch, off, bit);     k0 = static_cast<float>((ts.raw[off + (bit >> 3)] >> (bit & 7)) & MASK);
+                        k_code_location(BITS, r, ch + 1, off, bit); k1 = static_cast<float>((ts.raw[off + (bit >> 3)] >> (bit & 7)) & MASK);
+                        v_code_location(BITS, r, ch, off, bit);     v0 = static_cast<float>((ts.raw[off + (bit >> 3)] >> (bit & 7)) & MASK);
+                        v_code_location(BITS, r, ch + 1, off, bit); v1 = static_cast<float>((ts.raw[off + (bit >> 3)] >> (bit & 7)) & MASK);
+                    }
+                    *reinterpret_cast<unsigned*>(&ts.K[r][ch]) = pack_half2(k0, k1);
+                    *reinterpret_cast<unsigned*>(&ts.V[r][ch]) = pack_half2(v0, v1);
+                }
+                if (ch0 == 0) {
+                    float4 mt = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (live) {
+                        const __half* mh = reinterpret_cast<const __half*>(ts.raw + meta_location(BITS, r));
+                        mt = make_float4(__half2float(mh[0]), __half2float(mh[1]), __half2float(mh[2]), __half2float(mh[3]));
+                    }
+                    ts.meta[r] = mt;
+                    ts.pos[r] = live ? pos : -1;
+                }
+            }
+            __syncthreads();
+            consume();
+        }
+    }
+
+    // ---- (3) the chunk itself, causal: tiles 0 .. qt of its own rows (fp16 copies made by the preparation kernel)
+    for (int kt = 0; kt <= qt; ++kt) {
+        __syncthreads();
+        for (int item = tid; item < BN * 16; item += PF_THREADS) {
+            const int r = item >> 4, piece = item & 15, row = kt * BN + r;
+            uint4 kh = make_uint4(0, 0, 0, 0), vh = kh;
+            if (row < n_new) {
+                const long long off = (static_cast<long long>(first + row) * c.n_kv + h) * D + 8 * piece;
+                kh = __ldcg(reinterpret_cast<const uint4*>(P.KP + off));
+                vh = __ldcg(reinterpret_cast<const uint4*>(P.VP + off));
+            }
+            *reinterpret_cast<uint4*>(&ts.K[r][8 * piece]) = kh;
+            *reinterpret_cast<uint4*>(&ts.V[r][8 * piece]) = vh;
+            if (piece == 0) {
+                ts.meta[r] = make_float4(1.f, 0.f, 1.f, 0.f);
+                ts.pos[r] = row < n_new ? S0 + row : -1;
+            }
+        }
+        __syncthreads();
+        consume();
+    }
+
+    // ---- output: o_i = (sum_j p_ij v_hat_j) / sum_j p_ij
+    l_a += __shfl_xor_sync(FULLM, l_a, 1); l_a += __shfl_xor_sync(FULLM, l_a, 2);
+    l_b += __shfl_xor_sync(FULLM, l_b, 1); l_b += __shfl_xor_sync(FULLM, l_b, 2);
+    z_a += __shfl_xor_sync(FULLM, z_a, 1); z_a += __shfl_xor_sync(FULLM, z_a, 2);
+    z_b += __shfl_xor_sync(FULLM, z_b, 1); z_b += __shfl_xor_sync(FULLM, z_b, 2);
+    const float inv_a = l_a > 0.f ? 1.f / l_a : 0.f, inv_b = l_b > 0.f ? 1.f / l_b : 0.f;
+    if (row0 + g < n_new) {
+        float* dst = P.O + (static_cast<long long>(first + row0 + g) * c.n_q + jq) * D;
+#pragma unroll
+        for (int nb = 0; nb < 16; ++nb)
+            *reinterpret_cast<float2*>(dst + 8 * nb + 2 * t) = make_float2((o[nb][0] + z_a) * inv_a, (o[nb][1] + z_a) * inv_a);
+    }
+    if (row0 + g + 8 < n_new) {
+        float* dst = P.O + (static_cast<long long>(first + row0 + g + 8) * c.n_q + jq) * D;
+#pragma unroll
+        for (int nb = 0; nb < 16; ++nb)
+            *reinterpret_cast<float2*>(dst + 8 * nb + 2 * t) = make_float2((o[nb][2] + z_b) * inv_b, (o[nb][3] + z_b) * inv_b);
+    }
+}
+
+size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+
+struct PrefillPlan { size_t off_kp, off_vp, off_qp, off_qsum, total; };
+bool make_prefill_plan(const CacheView& c, int total_new, PrefillPlan& pl) {
+    if (total_new <= 0) return false;
+    size_t off = 0;
+    pl.off_kp = off;   off = align256(off + static_cast<size_t>(total_new) * c.n_kv * D * sizeof(__half));
+    pl.off_vp = off;   off = align256(off + static_cast<size_t>(total_new) * c.n_kv * D * sizeof(__half));
+    pl.off_qp = off;   off = align256(off + static_cast<size_t>(total_new) * c.n_q * D * sizeof(__half));
+    pl.off_qsum = off; off = align256(off + static_cast<size_t>(total_new) * c.n_q * sizeof(float));
+    pl.total = off;
+    return true;
+}
+
+}  // namespace
+}  // namespace wushkv
+
+using namespace wushkv;
+
+extern "C" size_t wushkv_prefill_workspace_bytes(const wushkv_cache* cache, int32_t batch, int32_t total_new) {
+    CacheView v;
+    if (make_view(cache, v) != WUSHKV_OK || batch <= 0) return 0;
+    PrefillPlan pl;
+    if (!make_prefill_plan(v, total_new, pl)) return 0;
+    return pl.total;
+}
+
+extern "C" int wushkv_prefill_attn(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
+                                   const int32_t* cu_new, int32_t total_new, int32_t max_new,
+                                   const uint16_t* K_new, const uint16_t* V_new, const uint16_t* Q_new, float* O,
+                                   void* workspace, size_t workspace_bytes, void* stream) {
+    PrefillParams P;
+    const int rc = make_view(cache, P.c);
+    if (rc != WUSHKV_OK) return rc;
+    if (batch <= 0 || !slot || !seq_len || !cu_new || total_new < 0 || max_new < 0 || max_new > total_new) return WUSHKV_EINVAL;
+    if (total_new == 0) return WUSHKV_OK;
+    if (!K_new || !V_new || !Q_new || !O || !workspace || !aligned(K_new, 16) || !aligned(V_new, 16) || !aligned(Q_new, 16) ||
+        !aligned(O, 16) || !aligned(workspace, 256))
+        return WUSHKV_EINVAL;
+    PrefillPlan pl;
+    if (!make_prefill_plan(P.c, total_new, pl)) return WUSHKV_EINVAL;
+    if (workspace_bytes < pl.total) return WUSHKV_ECAPACITY;
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
+    P.batch = batch; P.total_new = total_new; P.slot = slot; P.seq_len = seq_len; P.cu_new = cu_new;
+    P.K_new = K_new; P.V_new = V_new; P.Q_new = Q_new; P.O = O;
+    P.KP = reinterpret_cast<__half*>(ws + pl.off_kp);
+    P.VP = reinterpret_cast<__half*>(ws + pl.off_vp);
+    P.QP = reinterpret_cast<__half*>(ws + pl.off_qp);
+    P.qsum = reinterpret_cast<float*>(ws + pl.off_qsum);
+    P.tiles_per_seq = (max_new + BM - 1) / BM;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t smem_prep = (static_cast<size_t>(D) * (D + 1) + PREP_TOK * D) * sizeof(float);
+    if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(prefill_prep_kernel), static_cast<int>(smem_prep))) return WUSHKV_ECUDA;
+    prefill_prep_kernel<<<dim3((total_new + PREP_TOK - 1) / PREP_TOK, P.c.n_kv + P.c.n_q), 256, smem_prep, st>>>(P);
+    if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
+    const dim3 grid(static_cast<unsigned>(batch) * P.tiles_per_seq, P.c.n_q);
+    const size_t smem_attn = sizeof(TileSmem);
+    if (P.c.bits == 2) {
+        if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(prefill_attn_kernel<2>), static_cast<int>(smem_attn))) return WUSHKV_ECUDA;
+        prefill_attn_kernel<2><<<grid, PF_THREADS, smem_attn, st>>>(P);
+    } else {
+        if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(prefill_attn_kernel<4>), static_cast<int>(smem_attn))) return WUSHKV_ECUDA;
+        prefill_attn_kernel<4><<<grid, PF_THREADS, smem_attn, st>>>(P);
+    }
+    return cudaGetLastError() == cudaSuccess ? WUSHKV_OK : WUSHKV_ECUDA;
+}

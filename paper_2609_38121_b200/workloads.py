@@ -192,6 +192,12 @@ class LayerWorkload:
             yield pos0 + done, K, bf16_round_f32(V)
             done += n
 
+    def chunk_queries(self, b, positions):
+        """Queries of sequence ``b`` at several positions (a prefill chunk): [n][n_q][d] bf16-valued float32."""
+        rng = np.random.default_rng(np.random.SeedSequence(
+            entropy=self._ss_qry.entropy, spawn_key=self._ss_qry.spawn_key + (int(b), 1)))
+        return self._queries(rng, np.asarray(positions))
+
     def queries(self, b, position):
         """The decode-step query of sequence ``b`` at ``position``: [n_q][d] bf16-valued float32."""
         rng = np.random.default_rng(np.random.SeedSequence(

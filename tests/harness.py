@@ -36,7 +36,7 @@ class Layer:
     per-step new-token counts per sequence (list of lists) or None for prefill(S-1) + decode(1)."""
 
     def __init__(self, wl, lengths, bits, s_sink, s_keep, s_flush, lag=0, kappa_k=W.KAPPA_K, kappa_v=W.KAPPA_V,
-                 page_shuffle_seed=None, max_seq_len=None, ring_cap=None):
+                 page_shuffle_seed=None, max_seq_len=None, ring_cap=None, quantizer="affine"):
         import torch
         from paper_2609_38121_b200 import binding as B
         self.torch, self.B, self.wl = torch, B, wl
@@ -52,11 +52,11 @@ class Layer:
             order = np.random.default_rng(page_shuffle_seed).permutation(self.batch * max_pages)
         self.cache = B.PagedCache(wl.n_q, wl.n_kv, bits, self.batch, self.max_seq_len, s_sink, s_keep, s_flush,
                                   kappa_k, kappa_v, self.T, self.TinvT, boundary_lag=lag, page_order=order,
-                                  ring_cap=ring_cap)
+                                  ring_cap=ring_cap, quantizer=1 if quantizer == "quest" else 0)
         dev = self.cache.device
         self.slot = torch.arange(self.batch, dtype=torch.int32, device=dev)
         self.seq_len = torch.zeros(self.batch, dtype=torch.int32, device=dev)
-        self.oracle = [O.LayerCache(wl.n_kv, 128, bits, kappa_k, kappa_v, self.T) for _ in range(self.batch)]
+        self.oracle = [O.LayerCache(wl.n_kv, 128, bits, kappa_k, kappa_v, self.T, quantizer=quantizer) for _ in range(self.batch)]
         self.tokens = []
         for b, n in enumerate(self.lengths):
             ks, vs = [], []
@@ -180,6 +180,63 @@ class Layer:
                             1.0 / np.sqrt(128), lag=self.lag)
         assert np.all(np.isfinite(out)), "oracle read a position the GPU keeps no bf16 copy of"
         return out
+
+    def prefill(self, counts):
+        """Append counts[b] new tokens per sequence and compute their attention outputs with wushkv_prefill_attn.
+        Returns (O_gpu list per sequence [n][n_q][128], queries list per sequence)."""
+        torch, B = self.torch, self.B
+        counts = [int(c) for c in counts]
+        start = list(self.done)
+        Ks = [self.tokens[b][0][start[b]:start[b] + c] for b, c in enumerate(counts)]
+        Vs = [self.tokens[b][1][start[b]:start[b] + c] for b, c in enumerate(counts)]
+        self.append_step(counts)
+        total = sum(counts)
+        dev = self.cache.device
+        qs = [self.wl.chunk_queries(b, np.arange(start[b], start[b] + c)) if c else np.zeros((0, self.wl.n_q, 128), np.float32)
+              for b, c in enumerate(counts)]
+        bits16 = lambda x: torch.from_numpy(W.f32_to_bf16_bits(x).view(np.int16)).to(dev)  # noqa: E731
+        Kn, Vn, Qn = bits16(np.concatenate(Ks)), bits16(np.concatenate(Vs)), bits16(np.concatenate(qs))
+        cu = torch.tensor(np.concatenate([[0], np.cumsum(counts)]).astype(np.int32), device=dev)
+        Oo = torch.full((total, self.wl.n_q, 128), float("nan"), dtype=torch.float32, device=dev)
+        nbytes = B.prefill_workspace_bytes(self.cache.desc, self.batch, total)
+        ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        B.prefill_attn(self.cache.desc, self.batch, self.slot, self.seq_len, cu, total, max(counts), Kn, Vn, Qn, Oo, ws, nbytes)
+        torch.cuda.synchronize()
+        out = Oo.cpu().numpy().astype(np.float64)
+        offs = np.concatenate([[0], np.cumsum(counts)])
+        return [out[offs[b]:offs[b + 1]] for b in range(self.batch)], qs
+
+    def check_prefill_parity(self, counts, tol=DECODE_TOL, rows=None):
+        """Chunk attention of the GPU against the oracle's on the cache content the GPU stored (codes and meta of
+        the old positions; the bf16 roundings of the transformed keys for the window and chunk positions come from
+        the oracle's own cache, which the append parity check ties to the GPU's).  ``rows``: chunk rows to check
+        per sequence (default: all)."""
+        outs, qs = self.prefill(counts)
+        worst = 0.0
+        for b, c in enumerate(counts):
+            if c == 0:
+                continue
+            S = self.done[b]
+            n_kv = self.wl.n_kv
+            kc = np.zeros((S, n_kv, 128), np.uint8)
+            vc = np.zeros((S, n_kv, 128), np.uint8)
+            km = np.zeros((S, n_kv, 2))
+            vm = np.zeros((S, n_kv, 2))
+            for h in range(n_kv):
+                cc, sc, zc = self.gpu_codes(b, h, 0, n=S)
+                kc[:, h], km[:, h, 0], km[:, h, 1] = cc, sc, zc
+                cc, sc, zc = self.gpu_codes(b, h, 1, n=S)
+                vc[:, h], vm[:, h, 0], vm[:, h, 1] = cc, sc, zc
+            _, _, _, _, kb, vb = self.oracle[b].arrays()
+            sel = np.arange(c) if rows is None else np.asarray([r for r in rows if r < c])
+            ref = O.chunk_attn(qs[b], self.TinvT, kc, km, vc, vm, kb, vb, S, c, self.s_sink, self.s_keep, self.s_flush,
+                               1.0 / np.sqrt(128), lag=self.lag)
+            assert np.all(np.isfinite(outs[b])), "non-finite prefill output"
+            for r in sel:
+                err = np.max(np.abs(outs[b][r] - ref[r])) / np.max(np.abs(ref[r]))
+                worst = max(worst, err)
+                assert err <= tol, f"prefill mismatch: sequence {b}, chunk row {r}: {err:.3e} of max-abs"
+        return worst
 
     def check_decode_parity(self, tol=DECODE_TOL):
         Og, Q = self.decode()

@@ -112,6 +112,27 @@ def test_prefill_chunk_paths(path, test_option):
     assert L.cache.status() == 0
 
 
+@pytest.mark.parametrize("bits", [2, 4])
+def test_quest_quantizer_on_every_append_path(bits):
+    """Section 4.3, Eq. 5 instead of Eq. 6: step from the group's RMS, bin-centre reconstruction.  One sequence
+    goes through the tensor-core chunk path, one through the CUDA-core rows path, and every sequence gets a
+    decode-time token; the packed cache is then decoded as usual."""
+    wl = _wl(8, 2, seed=45, batch=3)
+    L = Layer(wl, [400, 90, 131], bits, 4, 64, 8, quantizer="quest")
+    L.append_step([399, 0, 0])        # chunk of >= 128 tokens: tensor-core transform, quad quantizer
+    L.append_step([0, 89, 130])       # tensor-core path again (max_new 130) with a ragged tile
+    L.append_step([1, 1, 1])          # single-token kernel
+    assert L.seq_len.cpu().tolist() == [400, 90, 131]
+    assert L.check_append_parity() <= CODE_MISMATCH_MAX
+    assert L.check_decode_parity() <= 2e-3
+    L2 = Layer(wl, [70, 33, 5], bits, 4, 64, 8, quantizer="quest")
+    L2.append_step([69, 32, 4])       # max_new < 128: CUDA-core rows path
+    L2.append_step([1, 1, 1])
+    assert L2.check_append_parity() <= CODE_MISMATCH_MAX
+    assert L2.check_decode_parity() <= 2e-3
+    assert L.cache.status() == 0 and L2.cache.status() == 0
+
+
 def test_window_edges_and_empty_sequences():
     """Degenerate cases of Section 4.4: nothing cached, everything inside the sink, nothing quantized
     yet (S <= S_sink + S_keep + S_flush - 1), exactly one flush group quantized."""

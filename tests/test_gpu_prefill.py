@@ -1,0 +1,66 @@
+"""GPU parity of chunk (prefill) attention over the mixed cache, wushkv_prefill_attn, against the oracle's
+chunk_attn: Algorithm 2 line 5 for a chunk, Sections 4.4 and 5.3."""
+import numpy as np
+import pytest
+
+from paper_2609_38121_b200 import workloads as W
+from tests.harness import CODE_MISMATCH_MAX, Layer
+
+pytestmark = pytest.mark.gpu
+
+
+def _wl(n_q, n_kv, seed, batch=1, theta=1e4, rmsnorm=False):
+    return W.LayerWorkload(dict(seed=seed, batch=batch, n_q=n_q, n_kv=n_kv, ctx=0, theta=theta, bits=2, s_sink=4,
+                                s_keep=64, rmsnorm=rmsnorm, ragged=None, prefill_chunk=0))
+
+
+@pytest.mark.parametrize("bits", [2, 4])
+def test_prefill_on_an_empty_cache(bits):
+    """The whole prompt as one chunk: every key is a chunk position (full precision, causal); several query tiles,
+    a ragged last tile, a sequence shorter than one tile."""
+    wl = _wl(8, 2, seed=91, batch=3)
+    L = Layer(wl, [333, 70, 9], bits, 4, 64, 1)
+    assert L.check_prefill_parity([333, 70, 9]) <= 2e-3
+    assert L.check_append_parity() <= CODE_MISMATCH_MAX
+    assert L.cache.status() == 0
+
+
+@pytest.mark.parametrize("bits,n_q,n_kv", [(2, 8, 2), (4, 14, 2)])
+def test_chunk_over_a_quantized_cache(bits, n_q, n_kv):
+    """A chunk appended to a long cache: sink rows, packed pages (first and last one partly outside the quantized
+    range), the old part of the recent window, then the chunk; ragged batch, shuffled page table, G = 4 and 7."""
+    wl = _wl(n_q, n_kv, seed=92, batch=3)
+    L = Layer(wl, [900, 450, 260], bits, 4, 64, 8, page_shuffle_seed=7)
+    L.append_step([700, 300, 259])
+    assert L.check_prefill_parity([200, 150, 1]) <= 2e-3        # the last sequence: a chunk of one token
+    assert L.check_decode_parity() <= 2e-3                       # the cache is in order for the next decode step
+    assert L.cache.status() == 0
+
+
+def test_chunk_shorter_than_the_recent_window_and_second_chunk():
+    """Chunks of 16 tokens as in the paper's perplexity runs (S_sink 16, S_keep 128, S_flush 16): old recent-window
+    rows come from the ring, the quantized boundary sits below the chunk; two chunks in a row."""
+    wl = _wl(8, 2, seed=93)
+    L = Layer(wl, [432], 2, 16, 128, 16)
+    L.append_step([400])
+    assert L.check_prefill_parity([16]) <= 2e-3
+    assert L.check_prefill_parity([16]) <= 2e-3
+    assert L.cache.status() == 0
+
+
+def test_literal_algorithm2_boundary():
+    """boundary_lag = chunk length: the boundary of Algorithm 2 lines 7-8 is moved after attention."""
+    wl = _wl(8, 2, seed=94)
+    n_new = 40
+    L = Layer(wl, [500], 2, 4, 64, 8, lag=n_new)
+    L.append_step([460])
+    assert L.check_prefill_parity([n_new]) <= 2e-3
+    assert L.cache.status() == 0
+
+
+def test_quest_cache_under_a_chunk():
+    wl = _wl(8, 2, seed=95)
+    L = Layer(wl, [600], 4, 4, 64, 1, quantizer="quest")
+    L.append_step([400])
+    assert L.check_prefill_parity([200]) <= 2e-3
+    assert L.cache.status() == 0
