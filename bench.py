@@ -47,6 +47,14 @@ NCU_TRAFFIC_BYTES = {"cfg1": 310668544 + 3688960, "cfg2": 362961408 + 3549440,
                      "cfg3": 76140032 + 3253760, "cfg4": None}
 
 
+def measured_tensor_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops_sustained"]), "measured"
+    except Exception:
+        return 1400.0, "fallback"
+
+
 def measured_hbm_peak():
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
@@ -113,6 +121,11 @@ class Session:
             self.K_chunk = self._dev_bf16(np.concatenate(ks))
             self.V_chunk = self._dev_bf16(np.concatenate(vs))
             self.cu_chunk = torch.arange(0, (self.batch + 1) * self.chunk, self.chunk, dtype=torch.int32, device=dev)
+            self.q_chunk_host = np.concatenate([wl.chunk_queries(b, np.arange(self.chunk)) for b in range(self.batch)])
+            self.Q_chunk = self._dev_bf16(self.q_chunk_host)
+            self.O_chunk = torch.zeros((self.batch * self.chunk, wl.n_q, 128), dtype=torch.float32, device=dev)
+            self.pf_bytes = B.prefill_workspace_bytes(self.cache.desc, self.batch, self.batch * self.chunk)
+            self.pf_ws = torch.empty(self.pf_bytes, dtype=torch.uint8, device=dev)
             n_step_tok = 0
         else:
             n_step_tok = n_steps
@@ -169,8 +182,9 @@ class Session:
         self.seq_len.copy_(self.base_len)
         self.step_index = 0
 
-    def step(self, mid_event=None):
-        """Enqueue one step (device-resident inputs)."""
+    def step(self, mid_event=None, pf_event=None):
+        """Enqueue one step (device-resident inputs).  Prefill config: append the chunk, compute the chunk's own
+        attention outputs (Algorithm 2 line 5), then one decode step over the resulting cache."""
         B = self.B
         if not self.chunk and mid_event is None:        # the fused call a user makes for a decode step
             i = self.step_index
@@ -189,6 +203,11 @@ class Session:
             self.step_index += 1
         if mid_event is not None:
             mid_event.record()
+        if self.chunk:
+            B.prefill_attn(self.cache.desc, self.batch, self.slot, self.seq_len, self.cu_chunk, self.batch * self.chunk,
+                           self.chunk, self.K_chunk, self.V_chunk, self.Q_chunk, self.O_chunk, self.pf_ws, self.pf_bytes)
+            if pf_event is not None:
+                pf_event.record()
         B.decode_attn(self.cache.desc, self.batch, self.slot, self.seq_len, self.max_seq_len, self.Q, self.O,
                       self.ws, self.ws_bytes)
 
@@ -211,9 +230,15 @@ class Session:
     def append_tokens(self):
         return self.batch * (self.chunk if self.chunk else 1)
 
+    def prefill_flops(self):
+        """Multiply-adds x 2 of the chunk attention (causal: row i sees i + 1 keys; both contractions)."""
+        n = self.chunk
+        return 4.0 * 128 * self.wl.n_q * self.batch * (n * (n + 1) / 2)
+
     def launches_per_step(self):
-        # chunk append: transform/quantize kernel + length update; token append: one kernel; decode: prep + main + combine
-        return (2 if self.chunk else 1) + 3
+        # chunk append: transform/quantize kernel + length update (+ prefill attention: preparation + attention);
+        # token append: one kernel; decode: prep + main + combine
+        return (4 if self.chunk else 1) + 3
 
 
 # ------------------------------------------------------------------------------------------------
@@ -531,6 +556,7 @@ def run_ours(args, rank, world):
     # Events between kernels switch programmatic dependent launch off, so region B's steps are a
     # little slower than region A's; the kernel's own duration is what is taken from here.
     mids = [ev() for _ in range(K)]
+    pfs = [ev() for _ in range(K)]
     kstart, kstop = [ev() for _ in range(K)], [ev() for _ in range(K)]
     for e in kstart + kstop:
         e.record()                    # materialise the handles
@@ -540,7 +566,7 @@ def run_ours(args, rank, world):
             flush_buf.fill_(i & 0xFF)
         B.set_profile_events(kstart[i], kstop[i])
         starts[i].record()
-        sess.step(mid_event=mids[i])
+        sess.step(mid_event=mids[i], pf_event=pfs[i])
         stops[i].record()
     B.set_profile_events(None, None)
     barrier()
@@ -550,6 +576,7 @@ def run_ours(args, rank, world):
     assert sess.cache.status() == 0, f"device status {sess.cache.status()}"
     step_ms = [s_.elapsed_time(e_) for s_, e_ in zip(starts, stops)]
     append_ms = [s_.elapsed_time(e_) for s_, e_ in zip(starts, mids)]
+    prefill_ms = [s_.elapsed_time(e_) for s_, e_ in zip(mids, pfs)] if sess.chunk else None
     kern_ms = [s_.elapsed_time(e_) for s_, e_ in zip(kstart, kstop)]
     ms_per_step = max_over_ranks(ms_per_step)
     bytes_step = float(np.mean([sess.decode_bytes(Wm + i + 1) for i in range(K)])) if not sess.chunk else float(cache_bytes)
@@ -649,6 +676,14 @@ def run_ours(args, rank, world):
                     "kernel_ms": kern_s * 1e3, "kernel_ms_min": min(kern_ms), "algorithmic_bytes": bytes_step,
                     "traffic": NCU_TRAFFIC_BYTES.get(args.config),
                     "kernel_cycles": (kern_s * 1e6 * sm_mhz) if sm_mhz else None}
+    roofline_pf = None
+    if sess.chunk:
+        tf_peak, tf_kind = measured_tensor_peak()
+        pf_s = statistics.mean(prefill_ms) * 1e-3
+        tf = sess.prefill_flops() / pf_s / 1e12
+        roofline_pf = {"bound": "tensor", "kernel": "prefill_attn_kernel (+ its preparation kernel)", "achieved": tf, "peak": tf_peak,
+                       "unit": "TFLOP/s", "frac": tf / tf_peak, "peak_kind": f"of {tf_kind} (bf16 matmul, sustained; fp16 has the same nominal rate)",
+                       "kernel_ms": pf_s * 1e3, "kernel_ms_min": min(prefill_ms), "algorithmic_flops": sess.prefill_flops(), "traffic": None}
     cpu = None
     if world == 1 and not args.no_cpu:
         smp, split = time_oracle_split(args.config, budget_s=args.cpu_seconds)
@@ -671,7 +706,7 @@ def run_ours(args, rank, world):
                    "s_flush": sess.s_flush, "page_tokens": 64, "prefill_chunk": sess.chunk,
                    "l2": ("flushed between steps (256 MB write)" if need_flush else "cache read per step exceeds L2 (no flush)"),
                    "replicas": world},
-        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
+        "roofline": roofline, "roofline_prefill_attn": roofline_pf, "cpu_baseline": cpu, "e2e": e2e,
         "value_sustained": sustained["value"] if sustained else None, "sustained": sustained,
         "gpu_launches": K * sess.launches_per_step(), "clocks": clocks,
         "decode_tokens_per_s": world * sess.batch / (ms_per_step * 1e-3),

@@ -50,8 +50,8 @@ struct PrefillParams {
     float* O;                             // [total_new][n_q][D]
     __half* KP;                           // [total_new][n_kv][D]  fp16(bf16(T_K k))
     __half* VP;                           // [total_new][n_kv][D]  fp16(v)
-    __half* QP;                           // [total_new][n_q][D]   fp16(T_K^{-T} q)
-    float* qsum;                          // [total_new][n_q]      sum over channels of the fp16 q'
+    __half* QP;                           // [2][total_new][n_q][D]  q' = T_K^{-T} q as fp16 value, then fp16 rounding remainder
+    float* qsum;                          // [total_new][n_q]      sum over channels of q' (value + remainder)
     int tiles_per_seq;                    // ceil(max_new / BM)
 };
 
@@ -115,15 +115,16 @@ __global__ void __launch_bounds__(256) prefill_prep_kernel(PrefillParams P) {
     for (int k = 0; k < 16; ++k) {
         const int tok = tok0 + tg * 16 + k;
         float val = acc[k];
-        __half hv;
+        __half hv, lv = __float2half_rn(0.f);
         if (is_key) hv = __float2half_rn(bf16_bits_to_float(float_to_bf16_bits(val)));   // the cache holds bf16(k')
-        else hv = __float2half_rn(val);
+        else { hv = __float2half_rn(val); lv = __float2half_rn(val - __half2float(hv)); }
         if (tok < P.total_new) {
-            __half* dst = (is_key ? P.KP : P.QP) + (static_cast<long long>(tok) * n_heads + head) * D + i;
-            *dst = hv;
+            const long long off = (static_cast<long long>(tok) * n_heads + head) * D + i;
+            if (is_key) P.KP[off] = hv;
+            else { P.QP[off] = hv; P.QP[static_cast<long long>(P.total_new) * n_heads * D + off] = lv; }
         }
-        if (!is_key) {                                                // sum of the rounded q' over the 128 channels
-            float s = __half2float(hv);
+        if (!is_key) {                                                // sum of the two-term q' over the 128 channels
+            float s = __half2float(hv) + __half2float(lv);
             for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(FULLM, s, o);
             if ((threadIdx.x & 31) == 0) rowsum[(tg * 16 + k) * 4 + ((threadIdx.x & 127) >> 5)] = s;
         }
@@ -151,6 +152,7 @@ __global__ void __launch_bounds__(256) prefill_prep_kernel(PrefillParams P) {
 // 2. attention
 // ------------------------------------------------------------------------------------------------
 struct TileSmem {
+    __half Q[2][BM][TILE_PITCH];   // the CTA's query rows: fp16 value and rounding remainder of q'
     __half K[BN][TILE_PITCH];
     __half V[BN][TILE_PITCH];
     float4 meta[BN];          // per key: Delta_k, x_min_k, Delta_v, x_min_v (1, 0, 1, 0 for a full-precision row)
@@ -186,17 +188,11 @@ __global__ void __launch_bounds__(PF_THREADS) prefill_attn_kernel(PrefillParams 
     // ---- this warp's 16 query rows as A fragments (kept in registers), and their channel sums
     const int row0 = qt * BM + warp * 16;                       // chunk-relative row of fragment row 0
     const int ra = min(row0 + g, n_new - 1), rb = min(row0 + g + 8, n_new - 1);
-    unsigned qa[8][4];
-    {
-        const __half* q0 = P.QP + (static_cast<long long>(first + ra) * c.n_q + jq) * D;
-        const __half* q1 = P.QP + (static_cast<long long>(first + rb) * c.n_q + jq) * D;
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            qa[ks][0] = __ldcg(reinterpret_cast<const unsigned*>(q0 + 16 * ks + 2 * t));
-            qa[ks][1] = __ldcg(reinterpret_cast<const unsigned*>(q1 + 16 * ks + 2 * t));
-            qa[ks][2] = __ldcg(reinterpret_cast<const unsigned*>(q0 + 16 * ks + 8 + 2 * t));
-            qa[ks][3] = __ldcg(reinterpret_cast<const unsigned*>(q1 + 16 * ks + 8 + 2 * t));
-        }
+    for (int item = tid; item < 2 * BM * 16; item += PF_THREADS) {       // 16-byte pieces of the query rows (rows past the chunk: the last row again)
+        const int part = item / (BM * 16), r = (item >> 4) % BM, piece = item & 15;
+        const int row = min(qt * BM + r, n_new - 1);
+        const __half* src = P.QP + static_cast<long long>(part) * P.total_new * c.n_q * D + (static_cast<long long>(first + row) * c.n_q + jq) * D + 8 * piece;
+        *reinterpret_cast<uint4*>(&ts.Q[part][r][8 * piece]) = __ldcg(reinterpret_cast<const uint4*>(src));
     }
     const float qs_a = __ldcg(P.qsum + static_cast<long long>(first + ra) * c.n_q + jq);
     const float qs_b = __ldcg(P.qsum + static_cast<long long>(first + rb) * c.n_q + jq);
@@ -214,12 +210,18 @@ __global__ void __launch_bounds__(PF_THREADS) prefill_attn_kernel(PrefillParams 
         for (int nb = 0; nb < 8; ++nb) s[nb][0] = s[nb][1] = s[nb][2] = s[nb][3] = 0.f;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
+            unsigned ah[4], al[4];                              // this warp's 16 rows x 16 channels: value, remainder
+            const int qrow = 16 * warp + (lane & 7) + 8 * ((lane >> 3) & 1), qcol = 16 * ks + 8 * (lane >> 4);
+            ldsm_x4(smem_addr(&ts.Q[0][qrow][qcol]), ah[0], ah[1], ah[2], ah[3]);
+            ldsm_x4(smem_addr(&ts.Q[1][qrow][qcol]), al[0], al[1], al[2], al[3]);
 #pragma unroll
             for (int nb2 = 0; nb2 < 4; ++nb2) {                 // two key blocks of 8 per ldmatrix.x4
                 unsigned b0, b1, b2, b3;
                 ldsm_x4(smem_addr(&ts.K[16 * nb2 + 8 * (lane >> 4) + (lane & 7)][16 * ks + 8 * ((lane >> 3) & 1)]), b0, b1, b2, b3);
-                hmma(s[2 * nb2], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
-                hmma(s[2 * nb2 + 1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b2, b3);
+                hmma(s[2 * nb2], ah[0], ah[1], ah[2], ah[3], b0, b1);
+                hmma(s[2 * nb2 + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
+                hmma(s[2 * nb2], al[0], al[1], al[2], al[3], b0, b1);
+                hmma(s[2 * nb2 + 1], al[0], al[1], al[2], al[3], b2, b3);
             }
         }
         // affine part, masks, row maxima (log2 domain)
@@ -409,7 +411,7 @@ bool make_prefill_plan(const CacheView& c, int total_new, PrefillPlan& pl) {
     size_t off = 0;
     pl.off_kp = off;   off = align256(off + static_cast<size_t>(total_new) * c.n_kv * D * sizeof(__half));
     pl.off_vp = off;   off = align256(off + static_cast<size_t>(total_new) * c.n_kv * D * sizeof(__half));
-    pl.off_qp = off;   off = align256(off + static_cast<size_t>(total_new) * c.n_q * D * sizeof(__half));
+    pl.off_qp = off;   off = align256(off + 2 * static_cast<size_t>(total_new) * c.n_q * D * sizeof(__half));
     pl.off_qsum = off; off = align256(off + static_cast<size_t>(total_new) * c.n_q * sizeof(float));
     pl.total = off;
     return true;

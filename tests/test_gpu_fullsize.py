@@ -77,6 +77,25 @@ def _check_decode_group(sess, out, b, h):
     return np.max(np.abs(got - ref)) / np.max(np.abs(ref))
 
 
+def _check_prefill_rows(sess, o_chunk, b, h, rows):
+    """Oracle chunk attention (empty cache before the chunk: every key is a chunk position, read as the bf16 rounding of
+    the transformed key) for the G query heads of KV head h of sequence b, at the given chunk rows."""
+    wl = sess.wl
+    G = wl.G
+    K, V = sess.host_tokens(b)
+    Kp = O.round_bf16(O.key_transform(sess.T[h].astype(np.float64), K[:, h]))
+    Vh = V[:, h].astype(np.float64)
+    q = sess.q_chunk_host.reshape(sess.batch, sess.chunk, wl.n_q, 128)[b]
+    errs = []
+    for r in rows:
+        for gq in range(G):
+            j = h * G + gq
+            qc = O.query_compensation(sess.TinvT[h].astype(np.float64), q[r, j][None].astype(np.float64))[0]
+            ref = O.attention_one_query(qc, Kp[:r + 1], Vh[:r + 1], 1.0 / np.sqrt(128))
+            errs.append(np.max(np.abs(o_chunk[b, r, j] - ref)) / np.max(np.abs(ref)))
+    return errs
+
+
 @pytest.mark.parametrize("name,groups", [
     ("cfg1", [(0, 0), (7, 3), (15, 7)]),          # Llama-3-8B-shaped, batch 16 x 32768, 2-bit
     ("cfg2", [(0, 0), (31, 5), (63, 7)]),         # 4-bit, batch 64, ragged 1024..8192
@@ -108,3 +127,12 @@ def test_full_size_config(name, groups):
     for (b, h) in groups:
         err = _check_decode_group(sess, out, b, h)
         assert err <= 2e-3, f"{name}: sequence {b} KV head {h}: {err:.3e}"
+    if sess.chunk:
+        # the chunk's own attention outputs (Algorithm 2 line 5) at full size: sampled rows of sampled
+        # (sequence, query head) pairs against the oracle's definition, row by row
+        o_chunk = sess.O_chunk.cpu().numpy().astype(np.float64).reshape(sess.batch, sess.chunk, sess.wl.n_q, 128)
+        assert np.all(np.isfinite(o_chunk))
+        rows = [0, 1, 63, 64, 65, 4095, 4096, sess.chunk - 65, sess.chunk - 1]
+        for (b, h) in groups:
+            errs = _check_prefill_rows(sess, o_chunk, b, h, rows)
+            assert max(errs) <= 2e-3, f"{name}: prefill rows of sequence {b} KV head {h}: {max(errs):.3e}"
