@@ -146,6 +146,26 @@ int wushkv_build_transforms(int32_t n_heads, int32_t d, const double* M, const d
                             float* T, float* T_invT);
 
 /*
+ * The same two calibration steps on the GPU (Algorithm 1 lines 4-5 and 7; Eq. 4; Eq. 1), for calibration sets
+ * of millions of tokens.  Results equal the host calls' up to summation order.
+ *   wushkv_accumulate_gram_device: K, Q (device) bf16 as above, 16-byte aligned; M, H (device, in/out) float64
+ *     [n_kv][d][d], zeroed by the caller before the first sequence.  d must be 128.  Products of the bf16
+ *     inputs are exact, sums are fp32 within groups of 128 tokens and float64 beyond (relative error below 1e-6).
+ *   wushkv_build_transforms_device: M, H (device) float64 [n_heads][d][d]; T, T_invT (device, out) fp32
+ *     [n_heads][d][d] with the same canonical form and bf16 rounding as the host call; status (device, out):
+ *     one int32 the caller zeroes, set to WUSHKV_ENOTPD if a damped matrix is not positive definite;
+ *     workspace (device): >= wushkv_build_transforms_workspace_bytes() bytes, 16-byte aligned.
+ * Both enqueue on `stream` and do not synchronise.
+ */
+int wushkv_accumulate_gram_device(int32_t n_kv, int32_t n_q, int32_t d, int64_t n_tok, const uint16_t* K, const uint16_t* Q,
+                                  double* M, double* H, void* stream);
+size_t wushkv_build_transforms_workspace_bytes(int32_t n_heads, int32_t d);
+int wushkv_build_transforms_device(int32_t n_heads, int32_t d, const double* M, const double* H, double gamma,
+                                   float* T, float* T_invT, int32_t* status, void* workspace, size_t workspace_bytes,
+                                   void* stream);
+
+
+/*
  * Quantize-on-append: Algorithm 2 lines 3-4 (key side) and 9-12, with Eq. 6 as the quantizer.
  * For sequence b (0 <= b < batch) the new tokens are rows cu_new[b] .. cu_new[b+1]-1 of K_new /
  * V_new and take positions seq_len[b], seq_len[b]+1, ...  Every new token is transformed

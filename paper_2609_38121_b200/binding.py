@@ -21,6 +21,7 @@ EXPORTS = (
     "wushkv_append", "wushkv_decode_workspace_bytes", "wushkv_decode_attn", "wushkv_unpack_debug",
     "wushkv_decode_step", "wushkv_step_staging_bytes", "wushkv_decode_step_host", "wushkv_set_profile_events",
     "wushkv_decode_attn_static", "wushkv_set_test_option", "wushkv_prefill_workspace_bytes", "wushkv_prefill_attn",
+    "wushkv_accumulate_gram_device", "wushkv_build_transforms_workspace_bytes", "wushkv_build_transforms_device",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -92,6 +93,14 @@ def _load():
     lib.wushkv_prefill_attn.restype = C.c_int
     lib.wushkv_prefill_attn.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.wushkv_accumulate_gram_device.restype = C.c_int
+    lib.wushkv_accumulate_gram_device.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                                  C.c_void_p, C.c_void_p]
+    lib.wushkv_build_transforms_workspace_bytes.restype = C.c_size_t
+    lib.wushkv_build_transforms_workspace_bytes.argtypes = [C.c_int32, C.c_int32]
+    lib.wushkv_build_transforms_device.restype = C.c_int
+    lib.wushkv_build_transforms_device.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_double, C.c_void_p, C.c_void_p,
+                                                   C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
     lib.wushkv_set_test_option.restype = C.c_int
     lib.wushkv_set_test_option.argtypes = [C.c_char_p, C.c_longlong]
     return lib
@@ -150,6 +159,32 @@ def build_transforms(M: np.ndarray, H: np.ndarray, gamma: float):
     _check(lib.wushkv_build_transforms(n, d, M.ctypes.data, H.ctypes.data, float(gamma), T.ctypes.data,
                                        TinvT.ctypes.data), "wushkv_build_transforms")
     return T, TinvT
+
+
+def accumulate_gram_device(K_bits, Q_bits, M, H, stream=None):
+    """wushkv_accumulate_gram_device: K_bits int16/uint16 [n_tok][n_kv][d], Q_bits [n_tok][n_q][d] (bf16 patterns) and
+    M, H float64 [n_kv][d][d], all CUDA tensors; M and H are updated in place."""
+    n_tok, n_kv, d = K_bits.shape
+    _check(lib.wushkv_accumulate_gram_device(n_kv, Q_bits.shape[1], d, n_tok, _ptr(K_bits), _ptr(Q_bits), _ptr(M), _ptr(H),
+                                             _stream_ptr(stream)), "wushkv_accumulate_gram_device")
+
+
+def build_transforms_device(M, H, gamma: float, stream=None):
+    """wushkv_build_transforms_device: M, H float64 CUDA tensors [n_heads][d][d]; returns (T, T_invT) fp32 CUDA tensors.
+    Raises with status ENOTPD if a damped matrix is not positive definite (this wrapper synchronises to find out)."""
+    import torch
+    n, d, _ = M.shape
+    T = torch.empty((n, d, d), dtype=torch.float32, device=M.device)
+    Ti = torch.empty_like(T)
+    status = torch.zeros(1, dtype=torch.int32, device=M.device)
+    nbytes = int(lib.wushkv_build_transforms_workspace_bytes(n, d))
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=M.device)
+    _check(lib.wushkv_build_transforms_device(n, d, _ptr(M), _ptr(H), float(gamma), _ptr(T), _ptr(Ti), _ptr(status), _ptr(ws),
+                                              nbytes, _stream_ptr(stream)), "wushkv_build_transforms_device")
+    st = int(status.item())
+    if st != 0:
+        raise WushkvError(st, "wushkv_build_transforms_device")
+    return T, Ti
 
 
 def append(cache: wushkv_cache, batch, slot, seq_len, cu_new, total_new, max_new, K_new, V_new, stream=None):
