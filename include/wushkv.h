@@ -302,6 +302,11 @@ int wushkv_decode_step_host(const wushkv_cache* cache, int32_t batch, const int3
  *   - Arguments and results are exactly those of wushkv_decode_attn, minus workspace.
  *   - A request whose wushkv_decode_workspace_bytes() exceeds WUSHKV_STATIC_SCRATCH_BYTES is
  *     refused with WUSHKV_ECAPACITY and nothing is launched; use wushkv_decode_attn then.
+ *     The workspace grows with batch * n_kv (8 KiB of query fragments each) and with the number
+ *     of warps of the main kernel (G * 528 bytes of partial result each; the "decode_ctas"
+ *     testing aid changes that number).  On a 148-SM GPU: 16 sequences x 8 KV heads x 32 query
+ *     heads need 6.0 MiB, 1 x 8 x 64 needs 7.2 MiB, 8 x 4 x 28 needs 6.6 MiB - they fit;
+ *     64 sequences x 8 KV heads x 32 query heads need 8.6 MiB and are refused.
  *   - The call allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).
  *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress,
  *     with that device current); make that first call before starting any stream capture.

@@ -21,7 +21,7 @@ Conventions
 
 Parity pins (tests/test_oracle_*.py, tests/test_golden.py) cover every function below (the error metric
 and the quantize-from-bf16 reading in test_oracle_attention.py, the QuEST quantizer in test_oracle_quest.py,
-chunk attention in test_oracle_chunk_attn.py); none is "parity unpinned" against the mathematics.  What the paper itself does not fix
+chunk attention in test_oracle_chunk_attn.py, Norm and RoPE in test_oracle_prologue.py); none is "parity unpinned" against the mathematics.  What the paper itself does not fix
 (quantile interpolation rule, tie rounding, storage precision of scale and
 zero, the boundary used at attention time) cannot be pinned to the paper; each
 such reading is listed where it is taken.
@@ -149,6 +149,43 @@ def build_transforms(M, H, gamma: float = 1e-2):
         T[h] = round_bf16(wush(M[h], H[h], gamma))
         TinvT[h] = round_fp32(np.linalg.inv(T[h]).T)
     return T, TinvT
+
+
+# --------------------------------------------------------------------------
+# normalisation and rotary embedding ahead of the transform  (Algorithm 2, lines 1-2)
+# --------------------------------------------------------------------------
+def rms_norm(x, weight=None, eps: float = 0.0):
+    """Algorithm 2 lines 1-2, "Norm": headwise RMS normalisation of every row of ``x`` ([..., d]),
+    x / sqrt(mean(x^2) + eps) times a per-channel weight ([d] or broadcastable; None: ones).
+    The paper names the step and cites the architecture (Section 4.1: keys are cached after
+    normalisation and rotation); the formula is the standard one of that architecture."""
+    x = np.asarray(x, dtype=np.float64)
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    y = x / np.sqrt(ms + eps)
+    return y if weight is None else y * np.asarray(weight, dtype=np.float64)
+
+
+def rope(x, positions, theta: float):
+    """Algorithm 2 lines 1-2, "RoPE": rotate channel pair (j, j + d/2) of every row by the angle
+    position * theta^(-2 j / d).  ``x`` is [n][..., d], ``positions`` [n] (absolute, 0-based).
+    Reading: the paper does not say how channels are paired; the half-split pairing is the one of the
+    model family it evaluates."""
+    x = np.asarray(x, dtype=np.float64)
+    d = x.shape[-1]
+    half = d // 2
+    j = np.arange(half, dtype=np.float64)
+    ang = np.asarray(positions, dtype=np.float64).reshape((-1,) + (1,) * (x.ndim - 1)) * theta ** (-2.0 * j / d)
+    c, s = np.cos(ang), np.sin(ang)
+    a, b = x[..., :half], x[..., half:]
+    return np.concatenate([a * c - b * s, a * s + b * c], axis=-1)
+
+
+def prepare_rows(x_proj, positions, theta: float, weight=None, eps: float = 0.0, normalise: bool = True):
+    """Algorithm 2 lines 1-2 for projected keys or queries ([n][heads][d], bf16-valued): optional Norm,
+    then RoPE, in float64, and ONE rounding to bf16 at the end (the model's activation format,
+    Section 5.3).  Reading: the paper fixes no rounding points inside the two steps."""
+    y = rms_norm(x_proj, weight, eps) if normalise else np.asarray(x_proj, dtype=np.float64)
+    return round_bf16(rope(y, positions, theta))
 
 
 def key_transform(T, k_rows):

@@ -37,6 +37,27 @@ def test_static_scratch_decode_matches_regular_decode_twice():
             err = np.max(np.abs(got[b] - ref[b])) / np.max(np.abs(ref[b]))
             assert err <= DECODE_TOL, f"call {call}, sequence {b}: {err:.3e}"
     assert L.cache.status() == 0
+    # The call allocates no device memory: after the calls above resolved the array's address, the
+    # driver's free-byte count is the same before and after two further calls, one of them on a
+    # stream of its own that is ordered after the first by an event.
+    out_a = torch.empty((L.batch, wl.n_q, 128), dtype=torch.float32, device="cuda")
+    out_b = torch.empty_like(out_a)
+    side = torch.cuda.Stream()
+    done = torch.cuda.Event()
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    B.decode_attn_static(L.cache.desc, L.batch, L.slot, L.seq_len, L.max_seq_len, Q, out_a)
+    done.record()
+    side.wait_event(done)
+    B.decode_attn_static(L.cache.desc, L.batch, L.slot, L.seq_len, L.max_seq_len, Q, out_b, stream=side)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, (free_before, free_after)
+    for o in (out_a, out_b):
+        got = o.cpu().numpy().astype(np.float64)
+        for b in range(L.batch):
+            assert np.max(np.abs(got[b] - ref[b])) / np.max(np.abs(ref[b])) <= DECODE_TOL
+    assert torch.equal(out_a, out_b)
     # a different query afterwards still gives the regular path's answer (nothing stale is read)
     q2 = np.stack([wl.queries(b, 5) for b in range(L.batch)])
     ref2, _ = L.decode(q2)
