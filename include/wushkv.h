@@ -67,6 +67,7 @@ extern "C" {
 #define WUSHKV_DEV_COPY_TIMEOUT    8  /* a staged page copy did not arrive within the wait limit */
 #define WUSHKV_DEV_BAD_COUNT      16  /* max_new == 1 was promised but a sequence brought more than one token: sequence skipped */
 #define WUSHKV_DEV_VALUE_RANGE    32  /* a stored value step Delta_v >= 1024: beyond the fp16 range of the decode value contraction */
+#define WUSHKV_DEV_ROPE_RANGE     64  /* a position beyond the rotary table of a *_projected call: rotated by the table's last angle */
 /* After PAGE_TABLE_FULL, BAD_PAGE_ID, BAD_SLOT or BAD_COUNT in wushkv_append the length of the affected
  * sequence is left as it was (tokens of the call that did fit are orphaned: nothing reads them). */
 
@@ -241,6 +242,43 @@ int wushkv_prefill_attn(const wushkv_cache* cache, int32_t batch, const int32_t*
                         const int32_t* cu_new, int32_t total_new, int32_t max_new,
                         const uint16_t* K_new, const uint16_t* V_new, const uint16_t* Q_new, float* O,
                         void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Projected inputs: Algorithm 2 lines 1-2 (Norm, RoPE) fused into the kernels that apply line 3, so that
+ * keys and queries are read once, in the form the projections W_K x, W_Q x left them, and their normalised,
+ * rotated form never goes through memory (Section 4.1: keys are cached after normalisation and rotation).
+ *   Norm: headwise RMS normalisation x / sqrt(mean(x^2) + norm_eps), times a per-channel weight.
+ *   RoPE: channel pair (j, j + d/2) is rotated by the angle position * theta^(-2j/d); the position of a new
+ *         key is its index in the sequence, the position of the decode query is seq_len[b] - 1.
+ *   Arithmetic: fp32, one rounding to bf16 after the rotation; from there on the call is bit-identical to its
+ *         plain counterpart given those bf16 values.
+ *   wushkv_prologue (host struct; its pointers are DEVICE pointers, caller-owned, read-only):
+ *     rope_table       fp32 [rope_positions][d/2][2] = (cos, sin), written by wushkv_build_rope_table
+ *     rope_positions   positions the table covers; a token beyond it sets WUSHKV_DEV_ROPE_RANGE and is
+ *                      rotated by the table's last angle (drop the sequence)
+ *     normalise        0: no Norm step (RoPE only); 1: RMS normalisation
+ *     k_norm_weight    fp32 [n_kv][d] or NULL (ones);  q_norm_weight  fp32 [n_q][d] or NULL (ones)
+ *     norm_eps         >= 0
+ * wushkv_build_rope_table: cosines and sines in double precision, rounded to fp32 (device kernel; d must be 128).
+ * wushkv_append_projected / wushkv_decode_attn_projected: arguments, results and errors of wushkv_append /
+ * wushkv_decode_attn, with K_proj / Q_proj in place of K_new / Q and WUSHKV_EINVAL for a NULL or malformed
+ * prologue.  Values are never normalised or rotated (V_new is passed as before).
+ */
+typedef struct wushkv_prologue {
+    const float* rope_table;
+    int32_t rope_positions;
+    int32_t normalise;
+    const float* k_norm_weight;
+    const float* q_norm_weight;
+    float norm_eps;
+} wushkv_prologue;
+int wushkv_build_rope_table(double theta, int32_t n_positions, int32_t d, float* table, void* stream);
+int wushkv_append_projected(const wushkv_cache* cache, int32_t batch, const int32_t* slot, int32_t* seq_len,
+                            const int32_t* cu_new, int32_t total_new, int32_t max_new,
+                            const uint16_t* K_proj, const uint16_t* V_new, const wushkv_prologue* prologue, void* stream);
+int wushkv_decode_attn_projected(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
+                                 int32_t max_seq_len, const uint16_t* Q_proj, const wushkv_prologue* prologue, float* O,
+                                 void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Read back the logical content of the packed cache (test / debugging aid): for positions

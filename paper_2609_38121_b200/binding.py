@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libwushkv.so")
 OK, EINVAL, ENOTPD, ECUDA, ECAPACITY = 0, 1, 2, 3, 4
 QUANTIZER_AFFINE, QUANTIZER_QUEST = 0, 1
 DEV_PAGE_TABLE_FULL, DEV_BAD_PAGE_ID, DEV_BAD_SLOT, DEV_COPY_TIMEOUT, DEV_BAD_COUNT, DEV_VALUE_RANGE = 1, 2, 4, 8, 16, 32
+DEV_ROPE_RANGE = 64
 
 EXPORTS = (
     "wushkv_page_bytes", "wushkv_status_string", "wushkv_accumulate_gram", "wushkv_build_transforms",
@@ -22,6 +23,7 @@ EXPORTS = (
     "wushkv_decode_step", "wushkv_step_staging_bytes", "wushkv_decode_step_host", "wushkv_set_profile_events",
     "wushkv_decode_attn_static", "wushkv_set_test_option", "wushkv_prefill_workspace_bytes", "wushkv_prefill_attn",
     "wushkv_accumulate_gram_device", "wushkv_build_transforms_workspace_bytes", "wushkv_build_transforms_device",
+    "wushkv_build_rope_table", "wushkv_append_projected", "wushkv_decode_attn_projected",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -45,6 +47,12 @@ class wushkv_cache(C.Structure):
         ("pages", C.c_void_p), ("page_table", C.c_void_p), ("sink_kv", C.c_void_p), ("ring_kv", C.c_void_p),
         ("T_K", C.c_void_p), ("T_K_invT", C.c_void_p), ("dev_status", C.c_void_p),
     ]
+
+
+class wushkv_prologue(C.Structure):
+    """Mirror of ``struct wushkv_prologue`` (device pointers)."""
+    _fields_ = [("rope_table", C.c_void_p), ("rope_positions", C.c_int32), ("normalise", C.c_int32),
+                ("k_norm_weight", C.c_void_p), ("q_norm_weight", C.c_void_p), ("norm_eps", C.c_float)]
 
 
 def _load():
@@ -101,6 +109,14 @@ def _load():
     lib.wushkv_build_transforms_device.restype = C.c_int
     lib.wushkv_build_transforms_device.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_double, C.c_void_p, C.c_void_p,
                                                    C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.wushkv_build_rope_table.restype = C.c_int
+    lib.wushkv_build_rope_table.argtypes = [C.c_double, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+    lib.wushkv_append_projected.restype = C.c_int
+    lib.wushkv_append_projected.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                            C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(wushkv_prologue), C.c_void_p]
+    lib.wushkv_decode_attn_projected.restype = C.c_int
+    lib.wushkv_decode_attn_projected.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_void_p, C.c_void_p, C.c_int32,
+                                                 C.c_void_p, C.POINTER(wushkv_prologue), C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
     lib.wushkv_set_test_option.restype = C.c_int
     lib.wushkv_set_test_option.argtypes = [C.c_char_p, C.c_longlong]
     return lib
@@ -190,6 +206,38 @@ def build_transforms_device(M, H, gamma: float, stream=None):
 def append(cache: wushkv_cache, batch, slot, seq_len, cu_new, total_new, max_new, K_new, V_new, stream=None):
     _check(lib.wushkv_append(C.byref(cache), batch, _ptr(slot), _ptr(seq_len), _ptr(cu_new), total_new, max_new,
                              _ptr(K_new), _ptr(V_new), _stream_ptr(stream)), "wushkv_append")
+
+
+class Prologue:
+    """Holds the device tensors a ``wushkv_prologue`` points to (rotary table from wushkv_build_rope_table, optional
+    normalisation weights [n_kv][d] / [n_q][d]) and the struct itself."""
+
+    def __init__(self, theta: float, n_positions: int, normalise: bool = False, k_weight=None, q_weight=None,
+                 eps: float = 0.0, device="cuda", d: int = 128):
+        import torch
+        self.table = torch.empty((n_positions, d // 2, 2), dtype=torch.float32, device=device)
+        _check(lib.wushkv_build_rope_table(float(theta), n_positions, d, _ptr(self.table), _stream_ptr(None)),
+               "wushkv_build_rope_table")
+        as_dev = lambda w: None if w is None else torch.as_tensor(np.ascontiguousarray(w, dtype=np.float32)).to(device)
+        self.k_weight, self.q_weight = as_dev(k_weight), as_dev(q_weight)
+        self.desc = wushkv_prologue(_ptr(self.table), n_positions, 1 if normalise else 0, _ptr(self.k_weight),
+                                    _ptr(self.q_weight), float(eps))
+
+
+def append_projected(cache: wushkv_cache, batch, slot, seq_len, cu_new, total_new, max_new, K_proj, V_new,
+                     prologue: wushkv_prologue, stream=None):
+    """wushkv_append_projected: wushkv_append on projected keys (Norm and RoPE applied inside the kernels)."""
+    _check(lib.wushkv_append_projected(C.byref(cache), batch, _ptr(slot), _ptr(seq_len), _ptr(cu_new), total_new, max_new,
+                                       _ptr(K_proj), _ptr(V_new), C.byref(prologue), _stream_ptr(stream)),
+           "wushkv_append_projected")
+
+
+def decode_attn_projected(cache: wushkv_cache, batch, slot, seq_len, max_seq_len, Q_proj, prologue: wushkv_prologue, O,
+                          workspace, workspace_bytes, stream=None):
+    """wushkv_decode_attn_projected: wushkv_decode_attn on projected queries."""
+    _check(lib.wushkv_decode_attn_projected(C.byref(cache), batch, _ptr(slot), _ptr(seq_len), max_seq_len, _ptr(Q_proj),
+                                            C.byref(prologue), _ptr(O), _ptr(workspace), workspace_bytes,
+                                            _stream_ptr(stream)), "wushkv_decode_attn_projected")
 
 
 def decode_workspace_bytes(cache: wushkv_cache, batch: int, max_seq_len: int) -> int:

@@ -19,6 +19,7 @@
 #include <cstdlib>
 
 #include "host_common.h"
+#include "prologue.cuh"
 #include "layout.cuh"
 
 namespace wushkv {
@@ -46,6 +47,7 @@ struct AppendParams {
     ClipRule rule_k, rule_v;
     int wait_limit;          // poll limit of the chunk kernel's MMA barrier wait (0: default, about two seconds)
     int drop_mma_commit;     // testing aid: the first tile's MMAs are never committed to their barrier
+    Prologue pro;            // pro.rope != nullptr: K_new holds projected keys, normalised and rotated here (Algorithm 2 lines 1-2)
 };
 
 __device__ __forceinline__ void cswap_desc(unsigned& a, unsigned& b) {
@@ -234,6 +236,7 @@ __global__ void __launch_bounds__(256) append_rows_kernel(AppendParams P) {
         const uint2 kraw = __ldg(reinterpret_cast<const uint2*>(P.K_new + row) + lane);
         float kin[4] = {bf16_bits_to_float(kraw.x & 0xffff), bf16_bits_to_float(kraw.x >> 16),
                         bf16_bits_to_float(kraw.y & 0xffff), bf16_bits_to_float(kraw.y >> 16)};
+        if (P.pro.rope) norm_rope_warp(kin, lane, P.pro, head, prologue_position(P.pro, ts.pos, P.c.dev_status, lane == 0));
         float x[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 4
         for (int jj = 0; jj < 32; ++jj) {
@@ -300,6 +303,16 @@ __global__ void __launch_bounds__(1024) append_token_kernel(AppendParams P) {
     if (warp >= n_kv && warp < 2 * n_kv) v_pre = __ldg(reinterpret_cast<const uint2*>(P.V_new + row0 + (warp - n_kv) * D) + lane);
     for (int idx = threadIdx.x; idx < n_kv * D; idx += blockDim.x) kin_s[idx] = bf16_bits_to_float(__ldg(P.K_new + row0 + idx));
     __syncthreads();
+    if (P.pro.rope) {                                    // projected keys: Norm and RoPE first, one warp per head
+        for (int h = warp; h < n_kv; h += nwarps) {
+            float4* kv = reinterpret_cast<float4*>(kin_s + h * D) + lane;
+            const float4 v = *kv;
+            float x[4] = {v.x, v.y, v.z, v.w};
+            norm_rope_warp(x, lane, P.pro, h, prologue_position(P.pro, s0, P.c.dev_status, lane == 0 && h == 0));
+            *kv = make_float4(x[0], x[1], x[2], x[3]);
+        }
+        __syncthreads();
+    }
     // k'[h][i] = sum_j T[h][i][j] k[h][j]: a warp takes 32 consecutive rows of one head; every row is
     // read as one coalesced 512-byte line (lane L holds columns 4L..4L+3), the 32 partial sums per lane
     // are then reduced across lanes with a transposing butterfly.
@@ -608,6 +621,65 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
             rows[tid] = ri;
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
+        if (P.pro.rope) {
+            // Projected keys: normalise and rotate the staged tile in place (Algorithm 2 lines 1-2).  Four threads
+            // share a row; thread q of a row owns channels 16q..16q+15 and their rotation partners 64+16q..64+16q+15,
+            // i.e. k chunks 2q, 2q+1, 8+2q, 9+2q of the operand layout.
+            __syncthreads();                                  // the copies and the row records of the other threads
+            const int row = tid >> 2, q = tid & 3;
+            const RowInfo ri = rows[row];
+            unsigned char* base = sA + (row >> 3) * TC_SBO + (row & 7) * 16;
+            uint4 raw[4];
+            raw[0] = *reinterpret_cast<const uint4*>(base + (2 * q) * TC_LBO);
+            raw[1] = *reinterpret_cast<const uint4*>(base + (2 * q + 1) * TC_LBO);
+            raw[2] = *reinterpret_cast<const uint4*>(base + (8 + 2 * q) * TC_LBO);
+            raw[3] = *reinterpret_cast<const uint4*>(base + (9 + 2 * q) * TC_LBO);
+            float a[16], b[16];
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const unsigned wa[4] = {raw[k].x, raw[k].y, raw[k].z, raw[k].w}, wb[4] = {raw[2 + k].x, raw[2 + k].y, raw[2 + k].z, raw[2 + k].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    a[8 * k + 2 * e] = bf16_bits_to_float(wa[e] & 0xffff); a[8 * k + 2 * e + 1] = bf16_bits_to_float(wa[e] >> 16);
+                    b[8 * k + 2 * e] = bf16_bits_to_float(wb[e] & 0xffff); b[8 * k + 2 * e + 1] = bf16_bits_to_float(wb[e] >> 16);
+                }
+            }
+            if (P.pro.normalise) {
+                float ss = 0.f;
+#pragma unroll
+                for (int e = 0; e < 16; ++e) ss = fmaf(a[e], a[e], fmaf(b[e], b[e], ss));
+                ss += __shfl_xor_sync(FULL, ss, 1);
+                ss += __shfl_xor_sync(FULL, ss, 2);
+                const float r = ss > 0.f ? 1.f / sqrtf(ss * (1.f / D) + P.pro.eps) : 0.f;
+                if (P.pro.weight) {
+                    const float4* wa = reinterpret_cast<const float4*>(P.pro.weight + static_cast<long long>(head) * D + 16 * q);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float4 u = __ldg(wa + e), v = __ldg(wa + 16 + e);
+                        a[4 * e] *= r * u.x; a[4 * e + 1] *= r * u.y; a[4 * e + 2] *= r * u.z; a[4 * e + 3] *= r * u.w;
+                        b[4 * e] *= r * v.x; b[4 * e + 1] *= r * v.y; b[4 * e + 2] *= r * v.z; b[4 * e + 3] *= r * v.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) { a[e] *= r; b[e] *= r; }
+                }
+            }
+            const int pos = prologue_position(P.pro, ri.pos, P.c.dev_status, ri.rec_off >= 0 && q == 0);
+            const float4* tab = reinterpret_cast<const float4*>(P.pro.rope + static_cast<long long>(pos) * (D / 2) + 16 * q);
+            unsigned outa[8], outb[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float4 cs = __ldg(tab + e);             // (cos, sin) of pairs 16q + 2e, 16q + 2e + 1
+                const float ya0 = fmaf(a[2 * e], cs.x, -b[2 * e] * cs.y), yb0 = fmaf(a[2 * e], cs.y, b[2 * e] * cs.x);
+                const float ya1 = fmaf(a[2 * e + 1], cs.z, -b[2 * e + 1] * cs.w), yb1 = fmaf(a[2 * e + 1], cs.w, b[2 * e + 1] * cs.z);
+                outa[e] = float_to_bf16_bits(ya0) | (static_cast<unsigned>(float_to_bf16_bits(ya1)) << 16);
+                outb[e] = float_to_bf16_bits(yb0) | (static_cast<unsigned>(float_to_bf16_bits(yb1)) << 16);
+            }
+            *reinterpret_cast<uint4*>(base + (2 * q) * TC_LBO) = make_uint4(outa[0], outa[1], outa[2], outa[3]);
+            *reinterpret_cast<uint4*>(base + (2 * q + 1) * TC_LBO) = make_uint4(outa[4], outa[5], outa[6], outa[7]);
+            *reinterpret_cast<uint4*>(base + (8 + 2 * q) * TC_LBO) = make_uint4(outb[0], outb[1], outb[2], outb[3]);
+            *reinterpret_cast<uint4*>(base + (9 + 2 * q) * TC_LBO) = make_uint4(outb[4], outb[5], outb[6], outb[7]);
+        }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // generic-proxy writes -> visible to the tensor core
         __syncthreads();
         // ---- one thread issues the 8 k-steps and commits them to the barrier
@@ -931,12 +1003,14 @@ static ClipRule make_rule(float kappa) {
 
 using namespace wushkv;
 
-extern "C" int wushkv_append(const wushkv_cache* cache, int32_t batch, const int32_t* slot, int32_t* seq_len,
-                             const int32_t* cu_new, int32_t total_new, int32_t max_new,
-                             const uint16_t* K_new, const uint16_t* V_new, void* stream) {
+static int append_impl(const wushkv_cache* cache, int32_t batch, const int32_t* slot, int32_t* seq_len,
+                       const int32_t* cu_new, int32_t total_new, int32_t max_new,
+                       const uint16_t* K_new, const uint16_t* V_new, const wushkv_prologue* prologue, void* stream) {
     AppendParams P;
     const int rc = make_view(cache, P.c);
     if (rc != WUSHKV_OK) return rc;
+    P.pro = Prologue{nullptr, 0, 0, nullptr, 0.f};
+    if (prologue && !make_prologue(prologue, prologue->k_norm_weight, P.pro)) return WUSHKV_EINVAL;
     if (batch <= 0 || !slot || !seq_len || !cu_new || total_new < 0 || max_new < 0 || max_new > total_new) return WUSHKV_EINVAL;
     if (total_new == 0) return WUSHKV_OK;
     if (!K_new || !V_new || !aligned(K_new, 16) || !aligned(V_new, 16)) return WUSHKV_EINVAL;
@@ -1021,6 +1095,37 @@ extern "C" int wushkv_append(const wushkv_cache* cache, int32_t batch, const int
     advance_len_kernel<<<(batch + 127) / 128, 128, 0, st>>>(P.c, batch, slot, seq_len, cu_new);
     if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
     return WUSHKV_OK;
+}
+
+extern "C" int wushkv_append(const wushkv_cache* cache, int32_t batch, const int32_t* slot, int32_t* seq_len,
+                             const int32_t* cu_new, int32_t total_new, int32_t max_new,
+                             const uint16_t* K_new, const uint16_t* V_new, void* stream) {
+    return append_impl(cache, batch, slot, seq_len, cu_new, total_new, max_new, K_new, V_new, nullptr, stream);
+}
+
+extern "C" int wushkv_append_projected(const wushkv_cache* cache, int32_t batch, const int32_t* slot, int32_t* seq_len,
+                                       const int32_t* cu_new, int32_t total_new, int32_t max_new,
+                                       const uint16_t* K_proj, const uint16_t* V_new, const wushkv_prologue* prologue, void* stream) {
+    if (!prologue) return WUSHKV_EINVAL;
+    return append_impl(cache, batch, slot, seq_len, cu_new, total_new, max_new, K_proj, V_new, prologue, stream);
+}
+
+// cosines and sines of position * theta^(-2j/d) in double precision, rounded to fp32
+__global__ void rope_table_kernel(double theta, int n_pos, float2* table) {
+    const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (idx >= static_cast<long long>(n_pos) * (D / 2)) return;
+    const int j = static_cast<int>(idx % (D / 2));
+    const double pos = static_cast<double>(idx / (D / 2));
+    double sn, cs;
+    sincos(pos * pow(theta, -2.0 * j / D), &sn, &cs);
+    table[idx] = make_float2(static_cast<float>(cs), static_cast<float>(sn));
+}
+
+extern "C" int wushkv_build_rope_table(double theta, int32_t n_positions, int32_t d, float* table, void* stream) {
+    if (!(theta > 0.0) || n_positions <= 0 || d != D || !table || !aligned(table, 16)) return WUSHKV_EINVAL;
+    const long long n = static_cast<long long>(n_positions) * (D / 2);
+    rope_table_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(theta, n_positions, reinterpret_cast<float2*>(table));
+    return cudaGetLastError() == cudaSuccess ? WUSHKV_OK : WUSHKV_ECUDA;
 }
 
 extern "C" int wushkv_unpack_debug(const wushkv_cache* cache, int32_t slot, int32_t kv_head, int32_t which,

@@ -37,6 +37,7 @@
 #include <cstdlib>
 
 #include "host_common.h"
+#include "prologue.cuh"
 #include "layout.cuh"
 
 namespace wushkv {
@@ -85,6 +86,7 @@ struct DecodeParams {
     long long drop_unit; // testing aid: flattened index of a unit whose copy is never issued (-1: none)
     int q_early;         // 1: Q was final before the kernel ahead of the preparation kernel started
     int stream_pages;    // 1: the packed pages of a step cannot stay in L2 anyway: copy them with an evict-first hint
+    Prologue pro;        // pro.rope != nullptr: Q holds projected queries, normalised and rotated by the preparation kernel
 };
 
 // shift of the code field used by k-step / channel block idx (0..7) inside its 16-bit lane, after
@@ -151,6 +153,17 @@ __global__ void __launch_bounds__(PREP_THREADS) decode_prep_kernel(DecodeParams 
     for (int k = i; k < G * D; k += PREP_THREADS)
         q_s[k >> 7][k & (D - 1)] = bf16_bits_to_float(P.Q[(static_cast<long long>(b) * P.c.n_q + h * G) * D + k]);
     __syncthreads();
+    if (P.pro.rope) {                     // projected queries: Norm and RoPE at the newest position (Algorithm 2 lines 1-2)
+        if (warp < G) {
+            const int S = __ldcg(P.seq_len + b);
+            float4* qv = reinterpret_cast<float4*>(&q_s[warp][0]) + lane;
+            const float4 v = *qv;
+            float x[4] = {v.x, v.y, v.z, v.w};
+            norm_rope_warp(x, lane, P.pro, h * G + warp, prologue_position(P.pro, max(S - 1, 0), P.c.dev_status, lane == 0 && S > P.pro.n_pos));
+            *qv = make_float4(x[0], x[1], x[2], x[3]);
+        }
+        __syncthreads();
+    }
     // q'[g][i] = sum_j T_invT[h][i][j] q[g][j].  Each of the 16 warps takes 8 rows, all of their loads in
     // flight together; a row is one coalesced 512-byte read (lane L holds columns 4L..4L+3); rows are
     // handled 32/GP at a time so that the GP x rows partial sums fit a 32-value transposing butterfly
@@ -1123,7 +1136,8 @@ extern "C" size_t wushkv_decode_workspace_bytes(const wushkv_cache* cache, int32
 
 static int decode_attn_impl(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
                             int32_t max_seq_len, const uint16_t* Q, float* O,
-                            void* workspace, size_t workspace_bytes, void* stream, int q_early) {
+                            void* workspace, size_t workspace_bytes, void* stream, int q_early,
+                            const wushkv_prologue* prologue = nullptr) {
     DecodeParams P;
     P.q_early = q_early;
     const int rc = make_view(cache, P.c);
@@ -1143,6 +1157,8 @@ static int decode_attn_impl(const wushkv_cache* cache, int32_t batch, const int3
     P.n_warps = pl.n_warps;
     P.wait_limit = static_cast<int>(std::min<long long>(std::max<long long>(knobs().wait_limit, 0), 1 << 30));
     P.drop_unit = knobs().drop_copy_unit;
+    P.pro = Prologue{nullptr, 0, 0, nullptr, 0.f};
+    if (prologue && !make_prologue(prologue, prologue->q_norm_weight, P.pro)) return WUSHKV_EINVAL;
     {   // upper bound of the packed bytes one step reads against the L2 size
         static int l2_bytes[64] = {};
         int dev = 0;
@@ -1166,6 +1182,14 @@ extern "C" int wushkv_decode_attn(const wushkv_cache* cache, int32_t batch, cons
                                   int32_t max_seq_len, const uint16_t* Q, float* O,
                                   void* workspace, size_t workspace_bytes, void* stream) {
     return decode_attn_impl(cache, batch, slot, seq_len, max_seq_len, Q, O, workspace, workspace_bytes, stream, 0);
+}
+
+extern "C" int wushkv_decode_attn_projected(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
+                                            int32_t max_seq_len, const uint16_t* Q_proj, const wushkv_prologue* prologue, float* O,
+                                            void* workspace, size_t workspace_bytes, void* stream) {
+    if (!prologue) return WUSHKV_EINVAL;
+    // the query's position is the final length minus one: the preparation kernel waits for the kernel ahead of it
+    return decode_attn_impl(cache, batch, slot, seq_len, max_seq_len, Q_proj, O, workspace, workspace_bytes, stream, 0, prologue);
 }
 
 extern "C" int wushkv_decode_step(const wushkv_cache* cache, int32_t batch, const int32_t* slot, int32_t* seq_len,

@@ -198,6 +198,16 @@ class LayerWorkload:
             entropy=self._ss_qry.entropy, spawn_key=self._ss_qry.spawn_key + (int(b), 1)))
         return self._queries(rng, np.asarray(positions))
 
+    def projected(self, b, n_tokens):
+        """Projected (pre-Norm, pre-RoPE) keys [n][n_kv][d] and queries [n][n_q][d] of sequence ``b``: the same
+        channel-scaled Gaussians the other draws start from, rounded to bf16, for callers that apply
+        normalisation and rotation themselves."""
+        rng = np.random.default_rng(np.random.SeedSequence(
+            entropy=self._ss_tok.entropy, spawn_key=self._ss_tok.spawn_key + (int(b), 2)))
+        k = rng.standard_normal((n_tokens, self.n_kv, self.d), dtype=np.float32) * self.s_k[None]
+        q = rng.standard_normal((n_tokens, self.n_q, self.d), dtype=np.float32) * self.s_q[None] * self.alpha[None, :, None]
+        return bf16_round_f32(k), bf16_round_f32(q)
+
     def queries(self, b, position):
         """The decode-step query of sequence ``b`` at ``position``: [n_q][d] bf16-valued float32."""
         rng = np.random.default_rng(np.random.SeedSequence(

@@ -66,6 +66,7 @@ class Layer:
             self.tokens.append((np.concatenate(ks) if ks else np.zeros((0, wl.n_kv, 128), np.float32),
                                 np.concatenate(vs) if vs else np.zeros((0, wl.n_kv, 128), np.float32)))
         self.done = [0] * self.batch
+        self.prologue = None          # a binding.Prologue: appends then go through wushkv_append_projected
 
     def append_step(self, counts, oracle_too=True):
         """Append counts[b] new tokens to sequence b on the GPU (one library call) and in the oracle."""
@@ -86,7 +87,11 @@ class Layer:
             Vn = torch.from_numpy(W.f32_to_bf16_bits(np.concatenate(Vs)).view(np.int16)).to(self.cache.device)
         else:
             Kn = Vn = torch.zeros(8, dtype=torch.int16, device=self.cache.device)
-        B.append(self.cache.desc, self.batch, self.slot, self.seq_len, cu, total, max(counts), Kn, Vn)
+        if self.prologue is not None:
+            B.append_projected(self.cache.desc, self.batch, self.slot, self.seq_len, cu, total, max(counts), Kn, Vn,
+                               self.prologue.desc)
+        else:
+            B.append(self.cache.desc, self.batch, self.slot, self.seq_len, cu, total, max(counts), Kn, Vn)
         torch.cuda.synchronize()
 
     def fill(self, last_step=1):
@@ -148,8 +153,9 @@ class Layer:
                 vb[p] = ring[:, 1, p % c.ring_cap]
         return kb, vb
 
-    def decode(self, queries=None):
-        """One decode step on the GPU; returns (O_gpu [batch][n_q][128], Q float32 used)."""
+    def decode(self, queries=None, projected=False):
+        """One decode step on the GPU; returns (O_gpu [batch][n_q][128], Q float32 used).  ``projected``: the
+        queries are projected ones and go through wushkv_decode_attn_projected with this layer's prologue."""
         torch, B = self.torch, self.B
         if queries is None:
             queries = np.stack([self.wl.queries(b, max(self.lengths[b] - 1, 0)) for b in range(self.batch)])
@@ -158,7 +164,11 @@ class Layer:
         nbytes = B.decode_workspace_bytes(self.cache.desc, self.batch, self.max_seq_len)
         assert nbytes > 0
         ws = torch.empty(nbytes, dtype=torch.uint8, device=self.cache.device)
-        B.decode_attn(self.cache.desc, self.batch, self.slot, self.seq_len, self.max_seq_len, Q, Oo, ws, nbytes)
+        if projected:
+            B.decode_attn_projected(self.cache.desc, self.batch, self.slot, self.seq_len, self.max_seq_len, Q,
+                                    self.prologue.desc, Oo, ws, nbytes)
+        else:
+            B.decode_attn(self.cache.desc, self.batch, self.slot, self.seq_len, self.max_seq_len, Q, Oo, ws, nbytes)
         torch.cuda.synchronize()
         return Oo.cpu().numpy().astype(np.float64), queries
 
