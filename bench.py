@@ -43,8 +43,8 @@ FALLBACK_HBM_GBS = 6650.0
 L2_BYTES = 126 * 2 ** 20
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel at the named workload,
 # from one ncu capture each (None where not captured).
-NCU_TRAFFIC_BYTES = {"cfg1": 310668544 + 3688960, "cfg2": 362961408 + 3549440,
-                     "cfg3": 76140032 + 3253760, "cfg4": None}
+NCU_TRAFFIC_BYTES = {"cfg1": 314262000, "cfg2": 365696000, "cfg3": 78262000,
+                     "cfg4": 134600000 + 13600000}
 
 
 def measured_tensor_peak():

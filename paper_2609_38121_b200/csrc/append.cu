@@ -269,89 +269,90 @@ __global__ void __launch_bounds__(256) append_rows_kernel(AppendParams P) {
     }
 }
 
-// Decode-time append: exactly one new token per sequence (or none).  One CTA per sequence handles
-// all KV heads: every thread computes outputs of k' = T_K k as a row dot product (the rows of T_K
-// come straight from L2), then one warp per vector quantizes and packs keys and values.  The CTA
-// is the only reader of its sequence's length, so it also advances it: no second launch.
+// Decode-time append: exactly one new token per sequence (or none).  One CTA of four warps per (KV head,
+// sequence); the CTAs of a sequence form a thread-block cluster.  Every warp computes 32 outputs of
+// k' = T_K k as row dot products (the rows of T_K come straight from L2, 64 KB per CTA, so the read is
+// spread over n_kv SMs per sequence instead of one), then one warp quantizes and packs the key, another
+// the value.  The cluster is the only reader of its sequence's length, so it also advances it: every CTA
+// reads the old length, the cluster meets at its barrier, then the first CTA stores the new one.
 template <int BITS>
-__global__ void __launch_bounds__(1024) append_token_kernel(AppendParams P) {
-    extern __shared__ __align__(16) float tok_s[];       // [n_kv][128] input key, [n_kv][128] transformed key
+__global__ void __launch_bounds__(128) append_token_kernel(AppendParams P) {
+    __shared__ __align__(16) float kin_s[D];             // input key
+    __shared__ __align__(16) float kp_s[D];              // transformed key
     // Launched programmatically: the CTAs may be resident before the kernel ahead in the stream has
     // finished, so wait for it (and its memory) first; then let the next kernel's CTAs come in early
     // too (that kernel waits for this one itself).
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const int b = blockIdx.x;
+    const int head = blockIdx.x, b = blockIdx.y;
     const int n_kv = P.c.n_kv;
-    float* kin_s = tok_s;
-    float* kp_s = tok_s + n_kv * D;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int first = __ldg(P.cu_new + b), n_new = __ldg(P.cu_new + b + 1) - first;
-    if (n_new <= 0) return;
-    if (n_new > 1) {                                     // the host promised one token per sequence
-        if (threadIdx.x == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_COUNT);
-        return;
+    const int s0 = n_new > 0 ? P.seq_len[b] : 0;         // written by this cluster: not through the read-only path
+    // every CTA of the sequence has read the old length once all have arrived here
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    bool ok = n_new == 1;
+    if (n_new > 1 && threadIdx.x == 0 && head == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_COUNT);   // the host promised one token per sequence
+    int slot0 = 0, page = -1;
+    if (ok) {
+        slot0 = __ldg(P.slot + b);                       // the page lookup does not depend on the transform: start it now
+        if (slot0 >= 0 && slot0 < P.c.n_slots && s0 >= 0 && s0 / PAGE_TOKENS < P.c.max_pages)
+            page = __ldg(P.c.page_table + static_cast<long long>(slot0) * P.c.max_pages + s0 / PAGE_TOKENS);
     }
-    const int s0 = P.seq_len[b];                         // written by this kernel: not through the read-only path
-    const int slot0 = __ldg(P.slot + b);                 // the page lookup does not depend on the transform: start it now
-    int page = -1;
-    if (slot0 >= 0 && slot0 < P.c.n_slots && s0 >= 0 && s0 / PAGE_TOKENS < P.c.max_pages)
-        page = __ldg(P.c.page_table + static_cast<long long>(slot0) * P.c.max_pages + s0 / PAGE_TOKENS);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    const long long row0 = static_cast<long long>(first) * n_kv * D;
-    // a warp that will quantize a value vector requests it now; it is used after the transform
-    uint2 v_pre = make_uint2(0u, 0u);
-    if (warp >= n_kv && warp < 2 * n_kv) v_pre = __ldg(reinterpret_cast<const uint2*>(P.V_new + row0 + (warp - n_kv) * D) + lane);
-    for (int idx = threadIdx.x; idx < n_kv * D; idx += blockDim.x) kin_s[idx] = bf16_bits_to_float(__ldg(P.K_new + row0 + idx));
-    __syncthreads();
-    if (P.pro.rope) {                                    // projected keys: Norm and RoPE first, one warp per head
-        for (int h = warp; h < n_kv; h += nwarps) {
-            float4* kv = reinterpret_cast<float4*>(kin_s + h * D) + lane;
-            const float4 v = *kv;
-            float x[4] = {v.x, v.y, v.z, v.w};
-            norm_rope_warp(x, lane, P.pro, h, prologue_position(P.pro, s0, P.c.dev_status, lane == 0 && h == 0));
-            *kv = make_float4(x[0], x[1], x[2], x[3]);
+    if (ok) {
+        const long long row0 = (static_cast<long long>(first) * n_kv + head) * D;
+        // the warp that will quantize the value vector requests it now; it is used after the transform
+        uint2 v_pre = make_uint2(0u, 0u);
+        if (warp == 1) v_pre = __ldg(reinterpret_cast<const uint2*>(P.V_new + row0) + lane);
+        kin_s[threadIdx.x] = bf16_bits_to_float(__ldg(P.K_new + row0 + threadIdx.x));
+        __syncthreads();
+        if (P.pro.rope) {                                // projected keys: Norm and RoPE first
+            if (warp == 0) {
+                float4* kv = reinterpret_cast<float4*>(kin_s) + lane;
+                const float4 v = *kv;
+                float x[4] = {v.x, v.y, v.z, v.w};
+                norm_rope_warp(x, lane, P.pro, head, prologue_position(P.pro, s0, P.c.dev_status, lane == 0 && head == 0));
+                *kv = make_float4(x[0], x[1], x[2], x[3]);
+            }
+            __syncthreads();
+        }
+        // k'[i] = sum_j T[i][j] k[j]: a warp takes 32 consecutive rows; every row is read as one coalesced
+        // 512-byte line (lane L holds columns 4L..4L+3), the 32 partial sums per lane are then reduced across
+        // lanes with a transposing butterfly.
+        {
+            const int r0 = warp * 32;
+            const float4 kv = *reinterpret_cast<const float4*>(kin_s + 4 * lane);
+            const float4* Tbase = reinterpret_cast<const float4*>(P.c.T_K + (static_cast<long long>(head) * D + r0) * D) + lane;
+            float part[32];
+#pragma unroll
+            for (int r = 0; r < 32; ++r) {
+                const float4 t = __ldg(Tbase + r * (D / 4));
+                part[r] = fmaf(t.x, kv.x, fmaf(t.y, kv.y, fmaf(t.z, kv.z, t.w * kv.w)));
+            }
+            kp_s[r0 + lane] = warp_transpose_reduce(part, lane);
         }
         __syncthreads();
-    }
-    // k'[h][i] = sum_j T[h][i][j] k[h][j]: a warp takes 32 consecutive rows of one head; every row is
-    // read as one coalesced 512-byte line (lane L holds columns 4L..4L+3), the 32 partial sums per lane
-    // are then reduced across lanes with a transposing butterfly.
-    for (int task = warp; task < n_kv * 4; task += nwarps) {
-        const int h = task >> 2, r0 = (task & 3) * 32;
-        const float4 kv = *reinterpret_cast<const float4*>(kin_s + h * D + 4 * lane);
-        const float4* Tbase = reinterpret_cast<const float4*>(P.c.T_K + (static_cast<long long>(h) * D + r0) * D) + lane;
-        float part[32];
-#pragma unroll
-        for (int r = 0; r < 32; ++r) {
-            const float4 t = __ldg(Tbase + r * (D / 4));
-            part[r] = fmaf(t.x, kv.x, fmaf(t.y, kv.y, fmaf(t.z, kv.z, t.w * kv.w)));
+        TokenSlot ts;
+        ts.b = b; ts.slot = slot0; ts.pos = s0; ts.s_final = s0 + 1;
+        if (ts.slot < 0 || ts.slot >= P.c.n_slots || s0 < 0) { if (threadIdx.x == 0 && head == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_SLOT); ok = false; }
+        if (ok) {
+            const int pidx = ts.pos / PAGE_TOKENS;
+            if (pidx >= P.c.max_pages) { if (threadIdx.x == 0 && head == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_PAGE_TABLE_FULL); ok = false; }
+            else if (page < 0 || page >= P.c.n_pages) { if (threadIdx.x == 0 && head == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_PAGE_ID); ok = false; }
         }
-        kp_s[h * D + r0 + lane] = warp_transpose_reduce(part, lane);
-    }
-    __syncthreads();
-    TokenSlot ts;
-    ts.b = b; ts.slot = slot0; ts.pos = s0; ts.s_final = s0 + 1;
-    bool ok = true;
-    if (ts.slot < 0 || ts.slot >= P.c.n_slots || s0 < 0) { if (threadIdx.x == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_SLOT); ok = false; }
-    if (ok) {
-        const int pidx = ts.pos / PAGE_TOKENS;
-        if (pidx >= P.c.max_pages) { if (threadIdx.x == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_PAGE_TABLE_FULL); ok = false; }
-        else if (page < 0 || page >= P.c.n_pages) { if (threadIdx.x == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_BAD_PAGE_ID); ok = false; }
-    }
-    if (ok) {
-        ts.r = ts.pos % PAGE_TOKENS;
-        for (int v = warp; v < 2 * n_kv; v += nwarps) {
-            const int which = v >= n_kv ? 1 : 0, head = which ? v - n_kv : v;
+        if (ok && warp < 2) {
+            const int which = warp;                      // warp 0: key, warp 1: value
+            ts.r = ts.pos % PAGE_TOKENS;
             ts.rec = P.c.pages + (static_cast<long long>(page) * n_kv + head) * record_bytes(BITS);
             float x[4];
             uint2 copy;
             if (which == 0) {
-                const float4 kp = *reinterpret_cast<const float4*>(kp_s + head * D + 4 * lane);
+                const float4 kp = *reinterpret_cast<const float4*>(kp_s + 4 * lane);
                 x[0] = kp.x; x[1] = kp.y; x[2] = kp.z; x[3] = kp.w;
                 copy.x = float_to_bf16_bits(x[0]) | (static_cast<unsigned>(float_to_bf16_bits(x[1])) << 16);
                 copy.y = float_to_bf16_bits(x[2]) | (static_cast<unsigned>(float_to_bf16_bits(x[3])) << 16);
             } else {
-                copy = (v == warp) ? v_pre : __ldg(reinterpret_cast<const uint2*>(P.V_new + row0 + head * D) + lane);
+                copy = v_pre;
                 x[0] = bf16_bits_to_float(copy.x & 0xffff); x[1] = bf16_bits_to_float(copy.x >> 16);
                 x[2] = bf16_bits_to_float(copy.y & 0xffff); x[3] = bf16_bits_to_float(copy.y >> 16);
             }
@@ -364,7 +365,9 @@ __global__ void __launch_bounds__(1024) append_token_kernel(AppendParams P) {
             store_window_copy(P, ts, head, which, copy, lane);
         }
     }
-    if (ok && threadIdx.x == 0) P.seq_len[b] = s0 + 1;    // every read of the old length happened before the barriers above
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    // the conditions that clear `ok` are the same for every head of the sequence, so the first CTA decides for all
+    if (ok && head == 0 && threadIdx.x == 0) P.seq_len[b] = s0 + 1;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -470,7 +473,7 @@ template <int BITS, int KK>
 __device__ __forceinline__ void quad_quantize(const float (&x)[32], ClipRule rule, int (&code)[32], __half& step_h, __half& xmin_h,
                                               int* value_status = nullptr, bool flag_lane = false) {
     constexpr int LEVELS = (1 << BITS) - 1;
-    if (rule.quest > 0.f) {                     // Eq. 5 (see quantize_vec)
+    if constexpr (KK < 0) {                     // Eq. 5 (see quantize_vec); a compile-time choice keeps it out of the Eq. 6 kernels
         float ss = 0.f;
 #pragma unroll
         for (int i = 0; i < 32; ++i) ss = fmaf(x[i], x[i], ss);
@@ -487,8 +490,7 @@ __device__ __forceinline__ void quad_quantize(const float (&x)[32], ClipRule rul
             const float t = fminf(fmaxf(floorf(x[i] * inv) + HALF, 0.f), static_cast<float>(LEVELS));
             code[i] = step_s > 0.f ? static_cast<int>(t) : 0;
         }
-        return;
-    }
+    } else {
     unsigned top[KK];
 #pragma unroll
     for (int g0 = 0; g0 < 32; g0 += KK) {
@@ -538,10 +540,11 @@ __device__ __forceinline__ void quad_quantize(const float (&x)[32], ClipRule rul
         const float t = fminf(fmaxf((x[i] - xmin_s) * inv, 0.f), static_cast<float>(LEVELS));
         code[i] = static_cast<int>(__float_as_uint(t + 12582912.f) & 0xFu);
     }
+    }
 }
 
-// KK_K / KK_V: list length of the quad quantizer for keys / values (8 or 16, >= the rule's rounds), or 0 for
-// the warp-per-vector quantizer (any kappa).
+// KK_K / KK_V: list length of the quad quantizer for keys / values (8 or 16, >= the rule's rounds), 0 for
+// the warp-per-vector quantizer (any kappa), or -1 for the QuEST rule (Eq. 5, no order statistics).
 template <int BITS, int KK_K, int KK_V>
 __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParams P) {
     extern __shared__ __align__(1024) unsigned char tc_smem[];
@@ -601,7 +604,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
                 cp_async16(smem_addr_u32(sA + rg * TC_SBO + kc * TC_LBO + r8 * 16),
                            P.K_new + (static_cast<long long>(in_range ? tok : 0) * P.c.n_kv + head) * D + kc * 8, in_range ? 16u : 0u);
             }
-            if (KK_V > 0) {
+            if (KK_V != 0) {
                 for (int item = tid; item < TC_TILE * 16; item += TC_THREADS) {
                     const int row = item >> 4, ch = item & 15;
                     const bool in_range = tok0 + row < P.total_new;
@@ -700,8 +703,8 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
                 asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr_u32(mbar)) : "memory");
         }
         // ---- while the tensor core runs: values of this tile (no transform)
-        if (KK_V > 0) {
-            constexpr int KQ = KK_V > 0 ? KK_V : 8;
+        if (KK_V != 0) {
+            constexpr int KQ = KK_V != 0 ? KK_V : 8;
             const int row = 8 * warp + (lane >> 2), qd = lane & 3;
             const RowInfo ri = rows[row];
             const bool live = ri.rec_off >= 0;
@@ -825,8 +828,8 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
         // ---- keys of this tile: quantize the fp32 rows
-        if (KK_K > 0) {
-            constexpr int KQ = KK_K > 0 ? KK_K : 8;
+        if (KK_K != 0) {
+            constexpr int KQ = KK_K != 0 ? KK_K : 8;
             const int row = 8 * warp + (lane >> 2), qd = lane & 3;
             const RowInfo ri = rows[row];
             const bool live = ri.rec_off >= 0;
@@ -1026,20 +1029,21 @@ static int append_impl(const wushkv_cache* cache, int32_t batch, const int32_t* 
     }
     P.wait_limit = static_cast<int>(std::min<long long>(std::max<long long>(knobs().wait_limit, 0), 1 << 30));
     P.drop_mma_commit = knobs().drop_chunk_mma;
-    if (max_new == 1) {                 // decode-time append: one CTA per sequence, single launch
-        const int threads = std::min(1024, P.c.n_kv * D);
-        const size_t smem1 = static_cast<size_t>(2) * P.c.n_kv * D * sizeof(float);
-        if (smem1 > 48 * 1024) return WUSHKV_EINVAL;
-        cudaLaunchAttribute attr[1];
+    if (max_new == 1 && P.c.n_kv <= 8 && batch <= 65535) {    // decode-time append: a cluster of one CTA per KV head for every sequence, single launch
+        cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = P.c.n_kv;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(batch);
-        cfg.blockDim = dim3(threads);
-        cfg.dynamicSmemBytes = smem1;
+        cfg.gridDim = dim3(P.c.n_kv, batch);
+        cfg.blockDim = dim3(128);
+        cfg.dynamicSmemBytes = 0;
         cfg.stream = st;
         cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        cfg.numAttrs = 2;
         const cudaError_t e1 = P.c.bits == 2 ? cudaLaunchKernelEx(&cfg, append_token_kernel<2>, P)
                                              : cudaLaunchKernelEx(&cfg, append_token_kernel<4>, P);
         return e1 == cudaSuccess ? WUSHKV_OK : WUSHKV_ECUDA;
@@ -1051,8 +1055,9 @@ static int append_impl(const wushkv_cache* cache, int32_t batch, const int32_t* 
         const dim3 grid_tc(per_head, P.c.n_kv);
         // list length of the quad quantizer: the rule's rounds must fit (kappa >= ~0.945 -> 8, >= ~0.882 -> 16)
         const int need = std::max(P.rule_k.rounds, P.rule_v.rounds);
-        const int kk_k = need > 16 ? 0 : (P.rule_k.rounds <= 8 ? 8 : 16);
-        const int kk_v = need > 16 ? 0 : (P.rule_v.rounds <= 8 ? 8 : 16);
+        const bool quest = P.rule_k.quest > 0.f;
+        const int kk_k = quest ? -1 : need > 16 ? 0 : (P.rule_k.rounds <= 8 ? 8 : 16);
+        const int kk_v = quest ? -1 : need > 16 ? 0 : (P.rule_v.rounds <= 8 ? 8 : 16);
         auto launch = [&](auto kernel) -> bool {
             if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(kernel), TC_SMEM_TOTAL)) return false;
             kernel<<<grid_tc, TC_THREADS, TC_SMEM_TOTAL, st>>>(P);
@@ -1060,13 +1065,15 @@ static int append_impl(const wushkv_cache* cache, int32_t batch, const int32_t* 
         };
         bool ok;
         if (P.c.bits == 2) {
-            if (kk_k == 0) ok = launch(append_chunk_kernel<2, 0, 0>);
+            if (kk_k < 0) ok = launch(append_chunk_kernel<2, -1, -1>);
+            else if (kk_k == 0) ok = launch(append_chunk_kernel<2, 0, 0>);
             else if (kk_k == 8 && kk_v == 8) ok = launch(append_chunk_kernel<2, 8, 8>);
             else if (kk_k == 8) ok = launch(append_chunk_kernel<2, 8, 16>);
             else if (kk_v == 8) ok = launch(append_chunk_kernel<2, 16, 8>);
             else ok = launch(append_chunk_kernel<2, 16, 16>);
         } else {
-            if (kk_k == 0) ok = launch(append_chunk_kernel<4, 0, 0>);
+            if (kk_k < 0) ok = launch(append_chunk_kernel<4, -1, -1>);
+            else if (kk_k == 0) ok = launch(append_chunk_kernel<4, 0, 0>);
             else if (kk_k == 8 && kk_v == 8) ok = launch(append_chunk_kernel<4, 8, 8>);
             else if (kk_k == 8) ok = launch(append_chunk_kernel<4, 8, 16>);
             else if (kk_v == 8) ok = launch(append_chunk_kernel<4, 16, 8>);
