@@ -86,12 +86,14 @@ def library_transforms(wl):
 class Session:
     """A filled cache plus the per-step inputs of one config, resident on one GPU."""
 
-    def __init__(self, name, n_steps, device="cuda", seed_offset=0, verbose=False):
+    def __init__(self, name, n_steps, device="cuda", seed_offset=0, verbose=False, bits=None):
         import torch
         from paper_2609_38121_b200 import binding as B
         self.torch, self.B = torch, B
         cfg = dict(W.CONFIGS[name])
         cfg["seed"] += 1000 * seed_offset
+        if bits:
+            cfg["bits"] = bits
         self.name, self.cfg = name, cfg
         wl = self.wl = W.LayerWorkload(cfg)
         self.n_steps = n_steps
@@ -218,7 +220,7 @@ class Session:
 
     def decode_bytes(self, step_no=1):
         c = self.cfg
-        per_q = 72 if c["bits"] == 2 else 136
+        per_q = 2 * 128 * c["bits"] // 8 + 8
         total = 0
         for S in self.lengths_at(step_no):
             S = int(S)
@@ -410,7 +412,7 @@ class OracleSample:
 
     def bytes_per_step(self):
         c = self.cfg
-        per_q = 72 if c["bits"] == 2 else 136
+        per_q = 2 * 128 * c["bits"] // 8 + 8
         S = self.S
         nq = max(S - c["s_keep"] - c["s_sink"], 0)
         return nq * per_q + (S - nq) * 512
@@ -513,7 +515,7 @@ def run_ours(args, rank, world):
     torch.cuda.set_device(local)
     K, Wm = args.steps, args.warmup
     n_total_steps = Wm + K            # device-timed region
-    sess = Session(args.config, n_steps=3 * n_total_steps + 2, seed_offset=rank, verbose=(rank == 0 and args.verbose))
+    sess = Session(args.config, n_steps=3 * n_total_steps + 2, seed_offset=rank, verbose=(rank == 0 and args.verbose), bits=args.bits)
     cache_bytes = sess.decode_bytes(1)
     need_flush = cache_bytes < 2 * L2_BYTES
     flush_buf = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device="cuda") if need_flush else None
@@ -656,7 +658,7 @@ def run_ours(args, rank, world):
     if sess.chunk:
         # prefill config: the dominant kernel is the chunk append (tensor-core transform + quantize + pack); its
         # algorithmic bytes are the bf16 keys and values read plus the packed records written
-        per_tok = 2 * 128 * 2 + (72 if sess.cfg["bits"] == 2 else 136)
+        per_tok = 2 * 128 * 2 + 2 * 128 * sess.cfg["bits"] // 8 + 8
         app_bytes = float(sess.append_tokens() * sess.wl.n_kv * per_tok)
         app_s = statistics.mean(append_ms) * 1e-3
         achieved = app_bytes / app_s / 1e9
@@ -674,7 +676,7 @@ def run_ours(args, rank, world):
         roofline = {"bound": "hbm", "kernel": "decode_main_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                     "kernel_ms": kern_s * 1e3, "kernel_ms_min": min(kern_ms), "algorithmic_bytes": bytes_step,
-                    "traffic": NCU_TRAFFIC_BYTES.get(args.config),
+                    "traffic": None if args.bits else NCU_TRAFFIC_BYTES.get(args.config),
                     "kernel_cycles": (kern_s * 1e6 * sm_mhz) if sm_mhz else None}
     roofline_pf = None
     if sess.chunk:
@@ -701,7 +703,7 @@ def run_ours(args, rank, world):
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": args.config, "batch": sess.batch, "n_q": c["n_q"], "n_kv": c["n_kv"], "head_dim": 128,
+        "config": {"workload": args.config + (f"@{args.bits}bit" if args.bits else ""), "batch": sess.batch, "n_q": c["n_q"], "n_kv": c["n_kv"], "head_dim": 128,
                    "context": int(sess.final.max()), "bits": c["bits"], "s_sink": c["s_sink"], "s_keep": c["s_keep"],
                    "s_flush": sess.s_flush, "page_tokens": 64, "prefill_chunk": sess.chunk,
                    "l2": ("flushed between steps (256 MB write)" if need_flush else "cache read per step exceeds L2 (no flush)"),
@@ -728,6 +730,8 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-sustained", action="store_true", help="skip the second-long back-to-back leg")
     ap.add_argument("--sustained-seconds", type=float, default=1.0)
+    ap.add_argument("--bits", type=int, default=0, choices=[0, 2, 3, 4],
+                    help="override the configuration's bit width (0: as the configuration says); the workload name then carries it")
     ap.add_argument("--verbose", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)

@@ -6,7 +6,7 @@
  *       (WUSH closed form, Section 3 Eq. 1, specialised to keys by Eq. 4 / Algorithm 1),
  *   (2) quantize-on-append: k' = T_K k for each new post-RoPE key, values taken as they
  *       are (already in the weight-folded basis, Section 4.2), the per-token
- *       percentile-clipped affine quantizer of Section 5.3 Eq. 6 at 2 or 4 bits, and packing of
+ *       percentile-clipped affine quantizer of Section 5.3 Eq. 6 at 2, 3 or 4 bits, and packing of
  *       codes + (scale, zero) into a paged cache (Algorithm 2 lines 3-4, 9-12),
  *   (3) decode attention over that packed cache for one new query per sequence
  *       (Algorithm 2 lines 3 and 5; Eq. 2; Eq. 3), reading the first S_sink and the most
@@ -26,7 +26,7 @@
  *   - Problems that only the device can see (a position beyond the page table, a page id
  *     outside the pool, a copy that never arrived) never trap: the offending access is
  *     skipped and a bit is OR-ed into *dev_status, which the caller reads when it likes.
- *   - Head dimension d must be 128 and page_tokens must be 64.  bits is 2 or 4.  The query
+ *   - Head dimension d must be 128 and page_tokens must be 64.  bits is 2, 3 or 4 (3-bit codes are stored as a 2-bit plane plus a 1-bit plane: 48 bytes per vector).  The query
  *     group size n_q / n_kv must be an integer between 1 and 8.
  *
  * Conventions

@@ -345,25 +345,25 @@ def quest_quantize(x, bits: int):
 
 
 def pack_codes(codes, bits: int) -> np.ndarray:
-    """Reference bit packing (storage definition only): channel i occupies
-    bits [bits*(i % per), bits*(i % per + 1)) of byte i // per, per = 8/bits.
-    The CUDA library is free to permute its physical layout; parity is checked
-    on logical codes."""
+    """Reference bit packing (storage definition only): the codes of a vector form one little-endian
+    bit stream, channel i occupying stream bits [bits*i, bits*(i+1)); d*bits/8 bytes per vector
+    (32 / 48 / 64 bytes at 2 / 3 / 4 bits for d = 128).  For 2 and 4 bits this is "channel i in bits
+    bits*(i % per) of byte i // per", per = 8/bits.  The CUDA library is free to permute its physical
+    layout; parity is checked on logical codes."""
     codes = np.asarray(codes, dtype=np.uint8)
-    per = 8 // bits
-    c = codes.reshape(codes.shape[:-1] + (codes.shape[-1] // per, per)).astype(np.uint16)
-    out = np.zeros(c.shape[:-1], dtype=np.uint16)
-    for j in range(per):
-        out |= c[..., j] << (bits * j)
-    return out.astype(np.uint8)
+    d = codes.shape[-1]
+    assert (d * bits) % 8 == 0
+    planes = ((codes[..., None] >> np.arange(bits, dtype=np.uint8)) & 1).astype(np.uint8)     # [..., d, bits], low bit first
+    stream = planes.reshape(codes.shape[:-1] + (d * bits,))
+    return np.packbits(stream, axis=-1, bitorder="little")
 
 
 def unpack_codes(packed, bits: int) -> np.ndarray:
     packed = np.asarray(packed, dtype=np.uint8)
-    per = 8 // bits
-    mask = (1 << bits) - 1
-    parts = [(packed >> (bits * j)) & mask for j in range(per)]
-    return np.stack(parts, axis=-1).reshape(packed.shape[:-1] + (packed.shape[-1] * per,))
+    stream = np.unpackbits(packed, axis=-1, bitorder="little")
+    d = stream.shape[-1] // bits
+    planes = stream.reshape(packed.shape[:-1] + (d, bits)).astype(np.uint16)
+    return (planes << np.arange(bits, dtype=np.uint16)).sum(axis=-1).astype(np.uint8)
 
 
 # --------------------------------------------------------------------------

@@ -33,7 +33,7 @@ extern "C" int wushkv_set_test_option(const char* name, long long value) {
 }
 
 extern "C" size_t wushkv_page_bytes(int32_t n_kv, int32_t d, int32_t bits, int32_t page_tokens) {
-    if (n_kv <= 0 || d != wushkv::D || page_tokens != wushkv::PAGE_TOKENS || (bits != 2 && bits != 4)) return 0;
+    if (n_kv <= 0 || d != wushkv::D || page_tokens != wushkv::PAGE_TOKENS || (bits != 2 && bits != 3 && bits != 4)) return 0;
     return static_cast<size_t>(n_kv) * wushkv::record_bytes(bits);
 }
 

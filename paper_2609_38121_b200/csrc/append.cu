@@ -127,39 +127,57 @@ __device__ __forceinline__ void quantize_vec(const float (&x)[4], ClipRule rule,
 // of the word of fragment lane t = 2 (lane & 1) + (e >> 1).
 template <int BITS>
 __device__ __forceinline__ void store_k_codes(unsigned char* rec, int r, const int (&code)[4], int lane) {
+    constexpr bool PLANES = BITS == 3;                  // 3 bits: low two bits here (2-bit layout), high bit below
+    constexpr bool TWO = BITS == 2 || BITS == 3;
     const int bi = r >> 4, rr = r & 15, g = rr & 7, rs = rr >> 3;
     const int s = lane >> 3, b0 = 2 * ((lane >> 1) & 1);
-    const int sh = 8 * b0 + ((BITS == 2) ? 2 * s : 4 * (s & 1));
-    unsigned wa = (static_cast<unsigned>(code[0]) << sh) | (static_cast<unsigned>(code[1]) << (8 + sh));   // t = 2 (lane & 1)
-    unsigned wb = (static_cast<unsigned>(code[2]) << sh) | (static_cast<unsigned>(code[3]) << (8 + sh));   // t = 2 (lane & 1) + 1
+    const int sh = 8 * b0 + (TWO ? 2 * s : 4 * (s & 1));
+    const unsigned lowmask = PLANES ? 3u : 0xFu;
+    unsigned wa = ((static_cast<unsigned>(code[0]) & lowmask) << sh) | ((static_cast<unsigned>(code[1]) & lowmask) << (8 + sh));   // t = 2 (lane & 1)
+    unsigned wb = ((static_cast<unsigned>(code[2]) & lowmask) << sh) | ((static_cast<unsigned>(code[3]) & lowmask) << (8 + sh));   // t = 2 (lane & 1) + 1
     wa |= __shfl_xor_sync(FULL, wa, 2);  wb |= __shfl_xor_sync(FULL, wb, 2);       // the other byte pair
     wa |= __shfl_xor_sync(FULL, wa, 8);  wb |= __shfl_xor_sync(FULL, wb, 8);       // the fields / nibbles of the same byte
-    if (BITS == 2) { wa |= __shfl_xor_sync(FULL, wa, 16); wb |= __shfl_xor_sync(FULL, wb, 16); }
+    if (TWO) { wa |= __shfl_xor_sync(FULL, wa, 16); wb |= __shfl_xor_sync(FULL, wb, 16); }
     const int hh = (lane >> 2) & 1, ta = 2 * (lane & 1), j = rs + 2 * hh;
-    const bool writer = BITS == 2 ? (lane & 26) == 0 : (lane & 10) == 0;
+    const bool writer = TWO ? (lane & 26) == 0 : (lane & 10) == 0;
     if (writer) {
         unsigned char* p = rec + bi * code_block_bytes(BITS) + (BITS == 4 ? 512 * (lane >> 4) : 0) + 16 * (4 * g + ta) + 4 * j;
         *reinterpret_cast<unsigned*>(p) = wa;
         *reinterpret_cast<unsigned*>(p + 16) = wb;
     }
+    if (PLANES) {                                       // 1-bit plane: word rs of lane (g,t), byte b, bit 2s + hh
+        const int shb = 8 * b0 + 2 * s + hh;
+        unsigned ha = ((static_cast<unsigned>(code[0]) >> 2) << shb) | ((static_cast<unsigned>(code[1]) >> 2) << (8 + shb));
+        unsigned hb = ((static_cast<unsigned>(code[2]) >> 2) << shb) | ((static_cast<unsigned>(code[3]) >> 2) << (8 + shb));
+#pragma unroll
+        for (int o = 2; o <= 16; o <<= 1) { ha |= __shfl_xor_sync(FULL, ha, o); hb |= __shfl_xor_sync(FULL, hb, o); }
+        if ((lane & 30) == 0) {
+            unsigned char* p = rec + k_hi_offset(3) + bi * 256 + 8 * (4 * g + ta) + 4 * rs;
+            *reinterpret_cast<unsigned*>(p) = ha;
+            *reinterpret_cast<unsigned*>(p + 8) = hb;
+        }
+    }
 }
 
 template <int BITS>
 __device__ __forceinline__ void store_v_codes(unsigned char* rec, int r, const int (&code)[4], int lane) {
+    constexpr bool PLANES = BITS == 3;
+    constexpr bool TWO = BITS == 2 || BITS == 3;
     const int bi = r >> 4, rr = r & 15, ps = rr >> 3, t = (rr & 7) >> 1, hi = rr & 1;
     const int i = lane >> 2;                            // channel block of this lane's channels
-    const int sh = (BITS == 2) ? 2 * i : 4 * (i & 3);
-    unsigned wa = (static_cast<unsigned>(code[0]) << sh) | (static_cast<unsigned>(code[1]) << (16 + sh));
-    unsigned wb = (static_cast<unsigned>(code[2]) << sh) | (static_cast<unsigned>(code[3]) << (16 + sh));
+    const int sh = TWO ? 2 * i : 4 * (i & 3);
+    const unsigned lowmask = PLANES ? 3u : 0xFu;
+    unsigned wa = ((static_cast<unsigned>(code[0]) & lowmask) << sh) | ((static_cast<unsigned>(code[1]) & lowmask) << (16 + sh));
+    unsigned wb = ((static_cast<unsigned>(code[2]) & lowmask) << sh) | ((static_cast<unsigned>(code[3]) & lowmask) << (16 + sh));
     wa |= __shfl_xor_sync(FULL, wa, 4);  wb |= __shfl_xor_sync(FULL, wb, 4);
     wa |= __shfl_xor_sync(FULL, wa, 8);  wb |= __shfl_xor_sync(FULL, wb, 8);
-    if (BITS == 2) { wa |= __shfl_xor_sync(FULL, wa, 16); wb |= __shfl_xor_sync(FULL, wb, 16); }
+    if (TWO) { wa |= __shfl_xor_sync(FULL, wa, 16); wb |= __shfl_xor_sync(FULL, wb, 16); }
     const int rsel = (lane & 3) >> 1, g0 = 4 * (lane & 1);
     unsigned char* base;
     bool writer;
-    if (BITS == 2) {
+    if (TWO) {
         writer = lane < 4;
-        base = rec + v_codes_offset(2) + bi * 512 + 4 * (2 * ps + rsel) + 2 * hi;
+        base = rec + v_codes_offset(BITS) + bi * 512 + 4 * (2 * ps + rsel) + 2 * hi;
     } else {
         writer = (lane & 12) == 0;
         base = rec + v_codes_offset(4) + bi * 1024 + 512 * ps + 4 * (2 * rsel + (lane >> 4)) + 2 * hi;
@@ -169,6 +187,20 @@ __device__ __forceinline__ void store_v_codes(unsigned char* rec, int r, const i
         *reinterpret_cast<unsigned short*>(base + 16 * (4 * (g0 + 1) + t)) = static_cast<unsigned short>(wa >> 16);
         *reinterpret_cast<unsigned short*>(base + 16 * (4 * (g0 + 2) + t)) = static_cast<unsigned short>(wb & 0xffffu);
         *reinterpret_cast<unsigned short*>(base + 16 * (4 * (g0 + 3) + t)) = static_cast<unsigned short>(wb >> 16);
+    }
+    if (PLANES) {                                       // 1-bit plane: half-word hi of word ps of lane (g,t), bit v1_bit(rsel, i)
+        const int shb = v1_bit(rsel, i);
+        unsigned ha = ((static_cast<unsigned>(code[0]) >> 2) << shb) | ((static_cast<unsigned>(code[1]) >> 2) << (16 + shb));
+        unsigned hb = ((static_cast<unsigned>(code[2]) >> 2) << shb) | ((static_cast<unsigned>(code[3]) >> 2) << (16 + shb));
+#pragma unroll
+        for (int o = 2; o <= 16; o <<= 1) { ha |= __shfl_xor_sync(FULL, ha, o); hb |= __shfl_xor_sync(FULL, hb, o); }
+        if (lane < 2) {
+            unsigned char* hbase = rec + v_hi_offset(3) + bi * 256 + 4 * ps + 2 * hi;
+            *reinterpret_cast<unsigned short*>(hbase + 8 * (4 * (g0 + 0) + t)) = static_cast<unsigned short>(ha & 0xffffu);
+            *reinterpret_cast<unsigned short*>(hbase + 8 * (4 * (g0 + 1) + t)) = static_cast<unsigned short>(ha >> 16);
+            *reinterpret_cast<unsigned short*>(hbase + 8 * (4 * (g0 + 2) + t)) = static_cast<unsigned short>(hb & 0xffffu);
+            *reinterpret_cast<unsigned short*>(hbase + 8 * (4 * (g0 + 3) + t)) = static_cast<unsigned short>(hb >> 16);
+        }
     }
 }
 
@@ -720,18 +752,35 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
             int code[32];
             __half step_h, xmin_h;
             quad_quantize<BITS, KQ>(x, P.rule_v, code, step_h, xmin_h, P.c.dev_status, live && qd == 0);
+            unsigned hplane[4] = {0u, 0u, 0u, 0u};           // 3 bits: the 1-bit plane's half-words, both row halves joined
+            if (BITS == 3) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    unsigned h0 = 0, h1 = 0;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        h0 |= static_cast<unsigned>(code[4 * k + e] >> 2) << v1_bit(0, k);
+                        h1 |= static_cast<unsigned>(code[4 * k + e] >> 2) << v1_bit(1, k);
+                    }
+                    const unsigned mine = (qd >> 1) ? h1 : h0;
+                    hplane[e] = mine | __shfl_xor_sync(FULL, mine, 2);     // lane qd ^ 2 holds the other row half of the same rows
+                }
+            }
             if (live) {
                 unsigned char* rec = P.c.pages + ri.rec_off;
                 const int bi = ri.r >> 4, rr = ri.r & 15, ps = rr >> 3, t = (rr & 7) >> 1, hi = rr & 1;
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {                 // channel residue c16 = 4 qd + e: one half-word per 8 (or 4) channel blocks
                     const int c16 = 4 * qd + e, g = c16 & 7, rsel = c16 >> 3;
-                    if (BITS == 2) {
+                    if (BITS == 2 || BITS == 3) {
                         unsigned hw = 0;
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) hw |= static_cast<unsigned>(code[4 * k + e]) << (2 * k);
-                        *reinterpret_cast<unsigned short*>(rec + v_codes_offset(2) + bi * 512 + 16 * (4 * g + t) + 4 * (2 * ps + rsel) + 2 * hi) =
+                        for (int k = 0; k < 8; ++k) hw |= static_cast<unsigned>(code[4 * k + e] & 3) << (2 * k);
+                        *reinterpret_cast<unsigned short*>(rec + v_codes_offset(BITS) + bi * 512 + 16 * (4 * g + t) + 4 * (2 * ps + rsel) + 2 * hi) =
                             static_cast<unsigned short>(hw);
+                        if (BITS == 3 && qd < 2)
+                            *reinterpret_cast<unsigned short*>(rec + v_hi_offset(3) + bi * 256 + 8 * (4 * g + t) + 4 * ps + 2 * hi) =
+                                static_cast<unsigned short>(hplane[e]);
                     } else {
 #pragma unroll
                         for (int j = 0; j < 2; ++j) {
@@ -847,15 +896,23 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
                 unsigned char* rec = P.c.pages + ri.rec_off;
                 const int bi = ri.r >> 4, rr = ri.r & 15, g = rr & 7, rs = rr >> 3;
                 // entry 4k + j is byte j of the word of channel half k & 1, field / nibble of k-step k >> 1
-                if (BITS == 2) {
+                if (BITS == 2 || BITS == 3) {
                     unsigned w[2] = {0u, 0u};
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) w[k & 1] |= static_cast<unsigned>(code[4 * k + j]) << (8 * j + 2 * (k >> 1));
+                        for (int j = 0; j < 4; ++j) w[k & 1] |= static_cast<unsigned>(code[4 * k + j] & 3) << (8 * j + 2 * (k >> 1));
                     unsigned char* p = rec + bi * 512 + 16 * (4 * g + qd) + 4 * rs;
                     *reinterpret_cast<unsigned*>(p) = w[0];
                     *reinterpret_cast<unsigned*>(p + 8) = w[1];
+                    if (BITS == 3) {                          // 1-bit plane: byte j, bit 2 (k >> 1) + (k & 1) = k
+                        unsigned wh = 0u;
+#pragma unroll
+                        for (int k = 0; k < 8; ++k)
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) wh |= static_cast<unsigned>(code[4 * k + j] >> 2) << (8 * j + k);
+                        *reinterpret_cast<unsigned*>(rec + k_hi_offset(3) + bi * 256 + 8 * (4 * g + qd) + 4 * rs) = wh;
+                    }
                 } else {
                     unsigned w[2][2] = {{0u, 0u}, {0u, 0u}};      // [512-byte half][channel half]
 #pragma unroll
@@ -949,7 +1006,12 @@ __global__ void unpack_debug_kernel(CacheView c, int slot, int head, int which, 
     int off, bit;
     if (which == 0) k_code_location(c.bits, r, ch, off, bit); else v_code_location(c.bits, r, ch, off, bit);
     const unsigned byte = rec[off + (bit >> 3)];          // little-endian half-words: bit 8.. is the second byte
-    codes[idx] = static_cast<unsigned char>((byte >> (bit & 7)) & ((1u << c.bits) - 1u));
+    unsigned code = (byte >> (bit & 7)) & ((1u << (c.bits == 3 ? 2 : c.bits)) - 1u);
+    if (c.bits == 3) {                                    // the third bit lives in the 1-bit plane
+        if (which == 0) k_hi_location(r, ch, off, bit); else v_hi_location(r, ch, off, bit);
+        code |= ((static_cast<unsigned>(rec[off + (bit >> 3)]) >> (bit & 7)) & 1u) << 2;
+    }
+    codes[idx] = static_cast<unsigned char>(code);
     if (ch == 0) {
         const __half* meta = reinterpret_cast<const __half*>(rec + meta_location(c.bits, r));
         scale[tok] = __half2float(meta[2 * which]);
@@ -1045,6 +1107,7 @@ static int append_impl(const wushkv_cache* cache, int32_t batch, const int32_t* 
         cfg.attrs = attr;
         cfg.numAttrs = 2;
         const cudaError_t e1 = P.c.bits == 2 ? cudaLaunchKernelEx(&cfg, append_token_kernel<2>, P)
+                             : P.c.bits == 3 ? cudaLaunchKernelEx(&cfg, append_token_kernel<3>, P)
                                              : cudaLaunchKernelEx(&cfg, append_token_kernel<4>, P);
         return e1 == cudaSuccess ? WUSHKV_OK : WUSHKV_ECUDA;
     }
@@ -1071,6 +1134,13 @@ static int append_impl(const wushkv_cache* cache, int32_t batch, const int32_t* 
             else if (kk_k == 8) ok = launch(append_chunk_kernel<2, 8, 16>);
             else if (kk_v == 8) ok = launch(append_chunk_kernel<2, 16, 8>);
             else ok = launch(append_chunk_kernel<2, 16, 16>);
+        } else if (P.c.bits == 3) {
+            if (kk_k < 0) ok = launch(append_chunk_kernel<3, -1, -1>);
+            else if (kk_k == 0) ok = launch(append_chunk_kernel<3, 0, 0>);
+            else if (kk_k == 8 && kk_v == 8) ok = launch(append_chunk_kernel<3, 8, 8>);
+            else if (kk_k == 8) ok = launch(append_chunk_kernel<3, 8, 16>);
+            else if (kk_v == 8) ok = launch(append_chunk_kernel<3, 16, 8>);
+            else ok = launch(append_chunk_kernel<3, 16, 16>);
         } else {
             if (kk_k < 0) ok = launch(append_chunk_kernel<4, -1, -1>);
             else if (kk_k == 0) ok = launch(append_chunk_kernel<4, 0, 0>);
@@ -1094,6 +1164,9 @@ static int append_impl(const wushkv_cache* cache, int32_t batch, const int32_t* 
     if (P.c.bits == 2) {
         if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(append_rows_kernel<2>), static_cast<int>(smem))) return WUSHKV_ECUDA;
         append_rows_kernel<2><<<grid, 256, smem, st>>>(P);
+    } else if (P.c.bits == 3) {
+        if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(append_rows_kernel<3>), static_cast<int>(smem))) return WUSHKV_ECUDA;
+        append_rows_kernel<3><<<grid, 256, smem, st>>>(P);
     } else {
         if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(append_rows_kernel<4>), static_cast<int>(smem))) return WUSHKV_ECUDA;
         append_rows_kernel<4><<<grid, 256, smem, st>>>(P);

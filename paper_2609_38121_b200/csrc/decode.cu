@@ -93,7 +93,7 @@ struct DecodeParams {
 // the optional whole-word shift: the fp16 value of the masked field is code * 2^(field_shift - 24)
 template <int BITS>
 __host__ __device__ constexpr int field_shift(int idx) {
-    return BITS == 2 ? (idx < 5 ? 2 * idx : 2 * (idx - 5)) : 4 * (idx & 1);
+    return BITS != 4 ? (idx < 5 ? 2 * idx : 2 * (idx - 5)) : 4 * (idx & 1);     // 3 bits: its 2-bit plane
 }
 // bf16x2 bit pattern of (2^e, 2^e)
 __host__ __device__ constexpr unsigned bf16x2_pow2(int e) {
@@ -260,7 +260,7 @@ __global__ void __launch_bounds__(PREP_THREADS) decode_prep_kernel(DecodeParams 
     asm volatile("bar.sync 1, 128;" ::: "memory");
     if (i < G) {
         const int sum = red_isum[i][0] + red_isum[i][1] + red_isum[i][2] + red_isum[i][3];
-        constexpr float FS = BITS == 2 ? 4.f : 16.f;      // the integer score carries this factor (see the main kernel)
+        constexpr float FS = BITS != 4 ? 4.f : 16.f;      // the integer score carries this factor (see the main kernel)
         float* qs = P.qscal + (static_cast<long long>(b) * P.c.n_q + h * G + i) * 2;
         qs[0] = k2 * lam[i] * (1.f / FS);                 // score (log2 domain) = qs[0] * (Delta_k * sum_int + x_min_k * qs[1])
         qs[1] = FS * static_cast<float>(sum);
@@ -351,6 +351,11 @@ __device__ __forceinline__ void bulk_copy_g2s_stream(unsigned dst, const void* s
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(pol) : "memory");
 }
+__device__ __forceinline__ uint2 lds64(unsigned addr) {
+    uint2 v;
+    asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr) : "memory");
+    return v;
+}
 __device__ __forceinline__ uint4 lds128(unsigned addr) {
     uint4 v;
     asm("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
@@ -425,7 +430,7 @@ __device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(_
 // same word shifted right so that the upper fields fall into the low bits of each 16-bit lane.
 template <int BITS>
 __device__ __forceinline__ unsigned field(unsigned w, unsigned ws, int idx) {
-    if (BITS == 2) {
+    if (BITS != 4) {
         constexpr unsigned M0 = 0x00030003u;
         return idx < 5 ? (w & (M0 << (2 * idx))) : (ws & (M0 << (2 * (idx - 5))));
     } else {
@@ -433,7 +438,7 @@ __device__ __forceinline__ unsigned field(unsigned w, unsigned ws, int idx) {
         return idx < 2 ? (w & (M0 << (4 * idx))) : (ws & (M0 << (4 * (idx - 2))));
     }
 }
-template <int BITS> __device__ __forceinline__ unsigned pre_shift(unsigned w) { return BITS == 2 ? (w >> 10) : (w >> 8); }
+template <int BITS> __device__ __forceinline__ unsigned pre_shift(unsigned w) { return BITS != 4 ? (w >> 10) : (w >> 8); }
 
 // Per-warp running softmax state of one (sequence, KV head).  MODE 0: one head per thread (head t,
 // value and rounding-remainder columns).  MODE 1: two heads per thread (2t, 2t+1).
@@ -815,9 +820,9 @@ __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_ke
                         // position come out of the mask as the code itself, fields at an odd position as the code
                         // times FS (4 at 2 bits, 16 at 4 bits): the two kinds are summed separately (X, Y) and
                         // joined as FS * X + Y, which is FS times the exact integer dot product.
-                        constexpr int FS = BITS == 2 ? 4 : 16;
+                        constexpr int FS = BITS != 4 ? 4 : 16;
                         unsigned a[4][4];             // [k-step][A register]
-                        if (BITS == 2) {
+                        if (BITS != 4) {
                             const uint4 kw = lds128(rec + bi * CB + 16 * lane);      // (row g, ch half 0), (g+8, 0), (g, 1), (g+8, 1)
                             const unsigned sx = kw.x >> 4, sy = kw.y >> 4, sz = kw.z >> 4, sw = kw.w >> 4;
                             a[0][0] = kw.x & 0x03030303u; a[0][1] = kw.y & 0x03030303u; a[0][2] = kw.z & 0x03030303u; a[0][3] = kw.w & 0x03030303u;
@@ -843,12 +848,35 @@ __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_ke
 #pragma unroll
                             for (int e = 0; e < 4; ++e) dot[e] = X[e] * FS + Y[e];
                         }
+                        unsigned ah[4][4];            // 3 bits: A registers of the 1-bit plane (codes' high bits), one shift + mask each
+                        if (BITS == 3 && !(WUSHKV_ABL & 2)) {
+                            const uint2 kh = lds64(rec + k_hi_offset(3) + bi * 256 + 8 * lane);      // words of token rows g, g+8
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks) {
+                                ah[ks][0] = (kh.x >> (2 * ks)) & 0x01010101u;     ah[ks][1] = (kh.y >> (2 * ks)) & 0x01010101u;
+                                ah[ks][2] = (kh.x >> (2 * ks + 1)) & 0x01010101u; ah[ks][3] = (kh.y >> (2 * ks + 1)) & 0x01010101u;
+                            }
+                            int Z[4];
+                            mma_u8s8_zero(Z, ah[0][0], ah[0][1], ah[0][2], ah[0][3], qf[0][0], qf[0][1]);
+#pragma unroll
+                            for (int ks = 1; ks < 4; ++ks) mma_u8s8(Z, ah[ks][0], ah[ks][1], ah[ks][2], ah[ks][3], qf[ks][0], qf[ks][1]);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) dot[e] += 4 * FS * Z[e];       // code = low plane + 4 x high bit
+                        }
                         if (MODE == 1 && !(WUSHKV_ABL & 2)) {              // second fragment set: the low digits of the eight heads
                             int X[4], Y[4];
                             mma_u8s8_zero(X, a[0][0], a[0][1], a[0][2], a[0][3], qfl[0][0], qfl[0][1]);
                             mma_u8s8_zero(Y, a[1][0], a[1][1], a[1][2], a[1][3], qfl[1][0], qfl[1][1]);
                             mma_u8s8(X, a[2][0], a[2][1], a[2][2], a[2][3], qfl[2][0], qfl[2][1]);
                             mma_u8s8(Y, a[3][0], a[3][1], a[3][2], a[3][3], qfl[3][0], qfl[3][1]);
+                            if (BITS == 3) {
+                                int Z[4];
+                                mma_u8s8_zero(Z, ah[0][0], ah[0][1], ah[0][2], ah[0][3], qfl[0][0], qfl[0][1]);
+#pragma unroll
+                                for (int ks = 1; ks < 4; ++ks) mma_u8s8(Z, ah[ks][0], ah[ks][1], ah[ks][2], ah[ks][3], qfl[ks][0], qfl[ks][1]);
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) Y[e] += 4 * FS * Z[e];
+                            }
 #pragma unroll
                             for (int e = 0; e < 4; ++e) dot[e] = dot[e] * 256 + (X[e] * FS + Y[e]);
                         }
@@ -915,12 +943,26 @@ __global__ void __launch_bounds__(main_warps(BITS, MODE) * 32, 1) decode_main_ke
                         }
                         const unsigned b01 = movmatrix_trans(r0), b23 = movmatrix_trans(r1);
                         if (WUSHKV_ABL & 1) { st.o[bi][0] += __uint_as_float(b01 ^ b23); } else
-                        if (BITS == 2) {
-                            const uint4 vw = lds128(rec + v_codes_offset(2) + bi * CB + 16 * lane);
+                        if (BITS != 4) {
+                            const uint4 vw = lds128(rec + v_codes_offset(BITS) + bi * CB + 16 * lane);
                             const unsigned sx = pre_shift<2>(vw.x), sy = pre_shift<2>(vw.y), sz = pre_shift<2>(vw.z), sw = pre_shift<2>(vw.w);
 #pragma unroll
                             for (int i = 0; i < 8; ++i)
                                 mma_f16(st.o[i], field<2>(vw.x, sx, i), field<2>(vw.y, sy, i), field<2>(vw.z, sz, i), field<2>(vw.w, sw, i), b01, b23);
+                            if (BITS == 3) {
+                                // 1-bit plane: words of token halves ps = 0, 1; one of five shifts of a word puts the bit of
+                                // (row half, channel block i) two bits above the low plane's field of block i, so that it reads
+                                // as 4 x (high bit) in that field's unit and lands in the same accumulator
+                                const uint2 vh = lds64(rec + v_hi_offset(3) + bi * 256 + 8 * lane);
+                                const unsigned xv[5] = {vh.x, vh.x << 1, vh.x >> 9, vh.x >> 10, vh.x << 6};
+                                const unsigned yv[5] = {vh.y, vh.y << 1, vh.y >> 9, vh.y >> 10, vh.y << 6};
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) {
+                                    const unsigned m = 0x00010001u << v1_target(i);
+                                    const int r0 = i < 5 ? 0 : 2, r1 = i < 5 ? 1 : (i < 7 ? 3 : 4);
+                                    mma_f16(st.o[i], xv[r0] & m, xv[r1] & m, yv[r0] & m, yv[r1] & m, b01, b23);
+                                }
+                            }
                         } else {
                             const uint4 va = lds128(rec + v_codes_offset(4) + bi * CB + 16 * lane);         // tokens 2t,2t+1
                             const uint4 vb = lds128(rec + v_codes_offset(4) + bi * CB + 512 + 16 * lane);   // tokens 2t+8,2t+9
@@ -1169,12 +1211,13 @@ static int decode_attn_impl(const wushkv_cache* cache, int32_t batch, const int3
             if (dev >= 0 && dev < 64) l2_bytes[dev] = l2;
         }
         const double step_bytes = static_cast<double>(batch) * P.c.n_kv * ((max_seq_len + PAGE_TOKENS - 1) / PAGE_TOKENS) *
-                                  (P.c.bits == 2 ? record_bytes(2) : record_bytes(4));
+                                  record_bytes(P.c.bits);
         P.stream_pages = step_bytes > static_cast<double>(l2) ? 1 : 0;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool mode0 = P.c.G <= 4;
     if (P.c.bits == 2) return mode0 ? launch_decode<2, 0>(P, pl.n_ctas, st) : launch_decode<2, 1>(P, pl.n_ctas, st);
+    if (P.c.bits == 3) return mode0 ? launch_decode<3, 0>(P, pl.n_ctas, st) : launch_decode<3, 1>(P, pl.n_ctas, st);
     return mode0 ? launch_decode<4, 0>(P, pl.n_ctas, st) : launch_decode<4, 1>(P, pl.n_ctas, st);
 }
 

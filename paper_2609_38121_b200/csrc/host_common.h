@@ -14,7 +14,7 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 inline int make_view(const wushkv_cache* c, CacheView& v) {
     if (!c) return WUSHKV_EINVAL;
     if (c->d != D || c->page_tokens != PAGE_TOKENS) return WUSHKV_EINVAL;
-    if (c->bits != 2 && c->bits != 4) return WUSHKV_EINVAL;
+    if (c->bits != 2 && c->bits != 3 && c->bits != 4) return WUSHKV_EINVAL;
     if (c->n_kv <= 0 || c->n_q <= 0 || c->n_q % c->n_kv != 0) return WUSHKV_EINVAL;
     const int G = c->n_q / c->n_kv;
     if (G < 1 || G > 8) return WUSHKV_EINVAL;

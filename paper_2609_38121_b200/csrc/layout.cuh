@@ -2,7 +2,7 @@
 //
 // A record holds PAGE_TOKENS = 64 tokens as 4 blocks of 16 tokens:
 //     [K codes: 4 blocks][V codes: 4 blocks][meta: 4 blocks x 128 B]
-// with a code block of 16*128*bits/8 = 512 B (2-bit) or 1024 B (4-bit).  Inside a code block
+// with a code block of 512 B (2-bit) or 1024 B (4-bit); 3-bit records are described further down.  Inside a code block
 // byte 16*L .. 16*L+15 (of each 512-byte half) belongs to lane L = 4*g + t of the decode warp,
 // so that one 16-byte shared-memory load per lane yields exactly the words that lane turns into
 // mma A-fragments with a mask (and at most one shift) per register.
@@ -22,6 +22,13 @@
 //    Masked out of a 16-bit lane and read as an fp16 bit pattern, a code field that lies inside bits 0..10 is the
 //    exact value code * 2^(shift-24) (fp16 subnormals and the first binade are linear in the bit pattern), so
 //    no int->float conversion is executed; the powers of two are folded into the output epilogue.
+//  3-bit records store a code c as a 2-bit plane (c & 3, laid out exactly like the 2-bit blocks above) and a 1-bit
+//  plane (c >> 2) of 256 bytes per block, 8 bytes = two words per lane:
+//    K: word rs of lane (g,t), byte b, bit 2s + hh: (word >> (2s + hh)) & 0x01010101 is A register rs + 2hh of k-step s.
+//    V: word ps of lane (g,t), half-word hi; the bit of (rsel, channel block i) sits where one shift of the word puts
+//       it two bits above the 2-bit plane's field of block i (so that, read as fp16, it is 4 c1 on that field's
+//       scale and both planes accumulate into the same output fragment): v1_bit(rsel, i) below.
+//    record: [K 2-bit plane 4 x 512][K 1-bit plane 4 x 256][V 2-bit plane][V 1-bit plane][meta] = 6656 bytes.
 //  meta block bi: token rr -> 8 bytes {K step, K x_min, V step, V x_min} (fp16) at 128bi + 16(rr&7) + 8(rr>>3).
 #pragma once
 #include <cstdint>
@@ -34,11 +41,25 @@ constexpr int PAGE_TOKENS = 64;
 constexpr int BLOCK_TOKENS = 16;
 constexpr int BLOCKS_PER_PAGE = PAGE_TOKENS / BLOCK_TOKENS;
 
-__host__ __device__ constexpr int code_block_bytes(int bits) { return BLOCK_TOKENS * D * bits / 8; }
+// code_block_bytes: bytes of the (low-plane) code block the decode warp reads with one 16-byte load per lane and
+// 512-byte half: 512 at 2 and 3 bits, 1024 at 4 bits; a 3-bit record adds the 256-byte 1-bit-plane blocks.
+__host__ __device__ constexpr int code_block_bytes(int bits) { return bits == 4 ? 1024 : 512; }
+__host__ __device__ constexpr int hi_block_bytes(int bits) { return bits == 3 ? 256 : 0; }
+__host__ __device__ constexpr int side_bytes(int bits) { return BLOCKS_PER_PAGE * (code_block_bytes(bits) + hi_block_bytes(bits)); }
 __host__ __device__ constexpr int k_codes_offset(int) { return 0; }
-__host__ __device__ constexpr int v_codes_offset(int bits) { return BLOCKS_PER_PAGE * code_block_bytes(bits); }
-__host__ __device__ constexpr int meta_offset(int bits) { return 2 * BLOCKS_PER_PAGE * code_block_bytes(bits); }
+__host__ __device__ constexpr int k_hi_offset(int bits) { return BLOCKS_PER_PAGE * code_block_bytes(bits); }
+__host__ __device__ constexpr int v_codes_offset(int bits) { return side_bytes(bits); }
+__host__ __device__ constexpr int v_hi_offset(int bits) { return side_bytes(bits) + BLOCKS_PER_PAGE * code_block_bytes(bits); }
+__host__ __device__ constexpr int meta_offset(int bits) { return 2 * side_bytes(bits); }
 __host__ __device__ constexpr int record_bytes(int bits) { return meta_offset(bits) + PAGE_TOKENS * 8; }
+
+// Bit (inside its 16-bit half-word) of the V 1-bit-plane field of (row half rsel, channel block i), and the shift
+// that brings it to its target position 2 + field shift of block i (targets 2,4,6,8,10,2,4,6): a negative shift
+// is a left shift.  rsel 0: blocks 0-4 in place, blocks 5-7 from bits 11,13,15 (>> 9); rsel 1: blocks 0-4 from
+// bits 1,3,5,7,9 (<< 1), blocks 5,6 from bits 12,14 (>> 10), block 7 from bit 0 (<< 6).
+__host__ __device__ constexpr int v1_target(int i) { return i < 5 ? 2 * i + 2 : 2 * (i - 5) + 2; }
+__host__ __device__ constexpr int v1_shift(int rsel, int i) { return rsel == 0 ? (i < 5 ? 0 : 9) : (i < 5 ? -1 : (i < 7 ? 10 : -6)); }
+__host__ __device__ constexpr int v1_bit(int rsel, int i) { return v1_target(i) + v1_shift(rsel, i); }
 
 // Byte offset (within the record) of the byte holding K code (token r, channel ch) and the bit position
 // of the code inside that byte.
@@ -46,7 +67,7 @@ __host__ __device__ inline void k_code_location(int bits, int r, int ch, int& by
     const int bi = r >> 4, rr = r & 15, g = rr & 7, rs = rr >> 3;
     const int s = ch >> 5, hh = (ch >> 4) & 1, b = 2 * ((ch >> 3) & 1) + (ch & 1), t = (ch >> 1) & 3;
     const int L = 4 * g + t, j = rs + 2 * hh;
-    if (bits == 2) {
+    if (bits == 2 || bits == 3) {
         byte_off = bi * 512 + 16 * L + 4 * j + b;
         bit = 2 * s;
     } else {
@@ -60,13 +81,28 @@ __host__ __device__ inline void v_code_location(int bits, int r, int ch, int& by
     const int bi = r >> 4, rr = r & 15, ps = rr >> 3, t = (rr & 7) >> 1, hi = rr & 1;
     const int i = ch >> 4, r16 = ch & 15, rsel = r16 >> 3, g = r16 & 7;
     const int L = 4 * g + t;
-    if (bits == 2) {
-        byte_off = v_codes_offset(2) + bi * 512 + 16 * L + 4 * (2 * ps + rsel) + 2 * hi;
+    if (bits == 2 || bits == 3) {
+        byte_off = v_codes_offset(bits) + bi * 512 + 16 * L + 4 * (2 * ps + rsel) + 2 * hi;
         bit = 2 * i;
     } else {
         byte_off = v_codes_offset(4) + bi * 1024 + 512 * ps + 16 * L + 4 * (2 * rsel + (i >> 2)) + 2 * hi;
         bit = 4 * (i & 3);
     }
+}
+
+// 3-bit records: location of the high bit (c >> 2) of K / V code (token r, channel ch); byte offset of the byte (K)
+// or half-word (V) and the bit inside it.  (The functions above give the low two bits.)
+__host__ __device__ inline void k_hi_location(int r, int ch, int& byte_off, int& bit) {
+    const int bi = r >> 4, rr = r & 15, g = rr & 7, rs = rr >> 3;
+    const int s = ch >> 5, hh = (ch >> 4) & 1, b = 2 * ((ch >> 3) & 1) + (ch & 1), t = (ch >> 1) & 3;
+    byte_off = k_hi_offset(3) + bi * 256 + 8 * (4 * g + t) + 4 * rs + b;
+    bit = 2 * s + hh;
+}
+__host__ __device__ inline void v_hi_location(int r, int ch, int& byte_off, int& bit) {
+    const int bi = r >> 4, rr = r & 15, ps = rr >> 3, t = (rr & 7) >> 1, hi = rr & 1;
+    const int i = ch >> 4, r16 = ch & 15, rsel = r16 >> 3, g = r16 & 7;
+    byte_off = v_hi_offset(3) + bi * 256 + 8 * (4 * g + t) + 4 * ps + 2 * hi;
+    bit = v1_bit(rsel, i);
 }
 
 __host__ __device__ inline int meta_location(int bits, int r) {

@@ -333,15 +333,24 @@ __global__ void __launch_bounds__(PF_THREADS) prefill_attn_kernel(PrefillParams 
                 const int r = tid & 63, ch0 = (tid >> 6) * 64;
                 const int pos = pg * PAGE_TOKENS + r;
                 const bool live = page_ok && pos >= q_lo && pos < q_hi;
-                constexpr unsigned MASK = (1u << BITS) - 1u;
+                constexpr unsigned MASK = (1u << (BITS == 3 ? 2 : BITS)) - 1u;       // 3 bits: low two here, third bit below
+                auto field_at = [&](int off, int bit, unsigned mask) { return (static_cast<unsigned>(ts.raw[off + (bit >> 3)]) >> (bit & 7)) & mask; };
                 for (int ch = ch0; ch < ch0 + 64; ch += 2) {
                     float k0 = 0.f, k1 = 0.f, v0 = 0.f, v1 = 0.f;
                     if (live) {
                         int off, bit;
-                        k_code_location(BITS, r, ch, off, bit);     k0 = static_cast<float>((ts.raw[off + (bit >> 3)] >> (bit & 7)) & MASK);
-                        k_code_location(BITS, r, ch + 1, off, bit); k1 = static_cast<float>((ts.raw[off + (bit >> 3)] >> (bit & 7)) & MASK);
-                        v_code_location(BITS, r, ch, off, bit);     v0 = static_cast<float>((ts.raw[off + (bit >> 3)] >> (bit & 7)) & MASK);
-                        v_code_location(BITS, r, ch + 1, off, bit); v1 = static_cast<float>((ts.raw[off + (bit >> 3)] >> (bit & 7)) & MASK);
+                        unsigned ck[2], cv[2];
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            k_code_location(BITS, r, ch + e, off, bit); ck[e] = field_at(off, bit, MASK);
+                            v_code_location(BITS, r, ch + e, off, bit); cv[e] = field_at(off, bit, MASK);
+                            if (BITS == 3) {
+                                k_hi_location(r, ch + e, off, bit); ck[e] |= field_at(off, bit, 1u) << 2;
+                                v_hi_location(r, ch + e, off, bit); cv[e] |= field_at(off, bit, 1u) << 2;
+                            }
+                        }
+                        k0 = static_cast<float>(ck[0]); k1 = static_cast<float>(ck[1]);
+                        v0 = static_cast<float>(cv[0]); v1 = static_cast<float>(cv[1]);
                     }
                     *reinterpret_cast<unsigned*>(&ts.K[r][ch]) = pack_half2(k0, k1);
                     *reinterpret_cast<unsigned*>(&ts.V[r][ch]) = pack_half2(v0, v1);
@@ -463,6 +472,9 @@ extern "C" int wushkv_prefill_attn(const wushkv_cache* cache, int32_t batch, con
     if (P.c.bits == 2) {
         if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(prefill_attn_kernel<2>), static_cast<int>(smem_attn))) return WUSHKV_ECUDA;
         prefill_attn_kernel<2><<<grid, PF_THREADS, smem_attn, st>>>(P);
+    } else if (P.c.bits == 3) {
+        if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(prefill_attn_kernel<3>), static_cast<int>(smem_attn))) return WUSHKV_ECUDA;
+        prefill_attn_kernel<3><<<grid, PF_THREADS, smem_attn, st>>>(P);
     } else {
         if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(prefill_attn_kernel<4>), static_cast<int>(smem_attn))) return WUSHKV_ECUDA;
         prefill_attn_kernel<4><<<grid, PF_THREADS, smem_attn, st>>>(P);

@@ -46,7 +46,8 @@ def test_status_strings_and_page_bytes():
     assert "positive definite" in B.status_string(B.ENOTPD)
     assert B.page_bytes(8, 128, 2, 64) == 8 * 4608       # 64 tokens x (2 x 32 B codes + 8 B meta)
     assert B.page_bytes(8, 128, 4, 64) == 8 * 8704
-    assert B.page_bytes(8, 64, 2, 64) == 0 and B.page_bytes(8, 128, 3, 64) == 0
+    assert B.page_bytes(8, 128, 3, 64) == 8 * 6656       # 64 tokens x (2 x 48 B codes + 8 B meta)
+    assert B.page_bytes(8, 64, 2, 64) == 0 and B.page_bytes(8, 128, 5, 64) == 0
 
 
 def test_host_validation_rejects_bad_arguments_without_cuda():

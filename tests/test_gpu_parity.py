@@ -35,7 +35,7 @@ def _check_window_copies(L):
         assert np.mean(d > 0) < 2e-3
 
 
-@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 def test_config0_tiny_layer(bits):
     """Benchmark config 0: batch 1, 8 query / 2 KV heads, 2048 context, sink 4, recent 64."""
     wl = W.LayerWorkload("cfg0")
@@ -48,7 +48,8 @@ def test_config0_tiny_layer(bits):
     assert L.cache.status() == 0
 
 
-@pytest.mark.parametrize("n_q,n_kv,bits", [(8, 1, 2), (8, 1, 4), (7, 1, 2), (14, 2, 4), (2, 2, 2), (6, 2, 2), (5, 1, 4), (3, 1, 2)])
+@pytest.mark.parametrize("n_q,n_kv,bits", [(8, 1, 2), (8, 1, 4), (7, 1, 2), (14, 2, 4), (2, 2, 2), (6, 2, 2), (5, 1, 4), (3, 1, 2),
+                                            (8, 2, 3), (8, 1, 3), (3, 1, 3)])
 def test_group_sizes(n_q, n_kv, bits):
     """Every query-group size 1..8 takes one of the two fragment modes; G = 7 with RMSNorm is the
     Qwen-shaped layer of config 4, G = 8 the 70B-shaped layer of config 3."""
@@ -60,7 +61,7 @@ def test_group_sizes(n_q, n_kv, bits):
     assert L.cache.status() == 0
 
 
-@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 def test_ragged_batch_shuffled_pages_and_flush_sizes(bits):
     """Ragged lengths (config 2's structure, scaled down), page table in random order, S_flush > 1
     so that the recent window breathes, and appends that straddle page boundaries."""
@@ -94,15 +95,15 @@ def test_serving_window_sizes(s_sink, s_keep, s_flush):
     assert L.cache.status() == 0
 
 
-@pytest.mark.parametrize("path", ["tensor", "cuda"])
-def test_prefill_chunk_paths(path, test_option):
+@pytest.mark.parametrize("path,bits", [("tensor", 2), ("cuda", 2), ("tensor", 3), ("cuda", 3)])
+def test_prefill_chunk_paths(path, bits, test_option):
     """Config 4's structure scaled down: several sequences appended as one chunk each in ONE call
     (tile boundaries fall inside sequences and a ragged last tile), Qwen-shaped heads (G = 7, RMSNorm),
     through the tensor-core transform and through the CUDA-core chunk path; then one decode step."""
     if path == "cuda":
         test_option("append_path_cuda", 1)
     wl = _wl(28, 4, seed=41, batch=3, theta=1e6, rmsnorm=True)
-    L = Layer(wl, [700, 131, 390], 2, 4, 128, 1)
+    L = Layer(wl, [700, 131, 390], bits, 4, 128, 1)
     L.append_step([699, 130, 389])
     L.append_step([1, 1, 1])
     assert L.seq_len.cpu().tolist() == [700, 131, 390]
@@ -112,7 +113,7 @@ def test_prefill_chunk_paths(path, test_option):
     assert L.cache.status() == 0
 
 
-@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 def test_quest_quantizer_on_every_append_path(bits):
     """Section 4.3, Eq. 5 instead of Eq. 6: step from the group's RMS, bin-centre reconstruction.  One sequence
     goes through the tensor-core chunk path, one through the CUDA-core rows path, and every sequence gets a
@@ -171,7 +172,7 @@ def test_decode_is_deterministic_and_split_invariant(test_option):
     assert np.max(np.abs(outs[3] - outs[0])) <= 5e-4 * scale
 
 
-@pytest.mark.parametrize("bits,n_q,n_kv", [(2, 8, 2), (4, 14, 2)])
+@pytest.mark.parametrize("bits,n_q,n_kv", [(2, 8, 2), (4, 14, 2), (3, 8, 2)])
 def test_fused_step_equals_append_then_decode(bits, n_q, n_kv):
     """wushkv_decode_step (queries transformed beside the append) gives, bit for bit, the cache and the
     outputs of wushkv_append + wushkv_decode_attn; several steps are enqueued back to back."""

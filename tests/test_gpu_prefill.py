@@ -14,7 +14,7 @@ def _wl(n_q, n_kv, seed, batch=1, theta=1e4, rmsnorm=False):
                                 s_keep=64, rmsnorm=rmsnorm, ragged=None, prefill_chunk=0))
 
 
-@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 def test_prefill_on_an_empty_cache(bits):
     """The whole prompt as one chunk: every key is a chunk position (full precision, causal); several query tiles,
     a ragged last tile, a sequence shorter than one tile."""
@@ -25,7 +25,7 @@ def test_prefill_on_an_empty_cache(bits):
     assert L.cache.status() == 0
 
 
-@pytest.mark.parametrize("bits,n_q,n_kv", [(2, 8, 2), (4, 14, 2)])
+@pytest.mark.parametrize("bits,n_q,n_kv", [(2, 8, 2), (4, 14, 2), (3, 8, 2)])
 def test_chunk_over_a_quantized_cache(bits, n_q, n_kv):
     """A chunk appended to a long cache: sink rows, packed pages (first and last one partly outside the quantized
     range), the old part of the recent window, then the chunk; ragged batch, shuffled page table, G = 4 and 7."""

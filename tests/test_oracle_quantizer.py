@@ -129,7 +129,7 @@ def test_degenerate_groups():
         assert np.array_equal(O.dequantize(codes, delta, xmin), np.full(128, v))
 
 
-@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 def test_pack_roundtrip_and_layout(bits):
     rng = np.random.default_rng(17)
     codes = rng.integers(0, 1 << bits, size=(5, 3, 128), dtype=np.uint8)
@@ -140,6 +140,14 @@ def test_pack_roundtrip_and_layout(bits):
     one[:4] = [1, 2, 3, 1]
     if bits == 2:
         assert O.pack_codes(one, 2)[0] == 1 | (2 << 2) | (3 << 4) | (1 << 6)
+    elif bits == 3:
+        # 48 bytes per 128-channel vector; the stream 001 010 011 001 (low bit first per code) by hand:
+        # bits 0..11 = 1,0,0, 0,1,0, 1,1,0, 1,0,0 -> byte 0 = 0b11010001, byte 1 low nibble = 0b0010
+        one[:4] = [1, 2, 3, 1]
+        p3 = O.pack_codes(one, 3)
+        assert p3.shape == (48,) and p3[0] == 0b11010001 and p3[1] == 0b0010 and not p3[2:].any()
+        seven = np.full(128, 7, np.uint8)
+        assert np.all(O.pack_codes(seven, 3) == 0xFF)
     else:
         assert O.pack_codes(one, 4)[:2].tolist() == [1 | (2 << 4), 3 | (1 << 4)]
 
