@@ -21,7 +21,7 @@ Conventions
 
 Parity pins (tests/test_oracle_*.py, tests/test_golden.py) cover every function below (the error metric
 and the quantize-from-bf16 reading in test_oracle_attention.py, the QuEST quantizer in test_oracle_quest.py,
-chunk attention in test_oracle_chunk_attn.py, Norm and RoPE in test_oracle_prologue.py); none is "parity unpinned" against the mathematics.  What the paper itself does not fix
+chunk attention in test_oracle_chunk_attn.py, Norm and RoPE in test_oracle_prologue.py, the attention-aware Hessians in test_oracle_hessians.py); none is "parity unpinned" against the mathematics.  What the paper itself does not fix
 (quantile interpolation rule, tie rounding, storage precision of scale and
 zero, the boundary used at attention time) cannot be pinned to the paper; each
 such reading is listed where it is taken.
@@ -133,6 +133,53 @@ def gram_hessian(K, Q):
     for g in range(Q.shape[0]):
         H += Q[g].T @ Q[g]
     return M, 2.0 * H
+
+
+def causal_probabilities(Q, K, tau: float):
+    """Attention probabilities of one query head over one key head (Section 4.1): P[t, s] =
+    softmax_s(q_t . k_s / tau) over s <= t, zero for s > t.  Q, K are [S][d] rows."""
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    S = Q.shape[0]
+    logits = Q @ K.T / tau
+    logits[np.triu_indices(S, k=1)] = -np.inf
+    logits -= logits.max(axis=1, keepdims=True)
+    E = np.exp(logits)
+    return E / E.sum(axis=1, keepdims=True)
+
+
+def attention_hessians(Q, K, V, W_O, tau: float):
+    """Appendix C: the attention-aware Hessians of one key/value head over one calibration sequence, summed
+    over the perturbed position s as the WUSH-A aggregation does ("Aggregation for WUSH-A").
+      Q   [S][G][d_k]   queries of the G heads that read this key/value head (after Norm and RoPE)
+      K   [S][d_k], V [S][d_v]
+      W_O [G][d_v][d_model]   output-projection blocks
+    Returns (H_K [d_k][d_k], H_V [d_v][d_v]) with H = 2 sum_s sum_t J_{t,s}^T J_{t,s}, where J_{t,s} is the derivative
+    of the module output y_t with respect to a perturbation of k_s (key Jacobian) or of v_s (value Jacobian), taken
+    literally from the appendix:
+      key:   J = (1/tau) sum_g p_{g,t,s} W_O(g)^T (v_s - o_{g,t}) q_{g,t}^T      [d_model x d_k]
+      value: J = sum_g p_{g,t,s} W_O(g)^T                                       [d_model x d_v]
+    Plain loops over (s, t): for small calibration problems only."""
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    W_O = np.asarray(W_O, dtype=np.float64)
+    S, G, dk = Q.shape
+    dv = V.shape[1]
+    P = [causal_probabilities(Q[:, g], K, tau) for g in range(G)]          # [G] x [t][s]
+    Oh = [P[g] @ V for g in range(G)]                                      # head outputs o_{g,t}
+    H_K = np.zeros((dk, dk))
+    H_V = np.zeros((dv, dv))
+    for s in range(S):
+        for t in range(s, S):
+            Jk = np.zeros((W_O.shape[2], dk))
+            Jv = np.zeros((W_O.shape[2], dv))
+            for g in range(G):
+                Jk += P[g][t, s] * np.outer(W_O[g].T @ (V[s] - Oh[g][t]), Q[t, g]) / tau
+                Jv += P[g][t, s] * W_O[g].T
+            H_K += 2.0 * Jk.T @ Jk
+            H_V += 2.0 * Jv.T @ Jv
+    return H_K, H_V
 
 
 def build_transforms(M, H, gamma: float = 1e-2):
