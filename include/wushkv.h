@@ -244,6 +244,27 @@ int wushkv_prefill_attn(const wushkv_cache* cache, int32_t batch, const int32_t*
                         void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Attention-aware Hessians for the WUSH-A variant (Appendix C, "Aggregation for WUSH-A"): for ONE calibration
+ * sequence and every key/value head, the key Hessian and the value Hessian of the module-output error, summed over
+ * the perturbed cache position, added to the caller's float64 accumulators (call once per sequence; pass the sums
+ * to wushkv_build_transforms[_device] in place of Eq. 4's Hessians).  They depend on the causal attention
+ * probabilities p = softmax(q . k / tau), the head outputs and the output projection only (forward quantities).
+ *   K, Q, V (device): bf16 [n_tokens][n_kv][d], [n_tokens][n_q][d], [n_tokens][n_kv][d]; K and Q after Norm and RoPE,
+ *                     V as projected (not folded).
+ *   W_O (device):     fp32 [n_q][d][d_model], the output-projection block of every query head.
+ *   tau:              the logit temperature (sqrt(d) in the paper).
+ *   H_K, H_V (device, in/out): float64 [n_kv][d][d], accumulated.
+ *   workspace (device): >= wushkv_attention_hessians_workspace_bytes() bytes, 256-byte aligned, scratch.
+ * d must be 128 and the group size n_q / n_kv at most 4 (WUSHKV_EINVAL otherwise).  Cost O(n_tokens^2) per head.
+ * Arithmetic: fp32 with float64 accumulation of the sums over tokens.
+ */
+size_t wushkv_attention_hessians_workspace_bytes(int32_t n_kv, int32_t n_q, int32_t d, int64_t n_tokens);
+int wushkv_accumulate_attention_hessians_device(int32_t n_kv, int32_t n_q, int32_t d, int32_t d_model, int64_t n_tokens,
+                                                const uint16_t* K, const uint16_t* Q, const uint16_t* V, const float* W_O,
+                                                double tau, double* H_K, double* H_V,
+                                                void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Projected inputs: Algorithm 2 lines 1-2 (Norm, RoPE) fused into the kernels that apply line 3, so that
  * keys and queries are read once, in the form the projections W_K x, W_Q x left them, and their normalised,
  * rotated form never goes through memory (Section 4.1: keys are cached after normalisation and rotation).

@@ -24,6 +24,7 @@ EXPORTS = (
     "wushkv_decode_attn_static", "wushkv_set_test_option", "wushkv_prefill_workspace_bytes", "wushkv_prefill_attn",
     "wushkv_accumulate_gram_device", "wushkv_build_transforms_workspace_bytes", "wushkv_build_transforms_device",
     "wushkv_build_rope_table", "wushkv_append_projected", "wushkv_decode_attn_projected",
+    "wushkv_attention_hessians_workspace_bytes", "wushkv_accumulate_attention_hessians_device",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -117,6 +118,12 @@ def _load():
     lib.wushkv_decode_attn_projected.restype = C.c_int
     lib.wushkv_decode_attn_projected.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_void_p, C.c_void_p, C.c_int32,
                                                  C.c_void_p, C.POINTER(wushkv_prologue), C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.wushkv_attention_hessians_workspace_bytes.restype = C.c_size_t
+    lib.wushkv_attention_hessians_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int64]
+    lib.wushkv_accumulate_attention_hessians_device.restype = C.c_int
+    lib.wushkv_accumulate_attention_hessians_device.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_void_p,
+                                                                C.c_void_p, C.c_void_p, C.c_void_p, C.c_double, C.c_void_p,
+                                                                C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
     lib.wushkv_set_test_option.restype = C.c_int
     lib.wushkv_set_test_option.argtypes = [C.c_char_p, C.c_longlong]
     return lib
@@ -206,6 +213,21 @@ def build_transforms_device(M, H, gamma: float, stream=None):
 def append(cache: wushkv_cache, batch, slot, seq_len, cu_new, total_new, max_new, K_new, V_new, stream=None):
     _check(lib.wushkv_append(C.byref(cache), batch, _ptr(slot), _ptr(seq_len), _ptr(cu_new), total_new, max_new,
                              _ptr(K_new), _ptr(V_new), _stream_ptr(stream)), "wushkv_append")
+
+
+def accumulate_attention_hessians_device(K_bits, Q_bits, V_bits, W_O, tau: float, H_K, H_V, stream=None):
+    """wushkv_accumulate_attention_hessians_device: K_bits / V_bits [n_tok][n_kv][d], Q_bits [n_tok][n_q][d] (bf16 patterns),
+    W_O fp32 [n_q][d][d_model], H_K / H_V float64 [n_kv][d][d] (accumulated), all CUDA tensors; the scratch is allocated here."""
+    import torch
+    n_tok, n_kv, d = K_bits.shape
+    n_q, d_model = Q_bits.shape[1], W_O.shape[2]
+    nbytes = int(lib.wushkv_attention_hessians_workspace_bytes(n_kv, n_q, d, n_tok))
+    if nbytes == 0:
+        raise WushkvError(EINVAL, "wushkv_attention_hessians_workspace_bytes")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=K_bits.device)
+    _check(lib.wushkv_accumulate_attention_hessians_device(n_kv, n_q, d, d_model, n_tok, _ptr(K_bits), _ptr(Q_bits), _ptr(V_bits),
+                                                           _ptr(W_O), float(tau), _ptr(H_K), _ptr(H_V), _ptr(ws), nbytes,
+                                                           _stream_ptr(stream)), "wushkv_accumulate_attention_hessians_device")
 
 
 class Prologue:

@@ -15,7 +15,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libwushkv.so")
-SOURCES = ["api.cu", "transforms_host.cpp", "append.cu", "decode.cu", "decode_static.cu", "prefill.cu", "calibrate.cu"]
+SOURCES = ["api.cu", "transforms_host.cpp", "append.cu", "decode.cu", "decode_static.cu", "prefill.cu", "calibrate.cu", "hessians.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 
