@@ -52,6 +52,7 @@ struct Knobs {
     long long drop_copy_unit = -1;  // >= 0: the decode main kernel never issues the copy of this unit of the flattened list
     long long wait_limit = 0;       // > 0: poll limit of the device-side barrier waits (default: about a second)
     int drop_chunk_mma = 0;         // 1: the chunk append never commits its first tile's MMAs to the barrier
+    int prefill_legacy = 0;         // 1: chunk attention on the mma.sync kernel instead of the tcgen05 one
 };
 Knobs& knobs();
 

@@ -412,6 +412,392 @@ __global__ void __launch_bounds__(PF_THREADS) prefill_attn_kernel(PrefillParams 
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// 2b. attention on tcgen05 (the default path)
+// ------------------------------------------------------------------------------------------------
+// One CTA of 128 threads per (sequence, KV head, tile of R = 128 / G chunk positions): the G query heads that
+// read the KV head are packed into the M = 128 rows of the tile (row r = position r / G, head r % G), so a staged
+// key / value tile serves all of them.  Per 64-key tile:
+//   S = Q' K^T     16 x tcgen05.mma.kind::f16, M 128, N 64, K 16 (fp16 value and remainder of q' against the same
+//                  keys), fp32 accumulator in tensor memory (64 columns);
+//   softmax        thread r reads row r with tcgen05.ld, applies the affine factors and the causal mask, keeps a
+//                  lazily raised reference (the accumulator row in tensor memory is rescaled only when the row
+//                  maximum grows by more than 2^6) and writes (p Delta_v) as fp16 into the A-operand layout;
+//   O += P V       4 x tcgen05.mma, M 128, N 128, K 16, the value tile as an MN-major B operand, accumulator in
+//                  tensor memory (128 columns).
+// Operands use the no-swizzle canonical layouts: K-major tiles (Q', K, P) as 8-row x 16-byte core matrices at
+// (row / 8) * SBO + (k / 8) * 128 + (row % 8) * 16; the MN-major value tile as 8-key x 16-byte core matrices at
+// (channel / 8) * SBO + (key / 8) * 128 + (key % 8) * 16.  Every wait on the MMA barrier is bounded.
+constexpr int TM = 128;                       // rows of the packed query tile
+constexpr int TN = 64;                        // keys per tile (= one packed page)
+constexpr int TC_Q_BYTES = TM * D * 2;        // one fp16 query operand
+constexpr int TC_K_BYTES = TN * D * 2;        // key tile; reused for P (TM x TN fp16 is the same size)
+constexpr int TC_OFF_Q = 0;
+constexpr int TC_OFF_K = 2 * TC_Q_BYTES;
+constexpr int TC_OFF_V = TC_OFF_K + TC_K_BYTES;
+constexpr int TC_OFF_META = TC_OFF_V + TC_K_BYTES;             // float4[TN]
+constexpr int TC_OFF_POS = TC_OFF_META + TN * 16;              // int[TN]
+constexpr int TC_OFF_RAW = TC_OFF_POS + TN * 4;                // one packed record
+constexpr int TC_OFF_BAR = TC_OFF_RAW + 8704;                  // mbarrier, tensor-memory slot
+constexpr int TC_SMEM = TC_OFF_BAR + 64;
+constexpr float REF_SLACK = 6.f;              // log2 headroom of the lazily raised softmax reference
+constexpr unsigned TC_TMEM_COLS = 256;        // O: columns 0..127, S: columns 128..191
+constexpr unsigned TC_IDESC_S = (1u << 4) | ((TN >> 3) << 17) | ((TM >> 4) << 24);                  // fp32 <- fp16 x fp16, both K-major
+constexpr unsigned TC_IDESC_O = (1u << 4) | (1u << 16) | ((D >> 3) << 17) | ((TM >> 4) << 24);      // B (values) MN-major
+
+__device__ __forceinline__ unsigned long long tc_desc(unsigned addr, unsigned lbo, unsigned sbo) {
+    unsigned long long d = 0;
+    d |= static_cast<unsigned long long>((addr >> 4) & 0x3FFFu);
+    d |= static_cast<unsigned long long>((lbo >> 4) & 0x3FFFu) << 16;
+    d |= static_cast<unsigned long long>((sbo >> 4) & 0x3FFFu) << 32;
+    d |= 1ull << 46;
+    return d;
+}
+__device__ __forceinline__ void tc_mma(unsigned tmem, unsigned long long adesc, unsigned long long bdesc, unsigned idesc, unsigned accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+        ::"r"(tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(unsigned taddr, float (&v)[32]) {
+    unsigned r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tc_st32(unsigned taddr, const float (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        ::"r"(taddr),
+          "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+          "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+          "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+          "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
+          "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+          "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+          "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
+          "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+        : "memory");
+}
+__device__ __forceinline__ void cp16(unsigned dst, const void* src, unsigned bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P) {
+    extern __shared__ __align__(1024) unsigned char sm_tc[];
+    const CacheView& c = P.c;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int G = c.G, R = TM / G;                              // chunk positions per tile
+    const int qt = P.tiles_per_seq - 1 - static_cast<int>(blockIdx.x % P.tiles_per_seq);      // long tiles first
+    const int b = blockIdx.x / P.tiles_per_seq, h = blockIdx.y;
+    const int first = __ldg(P.cu_new + b), n_new = __ldg(P.cu_new + b + 1) - first;
+    if (qt * R >= n_new) return;
+    const int S = __ldg(P.seq_len + b), sl = __ldg(P.slot + b);
+    if (sl < 0 || sl >= c.n_slots || S < n_new) {
+        if (tid == 0) atomicOr(c.dev_status, WUSHKV_DEV_BAD_SLOT);
+        return;
+    }
+    unsigned char* sQ = sm_tc + TC_OFF_Q;
+    unsigned char* sK = sm_tc + TC_OFF_K;                       // key tile, then the probabilities of the same tile
+    unsigned char* sV = sm_tc + TC_OFF_V;
+    float4* meta = reinterpret_cast<float4*>(sm_tc + TC_OFF_META);
+    int* kpos = reinterpret_cast<int*>(sm_tc + TC_OFF_POS);
+    unsigned char* raw = sm_tc + TC_OFF_RAW;
+    unsigned long long* mbar = reinterpret_cast<unsigned long long*>(sm_tc + TC_OFF_BAR);
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(sm_tc + TC_OFF_BAR + 16);
+
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(TC_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(mbar)) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    const int S0 = S - n_new;
+    const int nq = n_quantized(S - c.lag, c.s_sink, c.s_keep, c.s_flush);
+    const int q_lo = c.s_sink, q_hi = min(c.s_sink + nq, S0);
+    const int a_hi = min(c.s_sink, S0);
+    const int c_lo = max(q_hi, a_hi);
+    const int n_old_fp = a_hi + max(S0 - c_lo, 0);
+    const float k2 = c.sm_scale * LOG2E_F;
+
+    // ---- the packed query tile: row r = chunk position qt R + r / G (clamped to the chunk), head h G + r % G
+    const int n_rows = min(R, n_new - qt * R) * G;              // rows that carry a query
+    for (int item = tid; item < 2 * TM * 16; item += TM) {
+        const int part = item / (TM * 16), r = (item >> 4) % TM, piece = item & 15;
+        const int rr = min(r, n_rows - 1);
+        const int tok = first + qt * R + rr / G, jq = h * G + rr % G;
+        const __half* src = P.QP + static_cast<long long>(part) * P.total_new * c.n_q * D + (static_cast<long long>(tok) * c.n_q + jq) * D + 8 * piece;
+        cp16(smem_addr(sQ + part * TC_Q_BYTES + (r >> 3) * 2048 + piece * 128 + (r & 7) * 16), src, 16u);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    const int my_r = min(tid, n_rows - 1);
+    const int my_tok = first + qt * R + my_r / G, my_jq = h * G + my_r % G;
+    const float my_qsum = __ldcg(P.qsum + static_cast<long long>(my_tok) * c.n_q + my_jq);
+    const int my_pos = S0 + qt * R + my_r / G;                  // causal limit of this thread's row
+    const int tile_pos_lo = S0 + qt * R;                        // smallest causal limit of the tile
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const unsigned tmem_base = *tmem_slot;
+    const unsigned tmem_row = tmem_base + (static_cast<unsigned>(warp * 32) << 16);
+    unsigned phase = 0;
+    bool failed = false, have_o = false;
+    float m_ref = -INFINITY, l = 0.f, z = 0.f;
+    const int wait_limit = 1 << 20;                            // polls that may sleep ~2 us each: about two seconds
+
+    auto wait_mma = [&]() -> bool {                             // bounded; the decision is uniform for the CTA
+        bool done = false;
+        for (int it = 0; it < wait_limit && !done; ++it) {
+            unsigned ok;
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                         : "=r"(ok) : "r"(smem_addr(mbar)), "r"(phase), "r"(2000u) : "memory");
+            done = ok != 0;
+        }
+        if (!__syncthreads_and(done ? 1 : 0)) return false;
+        phase ^= 1u;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        return true;
+    };
+
+    // One staged tile: S = Q' K^T, softmax of this thread's row, O += P V.  `masked`: some key of the tile may be
+    // invisible to some row (padding, or a chunk position beyond the row's own).
+    auto consume = [&](const bool masked) {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncthreads();
+        if (tid == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const unsigned long long bdesc = tc_desc(smem_addr(sK) + ks * 256, 128, 2048);
+                tc_mma(tmem_base + 128, tc_desc(smem_addr(sQ) + ks * 256, 128, 2048), bdesc, TC_IDESC_S, ks > 0 ? 1u : 0u);
+                tc_mma(tmem_base + 128, tc_desc(smem_addr(sQ + TC_Q_BYTES) + ks * 256, 128, 2048), bdesc, TC_IDESC_S, 1u);
+            }
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(mbar)) : "memory");
+        }
+        if (!wait_mma()) { failed = true; return; }
+        // ---- this thread's row of scores
+        float s[TN];
+        {
+            float lo[32], hi[32];
+            tc_ld32(tmem_row + 128, lo);
+            tc_ld32(tmem_row + 160, hi);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) { s[i] = lo[i]; s[32 + i] = hi[i]; }
+        }
+        float mx = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < TN; ++j) {
+            const float4 mt = meta[j];
+            float v = k2 * fmaf(mt.y, my_qsum, mt.x * s[j]);
+            if (masked) { const int kp = kpos[j]; if (kp < 0 || kp > my_pos) v = -INFINITY; }
+            s[j] = v;
+            mx = fmaxf(mx, v);
+        }
+        const bool raise = mx > m_ref + REF_SLACK;                 // also the first finite maximum (m_ref = -inf)
+        const float new_ref = raise ? mx : m_ref;
+        const float factor = raise ? fast_ex2(m_ref - new_ref) : 1.f;      // old reference -inf: factor 0, state is zero anyway
+        if (__any_sync(FULLM, raise) && have_o) {                  // rescale this warp's accumulator rows in tensor memory
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+                float o[32];
+                tc_ld32(tmem_row + 32 * q4, o);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o[i] *= factor;
+                tc_st32(tmem_row + 32 * q4, o);
+            }
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        }
+        l *= factor; z *= factor;
+        m_ref = new_ref;
+        const float ref = m_ref == -INFINITY ? 0.f : m_ref;
+        // ---- probabilities: (p Delta_v) as fp16 into the A-operand layout (over the key tile, which is consumed)
+        unsigned char* prow = sK + (tid >> 3) * 1024 + (tid & 7) * 16;
+#pragma unroll
+        for (int kc = 0; kc < TN / 8; ++kc) {
+            float w[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float4 mt = meta[8 * kc + e];
+                const float p = fast_ex2(s[8 * kc + e] - ref);
+                l += p;
+                z = fmaf(p, mt.w, z);
+                w[e] = p * mt.z;
+            }
+            *reinterpret_cast<uint4*>(prow + kc * 128) = make_uint4(pack_half2(w[0], w[1]), pack_half2(w[2], w[3]), pack_half2(w[4], w[5]), pack_half2(w[6], w[7]));
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncthreads();
+        if (tid == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+            for (int ks = 0; ks < TN / 16; ++ks)
+                tc_mma(tmem_base, tc_desc(smem_addr(sK) + ks * 256, 128, 1024), tc_desc(smem_addr(sV) + ks * 256, 128, 1024), TC_IDESC_O,
+                       (have_o || ks > 0) ? 1u : 0u);
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(mbar)) : "memory");
+        }
+        have_o = true;
+        if (!wait_mma()) { failed = true; return; }              // the tile buffers and the accumulator are free again
+    };
+
+    // ---- (1) full-precision old positions: sink [0, a_hi) and recent window [c_lo, S0), bf16 rows
+    for (int base = 0; base < n_old_fp && !failed; base += TN) {
+        for (int item = tid; item < TN * 16; item += TM) {
+            const int r = item >> 4, piece = item & 15, idx = base + r;
+            uint4 kh = make_uint4(0, 0, 0, 0), vh = kh;
+            if (idx < n_old_fp) {
+                const long long plane = (static_cast<long long>(sl) * c.n_kv + h) * 2;
+                const unsigned short *ksrc, *vsrc;
+                if (idx < a_hi) {
+                    ksrc = c.sink_kv + (plane * c.s_sink + idx) * D;
+                    vsrc = c.sink_kv + ((plane + 1) * c.s_sink + idx) * D;
+                } else {
+                    const int p = c_lo + (idx - a_hi);
+                    ksrc = c.ring_kv + (plane * c.ring_cap + p % c.ring_cap) * D;
+                    vsrc = c.ring_kv + ((plane + 1) * c.ring_cap + p % c.ring_cap) * D;
+                }
+                const uint4 kb16 = *reinterpret_cast<const uint4*>(ksrc + 8 * piece), vb16 = *reinterpret_cast<const uint4*>(vsrc + 8 * piece);
+                const unsigned kw[4] = {kb16.x, kb16.y, kb16.z, kb16.w}, vw[4] = {vb16.x, vb16.y, vb16.z, vb16.w};
+                unsigned ko[4], vo[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    ko[e] = pack_half2(bf16_bits_to_float(kw[e] & 0xffff), bf16_bits_to_float(kw[e] >> 16));
+                    vo[e] = pack_half2(bf16_bits_to_float(vw[e] & 0xffff), bf16_bits_to_float(vw[e] >> 16));
+                }
+                kh = make_uint4(ko[0], ko[1], ko[2], ko[3]); vh = make_uint4(vo[0], vo[1], vo[2], vo[3]);
+            }
+            *reinterpret_cast<uint4*>(sK + (r >> 3) * 2048 + piece * 128 + (r & 7) * 16) = kh;
+            *reinterpret_cast<uint4*>(sV + piece * 1024 + (r >> 3) * 128 + (r & 7) * 16) = vh;
+            if (piece == 0) {
+                meta[r] = make_float4(1.f, 0.f, 1.f, 0.f);
+                kpos[r] = idx < n_old_fp ? (idx < a_hi ? idx : c_lo + (idx - a_hi)) : -1;
+            }
+        }
+        consume(base + TN > n_old_fp);
+    }
+
+    // ---- (2) quantized positions below the chunk: one packed page per tile, staged as integer codes
+    if (q_hi > q_lo) {
+        constexpr int REC = record_bytes(BITS);
+        const int page_first = q_lo / PAGE_TOKENS, page_last = (q_hi - 1) / PAGE_TOKENS;
+        for (int pg = page_first; pg <= page_last && !failed; ++pg) {
+            int page = -1;
+            if (pg < c.max_pages) page = __ldg(c.page_table + static_cast<long long>(sl) * c.max_pages + pg);
+            const bool page_ok = page >= 0 && page < c.n_pages;
+            if (!page_ok && tid == 0) atomicOr(c.dev_status, pg < c.max_pages ? WUSHKV_DEV_BAD_PAGE_ID : WUSHKV_DEV_PAGE_TABLE_FULL);
+            if (page_ok) {
+                const uint4* src = reinterpret_cast<const uint4*>(c.pages + (static_cast<long long>(page) * c.n_kv + h) * REC);
+                for (int k = tid; k < REC / 16; k += TM) reinterpret_cast<uint4*>(raw)[k] = __ldg(src + k);
+            }
+            __syncthreads();
+            {   // thread -> token r = tid & 63, channels (tid >> 6) * 64 .. + 63, eight at a time
+                const int r = tid & 63, ch0 = (tid >> 6) * 64;
+                const int pos = pg * PAGE_TOKENS + r;
+                const bool live = page_ok && pos >= q_lo && pos < q_hi;
+                constexpr unsigned MASK = (1u << (BITS == 3 ? 2 : BITS)) - 1u;
+                auto field_at = [&](int off, int bit, unsigned mask) { return (static_cast<unsigned>(raw[off + (bit >> 3)]) >> (bit & 7)) & mask; };
+                for (int kc = ch0 / 8; kc < ch0 / 8 + 8; ++kc) {
+                    float kf[8], vf[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        unsigned ck = 0, cv = 0;
+                        if (live) {
+                            int off, bit;
+                            k_code_location(BITS, r, 8 * kc + e, off, bit); ck = field_at(off, bit, MASK);
+                            v_code_location(BITS, r, 8 * kc + e, off, bit); cv = field_at(off, bit, MASK);
+                            if (BITS == 3) {
+                                k_hi_location(r, 8 * kc + e, off, bit); ck |= field_at(off, bit, 1u) << 2;
+                                v_hi_location(r, 8 * kc + e, off, bit); cv |= field_at(off, bit, 1u) << 2;
+                            }
+                        }
+                        kf[e] = static_cast<float>(ck); vf[e] = static_cast<float>(cv);
+                    }
+                    *reinterpret_cast<uint4*>(sK + (r >> 3) * 2048 + kc * 128 + (r & 7) * 16) =
+                        make_uint4(pack_half2(kf[0], kf[1]), pack_half2(kf[2], kf[3]), pack_half2(kf[4], kf[5]), pack_half2(kf[6], kf[7]));
+                    *reinterpret_cast<uint4*>(sV + kc * 1024 + (r >> 3) * 128 + (r & 7) * 16) =
+                        make_uint4(pack_half2(vf[0], vf[1]), pack_half2(vf[2], vf[3]), pack_half2(vf[4], vf[5]), pack_half2(vf[6], vf[7]));
+                }
+                if (ch0 == 0) {
+                    float4 mt = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (live) {
+                        const __half* mh = reinterpret_cast<const __half*>(raw + meta_location(BITS, r));
+                        mt = make_float4(__half2float(mh[0]), __half2float(mh[1]), __half2float(mh[2]), __half2float(mh[3]));
+                    }
+                    meta[r] = mt;
+                    kpos[r] = live ? pos : -1;
+                }
+            }
+            consume(true);
+        }
+    }
+
+    // ---- (3) the chunk itself, causal: key tiles up to the tile's last position
+    const int last_row = min(qt * R + R, n_new) - 1;
+    for (int kt = 0; kt * TN <= last_row && !failed; ++kt) {
+        for (int item = tid; item < TN * 16; item += TM) {
+            const int r = item >> 4, piece = item & 15, row = kt * TN + r;
+            const bool in = row < n_new;
+            const long long off = (static_cast<long long>(first + (in ? row : 0)) * c.n_kv + h) * D + 8 * piece;
+            cp16(smem_addr(sK + (r >> 3) * 2048 + piece * 128 + (r & 7) * 16), P.KP + off, in ? 16u : 0u);
+            cp16(smem_addr(sV + piece * 1024 + (r >> 3) * 128 + (r & 7) * 16), P.VP + off, in ? 16u : 0u);
+            if (piece == 0) {
+                meta[r] = make_float4(1.f, 0.f, 1.f, 0.f);
+                kpos[r] = in ? S0 + row : -1;
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        // no mask needed when every key of the tile exists and lies at or below every row's own position
+        consume(!(kt * TN + TN <= n_new && S0 + kt * TN + TN - 1 <= tile_pos_lo));
+    }
+
+    // ---- output: o = (O + z) / l for the rows that carry a query
+    if (!failed && have_o) {
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        float* dst = P.O + (static_cast<long long>(my_tok) * c.n_q + my_jq) * D;
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+            float o[32];
+            tc_ld32(tmem_row + 32 * q4, o);
+            if (tid < n_rows) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 4)
+                    *reinterpret_cast<float4*>(dst + 32 * q4 + i) = make_float4((o[i] + z) * inv, (o[i + 1] + z) * inv, (o[i + 2] + z) * inv, (o[i + 3] + z) * inv);
+            }
+        }
+    }
+    if (failed) {
+        // commit whatever was issued once more and give it a bounded time, so that no MMA is still writing tensor
+        // memory when it is released below
+        if (tid == 0) {
+            atomicOr(c.dev_status, WUSHKV_DEV_COPY_TIMEOUT);
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(mbar)) : "memory");
+        }
+        for (int it = 0; it < 512; ++it) {
+            unsigned ok;
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                         : "=r"(ok) : "r"(smem_addr(mbar)), "r"(phase), "r"(2000u) : "memory");
+            if (ok) break;
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TC_TMEM_COLS) : "memory");
+}
+
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
 struct PrefillPlan { size_t off_kp, off_vp, off_qp, off_qsum, total; };
@@ -467,6 +853,20 @@ extern "C" int wushkv_prefill_attn(const wushkv_cache* cache, int32_t batch, con
     if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(prefill_prep_kernel), static_cast<int>(smem_prep))) return WUSHKV_ECUDA;
     prefill_prep_kernel<<<dim3((total_new + PREP_TOK - 1) / PREP_TOK, P.c.n_kv + P.c.n_q), 256, smem_prep, st>>>(P);
     if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
+    if (!knobs().prefill_legacy) {              // tcgen05 path: the G heads of a KV head share a 128-row tile
+        const int R = TM / P.c.G;
+        P.tiles_per_seq = (max_new + R - 1) / R;
+        const dim3 grid_tc(static_cast<unsigned>(batch) * P.tiles_per_seq, P.c.n_kv);
+        auto launch = [&](auto kernel) -> bool {
+            if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(kernel), TC_SMEM)) return false;
+            kernel<<<grid_tc, TM, TC_SMEM, st>>>(P);
+            return true;
+        };
+        const bool ok = P.c.bits == 2 ? launch(prefill_attn_tc_kernel<2>) : P.c.bits == 3 ? launch(prefill_attn_tc_kernel<3>)
+                                                                                         : launch(prefill_attn_tc_kernel<4>);
+        if (!ok) return WUSHKV_ECUDA;
+        return cudaGetLastError() == cudaSuccess ? WUSHKV_OK : WUSHKV_ECUDA;
+    }
     const dim3 grid(static_cast<unsigned>(batch) * P.tiles_per_seq, P.c.n_q);
     const size_t smem_attn = sizeof(TileSmem);
     if (P.c.bits == 2) {

@@ -9,6 +9,14 @@ from tests.harness import CODE_MISMATCH_MAX, Layer
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(params=["tcgen05", "mma_sync"], autouse=True)
+def attention_path(request, test_option):
+    """Every case runs on both attention kernels: the tcgen05 one (default) and the mma.sync one."""
+    if request.param == "mma_sync":
+        test_option("prefill_legacy", 1)
+    return request.param
+
+
 def _wl(n_q, n_kv, seed, batch=1, theta=1e4, rmsnorm=False):
     return W.LayerWorkload(dict(seed=seed, batch=batch, n_q=n_q, n_kv=n_kv, ctx=0, theta=theta, bits=2, s_sink=4,
                                 s_keep=64, rmsnorm=rmsnorm, ragged=None, prefill_chunk=0))
