@@ -23,6 +23,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <type_traits>
 
 #include "host_common.h"
 #include "layout.cuh"
@@ -76,75 +77,122 @@ __device__ __forceinline__ unsigned pack_half2(float lo, float hi) {
 // ------------------------------------------------------------------------------------------------
 // 1. transforms of the chunk (Algorithm 2 line 3)
 // ------------------------------------------------------------------------------------------------
-// One CTA per (tile of 32 tokens, head slot); head slots 0 .. n_kv-1 are the key heads, the rest the query heads.
-// The 128 x 128 transform sits transposed in shared memory; thread (channel i, token group) accumulates 16 tokens.
-constexpr int PREP_TOK = 32;
+// One CTA of 8 warps per (tile of 128 tokens, head slot); head slots 0 .. n_kv-1 are the key heads, the rest the
+// query heads.  out[token][i] = sum_j x[token][j] T[i][j] on tensor cores (mma.sync bf16, fp32 accumulation): the
+// token tile is the A operand as it comes (bf16), the transform the B operand.  T_K is bf16-valued (one term);
+// T_K^{-T} is fp32 and is fed as three bf16 terms (value, remainder, remainder of the remainder: 24 mantissa bits),
+// so the products are exact and the result is the fp32 dot product up to summation order.
+constexpr int PREP_TOK = 128;
+constexpr int PREP_PITCH = D + 8;             // bf16 per staged row (272 bytes: conflict-free ldmatrix)
+__device__ __forceinline__ void mma_bf16_prep(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0, unsigned b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
 __global__ void __launch_bounds__(256) prefill_prep_kernel(PrefillParams P) {
-    extern __shared__ __align__(16) float sm[];
-    float* Tt = sm;                               // [D][D + 1]: Tt[j][i] = T[i][j]
-    float* X = sm + D * (D + 1);                  // [PREP_TOK][D]
+    extern __shared__ __align__(16) unsigned short sm16[];
+    unsigned short* Xs = sm16;                            // [PREP_TOK][PREP_PITCH]
+    unsigned short* Ts = sm16 + PREP_TOK * PREP_PITCH;    // [terms][D][PREP_PITCH]: Ts[term][i][j] = term of T[i][j]
     const int hs = blockIdx.y, tok0 = blockIdx.x * PREP_TOK;
     const bool is_key = hs < P.c.n_kv;
     const int head = is_key ? hs : hs - P.c.n_kv;
     const int kvh = is_key ? head : head / P.c.G;
+    const int n_terms = is_key ? 1 : 3;
     const float* T = (is_key ? P.c.T_K : P.c.T_K_invT) + static_cast<long long>(kvh) * D * D;
-    for (int idx = threadIdx.x; idx < D * D; idx += 256) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+    for (int idx = tid; idx < D * D; idx += 256) {
         const int i = idx >> 7, j = idx & 127;
-        Tt[j * (D + 1) + i] = __ldg(T + idx);
+        float x = __ldg(T + idx);
+#pragma unroll
+        for (int term = 0; term < 3; ++term) {
+            if (term < n_terms) {
+                const unsigned short hb = float_to_bf16_bits(x);
+                Ts[(term * D + i) * PREP_PITCH + j] = hb;
+                x -= bf16_bits_to_float(hb);
+            }
+        }
     }
     const int n_heads = is_key ? P.c.n_kv : P.c.n_q;
     const unsigned short* src = is_key ? P.K_new : P.Q_new;
-    for (int idx = threadIdx.x; idx < PREP_TOK * D; idx += 256) {
-        const int tk = idx >> 7, ch = idx & 127;
-        const int tok = tok0 + tk;
-        X[idx] = tok < P.total_new ? bf16_bits_to_float(__ldg(src + (static_cast<long long>(tok) * n_heads + head) * D + ch)) : 0.f;
+    for (int item = tid; item < PREP_TOK * 16; item += 256) {
+        const int r = item >> 4, piece = item & 15, tok = tok0 + r;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (tok < P.total_new) v = __ldg(reinterpret_cast<const uint4*>(src + (static_cast<long long>(tok) * n_heads + head) * D + 8 * piece));
+        *reinterpret_cast<uint4*>(Xs + r * PREP_PITCH + 8 * piece) = v;
     }
-    __syncthreads();
-    const int i = threadIdx.x & 127, tg = threadIdx.x >> 7;          // output channel, token group (16 tokens each)
-    float acc[16];
-#pragma unroll
-    for (int k = 0; k < 16; ++k) acc[k] = 0.f;
-    for (int j = 0; j < D; ++j) {
-        const float tji = Tt[j * (D + 1) + i];
-#pragma unroll
-        for (int k = 0; k < 16; ++k) acc[k] = fmaf(tji, X[(tg * 16 + k) * D + j], acc[k]);
-    }
-    __syncthreads();                                                  // X is reused for the row sums
-    float* rowsum = X;                                                // [PREP_TOK][4 warps of this token group]
-#pragma unroll
-    for (int k = 0; k < 16; ++k) {
-        const int tok = tok0 + tg * 16 + k;
-        float val = acc[k];
-        __half hv, lv = __float2half_rn(0.f);
-        if (is_key) hv = __float2half_rn(bf16_bits_to_float(float_to_bf16_bits(val)));   // the cache holds bf16(k')
-        else { hv = __float2half_rn(val); lv = __float2half_rn(val - __half2float(hv)); }
-        if (tok < P.total_new) {
-            const long long off = (static_cast<long long>(tok) * n_heads + head) * D + i;
-            if (is_key) P.KP[off] = hv;
-            else { P.QP[off] = hv; P.QP[static_cast<long long>(P.total_new) * n_heads * D + off] = lv; }
-        }
-        if (!is_key) {                                                // sum of the two-term q' over the 128 channels
-            float s = __half2float(hv) + __half2float(lv);
-            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(FULLM, s, o);
-            if ((threadIdx.x & 31) == 0) rowsum[(tg * 16 + k) * 4 + ((threadIdx.x & 127) >> 5)] = s;
-        }
-    }
-    if (is_key) {                                                     // the chunk's values as fp16 (no transform)
-        for (int idx = threadIdx.x; idx < PREP_TOK * D; idx += 256) {
-            const int tk = idx >> 7, ch = idx & 127, tok = tok0 + tk;
+    if (is_key) {                                         // the chunk's values as fp16 (no transform)
+        for (int item = tid; item < PREP_TOK * 16; item += 256) {
+            const int r = item >> 4, piece = item & 15, tok = tok0 + r;
             if (tok < P.total_new) {
-                const long long off = (static_cast<long long>(tok) * P.c.n_kv + head) * D + ch;
-                P.VP[off] = __float2half_rn(bf16_bits_to_float(__ldg(P.V_new + off)));
+                const long long off = (static_cast<long long>(tok) * P.c.n_kv + head) * D + 8 * piece;
+                const uint4 v = __ldg(reinterpret_cast<const uint4*>(P.V_new + off));
+                const unsigned w[4] = {v.x, v.y, v.z, v.w};
+                unsigned o[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) o[e] = pack_half2(bf16_bits_to_float(w[e] & 0xffff), bf16_bits_to_float(w[e] >> 16));
+                *reinterpret_cast<uint4*>(P.VP + off) = make_uint4(o[0], o[1], o[2], o[3]);
             }
         }
-        return;
     }
     __syncthreads();
-    if (threadIdx.x < PREP_TOK) {
-        const int tok = tok0 + threadIdx.x;
-        if (tok < P.total_new)
-            P.qsum[static_cast<long long>(tok) * P.c.n_q + head] =
-                rowsum[threadIdx.x * 4] + rowsum[threadIdx.x * 4 + 1] + rowsum[threadIdx.x * 4 + 2] + rowsum[threadIdx.x * 4 + 3];
+    // warp w: token rows 16w .. 16w+15, all 128 output channels
+    float acc[16][4];
+#pragma unroll
+    for (int nb = 0; nb < 16; ++nb) acc[nb][0] = acc[nb][1] = acc[nb][2] = acc[nb][3] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+        unsigned a0, a1, a2, a3;
+        ldsm_x4(smem_addr(Xs + (16 * warp + (lane & 7) + 8 * ((lane >> 3) & 1)) * PREP_PITCH + 16 * ks + 8 * (lane >> 4)), a0, a1, a2, a3);
+        for (int term = 0; term < n_terms; ++term) {
+            const unsigned short* Tt = Ts + term * D * PREP_PITCH;
+#pragma unroll
+            for (int nb2 = 0; nb2 < 8; ++nb2) {           // two output-channel blocks of 8 per ldmatrix.x4
+                unsigned b0, b1, b2, b3;
+                ldsm_x4(smem_addr(Tt + (16 * nb2 + 8 * (lane >> 4) + (lane & 7)) * PREP_PITCH + 16 * ks + 8 * ((lane >> 3) & 1)), b0, b1, b2, b3);
+                mma_bf16_prep(acc[2 * nb2], a0, a1, a2, a3, b0, b1);
+                mma_bf16_prep(acc[2 * nb2 + 1], a0, a1, a2, a3, b2, b3);
+            }
+        }
+    }
+    // fragment: acc[nb][0..1] = row g, channels 8nb + 2t, +1; acc[nb][2..3] = row g + 8
+    const int tok_a = tok0 + 16 * warp + g, tok_b = tok_a + 8;
+    float sum_a = 0.f, sum_b = 0.f;
+#pragma unroll
+    for (int nb = 0; nb < 16; ++nb) {
+        const int ch = 8 * nb + 2 * t;
+        if (is_key) {                                     // the cache holds bf16(k')
+            const unsigned wa = pack_half2(bf16_bits_to_float(float_to_bf16_bits(acc[nb][0])), bf16_bits_to_float(float_to_bf16_bits(acc[nb][1])));
+            const unsigned wb = pack_half2(bf16_bits_to_float(float_to_bf16_bits(acc[nb][2])), bf16_bits_to_float(float_to_bf16_bits(acc[nb][3])));
+            if (tok_a < P.total_new) *reinterpret_cast<unsigned*>(P.KP + (static_cast<long long>(tok_a) * n_heads + head) * D + ch) = wa;
+            if (tok_b < P.total_new) *reinterpret_cast<unsigned*>(P.KP + (static_cast<long long>(tok_b) * n_heads + head) * D + ch) = wb;
+        } else {                                          // q' as fp16 value + fp16 rounding remainder
+            float hv[4], lv[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                hv[e] = __half2float(__float2half_rn(acc[nb][e]));
+                lv[e] = __half2float(__float2half_rn(acc[nb][e] - hv[e]));
+            }
+            sum_a += (hv[0] + lv[0]) + (hv[1] + lv[1]);
+            sum_b += (hv[2] + lv[2]) + (hv[3] + lv[3]);
+            const long long lo_off = static_cast<long long>(P.total_new) * n_heads * D;
+            if (tok_a < P.total_new) {
+                const long long off = (static_cast<long long>(tok_a) * n_heads + head) * D + ch;
+                *reinterpret_cast<unsigned*>(P.QP + off) = pack_half2(hv[0], hv[1]);
+                *reinterpret_cast<unsigned*>(P.QP + lo_off + off) = pack_half2(lv[0], lv[1]);
+            }
+            if (tok_b < P.total_new) {
+                const long long off = (static_cast<long long>(tok_b) * n_heads + head) * D + ch;
+                *reinterpret_cast<unsigned*>(P.QP + off) = pack_half2(hv[2], hv[3]);
+                *reinterpret_cast<unsigned*>(P.QP + lo_off + off) = pack_half2(lv[2], lv[3]);
+            }
+        }
+    }
+    if (!is_key) {                                        // sum of the two-term q' over the 128 channels
+        sum_a += __shfl_xor_sync(FULLM, sum_a, 1); sum_a += __shfl_xor_sync(FULLM, sum_a, 2);
+        sum_b += __shfl_xor_sync(FULLM, sum_b, 1); sum_b += __shfl_xor_sync(FULLM, sum_b, 2);
+        if (t == 0) {
+            if (tok_a < P.total_new) P.qsum[static_cast<long long>(tok_a) * P.c.n_q + head] = sum_a;
+            if (tok_b < P.total_new) P.qsum[static_cast<long long>(tok_b) * P.c.n_q + head] = sum_b;
+        }
     }
 }
 
@@ -556,14 +604,14 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P)
     unsigned phase = 0;
     bool failed = false, have_o = false;
     float m_ref = -INFINITY, l = 0.f, z = 0.f;
-    const int wait_limit = 1 << 20;                            // polls that may sleep ~2 us each: about two seconds
+    const int wait_limit = 1 << 24;                            // polls of at least ~60 ns each: a second or more
 
     auto wait_mma = [&]() -> bool {                             // bounded; the decision is uniform for the CTA
         bool done = false;
-        for (int it = 0; it < wait_limit && !done; ++it) {
+        for (int it = 0; it < wait_limit && !done; ++it) {       // short suspensions: the MMAs of a tile take about a microsecond
             unsigned ok;
             asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                         : "=r"(ok) : "r"(smem_addr(mbar)), "r"(phase), "r"(2000u) : "memory");
+                         : "=r"(ok) : "r"(smem_addr(mbar)), "r"(phase), "r"(64u) : "memory");
             done = ok != 0;
         }
         if (!__syncthreads_and(done ? 1 : 0)) return false;
@@ -572,9 +620,11 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P)
         return true;
     };
 
-    // One staged tile: S = Q' K^T, softmax of this thread's row, O += P V.  `masked`: some key of the tile may be
-    // invisible to some row (padding, or a chunk position beyond the row's own).
-    auto consume = [&](const bool masked) {
+    // One staged tile: S = Q' K^T, softmax of this thread's row, O += P V.  PACKED: the keys carry affine factors
+    // (codes of a packed page); MASKED: some key of the tile may be invisible to some row (padding, or a chunk
+    // position beyond the row's own).  Full-precision, fully visible tiles (most of a long chunk) take the short form.
+    auto consume = [&](auto packed_tag, auto masked_tag) {
+        constexpr bool PACKED = decltype(packed_tag)::value, MASKED = decltype(masked_tag)::value;
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncthreads();
@@ -589,7 +639,7 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P)
             asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(mbar)) : "memory");
         }
         if (!wait_mma()) { failed = true; return; }
-        // ---- this thread's row of scores
+        // ---- this thread's row of scores (log2 domain after the scaling below)
         float s[TN];
         {
             float lo[32], hi[32];
@@ -601,9 +651,10 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P)
         float mx = -INFINITY;
 #pragma unroll
         for (int j = 0; j < TN; ++j) {
-            const float4 mt = meta[j];
-            float v = k2 * fmaf(mt.y, my_qsum, mt.x * s[j]);
-            if (masked) { const int kp = kpos[j]; if (kp < 0 || kp > my_pos) v = -INFINITY; }
+            float v;
+            if (PACKED) { const float4 mt = meta[j]; v = k2 * fmaf(mt.y, my_qsum, mt.x * s[j]); }
+            else v = k2 * s[j];
+            if (MASKED) { const int kp = kpos[j]; if (kp < 0 || kp > my_pos) v = -INFINITY; }
             s[j] = v;
             mx = fmaxf(mx, v);
         }
@@ -631,11 +682,10 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P)
             float w[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-                const float4 mt = meta[8 * kc + e];
                 const float p = fast_ex2(s[8 * kc + e] - ref);
                 l += p;
-                z = fmaf(p, mt.w, z);
-                w[e] = p * mt.z;
+                if (PACKED) { const float4 mt = meta[8 * kc + e]; z = fmaf(p, mt.w, z); w[e] = p * mt.z; }
+                else w[e] = p;
             }
             *reinterpret_cast<uint4*>(prow + kc * 128) = make_uint4(pack_half2(w[0], w[1]), pack_half2(w[2], w[3]), pack_half2(w[4], w[5]), pack_half2(w[6], w[7]));
         }
@@ -687,7 +737,7 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P)
                 kpos[r] = idx < n_old_fp ? (idx < a_hi ? idx : c_lo + (idx - a_hi)) : -1;
             }
         }
-        consume(base + TN > n_old_fp);
+        if (base + TN > n_old_fp) consume(std::false_type{}, std::true_type{}); else consume(std::false_type{}, std::false_type{});
     }
 
     // ---- (2) quantized positions below the chunk: one packed page per tile, staged as integer codes
@@ -741,7 +791,7 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P)
                     kpos[r] = live ? pos : -1;
                 }
             }
-            consume(true);
+            consume(std::true_type{}, std::true_type{});
         }
     }
 
@@ -761,7 +811,8 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P)
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
         // no mask needed when every key of the tile exists and lies at or below every row's own position
-        consume(!(kt * TN + TN <= n_new && S0 + kt * TN + TN - 1 <= tile_pos_lo));
+        if (kt * TN + TN <= n_new && S0 + kt * TN + TN - 1 <= tile_pos_lo) consume(std::false_type{}, std::false_type{});
+        else consume(std::false_type{}, std::true_type{});
     }
 
     // ---- output: o = (O + z) / l for the rows that carry a query
@@ -849,7 +900,7 @@ extern "C" int wushkv_prefill_attn(const wushkv_cache* cache, int32_t batch, con
     P.qsum = reinterpret_cast<float*>(ws + pl.off_qsum);
     P.tiles_per_seq = (max_new + BM - 1) / BM;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const size_t smem_prep = (static_cast<size_t>(D) * (D + 1) + PREP_TOK * D) * sizeof(float);
+    const size_t smem_prep = static_cast<size_t>(PREP_TOK + 3 * D) * PREP_PITCH * sizeof(unsigned short);
     if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(prefill_prep_kernel), static_cast<int>(smem_prep))) return WUSHKV_ECUDA;
     prefill_prep_kernel<<<dim3((total_new + PREP_TOK - 1) / PREP_TOK, P.c.n_kv + P.c.n_q), 256, smem_prep, st>>>(P);
     if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
