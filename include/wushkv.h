@@ -225,8 +225,8 @@ int wushkv_decode_attn(const wushkv_cache* cache, int32_t batch, const int32_t* 
  * Chunk (prefill) attention: Algorithm 2 line 3 (q' = T_K^{-T} q, k' = T_K k) and line 5 for a chunk of new
  * positions, evaluated AFTER wushkv_append has stored the chunk (line 4).  Chunk position i of sequence b attends
  * to cached positions 0 .. seq_len[b] - n_new[b] + i (causal inside the chunk).  The chunk's own keys and values
- * are read in full precision (k' rounded to bf16, as the cache's window copies hold it; Section 4.4: "each new
- * chunk is first appended in full precision and is used to compute its attention output"; Section 5.3), older
+ * are read in full precision (k' rounded to bf16, as the cache's window copies hold it; Sections 4.4 and 5.3: a new
+ * chunk is appended in full precision and its attention output is computed from those copies), older
  * positions by the window rule at length seq_len[b] - boundary_lag: sink and recent window from the bf16 buffers,
  * the quantized middle from the packed pages.  boundary_lag = n_new reproduces Algorithm 2 literally (boundary
  * moved after attention); ring_cap must then cover s_keep + s_flush - 1 + boundary_lag positions.
@@ -235,7 +235,8 @@ int wushkv_decode_attn(const wushkv_cache* cache, int32_t batch, const int32_t* 
  *   Q_new (device): bf16 [total_new][n_q][d] post-Norm post-RoPE queries of the chunk, NOT compensated.
  *   O (device, out): fp32 [total_new][n_q][d] in the folded value basis.
  *   workspace (device): >= wushkv_prefill_workspace_bytes() bytes, 256-byte aligned, scratch.
- * Both contractions run on tensor cores (fp16 operands, fp32 accumulation); q' is rounded to fp16.
+ * Both contractions run on the tcgen05 tensor cores (fp16 operands, fp32 accumulators in tensor memory); q' enters as
+ * an fp16 value plus its fp16 rounding remainder.  The query heads of a KV head share one 128-row tile.
  */
 size_t wushkv_prefill_workspace_bytes(const wushkv_cache* cache, int32_t batch, int32_t total_new);
 int wushkv_prefill_attn(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
@@ -399,6 +400,7 @@ int wushkv_set_profile_events(void* start, void* stop);
  *   "wait_limit"        n > 0: poll limit of the device-side barrier waits (default: about a second); 0: default.
  *   "drop_chunk_mma"    1: the chunk append does not commit the MMAs of its first tile to their barrier (same
  *                       failure path in that kernel).
+ *   "prefill_legacy"    1: wushkv_prefill_attn runs its mma.sync kernel instead of the tcgen05 one.
  * Returns WUSHKV_EINVAL for an unknown name.
  */
 int wushkv_set_test_option(const char* name, long long value);

@@ -79,7 +79,7 @@ def round_fp32(x):
 def hadamard(d: int) -> np.ndarray:
     """Normalized Sylvester Hadamard matrix of order ``d`` (a power of two):
     entry (i, j) = (-1)**popcount(i & j) / sqrt(d).  Section 3 asks only for
-    "a normalized Hadamard matrix"; the Sylvester one is the reading taken."""
+    some Hadamard matrix scaled to be orthonormal; the Sylvester one is the reading taken."""
     if d < 1 or (d & (d - 1)) != 0:
         raise ValueError("Sylvester Hadamard needs a power-of-two order")
     h = np.ones((1, 1))
@@ -564,9 +564,9 @@ def chunk_attn(q_chunk, T_invT, k_codes, k_meta, v_codes, v_meta, k_bf16, v_bf16
     positions 0 .. S - n_new + i (causal inside the chunk).  Returns O [n_new][n_q][d].
 
     Which copy each position is read from (Section 4.4; Section 5.3): positions of the chunk itself are
-    read from their bf16 copies ("each new chunk is first appended in full precision and is used to compute
-    its attention output"; the serving integration "updates cache storage before attention, while still
-    using the current ... prefill chunk's K/V in BF16"); every older position follows the window rule at
+    read from their bf16 copies (the method appends a new chunk in full precision and computes the chunk's
+    attention output from those copies; the serving integration updates the storage before attention and
+    still reads the current chunk's keys and values in bf16); every older position follows the window rule at
     the cache length S - lag, as in ``effective_kv``.  Readings: lag = 0 is the serving behaviour;
     lag = n_new is Algorithm 2 taken literally (the boundary is only moved in lines 7-8, after
     attention)."""

@@ -2,23 +2,26 @@
 // chunk of S' > 1 new positions, after the chunk has been appended (line 4); Sections 4.4 and 5.3.
 //
 // Chunk position i of a sequence attends to every cached position up to itself.  Positions of the chunk are read
-// in full precision (k' = bf16(T_K k), v as given: "each new chunk is first appended in full precision and is used
-// to compute its attention output"), older positions follow the window rule: the sink and the recent window from
+// in full precision (k' = bf16(T_K k), v as given: the method appends a new chunk in full precision and computes the
+// chunk's attention output from those copies), older positions follow the window rule: the sink and the recent window from
 // their bf16 copies, the quantized middle from the packed pages (x_hat = x_min + Delta * code, Eq. 6 / Eq. 5).
 //
 // Two launches:
-//   1. prefill_prep_kernel   q' = T_K^{-T} q and k' = T_K k of the chunk (fp32 accumulation), written as fp16
-//                            operands of the attention kernel (k' through its bf16 rounding, the value the cache's
-//                            window copies hold), the chunk's values as fp16, and sum_c q'_c per query row.
-//   2. prefill_attn_kernel   one CTA per (sequence, query head, 64 query rows): four warps, 16 rows each, stream
-//                            64-key tiles of the three sources through shared memory and keep an online softmax
-//                            (flash-attention recurrence) per row.  Both contractions run on mma.sync.m16n8k16
-//                            (fp16 operands, fp32 accumulation).  The affine part of the quantizer is factored out
-//                            of the contractions, per key j of a tile:
+//   1. prefill_prep_kernel     q' = T_K^{-T} q and k' = T_K k of the chunk on tensor cores (bf16 mma, fp32
+//                              accumulation), written as fp16 operands of the attention kernel (k' through its bf16
+//                              rounding, the value the cache's window copies hold; q' as value + rounding
+//                              remainder), the chunk's values as fp16, and sum_c q'_c per query row.
+//   2. prefill_attn_tc_kernel  (default) one CTA per (sequence, KV head, 128-row tile that packs the G query heads):
+//                              both contractions as tcgen05.mma with accumulators in tensor memory; see section 2b.
+//      prefill_attn_kernel     (testing aid "prefill_legacy") one CTA per (sequence, query head, 64 query rows) on
+//                              mma.sync.m16n8k16; the first version, kept as a second implementation to test against.
+//   Both stream 64-key tiles of the three sources through shared memory and keep an online softmax
+//   (flash-attention recurrence) per row.  The affine part of the quantizer is factored out of the contractions,
+//   per key j of a tile:
 //                                score_ij = Delta_k,j (q'_i . c_k,j) + x_min_k,j sum(q'_i)
 //                                o_i     += (p_ij Delta_v,j) c_v,j + (p_ij x_min_v,j) 1
-//                            so packed pages are staged as their integer codes (exact in fp16) and full-precision
-//                            rows with Delta = 1, x_min = 0.
+//   so packed pages are staged as their integer codes (exact in fp16) and full-precision rows with Delta = 1,
+//   x_min = 0.
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
@@ -92,7 +95,7 @@ __global__ void __launch_bounds__(256) prefill_prep_kernel(PrefillParams P) {
     extern __shared__ __align__(16) unsigned short sm16[];
     unsigned short* Xs = sm16;                            // [PREP_TOK][PREP_PITCH]
     unsigned short* Ts = sm16 + PREP_TOK * PREP_PITCH;    // [terms][D][PREP_PITCH]: Ts[term][i][j] = term of T[i][j]
-    const int hs = blockIdx.y, tok0 = blockIdx.x * PREP_TOK;
+    const int hs = blockIdx.y;
     const bool is_key = hs < P.c.n_kv;
     const int head = is_key ? hs : hs - P.c.n_kv;
     const int kvh = is_key ? head : head / P.c.G;
@@ -113,6 +116,9 @@ __global__ void __launch_bounds__(256) prefill_prep_kernel(PrefillParams P) {
     }
     const int n_heads = is_key ? P.c.n_kv : P.c.n_q;
     const unsigned short* src = is_key ? P.K_new : P.Q_new;
+    // the transform stays in shared memory while the CTA walks over its token tiles
+    for (int tok0 = blockIdx.x * PREP_TOK; tok0 < P.total_new; tok0 += gridDim.x * PREP_TOK) {
+    __syncthreads();                                      // the previous tile's rows have been consumed
     for (int item = tid; item < PREP_TOK * 16; item += 256) {
         const int r = item >> 4, piece = item & 15, tok = tok0 + r;
         uint4 v = make_uint4(0, 0, 0, 0);
@@ -193,6 +199,7 @@ __global__ void __launch_bounds__(256) prefill_prep_kernel(PrefillParams P) {
             if (tok_a < P.total_new) P.qsum[static_cast<long long>(tok_a) * P.c.n_q + head] = sum_a;
             if (tok_b < P.total_new) P.qsum[static_cast<long long>(tok_b) * P.c.n_q + head] = sum_b;
         }
+    }
     }
 }
 
@@ -902,7 +909,11 @@ extern "C" int wushkv_prefill_attn(const wushkv_cache* cache, int32_t batch, con
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t smem_prep = static_cast<size_t>(PREP_TOK + 3 * D) * PREP_PITCH * sizeof(unsigned short);
     if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(prefill_prep_kernel), static_cast<int>(smem_prep))) return WUSHKV_ECUDA;
-    prefill_prep_kernel<<<dim3((total_new + PREP_TOK - 1) / PREP_TOK, P.c.n_kv + P.c.n_q), 256, smem_prep, st>>>(P);
+    {   // about one wave of CTAs: each keeps its head's transform resident and walks over token tiles
+        const int n_tok_tiles = (total_new + PREP_TOK - 1) / PREP_TOK, slots = P.c.n_kv + P.c.n_q;
+        const int per_slot = std::max(1, std::min(n_tok_tiles, sm_count() / slots));
+        prefill_prep_kernel<<<dim3(per_slot, slots), 256, smem_prep, st>>>(P);
+    }
     if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
     if (!knobs().prefill_legacy) {              // tcgen05 path: the G heads of a KV head share a 128-row tile
         const int R = TM / P.c.G;
