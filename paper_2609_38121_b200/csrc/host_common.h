@@ -53,6 +53,7 @@ struct Knobs {
     long long wait_limit = 0;       // > 0: poll limit of the device-side barrier waits (default: about a second)
     int drop_chunk_mma = 0;         // 1: the chunk append never commits its first tile's MMAs to the barrier
     int prefill_legacy = 0;         // 1: chunk attention on the mma.sync kernel instead of the tcgen05 one
+    int prefill_no_tma = 0;         // 1: the tcgen05 kernel stages the chunk's tiles with 16-byte copies instead of bulk tensor copies
 };
 Knobs& knobs();
 

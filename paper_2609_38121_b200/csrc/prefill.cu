@@ -22,10 +22,12 @@
 //                                o_i     += (p_ij Delta_v,j) c_v,j + (p_ij x_min_v,j) 1
 //   so packed pages are staged as their integer codes (exact in fp16) and full-precision rows with Delta = 1,
 //   x_min = 0.
+#include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstring>
 #include <type_traits>
 
 #include "host_common.h"
@@ -57,6 +59,7 @@ struct PrefillParams {
     __half* QP;                           // [2][total_new][n_q][D]  q' = T_K^{-T} q as fp16 value, then fp16 rounding remainder
     float* qsum;                          // [total_new][n_q]      sum over channels of q' (value + remainder)
     int tiles_per_seq;                    // ceil(max_new / BM)
+    int use_tma;                          // 1: the tcgen05 kernel stages the chunk's own tiles with bulk tensor copies
 };
 
 __device__ __forceinline__ unsigned smem_addr(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
@@ -494,7 +497,8 @@ constexpr int TC_OFF_META = TC_OFF_V + TC_K_BYTES;             // float4[TN]
 constexpr int TC_OFF_POS = TC_OFF_META + TN * 16;              // int[TN]
 constexpr int TC_OFF_RAW = TC_OFF_POS + TN * 4;                // one packed record
 constexpr int TC_OFF_BAR = TC_OFF_RAW + 8704;                  // mbarrier, tensor-memory slot
-constexpr int TC_SMEM = TC_OFF_BAR + 64;
+constexpr int TC_SMEM = TC_OFF_BAR + 64;                      // [0] MMA barrier, [8] tensor-copy barrier, [16] tensor-memory slot
+static_assert(TC_OFF_K % 1024 == 0 && TC_OFF_V % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 constexpr float REF_SLACK = 6.f;              // log2 headroom of the lazily raised softmax reference
 constexpr unsigned TC_TMEM_COLS = 256;        // O: columns 0..127, S: columns 128..191
 constexpr unsigned TC_IDESC_S = (1u << 4) | ((TN >> 3) << 17) | ((TM >> 4) << 24);                  // fp32 <- fp16 x fp16, both K-major
@@ -507,6 +511,12 @@ __device__ __forceinline__ unsigned long long tc_desc(unsigned addr, unsigned lb
     d |= static_cast<unsigned long long>((sbo >> 4) & 0x3FFFu) << 32;
     d |= 1ull << 46;
     return d;
+}
+// the same for a tile in the 128-byte-swizzled canonical layout (rows of 128 bytes, as a bulk tensor copy writes them)
+__device__ __forceinline__ unsigned long long tc_desc_sw128(unsigned addr, unsigned lbo, unsigned sbo) { return tc_desc(addr, lbo, sbo) | (2ull << 61); }
+__device__ __forceinline__ void tma_load_3d(unsigned dst, const CUtensorMap* map, int c0, int c1, int c2, unsigned bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(dst), "l"(reinterpret_cast<unsigned long long>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void tc_mma(unsigned tmem, unsigned long long adesc, unsigned long long bdesc, unsigned idesc, unsigned accumulate) {
     asm volatile(
@@ -548,7 +558,8 @@ __device__ __forceinline__ void cp16(unsigned dst, const void* src, unsigned byt
 }
 
 template <int BITS>
-__global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P) {
+__global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P, const __grid_constant__ CUtensorMap map_k,
+                                                                 const __grid_constant__ CUtensorMap map_v) {
     extern __shared__ __align__(1024) unsigned char sm_tc[];
     const CacheView& c = P.c;
     const int tid = threadIdx.x, warp = tid >> 5;
@@ -570,6 +581,8 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P)
     unsigned char* raw = sm_tc + TC_OFF_RAW;
     unsigned long long* mbar = reinterpret_cast<unsigned long long*>(sm_tc + TC_OFF_BAR);
     unsigned* tmem_slot = reinterpret_cast<unsigned*>(sm_tc + TC_OFF_BAR + 16);
+    const unsigned tbar = smem_addr(sm_tc + TC_OFF_BAR + 8);     // completion of the bulk tensor copies of a tile
+    unsigned tphase = 0;
 
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(TC_TMEM_COLS) : "memory");
@@ -577,6 +590,7 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P)
     }
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(mbar)) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(tbar) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     const int S0 = S - n_new;
@@ -630,16 +644,31 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P)
     // One staged tile: S = Q' K^T, softmax of this thread's row, O += P V.  PACKED: the keys carry affine factors
     // (codes of a packed page); MASKED: some key of the tile may be invisible to some row (padding, or a chunk
     // position beyond the row's own).  Full-precision, fully visible tiles (most of a long chunk) take the short form.
-    auto consume = [&](auto packed_tag, auto masked_tag) {
+    // `swz`: the key / value tile was written by bulk tensor copies (128-byte-swizzled rows, two 64-channel boxes each).
+    auto consume = [&](auto packed_tag, auto masked_tag, const bool swz) {
         constexpr bool PACKED = decltype(packed_tag)::value, MASKED = decltype(masked_tag)::value;
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        __syncthreads();
+        if (swz) {                                             // bounded wait for the tile's bulk copies
+            bool done = false;
+            for (int it = 0; it < wait_limit && !done; ++it) {
+                unsigned ok;
+                asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                             : "=r"(ok) : "r"(tbar), "r"(tphase), "r"(64u) : "memory");
+                done = ok != 0;
+            }
+            tphase ^= 1u;
+            if (!__syncthreads_and(done ? 1 : 0)) { failed = true; return; }
+        } else {
+            __syncthreads();
+        }
         if (tid == 0) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
-                const unsigned long long bdesc = tc_desc(smem_addr(sK) + ks * 256, 128, 2048);
+                // swizzled: channels 0-63 and 64-127 are two boxes of 8 KB; a k-step of 16 channels is 32 bytes inside the 128-byte row
+                const unsigned long long bdesc = swz ? tc_desc_sw128(smem_addr(sK) + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024)
+                                                     : tc_desc(smem_addr(sK) + ks * 256, 128, 2048);
                 tc_mma(tmem_base + 128, tc_desc(smem_addr(sQ) + ks * 256, 128, 2048), bdesc, TC_IDESC_S, ks > 0 ? 1u : 0u);
                 tc_mma(tmem_base + 128, tc_desc(smem_addr(sQ + TC_Q_BYTES) + ks * 256, 128, 2048), bdesc, TC_IDESC_S, 1u);
             }
@@ -702,8 +731,9 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P)
         if (tid == 0) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-            for (int ks = 0; ks < TN / 16; ++ks)
-                tc_mma(tmem_base, tc_desc(smem_addr(sK) + ks * 256, 128, 1024), tc_desc(smem_addr(sV) + ks * 256, 128, 1024), TC_IDESC_O,
+            for (int ks = 0; ks < TN / 16; ++ks)     // swizzled values: rows (keys) of 128 bytes, 8-key groups 1024 bytes apart, channel halves 8192 bytes apart
+                tc_mma(tmem_base, tc_desc(smem_addr(sK) + ks * 256, 128, 1024),
+                       swz ? tc_desc_sw128(smem_addr(sV) + ks * 2048, 8192, 1024) : tc_desc(smem_addr(sV) + ks * 256, 128, 1024), TC_IDESC_O,
                        (have_o || ks > 0) ? 1u : 0u);
             asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(mbar)) : "memory");
         }
@@ -744,7 +774,7 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P)
                 kpos[r] = idx < n_old_fp ? (idx < a_hi ? idx : c_lo + (idx - a_hi)) : -1;
             }
         }
-        if (base + TN > n_old_fp) consume(std::false_type{}, std::true_type{}); else consume(std::false_type{}, std::false_type{});
+        if (base + TN > n_old_fp) consume(std::false_type{}, std::true_type{}, false); else consume(std::false_type{}, std::false_type{}, false);
     }
 
     // ---- (2) quantized positions below the chunk: one packed page per tile, staged as integer codes
@@ -798,28 +828,46 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P)
                     kpos[r] = live ? pos : -1;
                 }
             }
-            consume(std::true_type{}, std::true_type{});
+            consume(std::true_type{}, std::true_type{}, false);
         }
     }
 
     // ---- (3) the chunk itself, causal: key tiles up to the tile's last position
     const int last_row = min(qt * R + R, n_new) - 1;
     for (int kt = 0; kt * TN <= last_row && !failed; ++kt) {
-        for (int item = tid; item < TN * 16; item += TM) {
-            const int r = item >> 4, piece = item & 15, row = kt * TN + r;
-            const bool in = row < n_new;
-            const long long off = (static_cast<long long>(first + (in ? row : 0)) * c.n_kv + h) * D + 8 * piece;
-            cp16(smem_addr(sK + (r >> 3) * 2048 + piece * 128 + (r & 7) * 16), P.KP + off, in ? 16u : 0u);
-            cp16(smem_addr(sV + piece * 1024 + (r >> 3) * 128 + (r & 7) * 16), P.VP + off, in ? 16u : 0u);
-            if (piece == 0) {
-                meta[r] = make_float4(1.f, 0.f, 1.f, 0.f);
-                kpos[r] = in ? S0 + row : -1;
+        if (P.use_tma) {
+            // four bulk tensor copies (keys / values x channel halves) of 64 rows x 128 bytes each; rows past the end of
+            // the chunk read zeros, rows of the next sequence are masked below
+            if (tid == 0) {
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(tbar), "r"(2u * TC_K_BYTES) : "memory");
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    tma_load_3d(smem_addr(sK) + hf * 8192, &map_k, 64 * hf, h, first + kt * TN, tbar);
+                    tma_load_3d(smem_addr(sV) + hf * 8192, &map_v, 64 * hf, h, first + kt * TN, tbar);
+                }
             }
+            if (tid < TN) {
+                const int row = kt * TN + tid;
+                meta[tid] = make_float4(1.f, 0.f, 1.f, 0.f);
+                kpos[tid] = row < n_new ? S0 + row : -1;
+            }
+        } else {
+            for (int item = tid; item < TN * 16; item += TM) {
+                const int r = item >> 4, piece = item & 15, row = kt * TN + r;
+                const bool in = row < n_new;
+                const long long off = (static_cast<long long>(first + (in ? row : 0)) * c.n_kv + h) * D + 8 * piece;
+                cp16(smem_addr(sK + (r >> 3) * 2048 + piece * 128 + (r & 7) * 16), P.KP + off, in ? 16u : 0u);
+                cp16(smem_addr(sV + piece * 1024 + (r >> 3) * 128 + (r & 7) * 16), P.VP + off, in ? 16u : 0u);
+                if (piece == 0) {
+                    meta[r] = make_float4(1.f, 0.f, 1.f, 0.f);
+                    kpos[r] = in ? S0 + row : -1;
+                }
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
         }
-        asm volatile("cp.async.commit_group;" ::: "memory");
         // no mask needed when every key of the tile exists and lies at or below every row's own position
-        if (kt * TN + TN <= n_new && S0 + kt * TN + TN - 1 <= tile_pos_lo) consume(std::false_type{}, std::false_type{});
-        else consume(std::false_type{}, std::true_type{});
+        if (kt * TN + TN <= n_new && S0 + kt * TN + TN - 1 <= tile_pos_lo) consume(std::false_type{}, std::false_type{}, P.use_tma != 0);
+        else consume(std::false_type{}, std::true_type{}, P.use_tma != 0);
     }
 
     // ---- output: o = (O + z) / l for the rows that carry a query
@@ -919,9 +967,36 @@ extern "C" int wushkv_prefill_attn(const wushkv_cache* cache, int32_t batch, con
         const int R = TM / P.c.G;
         P.tiles_per_seq = (max_new + R - 1) / R;
         const dim3 grid_tc(static_cast<unsigned>(batch) * P.tiles_per_seq, P.c.n_kv);
+        // tensor maps of the chunk's fp16 keys and values, [token][head][128 channels], boxes of 64 tokens x 64 channels
+        // written as 128-byte-swizzled rows; without the driver entry point the kernel stages with 16-byte copies
+        CUtensorMap map_k, map_v;
+        std::memset(&map_k, 0, sizeof(map_k));
+        std::memset(&map_v, 0, sizeof(map_v));
+        P.use_tma = 0;
+        {
+            typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                         const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                         CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+            static EncodeFn encode = [] {
+                void* fn = nullptr;
+                cudaDriverEntryPointQueryResult q;
+                if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) fn = nullptr;
+                return reinterpret_cast<EncodeFn>(fn);
+            }();
+            if (encode && !knobs().prefill_no_tma) {
+                const cuuint64_t gdim[3] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(P.c.n_kv), static_cast<cuuint64_t>(total_new)};
+                const cuuint64_t gstride[2] = {static_cast<cuuint64_t>(D) * 2, static_cast<cuuint64_t>(P.c.n_kv) * D * 2};
+                const cuuint32_t box[3] = {64, 1, TN}, estr[3] = {1, 1, 1};
+                const CUresult r1 = encode(&map_k, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, P.KP, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                const CUresult r2 = encode(&map_v, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, P.VP, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                P.use_tma = (r1 == CUDA_SUCCESS && r2 == CUDA_SUCCESS) ? 1 : 0;
+            }
+        }
         auto launch = [&](auto kernel) -> bool {
             if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(kernel), TC_SMEM)) return false;
-            kernel<<<grid_tc, TM, TC_SMEM, st>>>(P);
+            kernel<<<grid_tc, TM, TC_SMEM, st>>>(P, map_k, map_v);
             return true;
         };
         const bool ok = P.c.bits == 2 ? launch(prefill_attn_tc_kernel<2>) : P.c.bits == 3 ? launch(prefill_attn_tc_kernel<3>)

@@ -9,11 +9,14 @@ from tests.harness import CODE_MISMATCH_MAX, Layer
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(params=["tcgen05", "mma_sync"], autouse=True)
+@pytest.fixture(params=["tcgen05", "tcgen05_copies", "mma_sync"], autouse=True)
 def attention_path(request, test_option):
-    """Every case runs on both attention kernels: the tcgen05 one (default) and the mma.sync one."""
+    """Every case runs on the tcgen05 kernel with bulk tensor copies (default), on the same kernel with 16-byte copies,
+    and on the mma.sync kernel."""
     if request.param == "mma_sync":
         test_option("prefill_legacy", 1)
+    if request.param == "tcgen05_copies":
+        test_option("prefill_no_tma", 1)
     return request.param
 
 
