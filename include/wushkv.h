@@ -173,7 +173,8 @@ int wushkv_build_transforms_device(int32_t n_heads, int32_t d, const double* M, 
  * (keys only), quantized from the fp32 transform output, packed into its page, and its bf16
  * copy is written to the sink buffer (position < s_sink) and to the ring buffer (if it is among
  * the last ring_cap positions after this call).  Finally seq_len[b] += number of new tokens.
- *   slot (device): int32 [batch], cache slot of each sequence; slots must be distinct.
+ *   slot (device): int32 [batch], cache slot of each sequence; slots must be distinct (not checked: two sequences
+ *                  given the same slot write the same rows and no status bit is set).
  *   seq_len (device, in/out): int32 [batch].
  *   cu_new (device): int32 [batch+1] prefix sums, cu_new[0] = 0, cu_new[batch] = total_new.
  *   total_new, max_new (host): total and per-sequence maximum of new tokens.
