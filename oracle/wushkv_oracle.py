@@ -557,7 +557,7 @@ def decode_attn(q, T_invT, k_codes, k_meta, v_codes, v_meta, k_bf16, v_bf16, S,
 
 
 def chunk_attn(q_chunk, T_invT, k_codes, k_meta, v_codes, v_meta, k_bf16, v_bf16, S, n_new,
-               s_sink, s_keep, s_flush, sm_scale, lag=0):
+               s_sink, s_keep, s_flush, sm_scale, lag=0, rows=None):
     """Algorithm 2 lines 3 and 5 for a chunk of ``n_new`` > = 1 new positions of one sequence, AFTER they
     were appended (line 4): the cache holds S positions, the chunk is positions [S - n_new, S).
     q_chunk: [n_new][n_q][d] post-RoPE queries of the chunk (not compensated).  Chunk position i attends to
@@ -576,7 +576,7 @@ def chunk_attn(q_chunk, T_invT, k_codes, k_meta, v_codes, v_meta, k_bf16, v_bf16
     n_kv = T_invT.shape[0]
     G = n_q // n_kv
     S0 = S - n_new
-    out = np.empty((n_new, n_q, d))
+    out = np.full((n_new, n_q, d), np.nan)             # ``rows``: only these chunk rows are computed (the rest stay NaN)
     for h in range(n_kv):
         K_eff, V_eff = effective_kv(k_codes[:, h], k_meta[:, h], v_codes[:, h], v_meta[:, h],
                                     k_bf16[:, h], v_bf16[:, h], S, s_sink, s_keep, s_flush, lag)
@@ -585,7 +585,7 @@ def chunk_attn(q_chunk, T_invT, k_codes, k_meta, v_codes, v_meta, k_bf16, v_bf16
         for g in range(G):
             j = h * G + g
             qc = query_compensation(T_invT[h], q_chunk[:, j])            # [n_new][d]
-            for i in range(n_new):
+            for i in (range(n_new) if rows is None else rows):
                 n_vis = S0 + i + 1
                 out[i, j] = attention_one_query(qc[i], K_eff[:n_vis], V_eff[:n_vis], sm_scale)
     return out

@@ -240,7 +240,7 @@ class Layer:
             _, _, _, _, kb, vb = self.oracle[b].arrays()
             sel = np.arange(c) if rows is None else np.asarray([r for r in rows if r < c])
             ref = O.chunk_attn(qs[b], self.TinvT, kc, km, vc, vm, kb, vb, S, c, self.s_sink, self.s_keep, self.s_flush,
-                               1.0 / np.sqrt(128), lag=self.lag)
+                               1.0 / np.sqrt(128), lag=self.lag, rows=None if rows is None else [int(r) for r in sel])
             assert np.all(np.isfinite(outs[b])), "non-finite prefill output"
             for r in sel:
                 err = np.max(np.abs(outs[b][r] - ref[r])) / np.max(np.abs(ref[r]))

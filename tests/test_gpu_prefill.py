@@ -75,3 +75,16 @@ def test_quest_cache_under_a_chunk():
     L.append_step([400])
     assert L.check_prefill_parity([200]) <= 2e-3
     assert L.cache.status() == 0
+
+
+def test_long_chunk_over_a_long_quantized_cache(attention_path):
+    """A 2048-token chunk appended to a 32768-token cache (512 packed pages, then the window rows, then 32 causal
+    chunk tiles), sampled chunk rows against the oracle."""
+    if attention_path != "tcgen05":
+        pytest.skip("the long case runs on the default kernel only")
+    wl = _wl(8, 2, seed=97, theta=5e5)
+    L = Layer(wl, [32768 + 2048], 2, 4, 128, 1)
+    L.append_step([32768])
+    worst = L.check_prefill_parity([2048], rows=[0, 1, 17, 63, 64, 1023, 1024, 2000, 2047])
+    assert worst <= 2e-3
+    assert L.cache.status() == 0
