@@ -557,6 +557,59 @@ __device__ __forceinline__ void cp16(unsigned dst, const void* src, unsigned byt
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
 }
 
+// Eight consecutive channels 8 kc .. 8 kc + 7 of token r of a packed record as fp16 integers (keys and values), read
+// with 16-bit loads straight from the fragment-ordered layout (csrc/layout.cuh): a key half-word holds the two
+// channels 8 kc + 2 t, + 1 of fragment lane t; a value half-word holds the code fields of one channel for all channel
+// blocks.  Two codes c0, c1 become an fp16 pair by (c0 | c1 << 16 | 0x64006400) - (1024, 1024).
+template <int BITS>
+__device__ __forceinline__ void unpack_chunk8(const unsigned char* raw, int r, int kc, uint4& kout, uint4& vout) {
+    constexpr bool TWO = BITS != 4;                       // 2-bit fields (also the low plane of 3-bit records)
+    constexpr unsigned MASK = TWO ? 3u : 15u;
+    const int bi = r >> 4, rr = r & 15;
+    const __half2 bias = __halves2half2(__ushort_as_half(0x6400), __ushort_as_half(0x6400));
+    auto to_h2 = [&](unsigned c0, unsigned c1) {
+        const unsigned w = c0 | (c1 << 16) | 0x64006400u;
+        const __half2 h = __hsub2(*reinterpret_cast<const __half2*>(&w), bias);
+        return *reinterpret_cast<const unsigned*>(&h);
+    };
+    unsigned ko[4], vo[4];
+    {   // keys: token row -> (g, rs); chunk -> k-step s, channel half hh, byte pair bh
+        const int g = rr & 7, rs = rr >> 3, s4 = kc >> 2, hh = (kc >> 1) & 1, bh = kc & 1, j = rs + 2 * hh;
+        const int base = bi * code_block_bytes(BITS) + (TWO ? 0 : 512 * (s4 >> 1)) + 64 * g + 4 * j + 2 * bh;
+        const int sh = TWO ? 2 * s4 : 4 * (s4 & 1);
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const unsigned x = *reinterpret_cast<const unsigned short*>(raw + base + 16 * t);
+            unsigned c0 = (x >> sh) & MASK, c1 = (x >> (8 + sh)) & MASK;
+            if (BITS == 3) {
+                const unsigned y = *reinterpret_cast<const unsigned short*>(raw + k_hi_offset(3) + bi * 256 + 8 * (4 * g + t) + 4 * rs + 2 * bh);
+                c0 |= ((y >> (2 * s4 + hh)) & 1u) << 2;
+                c1 |= ((y >> (8 + 2 * s4 + hh)) & 1u) << 2;
+            }
+            ko[t] = to_h2(c0, c1);
+        }
+    }
+    {   // values: token -> (ps, t, hi); chunk -> channel block i, row half rsel; channel e of the chunk is fragment row g = e
+        const int ps = rr >> 3, tt = (rr & 7) >> 1, hi = rr & 1, i = kc >> 1, rsel = kc & 1;
+        const int base = v_codes_offset(BITS) + bi * code_block_bytes(BITS) + (TWO ? 4 * (2 * ps + rsel) : 512 * ps + 4 * (2 * rsel + (i >> 2))) + 16 * tt + 2 * hi;
+        const int sh = TWO ? 2 * i : 4 * (i & 3);
+        unsigned cv[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const unsigned x = *reinterpret_cast<const unsigned short*>(raw + base + 64 * e);
+            cv[e] = (x >> sh) & MASK;
+            if (BITS == 3) {
+                const unsigned y = *reinterpret_cast<const unsigned short*>(raw + v_hi_offset(3) + bi * 256 + 8 * (4 * e + tt) + 4 * ps + 2 * hi);
+                cv[e] |= ((y >> v1_bit(rsel, i)) & 1u) << 2;
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) vo[e] = to_h2(cv[2 * e], cv[2 * e + 1]);
+    }
+    kout = make_uint4(ko[0], ko[1], ko[2], ko[3]);
+    vout = make_uint4(vo[0], vo[1], vo[2], vo[3]);
+}
+
 template <int BITS>
 __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P, const __grid_constant__ CUtensorMap map_k,
                                                                  const __grid_constant__ CUtensorMap map_v) {
@@ -795,28 +848,12 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
                 const int r = tid & 63, ch0 = (tid >> 6) * 64;
                 const int pos = pg * PAGE_TOKENS + r;
                 const bool live = page_ok && pos >= q_lo && pos < q_hi;
-                constexpr unsigned MASK = (1u << (BITS == 3 ? 2 : BITS)) - 1u;
-                auto field_at = [&](int off, int bit, unsigned mask) { return (static_cast<unsigned>(raw[off + (bit >> 3)]) >> (bit & 7)) & mask; };
+                const uint4 zero4 = make_uint4(0, 0, 0, 0);
                 for (int kc = ch0 / 8; kc < ch0 / 8 + 8; ++kc) {
-                    float kf[8], vf[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        unsigned ck = 0, cv = 0;
-                        if (live) {
-                            int off, bit;
-                            k_code_location(BITS, r, 8 * kc + e, off, bit); ck = field_at(off, bit, MASK);
-                            v_code_location(BITS, r, 8 * kc + e, off, bit); cv = field_at(off, bit, MASK);
-                            if (BITS == 3) {
-                                k_hi_location(r, 8 * kc + e, off, bit); ck |= field_at(off, bit, 1u) << 2;
-                                v_hi_location(r, 8 * kc + e, off, bit); cv |= field_at(off, bit, 1u) << 2;
-                            }
-                        }
-                        kf[e] = static_cast<float>(ck); vf[e] = static_cast<float>(cv);
-                    }
-                    *reinterpret_cast<uint4*>(sK + (r >> 3) * 2048 + kc * 128 + (r & 7) * 16) =
-                        make_uint4(pack_half2(kf[0], kf[1]), pack_half2(kf[2], kf[3]), pack_half2(kf[4], kf[5]), pack_half2(kf[6], kf[7]));
-                    *reinterpret_cast<uint4*>(sV + kc * 1024 + (r >> 3) * 128 + (r & 7) * 16) =
-                        make_uint4(pack_half2(vf[0], vf[1]), pack_half2(vf[2], vf[3]), pack_half2(vf[4], vf[5]), pack_half2(vf[6], vf[7]));
+                    uint4 kq = zero4, vq = zero4;
+                    if (live) unpack_chunk8<BITS>(raw, r, kc, kq, vq);
+                    *reinterpret_cast<uint4*>(sK + (r >> 3) * 2048 + kc * 128 + (r & 7) * 16) = kq;
+                    *reinterpret_cast<uint4*>(sV + kc * 1024 + (r >> 3) * 128 + (r & 7) * 16) = vq;
                 }
                 if (ch0 == 0) {
                     float4 mt = make_float4(0.f, 0.f, 0.f, 0.f);
