@@ -48,6 +48,7 @@ struct AppendParams {
     int wait_limit;          // poll limit of the chunk kernel's MMA barrier wait (0: default, about two seconds)
     int drop_mma_commit;     // testing aid: the first tile's MMAs are never committed to their barrier
     Prologue pro;            // pro.rope != nullptr: K_new holds projected keys, normalised and rotated here (Algorithm 2 lines 1-2)
+    int use_tma;             // 1: the chunk kernel stages its key / value tiles with bulk tensor copies (128-byte-swizzled rows)
 };
 
 __device__ __forceinline__ void cswap_desc(unsigned& a, unsigned& b) {
@@ -439,6 +440,21 @@ __device__ __forceinline__ unsigned long long umma_smem_desc(unsigned smem_addr)
     d |= 1ull << 46;                                                             // descriptor version of sm_100
     return d;                                                                    // base offset 0, no swizzle
 }
+// The same for an operand written by a bulk tensor copy: rows of 128 bytes with the 128-byte swizzle, groups of 8 rows
+// 1024 bytes apart; a k-step of 16 channels advances the start address by 32 bytes inside the row.
+__device__ __forceinline__ unsigned long long umma_smem_desc_sw128(unsigned smem_addr) {
+    unsigned long long d = 0;
+    d |= static_cast<unsigned long long>((smem_addr >> 4) & 0x3FFFu);
+    d |= 1ull << 16;
+    d |= static_cast<unsigned long long>(1024u >> 4) << 32;
+    d |= 1ull << 46;
+    d |= 2ull << 61;
+    return d;
+}
+__device__ __forceinline__ void tma_tile_3d(unsigned dst, const CUtensorMap* map, int c0, int c1, int c2, unsigned bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(dst), "l"(reinterpret_cast<unsigned long long>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
+}
 // kind::f16 instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 128
 constexpr unsigned UMMA_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
@@ -578,7 +594,8 @@ __device__ __forceinline__ void quad_quantize(const float (&x)[32], ClipRule rul
 // KK_K / KK_V: list length of the quad quantizer for keys / values (8 or 16, >= the rule's rounds), 0 for
 // the warp-per-vector quantizer (any kappa), or -1 for the QuEST rule (Eq. 5, no order statistics).
 template <int BITS, int KK_K, int KK_V>
-__global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParams P) {
+__global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParams P, const __grid_constant__ CUtensorMap map_k,
+                                                                     const __grid_constant__ CUtensorMap map_v) {
     extern __shared__ __align__(1024) unsigned char tc_smem[];
     unsigned char* sB = tc_smem;
     unsigned char* sA = tc_smem + TC_SMEM_B;                         // A operand, later overwritten by the fp32 tile
@@ -596,8 +613,11 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr_u32(tmem_slot)), "r"(128u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    const unsigned tbar = smem_addr_u32(mbar) + 8;           // completion of a tile's bulk tensor copies
+    unsigned tphase = 0;
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr_u32(mbar)) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(tbar) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     {
@@ -627,7 +647,18 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
         // ---- A operand: key rows of this tile (zero rows past the end of the batch), and the value rows of the
         // tile into the part of the fp32 tile that is free until the MMAs are done; both as 16-byte
         // asynchronous copies, so that no register waits for them
-        {
+        if (P.use_tma) {
+            // four bulk tensor copies: keys and values x channel halves, 128 rows of 128 bytes each (rows past the end of
+            // the batch read zeros); the values go to the part of the fp32 tile that is free until the MMAs are done
+            if (tid == 0) {
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(tbar), "r"(KK_V != 0 ? 4u * 16384u : 2u * 16384u) : "memory");
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    tma_tile_3d(smem_addr_u32(sA) + hf * 16384, &map_k, 64 * hf, head, tok0, tbar);
+                    if (KK_V != 0) tma_tile_3d(smem_addr_u32(sV) + hf * 16384, &map_v, 64 * hf, head, tok0, tbar);
+                }
+            }
+        } else {
             const int r8 = lane & 7, cq = lane >> 3;
             for (int item = warp; item < 64; item += TC_THREADS / 32) {
                 const int rg = item >> 2, kc = (item & 3) * 4 + cq;
@@ -656,6 +687,22 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
             rows[tid] = ri;
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
+        if (P.use_tma) {                                      // bounded wait for the tile's bulk copies
+            bool arrived = false;
+            const int tma_wait_limit = P.wait_limit > 0 ? P.wait_limit : (1 << 22);
+            for (int it = 0; it < tma_wait_limit && !arrived; ++it) {
+                unsigned ok;
+                asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                             : "=r"(ok) : "r"(tbar), "r"(tphase), "r"(200u) : "memory");
+                arrived = ok != 0;
+            }
+            tphase ^= 1u;
+            if (!__syncthreads_and(arrived ? 1 : 0)) {
+                if (tid == 0) atomicOr(P.c.dev_status, WUSHKV_DEV_COPY_TIMEOUT);
+                failed = true;
+                break;
+            }
+        }
         if (P.pro.rope) {
             // Projected keys: normalise and rotate the staged tile in place (Algorithm 2 lines 1-2).  Four threads
             // share a row; thread q of a row owns channels 16q..16q+15 and their rotation partners 64+16q..64+16q+15,
@@ -724,10 +771,13 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
                 const unsigned accumulate = ks > 0 ? 1u : 0u;
+                // swizzled A: channels 0-63 and 64-127 are two boxes of 16 KB, a k-step is 32 bytes inside the 128-byte row
+                const unsigned long long a_ks = P.use_tma ? umma_smem_desc_sw128(smem_addr_u32(sA) + (ks >> 2) * 16384 + (ks & 3) * 32)
+                                                          : adesc + static_cast<unsigned long long>(ks * 2 * TC_LBO >> 4);
                 asm volatile(
                     "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
                     "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
-                    ::"r"(tmem_base), "l"(adesc + static_cast<unsigned long long>(ks * 2 * TC_LBO >> 4)),
+                    ::"r"(tmem_base), "l"(a_ks),
                       "l"(bdesc + static_cast<unsigned long long>(ks * 2 * TC_LBO >> 4)), "r"(UMMA_IDESC), "r"(accumulate),
                       "r"(0u), "r"(0u), "r"(0u), "r"(0u) : "memory");
             }
@@ -745,7 +795,12 @@ __global__ void __launch_bounds__(TC_THREADS, 2) append_chunk_kernel(AppendParam
             uint2 raw[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
-                raw[k] = live ? *reinterpret_cast<const uint2*>(vrow + 32 * k) : make_uint2(0u, 0u);
+                // channels 16k + 4qd .. +3: byte 32k + 8qd of the row; in a swizzled tile the row is 2 x 128 bytes (two
+                // boxes) and its 16-byte pieces are XOR-ed with the row index
+                const int o = 32 * k + 8 * qd;
+                const unsigned char* src = P.use_tma ? sV + (o >> 7) * 16384 + row * 128 + ((((o & 127) >> 4) ^ (row & 7)) << 4) + (o & 15)
+                                                     : vrow + 32 * k;
+                raw[k] = live ? *reinterpret_cast<const uint2*>(src) : make_uint2(0u, 0u);
                 x[4 * k + 0] = bf16_bits_to_float(raw[k].x & 0xffff); x[4 * k + 1] = bf16_bits_to_float(raw[k].x >> 16);
                 x[4 * k + 2] = bf16_bits_to_float(raw[k].y & 0xffff); x[4 * k + 3] = bf16_bits_to_float(raw[k].y >> 16);
             }
@@ -1075,6 +1130,7 @@ static int append_impl(const wushkv_cache* cache, int32_t batch, const int32_t* 
     const int rc = make_view(cache, P.c);
     if (rc != WUSHKV_OK) return rc;
     P.pro = Prologue{nullptr, 0, 0, nullptr, 0.f};
+    P.use_tma = 0;
     if (prologue && !make_prologue(prologue, prologue->k_norm_weight, P.pro)) return WUSHKV_EINVAL;
     if (batch <= 0 || !slot || !seq_len || !cu_new || total_new < 0 || max_new < 0 || max_new > total_new) return WUSHKV_EINVAL;
     if (total_new == 0) return WUSHKV_OK;
@@ -1121,9 +1177,14 @@ static int append_impl(const wushkv_cache* cache, int32_t batch, const int32_t* 
         const bool quest = P.rule_k.quest > 0.f;
         const int kk_k = quest ? -1 : need > 16 ? 0 : (P.rule_k.rounds <= 8 ? 8 : 16);
         const int kk_v = quest ? -1 : need > 16 ? 0 : (P.rule_v.rounds <= 8 ? 8 : 16);
+        // tensor maps of the new keys and values (not for projected keys, whose tile is rewritten in place in the plain layout)
+        CUtensorMap map_k, map_v;
+        const bool mk = make_row_tensor_map(map_k, true, K_new, P.c.n_kv, total_new, TC_TILE);
+        const bool mv = make_row_tensor_map(map_v, true, V_new, P.c.n_kv, total_new, TC_TILE);
+        P.use_tma = (mk && mv && !P.pro.rope && !knobs().append_no_tma) ? 1 : 0;
         auto launch = [&](auto kernel) -> bool {
             if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(kernel), TC_SMEM_TOTAL)) return false;
-            kernel<<<grid_tc, TC_THREADS, TC_SMEM_TOTAL, st>>>(P);
+            kernel<<<grid_tc, TC_THREADS, TC_SMEM_TOTAL, st>>>(P, map_k, map_v);
             return true;
         };
         bool ok;

@@ -1,6 +1,8 @@
 // Host-side argument validation shared by the entry points.
 #pragma once
 #include <cstdint>
+#include <cstring>
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include "../../include/wushkv.h"
@@ -54,6 +56,7 @@ struct Knobs {
     int drop_chunk_mma = 0;         // 1: the chunk append never commits its first tile's MMAs to the barrier
     int prefill_legacy = 0;         // 1: chunk attention on the mma.sync kernel instead of the tcgen05 one
     int prefill_no_tma = 0;         // 1: the tcgen05 kernel stages the chunk's tiles with 16-byte copies instead of bulk tensor copies
+    int append_no_tma = 0;          // 1: the chunk append stages its tiles with 16-byte copies instead of bulk tensor copies
 };
 Knobs& knobs();
 
@@ -74,6 +77,29 @@ inline bool opt_in_dynamic_smem(const void* fn, int bytes) {
         return true;
     }
     return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+}
+
+// Tensor map of a 16-bit row tensor [rows][n_heads][128 channels]: boxes of box_rows x 64 channels (128 bytes), written to
+// shared memory as 128-byte-swizzled rows.  Coordinates of a copy: (channel 0 or 64, head, first row).  False when the
+// driver entry point is missing or refuses (callers then stage with 16-byte copies).
+inline bool make_row_tensor_map(CUtensorMap& map, bool bf16, const void* base, int n_heads, long long rows, int box_rows) {
+    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                 const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeFn encode = [] {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) fn = nullptr;
+        return reinterpret_cast<EncodeFn>(fn);
+    }();
+    std::memset(&map, 0, sizeof(map));
+    if (!encode || rows <= 0 || n_heads <= 0) return false;
+    const cuuint64_t gdim[3] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(n_heads), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t gstride[2] = {static_cast<cuuint64_t>(D) * 2, static_cast<cuuint64_t>(n_heads) * D * 2};
+    const cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(box_rows)}, estr[3] = {1, 1, 1};
+    return encode(&map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), gdim, gstride, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 inline int sm_count() {

@@ -1007,30 +1007,9 @@ extern "C" int wushkv_prefill_attn(const wushkv_cache* cache, int32_t batch, con
         // tensor maps of the chunk's fp16 keys and values, [token][head][128 channels], boxes of 64 tokens x 64 channels
         // written as 128-byte-swizzled rows; without the driver entry point the kernel stages with 16-byte copies
         CUtensorMap map_k, map_v;
-        std::memset(&map_k, 0, sizeof(map_k));
-        std::memset(&map_v, 0, sizeof(map_v));
-        P.use_tma = 0;
-        {
-            typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                         const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                         CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-            static EncodeFn encode = [] {
-                void* fn = nullptr;
-                cudaDriverEntryPointQueryResult q;
-                if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) fn = nullptr;
-                return reinterpret_cast<EncodeFn>(fn);
-            }();
-            if (encode && !knobs().prefill_no_tma) {
-                const cuuint64_t gdim[3] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(P.c.n_kv), static_cast<cuuint64_t>(total_new)};
-                const cuuint64_t gstride[2] = {static_cast<cuuint64_t>(D) * 2, static_cast<cuuint64_t>(P.c.n_kv) * D * 2};
-                const cuuint32_t box[3] = {64, 1, TN}, estr[3] = {1, 1, 1};
-                const CUresult r1 = encode(&map_k, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, P.KP, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-                const CUresult r2 = encode(&map_v, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, P.VP, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-                P.use_tma = (r1 == CUDA_SUCCESS && r2 == CUDA_SUCCESS) ? 1 : 0;
-            }
-        }
+        const bool mk = make_row_tensor_map(map_k, false, P.KP, P.c.n_kv, total_new, TN);
+        const bool mv = make_row_tensor_map(map_v, false, P.VP, P.c.n_kv, total_new, TN);
+        P.use_tma = (mk && mv && !knobs().prefill_no_tma) ? 1 : 0;
         auto launch = [&](auto kernel) -> bool {
             if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(kernel), TC_SMEM)) return false;
             kernel<<<grid_tc, TM, TC_SMEM, st>>>(P, map_k, map_v);

@@ -95,13 +95,15 @@ def test_serving_window_sizes(s_sink, s_keep, s_flush):
     assert L.cache.status() == 0
 
 
-@pytest.mark.parametrize("path,bits", [("tensor", 2), ("cuda", 2), ("tensor", 3), ("cuda", 3)])
+@pytest.mark.parametrize("path,bits", [("tensor", 2), ("cuda", 2), ("tensor", 3), ("cuda", 3), ("tensor_copies", 2), ("tensor_copies", 4)])
 def test_prefill_chunk_paths(path, bits, test_option):
     """Config 4's structure scaled down: several sequences appended as one chunk each in ONE call
     (tile boundaries fall inside sequences and a ragged last tile), Qwen-shaped heads (G = 7, RMSNorm),
     through the tensor-core transform and through the CUDA-core chunk path; then one decode step."""
     if path == "cuda":
         test_option("append_path_cuda", 1)
+    if path == "tensor_copies":                     # the tensor-core path staged with 16-byte copies instead of bulk tensor copies
+        test_option("append_no_tma", 1)
     wl = _wl(28, 4, seed=41, batch=3, theta=1e6, rmsnorm=True)
     L = Layer(wl, [700, 131, 390], bits, 4, 128, 1)
     L.append_step([699, 130, 389])
