@@ -404,6 +404,8 @@ int wushkv_set_profile_events(void* start, void* stop);
  *   "prefill_legacy"    1: wushkv_prefill_attn runs its mma.sync kernel instead of the tcgen05 one.
  *   "prefill_no_tma"    1: the tcgen05 kernel stages the chunk's own tiles with 16-byte copies, not bulk tensor copies.
  *   "append_no_tma"     1: the same for the key / value tiles of the tensor-core chunk append.
+ *   "drop_prefill"      1: the tcgen05 chunk attention never commits the score MMAs of a CTA's first tile; 2: it announces
+ *                       but never issues one bulk copy of a CTA's first chunk tile (the bounded wait runs out either way).
  * Returns WUSHKV_EINVAL for an unknown name.
  */
 int wushkv_set_test_option(const char* name, long long value);

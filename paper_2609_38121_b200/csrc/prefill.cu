@@ -60,6 +60,9 @@ struct PrefillParams {
     float* qsum;                          // [total_new][n_q]      sum over channels of q' (value + remainder)
     int tiles_per_seq;                    // ceil(max_new / BM)
     int use_tma;                          // 1: the tcgen05 kernel stages the chunk's own tiles with bulk tensor copies
+    int wait_limit;                       // poll limit of the barrier waits (0: default, a second or more)
+    int drop;                             // testing aid: 1 the first tile's score MMAs are never committed, 2 the first bulk copy of a
+                                          // CTA's first chunk tile is announced but never issued (the wait then runs into its limit)
 };
 
 __device__ __forceinline__ unsigned smem_addr(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
@@ -678,7 +681,8 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
     unsigned phase = 0;
     bool failed = false, have_o = false;
     float m_ref = -INFINITY, l = 0.f, z = 0.f;
-    const int wait_limit = 1 << 24;                            // polls of at least ~60 ns each: a second or more
+    const int wait_limit = P.wait_limit > 0 ? P.wait_limit : (1 << 24);      // polls of at least ~60 ns each: a second or more
+    bool first_tile = true;
 
     auto wait_mma = [&]() -> bool {                             // bounded; the decision is uniform for the CTA
         bool done = false;
@@ -725,8 +729,10 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
                 tc_mma(tmem_base + 128, tc_desc(smem_addr(sQ) + ks * 256, 128, 2048), bdesc, TC_IDESC_S, ks > 0 ? 1u : 0u);
                 tc_mma(tmem_base + 128, tc_desc(smem_addr(sQ + TC_Q_BYTES) + ks * 256, 128, 2048), bdesc, TC_IDESC_S, 1u);
             }
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(mbar)) : "memory");
+            if (!(P.drop == 1 && first_tile))
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(mbar)) : "memory");
         }
+        first_tile = false;
         if (!wait_mma()) { failed = true; return; }
         // ---- this thread's row of scores (log2 domain after the scaling below)
         float s[TN];
@@ -879,7 +885,8 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(tbar), "r"(2u * TC_K_BYTES) : "memory");
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf) {
-                    tma_load_3d(smem_addr(sK) + hf * 8192, &map_k, 64 * hf, h, first + kt * TN, tbar);
+                    if (!(P.drop == 2 && kt == 0 && hf == 0))
+                        tma_load_3d(smem_addr(sK) + hf * 8192, &map_k, 64 * hf, h, first + kt * TN, tbar);
                     tma_load_3d(smem_addr(sV) + hf * 8192, &map_v, 64 * hf, h, first + kt * TN, tbar);
                 }
             }
@@ -986,6 +993,9 @@ extern "C" int wushkv_prefill_attn(const wushkv_cache* cache, int32_t batch, con
     unsigned char* ws = static_cast<unsigned char*>(workspace);
     P.batch = batch; P.total_new = total_new; P.slot = slot; P.seq_len = seq_len; P.cu_new = cu_new;
     P.K_new = K_new; P.V_new = V_new; P.Q_new = Q_new; P.O = O;
+    P.use_tma = 0;
+    P.wait_limit = static_cast<int>(std::min<long long>(std::max<long long>(knobs().wait_limit, 0), 1 << 30));
+    P.drop = knobs().drop_prefill;
     P.KP = reinterpret_cast<__half*>(ws + pl.off_kp);
     P.VP = reinterpret_cast<__half*>(ws + pl.off_vp);
     P.QP = reinterpret_cast<__half*>(ws + pl.off_qp);

@@ -54,6 +54,25 @@ def test_chunk_mma_that_is_never_committed_is_flagged(test_option):
     assert ok.check_decode_parity() <= 2e-3
 
 
+@pytest.mark.parametrize("what", [1, 2])
+def test_chunk_attention_wait_that_runs_out_is_flagged(what, test_option):
+    """The tcgen05 chunk attention with score MMAs that are never committed (1) or a bulk tensor copy that is announced
+    but never issued (2): the bounded wait runs out, the kernel flags it, frees its tensor memory and returns; the next
+    call is healthy."""
+    from paper_2609_38121_b200 import binding as B
+    wl = _wl(8, 2, seed=66)
+    L = Layer(wl, [300], 2, 4, 64, 1)
+    test_option("drop_prefill", what)
+    test_option("wait_limit", 2000)
+    outs, _ = L.prefill([300])
+    assert L.cache.status() & B.DEV_COPY_TIMEOUT
+    test_option("drop_prefill", 0)
+    test_option("wait_limit", 0)
+    ok = Layer(wl, [300], 2, 4, 64, 1)
+    assert ok.check_prefill_parity([300]) <= 2e-3
+    assert ok.cache.status() == 0
+
+
 def test_more_tokens_than_the_decode_hint_promised():
     """max_new == 1 selects the single-token kernel; a sequence that brings two tokens is flagged and left alone."""
     import torch
