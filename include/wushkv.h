@@ -283,8 +283,8 @@ int wushkv_accumulate_attention_hessians_device(int32_t n_kv, int32_t n_q, int32
  *     k_norm_weight    fp32 [n_kv][d] or NULL (ones);  q_norm_weight  fp32 [n_q][d] or NULL (ones)
  *     norm_eps         >= 0
  * wushkv_build_rope_table: cosines and sines in double precision, rounded to fp32 (device kernel; d must be 128).
- * wushkv_append_projected / wushkv_decode_attn_projected: arguments, results and errors of wushkv_append /
- * wushkv_decode_attn, with K_proj / Q_proj in place of K_new / Q and WUSHKV_EINVAL for a NULL or malformed
+ * wushkv_append_projected / wushkv_decode_attn_projected / wushkv_prefill_attn_projected: arguments, results and errors
+ * of wushkv_append / wushkv_decode_attn / wushkv_prefill_attn, with K_proj / Q_proj in place of K_new / Q and WUSHKV_EINVAL for a NULL or malformed
  * prologue.  Values are never normalised or rotated (V_new is passed as before).
  */
 typedef struct wushkv_prologue {
@@ -302,6 +302,13 @@ int wushkv_append_projected(const wushkv_cache* cache, int32_t batch, const int3
 int wushkv_decode_attn_projected(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
                                  int32_t max_seq_len, const uint16_t* Q_proj, const wushkv_prologue* prologue, float* O,
                                  void* workspace, size_t workspace_bytes, void* stream);
+/* wushkv_prefill_attn on projected keys and queries of the chunk (K_proj: what wushkv_append_projected received; the
+ * position of chunk token i of sequence b is seq_len[b] - n_new[b] + i); otherwise as wushkv_prefill_attn. */
+int wushkv_prefill_attn_projected(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
+                                  const int32_t* cu_new, int32_t total_new, int32_t max_new,
+                                  const uint16_t* K_proj, const uint16_t* V_new, const uint16_t* Q_proj,
+                                  const wushkv_prologue* prologue, float* O,
+                                  void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Read back the logical content of the packed cache (test / debugging aid): for positions

@@ -25,6 +25,7 @@ EXPORTS = (
     "wushkv_accumulate_gram_device", "wushkv_build_transforms_workspace_bytes", "wushkv_build_transforms_device",
     "wushkv_build_rope_table", "wushkv_append_projected", "wushkv_decode_attn_projected",
     "wushkv_attention_hessians_workspace_bytes", "wushkv_accumulate_attention_hessians_device",
+    "wushkv_prefill_attn_projected",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -118,6 +119,10 @@ def _load():
     lib.wushkv_decode_attn_projected.restype = C.c_int
     lib.wushkv_decode_attn_projected.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_void_p, C.c_void_p, C.c_int32,
                                                  C.c_void_p, C.POINTER(wushkv_prologue), C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.wushkv_prefill_attn_projected.restype = C.c_int
+    lib.wushkv_prefill_attn_projected.argtypes = [C.POINTER(wushkv_cache), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                                  C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(wushkv_prologue), C.c_void_p, C.c_void_p,
+                                                  C.c_size_t, C.c_void_p]
     lib.wushkv_attention_hessians_workspace_bytes.restype = C.c_size_t
     lib.wushkv_attention_hessians_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int64]
     lib.wushkv_accumulate_attention_hessians_device.restype = C.c_int
@@ -260,6 +265,14 @@ def decode_attn_projected(cache: wushkv_cache, batch, slot, seq_len, max_seq_len
     _check(lib.wushkv_decode_attn_projected(C.byref(cache), batch, _ptr(slot), _ptr(seq_len), max_seq_len, _ptr(Q_proj),
                                             C.byref(prologue), _ptr(O), _ptr(workspace), workspace_bytes,
                                             _stream_ptr(stream)), "wushkv_decode_attn_projected")
+
+
+def prefill_attn_projected(cache: wushkv_cache, batch, slot, seq_len, cu_new, total_new, max_new, K_proj, V_new, Q_proj,
+                           prologue: wushkv_prologue, O, workspace, workspace_bytes, stream=None):
+    """wushkv_prefill_attn_projected: wushkv_prefill_attn on projected keys and queries."""
+    _check(lib.wushkv_prefill_attn_projected(C.byref(cache), batch, _ptr(slot), _ptr(seq_len), _ptr(cu_new), total_new, max_new,
+                                             _ptr(K_proj), _ptr(V_new), _ptr(Q_proj), C.byref(prologue), _ptr(O), _ptr(workspace),
+                                             workspace_bytes, _stream_ptr(stream)), "wushkv_prefill_attn_projected")
 
 
 def decode_workspace_bytes(cache: wushkv_cache, batch: int, max_seq_len: int) -> int:

@@ -32,6 +32,7 @@
 
 #include "host_common.h"
 #include "layout.cuh"
+#include "prologue.cuh"
 
 namespace wushkv {
 
@@ -60,6 +61,8 @@ struct PrefillParams {
     float* qsum;                          // [total_new][n_q]      sum over channels of q' (value + remainder)
     int tiles_per_seq;                    // ceil(max_new / BM)
     int use_tma;                          // 1: the tcgen05 kernel stages the chunk's own tiles with bulk tensor copies
+    Prologue pro;                         // pro.rope != nullptr: K_new / Q_new are projected; Norm and RoPE are applied by the
+    const float* q_weight;                // transform kernel (pro.weight: key weights, q_weight: query weights)
     int wait_limit;                       // poll limit of the barrier waits (0: default, a second or more)
     int drop;                             // testing aid: 1 the first tile's score MMAs are never committed, 2 the first bulk copy of a
                                           // CTA's first chunk tile is announced but never issued (the wait then runs into its limit)
@@ -146,6 +149,47 @@ __global__ void __launch_bounds__(256) prefill_prep_kernel(PrefillParams P) {
         }
     }
     __syncthreads();
+    if (P.pro.rope) {
+        // Projected keys / queries: normalise and rotate the staged rows in place (Algorithm 2 lines 1-2, fp32, one rounding
+        // to bf16).  Two threads share a row: thread u of the pair owns channels 32u .. 32u+31 and their rotation
+        // partners 64+32u .. 64+32u+31.
+        const int row = tid >> 1, u = tid & 1, tok = tok0 + row;
+        unsigned short* xa = Xs + row * PREP_PITCH + 32 * u;
+        unsigned short* xb = xa + 64;
+        float a[32], b[32];
+#pragma unroll
+        for (int k = 0; k < 32; ++k) { a[k] = bf16_bits_to_float(xa[k]); b[k] = bf16_bits_to_float(xb[k]); }
+        if (P.pro.normalise) {
+            float ss = 0.f;
+#pragma unroll
+            for (int k = 0; k < 32; ++k) ss = fmaf(a[k], a[k], fmaf(b[k], b[k], ss));
+            ss += __shfl_xor_sync(FULLM, ss, 1);
+            const float rn = ss > 0.f ? 1.f / sqrtf(ss * (1.f / D) + P.pro.eps) : 0.f;
+            const float* w = is_key ? P.pro.weight : P.q_weight;
+#pragma unroll
+            for (int k = 0; k < 32; ++k) {
+                const float wa = w ? __ldg(w + static_cast<long long>(head) * D + 32 * u + k) : 1.f;
+                const float wb = w ? __ldg(w + static_cast<long long>(head) * D + 64 + 32 * u + k) : 1.f;
+                a[k] *= rn * wa; b[k] *= rn * wb;
+            }
+        }
+        int pos = 0;
+        if (tok < P.total_new) {                           // position of the token: its sequence's length before the chunk + its index
+            int lo = 0, hi = P.batch;
+            while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (__ldg(P.cu_new + mid) <= tok) lo = mid; else hi = mid; }
+            const int f0 = __ldg(P.cu_new + lo), n_b = __ldg(P.cu_new + lo + 1) - f0;
+            pos = __ldg(P.seq_len + lo) - n_b + (tok - f0);
+        }
+        pos = prologue_position(P.pro, pos, P.c.dev_status, u == 0 && tok < P.total_new);
+        const float2* tab = P.pro.rope + static_cast<long long>(pos) * (D / 2) + 32 * u;
+#pragma unroll
+        for (int k = 0; k < 32; ++k) {
+            const float2 cs = __ldg(tab + k);
+            xa[k] = float_to_bf16_bits(fmaf(a[k], cs.x, -b[k] * cs.y));
+            xb[k] = float_to_bf16_bits(fmaf(a[k], cs.y, b[k] * cs.x));
+        }
+        __syncthreads();
+    }
     // warp w: token rows 16w .. 16w+15, all 128 output channels
     float acc[16][4];
 #pragma unroll
@@ -975,13 +1019,19 @@ extern "C" size_t wushkv_prefill_workspace_bytes(const wushkv_cache* cache, int3
     return pl.total;
 }
 
-extern "C" int wushkv_prefill_attn(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
-                                   const int32_t* cu_new, int32_t total_new, int32_t max_new,
-                                   const uint16_t* K_new, const uint16_t* V_new, const uint16_t* Q_new, float* O,
-                                   void* workspace, size_t workspace_bytes, void* stream) {
+static int prefill_attn_impl(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
+                             const int32_t* cu_new, int32_t total_new, int32_t max_new,
+                             const uint16_t* K_new, const uint16_t* V_new, const uint16_t* Q_new, float* O,
+                             void* workspace, size_t workspace_bytes, void* stream, const wushkv_prologue* prologue) {
     PrefillParams P;
     const int rc = make_view(cache, P.c);
     if (rc != WUSHKV_OK) return rc;
+    P.pro = Prologue{nullptr, 0, 0, nullptr, 0.f};
+    P.q_weight = nullptr;
+    if (prologue) {
+        if (!make_prologue(prologue, prologue->k_norm_weight, P.pro) || (reinterpret_cast<uintptr_t>(prologue->q_norm_weight) & 15)) return WUSHKV_EINVAL;
+        P.q_weight = prologue->q_norm_weight;
+    }
     if (batch <= 0 || !slot || !seq_len || !cu_new || total_new < 0 || max_new < 0 || max_new > total_new) return WUSHKV_EINVAL;
     if (total_new == 0) return WUSHKV_OK;
     if (!K_new || !V_new || !Q_new || !O || !workspace || !aligned(K_new, 16) || !aligned(V_new, 16) || !aligned(Q_new, 16) ||
@@ -1043,4 +1093,22 @@ extern "C" int wushkv_prefill_attn(const wushkv_cache* cache, int32_t batch, con
         prefill_attn_kernel<4><<<grid, PF_THREADS, smem_attn, st>>>(P);
     }
     return cudaGetLastError() == cudaSuccess ? WUSHKV_OK : WUSHKV_ECUDA;
+}
+
+extern "C" int wushkv_prefill_attn(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
+                                   const int32_t* cu_new, int32_t total_new, int32_t max_new,
+                                   const uint16_t* K_new, const uint16_t* V_new, const uint16_t* Q_new, float* O,
+                                   void* workspace, size_t workspace_bytes, void* stream) {
+    return prefill_attn_impl(cache, batch, slot, seq_len, cu_new, total_new, max_new, K_new, V_new, Q_new, O, workspace, workspace_bytes,
+                             stream, nullptr);
+}
+
+extern "C" int wushkv_prefill_attn_projected(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
+                                             const int32_t* cu_new, int32_t total_new, int32_t max_new,
+                                             const uint16_t* K_proj, const uint16_t* V_new, const uint16_t* Q_proj,
+                                             const wushkv_prologue* prologue, float* O,
+                                             void* workspace, size_t workspace_bytes, void* stream) {
+    if (!prologue) return WUSHKV_EINVAL;
+    return prefill_attn_impl(cache, batch, slot, seq_len, cu_new, total_new, max_new, K_proj, V_new, Q_proj, O, workspace, workspace_bytes,
+                             stream, prologue);
 }

@@ -191,8 +191,9 @@ class Layer:
         assert np.all(np.isfinite(out)), "oracle read a position the GPU keeps no bf16 copy of"
         return out
 
-    def prefill(self, counts):
-        """Append counts[b] new tokens per sequence and compute their attention outputs with wushkv_prefill_attn.
+    def prefill(self, counts, queries=None):
+        """Append counts[b] new tokens per sequence and compute their attention outputs with wushkv_prefill_attn (with
+        wushkv_prefill_attn_projected if this layer has a prologue; ``queries`` then holds the projected queries).
         Returns (O_gpu list per sequence [n][n_q][128], queries list per sequence)."""
         torch, B = self.torch, self.B
         counts = [int(c) for c in counts]
@@ -202,15 +203,20 @@ class Layer:
         self.append_step(counts)
         total = sum(counts)
         dev = self.cache.device
-        qs = [self.wl.chunk_queries(b, np.arange(start[b], start[b] + c)) if c else np.zeros((0, self.wl.n_q, 128), np.float32)
-              for b, c in enumerate(counts)]
+        qs = queries if queries is not None else [
+            self.wl.chunk_queries(b, np.arange(start[b], start[b] + c)) if c else np.zeros((0, self.wl.n_q, 128), np.float32)
+            for b, c in enumerate(counts)]
         bits16 = lambda x: torch.from_numpy(W.f32_to_bf16_bits(x).view(np.int16)).to(dev)  # noqa: E731
         Kn, Vn, Qn = bits16(np.concatenate(Ks)), bits16(np.concatenate(Vs)), bits16(np.concatenate(qs))
         cu = torch.tensor(np.concatenate([[0], np.cumsum(counts)]).astype(np.int32), device=dev)
         Oo = torch.full((total, self.wl.n_q, 128), float("nan"), dtype=torch.float32, device=dev)
         nbytes = B.prefill_workspace_bytes(self.cache.desc, self.batch, total)
         ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
-        B.prefill_attn(self.cache.desc, self.batch, self.slot, self.seq_len, cu, total, max(counts), Kn, Vn, Qn, Oo, ws, nbytes)
+        if self.prologue is not None:
+            B.prefill_attn_projected(self.cache.desc, self.batch, self.slot, self.seq_len, cu, total, max(counts), Kn, Vn, Qn,
+                                     self.prologue.desc, Oo, ws, nbytes)
+        else:
+            B.prefill_attn(self.cache.desc, self.batch, self.slot, self.seq_len, cu, total, max(counts), Kn, Vn, Qn, Oo, ws, nbytes)
         torch.cuda.synchronize()
         out = Oo.cpu().numpy().astype(np.float64)
         offs = np.concatenate([[0], np.cumsum(counts)])

@@ -141,6 +141,34 @@ def test_projected_decode_matches_the_oracle(n_q, n_kv):
     assert fused.cache.status() == 0
 
 
+def test_projected_chunk_attention_matches_the_oracle():
+    """wushkv_prefill_attn_projected after wushkv_append_projected: a first chunk on the empty cache, then a second chunk
+    over it, against the oracle's chunk attention on oracle-prepared keys and queries (cache content: the GPU's codes)."""
+    wl = _wl(53, 2, 8, 2, 2)
+    lengths = [450, 290]
+    plain, fused, masks, qproj = _pair(wl, lengths, 2, True)
+    done = [0, 0]
+    for counts in ([300, 200], [150, 90]):
+        qs = [qproj[b][done[b]:done[b] + c] for b, c in enumerate(counts)]
+        outs, _ = fused.prefill(counts, queries=qs)
+        plain.append_step(counts)                               # the oracle's cache of the prepared keys (and the plain GPU cache)
+        for b, c in enumerate(counts):
+            S = done[b] + c
+            kc = np.zeros((S, wl.n_kv, 128), np.uint8); vc = np.zeros_like(kc)
+            km = np.zeros((S, wl.n_kv, 2)); vm = np.zeros_like(km)
+            for h in range(wl.n_kv):
+                cc, sc, zc = fused.gpu_codes(b, h, 0, n=S); kc[:, h], km[:, h, 0], km[:, h, 1] = cc, sc, zc
+                cc, sc, zc = fused.gpu_codes(b, h, 1, n=S); vc[:, h], vm[:, h, 0], vm[:, h, 1] = cc, sc, zc
+            _, _, _, _, kb, vb = plain.oracle[b].arrays()
+            qprep, _ = _prepared(qs[b], np.arange(done[b], S), wl.theta, wl.gain_q[None], True)
+            ref = O.chunk_attn(qprep, fused.TinvT, kc, km, vc, vm, kb, vb, S, c, 4, 64, 1, 1.0 / np.sqrt(128))
+            for r in range(c):
+                err = np.max(np.abs(outs[b][r] - ref[r])) / np.max(np.abs(ref[r]))
+                assert err <= DECODE_TOL, (b, r, err)
+            done[b] = S
+    assert fused.cache.status() == 0
+
+
 def test_position_beyond_the_rotary_table_is_flagged():
     from paper_2609_38121_b200 import binding as B
     wl = _wl(49, 1, 8, 2, 2)
