@@ -257,7 +257,7 @@ int wushkv_prefill_attn(const wushkv_cache* cache, int32_t batch, const int32_t*
  *   tau:              the logit temperature (sqrt(d) in the paper).
  *   H_K, H_V (device, in/out): float64 [n_kv][d][d], accumulated.
  *   workspace (device): >= wushkv_attention_hessians_workspace_bytes() bytes, 256-byte aligned, scratch.
- * d must be 128 and the group size n_q / n_kv at most 4 (WUSHKV_EINVAL otherwise).  Cost O(n_tokens^2) per head.
+ * d must be 128 and the group size n_q / n_kv at most 8 (WUSHKV_EINVAL otherwise).  Cost O(n_tokens^2) per head.
  * Arithmetic: fp32 with float64 accumulation of the sums over tokens.
  */
 size_t wushkv_attention_hessians_workspace_bytes(int32_t n_kv, int32_t n_q, int32_t d, int64_t n_tokens);

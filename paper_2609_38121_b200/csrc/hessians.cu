@@ -17,6 +17,7 @@
 //   reduce_kernel     H_K and H_V (float64, added to the caller's accumulators)
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cmath>
 
 #include "host_common.h"
@@ -116,9 +117,10 @@ __device__ __noinline__ void gamma_matvec(const float* gam, const float (&x)[4],
 }
 
 // One warp per (position, ordered pair): u_{gg'}(t) = Gamma_{gg'} o_{g',t} and alpha_{gg'}(s) = v_s . Gamma_{gg'} v_s.
-// grid (S, n_kv), G*G warps.
+// grid (S, n_kv), up to 16 warps that share the G*G ordered pairs.
 __global__ void project_kernel(HessParams P) {
-    const int t = blockIdx.x, h = blockIdx.y, w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t = blockIdx.x, h = blockIdx.y, lane = threadIdx.x & 31;
+    for (int w = threadIdx.x >> 5; w < P.G * P.G; w += blockDim.x >> 5) {
     const int g = w / P.G, gp = w % P.G;
     const float* gam = P.gamma + (static_cast<long long>(h * P.G + g) * P.G + gp) * D * D;
     float x[4], y[4];
@@ -144,6 +146,7 @@ __global__ void project_kernel(HessParams P) {
 #pragma unroll
     for (int off = 16; off >= 1; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
     if (lane == 0) P.alpha[(static_cast<long long>(t) * P.n_kv + h) * P.G * P.G + w] = dot;
+    }
 }
 
 // One CTA of 128 threads (one per channel) per (t, h): the pair sums W0, W1, W2 over s <= t, then A_{gg'}(t).
@@ -314,7 +317,7 @@ HessLayout hess_layout(int n_kv, int n_q, long long S) {
 using namespace wushkv;
 
 extern "C" size_t wushkv_attention_hessians_workspace_bytes(int32_t n_kv, int32_t n_q, int32_t d, int64_t n_tokens) {
-    if (d != D || n_kv <= 0 || n_q <= 0 || n_q % n_kv != 0 || n_q / n_kv > 4 || n_tokens <= 0) return 0;
+    if (d != D || n_kv <= 0 || n_q <= 0 || n_q % n_kv != 0 || n_q / n_kv > 8 || n_tokens <= 0) return 0;
     return hess_layout(n_kv, n_q, n_tokens).total;
 }
 
@@ -324,7 +327,7 @@ extern "C" int wushkv_accumulate_attention_hessians_device(int32_t n_kv, int32_t
                                                            void* workspace, size_t workspace_bytes, void* stream) {
     if (d != D || n_kv <= 0 || n_q <= 0 || n_q % n_kv != 0 || d_model <= 0 || n_tokens <= 0 || n_tokens > (1 << 24)) return WUSHKV_EINVAL;
     const int G = n_q / n_kv;
-    if (G > 4) return WUSHKV_EINVAL;          // pair accumulators are kept in registers: group sizes 1..4
+    if (G > 8) return WUSHKV_EINVAL;          // the library's group sizes: 1..8
     if (!K || !Q || !V || !W_O || !H_K || !H_V || !workspace || !(tau > 0.0)) return WUSHKV_EINVAL;
     if (!aligned(K, 16) || !aligned(Q, 16) || !aligned(V, 16) || !aligned(W_O, 16) || !aligned(workspace, 256)) return WUSHKV_EINVAL;
     const HessLayout L = hess_layout(n_kv, n_q, n_tokens);
@@ -342,13 +345,17 @@ extern "C" int wushkv_accumulate_attention_hessians_device(int32_t n_kv, int32_t
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     gamma_kernel<<<dim3(D / 16, D / 16, n_kv * G * G), dim3(16, 16), 0, st>>>(P);
     rows_kernel<<<dim3(P.S, n_kv), 32 * G, 0, st>>>(P);
-    project_kernel<<<dim3(P.S, n_kv), 32 * G * G, 0, st>>>(P);
+    project_kernel<<<dim3(P.S, n_kv), 32 * std::min(G * G, 16), 0, st>>>(P);
     const dim3 grid_t(P.S, n_kv), grid_r(D / 16, D / 16, n_kv);
     switch (G) {
         case 1: pairs_kernel<1><<<grid_t, 128, 0, st>>>(P); reduce_kernel<1><<<grid_r, dim3(16, 16), 0, st>>>(P); break;
         case 2: pairs_kernel<2><<<grid_t, 128, 0, st>>>(P); reduce_kernel<2><<<grid_r, dim3(16, 16), 0, st>>>(P); break;
         case 3: pairs_kernel<3><<<grid_t, 128, 0, st>>>(P); reduce_kernel<3><<<grid_r, dim3(16, 16), 0, st>>>(P); break;
-        default: pairs_kernel<4><<<grid_t, 128, 0, st>>>(P); reduce_kernel<4><<<grid_r, dim3(16, 16), 0, st>>>(P); break;
+        case 4: pairs_kernel<4><<<grid_t, 128, 0, st>>>(P); reduce_kernel<4><<<grid_r, dim3(16, 16), 0, st>>>(P); break;
+        case 5: pairs_kernel<5><<<grid_t, 128, 0, st>>>(P); reduce_kernel<5><<<grid_r, dim3(16, 16), 0, st>>>(P); break;
+        case 6: pairs_kernel<6><<<grid_t, 128, 0, st>>>(P); reduce_kernel<6><<<grid_r, dim3(16, 16), 0, st>>>(P); break;
+        case 7: pairs_kernel<7><<<grid_t, 128, 0, st>>>(P); reduce_kernel<7><<<grid_r, dim3(16, 16), 0, st>>>(P); break;
+        default: pairs_kernel<8><<<grid_t, 128, 0, st>>>(P); reduce_kernel<8><<<grid_r, dim3(16, 16), 0, st>>>(P); break;
     }
     return cudaGetLastError() == cudaSuccess ? WUSHKV_OK : WUSHKV_ECUDA;
 }

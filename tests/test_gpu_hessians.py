@@ -35,7 +35,7 @@ def _gpu(K, Q, V, WO, tau, calls=1):
     return HK.cpu().numpy(), HV.cpu().numpy()
 
 
-@pytest.mark.parametrize("n_q,n_kv,n_tok", [(8, 2, 70), (3, 1, 45), (2, 2, 33)])
+@pytest.mark.parametrize("n_q,n_kv,n_tok", [(8, 2, 70), (3, 1, 45), (2, 2, 33), (8, 1, 40), (7, 1, 36)])
 def test_attention_hessians_match_the_oracle(n_q, n_kv, n_tok):
     wl, K, Q, V, WO = _inputs(n_q, n_kv, n_tok, 32)
     tau = float(np.sqrt(128))
@@ -66,6 +66,7 @@ def test_hessians_accumulate_over_calls_and_feed_the_transform_builder():
     assert np.all(np.abs(T - To) <= ulp) and np.mean(T != To) < 2e-3
 
 
-def test_group_sizes_beyond_four_are_refused():
+def test_group_sizes_beyond_eight_are_refused():
     from paper_2609_38121_b200 import binding as B
-    assert B.lib.wushkv_attention_hessians_workspace_bytes(1, 8, 128, 64) == 0
+    assert B.lib.wushkv_attention_hessians_workspace_bytes(1, 9, 128, 64) == 0
+    assert B.lib.wushkv_attention_hessians_workspace_bytes(1, 8, 128, 64) > 0
