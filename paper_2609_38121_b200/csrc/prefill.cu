@@ -547,7 +547,7 @@ constexpr int TC_OFF_BAR = TC_OFF_RAW + 8704;                  // mbarrier, tens
 constexpr int TC_SMEM = TC_OFF_BAR + 64;                      // [0] MMA barrier, [8] tensor-copy barrier, [16] tensor-memory slot
 static_assert(TC_OFF_K % 1024 == 0 && TC_OFF_V % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 constexpr float REF_SLACK = 6.f;              // log2 headroom of the lazily raised softmax reference
-constexpr unsigned TC_TMEM_COLS = 256;        // O: columns 0..127, S: columns 128..191
+constexpr unsigned TC_TMEM_COLS = 256;        // O: columns 0..127, S: columns 128..191, P (fp16 pairs): columns 192..223
 constexpr unsigned TC_IDESC_S = (1u << 4) | ((TN >> 3) << 17) | ((TM >> 4) << 24);                  // fp32 <- fp16 x fp16, both K-major
 constexpr unsigned TC_IDESC_O = (1u << 4) | (1u << 16) | ((D >> 3) << 17) | ((TM >> 4) << 24);      // B (values) MN-major
 
@@ -570,6 +570,22 @@ __device__ __forceinline__ void tc_mma(unsigned tmem, unsigned long long adesc, 
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
         ::"r"(tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u) : "memory");
+}
+// the same with the A operand in tensor memory (lane = row, a 32-bit column = two consecutive K elements)
+__device__ __forceinline__ void tc_mma_ts(unsigned tmem_d, unsigned tmem_a, unsigned long long bdesc, unsigned idesc, unsigned accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void tc_st32u(unsigned taddr, const unsigned (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]),
+          "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]),
+          "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
 }
 __device__ __forceinline__ void tc_ld32(unsigned taddr, float (&v)[32]) {
     unsigned r[32];
@@ -814,8 +830,8 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
         l *= factor; z *= factor;
         m_ref = new_ref;
         const float ref = m_ref == -INFINITY ? 0.f : m_ref;
-        // ---- probabilities: (p Delta_v) as fp16 into the A-operand layout (over the key tile, which is consumed)
-        unsigned char* prow = sK + (tid >> 3) * 1024 + (tid & 7) * 16;
+        // ---- probabilities: (p Delta_v) as fp16 pairs into tensor memory (columns 192..223), the A operand of O += P V
+        unsigned pk[32];
 #pragma unroll
         for (int kc = 0; kc < TN / 8; ++kc) {
             float w[8];
@@ -826,8 +842,11 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
                 if (PACKED) { const float4 mt = meta[8 * kc + e]; z = fmaf(p, mt.w, z); w[e] = p * mt.z; }
                 else w[e] = p;
             }
-            *reinterpret_cast<uint4*>(prow + kc * 128) = make_uint4(pack_half2(w[0], w[1]), pack_half2(w[2], w[3]), pack_half2(w[4], w[5]), pack_half2(w[6], w[7]));
+#pragma unroll
+            for (int e = 0; e < 4; ++e) pk[4 * kc + e] = pack_half2(w[2 * e], w[2 * e + 1]);
         }
+        tc_st32u(tmem_row + 192, pk);
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncthreads();
@@ -835,9 +854,9 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
             for (int ks = 0; ks < TN / 16; ++ks)     // swizzled values: rows (keys) of 128 bytes, 8-key groups 1024 bytes apart, channel halves 8192 bytes apart
-                tc_mma(tmem_base, tc_desc(smem_addr(sK) + ks * 256, 128, 1024),
-                       swz ? tc_desc_sw128(smem_addr(sV) + ks * 2048, 8192, 1024) : tc_desc(smem_addr(sV) + ks * 256, 128, 1024), TC_IDESC_O,
-                       (have_o || ks > 0) ? 1u : 0u);
+                tc_mma_ts(tmem_base, tmem_base + 192 + 8 * ks,
+                          swz ? tc_desc_sw128(smem_addr(sV) + ks * 2048, 8192, 1024) : tc_desc(smem_addr(sV) + ks * 256, 128, 1024), TC_IDESC_O,
+                          (have_o || ks > 0) ? 1u : 0u);
             asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(mbar)) : "memory");
         }
         have_o = true;
