@@ -539,12 +539,13 @@ constexpr int TC_Q_BYTES = TM * D * 2;        // one fp16 query operand
 constexpr int TC_K_BYTES = TN * D * 2;        // key tile; reused for P (TM x TN fp16 is the same size)
 constexpr int TC_OFF_Q = 0;
 constexpr int TC_OFF_K = 2 * TC_Q_BYTES;
-constexpr int TC_OFF_V = TC_OFF_K + TC_K_BYTES;
-constexpr int TC_OFF_META = TC_OFF_V + TC_K_BYTES;             // float4[TN]
-constexpr int TC_OFF_POS = TC_OFF_META + TN * 16;              // int[TN]
-constexpr int TC_OFF_RAW = TC_OFF_POS + TN * 4;                // one packed record
-constexpr int TC_OFF_BAR = TC_OFF_RAW + 8704;                  // mbarrier, tensor-memory slot
-constexpr int TC_SMEM = TC_OFF_BAR + 64;                      // [0] MMA barrier, [8] tensor-copy barrier, [16] tensor-memory slot
+constexpr int TC_OFF_V = TC_OFF_K + TC_K_BYTES;                // two value tiles (the next one is staged while the current one is read)
+constexpr int TC_OFF_META = TC_OFF_V + 2 * TC_K_BYTES;         // uint2[TN]: four fp16 per key
+constexpr int TC_OFF_POS = TC_OFF_META + TN * 8;               // int[TN]
+constexpr int TC_OFF_BAR = TC_OFF_POS + TN * 4;                // barriers, tensor-memory slot
+constexpr int TC_SMEM = TC_OFF_BAR + 64;                      // [0] score-MMA barrier, [8] tensor-copy barrier, [16] tensor-memory slot, [24] P V barrier
+static_assert(2 * (TC_SMEM + 1024) <= 233472, "two CTAs per SM");
+static_assert(8704 <= TC_K_BYTES, "a packed record is staged in the idle value buffer");
 static_assert(TC_OFF_K % 1024 == 0 && TC_OFF_V % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 constexpr float REF_SLACK = 6.f;              // log2 headroom of the lazily raised softmax reference
 constexpr unsigned TC_TMEM_COLS = 256;        // O: columns 0..127, S: columns 128..191, P (fp16 pairs): columns 192..223
@@ -624,6 +625,8 @@ __device__ __forceinline__ void cp16(unsigned dst, const void* src, unsigned byt
 // with 16-bit loads straight from the fragment-ordered layout (csrc/layout.cuh): a key half-word holds the two
 // channels 8 kc + 2 t, + 1 of fragment lane t; a value half-word holds the code fields of one channel for all channel
 // blocks.  Two codes c0, c1 become an fp16 pair by (c0 | c1 << 16 | 0x64006400) - (1024, 1024).
+__device__ __forceinline__ float2 h2f2u(unsigned u) { return __half22float2(*reinterpret_cast<const __half2*>(&u)); }
+
 template <int BITS>
 __device__ __forceinline__ void unpack_chunk8(const unsigned char* raw, int r, int kc, uint4& kout, uint4& vout) {
     constexpr bool TWO = BITS != 4;                       // 2-bit fields (also the low plane of 3-bit records)
@@ -690,12 +693,16 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
         return;
     }
     unsigned char* sQ = sm_tc + TC_OFF_Q;
-    unsigned char* sK = sm_tc + TC_OFF_K;                       // key tile, then the probabilities of the same tile
-    unsigned char* sV = sm_tc + TC_OFF_V;
-    float4* meta = reinterpret_cast<float4*>(sm_tc + TC_OFF_META);
+    unsigned char* sK = sm_tc + TC_OFF_K;
+    unsigned char* sVb = sm_tc + TC_OFF_V;                      // two value buffers; `vb` selects the one of the tile being staged / consumed
+    int vb = 0;
+    uint2* meta = reinterpret_cast<uint2*>(sm_tc + TC_OFF_META);
     int* kpos = reinterpret_cast<int*>(sm_tc + TC_OFF_POS);
-    unsigned char* raw = sm_tc + TC_OFF_RAW;
     unsigned long long* mbar = reinterpret_cast<unsigned long long*>(sm_tc + TC_OFF_BAR);
+    const unsigned obar = smem_addr(sm_tc + TC_OFF_BAR + 24);    // completion of O += P V of a tile
+    unsigned ophase = 0;
+    bool pv_pending = false;
+    const uint2 META_PLAIN = make_uint2(0x00003C00u, 0x00003C00u);   // (1, 0, 1, 0) as fp16: a full-precision key
     unsigned* tmem_slot = reinterpret_cast<unsigned*>(sm_tc + TC_OFF_BAR + 16);
     const unsigned tbar = smem_addr(sm_tc + TC_OFF_BAR + 8);     // completion of the bulk tensor copies of a tile
     unsigned tphase = 0;
@@ -707,6 +714,7 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(mbar)) : "memory");
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(tbar) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(obar) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     const int S0 = S - n_new;
@@ -758,12 +766,32 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
         return true;
     };
 
+    // O += P V of the previous tile is only awaited where its operands or its accumulator are needed again
+    auto drain_pv = [&]() -> bool {
+        if (!pv_pending) return true;
+        bool done = false;
+        for (int it = 0; it < wait_limit && !done; ++it) {
+            unsigned ok;
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                         : "=r"(ok) : "r"(obar), "r"(ophase), "r"(64u) : "memory");
+            done = ok != 0;
+        }
+        pv_pending = false;
+        ophase ^= 1u;
+        if (!__syncthreads_and(done ? 1 : 0)) return false;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        return true;
+    };
+
     // One staged tile: S = Q' K^T, softmax of this thread's row, O += P V.  PACKED: the keys carry affine factors
     // (codes of a packed page); MASKED: some key of the tile may be invisible to some row (padding, or a chunk
     // position beyond the row's own).  Full-precision, fully visible tiles (most of a long chunk) take the short form.
     // `swz`: the key / value tile was written by bulk tensor copies (128-byte-swizzled rows, two 64-channel boxes each).
-    auto consume = [&](auto packed_tag, auto masked_tag, const bool swz) {
+    // `next_row` >= 0: the first token row of the next tile, to be fetched by bulk tensor copies as soon as the scores of
+    // this tile are done (the key buffer is free then, the other value buffer has been free since the previous tile).
+    auto consume = [&](auto packed_tag, auto masked_tag, const bool swz, const int next_row) {
         constexpr bool PACKED = decltype(packed_tag)::value, MASKED = decltype(masked_tag)::value;
+        unsigned char* sV = sVb + vb * TC_K_BYTES;
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         if (swz) {                                             // bounded wait for the tile's bulk copies
@@ -794,6 +822,14 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
         }
         first_tile = false;
         if (!wait_mma()) { failed = true; return; }
+        if (next_row >= 0 && tid == 0) {
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(tbar), "r"(2u * TC_K_BYTES) : "memory");
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                tma_load_3d(smem_addr(sK) + hf * 8192, &map_k, 64 * hf, h, next_row, tbar);
+                tma_load_3d(smem_addr(sVb + (vb ^ 1) * TC_K_BYTES) + hf * 8192, &map_v, 64 * hf, h, next_row, tbar);
+            }
+        }
         // ---- this thread's row of scores (log2 domain after the scaling below)
         float s[TN];
         {
@@ -807,7 +843,7 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
 #pragma unroll
         for (int j = 0; j < TN; ++j) {
             float v;
-            if (PACKED) { const float4 mt = meta[j]; v = k2 * fmaf(mt.y, my_qsum, mt.x * s[j]); }
+            if (PACKED) { const float2 mk = h2f2u(meta[j].x); v = k2 * fmaf(mk.y, my_qsum, mk.x * s[j]); }
             else v = k2 * s[j];
             if (MASKED) { const int kp = kpos[j]; if (kp < 0 || kp > my_pos) v = -INFINITY; }
             s[j] = v;
@@ -816,6 +852,7 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
         const bool raise = mx > m_ref + REF_SLACK;                 // also the first finite maximum (m_ref = -inf)
         const float new_ref = raise ? mx : m_ref;
         const float factor = raise ? fast_ex2(m_ref - new_ref) : 1.f;      // old reference -inf: factor 0, state is zero anyway
+        if (!drain_pv()) { failed = true; return; }                // the accumulator and the probability columns are free again
         if (__any_sync(FULLM, raise) && have_o) {                  // rescale this warp's accumulator rows in tensor memory
 #pragma unroll
             for (int q4 = 0; q4 < 4; ++q4) {
@@ -839,7 +876,7 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
             for (int e = 0; e < 8; ++e) {
                 const float p = fast_ex2(s[8 * kc + e] - ref);
                 l += p;
-                if (PACKED) { const float4 mt = meta[8 * kc + e]; z = fmaf(p, mt.w, z); w[e] = p * mt.z; }
+                if (PACKED) { const float2 mv = h2f2u(meta[8 * kc + e].y); z = fmaf(p, mv.y, z); w[e] = p * mv.x; }
                 else w[e] = p;
             }
 #pragma unroll
@@ -857,14 +894,16 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
                 tc_mma_ts(tmem_base, tmem_base + 192 + 8 * ks,
                           swz ? tc_desc_sw128(smem_addr(sV) + ks * 2048, 8192, 1024) : tc_desc(smem_addr(sV) + ks * 256, 128, 1024), TC_IDESC_O,
                           (have_o || ks > 0) ? 1u : 0u);
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(mbar)) : "memory");
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(obar) : "memory");
         }
         have_o = true;
-        if (!wait_mma()) { failed = true; return; }              // the tile buffers and the accumulator are free again
+        pv_pending = true;                                       // awaited by the next tile (or the epilogue)
+        vb ^= 1;
     };
 
     // ---- (1) full-precision old positions: sink [0, a_hi) and recent window [c_lo, S0), bf16 rows
     for (int base = 0; base < n_old_fp && !failed; base += TN) {
+        unsigned char* sV = sVb + vb * TC_K_BYTES;
         for (int item = tid; item < TN * 16; item += TM) {
             const int r = item >> 4, piece = item & 15, idx = base + r;
             uint4 kh = make_uint4(0, 0, 0, 0), vh = kh;
@@ -892,11 +931,11 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
             *reinterpret_cast<uint4*>(sK + (r >> 3) * 2048 + piece * 128 + (r & 7) * 16) = kh;
             *reinterpret_cast<uint4*>(sV + piece * 1024 + (r >> 3) * 128 + (r & 7) * 16) = vh;
             if (piece == 0) {
-                meta[r] = make_float4(1.f, 0.f, 1.f, 0.f);
+                meta[r] = META_PLAIN;
                 kpos[r] = idx < n_old_fp ? (idx < a_hi ? idx : c_lo + (idx - a_hi)) : -1;
             }
         }
-        if (base + TN > n_old_fp) consume(std::false_type{}, std::true_type{}, false); else consume(std::false_type{}, std::false_type{}, false);
+        if (base + TN > n_old_fp) consume(std::false_type{}, std::true_type{}, false, -1); else consume(std::false_type{}, std::false_type{}, false, -1);
     }
 
     // ---- (2) quantized positions below the chunk: one packed page per tile, staged as integer codes
@@ -908,6 +947,9 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
             if (pg < c.max_pages) page = __ldg(c.page_table + static_cast<long long>(sl) * c.max_pages + pg);
             const bool page_ok = page >= 0 && page < c.n_pages;
             if (!page_ok && tid == 0) atomicOr(c.dev_status, pg < c.max_pages ? WUSHKV_DEV_BAD_PAGE_ID : WUSHKV_DEV_PAGE_TABLE_FULL);
+            if (!drain_pv()) { failed = true; break; }          // the record is staged in the value buffer of the previous tile
+            unsigned char* sV = sVb + vb * TC_K_BYTES;
+            unsigned char* raw = sVb + (vb ^ 1) * TC_K_BYTES;
             if (page_ok) {
                 const uint4* src = reinterpret_cast<const uint4*>(c.pages + (static_cast<long long>(page) * c.n_kv + h) * REC);
                 for (int k = tid; k < REC / 16; k += TM) reinterpret_cast<uint4*>(raw)[k] = __ldg(src + k);
@@ -925,37 +967,34 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
                     *reinterpret_cast<uint4*>(sV + kc * 1024 + (r >> 3) * 128 + (r & 7) * 16) = vq;
                 }
                 if (ch0 == 0) {
-                    float4 mt = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (live) {
-                        const __half* mh = reinterpret_cast<const __half*>(raw + meta_location(BITS, r));
-                        mt = make_float4(__half2float(mh[0]), __half2float(mh[1]), __half2float(mh[2]), __half2float(mh[3]));
-                    }
-                    meta[r] = mt;
+                    meta[r] = live ? *reinterpret_cast<const uint2*>(raw + meta_location(BITS, r)) : make_uint2(0u, 0u);
                     kpos[r] = live ? pos : -1;
                 }
             }
-            consume(std::true_type{}, std::true_type{}, false);
+            consume(std::true_type{}, std::true_type{}, false, -1);
         }
     }
 
     // ---- (3) the chunk itself, causal: key tiles up to the tile's last position
     const int last_row = min(qt * R + R, n_new) - 1;
     for (int kt = 0; kt * TN <= last_row && !failed; ++kt) {
+        unsigned char* sV = sVb + vb * TC_K_BYTES;
         if (P.use_tma) {
             // four bulk tensor copies (keys / values x channel halves) of 64 rows x 128 bytes each; rows past the end of
-            // the chunk read zeros, rows of the next sequence are masked below
-            if (tid == 0) {
+            // the chunk read zeros, rows of the next sequence are masked below.  Only the first tile is fetched here: every
+            // later one was requested while its predecessor's softmax ran (see consume).
+            if (kt == 0 && tid == 0) {
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(tbar), "r"(2u * TC_K_BYTES) : "memory");
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf) {
-                    if (!(P.drop == 2 && kt == 0 && hf == 0))
-                        tma_load_3d(smem_addr(sK) + hf * 8192, &map_k, 64 * hf, h, first + kt * TN, tbar);
-                    tma_load_3d(smem_addr(sV) + hf * 8192, &map_v, 64 * hf, h, first + kt * TN, tbar);
+                    if (!(P.drop == 2 && hf == 0))
+                        tma_load_3d(smem_addr(sK) + hf * 8192, &map_k, 64 * hf, h, first, tbar);
+                    tma_load_3d(smem_addr(sV) + hf * 8192, &map_v, 64 * hf, h, first, tbar);
                 }
             }
             if (tid < TN) {
                 const int row = kt * TN + tid;
-                meta[tid] = make_float4(1.f, 0.f, 1.f, 0.f);
+                meta[tid] = META_PLAIN;
                 kpos[tid] = row < n_new ? S0 + row : -1;
             }
         } else {
@@ -966,18 +1005,20 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
                 cp16(smem_addr(sK + (r >> 3) * 2048 + piece * 128 + (r & 7) * 16), P.KP + off, in ? 16u : 0u);
                 cp16(smem_addr(sV + piece * 1024 + (r >> 3) * 128 + (r & 7) * 16), P.VP + off, in ? 16u : 0u);
                 if (piece == 0) {
-                    meta[r] = make_float4(1.f, 0.f, 1.f, 0.f);
+                    meta[r] = META_PLAIN;
                     kpos[r] = in ? S0 + row : -1;
                 }
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
         }
+        const int next_row = (P.use_tma && (kt + 1) * TN <= last_row) ? first + (kt + 1) * TN : -1;
         // no mask needed when every key of the tile exists and lies at or below every row's own position
-        if (kt * TN + TN <= n_new && S0 + kt * TN + TN - 1 <= tile_pos_lo) consume(std::false_type{}, std::false_type{}, P.use_tma != 0);
-        else consume(std::false_type{}, std::true_type{}, P.use_tma != 0);
+        if (kt * TN + TN <= n_new && S0 + kt * TN + TN - 1 <= tile_pos_lo) consume(std::false_type{}, std::false_type{}, P.use_tma != 0, next_row);
+        else consume(std::false_type{}, std::true_type{}, P.use_tma != 0, next_row);
     }
 
     // ---- output: o = (O + z) / l for the rows that carry a query
+    if (!failed && !drain_pv()) failed = true;
     if (!failed && have_o) {
         const float inv = l > 0.f ? 1.f / l : 0.f;
         float* dst = P.O + (static_cast<long long>(my_tok) * c.n_q + my_jq) * D;
