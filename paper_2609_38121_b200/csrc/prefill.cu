@@ -27,6 +27,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstdio>
 #include <cstring>
 #include <type_traits>
 
@@ -569,15 +570,15 @@ __device__ __forceinline__ void tma_load_3d(unsigned dst, const CUtensorMap* map
 __device__ __forceinline__ void tc_mma(unsigned tmem, unsigned long long adesc, unsigned long long bdesc, unsigned idesc, unsigned accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
-        ::"r"(tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u) : "memory");
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 // the same with the A operand in tensor memory (lane = row, a 32-bit column = two consecutive K elements)
 __device__ __forceinline__ void tc_mma_ts(unsigned tmem_d, unsigned tmem_a, unsigned long long bdesc, unsigned idesc, unsigned accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %6, %7, %8}, p;\n\t}"
-        ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u) : "memory");
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void tc_st32u(unsigned taddr, const unsigned (&v)[32]) {
     asm volatile(
@@ -1052,6 +1053,563 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TC_TMEM_COLS) : "memory");
 }
 
+// ------------------------------------------------------------------------------------------------
+// 2c. attention on tcgen05, warp-specialised (the default path)
+// ------------------------------------------------------------------------------------------------
+// One CTA of 384 threads per (sequence, KV head, PAIR of consecutive 128-row query tiles), one CTA per SM.  The
+// three roles run on their own and meet only at mbarriers, so that the tensor pipe computes the scores of the next key
+// tile while the softmax warps work on the current one:
+//   warps 0-3 / 4-7   softmax of query tile 0 / 1: thread r owns row r.  Per key tile: wait for S, read the row with
+//                     tcgen05.ld, scale / mask, raise the lazy reference (rescaling the accumulator rows in tensor memory
+//                     only then), write (p Delta_v) as fp16 pairs over the first 32 columns of the score buffer just read,
+//                     arrive on the tile's "probabilities ready" barrier.
+//   warps 8 / 11      issue the tcgen05.mma of query tile 0 / 1 (one lane each): S_t(g+1) = Q'_t K(g+1)^T as soon as the
+//                     key tile has landed, then O_t += P_t(g) V(g) once the probabilities are ready; commits release the
+//                     key / value stages (two arrivals each) and signal the softmax warps.
+//   warps 9-10        stage the key / value tiles into rings of three / two stages: bf16 window rows and packed pages (the
+//                     raw record arrives by a bulk copy one tile ahead and is unpacked into fp16 codes) are written by the
+//                     64 threads, the chunk's own tiles are bulk tensor copies issued by one lane of warp 9 (keys) and
+//                     one of warp 10 (values).
+// Tensor memory (512 columns): query tile t owns columns 256 t .. 256 t + 255: O (128), two score buffers (64 each).
+// Every wait is bounded; a wait that runs out raises a CTA-wide flag that ends all roles.
+constexpr int WS_THREADS = 384;
+constexpr int WS_KS = 3, WS_VS = 2;                              // ring depths of the key / value stages: a bulk tensor copy takes longer than
+                                                                 // one tile's MMAs, so a key tile is requested three tiles ahead of its scores
+constexpr int WS_RAW_BYTES = 8704;                               // largest packed record (4 bits)
+constexpr int WS_OFF_Q = 0;                                      // (tile 0 value, remainder), (tile 1 value, remainder)
+constexpr int WS_OFF_K = 4 * TC_Q_BYTES;
+constexpr int WS_OFF_V = WS_OFF_K + WS_KS * TC_K_BYTES;
+constexpr int WS_OFF_RAW = WS_OFF_V + WS_VS * TC_K_BYTES;        // two raw records
+constexpr int WS_OFF_META = WS_OFF_RAW + 2 * WS_RAW_BYTES;       // uint2[WS_VS][TN]: per-key factors of a packed tile
+constexpr int WS_OFF_LIVE = WS_OFF_META + WS_VS * TN * 8;        // uint2[WS_VS]: which keys of a packed tile exist
+enum { WB_KFULL = 0, WB_KEMPTY = WB_KFULL + WS_KS, WB_VFULL = WB_KEMPTY + WS_KS, WB_VEMPTY = WB_VFULL + WS_VS,
+       WB_S = WB_VEMPTY + WS_VS, WB_PV = WB_S + 4, WB_PREADY = WB_PV + 2, WB_RAW = WB_PREADY + 2, WB_Q = WB_RAW + 2,
+       WB_DRAIN, WB_COUNT };
+constexpr int WS_OFF_BAR = WS_OFF_LIVE + WS_VS * 8;
+constexpr int WS_OFF_MISC = WS_OFF_BAR + WB_COUNT * 8;           // [0] tensor-memory slot, [4] abort flag
+constexpr int WS_SMEM = WS_OFF_MISC + 16;
+static_assert(WS_SMEM <= 232448, "the dynamic shared memory of one CTA");
+static_assert(WS_OFF_K % 1024 == 0 && WS_OFF_V % 1024 == 0 && WS_OFF_RAW % 16 == 0 && WS_RAW_BYTES % 16 == 0, "alignment of the stages");
+static_assert(record_bytes(4) <= WS_RAW_BYTES && record_bytes(3) <= WS_RAW_BYTES, "raw record buffer");
+
+// Bounded wait for a phase of an mbarrier; gives up early when another role has raised the abort flag and raises it
+// itself when the limit runs out.
+__device__ __forceinline__ bool ws_wait(unsigned bar, unsigned parity, int limit, volatile int* abort_flag) {
+    for (int it = 0; it < limit; ++it) {
+        unsigned ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(bar), "r"(parity), "r"(64u) : "memory");
+        if (ok) return true;
+        if ((it & 7) == 7 && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void ws_arrive(unsigned bar) { asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory"); }
+__device__ __forceinline__ void ws_expect_tx(unsigned bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void ws_commit(unsigned bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void ws_bulk_g2s(unsigned dst, const void* src, unsigned bytes, unsigned bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// AND of a predicate over the 64 staging threads (named barrier 1): keeps their give-up decision uniform
+__device__ __forceinline__ bool ws_stagers_and(bool pred) {
+    unsigned r;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred p, 1, 64, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(r) : "r"(pred ? 1u : 0u) : "memory");
+    return r != 0;
+}
+
+#ifndef WUSHKV_WS_TIMING
+#define WUSHKV_WS_TIMING 0      // timing experiments only: per-role cycle counters of CTA (0, 0)
+#endif
+#if WUSHKV_WS_TIMING
+__device__ unsigned long long g_ws_t[32];
+#define WST_DECL long long wst_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long wst_last = clock64()
+#define WST(slot) do { const long long now = clock64(); wst_acc[slot] += now - wst_last; wst_last = now; } while (0)
+#define WST_FLUSH do { if (blockIdx.x == 0 && blockIdx.y == 0 && lane == 0 && (warp == 0 || warp == 8 || warp == 9)) \
+    for (int i = 0; i < 8; ++i) g_ws_t[(warp == 8 ? 16 : warp == 9 ? 24 : 0) + i] += wst_acc[i]; } while (0)
+#else
+#define WST_DECL
+#define WST(slot) do { } while (0)
+#define WST_FLUSH do { } while (0)
+#endif
+
+template <int BITS>
+__global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillParams P, const __grid_constant__ CUtensorMap map_k,
+                                                                        const __grid_constant__ CUtensorMap map_v) {
+    extern __shared__ __align__(1024) unsigned char sm_ws[];
+    constexpr int REC = record_bytes(BITS);
+    const CacheView& c = P.c;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int G = c.G, R = TM / G;                              // chunk positions per query tile
+    const int pairs = (P.tiles_per_seq + 1) >> 1;
+    const int pr = pairs - 1 - static_cast<int>(blockIdx.x % pairs);      // long pairs first
+    const int b = blockIdx.x / pairs, h = blockIdx.y;
+    const int first = __ldg(P.cu_new + b), n_new = __ldg(P.cu_new + b + 1) - first;
+    if (2 * pr * R >= n_new) return;
+    const int S = __ldg(P.seq_len + b), sl = __ldg(P.slot + b);
+    if (sl < 0 || sl >= c.n_slots || S < n_new) {
+        if (tid == 0) atomicOr(c.dev_status, WUSHKV_DEV_BAD_SLOT);
+        return;
+    }
+    const unsigned bar0 = smem_addr(sm_ws + WS_OFF_BAR);
+    auto bar = [&](int i) -> unsigned { return bar0 + 8u * static_cast<unsigned>(i); };
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(sm_ws + WS_OFF_MISC);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm_ws + WS_OFF_MISC + 4);
+    uint2* meta_all = reinterpret_cast<uint2*>(sm_ws + WS_OFF_META);
+    uint2* live_all = reinterpret_cast<uint2*>(sm_ws + WS_OFF_LIVE);
+
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+        for (int i = 0; i < WB_COUNT; ++i) {
+            // probabilities: the 128 softmax threads of a tile; stage releases: the two issuing warps; queries: warps 0-8
+            const unsigned count = (i == WB_PREADY || i == WB_PREADY + 1) ? 128u : i == WB_Q ? 288u
+                                 : (i >= WB_KEMPTY && i < WB_KEMPTY + WS_KS) || (i >= WB_VEMPTY && i < WB_VEMPTY + WS_VS) ? 2u : 1u;
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar(i)), "r"(count) : "memory");
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // ---- geometry of the key side (as in the one-tile kernel) and of the two query tiles
+    const int S0 = S - n_new;
+    const int nq = n_quantized(S - c.lag, c.s_sink, c.s_keep, c.s_flush);
+    const int q_lo = c.s_sink, q_hi = min(c.s_sink + nq, S0);
+    const int a_hi = min(c.s_sink, S0);
+    const int c_lo = max(q_hi, a_hi);
+    const int n_old_fp = a_hi + max(S0 - c_lo, 0);
+    const float k2 = c.sm_scale * LOG2E_F;
+    const int nA = (n_old_fp + TN - 1) / TN;                    // tiles of full-precision old positions
+    const int page_first = q_lo / PAGE_TOKENS;
+    const int nB = q_hi > q_lo ? (q_hi - 1) / PAGE_TOKENS - page_first + 1 : 0;      // packed pages
+    const int gC = nA + nB;                                     // first tile of the chunk itself
+    int n_rows[2], n_tiles[2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        const int qt = 2 * pr + t, np = min(R, n_new - qt * R);
+        n_rows[t] = max(np, 0) * G;
+        n_tiles[t] = np > 0 ? gC + (min(qt * R + R, n_new) - 1) / TN + 1 : 0;
+    }
+    const int NT = max(n_tiles[0], n_tiles[1]);
+    const int wait_limit = P.wait_limit > 0 ? P.wait_limit : (1 << 24);      // polls of at least ~60 ns each: a second or more
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const unsigned tmem_base = *tmem_slot;
+
+    // ---- the packed query tiles: row r of tile t = chunk position (2 pr + t) R + r / G (clamped), head h G + r % G
+    // (staged by the softmax and MMA warps; the staging warps start on the key side at once)
+    for (int item = tid; item < 4 * TM * 16 && warp < 9; item += 288) {
+        const int q = item >> 11, part = q & 1, r = (item >> 4) & (TM - 1), piece = item & 15;
+        const int t = n_rows[q >> 1] > 0 ? (q >> 1) : 0;        // a tile without rows aliases tile 0's (never used)
+        const int rr = min(r, n_rows[t] - 1);
+        const int tok = first + (2 * pr + t) * R + rr / G, jq = h * G + rr % G;
+        const __half* src = P.QP + static_cast<long long>(part) * P.total_new * c.n_q * D + (static_cast<long long>(tok) * c.n_q + jq) * D + 8 * piece;
+        cp16(smem_addr(sm_ws + WS_OFF_Q + q * TC_Q_BYTES + (r >> 3) * 2048 + piece * 128 + (r & 7) * 16), src, 16u);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    if (warp < 9) ws_arrive(bar(WB_Q));
+
+    if (warp < 8) {
+        // =============================== softmax of query tile t ==========================================
+        const int t = warp >> 2, wt = tid & 127;
+        if (n_tiles[t] > 0) {
+            const int qt = 2 * pr + t;
+            const int my_r = min(wt, n_rows[t] - 1);
+            const int my_tok = first + qt * R + my_r / G, my_jq = h * G + my_r % G;
+            const float my_qsum = __ldcg(P.qsum + static_cast<long long>(my_tok) * c.n_q + my_jq);
+            const int my_row = qt * R + my_r / G;               // this row sees the chunk's rows 0 .. my_row
+            const int tile_row_lo = qt * R;                     // smallest such limit of the tile
+            const unsigned tmem_row = tmem_base + (static_cast<unsigned>((warp & 3) * 32) << 16) + 256u * t;
+            float m_ref = -INFINITY, l = 0.f, z = 0.f;
+            bool ok = true;
+            WST_DECL;
+
+            // One key tile.  PACKED: the keys carry affine factors (a packed page; factors and the set of existing keys
+            // come with the value stage).  MASKED: key j exists if bit j of (live_lo, live_hi) is set and is visible to
+            // this row if crow0 + j <= my_row (crow0: chunk row of the tile's first key, very negative for old positions).
+            auto soft = [&](auto packed_tag, auto masked_tag, const int g, unsigned live_lo, unsigned live_hi, const int crow0) {
+                constexpr bool PACKED = decltype(packed_tag)::value, MASKED = decltype(masked_tag)::value;
+                const unsigned sbuf = tmem_row + 128u + 64u * (g & 1);
+                WST(0);
+                // one barrier per score buffer: its next phase (tile g + 2) cannot complete before this tile's probabilities are ready
+                if (!__all_sync(FULLM, ws_wait(bar(WB_S + 2 * t + (g & 1)), (g >> 1) & 1, wait_limit, abort_flag))) { ok = false; return; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint2* meta = meta_all + (g % WS_VS) * TN;
+                if (PACKED) {
+                    if (!__all_sync(FULLM, ws_wait(bar(WB_VFULL + g % WS_VS), (g / WS_VS) & 1, wait_limit, abort_flag))) { ok = false; return; }
+                    const uint2 lv = live_all[g % WS_VS];
+                    live_lo = lv.x; live_hi = lv.y;
+                }
+                WST(1);
+                float s[TN];
+                {
+                    float lo[32], hi[32];
+                    tc_ld32(sbuf, lo);
+                    tc_ld32(sbuf + 32, hi);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) { s[i] = lo[i]; s[32 + i] = hi[i]; }
+                }
+                WST(2);
+                float mx = -INFINITY;
+#pragma unroll
+                for (int j = 0; j < TN; ++j) {
+                    float v;
+                    if (PACKED) { const float2 mk = h2f2u(meta[j].x); v = k2 * fmaf(mk.y, my_qsum, mk.x * s[j]); }
+                    else v = k2 * s[j];
+                    if (MASKED) {
+                        const bool live = ((j < 32 ? live_lo >> j : live_hi >> (j - 32)) & 1u) != 0u;
+                        if (!live || crow0 + j > my_row) v = -INFINITY;
+                    }
+                    s[j] = v;
+                    mx = fmaxf(mx, v);
+                }
+                const bool raise = mx > m_ref + REF_SLACK;                 // also the first finite maximum (m_ref = -inf)
+                const float new_ref = raise ? mx : m_ref;
+                const float factor = raise ? fast_ex2(m_ref - new_ref) : 1.f;      // old reference -inf: factor 0, state is zero anyway
+                WST(3);
+                if (g > 0) {                                               // O += P V of the previous tile: long done as a rule
+                    if (!__all_sync(FULLM, ws_wait(bar(WB_PV + t), (g - 1) & 1, wait_limit, abort_flag))) { ok = false; return; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    if (__any_sync(FULLM, raise)) {                        // rescale this warp's accumulator rows in tensor memory
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            float o[32];
+                            tc_ld32(tmem_row + 32 * q4, o);
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) o[i] *= factor;
+                            tc_st32(tmem_row + 32 * q4, o);
+                        }
+                    }
+                }
+                WST(4);
+                l *= factor; z *= factor;
+                m_ref = new_ref;
+                const float ref = m_ref == -INFINITY ? 0.f : m_ref;
+                // ---- probabilities: (p Delta_v) as fp16 pairs over the first 32 columns of the score buffer just read
+                unsigned pk[32];
+#pragma unroll
+                for (int kc = 0; kc < TN / 8; ++kc) {
+                    float w[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const float p = fast_ex2(s[8 * kc + e] - ref);
+                        l += p;
+                        if (PACKED) { const float2 mv = h2f2u(meta[8 * kc + e].y); z = fmaf(p, mv.y, z); w[e] = p * mv.x; }
+                        else w[e] = p;
+                    }
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) pk[4 * kc + e] = pack_half2(w[2 * e], w[2 * e + 1]);
+                }
+                WST(5);
+                tc_st32u(sbuf, pk);
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                ws_arrive(bar(WB_PREADY + t));
+                WST(6);
+            };
+
+            constexpr int FAR_BELOW = -(1 << 30);
+            for (int g = 0; g < n_tiles[t] && ok; ++g) {
+                if (g < nA) {
+                    const int nv = min(TN, n_old_fp - g * TN);
+                    if (nv == TN) soft(std::false_type{}, std::false_type{}, g, 0u, 0u, FAR_BELOW);
+                    else soft(std::false_type{}, std::true_type{}, g, nv >= 32 ? 0xffffffffu : (1u << nv) - 1u,
+                              nv >= 32 ? (1u << (nv - 32)) - 1u : 0u, FAR_BELOW);
+                } else if (g < gC) {
+                    soft(std::true_type{}, std::true_type{}, g, 0u, 0u, FAR_BELOW);
+                } else {
+                    const int kt = g - gC, nv = min(TN, n_new - kt * TN);
+                    // no mask needed when every key of the tile exists and lies at or below every row's own position
+                    if (nv == TN && kt * TN + TN - 1 <= tile_row_lo) soft(std::false_type{}, std::false_type{}, g, 0u, 0u, 0);
+                    else soft(std::false_type{}, std::true_type{}, g, nv >= 32 ? 0xffffffffu : (1u << nv) - 1u,
+                              nv >= 32 ? (nv == TN ? 0xffffffffu : (1u << (nv - 32)) - 1u) : 0u, kt * TN);
+                }
+            }
+            WST_FLUSH;
+            // ---- output: o = (O + z) / l for the rows that carry a query
+            if (ok && !__all_sync(FULLM, ws_wait(bar(WB_PV + t), (n_tiles[t] - 1) & 1, wait_limit, abort_flag))) ok = false;
+            if (ok) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const float inv = l > 0.f ? 1.f / l : 0.f;
+                float* dst = P.O + (static_cast<long long>(my_tok) * c.n_q + my_jq) * D;
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    float o[32];
+                    tc_ld32(tmem_row + 32 * q4, o);
+                    if (wt < n_rows[t]) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4)
+                            *reinterpret_cast<float4*>(dst + 32 * q4 + i) = make_float4((o[i] + z) * inv, (o[i + 1] + z) * inv, (o[i + 2] + z) * inv, (o[i + 3] + z) * inv);
+                    }
+                }
+            }
+        }
+    }
+    else if (warp == 8 || warp == 11) {
+        // =============================== MMA issue for query tile t ========================================
+        // One issuing warp per query tile: with the 64-key tiles an MMA takes the pipe 48-64 cycles, about what one thread
+        // needs to issue it, so a single thread for both tiles left the pipe half idle.
+        const int t = warp == 8 ? 0 : 1;
+        const int mine = n_tiles[t];                            // tiles of this query tile; the other one may have more
+        WST_DECL;
+        bool ok = __all_sync(FULLM, ws_wait(bar(WB_Q), 0u, wait_limit, abort_flag));
+        WST(0);
+        // Descriptors are built once; their low bits hold the start address / 16, so a byte offset is added as offset / 16.
+        const unsigned long long q_desc = tc_desc(smem_addr(sm_ws + WS_OFF_Q + 2 * t * TC_Q_BYTES), 128, 2048);
+        const unsigned long long k_plain0 = tc_desc(smem_addr(sm_ws + WS_OFF_K), 128, 2048), k_swz0 = tc_desc_sw128(smem_addr(sm_ws + WS_OFF_K), 16, 1024);
+        const unsigned long long v_plain0 = tc_desc(smem_addr(sm_ws + WS_OFF_V), 128, 1024), v_swz0 = tc_desc_sw128(smem_addr(sm_ws + WS_OFF_V), 8192, 1024);
+        const unsigned acc_o = tmem_base + 256u * t;
+        auto scores_of = [&](auto swz_tag, const int g, const int st) {      // lane 0: the MMAs of S_t(g)
+            constexpr bool SWZ = decltype(swz_tag)::value;
+            const unsigned long long kb = (SWZ ? k_swz0 : k_plain0) + static_cast<unsigned>(st * (TC_K_BYTES >> 4));
+            const unsigned acc = acc_o + 128u + 64u * (g & 1);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                // swizzled: channels 0-63 and 64-127 are two boxes of 8 KB; a k-step of 16 channels is 32 bytes inside the 128-byte row
+                const unsigned long long bdesc = kb + static_cast<unsigned>((SWZ ? (ks >> 2) * 8192 + (ks & 3) * 32 : ks * 256) >> 4);
+                tc_mma(acc, q_desc + static_cast<unsigned>(ks * 256 >> 4), bdesc, TC_IDESC_S, ks > 0 ? 1u : 0u);
+                tc_mma(acc, q_desc + static_cast<unsigned>((TC_Q_BYTES + ks * 256) >> 4), bdesc, TC_IDESC_S, 1u);
+            }
+            if (!(P.drop == 1 && g == 0)) ws_commit(bar(WB_S + 2 * t + (g & 1)));
+            ws_commit(bar(WB_KEMPTY + st));
+        };
+        auto issue_scores = [&](const int g) -> bool {          // S_t(g) = Q'_t K(g)^T
+            const int st = g % WS_KS;
+#if WUSHKV_WS_TIMING
+            WST(6);
+            if (!__all_sync(FULLM, ws_wait(bar(WB_Q), 0u, wait_limit, abort_flag))) return false;      // measurement only: a wait that is satisfied
+            WST(7);
+#endif
+            if (!__all_sync(FULLM, ws_wait(bar(WB_KFULL + st), (g / WS_KS) & 1, wait_limit, abort_flag))) return false;
+            WST(1);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (lane == 0) {
+                if (g >= mine) ws_arrive(bar(WB_KEMPTY + st));  // a tile only the other query tile reads: just release the stage
+                else if (g >= gC && P.use_tma) scores_of(std::true_type{}, g, st);
+                else scores_of(std::false_type{}, g, st);
+            }
+            __syncwarp();
+            WST(2);
+            return true;
+        };
+        auto issue_values = [&](const int g) -> bool {          // O_t += P_t(g) V(g)
+            const int st = g % WS_VS;
+            if (!__all_sync(FULLM, ws_wait(bar(WB_VFULL + st), (g / WS_VS) & 1, wait_limit, abort_flag))) return false;
+            WST(3);
+            if (g >= mine) {
+                if (lane == 0) ws_arrive(bar(WB_VEMPTY + st));
+                __syncwarp();
+                return true;
+            }
+            const bool swz = g >= gC && P.use_tma;
+            // swizzled values: rows (keys) of 128 bytes, 8-key groups 1024 bytes apart, channel halves 8192 bytes apart: 16 keys = 2048 bytes
+            const unsigned long long vb = (swz ? v_swz0 : v_plain0) + static_cast<unsigned>(st * (TC_K_BYTES >> 4));
+            const unsigned vstep = swz ? (2048u >> 4) : (256u >> 4);
+            if (!__all_sync(FULLM, ws_wait(bar(WB_PREADY + t), g & 1, wait_limit, abort_flag))) return false;
+            WST(4);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (lane == 0) {
+                const unsigned prob = acc_o + 128u + 64u * (g & 1);
+#pragma unroll
+                for (int ks = 0; ks < TN / 16; ++ks)
+                    tc_mma_ts(acc_o, prob + 8 * ks, vb + ks * vstep, TC_IDESC_O, (g > 0 || ks > 0) ? 1u : 0u);
+                ws_commit(bar(WB_PV + t));
+                ws_commit(bar(WB_VEMPTY + st));
+            }
+            __syncwarp();
+            WST(5);
+            return true;
+        };
+        if (ok) ok = issue_scores(0);
+        for (int g = 0; g < NT && ok; ++g) {
+            if (g + 1 < NT) ok = issue_scores(g + 1);
+            if (ok) ok = issue_values(g);
+        }
+        WST_FLUSH;
+    } else {
+        // =============================== staging of key / value tiles =====================================
+        const int ptid = tid - 288;
+        const int n_staged = P.use_tma ? gC : NT;               // tiles written by the 64 threads
+        int raw_uses[2] = {0, 0};                               // records fetched so far into each raw buffer
+        auto page_of = [&](const int gb) -> int {               // page id of packed tile gb, -1 if it cannot be read
+            const int pg = page_first + gb;
+            int page = -1;
+            if (pg < c.max_pages) page = __ldg(c.page_table + static_cast<long long>(sl) * c.max_pages + pg);
+            return (page >= 0 && page < c.n_pages) ? page : -1;
+        };
+        auto fetch_record = [&](const int gb) {                 // one thread: bulk copy of the record into raw buffer gb & 1
+            const int page = page_of(gb);
+            if (page < 0) {
+                atomicOr(c.dev_status, page_first + gb < c.max_pages ? WUSHKV_DEV_BAD_PAGE_ID : WUSHKV_DEV_PAGE_TABLE_FULL);
+                return;
+            }
+            ws_expect_tx(bar(WB_RAW + (gb & 1)), REC);
+            ws_bulk_g2s(smem_addr(sm_ws + WS_OFF_RAW + (gb & 1) * WS_RAW_BYTES), c.pages + (static_cast<long long>(page) * c.n_kv + h) * REC, REC,
+                        bar(WB_RAW + (gb & 1)));
+        };
+        if (nB > 0 && ptid == 0) fetch_record(0);
+        bool ok = true;
+        for (int g = 0; g < n_staged && ok; ++g) {
+            const int ks = g % WS_KS, vs = g % WS_VS;
+            unsigned char* sK = sm_ws + WS_OFF_K + ks * TC_K_BYTES;
+            unsigned char* sV = sm_ws + WS_OFF_V + vs * TC_K_BYTES;
+            bool mine = true;
+            if (g >= WS_KS) mine = ws_wait(bar(WB_KEMPTY + ks), ((g / WS_KS) - 1) & 1, wait_limit, abort_flag);
+            if (mine && g >= WS_VS) mine = ws_wait(bar(WB_VEMPTY + vs), ((g / WS_VS) - 1) & 1, wait_limit, abort_flag);
+            mine = __all_sync(FULLM, mine);                     // warp-uniform from here on
+            if (g < nA) {
+                // ---- full-precision old positions: sink [0, a_hi) and recent window [c_lo, S0), bf16 rows
+                for (int item = ptid; item < TN * 16 && mine; item += 64) {
+                    const int r = item & (TN - 1), piece = item >> 6, idx = g * TN + r;
+                    uint4 kh = make_uint4(0, 0, 0, 0), vh = kh;
+                    if (idx < n_old_fp) {
+                        const long long plane = (static_cast<long long>(sl) * c.n_kv + h) * 2;
+                        const unsigned short *ksrc, *vsrc;
+                        if (idx < a_hi) {
+                            ksrc = c.sink_kv + (plane * c.s_sink + idx) * D;
+                            vsrc = c.sink_kv + ((plane + 1) * c.s_sink + idx) * D;
+                        } else {
+                            const int p = c_lo + (idx - a_hi);
+                            ksrc = c.ring_kv + (plane * c.ring_cap + p % c.ring_cap) * D;
+                            vsrc = c.ring_kv + ((plane + 1) * c.ring_cap + p % c.ring_cap) * D;
+                        }
+                        const uint4 kb16 = *reinterpret_cast<const uint4*>(ksrc + 8 * piece), vb16 = *reinterpret_cast<const uint4*>(vsrc + 8 * piece);
+                        const unsigned kw[4] = {kb16.x, kb16.y, kb16.z, kb16.w}, vw[4] = {vb16.x, vb16.y, vb16.z, vb16.w};
+                        unsigned ko[4], vo[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            ko[e] = pack_half2(bf16_bits_to_float(kw[e] & 0xffff), bf16_bits_to_float(kw[e] >> 16));
+                            vo[e] = pack_half2(bf16_bits_to_float(vw[e] & 0xffff), bf16_bits_to_float(vw[e] >> 16));
+                        }
+                        kh = make_uint4(ko[0], ko[1], ko[2], ko[3]); vh = make_uint4(vo[0], vo[1], vo[2], vo[3]);
+                    }
+                    *reinterpret_cast<uint4*>(sK + (r >> 3) * 2048 + piece * 128 + (r & 7) * 16) = kh;
+                    *reinterpret_cast<uint4*>(sV + piece * 1024 + (r >> 3) * 128 + (r & 7) * 16) = vh;
+                }
+            } else if (g < gC) {
+                // ---- a packed page: the record was requested one tile ahead; unpack it into integer codes (exact in fp16)
+                const int gb = g - nA, rb = gb & 1;
+                // the other raw buffer was last read for tile gb - 1, which every staging thread has left
+                if (gb + 1 < nB && ptid == 0) fetch_record(gb + 1);
+                const bool page_ok = page_of(gb) >= 0;
+                if (page_ok && mine) mine = __all_sync(FULLM, ws_wait(bar(WB_RAW + rb), raw_uses[rb] & 1, wait_limit, abort_flag));
+                if (page_ok) ++raw_uses[rb];
+                const unsigned char* raw = sm_ws + WS_OFF_RAW + rb * WS_RAW_BYTES;
+                const uint4 zero4 = make_uint4(0, 0, 0, 0);
+                for (int item = ptid; item < TN * 16 && mine; item += 64) {
+                    const int r = item & (TN - 1), kc = item >> 6;
+                    const int pos = (page_first + gb) * PAGE_TOKENS + r;
+                    const bool live = page_ok && pos >= q_lo && pos < q_hi;
+                    uint4 kq = zero4, vq = zero4;
+                    if (live) unpack_chunk8<BITS>(raw, r, kc, kq, vq);
+                    *reinterpret_cast<uint4*>(sK + (r >> 3) * 2048 + kc * 128 + (r & 7) * 16) = kq;
+                    *reinterpret_cast<uint4*>(sV + kc * 1024 + (r >> 3) * 128 + (r & 7) * 16) = vq;
+                }
+                if (mine) {                                     // factors and existence of key ptid (the 64 threads = the 64 keys)
+                    const int pos = (page_first + gb) * PAGE_TOKENS + ptid;
+                    const bool live = page_ok && pos >= q_lo && pos < q_hi;
+                    meta_all[vs * TN + ptid] = live ? *reinterpret_cast<const uint2*>(raw + meta_location(BITS, ptid)) : make_uint2(0u, 0u);
+                    const unsigned word = __ballot_sync(FULLM, live);
+                    if (lane == 0) reinterpret_cast<unsigned*>(live_all + vs)[ptid >> 5] = word;
+                }
+            } else {
+                // ---- the chunk's own rows by 16-byte loads (testing aid; bulk tensor copies otherwise)
+                const int kt = g - gC;
+                for (int item = ptid; item < TN * 16 && mine; item += 64) {
+                    const int r = item & (TN - 1), piece = item >> 6, row = kt * TN + r;
+                    uint4 kh = make_uint4(0, 0, 0, 0), vh = kh;
+                    if (row < n_new) {
+                        const long long off = (static_cast<long long>(first + row) * c.n_kv + h) * D + 8 * piece;
+                        kh = *reinterpret_cast<const uint4*>(P.KP + off);
+                        vh = *reinterpret_cast<const uint4*>(P.VP + off);
+                    }
+                    *reinterpret_cast<uint4*>(sK + (r >> 3) * 2048 + piece * 128 + (r & 7) * 16) = kh;
+                    *reinterpret_cast<uint4*>(sV + piece * 1024 + (r >> 3) * 128 + (r & 7) * 16) = vh;
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            ok = ws_stagers_and(mine);
+            if (ok && ptid == 0) { ws_arrive(bar(WB_KFULL + ks)); ws_arrive(bar(WB_VFULL + vs)); }
+        }
+        // ---- the chunk itself: four bulk tensor copies per tile (keys / values x channel halves) of 64 rows x 128 bytes;
+        // rows past the end of the chunk read zeros or the next sequence's rows, both masked by the softmax warps.
+        // Warp 9 requests the key tiles, warp 10 the value tiles: the two rings advance on their own.
+        int armed[3] = {-1, -1, -1};                            // last tile whose copies this warp announced on each stage
+        if (P.use_tma && warp <= 10) {
+            const bool keys = warp == 9;
+            const int depth = keys ? WS_KS : WS_VS, full0 = keys ? WB_KFULL : WB_VFULL, empty0 = keys ? WB_KEMPTY : WB_VEMPTY;
+            const CUtensorMap* map = keys ? &map_k : &map_v;
+            unsigned char* ring = sm_ws + (keys ? WS_OFF_K : WS_OFF_V);
+            WST_DECL;
+            for (int g = gC; g < NT && ok; ++g) {
+                const int st = g % depth, row = first + (g - gC) * TN;
+                WST(0);
+                if (g >= depth && !__all_sync(FULLM, ws_wait(bar(empty0 + st), ((g / depth) - 1) & 1, wait_limit, abort_flag))) { ok = false; break; }
+                WST(1);
+                if (lane == 0) {
+                    ws_expect_tx(bar(full0 + st), TC_K_BYTES);
+#pragma unroll
+                    for (int hf = 0; hf < 2; ++hf)
+                        if (!(P.drop == 2 && keys && g == gC && hf == 0))
+                            tma_load_3d(smem_addr(ring + st * TC_K_BYTES) + hf * 8192, map, 64 * hf, h, row, bar(full0 + st));
+                }
+#pragma unroll
+                for (int i = 0; i < 3; ++i) if (i == st) armed[i] = g;
+#if WUSHKV_WS_TIMING
+                WST(2);
+                ws_wait(bar(full0 + st), (g / depth) & 1, wait_limit, abort_flag);      // measurement only: how long the copies take
+                WST(3);
+#endif
+            }
+            WST_FLUSH;
+            // after a failure elsewhere: give the copies this warp announced a bounded time to land, so that none is
+            // still writing shared memory when the CTA ends
+            if (lane == 0 && *abort_flag) {
+#pragma unroll
+                for (int i = 0; i < 3; ++i)
+                    if (i < depth && armed[i] >= 0)
+                        for (int it = 0; it < 512 && !ws_wait(bar(full0 + i), (armed[i] / depth) & 1, 1, abort_flag); ++it) __nanosleep(2000);
+            }
+        }
+        if (tid == 288 && *abort_flag) {                        // the same for the record copies
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+                if (nB > i) for (int it = 0; it < 64 && !ws_wait(bar(WB_RAW + i), raw_uses[i] & 1, 1, abort_flag); ++it) __nanosleep(2000);
+        }
+    }
+
+    // ---- all roles are done (or gave up)
+    __syncthreads();
+    if (*abort_flag) {
+        // commit whatever was issued once more and give it a bounded time, so that no MMA is still writing tensor
+        // memory when it is released below
+        if (tid == 256) {
+            atomicOr(c.dev_status, WUSHKV_DEV_COPY_TIMEOUT);
+            ws_commit(bar(WB_DRAIN));
+            for (int it = 0; it < 512; ++it) {
+                unsigned done;
+                asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                             : "=r"(done) : "r"(bar(WB_DRAIN)), "r"(0u), "r"(2000u) : "memory");
+                if (done) break;
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+}
+
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
 struct PrefillPlan { size_t off_kp, off_vp, off_qp, off_qsum, total; };
@@ -1130,6 +1688,32 @@ static int prefill_attn_impl(const wushkv_cache* cache, int32_t batch, const int
         const bool mk = make_row_tensor_map(map_k, false, P.KP, P.c.n_kv, total_new, TN);
         const bool mv = make_row_tensor_map(map_v, false, P.VP, P.c.n_kv, total_new, TN);
         P.use_tma = (mk && mv && !knobs().prefill_no_tma) ? 1 : 0;
+        if (!knobs().prefill_one_tile) {        // warp-specialised kernel: a pair of query tiles per CTA
+            const dim3 grid_ws(static_cast<unsigned>(batch) * ((P.tiles_per_seq + 1) / 2), P.c.n_kv);
+            auto launch_ws = [&](auto kernel) -> bool {
+                if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(kernel), WS_SMEM)) return false;
+                kernel<<<grid_ws, WS_THREADS, WS_SMEM, st>>>(P, map_k, map_v);
+                return true;
+            };
+            const bool ok = P.c.bits == 2 ? launch_ws(prefill_attn_ws_kernel<2>) : P.c.bits == 3 ? launch_ws(prefill_attn_ws_kernel<3>)
+                                                                                             : launch_ws(prefill_attn_ws_kernel<4>);
+            if (!ok) return WUSHKV_ECUDA;
+#if WUSHKV_WS_TIMING
+            {
+                cudaDeviceSynchronize();
+                unsigned long long t[32];
+                cudaMemcpyFromSymbol(t, g_ws_t, sizeof(t));
+                std::fprintf(stderr, "ws timing softmax:");
+                for (int i = 0; i < 8; ++i) std::fprintf(stderr, " %llu", t[i]);
+                std::fprintf(stderr, "\nws timing mma:");
+                for (int i = 16; i < 32; ++i) std::fprintf(stderr, " %llu", t[i]);
+                std::fprintf(stderr, "\n");
+                std::memset(t, 0, sizeof(t));
+                cudaMemcpyToSymbol(g_ws_t, t, sizeof(t));
+            }
+#endif
+            return cudaGetLastError() == cudaSuccess ? WUSHKV_OK : WUSHKV_ECUDA;
+        }
         auto launch = [&](auto kernel) -> bool {
             if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(kernel), TC_SMEM)) return false;
             kernel<<<grid_tc, TM, TC_SMEM, st>>>(P, map_k, map_v);

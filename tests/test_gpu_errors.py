@@ -54,14 +54,16 @@ def test_chunk_mma_that_is_never_committed_is_flagged(test_option):
     assert ok.check_decode_parity() <= 2e-3
 
 
+@pytest.mark.parametrize("one_tile", [0, 1])
 @pytest.mark.parametrize("what", [1, 2])
-def test_chunk_attention_wait_that_runs_out_is_flagged(what, test_option):
+def test_chunk_attention_wait_that_runs_out_is_flagged(what, one_tile, test_option):
     """The tcgen05 chunk attention with score MMAs that are never committed (1) or a bulk tensor copy that is announced
     but never issued (2): the bounded wait runs out, the kernel flags it, frees its tensor memory and returns; the next
     call is healthy."""
     from paper_2609_38121_b200 import binding as B
     wl = _wl(8, 2, seed=66)
     L = Layer(wl, [300], 2, 4, 64, 1)
+    test_option("prefill_one_tile", one_tile)
     test_option("drop_prefill", what)
     test_option("wait_limit", 2000)
     outs, _ = L.prefill([300])

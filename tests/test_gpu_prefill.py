@@ -9,13 +9,15 @@ from tests.harness import CODE_MISMATCH_MAX, Layer
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(params=["tcgen05", "tcgen05_copies", "mma_sync"], autouse=True)
+@pytest.fixture(params=["tcgen05", "tcgen05_copies", "tcgen05_one_tile", "tcgen05_one_tile_copies", "mma_sync"], autouse=True)
 def attention_path(request, test_option):
-    """Every case runs on the tcgen05 kernel with bulk tensor copies (default), on the same kernel with 16-byte copies,
-    and on the mma.sync kernel."""
+    """Every case runs on the warp-specialised tcgen05 kernel with bulk tensor copies (default), on the same kernel with
+    plain 16-byte loads, on the one-tile-per-CTA tcgen05 kernel (both ways) and on the mma.sync kernel."""
     if request.param == "mma_sync":
         test_option("prefill_legacy", 1)
-    if request.param == "tcgen05_copies":
+    if request.param.startswith("tcgen05_one_tile"):
+        test_option("prefill_one_tile", 1)
+    if request.param.endswith("copies"):
         test_option("prefill_no_tma", 1)
     return request.param
 
