@@ -1083,7 +1083,7 @@ constexpr int WS_OFF_RAW = WS_OFF_V + WS_VS * TC_K_BYTES;        // two raw reco
 constexpr int WS_OFF_META = WS_OFF_RAW + 2 * WS_RAW_BYTES;       // uint2[WS_VS][TN]: per-key factors of a packed tile
 constexpr int WS_OFF_LIVE = WS_OFF_META + WS_VS * TN * 8;        // uint2[WS_VS]: which keys of a packed tile exist
 enum { WB_KFULL = 0, WB_KEMPTY = WB_KFULL + WS_KS, WB_VFULL = WB_KEMPTY + WS_KS, WB_VEMPTY = WB_VFULL + WS_VS,
-       WB_S = WB_VEMPTY + WS_VS, WB_PV = WB_S + 4, WB_PREADY = WB_PV + 2, WB_RAW = WB_PREADY + 2, WB_Q = WB_RAW + 2,
+       WB_S = WB_VEMPTY + WS_VS, WB_PV = WB_S + 4, WB_PREADY = WB_PV + 4, WB_RAW = WB_PREADY + 4, WB_Q = WB_RAW + 2,
        WB_DRAIN, WB_COUNT };
 constexpr int WS_OFF_BAR = WS_OFF_LIVE + WS_VS * 8;
 constexpr int WS_OFF_MISC = WS_OFF_BAR + WB_COUNT * 8;           // [0] tensor-memory slot, [4] abort flag
@@ -1095,6 +1095,12 @@ static_assert(record_bytes(4) <= WS_RAW_BYTES && record_bytes(3) <= WS_RAW_BYTES
 // Bounded wait for a phase of an mbarrier; gives up early when another role has raised the abort flag and raises it
 // itself when the limit runs out.
 __device__ __forceinline__ bool ws_wait(unsigned bar, unsigned parity, int limit, volatile int* abort_flag) {
+    {   // the common case: the phase is complete already (a test is cheaper than a wait that may suspend the thread)
+        unsigned ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+    }
     for (int it = 0; it < limit; ++it) {
         unsigned ok;
         asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
@@ -1171,7 +1177,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
     if (tid == 0) {
         for (int i = 0; i < WB_COUNT; ++i) {
             // probabilities: the 128 softmax threads of a tile; stage releases: the two issuing warps; queries: warps 0-8
-            const unsigned count = (i == WB_PREADY || i == WB_PREADY + 1) ? 128u : i == WB_Q ? 288u
+            const unsigned count = (i >= WB_PREADY && i < WB_PREADY + 4) ? 128u : i == WB_Q ? 288u
                                  : (i >= WB_KEMPTY && i < WB_KEMPTY + WS_KS) || (i >= WB_VEMPTY && i < WB_VEMPTY + WS_VS) ? 2u : 1u;
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar(i)), "r"(count) : "memory");
         }
@@ -1278,18 +1284,18 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 const float new_ref = raise ? mx : m_ref;
                 const float factor = raise ? fast_ex2(m_ref - new_ref) : 1.f;      // old reference -inf: factor 0, state is zero anyway
                 WST(3);
-                if (g > 0) {                                               // O += P V of the previous tile: long done as a rule
-                    if (!__all_sync(FULLM, ws_wait(bar(WB_PV + t), (g - 1) & 1, wait_limit, abort_flag))) { ok = false; return; }
+                // The accumulator rows in tensor memory are touched only when the reference grew: only then is O += P V of
+                // the previous tile awaited (one barrier per tile parity, so that a warp may skip any number of them).
+                if (g > 0 && __any_sync(FULLM, raise)) {
+                    if (!__all_sync(FULLM, ws_wait(bar(WB_PV + 2 * t + ((g - 1) & 1)), ((g - 1) >> 1) & 1, wait_limit, abort_flag))) { ok = false; return; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    if (__any_sync(FULLM, raise)) {                        // rescale this warp's accumulator rows in tensor memory
 #pragma unroll
-                        for (int q4 = 0; q4 < 4; ++q4) {
-                            float o[32];
-                            tc_ld32(tmem_row + 32 * q4, o);
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        float o[32];
+                        tc_ld32(tmem_row + 32 * q4, o);
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) o[i] *= factor;
-                            tc_st32(tmem_row + 32 * q4, o);
-                        }
+                        for (int i = 0; i < 32; ++i) o[i] *= factor;
+                        tc_st32(tmem_row + 32 * q4, o);
                     }
                 }
                 WST(4);
@@ -1315,7 +1321,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 tc_st32u(sbuf, pk);
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                ws_arrive(bar(WB_PREADY + t));
+                // one barrier per tile parity: the softmax of tile g + 1 does not wait for the issuing warp, that of tile g + 2 does
+                ws_arrive(bar(WB_PREADY + 2 * t + (g & 1)));
                 WST(6);
             };
 
@@ -1338,7 +1345,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
             }
             WST_FLUSH;
             // ---- output: o = (O + z) / l for the rows that carry a query
-            if (ok && !__all_sync(FULLM, ws_wait(bar(WB_PV + t), (n_tiles[t] - 1) & 1, wait_limit, abort_flag))) ok = false;
+            if (ok && !__all_sync(FULLM, ws_wait(bar(WB_PV + 2 * t + ((n_tiles[t] - 1) & 1)), ((n_tiles[t] - 1) >> 1) & 1, wait_limit, abort_flag))) ok = false;
             if (ok) {
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const float inv = l > 0.f ? 1.f / l : 0.f;
@@ -1384,58 +1391,53 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
             if (!(P.drop == 1 && g == 0)) ws_commit(bar(WB_S + 2 * t + (g & 1)));
             ws_commit(bar(WB_KEMPTY + st));
         };
-        auto issue_scores = [&](const int g) -> bool {          // S_t(g) = Q'_t K(g)^T
+        // Only lane 0 runs the loop.  Order per tile g: wait for the probabilities, O_t += P_t(g) V(g), S_t(g+2) (its score
+        // buffer is the one P_t(g) sits in, so it must follow that product in the pipe), then, off the critical path, the
+        // wait for the value stage the next round needs.
+        auto scores = [&](const int g) -> bool {                // key stage of tile g has landed (awaited by the caller)
             const int st = g % WS_KS;
-#if WUSHKV_WS_TIMING
-            WST(6);
-            if (!__all_sync(FULLM, ws_wait(bar(WB_Q), 0u, wait_limit, abort_flag))) return false;      // measurement only: a wait that is satisfied
-            WST(7);
-#endif
-            if (!__all_sync(FULLM, ws_wait(bar(WB_KFULL + st), (g / WS_KS) & 1, wait_limit, abort_flag))) return false;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (g >= mine) ws_arrive(bar(WB_KEMPTY + st));      // a tile only the other query tile reads: just release the stage
+            else if (g >= gC && P.use_tma) scores_of(std::true_type{}, g, st);
+            else scores_of(std::false_type{}, g, st);
+            return true;
+        };
+        auto key_landed = [&](const int g) -> bool { return ws_wait(bar(WB_KFULL + g % WS_KS), (g / WS_KS) & 1, wait_limit, abort_flag); };
+        auto value_landed = [&](const int g) -> bool { return ws_wait(bar(WB_VFULL + g % WS_VS), (g / WS_VS) & 1, wait_limit, abort_flag); };
+        if (lane == 0 && ok) {
+            ok = key_landed(0) && scores(0);
+            if (ok && NT > 1) ok = key_landed(1) && scores(1);
+            if (ok) ok = value_landed(0);
             WST(1);
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            if (lane == 0) {
-                if (g >= mine) ws_arrive(bar(WB_KEMPTY + st));  // a tile only the other query tile reads: just release the stage
-                else if (g >= gC && P.use_tma) scores_of(std::true_type{}, g, st);
-                else scores_of(std::false_type{}, g, st);
-            }
-            __syncwarp();
-            WST(2);
-            return true;
-        };
-        auto issue_values = [&](const int g) -> bool {          // O_t += P_t(g) V(g)
-            const int st = g % WS_VS;
-            if (!__all_sync(FULLM, ws_wait(bar(WB_VFULL + st), (g / WS_VS) & 1, wait_limit, abort_flag))) return false;
-            WST(3);
-            if (g >= mine) {
-                if (lane == 0) ws_arrive(bar(WB_VEMPTY + st));
-                __syncwarp();
-                return true;
-            }
-            const bool swz = g >= gC && P.use_tma;
-            // swizzled values: rows (keys) of 128 bytes, 8-key groups 1024 bytes apart, channel halves 8192 bytes apart: 16 keys = 2048 bytes
-            const unsigned long long vb = (swz ? v_swz0 : v_plain0) + static_cast<unsigned>(st * (TC_K_BYTES >> 4));
-            const unsigned vstep = swz ? (2048u >> 4) : (256u >> 4);
-            if (!__all_sync(FULLM, ws_wait(bar(WB_PREADY + t), g & 1, wait_limit, abort_flag))) return false;
-            WST(4);
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            if (lane == 0) {
-                const unsigned prob = acc_o + 128u + 64u * (g & 1);
+            for (int g = 0; g < NT && ok; ++g) {
+                const int st = g % WS_VS;
+                if (g < mine) {
+                    if (!ws_wait(bar(WB_PREADY + 2 * t + (g & 1)), (g >> 1) & 1, wait_limit, abort_flag)) { ok = false; break; }
+                    WST(2);
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const bool swz = g >= gC && P.use_tma;
+                    // swizzled values: rows (keys) of 128 bytes, 8-key groups 1024 bytes apart, channel halves 8192 bytes apart: 16 keys = 2048 bytes
+                    const unsigned long long vb = (swz ? v_swz0 : v_plain0) + static_cast<unsigned>(st * (TC_K_BYTES >> 4));
+                    const unsigned vstep = swz ? (2048u >> 4) : (256u >> 4);
+                    const unsigned prob = acc_o + 128u + 64u * (g & 1);
 #pragma unroll
-                for (int ks = 0; ks < TN / 16; ++ks)
-                    tc_mma_ts(acc_o, prob + 8 * ks, vb + ks * vstep, TC_IDESC_O, (g > 0 || ks > 0) ? 1u : 0u);
-                ws_commit(bar(WB_PV + t));
-                ws_commit(bar(WB_VEMPTY + st));
+                    for (int ks = 0; ks < TN / 16; ++ks)
+                        tc_mma_ts(acc_o, prob + 8 * ks, vb + ks * vstep, TC_IDESC_O, (g > 0 || ks > 0) ? 1u : 0u);
+                    ws_commit(bar(WB_PV + 2 * t + (g & 1)));
+                    ws_commit(bar(WB_VEMPTY + st));
+                } else {
+                    ws_arrive(bar(WB_VEMPTY + st));
+                }
+                WST(3);
+                // (a key tile written by the staging threads comes together with its value tile, whose stage the product
+                // just issued releases: its arrival cannot be awaited any earlier than here)
+                if (g + 2 < NT) { if (!key_landed(g + 2)) { ok = false; break; } scores(g + 2); }
+                WST(4);
+                if (g + 1 < NT && !value_landed(g + 1)) { ok = false; break; }
+                WST(5);
             }
-            __syncwarp();
-            WST(5);
-            return true;
-        };
-        if (ok) ok = issue_scores(0);
-        for (int g = 0; g < NT && ok; ++g) {
-            if (g + 1 < NT) ok = issue_scores(g + 1);
-            if (ok) ok = issue_values(g);
         }
+        __syncwarp();
         WST_FLUSH;
     } else {
         // =============================== staging of key / value tiles =====================================
