@@ -84,7 +84,7 @@ inline bool opt_in_dynamic_smem(const void* fn, int bytes) {
 // Tensor map of a 16-bit row tensor [rows][n_heads][128 channels]: boxes of box_rows x 64 channels (128 bytes), written to
 // shared memory as 128-byte-swizzled rows.  Coordinates of a copy: (channel 0 or 64, head, first row).  False when the
 // driver entry point is missing or refuses (callers then stage with 16-byte copies).
-inline bool make_row_tensor_map(CUtensorMap& map, bool bf16, const void* base, int n_heads, long long rows, int box_rows) {
+inline bool make_row_tensor_map(CUtensorMap& map, bool bf16, const void* base, int n_heads, long long rows, int box_rows, int box_heads = 1) {
     typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -98,7 +98,7 @@ inline bool make_row_tensor_map(CUtensorMap& map, bool bf16, const void* base, i
     if (!encode || rows <= 0 || n_heads <= 0) return false;
     const cuuint64_t gdim[3] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(n_heads), static_cast<cuuint64_t>(rows)};
     const cuuint64_t gstride[2] = {static_cast<cuuint64_t>(D) * 2, static_cast<cuuint64_t>(n_heads) * D * 2};
-    const cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(box_rows)}, estr[3] = {1, 1, 1};
+    const cuuint32_t box[3] = {64, static_cast<cuuint32_t>(box_heads), static_cast<cuuint32_t>(box_rows)}, estr[3] = {1, 1, 1};
     return encode(&map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), gdim, gstride, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;

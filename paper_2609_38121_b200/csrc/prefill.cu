@@ -1147,7 +1147,9 @@ __device__ unsigned long long g_ws_t[32];
 
 template <int BITS>
 __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillParams P, const __grid_constant__ CUtensorMap map_k,
-                                                                        const __grid_constant__ CUtensorMap map_v) {
+                                                                        const __grid_constant__ CUtensorMap map_v,
+                                                                        const __grid_constant__ CUtensorMap map_q0,
+                                                                        const __grid_constant__ CUtensorMap map_q1) {
     extern __shared__ __align__(1024) unsigned char sm_ws[];
     constexpr int REC = record_bytes(BITS);
     const CacheView& c = P.c;
@@ -1176,8 +1178,9 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
     }
     if (tid == 0) {
         for (int i = 0; i < WB_COUNT; ++i) {
-            // probabilities: the 128 softmax threads of a tile; stage releases: the two issuing warps; queries: warps 0-8
-            const unsigned count = (i >= WB_PREADY && i < WB_PREADY + 4) ? 128u : i == WB_Q ? 288u
+            // probabilities: the 128 softmax threads of a tile; stage releases: the two issuing warps; queries: one announcement
+            // of bulk tensor copies, or warps 0-8 with their 16-byte copies
+            const unsigned count = (i >= WB_PREADY && i < WB_PREADY + 4) ? 128u : i == WB_Q ? (P.use_tma ? 1u : 288u)
                                  : (i >= WB_KEMPTY && i < WB_KEMPTY + WS_KS) || (i >= WB_VEMPTY && i < WB_VEMPTY + WS_VS) ? 2u : 1u;
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar(i)), "r"(count) : "memory");
         }
@@ -1211,20 +1214,37 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const unsigned tmem_base = *tmem_slot;
 
-    // ---- the packed query tiles: row r of tile t = chunk position (2 pr + t) R + r / G (clamped), head h G + r % G
-    // (staged by the softmax and MMA warps; the staging warps start on the key side at once)
-    for (int item = tid; item < 4 * TM * 16 && warp < 9; item += 288) {
-        const int q = item >> 11, part = q & 1, r = (item >> 4) & (TM - 1), piece = item & 15;
-        const int t = n_rows[q >> 1] > 0 ? (q >> 1) : 0;        // a tile without rows aliases tile 0's (never used)
-        const int rr = min(r, n_rows[t] - 1);
-        const int tok = first + (2 * pr + t) * R + rr / G, jq = h * G + rr % G;
-        const __half* src = P.QP + static_cast<long long>(part) * P.total_new * c.n_q * D + (static_cast<long long>(tok) * c.n_q + jq) * D + 8 * piece;
-        cp16(smem_addr(sm_ws + WS_OFF_Q + q * TC_Q_BYTES + (r >> 3) * 2048 + piece * 128 + (r & 7) * 16), src, 16u);
+    // ---- the packed query tiles: row r of tile t = chunk position (2 pr + t) R + r / G, head h G + r % G.  With bulk tensor
+    // copies a box of (64 channels, G heads, R positions) lands as R G rows of 128 bytes in exactly that order (128-byte
+    // swizzle; rows past the chunk hold zeros or the next sequence's queries and are never stored); otherwise the softmax
+    // and MMA warps place 16-byte pieces (rows clamped to the chunk) while the staging warps start on the key side at once.
+    if (P.use_tma) {
+        if (tid == 288) {
+            const unsigned box_bytes = 128u * static_cast<unsigned>(G * R);
+            ws_expect_tx(bar(WB_Q), 4u * box_bytes * ((n_tiles[0] > 0 ? 1u : 0u) + (n_tiles[1] > 0 ? 1u : 0u)));
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (n_tiles[q >> 1] == 0) continue;
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf)
+                    tma_load_3d(smem_addr(sm_ws + WS_OFF_Q + q * TC_Q_BYTES + hf * 16384), (q & 1) ? &map_q1 : &map_q0, 64 * hf, h * G,
+                                first + (2 * pr + (q >> 1)) * R, bar(WB_Q));
+            }
+        }
+    } else {
+        for (int item = tid; item < 4 * TM * 16 && warp < 9; item += 288) {
+            const int q = item >> 11, part = q & 1, r = (item >> 4) & (TM - 1), piece = item & 15;
+            const int t = n_rows[q >> 1] > 0 ? (q >> 1) : 0;        // a tile without rows aliases tile 0's (never used)
+            const int rr = min(r, n_rows[t] - 1);
+            const int tok = first + (2 * pr + t) * R + rr / G, jq = h * G + rr % G;
+            const __half* src = P.QP + static_cast<long long>(part) * P.total_new * c.n_q * D + (static_cast<long long>(tok) * c.n_q + jq) * D + 8 * piece;
+            cp16(smem_addr(sm_ws + WS_OFF_Q + q * TC_Q_BYTES + (r >> 3) * 2048 + piece * 128 + (r & 7) * 16), src, 16u);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        if (warp < 9) ws_arrive(bar(WB_Q));
     }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    if (warp < 9) ws_arrive(bar(WB_Q));
 
     if (warp < 8) {
         // =============================== softmax of query tile t ==========================================
@@ -1373,7 +1393,9 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
         bool ok = __all_sync(FULLM, ws_wait(bar(WB_Q), 0u, wait_limit, abort_flag));
         WST(0);
         // Descriptors are built once; their low bits hold the start address / 16, so a byte offset is added as offset / 16.
-        const unsigned long long q_desc = tc_desc(smem_addr(sm_ws + WS_OFF_Q + 2 * t * TC_Q_BYTES), 128, 2048);
+        const bool q_swz = P.use_tma != 0;                      // query tiles written by bulk tensor copies: 128-byte-swizzled rows, two 16 KB boxes
+        const unsigned long long q_desc = q_swz ? tc_desc_sw128(smem_addr(sm_ws + WS_OFF_Q + 2 * t * TC_Q_BYTES), 16, 1024)
+                                                : tc_desc(smem_addr(sm_ws + WS_OFF_Q + 2 * t * TC_Q_BYTES), 128, 2048);
         const unsigned long long k_plain0 = tc_desc(smem_addr(sm_ws + WS_OFF_K), 128, 2048), k_swz0 = tc_desc_sw128(smem_addr(sm_ws + WS_OFF_K), 16, 1024);
         const unsigned long long v_plain0 = tc_desc(smem_addr(sm_ws + WS_OFF_V), 128, 1024), v_swz0 = tc_desc_sw128(smem_addr(sm_ws + WS_OFF_V), 8192, 1024);
         const unsigned acc_o = tmem_base + 256u * t;
@@ -1385,8 +1407,9 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
             for (int ks = 0; ks < 8; ++ks) {
                 // swizzled: channels 0-63 and 64-127 are two boxes of 8 KB; a k-step of 16 channels is 32 bytes inside the 128-byte row
                 const unsigned long long bdesc = kb + static_cast<unsigned>((SWZ ? (ks >> 2) * 8192 + (ks & 3) * 32 : ks * 256) >> 4);
-                tc_mma(acc, q_desc + static_cast<unsigned>(ks * 256 >> 4), bdesc, TC_IDESC_S, ks > 0 ? 1u : 0u);
-                tc_mma(acc, q_desc + static_cast<unsigned>((TC_Q_BYTES + ks * 256) >> 4), bdesc, TC_IDESC_S, 1u);
+                const unsigned long long adesc = q_desc + static_cast<unsigned>((q_swz ? (ks >> 2) * 16384 + (ks & 3) * 32 : ks * 256) >> 4);
+                tc_mma(acc, adesc, bdesc, TC_IDESC_S, ks > 0 ? 1u : 0u);
+                tc_mma(acc, adesc + static_cast<unsigned>(TC_Q_BYTES >> 4), bdesc, TC_IDESC_S, 1u);
             }
             if (!(P.drop == 1 && g == 0)) ws_commit(bar(WB_S + 2 * t + (g & 1)));
             ws_commit(bar(WB_KEMPTY + st));
@@ -1584,7 +1607,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                         for (int it = 0; it < 512 && !ws_wait(bar(full0 + i), (armed[i] / depth) & 1, 1, abort_flag); ++it) __nanosleep(2000);
             }
         }
-        if (tid == 288 && *abort_flag) {                        // the same for the record copies
+        if (tid == 288 && *abort_flag) {                        // the same for the query and record copies
+            if (P.use_tma) for (int it = 0; it < 512 && !ws_wait(bar(WB_Q), 0u, 1, abort_flag); ++it) __nanosleep(2000);
 #pragma unroll
             for (int i = 0; i < 2; ++i)
                 if (nB > i) for (int it = 0; it < 64 && !ws_wait(bar(WB_RAW + i), raw_uses[i] & 1, 1, abort_flag); ++it) __nanosleep(2000);
@@ -1692,9 +1716,14 @@ static int prefill_attn_impl(const wushkv_cache* cache, int32_t batch, const int
         P.use_tma = (mk && mv && !knobs().prefill_no_tma) ? 1 : 0;
         if (!knobs().prefill_one_tile) {        // warp-specialised kernel: a pair of query tiles per CTA
             const dim3 grid_ws(static_cast<unsigned>(batch) * ((P.tiles_per_seq + 1) / 2), P.c.n_kv);
+            // the query operands (value, remainder) as [token][query head][128 channels]: a box is one tile's (G heads, R positions)
+            CUtensorMap map_q0, map_q1;
+            const bool mq = make_row_tensor_map(map_q0, false, P.QP, P.c.n_q, total_new, R, P.c.G) &&
+                            make_row_tensor_map(map_q1, false, P.QP + static_cast<size_t>(total_new) * P.c.n_q * D, P.c.n_q, total_new, R, P.c.G);
+            if (!mq) P.use_tma = 0;
             auto launch_ws = [&](auto kernel) -> bool {
                 if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(kernel), WS_SMEM)) return false;
-                kernel<<<grid_ws, WS_THREADS, WS_SMEM, st>>>(P, map_k, map_v);
+                kernel<<<grid_ws, WS_THREADS, WS_SMEM, st>>>(P, map_k, map_v, map_q0, map_q1);
                 return true;
             };
             const bool ok = P.c.bits == 2 ? launch_ws(prefill_attn_ws_kernel<2>) : P.c.bits == 3 ? launch_ws(prefill_attn_ws_kernel<3>)
