@@ -1636,6 +1636,217 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
 }
 
+// ------------------------------------------------------------------------------------------------
+// 1b. transforms of the chunk on tcgen05 (the default for plain, i.e. not projected, inputs)
+// ------------------------------------------------------------------------------------------------
+// The same arithmetic as prefill_prep_kernel (bf16 x bf16 products, exact in the fp32 accumulator; T_K^{-T} as three bf16
+// terms), as tcgen05.mma with the accumulator in tensor memory.  A CTA keeps its head's transform in shared memory as the
+// B operand and walks over 128-token tiles:
+//   warp 16  one lane requests the token tiles: two bulk tensor copies (channel halves) of 128 rows x 128 bytes into a
+//            two-deep ring, the A operand as it comes;
+//   warp 17  one lane issues 8 MMAs (M 128, N 128, K 16) per term into one of two 128-column accumulators;
+//   warps 0-15  a thread owns 32 channels of one token of the tile (one warp alone per scheduler spends its time on
+//            instruction latency): tcgen05.ld, the roundings (k' through bf16 to fp16; q' as fp16 value + fp16 remainder,
+//            and their sum over the channels); the rows go through a shared-memory tile so that the stores to global memory
+//            are whole 256-byte rows.  Key-head CTAs also convert the chunk's values.
+// Barriers come in pairs (one per ring slot), every wait is bounded.
+constexpr int PT_THREADS = 576;                                  // warps 0-15 epilogue, 16 copies, 17 MMA issue
+constexpr int PT_OFF_T = 0;                                      // three terms of 128 x 128 bf16, K-major core matrices
+constexpr int PT_OFF_X = 3 * D * D * 2;                          // two token tiles (128-byte-swizzled rows, two 16 KB boxes each)
+constexpr int PT_X_BYTES = PREP_TOK * D * 2;
+enum { PB_XFULL = 0, PB_XEMPTY = 2, PB_DFULL = 4, PB_DEMPTY = 6, PB_DRAIN = 8, PB_COUNT = 9 };
+constexpr int PT_OUT_PITCH = D * 2 + 16;                         // bytes per staged output row (272: conflict-free 16-byte pieces)
+constexpr int PT_OFF_OUT = PT_OFF_X + 2 * PT_X_BYTES;            // one fp16 output tile on its way to global memory
+constexpr int PT_OFF_QS = PT_OFF_OUT + PREP_TOK * PT_OUT_PITCH;  // float[4][128]: partial sums of q' over channel quarters
+constexpr int PT_OFF_BAR = PT_OFF_QS + 4 * PREP_TOK * 4;
+constexpr int PT_OFF_MISC = PT_OFF_BAR + PB_COUNT * 8;           // [0] tensor-memory slot, [4] abort flag
+constexpr int PT_SMEM = PT_OFF_MISC + 16;
+constexpr unsigned PT_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((static_cast<unsigned>(D) >> 3) << 17) | ((static_cast<unsigned>(PREP_TOK) >> 4) << 24);   // fp32 <- bf16 x bf16, K-major
+static_assert(PT_OFF_X % 1024 == 0, "swizzled tiles need 1024-byte alignment");
+
+__global__ void __launch_bounds__(PT_THREADS, 1) prefill_prep_tc_kernel(PrefillParams P, const __grid_constant__ CUtensorMap map_k,
+                                                                        const __grid_constant__ CUtensorMap map_q) {
+    extern __shared__ __align__(1024) unsigned char sm_pt[];
+    const int hs = blockIdx.y;
+    const bool is_key = hs < P.c.n_kv;
+    const int head = is_key ? hs : hs - P.c.n_kv;
+    const int kvh = is_key ? head : head / P.c.G;
+    const int n_terms = is_key ? 1 : 3;
+    const int n_heads = is_key ? P.c.n_kv : P.c.n_q;
+    const float* T = (is_key ? P.c.T_K : P.c.T_K_invT) + static_cast<long long>(kvh) * D * D;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const unsigned bar0 = smem_addr(sm_pt + PT_OFF_BAR);
+    auto bar = [&](int i) -> unsigned { return bar0 + 8u * static_cast<unsigned>(i); };
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(sm_pt + PT_OFF_MISC);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm_pt + PT_OFF_MISC + 4);
+    const int n_my_tiles = (P.total_new + PREP_TOK - 1) / PREP_TOK > static_cast<int>(blockIdx.x)
+                               ? ((P.total_new + PREP_TOK - 1) / PREP_TOK - 1 - static_cast<int>(blockIdx.x)) / static_cast<int>(gridDim.x) + 1 : 0;
+    if (n_my_tiles == 0) return;
+
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(256u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+        for (int i = 0; i < PB_COUNT; ++i) {
+            const unsigned count = (i == PB_DEMPTY || i == PB_DEMPTY + 1) ? 512u : 1u;      // accumulator released by the 512 epilogue threads
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar(i)), "r"(count) : "memory");
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // the transform as the B operand: element (i, j) of term `term` at (i / 8) * 2048 + (j / 8) * 128 + (i % 8) * 16 + (j % 8) * 2
+    for (int idx = tid; idx < D * D; idx += PT_THREADS) {
+        const int i = idx >> 7, j = idx & 127;
+        float x = __ldg(T + idx);
+        const int off = (i >> 3) * 2048 + (j >> 3) * 128 + (i & 7) * 16 + (j & 7) * 2;
+#pragma unroll
+        for (int term = 0; term < 3; ++term) {
+            if (term < n_terms) {
+                const unsigned short hb = float_to_bf16_bits(x);
+                *reinterpret_cast<unsigned short*>(sm_pt + PT_OFF_T + term * (D * D * 2) + off) = hb;
+                x -= bf16_bits_to_float(hb);
+            }
+        }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const unsigned tmem_base = *tmem_slot;
+    const int wait_limit = P.wait_limit > 0 ? P.wait_limit : (1 << 24);
+
+    if (warp == 16) {
+        // ---- token tiles
+        int armed[2] = {-1, -1};
+        if (lane == 0) {
+            const CUtensorMap* map = is_key ? &map_k : &map_q;
+            for (int i = 0; i < n_my_tiles; ++i) {
+                const int s = i & 1, tok0 = (static_cast<int>(blockIdx.x) + i * static_cast<int>(gridDim.x)) * PREP_TOK;
+                if (i >= 2 && !ws_wait(bar(PB_XEMPTY + s), ((i >> 1) - 1) & 1, wait_limit, abort_flag)) break;
+                ws_expect_tx(bar(PB_XFULL + s), PT_X_BYTES);
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf)
+                    tma_load_3d(smem_addr(sm_pt + PT_OFF_X + s * PT_X_BYTES + hf * 16384), map, 64 * hf, head, tok0, bar(PB_XFULL + s));
+                if (s == 0) armed[0] = i; else armed[1] = i;
+            }
+            if (*abort_flag) {                                  // give announced copies a bounded time to land
+#pragma unroll
+                for (int s = 0; s < 2; ++s)
+                    if (armed[s] >= 0) for (int it = 0; it < 512 && !ws_wait(bar(PB_XFULL + s), (armed[s] >> 1) & 1, 1, abort_flag); ++it) __nanosleep(2000);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 17) {
+        // ---- MMA issue
+        if (lane == 0) {
+            const unsigned long long t_desc = tc_desc(smem_addr(sm_pt + PT_OFF_T), 128, 2048);
+            const unsigned long long x_desc = tc_desc_sw128(smem_addr(sm_pt + PT_OFF_X), 16, 1024);
+            for (int i = 0; i < n_my_tiles; ++i) {
+                const int s = i & 1;
+                if (!ws_wait(bar(PB_XFULL + s), (i >> 1) & 1, wait_limit, abort_flag)) break;
+                if (i >= 2 && !ws_wait(bar(PB_DEMPTY + s), ((i >> 1) - 1) & 1, wait_limit, abort_flag)) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const unsigned acc = tmem_base + 128u * s;
+                for (int term = 0; term < n_terms; ++term) {
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        tc_mma(acc, x_desc + static_cast<unsigned>((s * PT_X_BYTES + (ks >> 2) * 16384 + (ks & 3) * 32) >> 4),
+                               t_desc + static_cast<unsigned>((term * (D * D * 2) + ks * 256) >> 4), PT_IDESC, (term > 0 || ks > 0) ? 1u : 0u);
+                }
+                ws_commit(bar(PB_DFULL + s));
+                ws_commit(bar(PB_XEMPTY + s));
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---- epilogue: 16 warps; warp w reads rows 32 (w % 4) .. + 31 (its lanes of tensor memory), channels 32 (w / 4) .. + 31
+        constexpr int EPI = 512;
+        const int row = 32 * (warp & 3) + lane, cq = warp >> 2;
+        const unsigned tmem_row = tmem_base + (static_cast<unsigned>((warp & 3) * 32) << 16) + 32u * cq;
+        const long long lo_off = static_cast<long long>(P.total_new) * n_heads * D;
+        float* qs_part = reinterpret_cast<float*>(sm_pt + PT_OFF_QS);      // [4][128] partial channel sums
+        bool ok = true;
+        for (int i = 0; i < n_my_tiles && ok; ++i) {
+            const int s = i & 1, tok0 = (static_cast<int>(blockIdx.x) + i * static_cast<int>(gridDim.x)) * PREP_TOK;
+            if (is_key) {                                       // the chunk's values as fp16 (no transform); coalesced 16-byte pieces
+                for (int item = tid; item < PREP_TOK * 16; item += EPI) {
+                    const int r = item >> 4, piece = item & 15;
+                    if (tok0 + r < P.total_new) {
+                        const long long off = (static_cast<long long>(tok0 + r) * P.c.n_kv + head) * D + 8 * piece;
+                        const uint4 v = __ldg(reinterpret_cast<const uint4*>(P.V_new + off));
+                        const unsigned w[4] = {v.x, v.y, v.z, v.w};
+                        unsigned o[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) o[e] = pack_half2(bf16_bits_to_float(w[e] & 0xffff), bf16_bits_to_float(w[e] >> 16));
+                        *reinterpret_cast<uint4*>(P.VP + off) = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
+                }
+            }
+            {   // the give-up decision is taken by the 512 epilogue threads together (they meet at named barriers below)
+                const unsigned got = ws_wait(bar(PB_DFULL + s), (i >> 1) & 1, wait_limit, abort_flag) ? 1u : 0u;
+                unsigned all;
+                asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred p, 3, 512, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                             : "=r"(all) : "r"(got) : "memory");
+                if (!all) { ok = false; break; }
+            }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            float o[32];
+            tc_ld32(tmem_row + 128u * s, o);
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            ws_arrive(bar(PB_DEMPTY + s));                      // the accumulator is free again
+            float sum = 0.f;
+            unsigned hi[16], lo[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+                if (is_key) {                                   // the cache holds bf16(k')
+                    hi[e] = pack_half2(bf16_bits_to_float(float_to_bf16_bits(o[2 * e])), bf16_bits_to_float(float_to_bf16_bits(o[2 * e + 1])));
+                    lo[e] = 0u;
+                } else {                                        // q' as fp16 value + fp16 rounding remainder
+                    hi[e] = pack_half2(o[2 * e], o[2 * e + 1]);
+                    const float2 hv = h2f2u(hi[e]);
+                    lo[e] = pack_half2(o[2 * e] - hv.x, o[2 * e + 1] - hv.y);
+                    const float2 lv = h2f2u(lo[e]);
+                    sum += (hv.x + lv.x) + (hv.y + lv.y);
+                }
+            }
+            unsigned char* stage = sm_pt + PT_OFF_OUT + row * PT_OUT_PITCH + 64 * cq;
+            // the staged tile leaves as whole rows: 16 consecutive threads per 256-byte row
+            auto flush = [&](const unsigned (&w)[16], __half* base) {
+#pragma unroll
+                for (int e = 0; e < 16; e += 4) *reinterpret_cast<uint4*>(stage + 4 * e) = make_uint4(w[e], w[e + 1], w[e + 2], w[e + 3]);
+                asm volatile("bar.sync 2, 512;" ::: "memory");
+#pragma unroll
+                for (int item = tid; item < PREP_TOK * 16; item += EPI) {
+                    const int r = item >> 4, piece = item & 15;
+                    if (tok0 + r < P.total_new)
+                        *reinterpret_cast<uint4*>(base + (static_cast<long long>(tok0 + r) * n_heads + head) * D + 8 * piece) =
+                            *reinterpret_cast<const uint4*>(sm_pt + PT_OFF_OUT + r * PT_OUT_PITCH + 16 * piece);
+                }
+                asm volatile("bar.sync 2, 512;" ::: "memory");
+            };
+            if (!is_key) qs_part[cq * PREP_TOK + row] = sum;
+            flush(hi, is_key ? P.KP : P.QP);
+            if (!is_key) {
+                flush(lo, P.QP + lo_off);
+                if (cq == 0 && tok0 + row < P.total_new)
+                    P.qsum[static_cast<long long>(tok0 + row) * P.c.n_q + head] =
+                        (qs_part[row] + qs_part[PREP_TOK + row]) + (qs_part[2 * PREP_TOK + row] + qs_part[3 * PREP_TOK + row]);
+            }
+        }
+    }
+
+    __syncthreads();
+    if (*abort_flag && tid == 544) {                            // the issuing thread: let whatever was issued finish (bounded) before the release
+        atomicOr(P.c.dev_status, WUSHKV_DEV_COPY_TIMEOUT);
+        ws_commit(bar(PB_DRAIN));
+        for (int it = 0; it < 512 && !ws_wait(bar(PB_DRAIN), 0u, 1, abort_flag); ++it) __nanosleep(2000);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+}
+
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
 struct PrefillPlan { size_t off_kp, off_vp, off_qp, off_qsum, total; };
@@ -1701,7 +1912,14 @@ static int prefill_attn_impl(const wushkv_cache* cache, int32_t batch, const int
     {   // about one wave of CTAs: each keeps its head's transform resident and walks over token tiles
         const int n_tok_tiles = (total_new + PREP_TOK - 1) / PREP_TOK, slots = P.c.n_kv + P.c.n_q;
         const int per_slot = std::max(1, std::min(n_tok_tiles, sm_count() / slots));
-        prefill_prep_kernel<<<dim3(per_slot, slots), 256, smem_prep, st>>>(P);
+        // plain inputs: the tcgen05 kernel, fed by bulk tensor copies of the bf16 rows as they come
+        CUtensorMap in_k, in_q;
+        const bool tc_prep = !P.pro.rope && !knobs().prefill_legacy && !knobs().prefill_no_tma &&
+                             make_row_tensor_map(in_k, true, K_new, P.c.n_kv, total_new, PREP_TOK) &&
+                             make_row_tensor_map(in_q, true, Q_new, P.c.n_q, total_new, PREP_TOK) &&
+                             opt_in_dynamic_smem(reinterpret_cast<const void*>(prefill_prep_tc_kernel), PT_SMEM);
+        if (tc_prep) prefill_prep_tc_kernel<<<dim3(per_slot, slots), PT_THREADS, PT_SMEM, st>>>(P, in_k, in_q);
+        else prefill_prep_kernel<<<dim3(per_slot, slots), 256, smem_prep, st>>>(P);
     }
     if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
     if (!knobs().prefill_legacy) {              // tcgen05 path: the G heads of a KV head share a 128-row tile
