@@ -81,6 +81,25 @@ __device__ __forceinline__ void hmma(float (&c)[4], unsigned a0, unsigned a1, un
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ float fast_ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+// three-input maximum and packed fp32 arithmetic (two lanes per instruction)
+__device__ __forceinline__ float max3f(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float2 fma2f(float2 a, float m, float c) {        // (a.x m + c, a.y m + c)
+    float2 d;
+    asm("{\n\t.reg .b64 va, vm, vc, vd;\n\tmov.b64 va, {%2, %3};\n\tmov.b64 vm, {%4, %4};\n\tmov.b64 vc, {%5, %5};\n\t"
+        "fma.rn.f32x2 vd, va, vm, vc;\n\tmov.b64 {%0, %1}, vd;\n\t}"
+        : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(m), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float2 add2f(float2 a, float2 b) {
+    float2 d;
+    asm("{\n\t.reg .b64 va, vb, vd;\n\tmov.b64 va, {%2, %3};\n\tmov.b64 vb, {%4, %5};\n\tadd.rn.f32x2 vd, va, vb;\n\tmov.b64 {%0, %1}, vd;\n\t}"
+        : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return d;
+}
 __device__ __forceinline__ unsigned pack_half2(float lo, float hi) {
     unsigned d;
     asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
@@ -589,6 +608,13 @@ __device__ __forceinline__ void tc_st32u(unsigned taddr, const unsigned (&v)[32]
           "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
         : "memory");
 }
+__device__ __forceinline__ void tc_st16u(unsigned taddr, const unsigned (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]),
+          "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+        : "memory");
+}
 __device__ __forceinline__ void tc_ld32(unsigned taddr, float (&v)[32]) {
     unsigned r[32];
     asm volatile(
@@ -602,6 +628,29 @@ __device__ __forceinline__ void tc_ld32(unsigned taddr, float (&v)[32]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+// two 32-column loads in flight before the one wait
+__device__ __forceinline__ void tc_ld64(unsigned taddr, float (&v)[64]) {
+    unsigned r[64];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]),
+          "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]),
+          "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]),
+          "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+        : "r"(taddr + 32u) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 64; ++i) v[i] = __uint_as_float(r[i]);
 }
 __device__ __forceinline__ void tc_st32(unsigned taddr, const float (&v)[32]) {
     asm volatile(
@@ -1279,27 +1328,26 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 }
                 WST(1);
                 float s[TN];
-                {
-                    float lo[32], hi[32];
-                    tc_ld32(sbuf, lo);
-                    tc_ld32(sbuf + 32, hi);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) { s[i] = lo[i]; s[32 + i] = hi[i]; }
-                }
+                tc_ld64(sbuf, s);
                 WST(2);
-                float mx = -INFINITY;
+                // scores before the common factor k2 = scale * log2(e) > 0, which is folded into the exponent's multiply-add
+                // below: the maximum is taken of these (three-input max), then scaled once
+                if (PACKED || MASKED) {
 #pragma unroll
-                for (int j = 0; j < TN; ++j) {
-                    float v;
-                    if (PACKED) { const float2 mk = h2f2u(meta[j].x); v = k2 * fmaf(mk.y, my_qsum, mk.x * s[j]); }
-                    else v = k2 * s[j];
-                    if (MASKED) {
-                        const bool live = ((j < 32 ? live_lo >> j : live_hi >> (j - 32)) & 1u) != 0u;
-                        if (!live || crow0 + j > my_row) v = -INFINITY;
+                    for (int j = 0; j < TN; ++j) {
+                        float v = s[j];
+                        if (PACKED) { const float2 mk = h2f2u(meta[j].x); v = fmaf(mk.y, my_qsum, mk.x * v); }
+                        if (MASKED) {
+                            const bool live = ((j < 32 ? live_lo >> j : live_hi >> (j - 32)) & 1u) != 0u;
+                            if (!live || crow0 + j > my_row) v = -INFINITY;
+                        }
+                        s[j] = v;
                     }
-                    s[j] = v;
-                    mx = fmaxf(mx, v);
                 }
+                float mx_raw = fmaxf(s[0], s[1]);
+#pragma unroll
+                for (int j = 2; j < TN; j += 2) mx_raw = max3f(mx_raw, s[j], s[j + 1]);
+                const float mx = k2 * mx_raw;
                 const bool raise = mx > m_ref + REF_SLACK;                 // also the first finite maximum (m_ref = -inf)
                 const float new_ref = raise ? mx : m_ref;
                 const float factor = raise ? fast_ex2(m_ref - new_ref) : 1.f;      // old reference -inf: factor 0, state is zero anyway
@@ -1323,22 +1371,26 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 m_ref = new_ref;
                 const float ref = m_ref == -INFINITY ? 0.f : m_ref;
                 // ---- probabilities: (p Delta_v) as fp16 pairs over the first 32 columns of the score buffer just read
-                unsigned pk[32];
+                float2 lsum = make_float2(0.f, 0.f);                       // two partial sums
 #pragma unroll
-                for (int kc = 0; kc < TN / 8; ++kc) {
-                    float w[8];
+                for (int half = 0; half < 2; ++half) {                     // 32 keys = 16 columns of fp16 pairs at a time
+                    unsigned pk[16];
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const float p = fast_ex2(s[8 * kc + e] - ref);
-                        l += p;
-                        if (PACKED) { const float2 mv = h2f2u(meta[8 * kc + e].y); z = fmaf(p, mv.y, z); w[e] = p * mv.x; }
-                        else w[e] = p;
+                    for (int e16 = 0; e16 < 16; ++e16) {
+                        const int e = 16 * half + e16;
+                        float2 pr = make_float2(fast_ex2(fmaf(s[2 * e], k2, -ref)), fast_ex2(fmaf(s[2 * e + 1], k2, -ref)));     // k2 s - ref in one rounding
+                        lsum.x += pr.x; lsum.y += pr.y;
+                        if (PACKED) {
+                            const float2 mv0 = h2f2u(meta[2 * e].y), mv1 = h2f2u(meta[2 * e + 1].y);
+                            z = fmaf(pr.x, mv0.y, fmaf(pr.y, mv1.y, z));
+                            pr.x *= mv0.x; pr.y *= mv1.x;
+                        }
+                        pk[e16] = pack_half2(pr.x, pr.y);
                     }
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) pk[4 * kc + e] = pack_half2(w[2 * e], w[2 * e + 1]);
+                    tc_st16u(sbuf + 16 * half, pk);
                 }
+                l += lsum.x + lsum.y;
                 WST(5);
-                tc_st32u(sbuf, pk);
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 // one barrier per tile parity: the softmax of tile g + 1 does not wait for the issuing warp, that of tile g + 2 does
@@ -1348,20 +1400,22 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
 
             constexpr int FAR_BELOW = -(1 << 30);
             for (int g = 0; g < n_tiles[t] && ok; ++g) {
-                if (g < nA) {
-                    const int nv = min(TN, n_old_fp - g * TN);
-                    if (nv == TN) soft(std::false_type{}, std::false_type{}, g, 0u, 0u, FAR_BELOW);
-                    else soft(std::false_type{}, std::true_type{}, g, nv >= 32 ? 0xffffffffu : (1u << nv) - 1u,
-                              nv >= 32 ? (1u << (nv - 32)) - 1u : 0u, FAR_BELOW);
-                } else if (g < gC) {
-                    soft(std::true_type{}, std::true_type{}, g, 0u, 0u, FAR_BELOW);
-                } else {
-                    const int kt = g - gC, nv = min(TN, n_new - kt * TN);
+                // valid keys of the tile and the chunk row of its first key (old positions: visible to every row)
+                int nv = TN, crow0 = FAR_BELOW;
+                bool masked = false;
+                if (g < nA) { nv = min(TN, n_old_fp - g * TN); masked = nv < TN; }
+                else if (g >= gC) {
+                    const int kt = g - gC;
+                    nv = min(TN, n_new - kt * TN); crow0 = kt * TN;
                     // no mask needed when every key of the tile exists and lies at or below every row's own position
-                    if (nv == TN && kt * TN + TN - 1 <= tile_row_lo) soft(std::false_type{}, std::false_type{}, g, 0u, 0u, 0);
-                    else soft(std::false_type{}, std::true_type{}, g, nv >= 32 ? 0xffffffffu : (1u << nv) - 1u,
-                              nv >= 32 ? (nv == TN ? 0xffffffffu : (1u << (nv - 32)) - 1u) : 0u, kt * TN);
+                    masked = nv < TN || kt * TN + TN - 1 > tile_row_lo;
                 }
+                const unsigned live_lo = nv >= 32 ? 0xffffffffu : (1u << nv) - 1u;
+                const unsigned live_hi = nv >= TN ? 0xffffffffu : nv > 32 ? (1u << (nv - 32)) - 1u : 0u;
+                // (one call per variant, so that each is expanded in place)
+                if (g >= nA && g < gC) soft(std::true_type{}, std::true_type{}, g, 0u, 0u, FAR_BELOW);
+                else if (masked) soft(std::false_type{}, std::true_type{}, g, live_lo, live_hi, crow0);
+                else soft(std::false_type{}, std::false_type{}, g, 0u, 0u, 0);
             }
             WST_FLUSH;
             // ---- output: o = (O + z) / l for the rows that carry a query
