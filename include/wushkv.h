@@ -408,7 +408,9 @@ int wushkv_set_profile_events(void* start, void* stop);
  *   "wait_limit"        n > 0: poll limit of the device-side barrier waits (default: about a second); 0: default.
  *   "drop_chunk_mma"    1: the chunk append does not commit the MMAs of its first tile to their barrier (same
  *                       failure path in that kernel).
- *   "prefill_legacy"    1: wushkv_prefill_attn runs its mma.sync kernel instead of the tcgen05 one.
+ *   "prefill_legacy"    1: wushkv_prefill_attn runs its mma.sync kernels (attention and transforms) instead of the tcgen05 ones.
+ *   "prefill_one_tile"  1: the chunk attention runs on the tcgen05 kernel with one query tile per CTA and no role split
+ *                       instead of the warp-specialised one.
  *   "prefill_no_tma"    1: the tcgen05 kernel stages the chunk's own tiles with 16-byte copies, not bulk tensor copies.
  *   "append_no_tma"     1: the same for the key / value tiles of the tensor-core chunk append.
  *   "drop_prefill"      1: the tcgen05 chunk attention never commits the score MMAs of a CTA's first tile; 2: it announces

@@ -1105,23 +1105,24 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
 // ------------------------------------------------------------------------------------------------
 // 2c. attention on tcgen05, warp-specialised (the default path)
 // ------------------------------------------------------------------------------------------------
-// One CTA of 384 threads per (sequence, KV head, PAIR of consecutive 128-row query tiles), one CTA per SM.  The
-// three roles run on their own and meet only at mbarriers, so that the tensor pipe computes the scores of the next key
-// tile while the softmax warps work on the current one:
+// One CTA of 512 threads per (sequence, KV head, PAIR of consecutive 128-row query tiles), one CTA per SM.  The
+// roles run on their own and meet only at mbarriers, so that the tensor pipe computes the scores of later key tiles
+// while the softmax warps work on the current one:
 //   warps 0-3 / 4-7   softmax of query tile 0 / 1: thread r owns row r.  Per key tile: wait for S, read the row with
 //                     tcgen05.ld, scale / mask, raise the lazy reference (rescaling the accumulator rows in tensor memory
 //                     only then), write (p Delta_v) as fp16 pairs over the first 32 columns of the score buffer just read,
 //                     arrive on the tile's "probabilities ready" barrier.
-//   warps 8 / 11      issue the tcgen05.mma of query tile 0 / 1 (one lane each): S_t(g+1) = Q'_t K(g+1)^T as soon as the
-//                     key tile has landed, then O_t += P_t(g) V(g) once the probabilities are ready; commits release the
-//                     key / value stages (two arrivals each) and signal the softmax warps.
-//   warps 9-10        stage the key / value tiles into rings of three / two stages: bf16 window rows and packed pages (the
-//                     raw record arrives by a bulk copy one tile ahead and is unpacked into fp16 codes) are written by the
-//                     64 threads, the chunk's own tiles are bulk tensor copies issued by one lane of warp 9 (keys) and
-//                     one of warp 10 (values).
+//   warps 8 / 11      issue the tcgen05.mma of query tile 0 / 1 (one lane each): per key tile g, once the probabilities
+//                     are ready, O_t += P_t(g) V(g) and then S_t(g+2) = Q'_t K(g+2)^T (into the score buffer P_t(g) sat in);
+//                     commits release the key / value stages (two arrivals each) and signal the softmax warps.
+//   warps 9 / 10      one lane each requests the chunk's own key / value tiles (and warp 9 the query tiles) as bulk tensor
+//                     copies into rings of three / two stages.
+//   warps 12-15       write the other key / value tiles into the same rings: bf16 window rows, and packed pages (the raw
+//                     record arrives by a bulk copy one tile ahead and is unpacked into fp16 codes).
+// Registers are moved from warps 8-15 to the softmax warps (setmaxnreg, per group of four warps).
 // Tensor memory (512 columns): query tile t owns columns 256 t .. 256 t + 255: O (128), two score buffers (64 each).
 // Every wait is bounded; a wait that runs out raises a CTA-wide flag that ends all roles.
-constexpr int WS_THREADS = 384;
+constexpr int WS_THREADS = 512;
 constexpr int WS_KS = 3, WS_VS = 2;                              // ring depths of the key / value stages: a bulk tensor copy takes longer than
                                                                  // one tile's MMAs, so a key tile is requested three tiles ahead of its scores
 constexpr int WS_RAW_BYTES = 8704;                               // largest packed record (4 bits)
@@ -1133,7 +1134,7 @@ constexpr int WS_OFF_META = WS_OFF_RAW + 2 * WS_RAW_BYTES;       // uint2[WS_VS]
 constexpr int WS_OFF_LIVE = WS_OFF_META + WS_VS * TN * 8;        // uint2[WS_VS]: which keys of a packed tile exist
 enum { WB_KFULL = 0, WB_KEMPTY = WB_KFULL + WS_KS, WB_VFULL = WB_KEMPTY + WS_KS, WB_VEMPTY = WB_VFULL + WS_VS,
        WB_S = WB_VEMPTY + WS_VS, WB_PV = WB_S + 4, WB_PREADY = WB_PV + 4, WB_RAW = WB_PREADY + 4, WB_Q = WB_RAW + 2,
-       WB_DRAIN, WB_COUNT };
+       WB_STAGED, WB_DRAIN, WB_COUNT };
 constexpr int WS_OFF_BAR = WS_OFF_LIVE + WS_VS * 8;
 constexpr int WS_OFF_MISC = WS_OFF_BAR + WB_COUNT * 8;           // [0] tensor-memory slot, [4] abort flag
 constexpr int WS_SMEM = WS_OFF_MISC + 16;
@@ -1171,10 +1172,10 @@ __device__ __forceinline__ void ws_bulk_g2s(unsigned dst, const void* src, unsig
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-// AND of a predicate over the 64 staging threads (named barrier 1): keeps their give-up decision uniform
+// AND of a predicate over the 128 staging threads (named barrier 1): keeps their give-up decision uniform
 __device__ __forceinline__ bool ws_stagers_and(bool pred) {
     unsigned r;
-    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred p, 1, 64, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred p, 1, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
                  : "=r"(r) : "r"(pred ? 1u : 0u) : "memory");
     return r != 0;
 }
@@ -1229,7 +1230,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
         for (int i = 0; i < WB_COUNT; ++i) {
             // probabilities: the 128 softmax threads of a tile; stage releases: the two issuing warps; queries: one announcement
             // of bulk tensor copies, or warps 0-8 with their 16-byte copies
-            const unsigned count = (i >= WB_PREADY && i < WB_PREADY + 4) ? 128u : i == WB_Q ? (P.use_tma ? 1u : 288u)
+            const unsigned count = (i >= WB_PREADY && i < WB_PREADY + 4) ? 128u : i == WB_Q ? (P.use_tma ? 1u : 256u)
                                  : (i >= WB_KEMPTY && i < WB_KEMPTY + WS_KS) || (i >= WB_VEMPTY && i < WB_VEMPTY + WS_VS) ? 2u : 1u;
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar(i)), "r"(count) : "memory");
         }
@@ -1262,41 +1263,29 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const unsigned tmem_base = *tmem_slot;
-
+    // Registers move from the issuing / copying / staging warps to the softmax warps (per group of four warps; each group
+    // executes its own instruction at the head of its branch, so that the code below it is compiled for the new count).
     // ---- the packed query tiles: row r of tile t = chunk position (2 pr + t) R + r / G, head h G + r % G.  With bulk tensor
     // copies a box of (64 channels, G heads, R positions) lands as R G rows of 128 bytes in exactly that order (128-byte
     // swizzle; rows past the chunk hold zeros or the next sequence's queries and are never stored); otherwise the softmax
     // and MMA warps place 16-byte pieces (rows clamped to the chunk) while the staging warps start on the key side at once.
-    if (P.use_tma) {
-        if (tid == 288) {
-            const unsigned box_bytes = 128u * static_cast<unsigned>(G * R);
-            ws_expect_tx(bar(WB_Q), 4u * box_bytes * ((n_tiles[0] > 0 ? 1u : 0u) + (n_tiles[1] > 0 ? 1u : 0u)));
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                if (n_tiles[q >> 1] == 0) continue;
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf)
-                    tma_load_3d(smem_addr(sm_ws + WS_OFF_Q + q * TC_Q_BYTES + hf * 16384), (q & 1) ? &map_q1 : &map_q0, 64 * hf, h * G,
-                                first + (2 * pr + (q >> 1)) * R, bar(WB_Q));
-            }
-        }
-    } else {
-        for (int item = tid; item < 4 * TM * 16 && warp < 9; item += 288) {
-            const int q = item >> 11, part = q & 1, r = (item >> 4) & (TM - 1), piece = item & 15;
-            const int t = n_rows[q >> 1] > 0 ? (q >> 1) : 0;        // a tile without rows aliases tile 0's (never used)
-            const int rr = min(r, n_rows[t] - 1);
-            const int tok = first + (2 * pr + t) * R + rr / G, jq = h * G + rr % G;
-            const __half* src = P.QP + static_cast<long long>(part) * P.total_new * c.n_q * D + (static_cast<long long>(tok) * c.n_q + jq) * D + 8 * piece;
-            cp16(smem_addr(sm_ws + WS_OFF_Q + q * TC_Q_BYTES + (r >> 3) * 2048 + piece * 128 + (r & 7) * 16), src, 16u);
-        }
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        if (warp < 9) ws_arrive(bar(WB_Q));
-    }
-
     if (warp < 8) {
         // =============================== softmax of query tile t ==========================================
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 184;" ::: "memory");
+        if (!P.use_tma) {
+            for (int item = tid; item < 4 * TM * 16; item += 256) {
+                const int q = item >> 11, part = q & 1, r = (item >> 4) & (TM - 1), piece = item & 15;
+                const int tq = n_rows[q >> 1] > 0 ? (q >> 1) : 0;       // a tile without rows aliases tile 0's (never used)
+                const int rr = min(r, n_rows[tq] - 1);
+                const int tok = first + (2 * pr + tq) * R + rr / G, jq = h * G + rr % G;
+                const __half* src = P.QP + static_cast<long long>(part) * P.total_new * c.n_q * D + (static_cast<long long>(tok) * c.n_q + jq) * D + 8 * piece;
+                cp16(smem_addr(sm_ws + WS_OFF_Q + q * TC_Q_BYTES + (r >> 3) * 2048 + piece * 128 + (r & 7) * 16), src, 16u);
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            ws_arrive(bar(WB_Q));
+        }
         const int t = warp >> 2, wt = tid & 127;
         if (n_tiles[t] > 0) {
             const int qt = 2 * pr + t;
@@ -1437,7 +1426,21 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
             }
         }
     }
-    else if (warp == 8 || warp == 11) {
+    else if (warp < 12) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 56;" ::: "memory");
+      if (P.use_tma && tid == 288) {
+            const unsigned box_bytes = 128u * static_cast<unsigned>(G * R);
+            ws_expect_tx(bar(WB_Q), 4u * box_bytes * ((n_tiles[0] > 0 ? 1u : 0u) + (n_tiles[1] > 0 ? 1u : 0u)));
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (n_tiles[q >> 1] == 0) continue;
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf)
+                    tma_load_3d(smem_addr(sm_ws + WS_OFF_Q + q * TC_Q_BYTES + hf * 16384), (q & 1) ? &map_q1 : &map_q0, 64 * hf, h * G,
+                                first + (2 * pr + (q >> 1)) * R, bar(WB_Q));
+            }
+      }
+      if (warp == 8 || warp == 11) {
         // =============================== MMA issue for query tile t ========================================
         // One issuing warp per query tile: with the 64-key tiles an MMA takes the pipe 48-64 cycles, about what one thread
         // needs to issue it, so a single thread for both tiles left the pipe half idle.
@@ -1516,10 +1519,60 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
         }
         __syncwarp();
         WST_FLUSH;
-    } else {
-        // =============================== staging of key / value tiles =====================================
-        const int ptid = tid - 288;
-        const int n_staged = P.use_tma ? gC : NT;               // tiles written by the 64 threads
+      } else {
+        // =============================== the chunk itself: bulk tensor copies ==============================
+        // Four copies per tile (keys / values x channel halves) of 64 rows x 128 bytes; rows past the end of the chunk read
+        // zeros or the next sequence's rows, both masked by the softmax warps.  Warp 9 requests the key tiles, warp 10 the
+        // value tiles: the two rings advance on their own (a stage is requested once its previous tile was released, which
+        // for the first chunk tiles means: once the staging threads' last tiles went through).
+        int armed[3] = {-1, -1, -1};                            // last tile whose copies this warp announced on each stage
+        bool ok = true;
+        if (P.use_tma && gC > 0) ok = __all_sync(FULLM, ws_wait(bar(WB_STAGED), 0u, wait_limit, abort_flag));
+        if (P.use_tma) {
+            const bool keys = warp == 9;
+            const int depth = keys ? WS_KS : WS_VS, full0 = keys ? WB_KFULL : WB_VFULL, empty0 = keys ? WB_KEMPTY : WB_VEMPTY;
+            const CUtensorMap* map = keys ? &map_k : &map_v;
+            unsigned char* ring = sm_ws + (keys ? WS_OFF_K : WS_OFF_V);
+            WST_DECL;
+            for (int g = gC; g < NT && ok; ++g) {
+                const int st = g % depth, row = first + (g - gC) * TN;
+                WST(0);
+                if (g >= depth && !__all_sync(FULLM, ws_wait(bar(empty0 + st), ((g / depth) - 1) & 1, wait_limit, abort_flag))) { ok = false; break; }
+                WST(1);
+                if (lane == 0) {
+                    ws_expect_tx(bar(full0 + st), TC_K_BYTES);
+#pragma unroll
+                    for (int hf = 0; hf < 2; ++hf)
+                        if (!(P.drop == 2 && keys && g == gC && hf == 0))
+                            tma_load_3d(smem_addr(ring + st * TC_K_BYTES) + hf * 8192, map, 64 * hf, h, row, bar(full0 + st));
+                }
+#pragma unroll
+                for (int i = 0; i < 3; ++i) if (i == st) armed[i] = g;
+#if WUSHKV_WS_TIMING
+                WST(2);
+                ws_wait(bar(full0 + st), (g / depth) & 1, wait_limit, abort_flag);      // measurement only: how long the copies take
+                WST(3);
+#endif
+            }
+            WST_FLUSH;
+            // after a failure elsewhere: give the copies this warp announced a bounded time to land, so that none is
+            // still writing shared memory when the CTA ends
+            if (lane == 0 && *abort_flag) {
+#pragma unroll
+                for (int i = 0; i < 3; ++i)
+                    if (i < depth && armed[i] >= 0)
+                        for (int it = 0; it < 512 && !ws_wait(bar(full0 + i), (armed[i] / depth) & 1, 1, abort_flag); ++it) __nanosleep(2000);
+            }
+        }
+        if (tid == 288 && *abort_flag && P.use_tma)             // the same for the query copies
+            for (int it = 0; it < 512 && !ws_wait(bar(WB_Q), 0u, 1, abort_flag); ++it) __nanosleep(2000);
+      }
+    }
+    else {
+        // =============================== staging of key / value tiles by threads ===========================
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 88;" ::: "memory");
+        const int ptid = tid - 384;
+        const int n_staged = P.use_tma ? gC : NT;               // tiles written by the 128 threads
         int raw_uses[2] = {0, 0};                               // records fetched so far into each raw buffer
         auto page_of = [&](const int gb) -> int {               // page id of packed tile gb, -1 if it cannot be read
             const int pg = page_first + gb;
@@ -1549,7 +1602,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
             mine = __all_sync(FULLM, mine);                     // warp-uniform from here on
             if (g < nA) {
                 // ---- full-precision old positions: sink [0, a_hi) and recent window [c_lo, S0), bf16 rows
-                for (int item = ptid; item < TN * 16 && mine; item += 64) {
+                for (int item = ptid; item < TN * 16 && mine; item += 128) {
                     const int r = item & (TN - 1), piece = item >> 6, idx = g * TN + r;
                     uint4 kh = make_uint4(0, 0, 0, 0), vh = kh;
                     if (idx < n_old_fp) {
@@ -1586,7 +1639,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 if (page_ok) ++raw_uses[rb];
                 const unsigned char* raw = sm_ws + WS_OFF_RAW + rb * WS_RAW_BYTES;
                 const uint4 zero4 = make_uint4(0, 0, 0, 0);
-                for (int item = ptid; item < TN * 16 && mine; item += 64) {
+#pragma unroll 4
+                for (int item = ptid; item < (mine ? TN * 16 : 0); item += 128) {      // independent items: several in flight per thread
                     const int r = item & (TN - 1), kc = item >> 6;
                     const int pos = (page_first + gb) * PAGE_TOKENS + r;
                     const bool live = page_ok && pos >= q_lo && pos < q_hi;
@@ -1595,7 +1649,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                     *reinterpret_cast<uint4*>(sK + (r >> 3) * 2048 + kc * 128 + (r & 7) * 16) = kq;
                     *reinterpret_cast<uint4*>(sV + kc * 1024 + (r >> 3) * 128 + (r & 7) * 16) = vq;
                 }
-                if (mine) {                                     // factors and existence of key ptid (the 64 threads = the 64 keys)
+                if (mine && ptid < TN) {                        // warps 12 and 13: factors and existence of key ptid
                     const int pos = (page_first + gb) * PAGE_TOKENS + ptid;
                     const bool live = page_ok && pos >= q_lo && pos < q_hi;
                     meta_all[vs * TN + ptid] = live ? *reinterpret_cast<const uint2*>(raw + meta_location(BITS, ptid)) : make_uint2(0u, 0u);
@@ -1605,7 +1659,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
             } else {
                 // ---- the chunk's own rows by 16-byte loads (testing aid; bulk tensor copies otherwise)
                 const int kt = g - gC;
-                for (int item = ptid; item < TN * 16 && mine; item += 64) {
+                for (int item = ptid; item < TN * 16 && mine; item += 128) {
                     const int r = item & (TN - 1), piece = item >> 6, row = kt * TN + r;
                     uint4 kh = make_uint4(0, 0, 0, 0), vh = kh;
                     if (row < n_new) {
@@ -1621,48 +1675,10 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
             ok = ws_stagers_and(mine);
             if (ok && ptid == 0) { ws_arrive(bar(WB_KFULL + ks)); ws_arrive(bar(WB_VFULL + vs)); }
         }
-        // ---- the chunk itself: four bulk tensor copies per tile (keys / values x channel halves) of 64 rows x 128 bytes;
-        // rows past the end of the chunk read zeros or the next sequence's rows, both masked by the softmax warps.
-        // Warp 9 requests the key tiles, warp 10 the value tiles: the two rings advance on their own.
-        int armed[3] = {-1, -1, -1};                            // last tile whose copies this warp announced on each stage
-        if (P.use_tma && warp <= 10) {
-            const bool keys = warp == 9;
-            const int depth = keys ? WS_KS : WS_VS, full0 = keys ? WB_KFULL : WB_VFULL, empty0 = keys ? WB_KEMPTY : WB_VEMPTY;
-            const CUtensorMap* map = keys ? &map_k : &map_v;
-            unsigned char* ring = sm_ws + (keys ? WS_OFF_K : WS_OFF_V);
-            WST_DECL;
-            for (int g = gC; g < NT && ok; ++g) {
-                const int st = g % depth, row = first + (g - gC) * TN;
-                WST(0);
-                if (g >= depth && !__all_sync(FULLM, ws_wait(bar(empty0 + st), ((g / depth) - 1) & 1, wait_limit, abort_flag))) { ok = false; break; }
-                WST(1);
-                if (lane == 0) {
-                    ws_expect_tx(bar(full0 + st), TC_K_BYTES);
-#pragma unroll
-                    for (int hf = 0; hf < 2; ++hf)
-                        if (!(P.drop == 2 && keys && g == gC && hf == 0))
-                            tma_load_3d(smem_addr(ring + st * TC_K_BYTES) + hf * 8192, map, 64 * hf, h, row, bar(full0 + st));
-                }
-#pragma unroll
-                for (int i = 0; i < 3; ++i) if (i == st) armed[i] = g;
-#if WUSHKV_WS_TIMING
-                WST(2);
-                ws_wait(bar(full0 + st), (g / depth) & 1, wait_limit, abort_flag);      // measurement only: how long the copies take
-                WST(3);
-#endif
-            }
-            WST_FLUSH;
-            // after a failure elsewhere: give the copies this warp announced a bounded time to land, so that none is
-            // still writing shared memory when the CTA ends
-            if (lane == 0 && *abort_flag) {
-#pragma unroll
-                for (int i = 0; i < 3; ++i)
-                    if (i < depth && armed[i] >= 0)
-                        for (int it = 0; it < 512 && !ws_wait(bar(full0 + i), (armed[i] / depth) & 1, 1, abort_flag); ++it) __nanosleep(2000);
-            }
-        }
-        if (tid == 288 && *abort_flag) {                        // the same for the query and record copies
-            if (P.use_tma) for (int it = 0; it < 512 && !ws_wait(bar(WB_Q), 0u, 1, abort_flag); ++it) __nanosleep(2000);
+        // the copy-issuing warps may start on the chunk's own tiles now: a wait for a stage's release only tells the last two
+        // releases apart, so they must not look at a stage before the tiles staged here have gone through it
+        if (ok && ptid == 0) ws_arrive(bar(WB_STAGED));
+        if (tid == 384 && *abort_flag) {                        // give the record copies a bounded time to land
 #pragma unroll
             for (int i = 0; i < 2; ++i)
                 if (nB > i) for (int it = 0; it < 64 && !ws_wait(bar(WB_RAW + i), raw_uses[i] & 1, 1, abort_flag); ++it) __nanosleep(2000);
