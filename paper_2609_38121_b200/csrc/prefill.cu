@@ -1130,7 +1130,7 @@ constexpr int WS_OFF_Q = 0;                                      // (tile 0 valu
 constexpr int WS_OFF_K = 4 * TC_Q_BYTES;
 constexpr int WS_OFF_V = WS_OFF_K + WS_KS * TC_K_BYTES;
 constexpr int WS_OFF_RAW = WS_OFF_V + WS_VS * TC_K_BYTES;        // two raw records
-constexpr int WS_OFF_META = WS_OFF_RAW + 2 * WS_RAW_BYTES;       // uint2[WS_VS][TN]: per-key factors of a packed tile
+constexpr int WS_OFF_META = WS_OFF_RAW + 2 * WS_RAW_BYTES;       // unsigned[WS_VS][2][TN]: per-key factors of a packed tile (key side, value side)
 constexpr int WS_OFF_LIVE = WS_OFF_META + WS_VS * TN * 8;        // uint2[WS_VS]: which keys of a packed tile exist
 enum { WB_KFULL = 0, WB_KEMPTY = WB_KFULL + WS_KS, WB_VFULL = WB_KEMPTY + WS_KS, WB_VEMPTY = WB_VFULL + WS_VS,
        WB_S = WB_VEMPTY + WS_VS, WB_PV = WB_S + 4, WB_PREADY = WB_PV + 4, WB_RAW = WB_PREADY + 4, WB_Q = WB_RAW + 2,
@@ -1187,8 +1187,8 @@ __device__ __forceinline__ bool ws_stagers_and(bool pred) {
 __device__ unsigned long long g_ws_t[32];
 #define WST_DECL long long wst_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long wst_last = clock64()
 #define WST(slot) do { const long long now = clock64(); wst_acc[slot] += now - wst_last; wst_last = now; } while (0)
-#define WST_FLUSH do { if (blockIdx.x == 0 && blockIdx.y == 0 && lane == 0 && (warp == 0 || warp == 8 || warp == 9)) \
-    for (int i = 0; i < 8; ++i) g_ws_t[(warp == 8 ? 16 : warp == 9 ? 24 : 0) + i] += wst_acc[i]; } while (0)
+#define WST_FLUSH do { if (blockIdx.x == 0 && blockIdx.y == 0 && lane == 0 && (warp == 0 || warp == 8 || warp == 9 || warp == 12)) \
+    for (int i = 0; i < 8; ++i) g_ws_t[(warp == 8 ? 16 : warp == 9 ? 24 : warp == 12 ? 8 : 0) + i] += wst_acc[i]; } while (0)
 #else
 #define WST_DECL
 #define WST(slot) do { } while (0)
@@ -1219,7 +1219,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
     auto bar = [&](int i) -> unsigned { return bar0 + 8u * static_cast<unsigned>(i); };
     unsigned* tmem_slot = reinterpret_cast<unsigned*>(sm_ws + WS_OFF_MISC);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm_ws + WS_OFF_MISC + 4);
-    uint2* meta_all = reinterpret_cast<uint2*>(sm_ws + WS_OFF_META);
+    unsigned* meta_all = reinterpret_cast<unsigned*>(sm_ws + WS_OFF_META);     // [stage][key side, value side][key]: (step, offset) as fp16 pairs
     uint2* live_all = reinterpret_cast<uint2*>(sm_ws + WS_OFF_LIVE);
 
     if (warp == 0) {
@@ -1309,7 +1309,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 // one barrier per score buffer: its next phase (tile g + 2) cannot complete before this tile's probabilities are ready
                 if (!__all_sync(FULLM, ws_wait(bar(WB_S + 2 * t + (g & 1)), (g >> 1) & 1, wait_limit, abort_flag))) { ok = false; return; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint2* meta = meta_all + (g % WS_VS) * TN;
+                const uint4* kmeta = reinterpret_cast<const uint4*>(meta_all + (2 * (g % WS_VS)) * TN);       // four keys per load
+                const uint4* vmeta = kmeta + TN / 4;
                 if (PACKED) {
                     if (!__all_sync(FULLM, ws_wait(bar(WB_VFULL + g % WS_VS), (g / WS_VS) & 1, wait_limit, abort_flag))) { ok = false; return; }
                     const uint2 lv = live_all[g % WS_VS];
@@ -1323,14 +1324,21 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 // below: the maximum is taken of these (three-input max), then scaled once
                 if (PACKED || MASKED) {
 #pragma unroll
-                    for (int j = 0; j < TN; ++j) {
-                        float v = s[j];
-                        if (PACKED) { const float2 mk = h2f2u(meta[j].x); v = fmaf(mk.y, my_qsum, mk.x * v); }
-                        if (MASKED) {
-                            const bool live = ((j < 32 ? live_lo >> j : live_hi >> (j - 32)) & 1u) != 0u;
-                            if (!live || crow0 + j > my_row) v = -INFINITY;
+                    for (int j4 = 0; j4 < TN / 4; ++j4) {
+                        uint4 m4 = make_uint4(0u, 0u, 0u, 0u);
+                        if (PACKED) m4 = kmeta[j4];
+                        const unsigned mw[4] = {m4.x, m4.y, m4.z, m4.w};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const int j = 4 * j4 + q;
+                            float v = s[j];
+                            if (PACKED) { const float2 mk = h2f2u(mw[q]); v = fmaf(mk.y, my_qsum, mk.x * v); }
+                            if (MASKED) {
+                                const bool live = ((j < 32 ? live_lo >> j : live_hi >> (j - 32)) & 1u) != 0u;
+                                if (!live || crow0 + j > my_row) v = -INFINITY;
+                            }
+                            s[j] = v;
                         }
-                        s[j] = v;
                     }
                 }
                 float mx_raw = fmaxf(s[0], s[1]);
@@ -1365,16 +1373,22 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 for (int half = 0; half < 2; ++half) {                     // 32 keys = 16 columns of fp16 pairs at a time
                     unsigned pk[16];
 #pragma unroll
-                    for (int e16 = 0; e16 < 16; ++e16) {
-                        const int e = 16 * half + e16;
-                        float2 pr = make_float2(fast_ex2(fmaf(s[2 * e], k2, -ref)), fast_ex2(fmaf(s[2 * e + 1], k2, -ref)));     // k2 s - ref in one rounding
-                        lsum.x += pr.x; lsum.y += pr.y;
-                        if (PACKED) {
-                            const float2 mv0 = h2f2u(meta[2 * e].y), mv1 = h2f2u(meta[2 * e + 1].y);
-                            z = fmaf(pr.x, mv0.y, fmaf(pr.y, mv1.y, z));
-                            pr.x *= mv0.x; pr.y *= mv1.x;
+                    for (int e4 = 0; e4 < 8; ++e4) {                       // four keys = two fp16 pairs at a time
+                        uint4 m4 = make_uint4(0u, 0u, 0u, 0u);
+                        if (PACKED) m4 = vmeta[8 * half + e4];
+                        const unsigned mw[4] = {m4.x, m4.y, m4.z, m4.w};
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) {
+                            const int e = 16 * half + 2 * e4 + q;
+                            float2 pr = make_float2(fast_ex2(fmaf(s[2 * e], k2, -ref)), fast_ex2(fmaf(s[2 * e + 1], k2, -ref)));     // k2 s - ref in one rounding
+                            lsum.x += pr.x; lsum.y += pr.y;
+                            if (PACKED) {
+                                const float2 mv0 = h2f2u(mw[2 * q]), mv1 = h2f2u(mw[2 * q + 1]);
+                                z = fmaf(pr.x, mv0.y, fmaf(pr.y, mv1.y, z));
+                                pr.x *= mv0.x; pr.y *= mv1.x;
+                            }
+                            pk[2 * e4 + q] = pack_half2(pr.x, pr.y);
                         }
-                        pk[e16] = pack_half2(pr.x, pr.y);
                     }
                     tc_st16u(sbuf + 16 * half, pk);
                 }
@@ -1482,39 +1496,59 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
             else scores_of(std::false_type{}, g, st);
             return true;
         };
-        auto key_landed = [&](const int g) -> bool { return ws_wait(bar(WB_KFULL + g % WS_KS), (g / WS_KS) & 1, wait_limit, abort_flag); };
-        auto value_landed = [&](const int g) -> bool { return ws_wait(bar(WB_VFULL + g % WS_VS), (g / WS_VS) & 1, wait_limit, abort_flag); };
+        // Two streams of work, each in tile order: the scores S_t(sc) (once the key tile has landed and O += P V of tile
+        // sc - 2, which reads the probabilities out of the same score buffer, has been issued) and the products O_t += P_t(pv)
+        // V(pv) (once the value tile has landed and the probabilities are ready).  Neither may wait for the other: a key tile
+        // written by the staging threads arrives together with its value tile, whose stage only the product of two tiles
+        // before releases.  So the thread tests the barriers and issues whatever is ready.
+        auto landed = [&](const int full0, const int depth, const int g) -> bool {
+            unsigned ready;
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                         : "=r"(ready) : "r"(bar(full0 + g % depth)), "r"(static_cast<unsigned>((g / depth) & 1)) : "memory");
+            return ready != 0;
+        };
         if (lane == 0 && ok) {
-            ok = key_landed(0) && scores(0);
-            if (ok && NT > 1) ok = key_landed(1) && scores(1);
-            if (ok) ok = value_landed(0);
-            WST(1);
-            for (int g = 0; g < NT && ok; ++g) {
-                const int st = g % WS_VS;
-                if (g < mine) {
-                    if (!ws_wait(bar(WB_PREADY + 2 * t + (g & 1)), (g >> 1) & 1, wait_limit, abort_flag)) { ok = false; break; }
-                    WST(2);
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const bool swz = g >= gC && P.use_tma;
-                    // swizzled values: rows (keys) of 128 bytes, 8-key groups 1024 bytes apart, channel halves 8192 bytes apart: 16 keys = 2048 bytes
-                    const unsigned long long vb = (swz ? v_swz0 : v_plain0) + static_cast<unsigned>(st * (TC_K_BYTES >> 4));
-                    const unsigned vstep = swz ? (2048u >> 4) : (256u >> 4);
-                    const unsigned prob = acc_o + 128u + 64u * (g & 1);
+            int sc = 0, pv = 0, idle = 0;
+            while (pv < NT) {
+                bool progressed = false;
+                if (pv < sc && landed(WB_VFULL, WS_VS, pv)) {
+                    const int st = pv % WS_VS;
+                    if (pv >= mine) {                           // a tile only the other query tile reads: just release the stage
+                        ws_arrive(bar(WB_VEMPTY + st));
+                        ++pv; progressed = true;
+                    } else {
+                        unsigned ready;
+                        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                                     : "=r"(ready) : "r"(bar(WB_PREADY + 2 * t + (pv & 1))), "r"(static_cast<unsigned>((pv >> 1) & 1)) : "memory");
+                        if (ready) {
+                            WST(2);
+                            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                            const bool swz = pv >= gC && P.use_tma;
+                            // swizzled values: rows (keys) of 128 bytes, 8-key groups 1024 bytes apart, channel halves 8192 bytes apart: 16 keys = 2048 bytes
+                            const unsigned long long vb = (swz ? v_swz0 : v_plain0) + static_cast<unsigned>(st * (TC_K_BYTES >> 4));
+                            const unsigned vstep = swz ? (2048u >> 4) : (256u >> 4);
+                            const unsigned prob = acc_o + 128u + 64u * (pv & 1);
 #pragma unroll
-                    for (int ks = 0; ks < TN / 16; ++ks)
-                        tc_mma_ts(acc_o, prob + 8 * ks, vb + ks * vstep, TC_IDESC_O, (g > 0 || ks > 0) ? 1u : 0u);
-                    ws_commit(bar(WB_PV + 2 * t + (g & 1)));
-                    ws_commit(bar(WB_VEMPTY + st));
-                } else {
-                    ws_arrive(bar(WB_VEMPTY + st));
+                            for (int ks = 0; ks < TN / 16; ++ks)
+                                tc_mma_ts(acc_o, prob + 8 * ks, vb + ks * vstep, TC_IDESC_O, (pv > 0 || ks > 0) ? 1u : 0u);
+                            ws_commit(bar(WB_PV + 2 * t + (pv & 1)));
+                            ws_commit(bar(WB_VEMPTY + st));
+                            ++pv; progressed = true;
+                            WST(3);
+                        }
+                    }
                 }
-                WST(3);
-                // (a key tile written by the staging threads comes together with its value tile, whose stage the product
-                // just issued releases: its arrival cannot be awaited any earlier than here)
-                if (g + 2 < NT) { if (!key_landed(g + 2)) { ok = false; break; } scores(g + 2); }
-                WST(4);
-                if (g + 1 < NT && !value_landed(g + 1)) { ok = false; break; }
-                WST(5);
+                if (sc < NT && sc < pv + 2 && landed(WB_KFULL, WS_KS, sc)) {
+                    WST(6);
+                    scores(sc);
+                    ++sc; progressed = true;
+                    WST(4);
+                }
+                if (progressed) { idle = 0; continue; }
+                // nothing ready: a short pause keeps the polls off the softmax warps' issue slots; bounded like every wait
+                __nanosleep(40);
+                if (++idle >= wait_limit) { *abort_flag = 1; ok = false; break; }
+                if ((idle & 7) == 7 && *abort_flag) { ok = false; break; }
             }
         }
         __syncwarp();
@@ -1592,14 +1626,18 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
         };
         if (nB > 0 && ptid == 0) fetch_record(0);
         bool ok = true;
+        WST_DECL;
         for (int g = 0; g < n_staged && ok; ++g) {
+            WST(0);
             const int ks = g % WS_KS, vs = g % WS_VS;
             unsigned char* sK = sm_ws + WS_OFF_K + ks * TC_K_BYTES;
             unsigned char* sV = sm_ws + WS_OFF_V + vs * TC_K_BYTES;
             bool mine = true;
             if (g >= WS_KS) mine = ws_wait(bar(WB_KEMPTY + ks), ((g / WS_KS) - 1) & 1, wait_limit, abort_flag);
+            WST(4);
             if (mine && g >= WS_VS) mine = ws_wait(bar(WB_VEMPTY + vs), ((g / WS_VS) - 1) & 1, wait_limit, abort_flag);
             mine = __all_sync(FULLM, mine);                     // warp-uniform from here on
+            WST(1);
             if (g < nA) {
                 // ---- full-precision old positions: sink [0, a_hi) and recent window [c_lo, S0), bf16 rows
                 for (int item = ptid; item < TN * 16 && mine; item += 128) {
@@ -1652,7 +1690,9 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 if (mine && ptid < TN) {                        // warps 12 and 13: factors and existence of key ptid
                     const int pos = (page_first + gb) * PAGE_TOKENS + ptid;
                     const bool live = page_ok && pos >= q_lo && pos < q_hi;
-                    meta_all[vs * TN + ptid] = live ? *reinterpret_cast<const uint2*>(raw + meta_location(BITS, ptid)) : make_uint2(0u, 0u);
+                    const uint2 m = live ? *reinterpret_cast<const uint2*>(raw + meta_location(BITS, ptid)) : make_uint2(0u, 0u);
+                    meta_all[(2 * vs) * TN + ptid] = m.x;
+                    meta_all[(2 * vs + 1) * TN + ptid] = m.y;
                     const unsigned word = __ballot_sync(FULLM, live);
                     if (lane == 0) reinterpret_cast<unsigned*>(live_all + vs)[ptid >> 5] = word;
                 }
@@ -1671,12 +1711,15 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                     *reinterpret_cast<uint4*>(sV + piece * 1024 + (r >> 3) * 128 + (r & 7) * 16) = vh;
                 }
             }
+            WST(2);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             ok = ws_stagers_and(mine);
+            WST(3);
             if (ok && ptid == 0) { ws_arrive(bar(WB_KFULL + ks)); ws_arrive(bar(WB_VFULL + vs)); }
         }
         // the copy-issuing warps may start on the chunk's own tiles now: a wait for a stage's release only tells the last two
         // releases apart, so they must not look at a stage before the tiles staged here have gone through it
+        WST_FLUSH;
         if (ok && ptid == 0) ws_arrive(bar(WB_STAGED));
         if (tid == 384 && *abort_flag) {                        // give the record copies a bounded time to land
 #pragma unroll
@@ -2023,7 +2066,7 @@ static int prefill_attn_impl(const wushkv_cache* cache, int32_t batch, const int
                 unsigned long long t[32];
                 cudaMemcpyFromSymbol(t, g_ws_t, sizeof(t));
                 std::fprintf(stderr, "ws timing softmax:");
-                for (int i = 0; i < 8; ++i) std::fprintf(stderr, " %llu", t[i]);
+                for (int i = 0; i < 16; ++i) std::fprintf(stderr, " %llu", t[i]);
                 std::fprintf(stderr, "\nws timing mma:");
                 for (int i = 16; i < 32; ++i) std::fprintf(stderr, " %llu", t[i]);
                 std::fprintf(stderr, "\n");
