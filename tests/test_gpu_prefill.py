@@ -50,6 +50,18 @@ def test_chunk_over_a_quantized_cache(bits, n_q, n_kv):
     assert L.cache.status() == 0
 
 
+@pytest.mark.parametrize("n_q,n_kv", [(2, 2), (6, 2), (5, 1), (12, 2), (16, 2)])
+def test_head_group_sizes(n_q, n_kv):
+    """G = 1, 3, 5, 6 and 8 query heads per KV head: a 128-row tile packs 128 / G chunk positions, which leaves rows
+    unused when G does not divide 128, and a pair of tiles may end inside the chunk or be half empty; a chunk over a
+    short quantized cache, ragged batch."""
+    wl = _wl(n_q, n_kv, seed=96, batch=2)
+    L = Layer(wl, [500, 310], 2, 4, 64, 8)
+    L.append_step([300, 190])
+    assert L.check_prefill_parity([200, 120]) <= 2e-3
+    assert L.cache.status() == 0
+
+
 def test_chunk_shorter_than_the_recent_window_and_second_chunk():
     """Chunks of 16 tokens as in the paper's perplexity runs (S_sink 16, S_keep 128, S_flush 16): old recent-window
     rows come from the ring, the quantized boundary sits below the chunk; two chunks in a row."""
