@@ -1761,7 +1761,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
 //   warps 0-15  a thread owns 32 channels of one token of the tile (one warp alone per scheduler spends its time on
 //            instruction latency): tcgen05.ld, the roundings (k' through bf16 to fp16; q' as fp16 value + fp16 remainder,
 //            and their sum over the channels); the rows go through a shared-memory tile so that the stores to global memory
-//            are whole 256-byte rows.  Key-head CTAs also convert the chunk's values.
+//            are whole 256-byte rows.
+// Head slots past the query heads convert the chunk's values of one KV head to fp16 (plain loads and stores).
 // Barriers come in pairs (one per ring slot), every wait is bounded.
 constexpr int PT_THREADS = 576;                                  // warps 0-15 epilogue, 16 copies, 17 MMA issue
 constexpr int PT_OFF_T = 0;                                      // three terms of 128 x 128 bf16, K-major core matrices
@@ -1777,21 +1778,60 @@ constexpr int PT_SMEM = PT_OFF_MISC + 16;
 constexpr unsigned PT_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((static_cast<unsigned>(D) >> 3) << 17) | ((static_cast<unsigned>(PREP_TOK) >> 4) << 24);   // fp32 <- bf16 x bf16, K-major
 static_assert(PT_OFF_X % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 
+#if WUSHKV_WS_TIMING
+#define PST_DECL long long pst_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long pst_last = clock64()
+#define PST(slot) do { const long long now = clock64(); pst_acc[slot] += now - pst_last; pst_last = now; } while (0)
+#define PST_FLUSH(base) do { if (blockIdx.x == 0 && blockIdx.y == gridDim.y - 1 && lane == 0) for (int i_ = 0; i_ < 8; ++i_) g_ws_t[(base) + i_] += pst_acc[i_]; } while (0)
+#else
+#define PST_DECL
+#define PST(slot) do { } while (0)
+#define PST_FLUSH(base) do { } while (0)
+#endif
 __global__ void __launch_bounds__(PT_THREADS, 1) prefill_prep_tc_kernel(PrefillParams P, const __grid_constant__ CUtensorMap map_k,
                                                                         const __grid_constant__ CUtensorMap map_q) {
     extern __shared__ __align__(1024) unsigned char sm_pt[];
     const int hs = blockIdx.y;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (hs >= P.c.n_kv + P.c.n_q) {
+        // head slots past the query heads: the chunk's values of one KV head as fp16 (no transform), 16-byte pieces, four
+        // loads in flight per thread; the CTAs of a slot take interleaved 128-token tiles like the others
+        const int vh = hs - P.c.n_kv - P.c.n_q;
+        for (int tok0 = static_cast<int>(blockIdx.x) * PREP_TOK; tok0 < P.total_new; tok0 += static_cast<int>(gridDim.x) * PREP_TOK) {
+            uint4 v[4];
+            long long off[4];
+            bool in[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int item = tid + k * PT_THREADS, r = item >> 4, piece = item & 15;
+                in[k] = item < PREP_TOK * 16 && tok0 + r < P.total_new;
+                off[k] = (static_cast<long long>(tok0 + r) * P.c.n_kv + vh) * D + 8 * piece;
+                if (in[k]) v[k] = __ldg(reinterpret_cast<const uint4*>(P.V_new + off[k]));
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (!in[k]) continue;
+                const unsigned w[4] = {v[k].x, v[k].y, v[k].z, v[k].w};
+                unsigned o[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) o[e] = pack_half2(bf16_bits_to_float(w[e] & 0xffff), bf16_bits_to_float(w[e] >> 16));
+                *reinterpret_cast<uint4*>(P.VP + off[k]) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        }
+        return;
+    }
     const bool is_key = hs < P.c.n_kv;
     const int head = is_key ? hs : hs - P.c.n_kv;
     const int kvh = is_key ? head : head / P.c.G;
     const int n_terms = is_key ? 1 : 3;
     const int n_heads = is_key ? P.c.n_kv : P.c.n_q;
     const float* T = (is_key ? P.c.T_K : P.c.T_K_invT) + static_cast<long long>(kvh) * D * D;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned bar0 = smem_addr(sm_pt + PT_OFF_BAR);
     auto bar = [&](int i) -> unsigned { return bar0 + 8u * static_cast<unsigned>(i); };
     unsigned* tmem_slot = reinterpret_cast<unsigned*>(sm_pt + PT_OFF_MISC);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm_pt + PT_OFF_MISC + 4);
+#if WUSHKV_WS_TIMING
+    const long long t_entry = clock64();
+#endif
     const int n_my_tiles = (P.total_new + PREP_TOK - 1) / PREP_TOK > static_cast<int>(blockIdx.x)
                                ? ((P.total_new + PREP_TOK - 1) / PREP_TOK - 1 - static_cast<int>(blockIdx.x)) / static_cast<int>(gridDim.x) + 1 : 0;
     if (n_my_tiles == 0) return;
@@ -1828,6 +1868,9 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_prep_tc_kernel(PrefillP
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const unsigned tmem_base = *tmem_slot;
     const int wait_limit = P.wait_limit > 0 ? P.wait_limit : (1 << 24);
+#if WUSHKV_WS_TIMING
+    if (tid == 0 && blockIdx.x == 0 && blockIdx.y == gridDim.y - 1) g_ws_t[8] += clock64() - t_entry;
+#endif
 
     if (warp == 16) {
         // ---- token tiles
@@ -1855,10 +1898,14 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_prep_tc_kernel(PrefillP
         if (lane == 0) {
             const unsigned long long t_desc = tc_desc(smem_addr(sm_pt + PT_OFF_T), 128, 2048);
             const unsigned long long x_desc = tc_desc_sw128(smem_addr(sm_pt + PT_OFF_X), 16, 1024);
+            PST_DECL;
             for (int i = 0; i < n_my_tiles; ++i) {
                 const int s = i & 1;
+                PST(0);
                 if (!ws_wait(bar(PB_XFULL + s), (i >> 1) & 1, wait_limit, abort_flag)) break;
+                PST(1);
                 if (i >= 2 && !ws_wait(bar(PB_DEMPTY + s), ((i >> 1) - 1) & 1, wait_limit, abort_flag)) break;
+                PST(2);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const unsigned acc = tmem_base + 128u * s;
                 for (int term = 0; term < n_terms; ++term) {
@@ -1869,7 +1916,9 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_prep_tc_kernel(PrefillP
                 }
                 ws_commit(bar(PB_DFULL + s));
                 ws_commit(bar(PB_XEMPTY + s));
+                PST(3);
             }
+            PST_FLUSH(16);
         }
         __syncwarp();
     } else {
@@ -1880,22 +1929,10 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_prep_tc_kernel(PrefillP
         const long long lo_off = static_cast<long long>(P.total_new) * n_heads * D;
         float* qs_part = reinterpret_cast<float*>(sm_pt + PT_OFF_QS);      // [4][128] partial channel sums
         bool ok = true;
+        PST_DECL;
         for (int i = 0; i < n_my_tiles && ok; ++i) {
             const int s = i & 1, tok0 = (static_cast<int>(blockIdx.x) + i * static_cast<int>(gridDim.x)) * PREP_TOK;
-            if (is_key) {                                       // the chunk's values as fp16 (no transform); coalesced 16-byte pieces
-                for (int item = tid; item < PREP_TOK * 16; item += EPI) {
-                    const int r = item >> 4, piece = item & 15;
-                    if (tok0 + r < P.total_new) {
-                        const long long off = (static_cast<long long>(tok0 + r) * P.c.n_kv + head) * D + 8 * piece;
-                        const uint4 v = __ldg(reinterpret_cast<const uint4*>(P.V_new + off));
-                        const unsigned w[4] = {v.x, v.y, v.z, v.w};
-                        unsigned o[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) o[e] = pack_half2(bf16_bits_to_float(w[e] & 0xffff), bf16_bits_to_float(w[e] >> 16));
-                        *reinterpret_cast<uint4*>(P.VP + off) = make_uint4(o[0], o[1], o[2], o[3]);
-                    }
-                }
-            }
+            PST(0);
             {   // the give-up decision is taken by the 512 epilogue threads together (they meet at named barriers below)
                 const unsigned got = ws_wait(bar(PB_DFULL + s), (i >> 1) & 1, wait_limit, abort_flag) ? 1u : 0u;
                 unsigned all;
@@ -1903,6 +1940,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_prep_tc_kernel(PrefillP
                              : "=r"(all) : "r"(got) : "memory");
                 if (!all) { ok = false; break; }
             }
+            PST(1);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             float o[32];
             tc_ld32(tmem_row + 128u * s, o);
@@ -1939,17 +1977,24 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_prep_tc_kernel(PrefillP
                 asm volatile("bar.sync 2, 512;" ::: "memory");
             };
             if (!is_key) qs_part[cq * PREP_TOK + row] = sum;
+            PST(2);
             flush(hi, is_key ? P.KP : P.QP);
+            PST(3);
             if (!is_key) {
                 flush(lo, P.QP + lo_off);
+                PST(4);
                 if (cq == 0 && tok0 + row < P.total_new)
                     P.qsum[static_cast<long long>(tok0 + row) * P.c.n_q + head] =
                         (qs_part[row] + qs_part[PREP_TOK + row]) + (qs_part[2 * PREP_TOK + row] + qs_part[3 * PREP_TOK + row]);
             }
         }
+        if (warp == 0) PST_FLUSH(0);
     }
 
     __syncthreads();
+#if WUSHKV_WS_TIMING
+    if (tid == 0 && blockIdx.x == 0 && blockIdx.y == gridDim.y - 1) g_ws_t[9] += clock64() - t_entry;
+#endif
     if (*abort_flag && tid == 544) {                            // the issuing thread: let whatever was issued finish (bounded) before the release
         atomicOr(P.c.dev_status, WUSHKV_DEV_COPY_TIMEOUT);
         ws_commit(bar(PB_DRAIN));
@@ -2031,7 +2076,24 @@ static int prefill_attn_impl(const wushkv_cache* cache, int32_t batch, const int
                              make_row_tensor_map(in_k, true, K_new, P.c.n_kv, total_new, PREP_TOK) &&
                              make_row_tensor_map(in_q, true, Q_new, P.c.n_q, total_new, PREP_TOK) &&
                              opt_in_dynamic_smem(reinterpret_cast<const void*>(prefill_prep_tc_kernel), PT_SMEM);
-        if (tc_prep) prefill_prep_tc_kernel<<<dim3(per_slot, slots), PT_THREADS, PT_SMEM, st>>>(P, in_k, in_q);
+        if (tc_prep) {      // head slots: key heads, query heads, then one per KV head for the values
+            const int slots_tc = slots + P.c.n_kv, per_slot_tc = std::max(1, std::min(n_tok_tiles, sm_count() / slots_tc));
+            prefill_prep_tc_kernel<<<dim3(per_slot_tc, slots_tc), PT_THREADS, PT_SMEM, st>>>(P, in_k, in_q);
+        }
+#if WUSHKV_WS_TIMING
+        if (tc_prep) {
+            cudaDeviceSynchronize();
+            unsigned long long t[32];
+            cudaMemcpyFromSymbol(t, g_ws_t, sizeof(t));
+            std::fprintf(stderr, "prep timing epilogue:");
+            for (int i = 0; i < 10; ++i) std::fprintf(stderr, " %llu", t[i]);
+            std::fprintf(stderr, "\nprep timing mma:");
+            for (int i = 16; i < 24; ++i) std::fprintf(stderr, " %llu", t[i]);
+            std::fprintf(stderr, "\n");
+            std::memset(t, 0, sizeof(t));
+            cudaMemcpyToSymbol(g_ws_t, t, sizeof(t));
+        }
+#endif
         else prefill_prep_kernel<<<dim3(per_slot, slots), 256, smem_prep, st>>>(P);
     }
     if (cudaGetLastError() != cudaSuccess) return WUSHKV_ECUDA;
