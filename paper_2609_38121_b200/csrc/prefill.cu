@@ -726,6 +726,64 @@ __device__ __forceinline__ void unpack_chunk8(const unsigned char* raw, int r, i
     vout = make_uint4(vo[0], vo[1], vo[2], vo[3]);
 }
 
+// A whole 2-bit page (all 64 tokens live) as fp16 integer codes, by 128 threads: instead of gathering eight channels of a
+// token from 16-bit loads (unpack_chunk8), a thread reads the record the way it is laid out and scatters 16-byte chunks.
+//   keys:   thread (block bi, k-step s, fragment row g) loads the four 16-byte pieces of row g (fragment lanes t = 0..3: words
+//           j = rs + 2 hh, bytes b = 2 b1 + b0, field s of a byte = channel 32 s + 16 hh + 8 b1 + 2 t + b0 of token g + 8 rs)
+//           and writes, for (rs, hh, b1), the chunk of channels 8 (4 s + 2 hh + b1) .. + 7 of that token: pair t = (b0 0, 1).
+//   values: thread (block bi, word m = 2 ps + rsel, half ih of the channel blocks, token pair tt) loads word m of the eight
+//           pieces (e, tt) (half-word hi = token 8 ps + 2 tt + hi, field i = channel 16 i + 8 rsel + e) and writes, for
+//           (hi, i in 4 ih .. 4 ih + 3), the chunk of channels 8 (2 i + rsel) .. + 7 of that token: element e.
+__device__ __forceinline__ void unpack_page2(const unsigned char* raw, unsigned char* sK, unsigned char* sV, const int p) {
+    const __half2 bias = __halves2half2(__ushort_as_half(0x6400), __ushort_as_half(0x6400));
+    auto to_h2 = [&](const unsigned pair) {             // two codes (bits 0-1 and 16-17) -> fp16 pair: 1024 + c, minus 1024
+        const unsigned w = pair | 0x64006400u;
+        const __half2 hv = __hsub2(*reinterpret_cast<const __half2*>(&w), bias);
+        return *reinterpret_cast<const unsigned*>(&hv);
+    };
+    {
+        const int g = p & 7, s = (p >> 3) & 3, bi = p >> 5;
+        unsigned w[4][4];                                   // [t][j]
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const uint4 v = *reinterpret_cast<const uint4*>(raw + bi * 512 + 64 * g + 16 * t);
+            w[t][0] = v.x; w[t][1] = v.y; w[t][2] = v.z; w[t][3] = v.w;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {                       // j = rs + 2 hh
+#pragma unroll
+            for (int b1 = 0; b1 < 2; ++b1) {
+                unsigned out[4];
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const unsigned x = w[t][j] >> (16 * b1 + 2 * s);
+                    out[t] = to_h2((x & 3u) | ((x << 8) & 0x00030000u));
+                }
+                *reinterpret_cast<uint4*>(sK + (2 * bi + (j & 1)) * 2048 + (4 * s + 2 * (j >> 1) + b1) * 128 + g * 16) =
+                    make_uint4(out[0], out[1], out[2], out[3]);
+            }
+        }
+    }
+    {
+        const int tt = p & 3, ih = (p >> 2) & 1, m = (p >> 3) & 3, bi = p >> 5, ps = m >> 1, rsel = m & 1;
+        unsigned w[8];                                      // [e]
+#pragma unroll
+        for (int e = 0; e < 8; ++e) w[e] = *reinterpret_cast<const unsigned*>(raw + v_codes_offset(2) + bi * 512 + 16 * (4 * e + tt) + 4 * m);
+#pragma unroll
+        for (int hi = 0; hi < 2; ++hi) {
+#pragma unroll
+            for (int ii = 0; ii < 4; ++ii) {
+                const int i = 4 * ih + ii, sh = 16 * hi + 2 * i;
+                unsigned out[4];
+#pragma unroll
+                for (int e2 = 0; e2 < 4; ++e2) out[e2] = to_h2(((w[2 * e2] >> sh) & 3u) | (((w[2 * e2 + 1] >> sh) & 3u) << 16));
+                *reinterpret_cast<uint4*>(sV + (2 * i + rsel) * 1024 + (2 * bi + ps) * 128 + (2 * tt + hi) * 16) =
+                    make_uint4(out[0], out[1], out[2], out[3]);
+            }
+        }
+    }
+}
+
 template <int BITS>
 __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P, const __grid_constant__ CUtensorMap map_k,
                                                                  const __grid_constant__ CUtensorMap map_v) {
@@ -1677,8 +1735,11 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 if (page_ok) ++raw_uses[rb];
                 const unsigned char* raw = sm_ws + WS_OFF_RAW + rb * WS_RAW_BYTES;
                 const uint4 zero4 = make_uint4(0, 0, 0, 0);
+                const int page_pos = (page_first + gb) * PAGE_TOKENS;
+                const bool whole = BITS == 2 && page_ok && page_pos >= q_lo && page_pos + PAGE_TOKENS <= q_hi;
+                if (whole && mine) unpack_page2(raw, sK, sV, ptid);
 #pragma unroll 4
-                for (int item = ptid; item < (mine ? TN * 16 : 0); item += 128) {      // independent items: several in flight per thread
+                for (int item = ptid; item < (mine && !whole ? TN * 16 : 0); item += 128) {      // first / last page, other widths
                     const int r = item & (TN - 1), kc = item >> 6;
                     const int pos = (page_first + gb) * PAGE_TOKENS + r;
                     const bool live = page_ok && pos >= q_lo && pos < q_hi;
