@@ -1380,7 +1380,16 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 WST(2);
                 // scores before the common factor k2 = scale * log2(e) > 0, which is folded into the exponent's multiply-add
                 // below: the maximum is taken of these (three-input max), then scaled once
-                if (PACKED || MASKED) {
+                // (a packed page inside the quantized range has all its keys, and all of them lie below the chunk: no mask)
+                if (PACKED && (live_lo & live_hi) == 0xffffffffu) {
+#pragma unroll
+                    for (int j4 = 0; j4 < TN / 4; ++j4) {
+                        const uint4 m4 = kmeta[j4];
+                        const unsigned mw[4] = {m4.x, m4.y, m4.z, m4.w};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) { const float2 mk = h2f2u(mw[q]); s[4 * j4 + q] = fmaf(mk.y, my_qsum, mk.x * s[4 * j4 + q]); }
+                    }
+                } else if (PACKED || MASKED) {
 #pragma unroll
                     for (int j4 = 0; j4 < TN / 4; ++j4) {
                         uint4 m4 = make_uint4(0u, 0u, 0u, 0u);
