@@ -1174,15 +1174,15 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
 //                     are ready, O_t += P_t(g) V(g) and then S_t(g+2) = Q'_t K(g+2)^T (into the score buffer P_t(g) sat in);
 //                     commits release the key / value stages (two arrivals each) and signal the softmax warps.
 //   warps 9 / 10      one lane each requests the chunk's own key / value tiles (and warp 9 the query tiles) as bulk tensor
-//                     copies into rings of three / two stages.
+//                     copies into rings of two / three stages.
 //   warps 12-15       write the other key / value tiles into the same rings: bf16 window rows, and packed pages (the raw
 //                     record arrives by a bulk copy one tile ahead and is unpacked into fp16 codes).
 // Registers are moved from warps 8-15 to the softmax warps (setmaxnreg, per group of four warps).
 // Tensor memory (512 columns): query tile t owns columns 256 t .. 256 t + 255: O (128), two score buffers (64 each).
 // Every wait is bounded; a wait that runs out raises a CTA-wide flag that ends all roles.
 constexpr int WS_THREADS = 512;
-constexpr int WS_KS = 3, WS_VS = 2;                              // ring depths of the key / value stages: a bulk tensor copy takes longer than
-                                                                 // one tile's MMAs, so a key tile is requested three tiles ahead of its scores
+constexpr int WS_KS = 2, WS_VS = 3;                              // ring depths of the key / value stages: a key stage is free again when
+                                                                 // its scores are done, a value stage only after O += P V a softmax later
 constexpr int WS_RAW_BYTES = 8704;                               // largest packed record (4 bits)
 constexpr int WS_OFF_Q = 0;                                      // (tile 0 value, remainder), (tile 1 value, remainder)
 constexpr int WS_OFF_K = 4 * TC_Q_BYTES;
@@ -1626,7 +1626,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
         // zeros or the next sequence's rows, both masked by the softmax warps.  Warp 9 requests the key tiles, warp 10 the
         // value tiles: the two rings advance on their own (a stage is requested once its previous tile was released, which
         // for the first chunk tiles means: once the staging threads' last tiles went through).
-        int armed[3] = {-1, -1, -1};                            // last tile whose copies this warp announced on each stage
+        int armed[3] = {-1, -1, -1};                            // last tile whose copies this warp announced on each stage (<= 3 stages)
         bool ok = true;
         if (P.use_tma && gC > 0) ok = __all_sync(FULLM, ws_wait(bar(WB_STAGED), 0u, wait_limit, abort_flag));
         if (P.use_tma) {
