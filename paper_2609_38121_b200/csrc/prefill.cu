@@ -726,28 +726,41 @@ __device__ __forceinline__ void unpack_chunk8(const unsigned char* raw, int r, i
     vout = make_uint4(vo[0], vo[1], vo[2], vo[3]);
 }
 
-// A whole 2-bit page (all 64 tokens live) as fp16 integer codes, by 128 threads: instead of gathering eight channels of a
-// token from 16-bit loads (unpack_chunk8), a thread reads the record the way it is laid out and scatters 16-byte chunks.
+// A whole page (all 64 tokens live) as fp16 integer codes, by 128 threads: instead of gathering eight channels of a token
+// from 16-bit loads (unpack_chunk8), a thread reads the record the way it is laid out and scatters 16-byte chunks.
 //   keys:   thread (block bi, k-step s, fragment row g) loads the four 16-byte pieces of row g (fragment lanes t = 0..3: words
-//           j = rs + 2 hh, bytes b = 2 b1 + b0, field s of a byte = channel 32 s + 16 hh + 8 b1 + 2 t + b0 of token g + 8 rs)
-//           and writes, for (rs, hh, b1), the chunk of channels 8 (4 s + 2 hh + b1) .. + 7 of that token: pair t = (b0 0, 1).
-//   values: thread (block bi, word m = 2 ps + rsel, half ih of the channel blocks, token pair tt) loads word m of the eight
-//           pieces (e, tt) (half-word hi = token 8 ps + 2 tt + hi, field i = channel 16 i + 8 rsel + e) and writes, for
+//           j = rs + 2 hh, bytes b = 2 b1 + b0; the field of k-step s in a byte = channel 32 s + 16 hh + 8 b1 + 2 t + b0 of
+//           token g + 8 rs) and writes, for (rs, hh, b1), the chunk of channels 8 (4 s + 2 hh + b1) .. + 7 of that token:
+//           pair t = (b0 0, 1).  At 4 bits the k-steps 0-1 / 2-3 sit in two 512-byte halves, a nibble each.
+//   values: thread (block bi, token half ps, row half rsel, half ih of the channel blocks, token pair tt) loads one word of the
+//           eight pieces (e, tt) (half-word hi = token 8 ps + 2 tt + hi, field i = channel 16 i + 8 rsel + e) and writes, for
 //           (hi, i in 4 ih .. 4 ih + 3), the chunk of channels 8 (2 i + rsel) .. + 7 of that token: element e.
-__device__ __forceinline__ void unpack_page2(const unsigned char* raw, unsigned char* sK, unsigned char* sV, const int p) {
+//   3 bits: the 2-bit plane as above plus the high bit of every code from the 1-bit planes (csrc/layout.cuh).
+template <int BITS>
+__device__ __forceinline__ void unpack_page(const unsigned char* raw, unsigned char* sK, unsigned char* sV, const int p) {
+    constexpr bool TWO = BITS != 4;                         // 2-bit fields (also the low plane of 3-bit records)
+    constexpr unsigned MASK = TWO ? 3u : 15u, MASK_HI = MASK << 16;
+    constexpr int CB = code_block_bytes(BITS);
     const __half2 bias = __halves2half2(__ushort_as_half(0x6400), __ushort_as_half(0x6400));
-    auto to_h2 = [&](const unsigned pair) {             // two codes (bits 0-1 and 16-17) -> fp16 pair: 1024 + c, minus 1024
+    auto to_h2 = [&](const unsigned pair) {             // two codes (low bits of each half) -> fp16 pair: 1024 + c, minus 1024
         const unsigned w = pair | 0x64006400u;
         const __half2 hv = __hsub2(*reinterpret_cast<const __half2*>(&w), bias);
         return *reinterpret_cast<const unsigned*>(&hv);
     };
     {
         const int g = p & 7, s = (p >> 3) & 3, bi = p >> 5;
+        const unsigned char* src = raw + bi * CB + (TWO ? 0 : 512 * (s >> 1)) + 64 * g;
+        const int sh0 = TWO ? 2 * s : 4 * (s & 1);
         unsigned w[4][4];                                   // [t][j]
+        unsigned wh[4][2];                                  // 3 bits: [t][rs], bit 2 s + hh of byte b
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
-            const uint4 v = *reinterpret_cast<const uint4*>(raw + bi * 512 + 64 * g + 16 * t);
+            const uint4 v = *reinterpret_cast<const uint4*>(src + 16 * t);
             w[t][0] = v.x; w[t][1] = v.y; w[t][2] = v.z; w[t][3] = v.w;
+            if (BITS == 3) {
+                const uint2 y = *reinterpret_cast<const uint2*>(raw + k_hi_offset(3) + bi * 256 + 8 * (4 * g + t));
+                wh[t][0] = y.x; wh[t][1] = y.y;
+            }
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {                       // j = rs + 2 hh
@@ -756,8 +769,13 @@ __device__ __forceinline__ void unpack_page2(const unsigned char* raw, unsigned 
                 unsigned out[4];
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
-                    const unsigned x = w[t][j] >> (16 * b1 + 2 * s);
-                    out[t] = to_h2((x & 3u) | ((x << 8) & 0x00030000u));
+                    const unsigned x = w[t][j] >> (16 * b1 + sh0);
+                    unsigned pair = (x & MASK) | ((x << 8) & MASK_HI);
+                    if (BITS == 3) {
+                        const unsigned y = wh[t][j & 1] >> (16 * b1 + 2 * s + (j >> 1));
+                        pair |= ((y & 1u) | ((y << 8) & 0x00010000u)) << 2;
+                    }
+                    out[t] = to_h2(pair);
                 }
                 *reinterpret_cast<uint4*>(sK + (2 * bi + (j & 1)) * 2048 + (4 * s + 2 * (j >> 1) + b1) * 128 + g * 16) =
                     make_uint4(out[0], out[1], out[2], out[3]);
@@ -766,17 +784,27 @@ __device__ __forceinline__ void unpack_page2(const unsigned char* raw, unsigned 
     }
     {
         const int tt = p & 3, ih = (p >> 2) & 1, m = (p >> 3) & 3, bi = p >> 5, ps = m >> 1, rsel = m & 1;
-        unsigned w[8];                                      // [e]
+        const unsigned char* src = raw + v_codes_offset(BITS) + bi * CB + (TWO ? 4 * m : 512 * ps + 4 * (2 * rsel + ih)) + 16 * tt;
+        unsigned w[8], wh[8];                               // [e]; 3 bits: the word of token half ps (both half-words)
 #pragma unroll
-        for (int e = 0; e < 8; ++e) w[e] = *reinterpret_cast<const unsigned*>(raw + v_codes_offset(2) + bi * 512 + 16 * (4 * e + tt) + 4 * m);
+        for (int e = 0; e < 8; ++e) {
+            w[e] = *reinterpret_cast<const unsigned*>(src + 64 * e);
+            if (BITS == 3) wh[e] = *reinterpret_cast<const unsigned*>(raw + v_hi_offset(3) + bi * 256 + 8 * (4 * e + tt) + 4 * ps);
+        }
 #pragma unroll
         for (int hi = 0; hi < 2; ++hi) {
 #pragma unroll
             for (int ii = 0; ii < 4; ++ii) {
-                const int i = 4 * ih + ii, sh = 16 * hi + 2 * i;
+                const int i = 4 * ih + ii, sh = 16 * hi + (TWO ? 2 * i : 4 * ii);
+                // bit of the 1-bit plane for (rsel, i): rsel 0: 2 i + 2 (i < 5), 2 i + 1 (else); rsel 1: 2 i + 1 (i < 5), 2 i + 2 (i < 7), 0 (i = 7)
+                const int hb = 16 * hi + (rsel == 0 ? (i < 5 ? 2 * i + 2 : 2 * i + 1) : (i < 5 ? 2 * i + 1 : (i < 7 ? 2 * i + 2 : 0)));
                 unsigned out[4];
 #pragma unroll
-                for (int e2 = 0; e2 < 4; ++e2) out[e2] = to_h2(((w[2 * e2] >> sh) & 3u) | (((w[2 * e2 + 1] >> sh) & 3u) << 16));
+                for (int e2 = 0; e2 < 4; ++e2) {
+                    unsigned c0 = (w[2 * e2] >> sh) & MASK, c1 = (w[2 * e2 + 1] >> sh) & MASK;
+                    if (BITS == 3) { c0 |= ((wh[2 * e2] >> hb) & 1u) << 2; c1 |= ((wh[2 * e2 + 1] >> hb) & 1u) << 2; }
+                    out[e2] = to_h2(c0 | (c1 << 16));
+                }
                 *reinterpret_cast<uint4*>(sV + (2 * i + rsel) * 1024 + (2 * bi + ps) * 128 + (2 * tt + hi) * 16) =
                     make_uint4(out[0], out[1], out[2], out[3]);
             }
@@ -1745,10 +1773,10 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 const unsigned char* raw = sm_ws + WS_OFF_RAW + rb * WS_RAW_BYTES;
                 const uint4 zero4 = make_uint4(0, 0, 0, 0);
                 const int page_pos = (page_first + gb) * PAGE_TOKENS;
-                const bool whole = BITS == 2 && page_ok && page_pos >= q_lo && page_pos + PAGE_TOKENS <= q_hi;
-                if (whole && mine) unpack_page2(raw, sK, sV, ptid);
+                const bool whole = page_ok && page_pos >= q_lo && page_pos + PAGE_TOKENS <= q_hi;
+                if (whole && mine) unpack_page<BITS>(raw, sK, sV, ptid);
 #pragma unroll 4
-                for (int item = ptid; item < (mine && !whole ? TN * 16 : 0); item += 128) {      // first / last page, other widths
+                for (int item = ptid; item < (mine && !whole ? TN * 16 : 0); item += 128) {      // first / last page of the range
                     const int r = item & (TN - 1), kc = item >> 6;
                     const int pos = (page_first + gb) * PAGE_TOKENS + r;
                     const bool live = page_ok && pos >= q_lo && pos < q_hi;
