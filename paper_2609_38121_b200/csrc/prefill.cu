@@ -1211,22 +1211,26 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
 constexpr int WS_THREADS = 512;
 constexpr int WS_KS = 2, WS_VS = 3;                              // ring depths of the key / value stages: a key stage is free again when
                                                                  // its scores are done, a value stage only after O += P V a softmax later
-constexpr int WS_RAW_BYTES = 8704;                               // largest packed record (4 bits)
 constexpr int WS_OFF_Q = 0;                                      // (tile 0 value, remainder), (tile 1 value, remainder)
 constexpr int WS_OFF_K = 4 * TC_Q_BYTES;
 constexpr int WS_OFF_V = WS_OFF_K + WS_KS * TC_K_BYTES;
 constexpr int WS_OFF_RAW = WS_OFF_V + WS_VS * TC_K_BYTES;        // two raw records
-constexpr int WS_OFF_META = WS_OFF_RAW + 2 * WS_RAW_BYTES;       // unsigned[WS_VS][2][TN]: per-key factors of a packed tile (key side, value side)
-constexpr int WS_OFF_LIVE = WS_OFF_META + WS_VS * TN * 8;        // uint2[WS_VS]: which keys of a packed tile exist
 enum { WB_KFULL = 0, WB_KEMPTY = WB_KFULL + WS_KS, WB_VFULL = WB_KEMPTY + WS_KS, WB_VEMPTY = WB_VFULL + WS_VS,
        WB_S = WB_VEMPTY + WS_VS, WB_PV = WB_S + 4, WB_PREADY = WB_PV + 4, WB_RAW = WB_PREADY + 4, WB_Q = WB_RAW + 2,
        WB_STAGED, WB_DRAIN, WB_COUNT };
-constexpr int WS_OFF_BAR = WS_OFF_LIVE + WS_VS * 8;
-constexpr int WS_OFF_MISC = WS_OFF_BAR + WB_COUNT * 8;           // [0] tensor-memory slot, [4] abort flag
-constexpr int WS_SMEM = WS_OFF_MISC + 16;
-static_assert(WS_SMEM <= 232448, "the dynamic shared memory of one CTA");
-static_assert(WS_OFF_K % 1024 == 0 && WS_OFF_V % 1024 == 0 && WS_OFF_RAW % 16 == 0 && WS_RAW_BYTES % 16 == 0, "alignment of the stages");
-static_assert(record_bytes(4) <= WS_RAW_BYTES && record_bytes(3) <= WS_RAW_BYTES, "raw record buffer");
+// The rest of the layout depends on the record size.  Per-key factors of a packed tile, per value stage: (step, offset) of
+// the key side for the 64 keys, then of the value side; as fp32 pairs where the record leaves room for them (2 and 3 bits:
+// the softmax threads then load them ready to use, two keys per 16-byte load), as the record's fp16 pairs at 4 bits.
+__host__ __device__ constexpr bool ws_meta32(int bits) { return bits != 4; }
+__host__ __device__ constexpr int ws_meta_stage(int bits) { return 2 * TN * (ws_meta32(bits) ? 8 : 4); }
+__host__ __device__ constexpr int ws_off_meta(int bits) { return WS_OFF_RAW + 2 * record_bytes(bits); }
+__host__ __device__ constexpr int ws_off_live(int bits) { return ws_off_meta(bits) + WS_VS * ws_meta_stage(bits); }      // uint2[WS_VS]: which keys of a packed tile exist
+__host__ __device__ constexpr int ws_off_bar(int bits) { return ws_off_live(bits) + WS_VS * 8; }
+__host__ __device__ constexpr int ws_off_misc(int bits) { return ws_off_bar(bits) + WB_COUNT * 8; }                       // [0] tensor-memory slot, [4] abort flag
+__host__ __device__ constexpr int ws_smem(int bits) { return ws_off_misc(bits) + 16; }
+static_assert(ws_smem(2) <= 232448 && ws_smem(3) <= 232448 && ws_smem(4) <= 232448, "the dynamic shared memory of one CTA");
+static_assert(WS_OFF_K % 1024 == 0 && WS_OFF_V % 1024 == 0 && WS_OFF_RAW % 16 == 0, "alignment of the stages");
+static_assert(record_bytes(2) % 16 == 0 && record_bytes(3) % 16 == 0 && record_bytes(4) % 16 == 0, "raw records are copied in 16-byte units");
 
 // Bounded wait for a phase of an mbarrier; gives up early when another role has raised the abort flag and raises it
 // itself when the limit runs out.
@@ -1288,6 +1292,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                                                                         const __grid_constant__ CUtensorMap map_q1) {
     extern __shared__ __align__(1024) unsigned char sm_ws[];
     constexpr int REC = record_bytes(BITS);
+    constexpr bool META32 = ws_meta32(BITS);
+    constexpr int META_STAGE = ws_meta_stage(BITS);
     const CacheView& c = P.c;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = c.G, R = TM / G;                              // chunk positions per query tile
@@ -1301,12 +1307,12 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
         if (tid == 0) atomicOr(c.dev_status, WUSHKV_DEV_BAD_SLOT);
         return;
     }
-    const unsigned bar0 = smem_addr(sm_ws + WS_OFF_BAR);
+    const unsigned bar0 = smem_addr(sm_ws + ws_off_bar(BITS));
     auto bar = [&](int i) -> unsigned { return bar0 + 8u * static_cast<unsigned>(i); };
-    unsigned* tmem_slot = reinterpret_cast<unsigned*>(sm_ws + WS_OFF_MISC);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm_ws + WS_OFF_MISC + 4);
-    unsigned* meta_all = reinterpret_cast<unsigned*>(sm_ws + WS_OFF_META);     // [stage][key side, value side][key]: (step, offset) as fp16 pairs
-    uint2* live_all = reinterpret_cast<uint2*>(sm_ws + WS_OFF_LIVE);
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(sm_ws + ws_off_misc(BITS));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm_ws + ws_off_misc(BITS) + 4);
+    unsigned char* meta_all = sm_ws + ws_off_meta(BITS);         // [stage][key side, value side][key]: (step, offset)
+    uint2* live_all = reinterpret_cast<uint2*>(sm_ws + ws_off_live(BITS));
 
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(512u) : "memory");
@@ -1395,8 +1401,16 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 // one barrier per score buffer: its next phase (tile g + 2) cannot complete before this tile's probabilities are ready
                 if (!__all_sync(FULLM, ws_wait(bar(WB_S + 2 * t + (g & 1)), (g >> 1) & 1, wait_limit, abort_flag))) { ok = false; return; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint4* kmeta = reinterpret_cast<const uint4*>(meta_all + (2 * (g % WS_VS)) * TN);       // four keys per load
-                const uint4* vmeta = kmeta + TN / 4;
+                const unsigned char* kmeta = meta_all + (g % WS_VS) * META_STAGE, *vmeta = kmeta + META_STAGE / 2;
+                auto factors4 = [&](const unsigned char* side, const int j4, float2 (&f)[4]) {      // (step, offset) of keys 4 j4 .. 4 j4 + 3
+                    if constexpr (META32) {
+                        const float4 a = reinterpret_cast<const float4*>(side)[2 * j4], b2 = reinterpret_cast<const float4*>(side)[2 * j4 + 1];
+                        f[0] = make_float2(a.x, a.y); f[1] = make_float2(a.z, a.w); f[2] = make_float2(b2.x, b2.y); f[3] = make_float2(b2.z, b2.w);
+                    } else {
+                        const uint4 m4 = reinterpret_cast<const uint4*>(side)[j4];
+                        f[0] = h2f2u(m4.x); f[1] = h2f2u(m4.y); f[2] = h2f2u(m4.z); f[3] = h2f2u(m4.w);
+                    }
+                };
                 if (PACKED) {
                     if (!__all_sync(FULLM, ws_wait(bar(WB_VFULL + g % WS_VS), (g / WS_VS) & 1, wait_limit, abort_flag))) { ok = false; return; }
                     const uint2 lv = live_all[g % WS_VS];
@@ -1412,22 +1426,21 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 if (PACKED && (live_lo & live_hi) == 0xffffffffu) {
 #pragma unroll
                     for (int j4 = 0; j4 < TN / 4; ++j4) {
-                        const uint4 m4 = kmeta[j4];
-                        const unsigned mw[4] = {m4.x, m4.y, m4.z, m4.w};
+                        float2 mk[4];
+                        factors4(kmeta, j4, mk);
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) { const float2 mk = h2f2u(mw[q]); s[4 * j4 + q] = fmaf(mk.y, my_qsum, mk.x * s[4 * j4 + q]); }
+                        for (int q = 0; q < 4; ++q) s[4 * j4 + q] = fmaf(mk[q].y, my_qsum, mk[q].x * s[4 * j4 + q]);
                     }
                 } else if (PACKED || MASKED) {
 #pragma unroll
                     for (int j4 = 0; j4 < TN / 4; ++j4) {
-                        uint4 m4 = make_uint4(0u, 0u, 0u, 0u);
-                        if (PACKED) m4 = kmeta[j4];
-                        const unsigned mw[4] = {m4.x, m4.y, m4.z, m4.w};
+                        float2 mk[4];
+                        if (PACKED) factors4(kmeta, j4, mk);
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
                             const int j = 4 * j4 + q;
                             float v = s[j];
-                            if (PACKED) { const float2 mk = h2f2u(mw[q]); v = fmaf(mk.y, my_qsum, mk.x * v); }
+                            if (PACKED) v = fmaf(mk[q].y, my_qsum, mk[q].x * v);
                             if (MASKED) {
                                 const bool live = ((j < 32 ? live_lo >> j : live_hi >> (j - 32)) & 1u) != 0u;
                                 if (!live || crow0 + j > my_row) v = -INFINITY;
@@ -1469,16 +1482,15 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                     unsigned pk[16];
 #pragma unroll
                     for (int e4 = 0; e4 < 8; ++e4) {                       // four keys = two fp16 pairs at a time
-                        uint4 m4 = make_uint4(0u, 0u, 0u, 0u);
-                        if (PACKED) m4 = vmeta[8 * half + e4];
-                        const unsigned mw[4] = {m4.x, m4.y, m4.z, m4.w};
+                        float2 mv[4];
+                        if (PACKED) factors4(vmeta, 8 * half + e4, mv);
 #pragma unroll
                         for (int q = 0; q < 2; ++q) {
                             const int e = 16 * half + 2 * e4 + q;
                             float2 pr = make_float2(fast_ex2(fmaf(s[2 * e], k2, -ref)), fast_ex2(fmaf(s[2 * e + 1], k2, -ref)));     // k2 s - ref in one rounding
                             lsum.x += pr.x; lsum.y += pr.y;
                             if (PACKED) {
-                                const float2 mv0 = h2f2u(mw[2 * q]), mv1 = h2f2u(mw[2 * q + 1]);
+                                const float2 mv0 = mv[2 * q], mv1 = mv[2 * q + 1];
                                 z = fmaf(pr.x, mv0.y, fmaf(pr.y, mv1.y, z));
                                 pr.x *= mv0.x; pr.y *= mv1.x;
                             }
@@ -1716,7 +1728,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 return;
             }
             ws_expect_tx(bar(WB_RAW + (gb & 1)), REC);
-            ws_bulk_g2s(smem_addr(sm_ws + WS_OFF_RAW + (gb & 1) * WS_RAW_BYTES), c.pages + (static_cast<long long>(page) * c.n_kv + h) * REC, REC,
+            ws_bulk_g2s(smem_addr(sm_ws + WS_OFF_RAW + (gb & 1) * REC), c.pages + (static_cast<long long>(page) * c.n_kv + h) * REC, REC,
                         bar(WB_RAW + (gb & 1)));
         };
         if (nB > 0 && ptid == 0) fetch_record(0);
@@ -1770,7 +1782,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 const bool page_ok = page_of(gb) >= 0;
                 if (page_ok && mine) mine = __all_sync(FULLM, ws_wait(bar(WB_RAW + rb), raw_uses[rb] & 1, wait_limit, abort_flag));
                 if (page_ok) ++raw_uses[rb];
-                const unsigned char* raw = sm_ws + WS_OFF_RAW + rb * WS_RAW_BYTES;
+                const unsigned char* raw = sm_ws + WS_OFF_RAW + rb * REC;
                 const uint4 zero4 = make_uint4(0, 0, 0, 0);
                 const int page_pos = (page_first + gb) * PAGE_TOKENS;
                 const bool whole = page_ok && page_pos >= q_lo && page_pos + PAGE_TOKENS <= q_hi;
@@ -1789,8 +1801,14 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                     const int pos = (page_first + gb) * PAGE_TOKENS + ptid;
                     const bool live = page_ok && pos >= q_lo && pos < q_hi;
                     const uint2 m = live ? *reinterpret_cast<const uint2*>(raw + meta_location(BITS, ptid)) : make_uint2(0u, 0u);
-                    meta_all[(2 * vs) * TN + ptid] = m.x;
-                    meta_all[(2 * vs + 1) * TN + ptid] = m.y;
+                    unsigned char* kside = meta_all + vs * META_STAGE, *vside = kside + META_STAGE / 2;
+                    if constexpr (META32) {
+                        reinterpret_cast<float2*>(kside)[ptid] = h2f2u(m.x);
+                        reinterpret_cast<float2*>(vside)[ptid] = h2f2u(m.y);
+                    } else {
+                        reinterpret_cast<unsigned*>(kside)[ptid] = m.x;
+                        reinterpret_cast<unsigned*>(vside)[ptid] = m.y;
+                    }
                     const unsigned word = __ballot_sync(FULLM, live);
                     if (lane == 0) reinterpret_cast<unsigned*>(live_all + vs)[ptid >> 5] = word;
                 }
@@ -2212,13 +2230,14 @@ static int prefill_attn_impl(const wushkv_cache* cache, int32_t batch, const int
             const bool mq = make_row_tensor_map(map_q0, false, P.QP, P.c.n_q, total_new, R, P.c.G) &&
                             make_row_tensor_map(map_q1, false, P.QP + static_cast<size_t>(total_new) * P.c.n_q * D, P.c.n_q, total_new, R, P.c.G);
             if (!mq) P.use_tma = 0;
-            auto launch_ws = [&](auto kernel) -> bool {
-                if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(kernel), WS_SMEM)) return false;
-                kernel<<<grid_ws, WS_THREADS, WS_SMEM, st>>>(P, map_k, map_v, map_q0, map_q1);
+            auto launch_ws = [&](auto kernel, const int smem) -> bool {
+                if (!opt_in_dynamic_smem(reinterpret_cast<const void*>(kernel), smem)) return false;
+                kernel<<<grid_ws, WS_THREADS, smem, st>>>(P, map_k, map_v, map_q0, map_q1);
                 return true;
             };
-            const bool ok = P.c.bits == 2 ? launch_ws(prefill_attn_ws_kernel<2>) : P.c.bits == 3 ? launch_ws(prefill_attn_ws_kernel<3>)
-                                                                                             : launch_ws(prefill_attn_ws_kernel<4>);
+            const bool ok = P.c.bits == 2   ? launch_ws(prefill_attn_ws_kernel<2>, ws_smem(2))
+                            : P.c.bits == 3 ? launch_ws(prefill_attn_ws_kernel<3>, ws_smem(3))
+                                            : launch_ws(prefill_attn_ws_kernel<4>, ws_smem(4));
             if (!ok) return WUSHKV_ECUDA;
 #if WUSHKV_WS_TIMING
             {
