@@ -1721,8 +1721,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
             if (pg < c.max_pages) page = __ldg(c.page_table + static_cast<long long>(sl) * c.max_pages + pg);
             return (page >= 0 && page < c.n_pages) ? page : -1;
         };
-        auto fetch_record = [&](const int gb) {                 // one thread: bulk copy of the record into raw buffer gb & 1
-            const int page = page_of(gb);
+        auto fetch_record = [&](const int gb, const int page) {     // one thread: bulk copy of the record into raw buffer gb & 1
             if (page < 0) {
                 atomicOr(c.dev_status, page_first + gb < c.max_pages ? WUSHKV_DEV_BAD_PAGE_ID : WUSHKV_DEV_PAGE_TABLE_FULL);
                 return;
@@ -1731,7 +1730,9 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
             ws_bulk_g2s(smem_addr(sm_ws + WS_OFF_RAW + (gb & 1) * REC), c.pages + (static_cast<long long>(page) * c.n_kv + h) * REC, REC,
                         bar(WB_RAW + (gb & 1)));
         };
-        if (nB > 0 && ptid == 0) fetch_record(0);
+        // page ids are read two tiles ahead, so that neither the record request nor the unpacking waits for the page table
+        int page_cur = nB > 0 ? page_of(0) : -1, page_next = nB > 1 ? page_of(1) : -1;
+        if (nB > 0 && ptid == 0) fetch_record(0, page_cur);
         bool ok = true;
         WST_DECL;
         for (int g = 0; g < n_staged && ok; ++g) {
@@ -1778,8 +1779,10 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 // ---- a packed page: the record was requested one tile ahead; unpack it into integer codes (exact in fp16)
                 const int gb = g - nA, rb = gb & 1;
                 // the other raw buffer was last read for tile gb - 1, which every staging thread has left
-                if (gb + 1 < nB && ptid == 0) fetch_record(gb + 1);
-                const bool page_ok = page_of(gb) >= 0;
+                if (gb + 1 < nB && ptid == 0) fetch_record(gb + 1, page_next);
+                const bool page_ok = page_cur >= 0;
+                page_cur = page_next;
+                page_next = gb + 2 < nB ? page_of(gb + 2) : -1;
                 if (page_ok && mine) mine = __all_sync(FULLM, ws_wait(bar(WB_RAW + rb), raw_uses[rb] & 1, wait_limit, abort_flag));
                 if (page_ok) ++raw_uses[rb];
                 const unsigned char* raw = sm_ws + WS_OFF_RAW + rb * REC;
