@@ -7,15 +7,21 @@
 // their bf16 copies, the quantized middle from the packed pages (x_hat = x_min + Delta * code, Eq. 6 / Eq. 5).
 //
 // Two launches:
-//   1. prefill_prep_kernel     q' = T_K^{-T} q and k' = T_K k of the chunk on tensor cores (bf16 mma, fp32
+//   1. transforms              q' = T_K^{-T} q and k' = T_K k of the chunk on tensor cores (bf16 products, fp32
 //                              accumulation), written as fp16 operands of the attention kernel (k' through its bf16
 //                              rounding, the value the cache's window copies hold; q' as value + rounding
 //                              remainder), the chunk's values as fp16, and sum_c q'_c per query row.
-//   2. prefill_attn_tc_kernel  (default) one CTA per (sequence, KV head, 128-row tile that packs the G query heads):
-//                              both contractions as tcgen05.mma with accumulators in tensor memory; see section 2b.
-//      prefill_attn_kernel     (testing aid "prefill_legacy") one CTA per (sequence, query head, 64 query rows) on
-//                              mma.sync.m16n8k16; the first version, kept as a second implementation to test against.
-//   Both stream 64-key tiles of the three sources through shared memory and keep an online softmax
+//                              prefill_prep_tc_kernel (tcgen05, section 1b) for plain inputs; prefill_prep_kernel
+//                              (mma.sync, section 1) for projected inputs, whose rows it normalises and rotates first.
+//   2. attention               prefill_attn_ws_kernel (default, section 2c): one CTA per (sequence, KV head, pair of
+//                              128-row tiles that pack the G query heads), warp-specialised, both contractions as
+//                              tcgen05.mma with accumulators in tensor memory.
+//                              prefill_attn_tc_kernel (testing aid "prefill_one_tile", section 2b): the same contractions,
+//                              one tile per CTA, no role split.
+//                              prefill_attn_kernel (testing aid "prefill_legacy", section 2): one CTA per (sequence, query
+//                              head, 64 query rows) on mma.sync.m16n8k16; the first version.
+//                              The last two are kept as further implementations to test against.
+//   All stream 64-key tiles of the three sources through shared memory and keep an online softmax
 //   (flash-attention recurrence) per row.  The affine part of the quantizer is factored out of the contractions,
 //   per key j of a tile:
 //                                score_ij = Delta_k,j (q'_i . c_k,j) + x_min_k,j sum(q'_i)
@@ -538,7 +544,7 @@ __global__ void __launch_bounds__(PF_THREADS) prefill_attn_kernel(PrefillParams 
 }
 
 // ------------------------------------------------------------------------------------------------
-// 2b. attention on tcgen05 (the default path)
+// 2b. attention on tcgen05, one tile per CTA (testing aid "prefill_one_tile"; the default before section 2c)
 // ------------------------------------------------------------------------------------------------
 // One CTA of 128 threads per (sequence, KV head, tile of R = 128 / G chunk positions): the G query heads that
 // read the KV head are packed into the M = 128 rows of the tile (row r = position r / G, head r % G), so a staged
