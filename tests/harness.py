@@ -191,10 +191,12 @@ class Layer:
         assert np.all(np.isfinite(out)), "oracle read a position the GPU keeps no bf16 copy of"
         return out
 
-    def prefill(self, counts, queries=None):
+    def prefill(self, counts, queries=None, repeat=0):
         """Append counts[b] new tokens per sequence and compute their attention outputs with wushkv_prefill_attn (with
         wushkv_prefill_attn_projected if this layer has a prologue; ``queries`` then holds the projected queries).
-        Returns (O_gpu list per sequence [n][n_q][128], queries list per sequence)."""
+        Returns (O_gpu list per sequence [n][n_q][128], queries list per sequence).  ``repeat`` > 0: the attention call is
+        made that many more times on the same cache state into fresh buffers, and ``self.repeats`` holds those outputs
+        (whole arrays [total][n_q][128], float32) beside the first call's ``self.first``."""
         torch, B = self.torch, self.B
         counts = [int(c) for c in counts]
         start = list(self.done)
@@ -218,7 +220,18 @@ class Layer:
         else:
             B.prefill_attn(self.cache.desc, self.batch, self.slot, self.seq_len, cu, total, max(counts), Kn, Vn, Qn, Oo, ws, nbytes)
         torch.cuda.synchronize()
-        out = Oo.cpu().numpy().astype(np.float64)
+        self.first, self.repeats = Oo.cpu().numpy(), []
+        for _ in range(repeat):
+            O2 = torch.full((total, self.wl.n_q, 128), float("nan"), dtype=torch.float32, device=dev)
+            ws2 = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+            if self.prologue is not None:
+                B.prefill_attn_projected(self.cache.desc, self.batch, self.slot, self.seq_len, cu, total, max(counts), Kn, Vn, Qn,
+                                         self.prologue.desc, O2, ws2, nbytes)
+            else:
+                B.prefill_attn(self.cache.desc, self.batch, self.slot, self.seq_len, cu, total, max(counts), Kn, Vn, Qn, O2, ws2, nbytes)
+            torch.cuda.synchronize()
+            self.repeats.append(O2.cpu().numpy())
+        out = self.first.astype(np.float64)
         offs = np.concatenate([[0], np.cumsum(counts)])
         return [out[offs[b]:offs[b + 1]] for b in range(self.batch)], qs
 

@@ -62,6 +62,18 @@ def test_head_group_sizes(n_q, n_kv):
     assert L.cache.status() == 0
 
 
+def test_chunk_attention_is_bit_identical_from_run_to_run():
+    """The same call on the same cache state three times: the roles of the warp-specialised kernel meet in an order that
+    depends on timing, the arithmetic must not (tile order of every accumulation is fixed)."""
+    wl = _wl(14, 2, seed=98, batch=2)
+    L = Layer(wl, [1500, 700], 2, 4, 64, 8)
+    L.append_step([900, 300])
+    L.prefill([600, 400], repeat=2)
+    for other in L.repeats:
+        assert np.array_equal(L.first.view(np.uint32), other.view(np.uint32))
+    assert L.cache.status() == 0
+
+
 def test_chunk_shorter_than_the_recent_window_and_second_chunk():
     """Chunks of 16 tokens as in the paper's perplexity runs (S_sink 16, S_keep 128, S_flush 16): old recent-window
     rows come from the ring, the quantized boundary sits below the chunk; two chunks in a row."""
