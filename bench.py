@@ -691,7 +691,7 @@ def run_ours(args, rank, world):
         tf_peak, tf_kind = measured_tensor_peak()
         pf_s = statistics.mean(prefill_ms) * 1e-3
         tf = sess.prefill_flops() / pf_s / 1e12
-        roofline = {"bound": "tensor", "kernel": "prefill_attn_tc_kernel (+ prefill_prep_kernel)", "achieved": tf, "peak": tf_peak,
+        roofline = {"bound": "tensor", "kernel": "prefill_attn_ws_kernel (+ prefill_prep_tc_kernel)", "achieved": tf, "peak": tf_peak,
                     "unit": "TFLOP/s", "frac": tf / tf_peak, "peak_kind": f"of {tf_kind} (bf16 matmul, sustained; fp16 has the same nominal rate)",
                     "kernel_ms": pf_s * 1e3, "kernel_ms_min": min(prefill_ms), "algorithmic_flops": sess.prefill_flops(), "traffic": None}
     cpu = None
