@@ -11,8 +11,9 @@
 //                              accumulation), written as fp16 operands of the attention kernel (k' through its bf16
 //                              rounding, the value the cache's window copies hold; q' as value + rounding
 //                              remainder), the chunk's values as fp16, and sum_c q'_c per query row.
-//                              prefill_prep_tc_kernel (tcgen05, section 1b) for plain inputs; prefill_prep_kernel
-//                              (mma.sync, section 1) for projected inputs, whose rows it normalises and rotates first.
+//                              prefill_prep_tc_kernel (tcgen05, section 1b); prefill_prep_kernel (mma.sync, section 1)
+//                              without bulk tensor copies and as a testing aid.  Projected rows are normalised and
+//                              rotated in shared memory first (Algorithm 2 lines 1-2) by either.
 //   2. attention               prefill_attn_ws_kernel (default, section 2c): one CTA per (sequence, KV head, pair of
 //                              128-row tiles that pack the G query heads), warp-specialised, both contractions as
 //                              tcgen05.mma with accumulators in tensor memory.
@@ -1875,7 +1876,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
 }
 
 // ------------------------------------------------------------------------------------------------
-// 1b. transforms of the chunk on tcgen05 (the default for plain, i.e. not projected, inputs)
+// 1b. transforms of the chunk on tcgen05 (the default)
 // ------------------------------------------------------------------------------------------------
 // The same arithmetic as prefill_prep_kernel (bf16 x bf16 products, exact in the fp32 accumulator; T_K^{-T} as three bf16
 // terms), as tcgen05.mma with the accumulator in tensor memory.  A CTA keeps its head's transform in shared memory as the
@@ -1893,11 +1894,13 @@ constexpr int PT_THREADS = 576;                                  // warps 0-15 e
 constexpr int PT_OFF_T = 0;                                      // three terms of 128 x 128 bf16, K-major core matrices
 constexpr int PT_OFF_X = 3 * D * D * 2;                          // two token tiles (128-byte-swizzled rows, two 16 KB boxes each)
 constexpr int PT_X_BYTES = PREP_TOK * D * 2;
-enum { PB_XFULL = 0, PB_XEMPTY = 2, PB_DFULL = 4, PB_DEMPTY = 6, PB_DRAIN = 8, PB_COUNT = 9 };
+enum { PB_XFULL = 0, PB_XEMPTY = 2, PB_DFULL = 4, PB_DEMPTY = 6, PB_XREADY = 8, PB_DRAIN = 10, PB_COUNT = 11 };
 constexpr int PT_OUT_PITCH = D * 2 + 16;                         // bytes per staged output row (272: conflict-free 16-byte pieces)
 constexpr int PT_OFF_OUT = PT_OFF_X + 2 * PT_X_BYTES;            // one fp16 output tile on its way to global memory
 constexpr int PT_OFF_QS = PT_OFF_OUT + PREP_TOK * PT_OUT_PITCH;  // float[4][128]: partial sums of q' over channel quarters
-constexpr int PT_OFF_BAR = PT_OFF_QS + 4 * PREP_TOK * 4;
+constexpr int PT_MAX_SEQ = 1024;                                 // sequences whose chunk bounds are kept in shared memory (projected inputs)
+constexpr int PT_OFF_SEQ = PT_OFF_QS + 4 * PREP_TOK * 4;         // int[PT_MAX_SEQ + 1] first chunk token, int[PT_MAX_SEQ] position of token 0 minus its index
+constexpr int PT_OFF_BAR = PT_OFF_SEQ + (2 * PT_MAX_SEQ + 2) * 4;
 constexpr int PT_OFF_MISC = PT_OFF_BAR + PB_COUNT * 8;           // [0] tensor-memory slot, [4] abort flag
 constexpr int PT_SMEM = PT_OFF_MISC + 16;
 constexpr unsigned PT_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((static_cast<unsigned>(D) >> 3) << 17) | ((static_cast<unsigned>(PREP_TOK) >> 4) << 24);   // fp32 <- bf16 x bf16, K-major
@@ -1906,7 +1909,7 @@ static_assert(PT_OFF_X % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 #if WUSHKV_WS_TIMING
 #define PST_DECL long long pst_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long pst_last = clock64()
 #define PST(slot) do { const long long now = clock64(); pst_acc[slot] += now - pst_last; pst_last = now; } while (0)
-#define PST_FLUSH(base) do { if (blockIdx.x == 0 && blockIdx.y == gridDim.y - 1 && lane == 0) for (int i_ = 0; i_ < 8; ++i_) g_ws_t[(base) + i_] += pst_acc[i_]; } while (0)
+#define PST_FLUSH(base) do { if (blockIdx.x == 0 && blockIdx.y == P.c.n_kv && lane == 0) for (int i_ = 0; i_ < 8; ++i_) g_ws_t[(base) + i_] += pst_acc[i_]; } while (0)
 #else
 #define PST_DECL
 #define PST(slot) do { } while (0)
@@ -1967,11 +1970,23 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_prep_tc_kernel(PrefillP
     }
     if (tid == 0) {
         for (int i = 0; i < PB_COUNT; ++i) {
-            const unsigned count = (i == PB_DEMPTY || i == PB_DEMPTY + 1) ? 512u : 1u;      // accumulator released by the 512 epilogue threads
+            // accumulator released, and projected rows normalised and rotated, by the 512 epilogue threads
+            const unsigned count = (i == PB_DEMPTY || i == PB_DEMPTY + 1 || i == PB_XREADY || i == PB_XREADY + 1) ? 512u : 1u;
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar(i)), "r"(count) : "memory");
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // projected inputs: where every sequence's chunk starts and the position of its first token, for the row fix-up
+    int* seq_first = reinterpret_cast<int*>(sm_pt + PT_OFF_SEQ);
+    int* seq_base = seq_first + PT_MAX_SEQ + 1;
+    const bool seq_in_smem = P.pro.rope != nullptr && P.batch <= PT_MAX_SEQ;
+    if (seq_in_smem) {
+        for (int bq = tid; bq <= P.batch; bq += PT_THREADS) {
+            const int f0 = __ldg(P.cu_new + bq);
+            seq_first[bq] = f0;
+            if (bq < P.batch) seq_base[bq] = __ldg(P.seq_len + bq) - (__ldg(P.cu_new + bq + 1) - f0) - f0;
+        }
     }
     // the transform as the B operand: element (i, j) of term `term` at (i / 8) * 2048 + (j / 8) * 128 + (i % 8) * 16 + (j % 8) * 2
     for (int idx = tid; idx < D * D; idx += PT_THREADS) {
@@ -1993,6 +2008,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_prep_tc_kernel(PrefillP
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const unsigned tmem_base = *tmem_slot;
     const int wait_limit = P.wait_limit > 0 ? P.wait_limit : (1 << 24);
+    const bool fix_rows = P.pro.rope != nullptr;                // projected inputs: Algorithm 2 lines 1-2 on the staged rows
 #if WUSHKV_WS_TIMING
     if (tid == 0 && blockIdx.x == 0 && blockIdx.y == gridDim.y - 1) g_ws_t[8] += clock64() - t_entry;
 #endif
@@ -2027,7 +2043,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_prep_tc_kernel(PrefillP
             for (int i = 0; i < n_my_tiles; ++i) {
                 const int s = i & 1;
                 PST(0);
-                if (!ws_wait(bar(PB_XFULL + s), (i >> 1) & 1, wait_limit, abort_flag)) break;
+                if (!ws_wait(bar((fix_rows ? PB_XREADY : PB_XFULL) + s), (i >> 1) & 1, wait_limit, abort_flag)) break;
                 PST(1);
                 if (i >= 2 && !ws_wait(bar(PB_DEMPTY + s), ((i >> 1) - 1) & 1, wait_limit, abort_flag)) break;
                 PST(2);
@@ -2055,16 +2071,107 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_prep_tc_kernel(PrefillP
         float* qs_part = reinterpret_cast<float*>(sm_pt + PT_OFF_QS);      // [4][128] partial channel sums
         bool ok = true;
         PST_DECL;
+        // AND over the 512 epilogue threads (they meet at named barriers, so they give up together)
+        auto together = [&](const bool mine) -> bool {
+            unsigned all;
+            asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred p, 3, 512, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                         : "=r"(all) : "r"(mine ? 1u : 0u) : "memory");
+            return all != 0;
+        };
+        // Projected inputs: the rows of tile i, as the bulk tensor copies left them (128-byte-swizzled rows, channels 0-63 and
+        // 64-127 in two boxes), are normalised and rotated in place (Algorithm 2 lines 1-2: fp32, one rounding to bf16)
+        // before the MMAs may read them.
+        Prologue pro = P.pro;
+        pro.weight = is_key ? P.pro.weight : P.q_weight;
+        auto fix_tile = [&](const int i) -> bool {
+            const int s = i & 1, tok0 = (static_cast<int>(blockIdx.x) + i * static_cast<int>(gridDim.x)) * PREP_TOK;
+            PST(5);
+            if (!together(ws_wait(bar(PB_XFULL + s), (i >> 1) & 1, wait_limit, abort_flag))) return false;
+            PST(6);
+            unsigned char* xs = sm_pt + PT_OFF_X + s * PT_X_BYTES;
+            // four threads per row: thread q holds channels 16 q .. 16 q + 15 (two 16-byte chunks of the first box) and their
+            // rotation partners 64 + 16 q .. (the same chunks of the second box), so that a pair never leaves the thread
+            const int r = tid >> 2, q = tid & 3;
+            const bool valid = tok0 + r < P.total_new;      // rows past the chunk (zeros) go through the arithmetic and are not stored
+            const int tok = valid ? tok0 + r : P.total_new - 1;
+            {
+                int lo = 0, hi = P.batch, pos;              // the token's sequence by bisection of the chunk bounds, then its position
+                if (seq_in_smem) {
+                    while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (seq_first[mid] <= tok) lo = mid; else hi = mid; }
+                    pos = seq_base[lo] + tok;
+                } else {
+                    while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (__ldg(P.cu_new + mid) <= tok) lo = mid; else hi = mid; }
+                    const int f0 = __ldg(P.cu_new + lo), n_b = __ldg(P.cu_new + lo + 1) - f0;
+                    pos = __ldg(P.seq_len + lo) - n_b + (tok - f0);
+                }
+                pos = prologue_position(pro, pos, P.c.dev_status, q == 0 && valid);
+                uint4* cell[4];                             // [box][chunk]
+                uint4 raw[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    cell[k] = reinterpret_cast<uint4*>(xs + (k >> 1) * 16384 + r * 128 + (((2 * q + (k & 1)) ^ (r & 7)) << 4));
+                    raw[k] = *cell[k];
+                }
+                const float4* tab = reinterpret_cast<const float4*>(pro.rope + static_cast<long long>(pos) * (D / 2) + 16 * q);
+                float4 cs[8];                               // (cos, sin) of pairs 16 q .. 16 q + 15, two per load
+#pragma unroll
+                for (int k = 0; k < 8; ++k) cs[k] = __ldg(tab + k);
+                float x[4][8];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const unsigned w4[4] = {raw[k].x, raw[k].y, raw[k].z, raw[k].w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) { x[k][2 * e] = bf16_bits_to_float(w4[e] & 0xffff); x[k][2 * e + 1] = bf16_bits_to_float(w4[e] >> 16); }
+                }
+                if (pro.normalise) {
+                    float ss = 0.f;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) ss = fmaf(x[k][e], x[k][e], ss);
+                    ss += __shfl_xor_sync(FULLM, ss, 1);
+                    ss += __shfl_xor_sync(FULLM, ss, 2);
+                    const float rn = ss > 0.f ? 1.f / sqrtf(ss * (1.f / D) + pro.eps) : 0.f;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        float wv[8] = {1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f};
+                        if (pro.weight) {
+                            const float4* wp = reinterpret_cast<const float4*>(pro.weight + static_cast<long long>(head) * D + 64 * (k >> 1) + 16 * q + 8 * (k & 1));
+                            const float4 wa = __ldg(wp), wb = __ldg(wp + 1);
+                            wv[0] = wa.x; wv[1] = wa.y; wv[2] = wa.z; wv[3] = wa.w; wv[4] = wb.x; wv[5] = wb.y; wv[6] = wb.z; wv[7] = wb.w;
+                        }
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) x[k][e] *= pro.weight ? rn * wv[e] : rn;
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {               // chunk k of the first box with chunk k of the second
+                    unsigned oa[4], ob[4];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const float4 c2 = cs[4 * k + (e >> 1)];
+                        const float co = (e & 1) ? c2.z : c2.x, si = (e & 1) ? c2.w : c2.y;
+                        const float av = x[k][e], bv = x[2 + k][e];
+                        const unsigned ya = float_to_bf16_bits(fmaf(av, co, -bv * si)), yb = float_to_bf16_bits(fmaf(av, si, bv * co));
+                        if (e & 1) { oa[e >> 1] |= ya << 16; ob[e >> 1] |= yb << 16; } else { oa[e >> 1] = ya; ob[e >> 1] = yb; }
+                    }
+                    if (valid) {
+                        *cell[k] = make_uint4(oa[0], oa[1], oa[2], oa[3]);
+                        *cell[2 + k] = make_uint4(ob[0], ob[1], ob[2], ob[3]);
+                    }
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            ws_arrive(bar(PB_XREADY + s));
+            PST(7);
+            return true;
+        };
+        if (fix_rows) ok = fix_tile(0);
         for (int i = 0; i < n_my_tiles && ok; ++i) {
             const int s = i & 1, tok0 = (static_cast<int>(blockIdx.x) + i * static_cast<int>(gridDim.x)) * PREP_TOK;
+            if (fix_rows && i + 1 < n_my_tiles && !fix_tile(i + 1)) { ok = false; break; }
             PST(0);
-            {   // the give-up decision is taken by the 512 epilogue threads together (they meet at named barriers below)
-                const unsigned got = ws_wait(bar(PB_DFULL + s), (i >> 1) & 1, wait_limit, abort_flag) ? 1u : 0u;
-                unsigned all;
-                asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred p, 3, 512, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                             : "=r"(all) : "r"(got) : "memory");
-                if (!all) { ok = false; break; }
-            }
+            if (!together(ws_wait(bar(PB_DFULL + s), (i >> 1) & 1, wait_limit, abort_flag))) { ok = false; break; }
             PST(1);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             float o[32];
@@ -2195,9 +2302,10 @@ static int prefill_attn_impl(const wushkv_cache* cache, int32_t batch, const int
     {   // about one wave of CTAs: each keeps its head's transform resident and walks over token tiles
         const int n_tok_tiles = (total_new + PREP_TOK - 1) / PREP_TOK, slots = P.c.n_kv + P.c.n_q;
         const int per_slot = std::max(1, std::min(n_tok_tiles, sm_count() / slots));
-        // plain inputs: the tcgen05 kernel, fed by bulk tensor copies of the bf16 rows as they come
+        // the tcgen05 kernel, fed by bulk tensor copies of the bf16 rows as they come (projected rows are normalised and
+        // rotated in shared memory before the MMAs read them)
         CUtensorMap in_k, in_q;
-        const bool tc_prep = !P.pro.rope && !knobs().prefill_legacy && !knobs().prefill_no_tma &&
+        const bool tc_prep = !knobs().prefill_legacy && !knobs().prefill_no_tma &&
                              make_row_tensor_map(in_k, true, K_new, P.c.n_kv, total_new, PREP_TOK) &&
                              make_row_tensor_map(in_q, true, Q_new, P.c.n_q, total_new, PREP_TOK) &&
                              opt_in_dynamic_smem(reinterpret_cast<const void*>(prefill_prep_tc_kernel), PT_SMEM);

@@ -141,9 +141,13 @@ def test_projected_decode_matches_the_oracle(n_q, n_kv):
     assert fused.cache.status() == 0
 
 
-def test_projected_chunk_attention_matches_the_oracle():
+@pytest.mark.parametrize("copies", [0, 1])
+def test_projected_chunk_attention_matches_the_oracle(copies, test_option):
     """wushkv_prefill_attn_projected after wushkv_append_projected: a first chunk on the empty cache, then a second chunk
-    over it, against the oracle's chunk attention on oracle-prepared keys and queries (cache content: the GPU's codes)."""
+    over it, against the oracle's chunk attention on oracle-prepared keys and queries (cache content: the GPU's codes).
+    Once on the default kernels (tcgen05 transforms that normalise and rotate the rows the bulk tensor copies staged) and
+    once without bulk tensor copies (mma.sync transforms with their own row fix-up)."""
+    test_option("prefill_no_tma", copies)
     wl = _wl(53, 2, 8, 2, 2)
     lengths = [450, 290]
     plain, fused, masks, qproj = _pair(wl, lengths, 2, True)
