@@ -414,7 +414,8 @@ int wushkv_set_profile_events(void* start, void* stop);
  *   "prefill_no_tma"    1: the tcgen05 kernel stages the chunk's own tiles with 16-byte copies, not bulk tensor copies.
  *   "append_no_tma"     1: the same for the key / value tiles of the tensor-core chunk append.
  *   "drop_prefill"      1: the tcgen05 chunk attention never commits the score MMAs of a CTA's first tile; 2: it announces
- *                       but never issues one bulk copy of a CTA's first chunk tile (the bounded wait runs out either way).
+ *                       but never issues one bulk copy of a CTA's first chunk tile; 3: the tcgen05 transform kernel does the
+ *                       same with a copy of its first token tile (the bounded wait runs out in each case).
  * Returns WUSHKV_EINVAL for an unknown name.
  */
 int wushkv_set_test_option(const char* name, long long value);

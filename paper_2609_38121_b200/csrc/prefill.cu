@@ -73,7 +73,8 @@ struct PrefillParams {
     const float* q_weight;                // transform kernel (pro.weight: key weights, q_weight: query weights)
     int wait_limit;                       // poll limit of the barrier waits (0: default, a second or more)
     int drop;                             // testing aid: 1 the first tile's score MMAs are never committed, 2 the first bulk copy of a
-                                          // CTA's first chunk tile is announced but never issued (the wait then runs into its limit)
+                                          // CTA's first chunk tile is announced but never issued, 3 the same in the transform kernel
+                                          // (the wait then runs into its limit)
 };
 
 __device__ __forceinline__ unsigned smem_addr(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
@@ -2024,7 +2025,8 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_prep_tc_kernel(PrefillP
                 ws_expect_tx(bar(PB_XFULL + s), PT_X_BYTES);
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf)
-                    tma_load_3d(smem_addr(sm_pt + PT_OFF_X + s * PT_X_BYTES + hf * 16384), map, 64 * hf, head, tok0, bar(PB_XFULL + s));
+                    if (!(P.drop == 3 && i == 0 && hf == 0))    // testing aid: announced, never issued
+                        tma_load_3d(smem_addr(sm_pt + PT_OFF_X + s * PT_X_BYTES + hf * 16384), map, 64 * hf, head, tok0, bar(PB_XFULL + s));
                 if (s == 0) armed[0] = i; else armed[1] = i;
             }
             if (*abort_flag) {                                  // give announced copies a bounded time to land

@@ -54,6 +54,23 @@ def test_chunk_mma_that_is_never_committed_is_flagged(test_option):
     assert ok.check_decode_parity() <= 2e-3
 
 
+def test_chunk_transform_wait_that_runs_out_is_flagged(test_option):
+    """The tcgen05 transform kernel of the chunk attention with a bulk tensor copy that is announced but never issued: its
+    roles give up within the limit, the status bit is set, tensor memory is freed; the next call is healthy."""
+    from paper_2609_38121_b200 import binding as B
+    wl = _wl(8, 2, seed=67)
+    L = Layer(wl, [300], 2, 4, 64, 1)
+    test_option("drop_prefill", 3)
+    test_option("wait_limit", 2000)
+    L.prefill([300])
+    assert L.cache.status() & B.DEV_COPY_TIMEOUT
+    test_option("drop_prefill", 0)
+    test_option("wait_limit", 0)
+    ok = Layer(wl, [300], 2, 4, 64, 1)
+    assert ok.check_prefill_parity([300]) <= 2e-3
+    assert ok.cache.status() == 0
+
+
 @pytest.mark.parametrize("one_tile", [0, 1])
 @pytest.mark.parametrize("what", [1, 2])
 def test_chunk_attention_wait_that_runs_out_is_flagged(what, one_tile, test_option):
