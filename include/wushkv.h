@@ -411,6 +411,9 @@ int wushkv_set_profile_events(void* start, void* stop);
  *   "prefill_legacy"    1: wushkv_prefill_attn runs its mma.sync kernels (attention and transforms) instead of the tcgen05 ones.
  *   "prefill_one_tile"  1: the chunk attention runs on the tcgen05 kernel with one query tile per CTA and no role split
  *                       instead of the warp-specialised one.
+ *   "prefill_split"     n > 0: the warp-specialised chunk attention runs n CTAs per tile pair, each over a share of the key
+ *                       tiles, and merges their partial results (capped by what the workspace was sized for); 0: chosen from
+ *                       the number of tile pairs (several CTAs per pair only when the pairs alone would not fill the GPU).
  *   "prefill_no_tma"    1: the tcgen05 kernel stages the chunk's own tiles with 16-byte copies, not bulk tensor copies.
  *   "append_no_tma"     1: the same for the key / value tiles of the tensor-core chunk append.
  *   "drop_prefill"      1: the tcgen05 chunk attention never commits the score MMAs of a CTA's first tile; 2: it announces

@@ -31,6 +31,7 @@ extern "C" int wushkv_set_test_option(const char* name, long long value) {
     else if (!std::strcmp(name, "prefill_legacy")) k.prefill_legacy = value != 0;
     else if (!std::strcmp(name, "prefill_no_tma")) k.prefill_no_tma = value != 0;
     else if (!std::strcmp(name, "prefill_one_tile")) k.prefill_one_tile = value != 0;
+    else if (!std::strcmp(name, "prefill_split")) k.prefill_split = static_cast<int>(value);
     else if (!std::strcmp(name, "append_no_tma")) k.append_no_tma = value != 0;
     else if (!std::strcmp(name, "drop_prefill")) k.drop_prefill = static_cast<int>(value);
     else return WUSHKV_EINVAL;

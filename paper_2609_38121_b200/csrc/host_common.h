@@ -56,6 +56,7 @@ struct Knobs {
     int drop_chunk_mma = 0;         // 1: the chunk append never commits its first tile's MMAs to the barrier
     int prefill_legacy = 0;         // 1: chunk attention on the mma.sync kernel instead of the tcgen05 one
     int prefill_one_tile = 0;       // 1: chunk attention on the tcgen05 kernel with one query tile per CTA (no role split) instead of the warp-specialised one
+    int prefill_split = 0;          // > 0: CTAs per tile pair of the warp-specialised chunk attention (capped by what the workspace holds); 0: chosen by the grid size
     int prefill_no_tma = 0;         // 1: the tcgen05 kernel stages the chunk's tiles with 16-byte copies instead of bulk tensor copies
     int drop_prefill = 0;           // chunk attention: 1 the first tile's score MMAs are never committed, 2 one bulk copy is never issued, 3 one bulk copy of the transform kernel is never issued
     int append_no_tma = 0;          // 1: the chunk append stages its tiles with 16-byte copies instead of bulk tensor copies

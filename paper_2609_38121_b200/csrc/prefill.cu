@@ -71,6 +71,8 @@ struct PrefillParams {
     int use_tma;                          // 1: the tcgen05 kernel stages the chunk's own tiles with bulk tensor copies
     Prologue pro;                         // pro.rope != nullptr: K_new / Q_new are projected; Norm and RoPE are applied by the
     const float* q_weight;                // transform kernel (pro.weight: key weights, q_weight: query weights)
+    int n_split;                          // warp-specialised kernel: CTAs per tile pair, each over a share of the key tiles (1: none)
+    float* part;                          // n_split > 1: [n_split][total_new][n_q][PART_W] partial outputs
     int wait_limit;                       // poll limit of the barrier waits (0: default, a second or more)
     int drop;                             // testing aid: 1 the first tile's score MMAs are never committed, 2 the first bulk copy of a
                                           // CTA's first chunk tile is announced but never issued, 3 the same in the transform kernel
@@ -1214,9 +1216,12 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
 //   warps 12-15       write the other key / value tiles into the same rings: bf16 window rows, and packed pages (the raw
 //                     record arrives by a bulk copy one tile ahead and is unpacked into fp16 codes).
 // Registers are moved from warps 8-15 to the softmax warps (setmaxnreg, per group of four warps).
+// When the tile pairs of a call are too few to fill the GPU, n_split CTAs share a pair: each takes a contiguous share of the
+// pair's key tiles and writes a partial row (O + z, reference, sum) per query row; prefill_merge_kernel combines them.
 // Tensor memory (512 columns): query tile t owns columns 256 t .. 256 t + 255: O (128), two score buffers (64 each).
 // Every wait is bounded; a wait that runs out raises a CTA-wide flag that ends all roles.
 constexpr int WS_THREADS = 512;
+constexpr int PART_W = 132;                                      // floats of a partial row: O + z (128), reference, sum, padding
 constexpr int WS_KS = 2, WS_VS = 3;                              // ring depths of the key / value stages: a key stage is free again when
                                                                  // its scores are done, a value stage only after O += P V a softmax later
 constexpr int WS_OFF_Q = 0;                                      // (tile 0 value, remainder), (tile 1 value, remainder)
@@ -1305,9 +1310,12 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
     const CacheView& c = P.c;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = c.G, R = TM / G;                              // chunk positions per query tile
+    // n_split CTAs share a tile pair: each takes a contiguous share of the pair's key tiles and leaves a partial result
+    // (short chunks over long caches would otherwise occupy a few SMs only)
+    const int n_split = P.n_split, sp = static_cast<int>(blockIdx.x % n_split), bx = static_cast<int>(blockIdx.x / n_split);
     const int pairs = (P.tiles_per_seq + 1) >> 1;
-    const int pr = pairs - 1 - static_cast<int>(blockIdx.x % pairs);      // long pairs first
-    const int b = blockIdx.x / pairs, h = blockIdx.y;
+    const int pr = pairs - 1 - bx % pairs;                      // long pairs first
+    const int b = bx / pairs, h = blockIdx.y;
     const int first = __ldg(P.cu_new + b), n_new = __ldg(P.cu_new + b + 1) - first;
     if (2 * pr * R >= n_new) return;
     const int S = __ldg(P.seq_len + b), sl = __ldg(P.slot + b);
@@ -1345,18 +1353,27 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
     const int c_lo = max(q_hi, a_hi);
     const int n_old_fp = a_hi + max(S0 - c_lo, 0);
     const float k2 = c.sm_scale * LOG2E_F;
-    const int nA = (n_old_fp + TN - 1) / TN;                    // tiles of full-precision old positions
+    const int nA_all = (n_old_fp + TN - 1) / TN;                // tiles of full-precision old positions
     const int page_first = q_lo / PAGE_TOKENS;
-    const int nB = q_hi > q_lo ? (q_hi - 1) / PAGE_TOKENS - page_first + 1 : 0;      // packed pages
-    const int gC = nA + nB;                                     // first tile of the chunk itself
+    const int nB_all = q_hi > q_lo ? (q_hi - 1) / PAGE_TOKENS - page_first + 1 : 0;      // packed pages
+    const int gC_all = nA_all + nB_all;                         // first tile of the chunk itself
     int n_rows[2], n_tiles[2];
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
         const int qt = 2 * pr + t, np = min(R, n_new - qt * R);
         n_rows[t] = max(np, 0) * G;
-        n_tiles[t] = np > 0 ? gC + (min(qt * R + R, n_new) - 1) / TN + 1 : 0;
+        n_tiles[t] = np > 0 ? gC_all + (min(qt * R + R, n_new) - 1) / TN + 1 : 0;
     }
-    const int NT = max(n_tiles[0], n_tiles[1]);
+    // This CTA's share [g0, g0 + NT) of the pair's key tiles.  From here on tiles are counted from g0: nA and gC are the
+    // (possibly negative, possibly beyond NT) local indices where the packed pages and the chunk's own tiles begin.
+    const int NT_all = max(n_tiles[0], n_tiles[1]);
+    const int g0 = static_cast<int>(static_cast<long long>(NT_all) * sp / n_split);
+    const int NT = static_cast<int>(static_cast<long long>(NT_all) * (sp + 1) / n_split) - g0;
+    const int nA = nA_all - g0, gC = gC_all - g0;
+#pragma unroll
+    for (int t = 0; t < 2; ++t) n_tiles[t] = min(max(n_tiles[t] - g0, 0), NT);
+    const int n_staged = P.use_tma ? min(max(gC, 0), NT) : NT;                // tiles written by the staging threads
+    const int gb_first = max(-nA, 0), gb_end = max(min(gC, NT) - nA, gb_first);      // this CTA's packed pages [gb_first, gb_end)
     const int wait_limit = P.wait_limit > 0 ? P.wait_limit : (1 << 24);      // polls of at least ~60 ns each: a second or more
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -1521,7 +1538,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 // valid keys of the tile and the chunk row of its first key (old positions: visible to every row)
                 int nv = TN, crow0 = FAR_BELOW;
                 bool masked = false;
-                if (g < nA) { nv = min(TN, n_old_fp - g * TN); masked = nv < TN; }
+                if (g < nA) { nv = min(TN, n_old_fp - (g + g0) * TN); masked = nv < TN; }
                 else if (g >= gC) {
                     const int kt = g - gC;
                     nv = min(TN, n_new - kt * TN); crow0 = kt * TN;
@@ -1540,8 +1557,10 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
             if (ok && !__all_sync(FULLM, ws_wait(bar(WB_PV + 2 * t + ((n_tiles[t] - 1) & 1)), ((n_tiles[t] - 1) >> 1) & 1, wait_limit, abort_flag))) ok = false;
             if (ok) {
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const float inv = l > 0.f ? 1.f / l : 0.f;
-                float* dst = P.O + (static_cast<long long>(my_tok) * c.n_q + my_jq) * D;
+                // alone: o = (O + z) / l; one of several CTAs of the pair: the partial (O + z, reference, l) for the merge
+                const float inv = n_split > 1 ? 1.f : (l > 0.f ? 1.f / l : 0.f);
+                float* dst = n_split > 1 ? P.part + ((static_cast<long long>(sp) * P.total_new + my_tok) * c.n_q + my_jq) * PART_W
+                                         : P.O + (static_cast<long long>(my_tok) * c.n_q + my_jq) * D;
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
                     float o[32];
@@ -1552,7 +1571,16 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                             *reinterpret_cast<float4*>(dst + 32 * q4 + i) = make_float4((o[i] + z) * inv, (o[i + 1] + z) * inv, (o[i + 2] + z) * inv, (o[i + 3] + z) * inv);
                     }
                 }
+                if (n_split > 1 && wt < n_rows[t]) *reinterpret_cast<float2*>(dst + D) = make_float2(m_ref, l);
             }
+        } else if (n_split > 1 && wt < n_rows[t]) {
+            // none of this CTA's key tiles is the tile's: an empty partial (reference -inf, sum 0)
+            const int qt = 2 * pr + t;
+            const int my_tok = first + qt * R + wt / G, my_jq = h * G + wt % G;
+            float* dst = P.part + ((static_cast<long long>(sp) * P.total_new + my_tok) * c.n_q + my_jq) * PART_W;
+#pragma unroll
+            for (int i = 0; i < D; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(0.f, 0.f, 0.f, 0.f);
+            *reinterpret_cast<float2*>(dst + D) = make_float2(-INFINITY, 0.f);
         }
     }
     else if (warp < 12) {
@@ -1676,14 +1704,14 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
         // for the first chunk tiles means: once the staging threads' last tiles went through).
         int armed[3] = {-1, -1, -1};                            // last tile whose copies this warp announced on each stage (<= 3 stages)
         bool ok = true;
-        if (P.use_tma && gC > 0) ok = __all_sync(FULLM, ws_wait(bar(WB_STAGED), 0u, wait_limit, abort_flag));
+        if (P.use_tma && n_staged > 0) ok = __all_sync(FULLM, ws_wait(bar(WB_STAGED), 0u, wait_limit, abort_flag));
         if (P.use_tma) {
             const bool keys = warp == 9;
             const int depth = keys ? WS_KS : WS_VS, full0 = keys ? WB_KFULL : WB_VFULL, empty0 = keys ? WB_KEMPTY : WB_VEMPTY;
             const CUtensorMap* map = keys ? &map_k : &map_v;
             unsigned char* ring = sm_ws + (keys ? WS_OFF_K : WS_OFF_V);
             WST_DECL;
-            for (int g = gC; g < NT && ok; ++g) {
+            for (int g = max(gC, 0); g < NT && ok; ++g) {
                 const int st = g % depth, row = first + (g - gC) * TN;
                 WST(0);
                 if (g >= depth && !__all_sync(FULLM, ws_wait(bar(empty0 + st), ((g / depth) - 1) & 1, wait_limit, abort_flag))) { ok = false; break; }
@@ -1721,7 +1749,6 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
         // =============================== staging of key / value tiles by threads ===========================
         asm volatile("setmaxnreg.dec.sync.aligned.u32 88;" ::: "memory");
         const int ptid = tid - 384;
-        const int n_staged = P.use_tma ? gC : NT;               // tiles written by the 128 threads
         int raw_uses[2] = {0, 0};                               // records fetched so far into each raw buffer
         auto page_of = [&](const int gb) -> int {               // page id of packed tile gb, -1 if it cannot be read
             const int pg = page_first + gb;
@@ -1739,8 +1766,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                         bar(WB_RAW + (gb & 1)));
         };
         // page ids are read two tiles ahead, so that neither the record request nor the unpacking waits for the page table
-        int page_cur = nB > 0 ? page_of(0) : -1, page_next = nB > 1 ? page_of(1) : -1;
-        if (nB > 0 && ptid == 0) fetch_record(0, page_cur);
+        int page_cur = gb_end > gb_first ? page_of(gb_first) : -1, page_next = gb_end > gb_first + 1 ? page_of(gb_first + 1) : -1;
+        if (gb_end > gb_first && ptid == 0) fetch_record(gb_first, page_cur);
         bool ok = true;
         WST_DECL;
         for (int g = 0; g < n_staged && ok; ++g) {
@@ -1757,7 +1784,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
             if (g < nA) {
                 // ---- full-precision old positions: sink [0, a_hi) and recent window [c_lo, S0), bf16 rows
                 for (int item = ptid; item < TN * 16 && mine; item += 128) {
-                    const int r = item & (TN - 1), piece = item >> 6, idx = g * TN + r;
+                    const int r = item & (TN - 1), piece = item >> 6, idx = (g + g0) * TN + r;
                     uint4 kh = make_uint4(0, 0, 0, 0), vh = kh;
                     if (idx < n_old_fp) {
                         const long long plane = (static_cast<long long>(sl) * c.n_kv + h) * 2;
@@ -1787,10 +1814,10 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 // ---- a packed page: the record was requested one tile ahead; unpack it into integer codes (exact in fp16)
                 const int gb = g - nA, rb = gb & 1;
                 // the other raw buffer was last read for tile gb - 1, which every staging thread has left
-                if (gb + 1 < nB && ptid == 0) fetch_record(gb + 1, page_next);
+                if (gb + 1 < gb_end && ptid == 0) fetch_record(gb + 1, page_next);
                 const bool page_ok = page_cur >= 0;
                 page_cur = page_next;
-                page_next = gb + 2 < nB ? page_of(gb + 2) : -1;
+                page_next = gb + 2 < gb_end ? page_of(gb + 2) : -1;
                 if (page_ok && mine) mine = __all_sync(FULLM, ws_wait(bar(WB_RAW + rb), raw_uses[rb] & 1, wait_limit, abort_flag));
                 if (page_ok) ++raw_uses[rb];
                 const unsigned char* raw = sm_ws + WS_OFF_RAW + rb * REC;
@@ -1851,7 +1878,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
         if (tid == 384 && *abort_flag) {                        // give the record copies a bounded time to land
 #pragma unroll
             for (int i = 0; i < 2; ++i)
-                if (nB > i) for (int it = 0; it < 64 && !ws_wait(bar(WB_RAW + i), raw_uses[i] & 1, 1, abort_flag); ++it) __nanosleep(2000);
+                if (gb_end > gb_first) for (int it = 0; it < 64 && !ws_wait(bar(WB_RAW + i), raw_uses[i] & 1, 1, abort_flag); ++it) __nanosleep(2000);
         }
     }
 
@@ -1874,6 +1901,33 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+}
+
+// Merge of the partial results of the n_split CTAs of a tile pair: one CTA of 128 threads (one per channel) per
+// (query head, chunk token).  A partial holds O + z relative to its own reference m (2^m was factored out of its
+// probabilities) and the sum l of those probabilities; the output is sum_s 2^(m_s - M) (O + z)_s / sum_s 2^(m_s - M) l_s.
+__global__ void __launch_bounds__(D) prefill_merge_kernel(PrefillParams P) {
+    const CacheView& c = P.c;
+    const int jq = blockIdx.x, tok = blockIdx.y, ch = threadIdx.x;
+    {   // a sequence the attention kernel skipped leaves no partials: its rows stay untouched here as well
+        int lo = 0, hi = P.batch;
+        while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (__ldg(P.cu_new + mid) <= tok) lo = mid; else hi = mid; }
+        const int n_new = __ldg(P.cu_new + lo + 1) - __ldg(P.cu_new + lo), sl = __ldg(P.slot + lo);
+        if (sl < 0 || sl >= c.n_slots || __ldg(P.seq_len + lo) < n_new) return;
+    }
+    const long long row = static_cast<long long>(tok) * c.n_q + jq, stride = static_cast<long long>(P.total_new) * c.n_q * PART_W;
+    const float* p0 = P.part + row * PART_W;
+    float M = -INFINITY;
+    for (int s = 0; s < P.n_split; ++s) M = fmaxf(M, __ldcg(p0 + s * stride + D));
+    float acc = 0.f, lsum = 0.f;
+    for (int s = 0; s < P.n_split; ++s) {
+        const float m = __ldcg(p0 + s * stride + D);
+        if (m == -INFINITY) continue;
+        const float w = fast_ex2(m - M);
+        acc = fmaf(w, __ldcg(p0 + s * stride + ch), acc);
+        lsum = fmaf(w, __ldcg(p0 + s * stride + D + 1), lsum);
+    }
+    P.O[row * D + ch] = lsum > 0.f ? acc / lsum : 0.f;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -2241,7 +2295,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_prep_tc_kernel(PrefillP
 
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
-struct PrefillPlan { size_t off_kp, off_vp, off_qp, off_qsum, total; };
+struct PrefillPlan { size_t off_kp, off_vp, off_qp, off_qsum, off_part, total; int max_split; };
 bool make_prefill_plan(const CacheView& c, int total_new, PrefillPlan& pl) {
     if (total_new <= 0) return false;
     size_t off = 0;
@@ -2249,6 +2303,13 @@ bool make_prefill_plan(const CacheView& c, int total_new, PrefillPlan& pl) {
     pl.off_vp = off;   off = align256(off + static_cast<size_t>(total_new) * c.n_kv * D * sizeof(__half));
     pl.off_qp = off;   off = align256(off + 2 * static_cast<size_t>(total_new) * c.n_q * D * sizeof(__half));
     pl.off_qsum = off; off = align256(off + static_cast<size_t>(total_new) * c.n_q * sizeof(float));
+    // Partial results of the warp-specialised attention kernel when a call has too few tile pairs to fill the GPU: at
+    // least ceil(total_new / (2 R)) pairs per KV head exist, so at most sm_count / that many CTAs per pair are worth it.
+    const int R = 128 / c.G;
+    const long long min_ctas = (static_cast<long long>(total_new) + 2 * R - 1) / (2 * R) * c.n_kv;
+    pl.max_split = static_cast<int>(std::max<long long>(1, std::min<long long>(16, sm_count() / std::max<long long>(min_ctas, 1))));
+    pl.off_part = off;
+    if (pl.max_split > 1) off = align256(off + static_cast<size_t>(pl.max_split) * total_new * c.n_q * 132 * sizeof(float));
     pl.total = off;
     return true;
 }
@@ -2291,6 +2352,8 @@ static int prefill_attn_impl(const wushkv_cache* cache, int32_t batch, const int
     P.batch = batch; P.total_new = total_new; P.slot = slot; P.seq_len = seq_len; P.cu_new = cu_new;
     P.K_new = K_new; P.V_new = V_new; P.Q_new = Q_new; P.O = O;
     P.use_tma = 0;
+    P.n_split = 1;
+    P.part = nullptr;
     P.wait_limit = static_cast<int>(std::min<long long>(std::max<long long>(knobs().wait_limit, 0), 1 << 30));
     P.drop = knobs().drop_prefill;
     P.KP = reinterpret_cast<__half*>(ws + pl.off_kp);
@@ -2343,7 +2406,13 @@ static int prefill_attn_impl(const wushkv_cache* cache, int32_t batch, const int
         const bool mv = make_row_tensor_map(map_v, false, P.VP, P.c.n_kv, total_new, TN);
         P.use_tma = (mk && mv && !knobs().prefill_no_tma) ? 1 : 0;
         if (!knobs().prefill_one_tile) {        // warp-specialised kernel: a pair of query tiles per CTA
-            const dim3 grid_ws(static_cast<unsigned>(batch) * ((P.tiles_per_seq + 1) / 2), P.c.n_kv);
+            // few pairs (a short chunk): several CTAs per pair, each over a share of the key tiles, then a merge
+            const long long n_pairs = static_cast<long long>(batch) * ((P.tiles_per_seq + 1) / 2) * P.c.n_kv;
+            int n_split = static_cast<int>(std::max<long long>(1, std::min<long long>(pl.max_split, sm_count() / std::max<long long>(n_pairs, 1))));
+            if (knobs().prefill_split > 0) n_split = std::min(knobs().prefill_split, pl.max_split);
+            P.n_split = n_split;
+            P.part = reinterpret_cast<float*>(ws + pl.off_part);
+            const dim3 grid_ws(static_cast<unsigned>(batch) * ((P.tiles_per_seq + 1) / 2) * n_split, P.c.n_kv);
             // the query operands (value, remainder) as [token][query head][128 channels]: a box is one tile's (G heads, R positions)
             CUtensorMap map_q0, map_q1;
             const bool mq = make_row_tensor_map(map_q0, false, P.QP, P.c.n_q, total_new, R, P.c.G) &&
@@ -2358,6 +2427,7 @@ static int prefill_attn_impl(const wushkv_cache* cache, int32_t batch, const int
                             : P.c.bits == 3 ? launch_ws(prefill_attn_ws_kernel<3>, ws_smem(3))
                                             : launch_ws(prefill_attn_ws_kernel<4>, ws_smem(4));
             if (!ok) return WUSHKV_ECUDA;
+            if (n_split > 1) prefill_merge_kernel<<<dim3(P.c.n_q, total_new), D, 0, st>>>(P);
 #if WUSHKV_WS_TIMING
             {
                 cudaDeviceSynchronize();

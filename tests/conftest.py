@@ -32,7 +32,7 @@ def test_option():
     defaults when the test ends."""
     from paper_2609_38121_b200 import binding as B
     defaults = {"decode_ctas": 0, "append_path_cuda": 0, "host_io_copy": 0, "drop_copy_unit": -1, "wait_limit": 0,
-                "drop_chunk_mma": 0, "prefill_legacy": 0, "prefill_one_tile": 0, "prefill_no_tma": 0, "append_no_tma": 0, "drop_prefill": 0}
+                "drop_chunk_mma": 0, "prefill_legacy": 0, "prefill_one_tile": 0, "prefill_split": 0, "prefill_no_tma": 0, "append_no_tma": 0, "drop_prefill": 0}
     used = []
 
     def _set(name, value):

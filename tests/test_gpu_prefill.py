@@ -62,6 +62,21 @@ def test_head_group_sizes(n_q, n_kv):
     assert L.cache.status() == 0
 
 
+@pytest.mark.parametrize("split", [1, 2, 3, 7, 16])
+@pytest.mark.parametrize("bits", [2, 4])
+def test_key_tiles_shared_between_ctas(split, bits, attention_path, test_option):
+    """A short chunk over a long cache with the pair's key tiles cut into 1 .. 16 shares (one CTA each, partial results merged):
+    shares that hold only packed pages, only the chunk's own tiles, nothing at all for the earlier query tile, or no tile."""
+    if not attention_path.startswith("tcgen05") or "one_tile" in attention_path:
+        pytest.skip("shares exist in the warp-specialised kernel only")
+    test_option("prefill_split", split)
+    wl = _wl(8, 2, seed=99, batch=2)
+    L = Layer(wl, [1300, 200], bits, 4, 64, 8)
+    L.append_step([1200, 120])
+    assert L.check_prefill_parity([100, 80]) <= 2e-3
+    assert L.cache.status() == 0
+
+
 def test_chunk_attention_is_bit_identical_from_run_to_run():
     """The same call on the same cache state three times: the roles of the warp-specialised kernel meet in an order that
     depends on timing, the arithmetic must not (tile order of every accumulation is fixed)."""
