@@ -237,7 +237,9 @@ int wushkv_decode_attn(const wushkv_cache* cache, int32_t batch, const int32_t* 
  *   O (device, out): fp32 [total_new][n_q][d] in the folded value basis.
  *   workspace (device): >= wushkv_prefill_workspace_bytes() bytes, 256-byte aligned, scratch.
  * Both contractions run on the tcgen05 tensor cores (fp16 operands, fp32 accumulators in tensor memory); q' enters as
- * an fp16 value plus its fp16 rounding remainder.  The query heads of a KV head share one 128-row tile.
+ * an fp16 value plus its fp16 rounding remainder.  The query heads of a KV head share one 128-row tile.  A call whose
+ * chunk is too short to fill the GPU with tiles splits every tile's keys over several CTAs and merges their partial
+ * results (the workspace holds them); the result does not depend on timing, only on the call's shapes.
  */
 size_t wushkv_prefill_workspace_bytes(const wushkv_cache* cache, int32_t batch, int32_t total_new);
 int wushkv_prefill_attn(const wushkv_cache* cache, int32_t batch, const int32_t* slot, const int32_t* seq_len,
