@@ -1904,11 +1904,11 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
 }
 
 // Merge of the partial results of the n_split CTAs of a tile pair: one CTA of 128 threads (one per channel) per
-// (query head, chunk token).  A partial holds O + z relative to its own reference m (2^m was factored out of its
+// (chunk token, query head).  A partial holds O + z relative to its own reference m (2^m was factored out of its
 // probabilities) and the sum l of those probabilities; the output is sum_s 2^(m_s - M) (O + z)_s / sum_s 2^(m_s - M) l_s.
 __global__ void __launch_bounds__(D) prefill_merge_kernel(PrefillParams P) {
     const CacheView& c = P.c;
-    const int jq = blockIdx.x, tok = blockIdx.y, ch = threadIdx.x;
+    const int tok = blockIdx.x, jq = blockIdx.y, ch = threadIdx.x;
     {   // a sequence the attention kernel skipped leaves no partials: its rows stay untouched here as well
         int lo = 0, hi = P.batch;
         while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (__ldg(P.cu_new + mid) <= tok) lo = mid; else hi = mid; }
@@ -2427,7 +2427,7 @@ static int prefill_attn_impl(const wushkv_cache* cache, int32_t batch, const int
                             : P.c.bits == 3 ? launch_ws(prefill_attn_ws_kernel<3>, ws_smem(3))
                                             : launch_ws(prefill_attn_ws_kernel<4>, ws_smem(4));
             if (!ok) return WUSHKV_ECUDA;
-            if (n_split > 1) prefill_merge_kernel<<<dim3(P.c.n_q, total_new), D, 0, st>>>(P);
+            if (n_split > 1) prefill_merge_kernel<<<dim3(total_new, P.c.n_q), D, 0, st>>>(P);
 #if WUSHKV_WS_TIMING
             {
                 cudaDeviceSynchronize();
