@@ -118,14 +118,16 @@ def test_quest_cache_under_a_chunk():
     assert L.cache.status() == 0
 
 
-def test_long_chunk_over_a_long_quantized_cache(attention_path):
+@pytest.mark.parametrize("chunk", [2048, 96])
+def test_long_chunk_over_a_long_quantized_cache(chunk, attention_path):
     """A 2048-token chunk appended to a 32768-token cache (512 packed pages, then the window rows, then 32 causal
-    chunk tiles), sampled chunk rows against the oracle."""
+    chunk tiles; two CTAs per tile pair), and a 96-token chunk over the same cache (16 CTAs per tile pair, 33 key tiles
+    each); sampled chunk rows against the oracle."""
     if attention_path != "tcgen05":
         pytest.skip("the long case runs on the default kernel only")
     wl = _wl(8, 2, seed=97, theta=5e5)
-    L = Layer(wl, [32768 + 2048], 2, 4, 128, 1)
+    L = Layer(wl, [32768 + chunk], 2, 4, 128, 1)
     L.append_step([32768])
-    worst = L.check_prefill_parity([2048], rows=[0, 1, 17, 63, 64, 1023, 1024, 2000, 2047])
+    worst = L.check_prefill_parity([chunk], rows=[r for r in (0, 1, 17, 63, 64, 95, 1023, 1024, 2000, 2047) if r < chunk])
     assert worst <= 2e-3
     assert L.cache.status() == 0
