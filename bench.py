@@ -87,7 +87,7 @@ def library_transforms(wl):
 class Session:
     """A filled cache plus the per-step inputs of one config, resident on one GPU."""
 
-    def __init__(self, name, n_steps, device="cuda", seed_offset=0, verbose=False, bits=None):
+    def __init__(self, name, n_steps, device="cuda", seed_offset=0, verbose=False, bits=None, cached=0, chunk=0):
         import torch
         from paper_2609_38121_b200 import binding as B
         self.torch, self.B = torch, B
@@ -95,16 +95,22 @@ class Session:
         cfg["seed"] += 1000 * seed_offset
         if bits:
             cfg["bits"] = bits
+        if chunk and cfg["prefill_chunk"]:
+            cfg["prefill_chunk"] = cfg["ctx"] = int(chunk)
         self.name, self.cfg = name, cfg
         wl = self.wl = W.LayerWorkload(cfg)
         self.n_steps = n_steps
         self.chunk = cfg["prefill_chunk"]
         self.batch = wl.batch
         final = wl.lengths().astype(np.int64)
+        # prefill config only: `cached` tokens per sequence already sit in the cache (quantized, apart from the
+        # recent window) when the chunk arrives, so the chunk attention also reads packed pages
+        self.cached = int(cached) if self.chunk else 0
+        final = final + self.cached
         self.T, self.TinvT, self.TV = library_transforms(wl)
         self.s_flush = 1
         if self.chunk:
-            self.start_len = np.zeros(self.batch, np.int64)
+            self.start_len = np.full(self.batch, self.cached, np.int64)
             self.max_seq_len = int(final.max())
         else:
             self.start_len = final - 1
@@ -118,13 +124,13 @@ class Session:
         if self.chunk:
             ks, vs = [], []
             for b in range(self.batch):
-                _, K, V = next(wl.sequence_tokens(b, self.chunk, T_V=self.TV, chunk=self.chunk))
-                ks.append(K)
-                vs.append(V)
+                K, V = self.host_tokens(b)
+                ks.append(K[self.cached:])
+                vs.append(V[self.cached:])
             self.K_chunk = self._dev_bf16(np.concatenate(ks))
             self.V_chunk = self._dev_bf16(np.concatenate(vs))
             self.cu_chunk = torch.arange(0, (self.batch + 1) * self.chunk, self.chunk, dtype=torch.int32, device=dev)
-            self.q_chunk_host = np.concatenate([wl.chunk_queries(b, np.arange(self.chunk)) for b in range(self.batch)])
+            self.q_chunk_host = np.concatenate([wl.chunk_queries(b, self.cached + np.arange(self.chunk)) for b in range(self.batch)])
             self.Q_chunk = self._dev_bf16(self.q_chunk_host)
             self.O_chunk = torch.zeros((self.batch * self.chunk, wl.n_q, 128), dtype=torch.float32, device=dev)
             self.pf_bytes = B.prefill_workspace_bytes(self.cache.desc, self.batch, self.batch * self.chunk)
@@ -138,9 +144,12 @@ class Session:
         for b in range(self.batch):
             n_pre = int(self.start_len[b])
             ks, vs = [], []
-            for _, K, V in wl.sequence_tokens(b, n_pre + n_step_tok, T_V=self.TV):
-                ks.append(K)
-                vs.append(V)
+            if self.cached:
+                ks, vs = [[x] for x in self.host_tokens(b)]     # the stream whose tail is the chunk
+            else:
+                for _, K, V in wl.sequence_tokens(b, n_pre + n_step_tok, T_V=self.TV):
+                    ks.append(K)
+                    vs.append(V)
             K = np.concatenate(ks) if ks else np.zeros((0, wl.n_kv, 128), np.float32)
             V = np.concatenate(vs) if vs else np.zeros((0, wl.n_kv, 128), np.float32)
             if n_step_tok:
@@ -164,6 +173,8 @@ class Session:
         self.ws_bytes = B.decode_workspace_bytes(self.cache.desc, self.batch, self.max_seq_len)
         self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device=dev)
         self.base_len = self.seq_len.clone()
+        # rolling a sequence back to `cached` tokens also needs its recent window as it was then
+        self.ring_base = self.cache.ring_kv.clone() if self.cached else None
         self.final = final
         self.step_index = 0
         if verbose:
@@ -172,9 +183,12 @@ class Session:
     def host_tokens(self, b):
         """The (K, V) token rows of sequence b exactly as the constructor generated them (same stream,
         same chunking), positions 0 .. : used by tests to recompute sampled pieces with the oracle."""
-        if self.chunk:
+        if self.chunk and not self.cached:
             _, K, V = next(self.wl.sequence_tokens(b, self.chunk, T_V=self.TV, chunk=self.chunk))
             return K, V
+        if self.chunk:               # the cached tokens followed by the chunk's, one stream
+            toks = list(self.wl.sequence_tokens(b, self.cached + self.chunk, T_V=self.TV))
+            return np.concatenate([t[1] for t in toks]), np.concatenate([t[2] for t in toks])
         toks = list(self.wl.sequence_tokens(b, int(self.start_len[b]) + self.n_steps, T_V=self.TV))
         return np.concatenate([t[1] for t in toks]), np.concatenate([t[2] for t in toks])
 
@@ -196,7 +210,9 @@ class Session:
             self.step_index += 1
             return
         if self.chunk:
-            self.seq_len.zero_()
+            self.seq_len.copy_(self.base_len)
+            if self.ring_base is not None:
+                self.cache.ring_kv.copy_(self.ring_base)
             B.append(self.cache.desc, self.batch, self.slot, self.seq_len, self.cu_chunk, self.batch * self.chunk,
                      self.chunk, self.K_chunk, self.V_chunk)
         else:
@@ -234,14 +250,25 @@ class Session:
         return self.batch * (self.chunk if self.chunk else 1)
 
     def prefill_flops(self):
-        """Multiply-adds x 2 of the chunk attention (causal: row i sees i + 1 keys; both contractions)."""
+        """Multiply-adds x 2 of the chunk attention (causal: row i sees the cached tokens and i + 1 keys of the
+        chunk; both contractions)."""
         n = self.chunk
-        return 4.0 * 128 * self.wl.n_q * self.batch * (n * (n + 1) / 2)
+        return 4.0 * 128 * self.wl.n_q * self.batch * (n * self.cached + n * (n + 1) / 2)
 
     def launches_per_step(self):
         # chunk append: transform/quantize kernel + length update (+ prefill attention: preparation + attention);
         # token append: one kernel; decode: prep + main + combine
-        return (4 if self.chunk else 1) + 3
+        n = (4 if self.chunk else 1) + 3
+        if self.chunk:
+            # few query-tile pairs (a short chunk): the attention runs several CTAs per pair and a merge kernel follows
+            R = 128 // (self.wl.n_q // self.wl.n_kv)
+            tiles = -(-self.chunk // R)
+            pairs = self.batch * ((tiles + 1) // 2) * self.wl.n_kv
+            min_ctas = -(-self.batch * self.chunk // (2 * R)) * self.wl.n_kv
+            sms = self.torch.cuda.get_device_properties(self.cache.device).multi_processor_count
+            if min(max(1, min(16, sms // max(min_ctas, 1))), max(1, sms // pairs)) > 1:
+                n += 1
+        return n
 
 
 # ------------------------------------------------------------------------------------------------
@@ -516,7 +543,10 @@ def run_ours(args, rank, world):
     torch.cuda.set_device(local)
     K, Wm = args.steps, args.warmup
     n_total_steps = Wm + K            # device-timed region
-    sess = Session(args.config, n_steps=3 * n_total_steps + 2, seed_offset=rank, verbose=(rank == 0 and args.verbose), bits=args.bits)
+    if (args.cached_context or args.prefill_chunk) and not W.CONFIGS[args.config]["prefill_chunk"]:
+        raise SystemExit("--cached-context and --prefill-chunk apply to a prefill config (cfg4)")
+    sess = Session(args.config, n_steps=3 * n_total_steps + 2, seed_offset=rank, verbose=(rank == 0 and args.verbose), bits=args.bits,
+                   cached=args.cached_context, chunk=args.prefill_chunk)
     cache_bytes = sess.decode_bytes(1)
     need_flush = cache_bytes < 2 * L2_BYTES
     flush_buf = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device="cuda") if need_flush else None
@@ -711,9 +741,9 @@ def run_ours(args, rank, world):
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": args.config + (f"@{args.bits}bit" if args.bits else ""), "batch": sess.batch, "n_q": c["n_q"], "n_kv": c["n_kv"], "head_dim": 128,
+        "config": {"workload": args.config + (f"@{args.bits}bit" if args.bits else "") + (f"+chunk{sess.chunk}" if args.prefill_chunk else "") + (f"+cached{sess.cached}" if sess.cached else ""), "batch": sess.batch, "n_q": c["n_q"], "n_kv": c["n_kv"], "head_dim": 128,
                    "context": int(sess.final.max()), "bits": c["bits"], "s_sink": c["s_sink"], "s_keep": c["s_keep"],
-                   "s_flush": sess.s_flush, "page_tokens": 64, "prefill_chunk": sess.chunk,
+                   "s_flush": sess.s_flush, "page_tokens": 64, "prefill_chunk": sess.chunk, "cached_context": sess.cached,
                    "l2": ("flushed between steps (256 MB write)" if need_flush else "cache read per step exceeds L2 (no flush)"),
                    "replicas": world},
         "roofline": roofline, "roofline_append": roofline_append, "cpu_baseline": cpu, "e2e": e2e,
@@ -740,6 +770,11 @@ def main():
     ap.add_argument("--sustained-seconds", type=float, default=1.0)
     ap.add_argument("--bits", type=int, default=0, choices=[0, 2, 3, 4],
                     help="override the configuration's bit width (0: as the configuration says); the workload name then carries it")
+    ap.add_argument("--cached-context", type=int, default=0,
+                    help="prefill config: tokens per sequence already in the cache when the chunk arrives (default 0); "
+                         "not the headline configuration: a second workload, the chunk attention over packed pages")
+    ap.add_argument("--prefill-chunk", type=int, default=0,
+                    help="prefill config: tokens per sequence in the chunk (default: the config's own)")
     ap.add_argument("--verbose", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)

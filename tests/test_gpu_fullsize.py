@@ -136,3 +136,49 @@ def test_full_size_config(name, groups):
         for (b, h) in groups:
             errs = _check_prefill_rows(sess, o_chunk, b, h, rows)
             assert max(errs) <= 2e-3, f"{name}: prefill rows of sequence {b} KV head {h}: {max(errs):.3e}"
+
+
+def test_chunk_over_cached_context():
+    """The bench's second prefill workload: config 4's heads, a 512-token chunk per sequence arriving on 4096 cached
+    tokens.  Two steps, so the second one starts from the rolled-back cache (lengths and recent window restored):
+    codes around the roll-back point, sampled chunk rows and the decode that follows, each against the oracle."""
+    import torch
+    cached, chunk = 4096, 512
+    sess = bench.Session("cfg4", n_steps=4, cached=cached, chunk=chunk)
+    assert sess.chunk == chunk and sess.cached == cached
+    for _ in range(2):
+        sess.step()
+    torch.cuda.synchronize()
+    assert sess.cache.status() == 0
+    S_all = sess.seq_len.cpu().numpy()
+    assert np.all(S_all == cached + chunk)
+    cfg, wl = sess.cfg, sess.wl
+    G, S = wl.G, cached + chunk
+    # positions that left the recent window while the chunk was appended: quantized from the restored window rows
+    n_diff, n_codes = _check_append_samples(sess, 3, [(cached - 300, 600)])
+    assert n_codes == 2 * wl.n_kv * 128 * 600
+    assert n_diff <= 1e-4 * n_codes, (n_diff, n_codes)
+    out = sess.O.cpu().numpy().astype(np.float64)
+    o_chunk = sess.O_chunk.cpu().numpy().astype(np.float64).reshape(sess.batch, chunk, wl.n_q, 128)
+    assert np.all(np.isfinite(o_chunk))
+    q_all = sess.q_chunk_host.reshape(sess.batch, chunk, wl.n_q, 128)
+    rows = [0, 1, 17, 18, 255, 256, chunk - 2, chunk - 1]
+    for (b, h) in [(0, 0), (3, 2), (7, 3)]:
+        assert _check_decode_group(sess, out, b, h) <= 2e-3
+        kc, ks, kz = _unpack(sess, b, h, 0, 0, S)
+        vc, vs, vz = _unpack(sess, b, h, 1, 0, S)
+        km = np.stack([ks, kz], axis=1)[:, None, :]
+        vm = np.stack([vs, vz], axis=1)[:, None, :]
+        K, V = sess.host_tokens(b)
+        kb = np.full((S, 1, 128), np.nan)
+        vb = np.full((S, 1, 128), np.nan)
+        sink = sess.cache.sink_kv[b, h].float().cpu().numpy().astype(np.float64)
+        kb[:cfg["s_sink"], 0], vb[:cfg["s_sink"], 0] = sink[0], sink[1]
+        kb[cached:, 0] = O.round_bf16(O.key_transform(sess.T[h].astype(np.float64), K[cached:, h]))
+        vb[cached:, 0] = V[cached:, h]
+        ref = O.chunk_attn(q_all[b][:, h * G:(h + 1) * G], sess.TinvT[h:h + 1].astype(np.float64), kc[:, None], km, vc[:, None], vm,
+                           kb, vb, S, chunk, cfg["s_sink"], cfg["s_keep"], sess.s_flush, 1.0 / np.sqrt(128), rows=rows)
+        for r in rows:
+            got = o_chunk[b, r, h * G:(h + 1) * G]
+            err = np.max(np.abs(got - ref[r])) / np.max(np.abs(ref[r]))
+            assert err <= 2e-3, f"sequence {b} KV head {h} chunk row {r}: {err:.3e}"
