@@ -736,7 +736,7 @@ __device__ __forceinline__ void unpack_chunk8(const unsigned char* raw, int r, i
     vout = make_uint4(vo[0], vo[1], vo[2], vo[3]);
 }
 
-// A whole page (all 64 tokens live) as fp16 integer codes, by 128 threads: instead of gathering eight channels of a token
+// A whole page (all 64 tokens live) as fp16 key codes and fp16 values, by 128 threads: instead of gathering eight channels of a token
 // from 16-bit loads (unpack_chunk8), a thread reads the record the way it is laid out and scatters 16-byte chunks.
 //   keys:   thread (block bi, k-step s, fragment row g) loads the four 16-byte pieces of row g (fragment lanes t = 0..3: words
 //           j = rs + 2 hh, bytes b = 2 b1 + b0; the field of k-step s in a byte = channel 32 s + 16 hh + 8 b1 + 2 t + b0 of
@@ -746,10 +746,13 @@ __device__ __forceinline__ void unpack_chunk8(const unsigned char* raw, int r, i
 //           eight pieces (e, tt) (half-word hi = token 8 ps + 2 tt + hi, field i = channel 16 i + 8 rsel + e) and writes, for
 //           (hi, i in 4 ih .. 4 ih + 3), the chunk of channels 8 (2 i + rsel) .. + 7 of that token: element e.
 //   3 bits: the 2-bit plane as above plus the high bit of every code from the 1-bit planes (csrc/layout.cuh).
+// Keys are left as integer codes (exact in fp16; their factors are applied to the scores in fp32).  Values are written
+// dequantized, step * code + offset in one fp16 rounding: the probabilities that multiply them are fp16 already, and the
+// softmax then treats a packed page's values like any other's.
 template <int BITS>
 __device__ __forceinline__ void unpack_page(const unsigned char* raw, unsigned char* sK, unsigned char* sV, const int p) {
     constexpr bool TWO = BITS != 4;                         // 2-bit fields (also the low plane of 3-bit records)
-    constexpr unsigned MASK = TWO ? 3u : 15u, MASK_HI = MASK << 16;
+    constexpr unsigned MASK = TWO ? 3u : 15u, MASK_HI = MASK << 16, MASK2 = MASK * 0x00010001u;
     constexpr int CB = code_block_bytes(BITS);
     const __half2 bias = __halves2half2(__ushort_as_half(0x6400), __ushort_as_half(0x6400));
     auto to_h2 = [&](const unsigned pair) {             // two codes (low bits of each half) -> fp16 pair: 1024 + c, minus 1024
@@ -757,10 +760,21 @@ __device__ __forceinline__ void unpack_page(const unsigned char* raw, unsigned c
         const __half2 hv = __hsub2(*reinterpret_cast<const __half2*>(&w), bias);
         return *reinterpret_cast<const unsigned*>(&hv);
     };
+    // Two codes that sit at bit f of bytes 0 and 2 of `bytes` -> fp16 pair: (1024 + c 2^f) 2^-f - 1024 2^-f = c, one
+    // fused multiply-add (exact: c 2^f < 1024); mul = 2^-f and add = -2^(10 - f) in both halves.
+    auto field_h2 = [](const unsigned bytes, const unsigned mask, const unsigned mul, const unsigned add) {
+        const unsigned w = (bytes & mask) | 0x64006400u;
+        const __half2 hv = __hfma2(*reinterpret_cast<const __half2*>(&w), *reinterpret_cast<const __half2*>(&mul),
+                                   *reinterpret_cast<const __half2*>(&add));
+        return *reinterpret_cast<const unsigned*>(&hv);
+    };
+    auto pow2_neg = [](const int f) { return (0x3C00u - (static_cast<unsigned>(f) << 10)) * 0x00010001u; };            // 2^-f
+    auto bias_neg = [](const int f) { return (0x8000u | (static_cast<unsigned>(25 - f) << 10)) * 0x00010001u; };      // -2^(10 - f)
     {
         const int g = p & 7, s = (p >> 3) & 3, bi = p >> 5;
         const unsigned char* src = raw + bi * CB + (TWO ? 0 : 512 * (s >> 1)) + 64 * g;
         const int sh0 = TWO ? 2 * s : 4 * (s & 1);
+        const unsigned kmask = MASK2 << sh0, kmul = pow2_neg(sh0), kadd = bias_neg(sh0);
         unsigned w[4][4];                                   // [t][j]
         unsigned wh[4][2];                                  // 3 bits: [t][rs], bit 2 s + hh of byte b
 #pragma unroll
@@ -779,13 +793,16 @@ __device__ __forceinline__ void unpack_page(const unsigned char* raw, unsigned c
                 unsigned out[4];
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
-                    const unsigned x = w[t][j] >> (16 * b1 + sh0);
-                    unsigned pair = (x & MASK) | ((x << 8) & MASK_HI);
-                    if (BITS == 3) {
+                    if constexpr (BITS == 3) {
+                        const unsigned x = w[t][j] >> (16 * b1 + sh0);
+                        unsigned pair = (x & MASK) | ((x << 8) & MASK_HI);
                         const unsigned y = wh[t][j & 1] >> (16 * b1 + 2 * s + (j >> 1));
                         pair |= ((y & 1u) | ((y << 8) & 0x00010000u)) << 2;
+                        out[t] = to_h2(pair);
+                    } else {
+                        // bytes 2 b1 and 2 b1 + 1 of the word to bytes 0 and 2, then the thread's field of each
+                        out[t] = field_h2(__byte_perm(w[t][j], 0u, b1 ? 0x4342u : 0x4140u), kmask, kmul, kadd);
                     }
-                    out[t] = to_h2(pair);
                 }
                 *reinterpret_cast<uint4*>(sK + (2 * bi + (j & 1)) * 2048 + (4 * s + 2 * (j >> 1) + b1) * 128 + g * 16) =
                     make_uint4(out[0], out[1], out[2], out[3]);
@@ -803,6 +820,14 @@ __device__ __forceinline__ void unpack_page(const unsigned char* raw, unsigned c
         }
 #pragma unroll
         for (int hi = 0; hi < 2; ++hi) {
+            // the values are staged dequantized: step and offset of this half-word's token, in both halves of a pair
+            const unsigned mv = *reinterpret_cast<const unsigned*>(raw + meta_location(BITS, 16 * bi + 8 * ps + 2 * tt + hi) + 4);
+            const unsigned step2 = __byte_perm(mv, mv, 0x1010u), offs2 = __byte_perm(mv, mv, 0x3232u);
+            auto dequant = [&](const unsigned codes) {
+                const __half2 hv = __hfma2(*reinterpret_cast<const __half2*>(&codes), *reinterpret_cast<const __half2*>(&step2),
+                                           *reinterpret_cast<const __half2*>(&offs2));
+                return *reinterpret_cast<const unsigned*>(&hv);
+            };
 #pragma unroll
             for (int ii = 0; ii < 4; ++ii) {
                 const int i = 4 * ih + ii, sh = 16 * hi + (TWO ? 2 * i : 4 * ii);
@@ -811,9 +836,16 @@ __device__ __forceinline__ void unpack_page(const unsigned char* raw, unsigned c
                 unsigned out[4];
 #pragma unroll
                 for (int e2 = 0; e2 < 4; ++e2) {
-                    unsigned c0 = (w[2 * e2] >> sh) & MASK, c1 = (w[2 * e2 + 1] >> sh) & MASK;
-                    if (BITS == 3) { c0 |= ((wh[2 * e2] >> hb) & 1u) << 2; c1 |= ((wh[2 * e2 + 1] >> hb) & 1u) << 2; }
-                    out[e2] = to_h2(c0 | (c1 << 16));
+                    if constexpr (BITS == 3) {
+                        unsigned c0 = (w[2 * e2] >> sh) & MASK, c1 = (w[2 * e2 + 1] >> sh) & MASK;
+                        c0 |= ((wh[2 * e2] >> hb) & 1u) << 2; c1 |= ((wh[2 * e2 + 1] >> hb) & 1u) << 2;
+                        out[e2] = dequant(to_h2(c0 | (c1 << 16)));
+                    } else {
+                        // the byte that holds the field, of both words, to bytes 0 and 2 (the same for the fields of one byte)
+                        const int byte = TWO ? 2 * hi + ih : 2 * hi + (ii >> 1), f = TWO ? 2 * ii : 4 * (ii & 1);
+                        const unsigned both = __byte_perm(w[2 * e2], w[2 * e2 + 1], 0x0400u + 0x0101u * static_cast<unsigned>(byte));
+                        out[e2] = dequant(field_h2(both, MASK2 << f, pow2_neg(f), bias_neg(f)));
+                    }
                 }
                 *reinterpret_cast<uint4*>(sV + (2 * i + rsel) * 1024 + (2 * bi + ps) * 128 + (2 * tt + hi) * 16) =
                     make_uint4(out[0], out[1], out[2], out[3]);
@@ -1217,11 +1249,11 @@ __global__ void __launch_bounds__(TM, 2) prefill_attn_tc_kernel(PrefillParams P,
 //                     record arrives by a bulk copy one tile ahead and is unpacked into fp16 codes).
 // Registers are moved from warps 8-15 to the softmax warps (setmaxnreg, per group of four warps).
 // When the tile pairs of a call are too few to fill the GPU, n_split CTAs share a pair: each takes a contiguous share of the
-// pair's key tiles and writes a partial row (O + z, reference, sum) per query row; prefill_merge_kernel combines them.
+// pair's key tiles and writes a partial row (O, reference, sum) per query row; prefill_merge_kernel combines them.
 // Tensor memory (512 columns): query tile t owns columns 256 t .. 256 t + 255: O (128), two score buffers (64 each).
 // Every wait is bounded; a wait that runs out raises a CTA-wide flag that ends all roles.
 constexpr int WS_THREADS = 512;
-constexpr int PART_W = 132;                                      // floats of a partial row: O + z (128), reference, sum, padding
+constexpr int PART_W = 132;                                      // floats of a partial row: O (128), reference, sum, padding
 constexpr int WS_KS = 2, WS_VS = 3;                              // ring depths of the key / value stages: a key stage is free again when
                                                                  // its scores are done, a value stage only after O += P V a softmax later
 constexpr int WS_OFF_Q = 0;                                      // (tile 0 value, remainder), (tile 1 value, remainder)
@@ -1232,10 +1264,8 @@ enum { WB_KFULL = 0, WB_KEMPTY = WB_KFULL + WS_KS, WB_VFULL = WB_KEMPTY + WS_KS,
        WB_S = WB_VEMPTY + WS_VS, WB_PV = WB_S + 4, WB_PREADY = WB_PV + 4, WB_RAW = WB_PREADY + 4, WB_Q = WB_RAW + 2,
        WB_STAGED, WB_DRAIN, WB_COUNT };
 // The rest of the layout depends on the record size.  Per-key factors of a packed tile, per value stage: (step, offset) of
-// the key side for the 64 keys, then of the value side; as fp32 pairs where the record leaves room for them (2 and 3 bits:
-// the softmax threads then load them ready to use, two keys per 16-byte load), as the record's fp16 pairs at 4 bits.
-__host__ __device__ constexpr bool ws_meta32(int bits) { return bits != 4; }
-__host__ __device__ constexpr int ws_meta_stage(int bits) { return 2 * TN * (ws_meta32(bits) ? 8 : 4); }
+// the key side for the 64 keys as fp32 pairs (the softmax threads load them ready to use, two keys per 16-byte load).
+__host__ __device__ constexpr int ws_meta_stage(int) { return TN * 8; }
 __host__ __device__ constexpr int ws_off_meta(int bits) { return WS_OFF_RAW + 2 * record_bytes(bits); }
 __host__ __device__ constexpr int ws_off_live(int bits) { return ws_off_meta(bits) + WS_VS * ws_meta_stage(bits); }      // uint2[WS_VS]: which keys of a packed tile exist
 __host__ __device__ constexpr int ws_off_bar(int bits) { return ws_off_live(bits) + WS_VS * 8; }
@@ -1283,6 +1313,9 @@ __device__ __forceinline__ bool ws_stagers_and(bool pred) {
     return r != 0;
 }
 
+#ifndef WUSHKV_EXP
+#define WUSHKV_EXP 0
+#endif
 #ifndef WUSHKV_WS_TIMING
 #define WUSHKV_WS_TIMING 0      // timing experiments only: per-role cycle counters of CTA (0, 0)
 #endif
@@ -1305,7 +1338,6 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                                                                         const __grid_constant__ CUtensorMap map_q1) {
     extern __shared__ __align__(1024) unsigned char sm_ws[];
     constexpr int REC = record_bytes(BITS);
-    constexpr bool META32 = ws_meta32(BITS);
     constexpr int META_STAGE = ws_meta_stage(BITS);
     const CacheView& c = P.c;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -1412,12 +1444,12 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
             const int my_row = qt * R + my_r / G;               // this row sees the chunk's rows 0 .. my_row
             const int tile_row_lo = qt * R;                     // smallest such limit of the tile
             const unsigned tmem_row = tmem_base + (static_cast<unsigned>((warp & 3) * 32) << 16) + 256u * t;
-            float m_ref = -INFINITY, l = 0.f, z = 0.f;
+            float m_ref = -INFINITY, l = 0.f;
             bool ok = true;
             WST_DECL;
 
-            // One key tile.  PACKED: the keys carry affine factors (a packed page; factors and the set of existing keys
-            // come with the value stage).  MASKED: key j exists if bit j of (live_lo, live_hi) is set and is visible to
+            // One key tile.  PACKED: the keys are integer codes that carry affine factors (a packed page; the factors and the
+            // set of existing keys come with the value stage; the values of a packed page are staged dequantized).  MASKED: key j exists if bit j of (live_lo, live_hi) is set and is visible to
             // this row if crow0 + j <= my_row (crow0: chunk row of the tile's first key, very negative for old positions).
             auto soft = [&](auto packed_tag, auto masked_tag, const int g, unsigned live_lo, unsigned live_hi, const int crow0) {
                 constexpr bool PACKED = decltype(packed_tag)::value, MASKED = decltype(masked_tag)::value;
@@ -1426,15 +1458,10 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 // one barrier per score buffer: its next phase (tile g + 2) cannot complete before this tile's probabilities are ready
                 if (!__all_sync(FULLM, ws_wait(bar(WB_S + 2 * t + (g & 1)), (g >> 1) & 1, wait_limit, abort_flag))) { ok = false; return; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const unsigned char* kmeta = meta_all + (g % WS_VS) * META_STAGE, *vmeta = kmeta + META_STAGE / 2;
+                const unsigned char* kmeta = meta_all + (g % WS_VS) * META_STAGE;
                 auto factors4 = [&](const unsigned char* side, const int j4, float2 (&f)[4]) {      // (step, offset) of keys 4 j4 .. 4 j4 + 3
-                    if constexpr (META32) {
-                        const float4 a = reinterpret_cast<const float4*>(side)[2 * j4], b2 = reinterpret_cast<const float4*>(side)[2 * j4 + 1];
-                        f[0] = make_float2(a.x, a.y); f[1] = make_float2(a.z, a.w); f[2] = make_float2(b2.x, b2.y); f[3] = make_float2(b2.z, b2.w);
-                    } else {
-                        const uint4 m4 = reinterpret_cast<const uint4*>(side)[j4];
-                        f[0] = h2f2u(m4.x); f[1] = h2f2u(m4.y); f[2] = h2f2u(m4.z); f[3] = h2f2u(m4.w);
-                    }
+                    const float4 a = reinterpret_cast<const float4*>(side)[2 * j4], b2 = reinterpret_cast<const float4*>(side)[2 * j4 + 1];
+                    f[0] = make_float2(a.x, a.y); f[1] = make_float2(a.z, a.w); f[2] = make_float2(b2.x, b2.y); f[3] = make_float2(b2.z, b2.w);
                 };
                 if (PACKED) {
                     if (!__all_sync(FULLM, ws_wait(bar(WB_VFULL + g % WS_VS), (g / WS_VS) & 1, wait_limit, abort_flag))) { ok = false; return; }
@@ -1497,28 +1524,21 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                     }
                 }
                 WST(4);
-                l *= factor; z *= factor;
+                l *= factor;
                 m_ref = new_ref;
                 const float ref = m_ref == -INFINITY ? 0.f : m_ref;
-                // ---- probabilities: (p Delta_v) as fp16 pairs over the first 32 columns of the score buffer just read
+                // ---- probabilities as fp16 pairs over the first 32 columns of the score buffer just read
                 float2 lsum = make_float2(0.f, 0.f);                       // two partial sums
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {                     // 32 keys = 16 columns of fp16 pairs at a time
                     unsigned pk[16];
 #pragma unroll
                     for (int e4 = 0; e4 < 8; ++e4) {                       // four keys = two fp16 pairs at a time
-                        float2 mv[4];
-                        if (PACKED) factors4(vmeta, 8 * half + e4, mv);
 #pragma unroll
                         for (int q = 0; q < 2; ++q) {
                             const int e = 16 * half + 2 * e4 + q;
-                            float2 pr = make_float2(fast_ex2(fmaf(s[2 * e], k2, -ref)), fast_ex2(fmaf(s[2 * e + 1], k2, -ref)));     // k2 s - ref in one rounding
+                            const float2 pr = make_float2(fast_ex2(fmaf(s[2 * e], k2, -ref)), fast_ex2(fmaf(s[2 * e + 1], k2, -ref)));     // k2 s - ref in one rounding
                             lsum.x += pr.x; lsum.y += pr.y;
-                            if (PACKED) {
-                                const float2 mv0 = mv[2 * q], mv1 = mv[2 * q + 1];
-                                z = fmaf(pr.x, mv0.y, fmaf(pr.y, mv1.y, z));
-                                pr.x *= mv0.x; pr.y *= mv1.x;
-                            }
                             pk[2 * e4 + q] = pack_half2(pr.x, pr.y);
                         }
                     }
@@ -1548,16 +1568,20 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 const unsigned live_lo = nv >= 32 ? 0xffffffffu : (1u << nv) - 1u;
                 const unsigned live_hi = nv >= TN ? 0xffffffffu : nv > 32 ? (1u << (nv - 32)) - 1u : 0u;
                 // (one call per variant, so that each is expanded in place)
+#if WUSHKV_EXP == 1
+                if (g >= nA && g < gC) soft(std::false_type{}, std::false_type{}, g, 0u, 0u, FAR_BELOW);
+#else
                 if (g >= nA && g < gC) soft(std::true_type{}, std::true_type{}, g, 0u, 0u, FAR_BELOW);
+#endif
                 else if (masked) soft(std::false_type{}, std::true_type{}, g, live_lo, live_hi, crow0);
                 else soft(std::false_type{}, std::false_type{}, g, 0u, 0u, 0);
             }
             WST_FLUSH;
-            // ---- output: o = (O + z) / l for the rows that carry a query
+            // ---- output: o = O / l for the rows that carry a query
             if (ok && !__all_sync(FULLM, ws_wait(bar(WB_PV + 2 * t + ((n_tiles[t] - 1) & 1)), ((n_tiles[t] - 1) >> 1) & 1, wait_limit, abort_flag))) ok = false;
             if (ok) {
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                // alone: o = (O + z) / l; one of several CTAs of the pair: the partial (O + z, reference, l) for the merge
+                // alone: o = O / l; one of several CTAs of the pair: the partial (O, reference, l) for the merge
                 const float inv = n_split > 1 ? 1.f : (l > 0.f ? 1.f / l : 0.f);
                 float* dst = n_split > 1 ? P.part + ((static_cast<long long>(sp) * P.total_new + my_tok) * c.n_q + my_jq) * PART_W
                                          : P.O + (static_cast<long long>(my_tok) * c.n_q + my_jq) * D;
@@ -1568,7 +1592,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                     if (wt < n_rows[t]) {
 #pragma unroll
                         for (int i = 0; i < 32; i += 4)
-                            *reinterpret_cast<float4*>(dst + 32 * q4 + i) = make_float4((o[i] + z) * inv, (o[i + 1] + z) * inv, (o[i + 2] + z) * inv, (o[i + 3] + z) * inv);
+                            *reinterpret_cast<float4*>(dst + 32 * q4 + i) = make_float4(o[i] * inv, o[i + 1] * inv, o[i + 2] * inv, o[i + 3] * inv);
                     }
                 }
                 if (n_split > 1 && wt < n_rows[t]) *reinterpret_cast<float2*>(dst + D) = make_float2(m_ref, l);
@@ -1824,29 +1848,39 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 const uint4 zero4 = make_uint4(0, 0, 0, 0);
                 const int page_pos = (page_first + gb) * PAGE_TOKENS;
                 const bool whole = page_ok && page_pos >= q_lo && page_pos + PAGE_TOKENS <= q_hi;
+#if WUSHKV_EXP == 2
+                if (whole && mine && gb < 4) unpack_page<BITS>(raw, sK, sV, ptid);
+#else
                 if (whole && mine) unpack_page<BITS>(raw, sK, sV, ptid);
+#endif
 #pragma unroll 4
                 for (int item = ptid; item < (mine && !whole ? TN * 16 : 0); item += 128) {      // first / last page of the range
                     const int r = item & (TN - 1), kc = item >> 6;
                     const int pos = (page_first + gb) * PAGE_TOKENS + r;
                     const bool live = page_ok && pos >= q_lo && pos < q_hi;
                     uint4 kq = zero4, vq = zero4;
-                    if (live) unpack_chunk8<BITS>(raw, r, kc, kq, vq);
+                    if (live) {
+                        unpack_chunk8<BITS>(raw, r, kc, kq, vq);
+                        // values are staged dequantized (see unpack_page)
+                        const unsigned mv = *reinterpret_cast<const unsigned*>(raw + meta_location(BITS, r) + 4);
+                        const unsigned step2 = __byte_perm(mv, mv, 0x1010u), offs2 = __byte_perm(mv, mv, 0x3232u);
+                        unsigned* vw = reinterpret_cast<unsigned*>(&vq);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const __half2 hv = __hfma2(*reinterpret_cast<const __half2*>(vw + e), *reinterpret_cast<const __half2*>(&step2),
+                                                       *reinterpret_cast<const __half2*>(&offs2));
+                            vw[e] = *reinterpret_cast<const unsigned*>(&hv);
+                        }
+                    }
                     *reinterpret_cast<uint4*>(sK + (r >> 3) * 2048 + kc * 128 + (r & 7) * 16) = kq;
                     *reinterpret_cast<uint4*>(sV + kc * 1024 + (r >> 3) * 128 + (r & 7) * 16) = vq;
                 }
-                if (mine && ptid < TN) {                        // warps 12 and 13: factors and existence of key ptid
+                if (mine && ptid < TN) {                        // warps 12 and 13: key factors and existence of key ptid
                     const int pos = (page_first + gb) * PAGE_TOKENS + ptid;
                     const bool live = page_ok && pos >= q_lo && pos < q_hi;
-                    const uint2 m = live ? *reinterpret_cast<const uint2*>(raw + meta_location(BITS, ptid)) : make_uint2(0u, 0u);
-                    unsigned char* kside = meta_all + vs * META_STAGE, *vside = kside + META_STAGE / 2;
-                    if constexpr (META32) {
-                        reinterpret_cast<float2*>(kside)[ptid] = h2f2u(m.x);
-                        reinterpret_cast<float2*>(vside)[ptid] = h2f2u(m.y);
-                    } else {
-                        reinterpret_cast<unsigned*>(kside)[ptid] = m.x;
-                        reinterpret_cast<unsigned*>(vside)[ptid] = m.y;
-                    }
+                    const unsigned mk = live ? *reinterpret_cast<const unsigned*>(raw + meta_location(BITS, ptid)) : 0u;
+                    unsigned char* kside = meta_all + vs * META_STAGE;
+                    reinterpret_cast<float2*>(kside)[ptid] = h2f2u(mk);
                     const unsigned word = __ballot_sync(FULLM, live);
                     if (lane == 0) reinterpret_cast<unsigned*>(live_all + vs)[ptid >> 5] = word;
                 }
@@ -1904,8 +1938,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
 }
 
 // Merge of the partial results of the n_split CTAs of a tile pair: one CTA of 128 threads (one per channel) per
-// (chunk token, query head).  A partial holds O + z relative to its own reference m (2^m was factored out of its
-// probabilities) and the sum l of those probabilities; the output is sum_s 2^(m_s - M) (O + z)_s / sum_s 2^(m_s - M) l_s.
+// (chunk token, query head).  A partial holds O relative to its own reference m (2^m was factored out of its
+// probabilities) and the sum l of those probabilities; the output is sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.
 __global__ void __launch_bounds__(D) prefill_merge_kernel(PrefillParams P) {
     const CacheView& c = P.c;
     const int tok = blockIdx.x, jq = blockIdx.y, ch = threadIdx.x;
