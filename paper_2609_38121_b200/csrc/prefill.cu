@@ -810,24 +810,27 @@ __device__ __forceinline__ void unpack_page(const unsigned char* raw, unsigned c
         }
     }
     {
-        const int tt = p & 3, ih = (p >> 2) & 1, m = (p >> 3) & 3, bi = p >> 5, ps = m >> 1, rsel = m & 1;
-        const unsigned char* src = raw + v_codes_offset(BITS) + bi * CB + (TWO ? 4 * m : 512 * ps + 4 * (2 * rsel + ih)) + 16 * tt;
-        unsigned w[8], wh[8];                               // [e]; 3 bits: the word of token half ps (both half-words)
+        // (the half-word hi is a lane bit: the eight lanes of a quarter warp then write the eight 16-byte pieces of one 128-byte row)
+        const int tt = p & 3, hi = (p >> 2) & 1, m = (p >> 3) & 3, bi = p >> 5, ps = m >> 1, rsel = m & 1;
+        const unsigned char* src = raw + v_codes_offset(BITS) + bi * CB + (TWO ? 4 * m : 512 * ps + 8 * rsel) + 16 * tt;
+        // the values are staged dequantized: step and offset of this thread's token, in both halves of a pair
+        const unsigned mv = *reinterpret_cast<const unsigned*>(raw + meta_location(BITS, 16 * bi + 8 * ps + 2 * tt + hi) + 4);
+        const unsigned step2 = __byte_perm(mv, mv, 0x1010u), offs2 = __byte_perm(mv, mv, 0x3232u);
+        auto dequant = [&](const unsigned codes) {
+            const __half2 hv = __hfma2(*reinterpret_cast<const __half2*>(&codes), *reinterpret_cast<const __half2*>(&step2),
+                                       *reinterpret_cast<const __half2*>(&offs2));
+            return *reinterpret_cast<const unsigned*>(&hv);
+        };
+        unsigned wa[TWO ? 1 : 2][8], wh[8];                 // [ih][e] (2-bit fields: one word holds both); 3 bits: the word of token half ps
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-            w[e] = *reinterpret_cast<const unsigned*>(src + 64 * e);
+            wa[0][e] = *reinterpret_cast<const unsigned*>(src + 64 * e);
+            if (!TWO) wa[TWO ? 0 : 1][e] = *reinterpret_cast<const unsigned*>(src + 64 * e + 4);
             if (BITS == 3) wh[e] = *reinterpret_cast<const unsigned*>(raw + v_hi_offset(3) + bi * 256 + 8 * (4 * e + tt) + 4 * ps);
         }
 #pragma unroll
-        for (int hi = 0; hi < 2; ++hi) {
-            // the values are staged dequantized: step and offset of this half-word's token, in both halves of a pair
-            const unsigned mv = *reinterpret_cast<const unsigned*>(raw + meta_location(BITS, 16 * bi + 8 * ps + 2 * tt + hi) + 4);
-            const unsigned step2 = __byte_perm(mv, mv, 0x1010u), offs2 = __byte_perm(mv, mv, 0x3232u);
-            auto dequant = [&](const unsigned codes) {
-                const __half2 hv = __hfma2(*reinterpret_cast<const __half2*>(&codes), *reinterpret_cast<const __half2*>(&step2),
-                                           *reinterpret_cast<const __half2*>(&offs2));
-                return *reinterpret_cast<const unsigned*>(&hv);
-            };
+        for (int ih = 0; ih < 2; ++ih) {                    // half of the channel blocks
+            const unsigned (&w)[8] = wa[TWO ? 0 : ih];
 #pragma unroll
             for (int ii = 0; ii < 4; ++ii) {
                 const int i = 4 * ih + ii, sh = 16 * hi + (TWO ? 2 * i : 4 * ii);
@@ -1313,9 +1316,6 @@ __device__ __forceinline__ bool ws_stagers_and(bool pred) {
     return r != 0;
 }
 
-#ifndef WUSHKV_EXP
-#define WUSHKV_EXP 0
-#endif
 #ifndef WUSHKV_WS_TIMING
 #define WUSHKV_WS_TIMING 0      // timing experiments only: per-role cycle counters of CTA (0, 0)
 #endif
@@ -1568,11 +1568,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 const unsigned live_lo = nv >= 32 ? 0xffffffffu : (1u << nv) - 1u;
                 const unsigned live_hi = nv >= TN ? 0xffffffffu : nv > 32 ? (1u << (nv - 32)) - 1u : 0u;
                 // (one call per variant, so that each is expanded in place)
-#if WUSHKV_EXP == 1
-                if (g >= nA && g < gC) soft(std::false_type{}, std::false_type{}, g, 0u, 0u, FAR_BELOW);
-#else
                 if (g >= nA && g < gC) soft(std::true_type{}, std::true_type{}, g, 0u, 0u, FAR_BELOW);
-#endif
                 else if (masked) soft(std::false_type{}, std::true_type{}, g, live_lo, live_hi, crow0);
                 else soft(std::false_type{}, std::false_type{}, g, 0u, 0u, 0);
             }
@@ -1848,11 +1844,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
                 const uint4 zero4 = make_uint4(0, 0, 0, 0);
                 const int page_pos = (page_first + gb) * PAGE_TOKENS;
                 const bool whole = page_ok && page_pos >= q_lo && page_pos + PAGE_TOKENS <= q_hi;
-#if WUSHKV_EXP == 2
-                if (whole && mine && gb < 4) unpack_page<BITS>(raw, sK, sV, ptid);
-#else
                 if (whole && mine) unpack_page<BITS>(raw, sK, sV, ptid);
-#endif
 #pragma unroll 4
                 for (int item = ptid; item < (mine && !whole ? TN * 16 : 0); item += 128) {      // first / last page of the range
                     const int r = item & (TN - 1), kc = item >> 6;
