@@ -91,23 +91,10 @@ __device__ __forceinline__ void hmma(float (&c)[4], unsigned a0, unsigned a1, un
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ float fast_ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
-// three-input maximum and packed fp32 arithmetic (two lanes per instruction)
+// three-input maximum
 __device__ __forceinline__ float max3f(float a, float b, float c) {
     float d;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
-__device__ __forceinline__ float2 fma2f(float2 a, float m, float c) {        // (a.x m + c, a.y m + c)
-    float2 d;
-    asm("{\n\t.reg .b64 va, vm, vc, vd;\n\tmov.b64 va, {%2, %3};\n\tmov.b64 vm, {%4, %4};\n\tmov.b64 vc, {%5, %5};\n\t"
-        "fma.rn.f32x2 vd, va, vm, vc;\n\tmov.b64 {%0, %1}, vd;\n\t}"
-        : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(m), "f"(c));
-    return d;
-}
-__device__ __forceinline__ float2 add2f(float2 a, float2 b) {
-    float2 d;
-    asm("{\n\t.reg .b64 va, vb, vd;\n\tmov.b64 va, {%2, %3};\n\tmov.b64 vb, {%4, %5};\n\tadd.rn.f32x2 vd, va, vb;\n\tmov.b64 {%0, %1}, vd;\n\t}"
-        : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
     return d;
 }
 __device__ __forceinline__ unsigned pack_half2(float lo, float hi) {
@@ -752,18 +739,13 @@ __device__ __forceinline__ void unpack_chunk8(const unsigned char* raw, int r, i
 template <int BITS>
 __device__ __forceinline__ void unpack_page(const unsigned char* raw, unsigned char* sK, unsigned char* sV, const int p) {
     constexpr bool TWO = BITS != 4;                         // 2-bit fields (also the low plane of 3-bit records)
-    constexpr unsigned MASK = TWO ? 3u : 15u, MASK_HI = MASK << 16, MASK2 = MASK * 0x00010001u;
+    constexpr unsigned MASK = TWO ? 3u : 15u, MASK2 = MASK * 0x00010001u;
     constexpr int CB = code_block_bytes(BITS);
-    const __half2 bias = __halves2half2(__ushort_as_half(0x6400), __ushort_as_half(0x6400));
-    auto to_h2 = [&](const unsigned pair) {             // two codes (low bits of each half) -> fp16 pair: 1024 + c, minus 1024
-        const unsigned w = pair | 0x64006400u;
-        const __half2 hv = __hsub2(*reinterpret_cast<const __half2*>(&w), bias);
-        return *reinterpret_cast<const unsigned*>(&hv);
-    };
     // Two codes that sit at bit f of bytes 0 and 2 of `bytes` -> fp16 pair: (1024 + c 2^f) 2^-f - 1024 2^-f = c, one
-    // fused multiply-add (exact: c 2^f < 1024); mul = 2^-f and add = -2^(10 - f) in both halves.
-    auto field_h2 = [](const unsigned bytes, const unsigned mask, const unsigned mul, const unsigned add) {
-        const unsigned w = (bytes & mask) | 0x64006400u;
+    // fused multiply-add (exact: c 2^f < 1024); mul = 2^-f and add = -2^(10 - f) in both halves.  3 bits: `high` holds the
+    // codes' third bits, already at bit f + 2 of each half.
+    auto field_h2 = [](const unsigned bytes, const unsigned mask, const unsigned high, const unsigned mul, const unsigned add) {
+        const unsigned w = (bytes & mask) | 0x64006400u | high;
         const __half2 hv = __hfma2(*reinterpret_cast<const __half2*>(&w), *reinterpret_cast<const __half2*>(&mul),
                                    *reinterpret_cast<const __half2*>(&add));
         return *reinterpret_cast<const unsigned*>(&hv);
@@ -774,7 +756,7 @@ __device__ __forceinline__ void unpack_page(const unsigned char* raw, unsigned c
         const int g = p & 7, s = (p >> 3) & 3, bi = p >> 5;
         const unsigned char* src = raw + bi * CB + (TWO ? 0 : 512 * (s >> 1)) + 64 * g;
         const int sh0 = TWO ? 2 * s : 4 * (s & 1);
-        const unsigned kmask = MASK2 << sh0, kmul = pow2_neg(sh0), kadd = bias_neg(sh0);
+        const unsigned kmask = MASK2 << sh0, kmul = pow2_neg(sh0), kadd = bias_neg(sh0), khigh = 0x00010001u << (sh0 + 2);
         unsigned w[4][4];                                   // [t][j]
         unsigned wh[4][2];                                  // 3 bits: [t][rs], bit 2 s + hh of byte b
 #pragma unroll
@@ -793,16 +775,11 @@ __device__ __forceinline__ void unpack_page(const unsigned char* raw, unsigned c
                 unsigned out[4];
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
-                    if constexpr (BITS == 3) {
-                        const unsigned x = w[t][j] >> (16 * b1 + sh0);
-                        unsigned pair = (x & MASK) | ((x << 8) & MASK_HI);
-                        const unsigned y = wh[t][j & 1] >> (16 * b1 + 2 * s + (j >> 1));
-                        pair |= ((y & 1u) | ((y << 8) & 0x00010000u)) << 2;
-                        out[t] = to_h2(pair);
-                    } else {
-                        // bytes 2 b1 and 2 b1 + 1 of the word to bytes 0 and 2, then the thread's field of each
-                        out[t] = field_h2(__byte_perm(w[t][j], 0u, b1 ? 0x4342u : 0x4140u), kmask, kmul, kadd);
-                    }
+                    // bytes 2 b1 and 2 b1 + 1 of the word to bytes 0 and 2, then the thread's field of each
+                    unsigned high = 0u;
+                    if constexpr (BITS == 3)            // the same bytes of the 1-bit plane: bit 2 s + hh of each goes to bit 2 s + 2
+                        high = (__byte_perm(wh[t][j & 1], 0u, b1 ? 0x4342u : 0x4140u) << (2 - (j >> 1))) & khigh;
+                    out[t] = field_h2(__byte_perm(w[t][j], 0u, b1 ? 0x4342u : 0x4140u), kmask, high, kmul, kadd);
                 }
                 *reinterpret_cast<uint4*>(sK + (2 * bi + (j & 1)) * 2048 + (4 * s + 2 * (j >> 1) + b1) * 128 + g * 16) =
                     make_uint4(out[0], out[1], out[2], out[3]);
@@ -828,27 +805,29 @@ __device__ __forceinline__ void unpack_page(const unsigned char* raw, unsigned c
             if (!TWO) wa[TWO ? 0 : 1][e] = *reinterpret_cast<const unsigned*>(src + 64 * e + 4);
             if (BITS == 3) wh[e] = *reinterpret_cast<const unsigned*>(raw + v_hi_offset(3) + bi * 256 + 8 * (4 * e + tt) + 4 * ps);
         }
+        unsigned hw[4];                                     // 3 bits: this thread's half-word of the 1-bit plane, of the words 2 e2 and 2 e2 + 1
+        if constexpr (BITS == 3) {
+#pragma unroll
+            for (int e2 = 0; e2 < 4; ++e2) hw[e2] = __byte_perm(wh[2 * e2], wh[2 * e2 + 1], hi ? 0x7632u : 0x5410u);
+        }
 #pragma unroll
         for (int ih = 0; ih < 2; ++ih) {                    // half of the channel blocks
             const unsigned (&w)[8] = wa[TWO ? 0 : ih];
 #pragma unroll
             for (int ii = 0; ii < 4; ++ii) {
-                const int i = 4 * ih + ii, sh = 16 * hi + (TWO ? 2 * i : 4 * ii);
-                // bit of the 1-bit plane for (rsel, i): rsel 0: 2 i + 2 (i < 5), 2 i + 1 (else); rsel 1: 2 i + 1 (i < 5), 2 i + 2 (i < 7), 0 (i = 7)
-                const int hb = 16 * hi + (rsel == 0 ? (i < 5 ? 2 * i + 2 : 2 * i + 1) : (i < 5 ? 2 * i + 1 : (i < 7 ? 2 * i + 2 : 0)));
+                const int i = 4 * ih + ii;
+                // the field's byte (of both words, to bytes 0 and 2: the same for the fields of one byte) and its bit inside it
+                const int byte = TWO ? 2 * hi + ih : 2 * hi + (ii >> 1), f = TWO ? 2 * ii : 4 * (ii & 1);
+                // bit of the 1-bit plane for (rsel, i): rsel 0: 2 i + 2 (i < 5), 2 i + 1 (else); rsel 1: 2 i + 1 (i < 5), 2 i + 2 (i < 7), 0 (i = 7);
+                // a rotation takes it to bit f + 2 of each half
+                const int hb = rsel == 0 ? (i < 5 ? 2 * i + 2 : 2 * i + 1) : (i < 5 ? 2 * i + 1 : (i < 7 ? 2 * i + 2 : 0));
                 unsigned out[4];
 #pragma unroll
                 for (int e2 = 0; e2 < 4; ++e2) {
-                    if constexpr (BITS == 3) {
-                        unsigned c0 = (w[2 * e2] >> sh) & MASK, c1 = (w[2 * e2 + 1] >> sh) & MASK;
-                        c0 |= ((wh[2 * e2] >> hb) & 1u) << 2; c1 |= ((wh[2 * e2 + 1] >> hb) & 1u) << 2;
-                        out[e2] = dequant(to_h2(c0 | (c1 << 16)));
-                    } else {
-                        // the byte that holds the field, of both words, to bytes 0 and 2 (the same for the fields of one byte)
-                        const int byte = TWO ? 2 * hi + ih : 2 * hi + (ii >> 1), f = TWO ? 2 * ii : 4 * (ii & 1);
-                        const unsigned both = __byte_perm(w[2 * e2], w[2 * e2 + 1], 0x0400u + 0x0101u * static_cast<unsigned>(byte));
-                        out[e2] = dequant(field_h2(both, MASK2 << f, pow2_neg(f), bias_neg(f)));
-                    }
+                    unsigned high = 0u;
+                    if constexpr (BITS == 3) high = __funnelshift_r(hw[e2], hw[e2], (hb - (f + 2)) & 31) & (0x00010001u << (f + 2));
+                    const unsigned both = __byte_perm(w[2 * e2], w[2 * e2 + 1], 0x0400u + 0x0101u * static_cast<unsigned>(byte));
+                    out[e2] = dequant(field_h2(both, MASK2 << f, high, pow2_neg(f), bias_neg(f)));
                 }
                 *reinterpret_cast<uint4*>(sV + (2 * i + rsel) * 1024 + (2 * bi + ps) * 128 + (2 * tt + hi) * 16) =
                     make_uint4(out[0], out[1], out[2], out[3]);
