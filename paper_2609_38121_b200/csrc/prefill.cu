@@ -1399,7 +1399,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
     // and MMA warps place 16-byte pieces (rows clamped to the chunk) while the staging warps start on the key side at once.
     if (warp < 8) {
         // =============================== softmax of query tile t ==========================================
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 184;" ::: "memory");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 176;" ::: "memory");
         if (!P.use_tma) {
             for (int item = tid; item < 4 * TM * 16; item += 256) {
                 const int q = item >> 11, part = q & 1, r = (item >> 4) & (TM - 1), piece = item & 15;
@@ -1583,7 +1583,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
         }
     }
     else if (warp < 12) {
-      asm volatile("setmaxnreg.dec.sync.aligned.u32 56;" ::: "memory");
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 64;" ::: "memory");
       if (P.use_tma && tid == 288) {
             const unsigned box_bytes = 128u * static_cast<unsigned>(G * R);
             ws_expect_tx(bar(WB_Q), 4u * box_bytes * ((n_tiles[0] > 0 ? 1u : 0u) + (n_tiles[1] > 0 ? 1u : 0u)));
@@ -1746,7 +1746,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
     }
     else {
         // =============================== staging of key / value tiles by threads ===========================
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 88;" ::: "memory");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 96;" ::: "memory");
         const int ptid = tid - 384;
         int raw_uses[2] = {0, 0};                               // records fetched so far into each raw buffer
         auto page_of = [&](const int gb) -> int {               // page id of packed tile gb, -1 if it cannot be read
