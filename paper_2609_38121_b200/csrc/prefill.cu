@@ -1244,7 +1244,7 @@ constexpr int WS_OFF_V = WS_OFF_K + WS_KS * TC_K_BYTES;
 constexpr int WS_OFF_RAW = WS_OFF_V + WS_VS * TC_K_BYTES;        // two raw records
 enum { WB_KFULL = 0, WB_KEMPTY = WB_KFULL + WS_KS, WB_VFULL = WB_KEMPTY + WS_KS, WB_VEMPTY = WB_VFULL + WS_VS,
        WB_S = WB_VEMPTY + WS_VS, WB_PV = WB_S + 4, WB_PREADY = WB_PV + 4, WB_RAW = WB_PREADY + 4, WB_Q = WB_RAW + 2,
-       WB_STAGED, WB_DRAIN, WB_COUNT };
+       WB_STAGED, WB_DRAIN, WB_RAWFREE, WB_COUNT = WB_RAWFREE + 2 };
 // The rest of the layout depends on the record size.  Per-key factors of a packed tile, per value stage: (step, offset) of
 // the key side for the 64 keys as fp32 pairs (the softmax threads load them ready to use, two keys per 16-byte load).
 __host__ __device__ constexpr int ws_meta_stage(int) { return TN * 8; }
@@ -1703,7 +1703,29 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
         // for the first chunk tiles means: once the staging threads' last tiles went through).
         int armed[3] = {-1, -1, -1};                            // last tile whose copies this warp announced on each stage (<= 3 stages)
         bool ok = true;
-        if (P.use_tma && n_staged > 0) ok = __all_sync(FULLM, ws_wait(bar(WB_STAGED), 0u, wait_limit, abort_flag));
+        // Before that, warp 9 requests the records of the packed pages for the staging threads, by bulk copies into the two
+        // raw buffers: record gb as soon as the staging threads have left the record two before it.  (Done here because the
+        // request costs its thread several hundred cycles, which the staging threads do not have.)
+        int requested[2] = {0, 0};                              // records requested so far into each raw buffer
+        if (warp == 9) {
+            for (int gb = gb_first; gb < gb_end && ok; ++gb) {
+                const int rb = gb & 1, use = (gb - gb_first) >> 1;      // use-th record of this buffer
+                if (use >= 1 && !__all_sync(FULLM, ws_wait(bar(WB_RAWFREE + rb), (use - 1) & 1, wait_limit, abort_flag))) { ok = false; break; }
+                if (lane == 0) {
+                    const int pg = page_first + gb;
+                    const int page = pg < c.max_pages ? __ldg(c.page_table + static_cast<long long>(sl) * c.max_pages + pg) : -1;
+                    if (page < 0 || page >= c.n_pages) {
+                        atomicOr(c.dev_status, pg < c.max_pages ? WUSHKV_DEV_BAD_PAGE_ID : WUSHKV_DEV_PAGE_TABLE_FULL);
+                    } else {
+                        ws_expect_tx(bar(WB_RAW + rb), REC);
+                        ws_bulk_g2s(smem_addr(sm_ws + WS_OFF_RAW + rb * REC), c.pages + (static_cast<long long>(page) * c.n_kv + h) * REC, REC,
+                                    bar(WB_RAW + rb));
+                        ++requested[rb];
+                    }
+                }
+            }
+        }
+        if (ok && P.use_tma && n_staged > 0) ok = __all_sync(FULLM, ws_wait(bar(WB_STAGED), 0u, wait_limit, abort_flag));
         if (P.use_tma) {
             const bool keys = warp == 9;
             const int depth = keys ? WS_KS : WS_VS, full0 = keys ? WB_KFULL : WB_VFULL, empty0 = keys ? WB_KEMPTY : WB_VEMPTY;
@@ -1742,6 +1764,12 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
         }
         if (tid == 288 && *abort_flag && P.use_tma)             // the same for the query copies
             for (int it = 0; it < 512 && !ws_wait(bar(WB_Q), 0u, 1, abort_flag); ++it) __nanosleep(2000);
+        if (tid == 288 && *abort_flag) {                        // and for the record copies
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+                if (requested[i] > 0)
+                    for (int it = 0; it < 64 && !ws_wait(bar(WB_RAW + i), (requested[i] - 1) & 1, 1, abort_flag); ++it) __nanosleep(2000);
+        }
       }
     }
     else {
@@ -1749,24 +1777,16 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
         asm volatile("setmaxnreg.dec.sync.aligned.u32 96;" ::: "memory");
         const int ptid = tid - 384;
         int raw_uses[2] = {0, 0};                               // records fetched so far into each raw buffer
-        auto page_of = [&](const int gb) -> int {               // page id of packed tile gb, -1 if it cannot be read
+        // page id of packed tile gb as the table holds it (-1 beyond the table); it is range-checked where it is used, a tile
+        // later, so that nothing waits for the load
+        auto page_of = [&](const int gb) -> int {
             const int pg = page_first + gb;
-            int page = -1;
-            if (pg < c.max_pages) page = __ldg(c.page_table + static_cast<long long>(sl) * c.max_pages + pg);
-            return (page >= 0 && page < c.n_pages) ? page : -1;
+            return pg < c.max_pages ? __ldg(c.page_table + static_cast<long long>(sl) * c.max_pages + pg) : -1;
         };
-        auto fetch_record = [&](const int gb, const int page) {     // one thread: bulk copy of the record into raw buffer gb & 1
-            if (page < 0) {
-                atomicOr(c.dev_status, page_first + gb < c.max_pages ? WUSHKV_DEV_BAD_PAGE_ID : WUSHKV_DEV_PAGE_TABLE_FULL);
-                return;
-            }
-            ws_expect_tx(bar(WB_RAW + (gb & 1)), REC);
-            ws_bulk_g2s(smem_addr(sm_ws + WS_OFF_RAW + (gb & 1) * REC), c.pages + (static_cast<long long>(page) * c.n_kv + h) * REC, REC,
-                        bar(WB_RAW + (gb & 1)));
-        };
-        // page ids are read two tiles ahead, so that neither the record request nor the unpacking waits for the page table
-        int page_cur = gb_end > gb_first ? page_of(gb_first) : -1, page_next = gb_end > gb_first + 1 ? page_of(gb_first + 1) : -1;
-        if (gb_end > gb_first && ptid == 0) fetch_record(gb_first, page_cur);
+        auto page_valid = [&](const int page) { return page >= 0 && page < c.n_pages; };
+        // (the records themselves are requested by warp 9, up to two ahead; a page that cannot be read is reported there and
+        // its tile is staged as absent keys here)
+        int page_cur = gb_end > gb_first ? page_of(gb_first) : -1;
         bool ok = true;
         WST_DECL;
         for (int g = 0; g < n_staged && ok; ++g) {
@@ -1812,18 +1832,17 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
             } else if (g < gC) {
                 // ---- a packed page: the record was requested one tile ahead; unpack it into integer codes (exact in fp16)
                 const int gb = g - nA, rb = gb & 1;
-                // the other raw buffer was last read for tile gb - 1, which every staging thread has left
-                if (gb + 1 < gb_end && ptid == 0) fetch_record(gb + 1, page_next);
-                const bool page_ok = page_cur >= 0;
-                page_cur = page_next;
-                page_next = gb + 2 < gb_end ? page_of(gb + 2) : -1;
+                const bool page_ok = page_valid(page_cur);
+                page_cur = gb + 1 < gb_end ? page_of(gb + 1) : -1;          // read a tile ahead: nothing waits for the page table
                 if (page_ok && mine) mine = __all_sync(FULLM, ws_wait(bar(WB_RAW + rb), raw_uses[rb] & 1, wait_limit, abort_flag));
                 if (page_ok) ++raw_uses[rb];
+                WST(5);
                 const unsigned char* raw = sm_ws + WS_OFF_RAW + rb * REC;
                 const uint4 zero4 = make_uint4(0, 0, 0, 0);
                 const int page_pos = (page_first + gb) * PAGE_TOKENS;
                 const bool whole = page_ok && page_pos >= q_lo && page_pos + PAGE_TOKENS <= q_hi;
                 if (whole && mine) unpack_page<BITS>(raw, sK, sV, ptid);
+                WST(6);
 #pragma unroll 4
                 for (int item = ptid; item < (mine && !whole ? TN * 16 : 0); item += 128) {      // first / last page of the range
                     const int r = item & (TN - 1), kc = item >> 6;
@@ -1874,17 +1893,15 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             ok = ws_stagers_and(mine);
             WST(3);
-            if (ok && ptid == 0) { ws_arrive(bar(WB_KFULL + ks)); ws_arrive(bar(WB_VFULL + vs)); }
+            if (ok && ptid == 0) {
+                ws_arrive(bar(WB_KFULL + ks)); ws_arrive(bar(WB_VFULL + vs));
+                if (g >= nA && g < gC) ws_arrive(bar(WB_RAWFREE + ((g - nA) & 1)));      // every staging thread has left the raw record
+            }
         }
         // the copy-issuing warps may start on the chunk's own tiles now: a wait for a stage's release only tells the last two
         // releases apart, so they must not look at a stage before the tiles staged here have gone through it
         WST_FLUSH;
         if (ok && ptid == 0) ws_arrive(bar(WB_STAGED));
-        if (tid == 384 && *abort_flag) {                        // give the record copies a bounded time to land
-#pragma unroll
-            for (int i = 0; i < 2; ++i)
-                if (gb_end > gb_first) for (int it = 0; it < 64 && !ws_wait(bar(WB_RAW + i), raw_uses[i] & 1, 1, abort_flag); ++it) __nanosleep(2000);
-        }
     }
 
     // ---- all roles are done (or gave up)
