@@ -1708,12 +1708,19 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
         // request costs its thread several hundred cycles, which the staging threads do not have.)
         int requested[2] = {0, 0};                              // records requested so far into each raw buffer
         if (warp == 9) {
+            // (the page id is read a record ahead, so that the wait for the buffer covers the load)
+            auto page_id = [&](const int gb) {
+                const int pg = page_first + gb;
+                return (gb < gb_end && pg < c.max_pages) ? __ldg(c.page_table + static_cast<long long>(sl) * c.max_pages + pg) : -1;
+            };
+            int page_ahead = page_id(gb_first);
             for (int gb = gb_first; gb < gb_end && ok; ++gb) {
                 const int rb = gb & 1, use = (gb - gb_first) >> 1;      // use-th record of this buffer
+                const int page = page_ahead;
+                page_ahead = page_id(gb + 1);
                 if (use >= 1 && !__all_sync(FULLM, ws_wait(bar(WB_RAWFREE + rb), (use - 1) & 1, wait_limit, abort_flag))) { ok = false; break; }
                 if (lane == 0) {
                     const int pg = page_first + gb;
-                    const int page = pg < c.max_pages ? __ldg(c.page_table + static_cast<long long>(sl) * c.max_pages + pg) : -1;
                     if (page < 0 || page >= c.n_pages) {
                         atomicOr(c.dev_status, pg < c.max_pages ? WUSHKV_DEV_BAD_PAGE_ID : WUSHKV_DEV_PAGE_TABLE_FULL);
                     } else {
