@@ -1900,10 +1900,10 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             ok = ws_stagers_and(mine);
             WST(3);
-            if (ok && ptid == 0) {
-                ws_arrive(bar(WB_KFULL + ks)); ws_arrive(bar(WB_VFULL + vs));
-                if (g >= nA && g < gC) ws_arrive(bar(WB_RAWFREE + ((g - nA) & 1)));      // every staging thread has left the raw record
-            }
+            // (one arrival per warp: each costs its thread some tens of cycles)
+            if (ok && ptid == 0) ws_arrive(bar(WB_KFULL + ks));
+            if (ok && ptid == 32) ws_arrive(bar(WB_VFULL + vs));
+            if (ok && ptid == 64 && g >= nA && g < gC) ws_arrive(bar(WB_RAWFREE + ((g - nA) & 1)));      // every staging thread has left the raw record
         }
         // the copy-issuing warps may start on the chunk's own tiles now: a wait for a stage's release only tells the last two
         // releases apart, so they must not look at a stage before the tiles staged here have gone through it
