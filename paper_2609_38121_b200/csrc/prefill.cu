@@ -1516,8 +1516,15 @@ __global__ void __launch_bounds__(WS_THREADS, 1) prefill_attn_ws_kernel(PrefillP
 #pragma unroll
                         for (int q = 0; q < 2; ++q) {
                             const int e = 16 * half + 2 * e4 + q;
-                            const float2 pr = make_float2(fast_ex2(fmaf(s[2 * e], k2, -ref)), fast_ex2(fmaf(s[2 * e + 1], k2, -ref)));     // k2 s - ref in one rounding
-                            lsum.x += pr.x; lsum.y += pr.y;
+                            // k2 s - ref in one rounding, two lanes per instruction
+                            float2 pr;
+                            asm("{\n\t.reg .b64 va, vm, vc, vd;\n\tmov.b64 va, {%2, %3};\n\tmov.b64 vm, {%4, %4};\n\tmov.b64 vc, {%5, %5};\n\t"
+                                "fma.rn.f32x2 vd, va, vm, vc;\n\tmov.b64 {%0, %1}, vd;\n\t}"
+                                : "=f"(pr.x), "=f"(pr.y) : "f"(s[2 * e]), "f"(s[2 * e + 1]), "f"(k2), "f"(-ref));
+                            pr.x = fast_ex2(pr.x); pr.y = fast_ex2(pr.y);
+                            // so the running sums
+                            asm("{\n\t.reg .b64 va, vb, vd;\n\tmov.b64 va, {%2, %3};\n\tmov.b64 vb, {%4, %5};\n\tadd.rn.f32x2 vd, va, vb;\n\tmov.b64 {%0, %1}, vd;\n\t}"
+                                : "=f"(lsum.x), "=f"(lsum.y) : "f"(lsum.x), "f"(lsum.y), "f"(pr.x), "f"(pr.y));
                             pk[2 * e4 + q] = pack_half2(pr.x, pr.y);
                         }
                     }
